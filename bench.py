@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-attention step (multi-query vs multi-head) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch: the in-place append of the new
+token's key/value row, the split-m pass over the cache and the combine pass.  The headline
+workload is the long-context configuration (b=32, h=32, k=v=128, 8192-row cache); the other
+workloads (`--workload`, `--sweep`) are the parity configurations and the bandwidth sweep.
+Prints ONE JSON line (rank 0).  `value` is achieved HBM GB/s of the multi-query step
+(algorithmic bytes / time); the multi-head step on the same shapes is reported beside it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1911_02150_b200 import sharding, workloads as wl  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0      # the metric's stated denominator
+FALLBACK_HBM_GBS = 6650.0     # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+L2_BYTES = 126 * 2 ** 20
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+class StepState:
+    """Device-resident state of one variant: rotating cache sets (to keep reads out of L2), the
+    step's inputs and outputs, and the launch plan."""
+
+    def __init__(self, mqa, variant, w, device, seed, min_rotate_bytes):
+        self.mqa, self.variant, self.w, self.device = mqa, variant, w, device
+        b, h, m = w.b, w.h, w.m_max
+        self.kvh = 1 if variant == "mqa" else h
+        lens0 = wl.initial_lens(w, seed=0)
+        cache_bytes = 2 * b * self.kvh * m * 128 * 2
+        free, _ = torch.cuda.mem_get_info(device)
+        n_sets = max(1, -(-min_rotate_bytes // cache_bytes))
+        n_sets = int(min(n_sets, max(1, (free - 8 * 2 ** 30) // cache_bytes), 16))
+        self.sets = []
+        for i in range(n_sets):
+            inp = wl.make_inputs(b, h, m, variant, seed=seed + i, device=device)
+            self.sets.append(inp)
+        self.lens_before = torch.from_numpy(lens0).to(device)
+        self.lens_after = torch.from_numpy(lens0 + 1).to(device)
+        self.sum_lens = int((lens0 + 1).sum())
+        self.o = torch.empty(b, h, 128, dtype=torch.float32, device=device)
+        self.ws = mqa.alloc_workspace(b, h, m, device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.n_splits, self.chunk_rows = mqa.plan_splits(variant == "mqa", b, h, m)
+        self.bytes = wl.algorithmic_bytes(self.sum_lens, b, h, self.kvh)
+        self.cache_bytes = cache_bytes
+        self.append = mqa.kv_cache_append
+        self.step_fn = mqa.mqa_decode_step if variant == "mqa" else mqa.mha_decode_step
+        self.split_fn = mqa.mqa_decode_step_split if variant == "mqa" else mqa.mha_decode_step_split
+        self.combine_fn = mqa.mqa_decode_step_combine if variant == "mqa" else mqa.mha_decode_step_combine
+        self.launches_per_step = 2 + (1 if self.n_splits > 1 else 0)
+        # pinned host copies of the per-step inputs / result for the end-to-end leg
+        s0 = self.sets[0]
+        self.host_in = [s0[n].cpu().pin_memory() for n in ("q", "k_new", "v_new")]
+        self.host_o = torch.empty(b, h, 128, dtype=torch.float32).pin_memory()
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host_in)
+        self.d2h_bytes = self.host_o.numel() * 4
+
+    def step(self, i):
+        s = self.sets[i % len(self.sets)]
+        self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
+        self.step_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
+
+    def step_phases(self, i, ev0, ev1):
+        """Same launches as step(), with events around the pass over the cache."""
+        s = self.sets[i % len(self.sets)]
+        self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
+        ev0.record()
+        self.split_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
+        ev1.record()
+        self.combine_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
+
+    def step_e2e(self, i):
+        s = self.sets[i % len(self.sets)]
+        for name, src in zip(("q", "k_new", "v_new"), self.host_in):
+            s[name].copy_(src, non_blocking=True)
+        self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
+        self.step_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
+        self.host_o.copy_(self.o, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller needs o before the next token
+
+
+def time_region(fn, steps, device):
+    """Seconds for `steps` calls of fn(i), CUDA events on the launching stream, synchronised on both sides."""
+    sharding.barrier()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize(device)
+    sharding.barrier()
+    return e0.elapsed_time(e1) * 1e-3
+
+
+def run_variant(st: StepState, steps, warmup, device, sample_clocks):
+    for i in range(warmup):
+        st.step(i)
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(torch.cuda.current_device()) if sample_clocks else None
+    if sampler:
+        sampler.__enter__()
+    t0 = time.time()
+    n_rep = 0
+    secs = 0.0
+    # repeat the K-step region until ~0.4 s have been sampled by the clock monitor (short kernels)
+    regions = []
+    while True:
+        t = time_region(st.step, steps, device)
+        regions.append(t)
+        n_rep += 1
+        if not sample_clocks or time.time() - t0 > 0.5 or n_rep >= 200:
+            break
+    if sampler:
+        sampler.__exit__()
+    secs = regions[0]                                   # the reported region is the first, exactly K steps
+    # per-launch duration of the pass over the cache (the dominant kernel)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i in range(steps):
+        st.step_phases(i, *evs[i])
+    torch.cuda.synchronize(device)
+    kernel_s = statistics.mean(a.elapsed_time(c) for a, c in evs) * 1e-3
+    # end to end with host buffers
+    for i in range(min(warmup, 3)):
+        st.step_e2e(i)
+    e2e_s = time_region(st.step_e2e, steps, device)
+    status = int(st.status.item())
+    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status,
+            "clocks": sampler.summary() if sampler else None,
+            "median_region_s": statistics.median(regions), "regions": n_rep}
+
+
+def cpu_baseline(w, seed, budget_s=20.0):
+    """The oracle, as it stands, on the host cores: one multi-query step of the same workload on
+    as many whole sequences as fit the time budget."""
+    import oracle
+    inp = wl.make_inputs(min(w.b, 64), w.h, w.m_max, "mqa", seed=seed, device="cpu")
+    lens = (wl.initial_lens(w)[: inp["b"]] + 1).astype(np.int32)
+    qb, Kb, Vb = wl.bits(inp["q"]), wl.bits(inp["K"]), wl.bits(inp["V"])
+    t0 = time.perf_counter()
+    oracle.mqa_decode_step(qb[:1], Kb[:1], Vb[:1], lens[:1])
+    per_seq = max(time.perf_counter() - t0, 1e-6)       # one sequence, all heads in parallel
+    n = int(max(1, min(inp["b"], budget_s / per_seq)))
+    t0 = time.perf_counter()
+    oracle.mqa_decode_step(qb[:n], Kb[:n], Vb[:n], lens[:n])
+    dt = time.perf_counter() - t0
+    by = wl.algorithmic_bytes(int(lens[:n].sum()), n, w.h, 1)
+    return {"value": by / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n} of {w.b} sequences x {w.h} heads x {w.m_max} rows, one multi-query step, fp64, "
+                      f"{dt:.2f} s", "seconds": dt}
+
+
+def reference_arm(args, w):
+    """--impl reference: the CPU oracle timed on this machine's host cores, a bounded sample per step."""
+    rank, _, world = sharding.world_from_env()
+    if rank != 0:
+        return
+    import oracle
+    n_seq = min(w.b, 2)
+    inp = wl.make_inputs(n_seq, w.h, w.m_max, "mqa", seed=0, device="cpu")
+    lens = (wl.initial_lens(w)[:n_seq] + 1).astype(np.int32)
+    qb, Kb, Vb = wl.bits(inp["q"]), wl.bits(inp["K"]), wl.bits(inp["V"])
+    knb, vnb = wl.bits(inp["k_new"]), wl.bits(inp["v_new"])
+    lens_before = (lens - 1).astype(np.int32)
+
+    def one(_):
+        lb = lens_before.copy()
+        oracle.kv_cache_append(Kb, Vb, knb, vnb, lb, True)
+        oracle.mqa_decode_step(qb, Kb, Vb, lb)
+    for i in range(args.warmup):
+        one(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        one(i)
+    dt = (time.perf_counter() - t0) / args.steps
+    by = wl.algorithmic_bytes(int(lens.sum()), n_seq, w.h, 1)
+    val = by / dt / 1e9
+    sample = f"{n_seq} of {w.b} sequences x {w.h} heads x {w.m_max} rows per step (append + multi-query step), fp64 oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": "mqa_decode_step_hbm_gbs", "value": val, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(w), "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_name(w):
+    return (f"{w.name}: b={w.b} h={w.h} k=v=128 m_max={w.m_max} lens={w.lens}; one step = append of the new "
+            f"k/v row + attention over the prefix")
+
+
+def result_block(st, r, steps):
+    us = r["secs"] / steps * 1e6
+    gbs = st.bytes / (r["secs"] / steps) / 1e9
+    return {"us_per_step": us, "gbs": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_step": st.bytes,
+            "n_splits": st.n_splits, "chunk_rows": st.chunk_rows, "cache_sets": len(st.sets),
+            "kernel_us": r["kernel_s"] * 1e6, "status": r["status"],
+            "median_us_per_step": r["median_region_s"] / steps * 1e6}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long_context")
+    ap.add_argument("--no-mha", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="run every workload and write gpurun_out/sweep.json")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = wl.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        reference_arm(args, w)
+        return
+
+    rank, local_rank, world = sharding.world_from_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode step has no CPU path")
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    if world > 1:
+        sharding.init_process_group("nccl")
+    import paper_1911_02150_b200 as mqa
+    from paper_1911_02150_b200.build import build_library
+    if rank == 0 or world == 1:
+        build_library()
+    sharding.barrier()
+    mqa.lib()
+
+    if args.sweep:
+        run_sweep(mqa, args, device, rank)
+        return
+
+    peak, peak_kind = measured_peak()
+    seed = 1000 * rank                                  # every rank owns its own batch shard (weak scaling)
+    st = StepState(mqa, "mqa", w, device, seed, min_rotate_bytes=8 * L2_BYTES)
+    r = run_variant(st, args.steps, args.warmup, device, sample_clocks=True)
+    blk = result_block(st, r, args.steps)
+    secs_max = sharding.max_over_ranks(r["secs"], device)
+    e2e_max = sharding.max_over_ranks(r["e2e_s"], device)
+    total_bytes = sharding.sum_over_ranks(st.bytes, device)
+    value = total_bytes / (secs_max / args.steps) / 1e9
+    e2e_value = total_bytes / (e2e_max / args.steps) / 1e9
+    kernel_gbs = st.bytes / r["kernel_s"] / 1e9
+    out = {
+        "metric": "mqa_decode_step_hbm_gbs", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": secs_max / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(w), "parallelism": f"batch shards x{world}, no collective",
+                   "l2": f"rotating {len(st.sets)} cache sets of {st.cache_bytes >> 20} MiB (> L2) between steps",
+                   "n_splits": st.n_splits, "chunk_rows": st.chunk_rows},
+        "us_per_step": blk["us_per_step"], "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
+        "mqa": blk,
+        "roofline": {"bound": "hbm", "achieved": kernel_gbs, "peak": peak, "unit": "GB/s", "frac": kernel_gbs / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "kernel": "split pass of mqa_decode_step", "kernel_us": r["kernel_s"] * 1e6,
+                     "algorithmic_bytes": st.bytes},
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": st.h2d_bytes,
+                "d2h_bytes_per_step": st.d2h_bytes, "us_per_step": e2e_max / args.steps * 1e6,
+                "note": "per-step inputs q,k_new,v_new from pinned host memory, o read back; the KV cache is "
+                        "decoder state and stays resident in HBM"},
+        "gpu_launches": st.launches_per_step * args.steps,
+        "clocks": r["clocks"],
+    }
+    traffic = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic):
+        try:
+            out["roofline"]["traffic"] = json.load(open(traffic)).get(w.name, {}).get("mqa_split_dram_bytes")
+        except Exception:
+            pass
+    del st
+    torch.cuda.empty_cache()
+    if not args.no_mha:
+        sth = StepState(mqa, "mha", w, device, seed, min_rotate_bytes=2 * L2_BYTES)
+        rh = run_variant(sth, max(3, min(args.steps, 20)), 3, device, sample_clocks=False)
+        out["mha"] = result_block(sth, rh, max(3, min(args.steps, 20)))
+        out["mha"]["roofline_frac"] = sth.bytes / rh["kernel_s"] / 1e9 / peak
+        out["mqa_speedup_over_mha"] = out["mha"]["us_per_step"] / blk["us_per_step"]
+        del sth
+        torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w, seed)
+    if rank == 0:
+        print(json.dumps(out))
+
+
+def run_sweep(mqa, args, device, rank):
+    """Every workload, both variants: us per step and GB/s per point -> gpurun_out/sweep.json."""
+    peak, peak_kind = measured_peak()
+    rows = []
+    for name, w in wl.WORKLOADS.items():
+        if w.lens == "grow":
+            continue
+        for variant in ("mqa", "mha"):
+            kvh = 1 if variant == "mqa" else w.h
+            cache = 2 * w.b * kvh * w.m_max * 256
+            if cache > 100 * 2 ** 30:
+                rows.append({"workload": name, "variant": variant, "skipped": "cache exceeds 100 GiB"})
+                continue
+            free, _ = torch.cuda.mem_get_info(device)
+            if cache + 6 * 2 ** 30 > free:
+                rows.append({"workload": name, "variant": variant, "skipped": f"cache {cache >> 30} GiB does not fit"})
+                continue
+            st = StepState(mqa, variant, w, device, 0, min_rotate_bytes=4 * L2_BYTES)
+            steps = 20 if cache < 8 * 2 ** 30 else 5
+            r = run_variant(st, steps, 3, device, sample_clocks=False)
+            blk = result_block(st, r, steps)
+            blk.update({"workload": name, "variant": variant, "b": w.b, "h": w.h, "m": w.m_max,
+                        "frac_of_measured_copy": blk["gbs"] / peak})
+            rows.append(blk)
+            print(json.dumps(blk), file=sys.stderr)
+            del st
+            torch.cuda.empty_cache()
+    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+    with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
+        json.dump({"peak_gbs": peak, "peak_kind": peak_kind, "rows": rows}, f, indent=1)
+    if rank == 0:
+        print(json.dumps({"sweep_points": len(rows), "written": "gpurun_out/sweep.json"}))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,154 @@
+/*
+ * mqa_decode.h -- C ABI of the B200 (sm_100a) decode-attention library.
+ *
+ * One incremental-decoding attention step as stated in "Fast Transformer Decoding: One
+ * Write-Head is All You Need" (arXiv 1911.02150): for each sequence of a batch, h query
+ * heads attend over that sequence's key/value cache,
+ *
+ *     logits[b,h,j] = sum_c q[b,h,c] * K[..,j,c]          (no 1/sqrt(k) factor: the note
+ *     w[b,h,:]      = softmax_j(logits[b,h,:])             closing Section 2.2 folds it
+ *     o[b,h,c]      = sum_j w[b,h,j] * V[..,j,c]           into the projections)
+ *
+ * with j running over the valid prefix of the cache.  The multi-query form (Section 3)
+ * keeps ONE cache per sequence, K[b,m,k], V[b,m,v], shared by all heads; the multi-head
+ * form (Section 2.4) keeps one per head, K[b,h,m,k], V[b,h,m,v].  The new token's key and
+ * value row is appended to the cache in place before the step attends.
+ *
+ * Conventions for every entry point
+ *   - Every pointer is a DEVICE pointer owned by the caller unless said otherwise; tensors
+ *     are dense, row-major, innermost axis last.  q, K, V, k_new, v_new, o and the workspace
+ *     must be 16-byte aligned; lens and status 4-byte aligned.
+ *   - K, V, q, k_new, v_new hold bf16; o holds fp32; lens holds int32.
+ *   - k == v == 128 is the only supported head width; h >= 1.
+ *   - `stream` is a cudaStream_t passed as a plain pointer (NULL = the legacy default stream).
+ *     Calls only enqueue work on it: they never synchronise, never allocate device memory and
+ *     never free anything.  The launch configuration is chosen from the integer arguments and
+ *     the current device alone, never from device data.
+ *   - Return value: MQA_OK (0) or one of the positive codes below.  On any error NO kernel has
+ *     been launched and no buffer has been touched.
+ *   - Cache rows at or beyond lens[b] are don't-care: they may hold anything (NaN, Inf) and
+ *     do not influence o.  lens[b] outside [0, m_max] is clamped into it for the attention
+ *     and reported through `status`; nothing is read or written out of bounds.
+ *   - lens[b] == 0 gives o[b,:,:] = 0 (the paper's flow never produces an empty prefix, since
+ *     the append precedes the attention).
+ *   - Results are deterministic: the same inputs on the same device give the same bits.
+ *   - `status` (optional, may be NULL) is one int32 word on the device that kernels OR bits
+ *     into; the caller clears it.  Bits: MQA_STATUS_*.
+ */
+#ifndef MQA_DECODE_H_
+#define MQA_DECODE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* mqa_stream_t; /* a cudaStream_t */
+
+enum {
+    MQA_OK = 0,
+    MQA_ERR_INVALID_ARG = 1,         /* null or misaligned pointer, non-positive dimension   */
+    MQA_ERR_UNSUPPORTED = 2,         /* k or v != 128, or a size the launch grid cannot hold */
+    MQA_ERR_WORKSPACE_TOO_SMALL = 3, /* workspace_bytes < mqa_workspace_bytes(...)           */
+    MQA_ERR_CUDA = 4                 /* the CUDA runtime reported an error at launch         */
+};
+
+enum {
+    MQA_STATUS_APPEND_CACHE_FULL = 1,   /* kv_cache_append: some lens[b] >= m_max, that sequence skipped */
+    MQA_STATUS_APPEND_NEGATIVE_LEN = 2, /* kv_cache_append: some lens[b] < 0, that sequence skipped      */
+    MQA_STATUS_LEN_CLAMPED = 4,         /* decode step: some lens[b] outside [0, m_max] was clamped       */
+    MQA_STATUS_PIPELINE_TIMEOUT = 8     /* decode step: a bounded wait on an on-chip copy ran out; the
+                                           affected outputs are not valid                              */
+};
+
+/*
+ * kv_cache_append -- the concatenation of the new key/value row on the memory axis in the
+ * incremental functions of Sections 2.4 (multi-head) and 3 (multi-query), done in place in
+ * a cache padded to m_max rows.
+ *
+ *   K, V          [b, kv_heads, m_max, k], [b, kv_heads, m_max, v] bf16, read-write.
+ *                 kv_heads = 1 for the multi-query cache ([b, m_max, k]), h for multi-head.
+ *   k_new, v_new  [b, kv_heads, k], [b, kv_heads, v] bf16: the new token's rows.
+ *   lens          [b] int32: rows valid BEFORE the call; row lens[b] is the one written.
+ *   advance       non-zero: lens[b] += 1 on the device after the write (for written rows).
+ *   status        optional; CACHE_FULL / NEGATIVE_LEN when a sequence cannot take a row
+ *                 (that sequence is skipped: nothing written, lens[b] unchanged).
+ * The rows are copied as 16-bit words and never interpreted as numbers: bit-exact.
+ */
+int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new,
+                    int32_t* lens, int advance, int32_t* status,
+                    int b, int kv_heads, int m_max, int k, int v, mqa_stream_t stream);
+
+/*
+ * mqa_decode_step -- the three attention lines of the incremental multi-query function
+ * (Section 3): logits = einsum(bhk,bmk->bhm), softmax over m, o = einsum(bhm,bmv->bhv),
+ * over the first lens[b] rows of each sequence's shared cache.
+ *
+ *   q      [b, h, k] bf16          K, V   [b, m_max, k], [b, m_max, v] bf16 (read only)
+ *   lens   [b] int32: rows to attend over (i.e. AFTER the append)
+ *   o      [b, h, v] fp32, written
+ *   workspace, workspace_bytes   scratch for the per-split partial results; at least
+ *          mqa_workspace_bytes(b, h, m_max, k, v) bytes.  Contents on entry are ignored and
+ *          on return are unspecified.  Two calls that may overlap on the GPU need two
+ *          workspaces.  May be NULL when mqa_workspace_bytes(...) is 0.
+ *   status optional; LEN_CLAMPED, PIPELINE_TIMEOUT.
+ * The memory axis is cut into splits that run in parallel, each keeping a running maximum
+ * and sum (an exact re-association of the same softmax), and a second kernel combines the
+ * splits; shared K/V rows are read from HBM once and used for all h heads.
+ */
+int mqa_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                    void* workspace, size_t workspace_bytes, int32_t* status,
+                    int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+
+/*
+ * mha_decode_step -- the same three lines of the incremental multi-head function
+ * (Section 2.4): logits = einsum(bhk,bhmk->bhm), softmax over m, o = einsum(bhm,bhmv->bhv).
+ * Arguments as mqa_decode_step except K, V are [b, h, m_max, k], [b, h, m_max, v] (one
+ * cache per head); lens[b] is shared by the h heads of a sequence.
+ */
+int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                    void* workspace, size_t workspace_bytes, int32_t* status,
+                    int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+
+/*
+ * The two phases of a step, separately (mqa_decode_step == split then combine with the same
+ * arguments; likewise mha).  They exist so that a caller can time or schedule the phases on
+ * their own.  *_split runs the pass over the cache (Section 3 / 2.4 lines, per split) and
+ * leaves partial results in the workspace -- or final results in o when the plan has a single
+ * split; *_combine merges the splits into o and is a no-op (no launch) for a single split.
+ */
+int mqa_decode_step_split(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                          void* workspace, size_t workspace_bytes, int32_t* status,
+                          int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+int mqa_decode_step_combine(const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes,
+                            int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+int mha_decode_step_split(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                          void* workspace, size_t workspace_bytes, int32_t* status,
+                          int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes,
+                            int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+
+/*
+ * mqa_workspace_bytes -- bytes of scratch that mqa_decode_step and mha_decode_step need for
+ * these sizes on the current device (an upper bound valid for both; 0 if the arguments are
+ * not valid).  Host-only; touches no device memory.
+ */
+size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v);
+
+/*
+ * mqa_plan_splits -- how many splits of the memory axis the step will use for these sizes on
+ * the current device (`multi_query` non-zero: mqa_decode_step, zero: mha_decode_step), and,
+ * through *chunk_rows (optional), the rows per split.  Returns 0 for invalid arguments.
+ * Informational: lets a caller see the launch plan; host-only.
+ */
+int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int* chunk_rows);
+
+/* mqa_status_string -- a static, human-readable name for a return code. */
+const char* mqa_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MQA_DECODE_H_ */

@@ -1,0 +1,189 @@
+"""ctypes binding of ``libmqa_decode.so`` (the C ABI of ``include/mqa_decode.h``).
+
+Argument marshalling only: every function here checks tensor dtypes/shapes, takes device
+pointers and the current CUDA stream from PyTorch and calls the C entry point of the same
+name.  All arithmetic of the decode step runs inside the library's CUDA kernels.  There is
+no fallback: if the library is missing or was not built, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmqa_decode.so")
+
+MQA_OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 1, 2, 3, 4
+STATUS_APPEND_CACHE_FULL, STATUS_APPEND_NEGATIVE_LEN, STATUS_LEN_CLAMPED, STATUS_PIPELINE_TIMEOUT = 1, 2, 4, 8
+
+EXPORTS = (
+    "kv_cache_append", "mqa_decode_step", "mha_decode_step",
+    "mqa_decode_step_split", "mqa_decode_step_combine",
+    "mha_decode_step_split", "mha_decode_step_combine",
+    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string",
+)
+
+_lib = None
+
+
+class MqaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (code {code})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_1911_02150_b200.build` "
+                "(the decode step has no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, I, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.kv_cache_append.argtypes = [vp, vp, vp, vp, vp, I, vp, I, I, I, I, I, vp]
+        L.kv_cache_append.restype = I
+        for n in ("mqa_decode_step", "mha_decode_step", "mqa_decode_step_split", "mha_decode_step_split"):
+            f = getattr(L, n)
+            f.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, I, I, I, I, I, vp]
+            f.restype = I
+        for n in ("mqa_decode_step_combine", "mha_decode_step_combine"):
+            f = getattr(L, n)
+            f.argtypes = [vp, vp, vp, sz, I, I, I, I, I, vp]
+            f.restype = I
+        L.mqa_workspace_bytes.argtypes = [I, I, I, I, I]
+        L.mqa_workspace_bytes.restype = sz
+        L.mqa_plan_splits.argtypes = [I, I, I, I, I, I, ctypes.POINTER(I)]
+        L.mqa_plan_splits.restype = I
+        L.mqa_status_string.argtypes = [I]
+        L.mqa_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().mqa_status_string(int(code)).decode()
+
+
+def workspace_bytes(b: int, h: int, m_max: int, k: int = 128, v: int = 128) -> int:
+    return int(lib().mqa_workspace_bytes(b, h, m_max, k, v))
+
+
+def plan_splits(multi_query: bool, b: int, h: int, m_max: int, k: int = 128, v: int = 128):
+    """(n_splits, chunk_rows) the library will use for these sizes on the current device."""
+    chunk = ctypes.c_int(0)
+    n = lib().mqa_plan_splits(int(bool(multi_query)), b, h, m_max, k, v, ctypes.byref(chunk))
+    return int(n), int(chunk.value)
+
+
+def alloc_workspace(b: int, h: int, m_max: int, device, k: int = 128, v: int = 128) -> torch.Tensor:
+    """A byte tensor large enough for both step variants at these sizes (at least 16 bytes)."""
+    with torch.cuda.device(device):
+        n = workspace_bytes(b, h, m_max, k, v)
+    return torch.empty(max(n, 16), dtype=torch.uint8, device=device)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _need(t: torch.Tensor, dtype, shape, name: str):
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+
+
+def _check(rc: int, where: str):
+    if rc != MQA_OK:
+        raise MqaError(rc, where)
+
+
+def kv_cache_append(K, V, k_new, v_new, lens, advance: bool = True, status=None, stream=None) -> None:
+    """Write the new token's rows into row ``lens[b]`` of the cache, in place.
+
+    ``K``/``V``: ``[b,m_max,128]`` (multi-query) or ``[b,kv_heads,m_max,128]`` (multi-head) bf16;
+    ``k_new``/``v_new``: ``[b,128]`` or ``[b,kv_heads,128]``; ``lens``: int32 ``[b]``, advanced by one
+    on the device when ``advance``."""
+    if K.dim() == 3:
+        b, m_max, k = K.shape
+        kvh = 1
+        new_shape = (b, k)
+    else:
+        b, kvh, m_max, k = K.shape
+        new_shape = (b, kvh, k)
+    v = V.shape[-1]
+    _need(K, torch.bfloat16, K.shape, "K")
+    _need(V, torch.bfloat16, tuple(K.shape[:-1]) + (v,), "V")
+    _need(k_new, torch.bfloat16, new_shape, "k_new")
+    _need(v_new, torch.bfloat16, new_shape[:-1] + (v,), "v_new")
+    _need(lens, torch.int32, (b,), "lens")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    with torch.cuda.device(K.device):
+        rc = lib().kv_cache_append(_ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(lens), int(bool(advance)),
+                                   _ptr(status), b, kvh, m_max, k, v, _stream(stream))
+    _check(rc, "kv_cache_append")
+
+
+def _step(name: str, multi_query: bool, q, K, V, lens, o, workspace, status, stream, phase: str):
+    b, h, k = q.shape
+    m_max, v = K.shape[-2], V.shape[-1]
+    cache = (b, m_max) if multi_query else (b, h, m_max)
+    _need(q, torch.bfloat16, (b, h, k), "q")
+    _need(K, torch.bfloat16, cache + (k,), "K")
+    _need(V, torch.bfloat16, cache + (v,), "V")
+    _need(lens, torch.int32, (b,), "lens")
+    _need(o, torch.float32, (b, h, v), "o")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (_ptr(workspace), workspace.numel() * workspace.element_size())
+    with torch.cuda.device(q.device):
+        if phase == "combine":
+            rc = getattr(lib(), name)(_ptr(lens), _ptr(o), ws_ptr, ws_bytes, b, h, m_max, k, v, _stream(stream))
+        else:
+            rc = getattr(lib(), name)(_ptr(q), _ptr(K), _ptr(V), _ptr(lens), _ptr(o), ws_ptr, ws_bytes,
+                                      _ptr(status), b, h, m_max, k, v, _stream(stream))
+    _check(rc, name)
+    return o
+
+
+def mqa_decode_step(q, K, V, lens, o, workspace=None, status=None, stream=None):
+    """Multi-query step: ``q[b,h,128]`` over the shared ``K[b,m_max,128]``, ``V[b,m_max,128]`` (bf16),
+    first ``lens[b]`` rows -> ``o[b,h,128]`` fp32 (written in place and returned)."""
+    return _step("mqa_decode_step", True, q, K, V, lens, o, workspace, status, stream, "step")
+
+
+def mha_decode_step(q, K, V, lens, o, workspace=None, status=None, stream=None):
+    """Multi-head step: as above with per-head caches ``K[b,h,m_max,128]``, ``V[b,h,m_max,128]``."""
+    return _step("mha_decode_step", False, q, K, V, lens, o, workspace, status, stream, "step")
+
+
+def mqa_decode_step_split(q, K, V, lens, o, workspace=None, status=None, stream=None):
+    return _step("mqa_decode_step_split", True, q, K, V, lens, o, workspace, status, stream, "split")
+
+
+def mha_decode_step_split(q, K, V, lens, o, workspace=None, status=None, stream=None):
+    return _step("mha_decode_step_split", False, q, K, V, lens, o, workspace, status, stream, "split")
+
+
+def mqa_decode_step_combine(q, K, V, lens, o, workspace=None, status=None, stream=None):
+    return _step("mqa_decode_step_combine", True, q, K, V, lens, o, workspace, status, stream, "combine")
+
+
+def mha_decode_step_combine(q, K, V, lens, o, workspace=None, status=None, stream=None):
+    return _step("mha_decode_step_combine", False, q, K, V, lens, o, workspace, status, stream, "combine")

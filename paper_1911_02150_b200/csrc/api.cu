@@ -1,0 +1,228 @@
+// C-ABI entry points of the decode-attention library (declared in include/mqa_decode.h):
+// argument validation, the launch plan, and the kernel launches.  Host code here never
+// synchronises, allocates or frees device memory.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/mqa_decode.h"
+#include "append.cuh"
+#include "combine.cuh"
+#include "common.cuh"
+#include "decode_simt.cuh"
+
+namespace mqa {
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::atomic<int> g_sm_count[kMaxDevices];
+
+// Number of SMs of the current device (148 on a B200); 148 when no device can be queried,
+// so that the host-only planning calls still answer on a machine without a GPU.
+int sm_count() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+    if (dev < 0 || dev >= kMaxDevices) return 148;
+    int n = g_sm_count[dev].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return 148;
+    }
+    g_sm_count[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+
+struct Plan {
+    int n_splits = 0;     // 0 = invalid
+    int chunk_rows = 0;   // rows of the memory axis per split (multiple of 64)
+    size_t units = 0;     // b * h
+};
+
+bool dims_ok(int b, int h, int m_max) { return b > 0 && h > 0 && m_max > 0; }
+
+// Split plan for the CUDA-core kernel (one CTA per (unit, split)): enough CTAs to fill every
+// SM several times over, but never chunks shorter than 256 rows, and a single split (no
+// combine launch) when the cache is short.
+Plan plan_simt(int b, int h, int m_max) {
+    Plan p;
+    p.units = (size_t)b * h;
+    const long target_ctas = (long)sm_count() * 16;
+    long want = (target_ctas + (long)p.units - 1) / (long)p.units;
+    const long cap = m_max / 256 > 1 ? m_max / 256 : 1;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    int chunk = (int)((m_max + want - 1) / want);
+    chunk = (chunk + 63) / 64 * 64;
+    p.chunk_rows = chunk;
+    p.n_splits = (m_max + chunk - 1) / chunk;
+    return p;
+}
+
+Plan make_plan(bool multi_query, int b, int h, int m_max) {
+    (void)multi_query;
+    return plan_simt(b, h, m_max);
+}
+
+size_t plan_workspace_bytes(const Plan& p) {
+    if (p.n_splits <= 1) return 0;
+    return partial_ml_bytes(p.units, p.n_splits) + partial_acc_bytes(p.units, p.n_splits);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+int check_step_args(const void* q, const void* K, const void* V, const int32_t* lens, const float* o,
+                    const int32_t* status, int b, int h, int m_max, int k, int v) {
+    if (!q || !K || !V || !lens || !o) return MQA_ERR_INVALID_ARG;
+    if (!dims_ok(b, h, m_max) || k <= 0 || v <= 0) return MQA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(o) || !aligned4(lens) ||
+        !aligned4(status))
+        return MQA_ERR_INVALID_ARG;
+    if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
+    return MQA_OK;
+}
+
+int check_workspace(const Plan& p, const void* workspace, size_t workspace_bytes) {
+    const size_t need = plan_workspace_bytes(p);
+    if (need == 0) return MQA_OK;
+    if (!workspace || !aligned16(workspace)) return MQA_ERR_INVALID_ARG;
+    if (workspace_bytes < need) return MQA_ERR_WORKSPACE_TOO_SMALL;
+    return MQA_OK;
+}
+
+int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
+
+int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+              void* workspace, size_t workspace_bytes, int32_t* status,
+              int b, int h, int m_max, int k, int v, cudaStream_t stream) {
+    int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
+    if (rc) return rc;
+    const Plan p = make_plan(multi_query, b, h, m_max);
+    if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
+    rc = check_workspace(p, workspace, workspace_bytes);
+    if (rc) return rc;
+    float2* part_ml = reinterpret_cast<float2*>(workspace);
+    float* part_acc = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
+                                                           partial_ml_bytes(p.units, p.n_splits))
+                                : nullptr;
+    const unsigned grid = (unsigned)(p.units * (size_t)p.n_splits);
+    decode_split_simt_kernel<<<grid, kSimtThreads, 0, stream>>>(
+        static_cast<const uint4*>(q), static_cast<const uint4*>(K), static_cast<const uint4*>(V), lens, o,
+        part_ml, part_acc, status, h, multi_query ? h : 1, m_max, p.chunk_rows, p.n_splits);
+    return launch_status();
+}
+
+int run_combine(bool multi_query, const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes,
+                int b, int h, int m_max, int k, int v, cudaStream_t stream) {
+    if (!lens || !o || !dims_ok(b, h, m_max) || !aligned16(o) || !aligned4(lens)) return MQA_ERR_INVALID_ARG;
+    if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
+    const Plan p = make_plan(multi_query, b, h, m_max);
+    if (p.units > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
+    int rc = check_workspace(p, workspace, workspace_bytes);
+    if (rc) return rc;
+    if (p.n_splits <= 1) return MQA_OK;
+    const float2* part_ml = reinterpret_cast<const float2*>(workspace);
+    const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +
+                                                           partial_ml_bytes(p.units, p.n_splits));
+    combine_splits_kernel<<<(unsigned)p.units, kHeadDim, 0, stream>>>(part_ml, part_acc, lens, o, h, m_max,
+                                                                      p.chunk_rows, p.n_splits);
+    return launch_status();
+}
+
+int run_step(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+             void* workspace, size_t workspace_bytes, int32_t* status,
+             int b, int h, int m_max, int k, int v, cudaStream_t stream) {
+    int rc = run_split(multi_query, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream);
+    if (rc) return rc;
+    return run_combine(multi_query, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream);
+}
+
+}  // namespace
+}  // namespace mqa
+
+using namespace mqa;
+
+extern "C" {
+
+int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new, int32_t* lens, int advance,
+                    int32_t* status, int b, int kv_heads, int m_max, int k, int v, mqa_stream_t stream) {
+    if (!K || !V || !k_new || !v_new || !lens) return MQA_ERR_INVALID_ARG;
+    if (b <= 0 || kv_heads <= 0 || m_max <= 0 || k <= 0 || v <= 0) return MQA_ERR_INVALID_ARG;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(k_new) || !aligned16(v_new) || !aligned4(lens) ||
+        !aligned4(status))
+        return MQA_ERR_INVALID_ARG;
+    if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
+    kv_cache_append_kernel<<<(unsigned)b, kAppendThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<uint4*>(K), static_cast<uint4*>(V), static_cast<const uint4*>(k_new),
+        static_cast<const uint4*>(v_new), lens, advance, status, kv_heads, m_max);
+    return launch_status();
+}
+
+int mqa_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o, void* workspace,
+                    size_t workspace_bytes, int32_t* status, int b, int h, int m_max, int k, int v,
+                    mqa_stream_t stream) {
+    return run_step(true, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v,
+                    static_cast<cudaStream_t>(stream));
+}
+
+int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o, void* workspace,
+                    size_t workspace_bytes, int32_t* status, int b, int h, int m_max, int k, int v,
+                    mqa_stream_t stream) {
+    return run_step(false, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v,
+                    static_cast<cudaStream_t>(stream));
+}
+
+int mqa_decode_step_split(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                          void* workspace, size_t workspace_bytes, int32_t* status, int b, int h, int m_max,
+                          int k, int v, mqa_stream_t stream) {
+    return run_split(true, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int mqa_decode_step_combine(const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes, int b,
+                            int h, int m_max, int k, int v, mqa_stream_t stream) {
+    return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v,
+                       static_cast<cudaStream_t>(stream));
+}
+
+int mha_decode_step_split(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                          void* workspace, size_t workspace_bytes, int32_t* status, int b, int h, int m_max,
+                          int k, int v, mqa_stream_t stream) {
+    return run_split(false, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes, int b,
+                            int h, int m_max, int k, int v, mqa_stream_t stream) {
+    return run_combine(false, lens, o, workspace, workspace_bytes, b, h, m_max, k, v,
+                       static_cast<cudaStream_t>(stream));
+}
+
+size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v) {
+    if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
+    const size_t a = plan_workspace_bytes(make_plan(true, b, h, m_max));
+    const size_t c = plan_workspace_bytes(make_plan(false, b, h, m_max));
+    return a > c ? a : c;
+}
+
+int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int* chunk_rows) {
+    if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
+    const Plan p = make_plan(multi_query != 0, b, h, m_max);
+    if (chunk_rows) *chunk_rows = p.chunk_rows;
+    return p.n_splits;
+}
+
+const char* mqa_status_string(int code) {
+    switch (code) {
+        case MQA_OK: return "ok";
+        case MQA_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, non-positive dimension)";
+        case MQA_ERR_UNSUPPORTED: return "unsupported configuration (k and v must be 128)";
+        case MQA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small (see mqa_workspace_bytes)";
+        case MQA_ERR_CUDA: return "CUDA launch error";
+        default: return "unknown status code";
+    }
+}
+
+}  // extern "C"

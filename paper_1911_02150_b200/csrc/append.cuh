@@ -1,0 +1,38 @@
+// kv_cache_append kernel: one CTA per sequence copies the new token's key and value row of
+// every cache head into row lens[b] (the in-place form of the concatenation on the memory
+// axis in Sections 2.4 and 3).  Rows move as 16-byte words and are never interpreted.
+#pragma once
+#include "common.cuh"
+
+namespace mqa {
+
+constexpr int kAppendThreads = 256;  // 8 warps: one (cache head) row pair per warp per pass
+
+__global__ void __launch_bounds__(kAppendThreads)
+kv_cache_append_kernel(uint4* __restrict__ K, uint4* __restrict__ V,
+                       const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                       int32_t* __restrict__ lens, int advance, int32_t* __restrict__ status,
+                       int kv_heads, int m_max) {
+    const int bi = blockIdx.x;
+    const int row = lens[bi];
+    if (row < 0 || row >= m_max) {   // uniform over the CTA
+        if (threadIdx.x == 0 && status)
+            atomicOr(status, row < 0 ? kStatusAppendNegative : kStatusAppendFull);
+        return;
+    }
+    constexpr int kVecPerRow = kRowBytes / 16;               // 16 uint4 per row
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int vec = lane & (kVecPerRow - 1);
+    const bool is_v = lane >= kVecPerRow;                    // lanes 0-15 copy K, 16-31 copy V
+    for (int g = warp; g < kv_heads; g += kAppendThreads / 32) {
+        const size_t src = ((size_t)bi * kv_heads + g) * kVecPerRow + vec;
+        const size_t dst = (((size_t)bi * kv_heads + g) * m_max + row) * kVecPerRow + vec;
+        if (is_v) V[dst] = v_new[src]; else K[dst] = k_new[src];
+    }
+    if (advance) {
+        __syncthreads();             // every warp has read lens[bi] before it moves
+        if (threadIdx.x == 0) lens[bi] = row + 1;
+    }
+}
+
+}  // namespace mqa

@@ -1,0 +1,44 @@
+// Shared device helpers for the decode-attention kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mqa {
+
+constexpr int kHeadDim = 128;                 // k == v == 128 (Section 4.1: d_k = d_v = 128)
+constexpr int kRowBytes = kHeadDim * 2;       // one bf16 cache row
+constexpr float kLog2e = 1.4426950408889634f;
+
+// status bits (mirrors include/mqa_decode.h)
+constexpr int kStatusAppendFull = 1;
+constexpr int kStatusAppendNegative = 2;
+constexpr int kStatusLenClamped = 4;
+constexpr int kStatusPipelineTimeout = 8;
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// 16-byte read-only global load that does not allocate in L1 (each cache byte is used once).
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+// Clamp a sequence length into [0, m_max]; flag the status word if it had to move.
+__device__ __forceinline__ int clamp_len(int L, int m_max, int32_t* status) {
+    if (L < 0 || L > m_max) {
+        if (status) atomicOr(status, kStatusLenClamped);
+        L = L < 0 ? 0 : m_max;
+    }
+    return L;
+}
+
+}  // namespace mqa

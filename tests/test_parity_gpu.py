@@ -1,0 +1,356 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the
+same seeded bf16 inputs.
+
+Tolerance (from the build's stated target, bf16 inputs with fp32 accumulation):
+  * every element: |gpu - oracle| <= 4e-3;
+  * every (sequence, head) row: max_c |gpu - oracle| <= 1e-2 * max_c |oracle|  (relative to the
+    row's scale -- at long context the outputs are ~1e-2 and element-wise relative error is
+    ill-posed near zero crossings).
+The cache append is compared bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1911_02150_b200 as mqa
+from paper_1911_02150_b200 import binding, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+ABS_TOL = 4e-3
+REL_TOL = 1e-2
+DEV = "cuda:0"
+
+
+def check_close(got: np.ndarray, ref: np.ndarray, what: str = ""):
+    assert got.shape == ref.shape
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    err = np.abs(got.astype(np.float64) - ref)
+    assert err.max() <= ABS_TOL, f"{what}: max abs err {err.max():.3e}"
+    row_err = err.max(axis=-1)
+    row_ref = np.abs(ref).max(axis=-1)
+    bad = row_err > REL_TOL * row_ref
+    assert not bad.any(), f"{what}: {bad.sum()} rows over relative tolerance, worst {np.max(row_err / np.maximum(row_ref, 1e-300)):.3e}"
+
+
+def oracle_step(variant, q, K, V, lens_np, idx=None):
+    """Oracle on all sequences, or on the sampled ones in idx."""
+    if idx is not None:
+        sel = torch.as_tensor(idx, device=q.device)
+        q, K, V, lens_np = q[sel], K[sel], V[sel], lens_np[idx]
+    fn = oracle.mqa_decode_step if variant == "mqa" else oracle.mha_decode_step
+    return fn(wl.bits(q), wl.bits(K), wl.bits(V), lens_np.astype(np.int32))
+
+
+def gpu_step(variant, q, K, V, lens_t, expect_status=0):
+    b, h, _ = q.shape
+    o = torch.full((b, h, V.shape[-1]), float("nan"), dtype=torch.float32, device=q.device)
+    ws = mqa.alloc_workspace(b, h, K.shape[-2], q.device)
+    ws.fill_(0xFF)                                     # stale NaN bit patterns in the scratch
+    status = torch.zeros(1, dtype=torch.int32, device=q.device)
+    fn = mqa.mqa_decode_step if variant == "mqa" else mqa.mha_decode_step
+    fn(q, K, V, lens_t, o, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == expect_status
+    return o
+
+
+def run_case(variant, b, h, m_max, lens_np, seed=0, sample=None):
+    inp = wl.make_inputs(b, h, m_max, variant, seed=seed, device=DEV)
+    lens_np = np.asarray(lens_np, dtype=np.int32)
+    wl.poison_tail(inp["K"], lens_np)
+    wl.poison_tail(inp["V"], lens_np)
+    lens_t = torch.from_numpy(lens_np).to(DEV)
+    o = gpu_step(variant, inp["q"], inp["K"], inp["V"], lens_t)
+    got = o.cpu().numpy()
+    if sample is None:
+        ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], lens_np)
+    else:
+        ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], lens_np, sample)
+        got = got[sample]
+    check_close(got, ref, f"{variant} b={b} h={h} m_max={m_max}")
+    return inp, o
+
+
+SMALL = [
+    # b, h, m_max, lens
+    (1, 1, 1, [1]),
+    (1, 8, 128, [128]),                       # the single-step configuration
+    (3, 8, 300, [300, 1, 77]),                # ragged, several tiles, odd tails
+    (2, 16, 1000, [999, 513]),
+    (2, 32, 700, [700, 65]),
+    (4, 5, 257, [257, 256, 255, 2]),          # a head count outside {8, 16, 32}
+    (2, 12, 4096, [4096, 3000]),              # several splits
+    (5, 16, 64, [64, 63, 33, 17, 16]),
+    (1, 16, 20000, [19999]),                  # many splits of one sequence
+]
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+@pytest.mark.parametrize("b,h,m_max,lens", SMALL)
+def test_small_cases_match_oracle(variant, b, h, m_max, lens):
+    run_case(variant, b, h, m_max, lens, seed=b * 1000 + h)
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+@pytest.mark.parametrize("edge", range(60, 70))
+def test_every_length_around_a_tile_edge(variant, edge):
+    """lens = 60..69 crosses the 64-row boundary the kernels tile by."""
+    run_case(variant, 2, 8, 256, [edge, 256 - edge], seed=edge)
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_long_context_configuration(variant):
+    """b=32, h=32, m_max=8192: 8191 rows resident, the step appends row 8191 and attends over 8192."""
+    w = wl.WORKLOADS["long_context"]
+    inp = wl.make_inputs(w.b, w.h, w.m_max, variant, seed=0, device=DEV)
+    lens0 = wl.initial_lens(w)
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    Kbefore = inp["K"].clone() if variant == "mqa" else None
+    mqa.kv_cache_append(inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, advance=True)
+    o = gpu_step(variant, inp["q"], inp["K"], inp["V"], lens_t)
+    assert torch.equal(lens_t.cpu(), torch.from_numpy(lens0 + 1))
+    if Kbefore is not None:                            # only the appended row changed
+        same = (Kbefore.view(torch.int16) == inp["K"].view(torch.int16)).all(dim=-1)
+        assert bool(same[:, : w.m_max - 1].all())
+        assert torch.equal(inp["K"][:, w.m_max - 1].view(torch.int16), inp["k_new"].view(torch.int16))
+    sample = None if variant == "mqa" else [0, 7, 31]  # 3 of 32 sequences (all heads) for the 4 GiB cache
+    lens_np = lens0 + 1
+    ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], lens_np, sample)
+    got = o.cpu().numpy() if sample is None else o.cpu().numpy()[sample]
+    check_close(got, ref, f"long_context {variant}")
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_ragged_configuration(variant):
+    """b=256, h=16, m_max=2048, valid lengths uniform on [1, 2048], dead rows NaN-poisoned."""
+    w = wl.WORKLOADS["ragged"]
+    lens = wl.ragged_lens(w.b, w.m_max, seed=0)
+    assert lens.min() >= 1 and lens.max() <= w.m_max
+    sample = None if variant == "mqa" else list(range(0, 256, 16))
+    run_case(variant, w.b, w.h, w.m_max, lens, seed=0, sample=sample)
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_paper_incremental_decoding(variant):
+    """b=128, h=8: the cache grows from 1 to 128 rows over 128 steps (append, then attend over the
+    prefix); each step's output is checked against the oracle on the cache as it then stands."""
+    w = wl.WORKLOADS["paper_incremental"]
+    b, h, m_max = w.b, w.h, w.m_max
+    base = wl.make_inputs(b, h, m_max, variant, seed=0, device=DEV)
+    K, V = base["K"], base["V"]
+    nan = torch.tensor(wl.NAN_BITS, dtype=torch.int16, device=DEV)
+    K.view(torch.int16).fill_(nan)                     # nothing is valid before the first append
+    V.view(torch.int16).fill_(nan)
+    lens_t = torch.zeros(b, dtype=torch.int32, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    step_fn = mqa.mqa_decode_step if variant == "mqa" else mqa.mha_decode_step
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(1234)
+    new_shape = (b,) if variant == "mqa" else (b, h)
+    outs, qs = [], []
+    for t in range(w.steps):
+        q = wl.bf16_normal((b, h, 128), 128 ** -0.5, gen, DEV)
+        k_new = wl.bf16_normal(new_shape + (128,), 1.0, gen, DEV)
+        v_new = wl.bf16_normal(new_shape + (128,), 1.0, gen, DEV)
+        mqa.kv_cache_append(K, V, k_new, v_new, lens_t, advance=True, status=status)
+        o = torch.empty(b, h, 128, dtype=torch.float32, device=DEV)
+        step_fn(q, K, V, lens_t, o, ws, status)
+        outs.append(o)
+        qs.append(q)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(lens_t.cpu(), torch.full((b,), w.steps, dtype=torch.int32))
+    Kb, Vb = wl.bits(K), wl.bits(V)                    # rows are immutable once written
+    ofn = oracle.mqa_decode_step if variant == "mqa" else oracle.mha_decode_step
+    for t in range(w.steps):
+        ref = ofn(wl.bits(qs[t]), Kb, Vb, np.full(b, t + 1, np.int32))
+        check_close(outs[t].cpu().numpy(), ref, f"{variant} step {t + 1}")
+
+
+SWEEP = [("mqa", 1, 512), ("mha", 1, 512), ("mqa", 8, 4096), ("mha", 8, 4096), ("mqa", 64, 32768),
+         ("mha", 8, 32768), ("mqa", 256, 32768), ("mha", 64, 4096)]
+
+
+@pytest.mark.parametrize("variant,b,m", SWEEP)
+def test_sweep_points(variant, b, m):
+    """h=16 sweep points, full-length caches; large points are checked on sampled sequences."""
+    rng = np.random.default_rng(b * 7 + m)
+    n_s = 8 if m < 32768 else 3
+    sample = None if b <= n_s else sorted({0, b - 1, *rng.integers(0, b, size=n_s - 2).tolist()})
+    run_case(variant, b, 16, m, np.full(b, m, np.int32), seed=m + b, sample=sample)
+
+
+def test_largest_multihead_sweep_point_if_it_fits():
+    """b=256, m=32768, h=16 in multi-head form is a 64 GiB cache: 2^35 elements per tensor pair,
+    beyond 32-bit indexing.  Checked on three sampled sequences."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80 * 2 ** 30:
+        pytest.skip("less than 80 GiB free on this GPU")
+    b, h, m = 256, 16, 32768
+    run_case("mha", b, h, m, np.full(b, m, np.int32), seed=5, sample=[0, 129, 255])
+
+
+# ----------------------------------------------------------------------------- properties
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_dead_rows_never_contribute_bitwise(variant):
+    b, h, m_max = 6, 16, 1500
+    lens = np.array([1, 64, 65, 700, 1499, 1500], np.int32)
+    inp = wl.make_inputs(b, h, m_max, variant, seed=3, device=DEV)
+    lens_t = torch.from_numpy(lens).to(DEV)
+    outs = []
+    for pattern in (0x0000, wl.NAN_BITS, 0x7F80, 0xFF80, 0x7F7F):    # zeros, NaN, +inf, -inf, huge
+        K, V = inp["K"].clone(), inp["V"].clone()
+        wl.poison_tail(K, lens, pattern)
+        wl.poison_tail(V, lens, pattern)
+        outs.append(gpu_step(variant, inp["q"], K, V, lens_t))
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int32), outs[0].view(torch.int32))
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_two_runs_are_bit_identical(variant):
+    b, h, m_max = 16, 16, 5000
+    lens = wl.ragged_lens(b, m_max, seed=4)
+    inp = wl.make_inputs(b, h, m_max, variant, seed=4, device=DEV)
+    lens_t = torch.from_numpy(lens).to(DEV)
+    a = gpu_step(variant, inp["q"], inp["K"], inp["V"], lens_t)
+    c = gpu_step(variant, inp["q"], inp["K"], inp["V"], lens_t)
+    assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+
+
+def test_multiquery_equals_multihead_on_replicated_cache():
+    """Section 3: multi-query is multi-head whose heads share one K and V."""
+    b, h, m_max = 3, 16, 900
+    lens = np.array([900, 450, 3], np.int32)
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=5, device=DEV)
+    lens_t = torch.from_numpy(lens).to(DEV)
+    o_q = gpu_step("mqa", inp["q"], inp["K"], inp["V"], lens_t)
+    Krep = inp["K"][:, None].expand(b, h, m_max, 128).contiguous()
+    Vrep = inp["V"][:, None].expand(b, h, m_max, 128).contiguous()
+    o_h = gpu_step("mha", inp["q"], Krep, Vrep, lens_t)
+    assert float((o_q - o_h).abs().max()) <= 2e-5
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_dominant_logit_returns_that_row_exactly(variant):
+    b, h, m_max, star = 1, 8, 333, 201
+    inp = wl.make_inputs(b, h, m_max, variant, seed=6, device=DEV)
+    q = torch.zeros_like(inp["q"]); q[..., 0] = 1.0
+    K = torch.zeros_like(inp["K"]); K[..., star, 0] = 200.0
+    lens_t = torch.full((b,), m_max, dtype=torch.int32, device=DEV)
+    o = gpu_step(variant, q, K, inp["V"], lens_t)
+    want = inp["V"][..., star, :].float()
+    want = want.expand(b, h, 128) if variant == "mqa" else want
+    assert torch.equal(o, want.contiguous())
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_identical_keys_give_the_mean(variant):
+    b, h, m_max = 2, 8, 512
+    inp = wl.make_inputs(b, h, m_max, variant, seed=7, device=DEV)
+    K = inp["K"].clone()
+    K[..., :, :] = K[..., :1, :]
+    lens = np.array([512, 100], np.int32)
+    o = gpu_step(variant, inp["q"], K, inp["V"], torch.from_numpy(lens).to(DEV))
+    for s in range(b):
+        mean = inp["V"][s, ..., : lens[s], :].double().mean(dim=-2)
+        ref = mean.expand(h, 128) if variant == "mqa" else mean
+        assert float((o[s].double() - ref).abs().max()) <= 1e-5
+
+
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+def test_empty_and_out_of_range_lengths(variant):
+    b, h, m_max = 4, 8, 200
+    inp = wl.make_inputs(b, h, m_max, variant, seed=8, device=DEV)
+    lens = np.array([0, 200, -3, 999], np.int32)        # empty, full, negative (-> 0), too long (-> 200)
+    o = gpu_step(variant, inp["q"], inp["K"], inp["V"], torch.from_numpy(lens).to(DEV),
+                 expect_status=binding.STATUS_LEN_CLAMPED)
+    ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], np.array([0, 200, 0, 200], np.int32))
+    check_close(o.cpu().numpy()[[1, 3]], ref[[1, 3]], "clamped")
+    assert float(o[0].abs().max()) == 0.0 and float(o[2].abs().max()) == 0.0
+    # a batch made only of empty sequences, at a size that uses several splits
+    b2, m2 = 2, 8192
+    inp2 = wl.make_inputs(b2, h, m2, variant, seed=9, device=DEV)
+    o2 = gpu_step(variant, inp2["q"], inp2["K"], inp2["V"], torch.zeros(b2, dtype=torch.int32, device=DEV))
+    assert float(o2.abs().max()) == 0.0
+
+
+def test_split_and_combine_phases_equal_the_step():
+    b, h, m_max = 4, 16, 9000
+    lens = np.array([9000, 1, 4500, 8999], np.int32)
+    for variant in ("mqa", "mha"):
+        inp = wl.make_inputs(b, h, m_max, variant, seed=10, device=DEV)
+        lens_t = torch.from_numpy(lens).to(DEV)
+        whole = gpu_step(variant, inp["q"], inp["K"], inp["V"], lens_t)
+        o = torch.full_like(whole, float("nan"))
+        ws = mqa.alloc_workspace(b, h, m_max, DEV)
+        split = mqa.mqa_decode_step_split if variant == "mqa" else mqa.mha_decode_step_split
+        comb = mqa.mqa_decode_step_combine if variant == "mqa" else mqa.mha_decode_step_combine
+        split(inp["q"], inp["K"], inp["V"], lens_t, o, ws)
+        comb(inp["q"], inp["K"], inp["V"], lens_t, o, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(o.view(torch.int32), whole.view(torch.int32))
+
+
+# --------------------------------------------------------------------------------- append
+@pytest.mark.parametrize("kvh", [1, 8, 40])
+def test_append_is_bit_exact_and_touches_one_row(kvh):
+    b, m_max = 5, 37
+    g = torch.Generator(device="cpu"); g.manual_seed(11)
+    shape = (b, m_max, 128) if kvh == 1 else (b, kvh, m_max, 128)
+    new = (b, 128) if kvh == 1 else (b, kvh, 128)
+    rnd = lambda s: torch.randint(-32768, 32768, s, generator=g, dtype=torch.int16)
+    K, V, k_new, v_new = rnd(shape), rnd(shape), rnd(new), rnd(new)
+    k_new[..., :6] = torch.tensor([-32768, 1, 0x7FC1, -1, 0x7F80, -128], dtype=torch.int16)  # -0.0, subnormal, NaNs, infs
+    lens = np.array([0, 36, 37, 5, -1], np.int32)       # full and negative sequences are skipped
+    Kd, Vd = K.to(DEV).view(torch.bfloat16), V.to(DEV).view(torch.bfloat16)
+    lens_t = torch.from_numpy(lens).to(DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mqa.kv_cache_append(Kd, Vd, k_new.to(DEV).view(torch.bfloat16), v_new.to(DEV).view(torch.bfloat16), lens_t,
+                        advance=True, status=status)
+    torch.cuda.synchronize()
+    Kh, Vh, lens_h = K.numpy().view(np.uint16).copy(), V.numpy().view(np.uint16).copy(), lens.copy()
+    skipped = oracle.kv_cache_append(Kh, Vh, k_new.numpy().view(np.uint16), v_new.numpy().view(np.uint16), lens_h, True)
+    assert skipped == 2
+    assert int(status.item()) == binding.STATUS_APPEND_CACHE_FULL | binding.STATUS_APPEND_NEGATIVE_LEN
+    assert np.array_equal(wl.bits(Kd), Kh) and np.array_equal(wl.bits(Vd), Vh)
+    assert np.array_equal(lens_t.cpu().numpy(), lens_h)
+    # advance = 0 leaves lens alone
+    keep = lens_t.clone()
+    mqa.kv_cache_append(Kd, Vd, k_new.to(DEV).view(torch.bfloat16), v_new.to(DEV).view(torch.bfloat16), lens_t,
+                        advance=False)
+    torch.cuda.synchronize()
+    assert torch.equal(lens_t, keep)
+
+
+def test_errors_leave_outputs_untouched():
+    b, h, m_max = 1, 16, 32768
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=12, device=DEV)
+    lens_t = torch.full((b,), m_max, dtype=torch.int32, device=DEV)
+    o = torch.full((b, h, 128), 7.0, dtype=torch.float32, device=DEV)
+    n, _ = mqa.plan_splits(True, b, h, m_max)
+    assert n > 1
+    small = torch.empty(64, dtype=torch.uint8, device=DEV)
+    with pytest.raises(mqa.MqaError) as e:
+        mqa.mqa_decode_step(inp["q"], inp["K"], inp["V"], lens_t, o, small)
+    assert e.value.code == binding.ERR_WORKSPACE_TOO_SMALL
+    torch.cuda.synchronize()
+    assert bool((o == 7.0).all())
+
+
+def test_runs_on_a_side_stream():
+    b, h, m_max = 8, 16, 3000
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=13, device=DEV)
+    lens_t = torch.full((b,), m_max, dtype=torch.int32, device=DEV)
+    ref = gpu_step("mqa", inp["q"], inp["K"], inp["V"], lens_t)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    o = torch.zeros_like(ref)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    with torch.cuda.stream(s):
+        mqa.mqa_decode_step(inp["q"], inp["K"], inp["V"], lens_t, o, ws)
+    s.synchronize()
+    assert torch.equal(o.view(torch.int32), ref.view(torch.int32))
