@@ -1,6 +1,7 @@
 // C-ABI entry points of the decode-attention library (declared in include/mqa_decode.h):
 // argument validation, the launch plan, and the kernel launches.  Host code here never
 // synchronises, allocates or frees device memory.
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -10,6 +11,7 @@
 #include "append.cuh"
 #include "combine.cuh"
 #include "common.cuh"
+#include "decode_mma.cuh"
 #include "decode_simt.cuh"
 
 namespace mqa {
@@ -34,10 +36,13 @@ int sm_count() {
     return n;
 }
 
+enum class Kernel { kSimt, kMma1, kMma2 };
+
 struct Plan {
     int n_splits = 0;     // 0 = invalid
     int chunk_rows = 0;   // rows of the memory axis per split (multiple of 64)
     size_t units = 0;     // b * h
+    Kernel kernel = Kernel::kSimt;
 };
 
 bool dims_ok(int b, int h, int m_max) { return b > 0 && h > 0 && m_max > 0; }
@@ -60,8 +65,42 @@ Plan plan_simt(int b, int h, int m_max) {
     return p;
 }
 
+// Split plan for the tensor-core multi-query kernel (one CTA per (sequence, split), every CTA
+// serving all h heads).  A small cost model in units of "cache rows streamed by one SM":
+// CTAs run in waves over the resident slots, every CTA pays a fixed start-up/merge cost, and
+// every split adds partial results that are written once and read once by the combine pass.
+Plan plan_mma(int b, int h, int m_max) {
+    Plan p;
+    p.units = (size_t)b * h;
+    p.kernel = h <= 16 ? Kernel::kMma1 : Kernel::kMma2;
+    const int ctas_per_sm = h <= 16 ? MmaCfg<1>::kMinBlocks : MmaCfg<2>::kMinBlocks;
+    const long slots = (long)sm_count() * ctas_per_sm;
+    const double overhead_rows = 128.0;                               // start-up + merge, per CTA
+    const double partial_rows = (double)h * (kHeadDim + 2) * 4 * 2 / (2.0 * kRowBytes);   // per split
+    const int max_splits = m_max / 128 > 1 ? (m_max / 128 < 256 ? m_max / 128 : 256) : 1;
+    double best = 0;
+    for (int s = 1; s <= max_splits; ++s) {
+        int chunk = (m_max + s - 1) / s;
+        chunk = (chunk + kTileRows - 1) / kTileRows * kTileRows;
+        const int n = (m_max + chunk - 1) / chunk;
+        if (n != s) continue;                                         // same plan as a smaller s
+        const long ctas = (long)b * n;
+        const long waves = (ctas + slots - 1) / slots;
+        double cost = (double)waves * (chunk + overhead_rows) * ctas_per_sm;
+        if (n > 1) cost += (double)ctas * partial_rows / sm_count();
+        if (p.n_splits == 0 || cost < best) {
+            best = cost;
+            p.n_splits = n;
+            p.chunk_rows = chunk;
+        }
+    }
+    return p;
+}
+
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
-    (void)multi_query;
+    // heads beyond two 16-row tensor-core tiles, or a row space too large for the 32-bit TMA
+    // coordinates, go to the general CUDA-core kernel
+    if (multi_query && h <= 32 && (long long)b * m_max < 0x7fffffffLL) return plan_mma(b, h, m_max);
     return plan_simt(b, h, m_max);
 }
 
@@ -92,6 +131,66 @@ int check_workspace(const Plan& p, const void* workspace, size_t workspace_bytes
     return MQA_OK;
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+std::atomic<EncodeTiledFn> g_encode{nullptr};
+
+EncodeTiledFn encode_fn() {
+    EncodeTiledFn f = g_encode.load(std::memory_order_acquire);
+    if (f) return f;
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !sym) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    f = reinterpret_cast<EncodeTiledFn>(sym);
+    g_encode.store(f, std::memory_order_release);
+    return f;
+}
+
+// The cache of one tensor (K or V) as a 2-D bf16 tensor [rows = b * m_max][128 columns], fetched in
+// boxes of kTileRows rows x 64 columns (128 bytes, the span of the 128-byte swizzle).
+bool encode_cache_map(CUtensorMap* map, const void* base, long long rows) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
+    const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)kTileRows};
+    const cuuint32_t elem[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+std::atomic<int> g_smem_opt_in[kMaxDevices][2];
+
+template <int M_TILES>
+int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+               float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
+    using Cfg = MmaCfg<M_TILES>;
+    auto kernel = mqa_decode_split_mma_kernel<M_TILES>;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!g_smem_opt_in[dev][M_TILES - 1].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+        g_smem_opt_in[dev][M_TILES - 1].store(1, std::memory_order_release);
+    }
+    alignas(64) CUtensorMap map_k, map_v;
+    if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
+        return MQA_ERR_CUDA;
+    kernel<<<(unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream>>>(
+        map_k, map_v, static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
+        p.n_splits);
+    return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
+}
+
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
 
 int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
@@ -107,6 +206,10 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     float* part_acc = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits))
                                 : nullptr;
+    if (p.kernel == Kernel::kMma1)
+        return launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream);
+    if (p.kernel == Kernel::kMma2)
+        return launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream);
     const unsigned grid = (unsigned)(p.units * (size_t)p.n_splits);
     decode_split_simt_kernel<<<grid, kSimtThreads, 0, stream>>>(
         static_cast<const uint4*>(q), static_cast<const uint4*>(K), static_cast<const uint4*>(V), lens, o,

@@ -81,6 +81,8 @@ SMALL = [
     (2, 16, 1000, [999, 513]),
     (2, 32, 700, [700, 65]),
     (4, 5, 257, [257, 256, 255, 2]),          # a head count outside {8, 16, 32}
+    (2, 40, 600, [600, 31]),                  # more heads than two tensor-core tiles: general kernel
+    (3, 17, 95, [95, 32, 33]),                # 17 heads: second head tile nearly empty
     (2, 12, 4096, [4096, 3000]),              # several splits
     (5, 16, 64, [64, 63, 33, 17, 16]),
     (1, 16, 20000, [19999]),                  # many splits of one sequence
