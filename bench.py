@@ -141,14 +141,10 @@ class StepState:
         self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
         self.step_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
 
-    def step_phases(self, i, ev0, ev1):
-        """Same launches as step(), with events around the pass over the cache."""
+    def split_only(self, i):
+        """Only the pass over the cache (the dominant kernel) of step i."""
         s = self.sets[i % len(self.sets)]
-        self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
-        ev0.record()
         self.split_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
-        ev1.record()
-        self.combine_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
 
     def step_e2e(self, i):
         s = self.sets[i % len(self.sets)]
@@ -174,41 +170,60 @@ def time_region(fn, steps, device):
     return e0.elapsed_time(e1) * 1e-3
 
 
-def run_variant(st: StepState, steps, warmup, device, sample_clocks):
-    for i in range(warmup):
+def capture_graph(fn, steps):
+    """One CUDA graph holding `steps` calls of fn(i): the launch-bound loop is replayed with one
+    host call, so the device timeline has no host-side gaps between kernels."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(steps):
+            fn(i)
+    return g
+
+
+def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=True, min_warm_s=0.2):
+    t0 = time.time()
+    i = 0
+    while i < warmup or time.time() - t0 < min_warm_s:      # at least `warmup` steps, and clocks ramped up
         st.step(i)
+        i += 1
+        if i % 16 == 0:
+            torch.cuda.synchronize(device)
     torch.cuda.synchronize(device)
+    if use_graph:
+        g_step = capture_graph(st.step, steps)
+        g_split = capture_graph(st.split_only, steps)
+        g_step.replay(); g_split.replay()
+        torch.cuda.synchronize(device)
+        run_steps = lambda _i: g_step.replay()
+        run_split = lambda _i: g_split.replay()
+        calls = 1
+    else:
+        run_steps, run_split, calls = st.step, st.split_only, steps
     sampler = ClockSampler(torch.cuda.current_device()) if sample_clocks else None
     if sampler:
         sampler.__enter__()
     t0 = time.time()
-    n_rep = 0
-    secs = 0.0
-    # repeat the K-step region until ~0.4 s have been sampled by the clock monitor (short kernels)
     regions = []
+    # every region is exactly K steps between synchronisations; regions repeat until the clock
+    # monitor has seen ~0.5 s of load, and the median region is reported
     while True:
-        t = time_region(st.step, steps, device)
-        regions.append(t)
-        n_rep += 1
-        if not sample_clocks or time.time() - t0 > 0.5 or n_rep >= 200:
+        regions.append(time_region(run_steps, calls, device))
+        if not sample_clocks or time.time() - t0 > 0.5 or len(regions) >= 500:
             break
     if sampler:
         sampler.__exit__()
-    secs = regions[0]                                   # the reported region is the first, exactly K steps
-    # per-launch duration of the pass over the cache (the dominant kernel)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for i in range(steps):
-        st.step_phases(i, *evs[i])
-    torch.cuda.synchronize(device)
-    kernel_s = statistics.mean(a.elapsed_time(c) for a, c in evs) * 1e-3
-    # end to end with host buffers
-    for i in range(min(warmup, 3)):
+    secs = statistics.median(regions)
+    # per-launch duration of the pass over the cache (the dominant kernel): K back-to-back launches
+    kernel_regions = [time_region(run_split, calls, device) for _ in range(max(3, min(20, len(regions))))]
+    kernel_s = statistics.median(kernel_regions) / steps
+    # end to end with host buffers (eager: every step waits for its result)
+    for i in range(3):
         st.step_e2e(i)
     e2e_s = time_region(st.step_e2e, steps, device)
     status = int(st.status.item())
     return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status,
-            "clocks": sampler.summary() if sampler else None,
-            "median_region_s": statistics.median(regions), "regions": n_rep}
+            "clocks": sampler.summary() if sampler else None, "first_region_s": regions[0],
+            "min_region_s": min(regions), "regions": len(regions), "graph": bool(use_graph)}
 
 
 def cpu_baseline(w, seed, budget_s=20.0):
@@ -218,17 +233,20 @@ def cpu_baseline(w, seed, budget_s=20.0):
     inp = wl.make_inputs(min(w.b, 64), w.h, w.m_max, "mqa", seed=seed, device="cpu")
     lens = (wl.initial_lens(w)[: inp["b"]] + 1).astype(np.int32)
     qb, Kb, Vb = wl.bits(inp["q"]), wl.bits(inp["K"]), wl.bits(inp["V"])
-    t0 = time.perf_counter()
-    oracle.mqa_decode_step(qb[:1], Kb[:1], Vb[:1], lens[:1])
-    per_seq = max(time.perf_counter() - t0, 1e-6)       # one sequence, all heads in parallel
-    n = int(max(1, min(inp["b"], budget_s / per_seq)))
-    t0 = time.perf_counter()
-    oracle.mqa_decode_step(qb[:n], Kb[:n], Vb[:n], lens[:n])
-    dt = time.perf_counter() - t0
-    by = wl.algorithmic_bytes(int(lens[:n].sum()), n, w.h, 1)
-    return {"value": by / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{n} of {w.b} sequences x {w.h} heads x {w.m_max} rows, one multi-query step, fp64, "
-                      f"{dt:.2f} s", "seconds": dt}
+    threads = oracle.num_threads()
+    target_wall = budget_s / max(threads, 1)             # ~budget_s seconds of CPU work in total
+    n = inp["b"]
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        oracle.mqa_decode_step(qb[:n], Kb[:n], Vb[:n], lens[:n])
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= target_wall or reps >= 1000:
+            break
+    by = wl.algorithmic_bytes(int(lens[:n].sum()), n, w.h, 1) * reps
+    return {"value": by / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": f"{reps} multi-query steps over {n} of {w.b} sequences x {w.h} heads x {w.m_max} rows, fp64, "
+                      f"{dt:.2f} s wall on {threads} threads", "seconds": dt}
 
 
 def reference_arm(args, w):
@@ -279,7 +297,8 @@ def result_block(st, r, steps):
     return {"us_per_step": us, "gbs": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_step": st.bytes,
             "n_splits": st.n_splits, "chunk_rows": st.chunk_rows, "cache_sets": len(st.sets),
             "kernel_us": r["kernel_s"] * 1e6, "status": r["status"],
-            "median_us_per_step": r["median_region_s"] / steps * 1e6}
+            "first_region_us_per_step": r["first_region_s"] / steps * 1e6,
+            "min_us_per_step": r["min_region_s"] / steps * 1e6, "regions": r["regions"], "cuda_graph": r["graph"]}
 
 
 def main():
@@ -291,6 +310,7 @@ def main():
     ap.add_argument("--workload", default="long_context")
     ap.add_argument("--no-mha", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true", help="run every workload and write gpurun_out/sweep.json")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -321,7 +341,7 @@ def main():
     peak, peak_kind = measured_peak()
     seed = 1000 * rank                                  # every rank owns its own batch shard (weak scaling)
     st = StepState(mqa, "mqa", w, device, seed, min_rotate_bytes=8 * L2_BYTES)
-    r = run_variant(st, args.steps, args.warmup, device, sample_clocks=True)
+    r = run_variant(st, args.steps, args.warmup, device, sample_clocks=True, use_graph=not args.no_graph)
     blk = result_block(st, r, args.steps)
     secs_max = sharding.max_over_ranks(r["secs"], device)
     e2e_max = sharding.max_over_ranks(r["e2e_s"], device)
@@ -335,6 +355,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(w), "parallelism": f"batch shards x{world}, no collective",
                    "l2": f"rotating {len(st.sets)} cache sets of {st.cache_bytes >> 20} MiB (> L2) between steps",
+                   "launch": "K steps replayed as one CUDA graph" if r["graph"] else "K steps launched from the host",
                    "n_splits": st.n_splits, "chunk_rows": st.chunk_rows},
         "us_per_step": blk["us_per_step"], "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
         "mqa": blk,
@@ -359,7 +380,7 @@ def main():
     torch.cuda.empty_cache()
     if not args.no_mha:
         sth = StepState(mqa, "mha", w, device, seed, min_rotate_bytes=2 * L2_BYTES)
-        rh = run_variant(sth, max(3, min(args.steps, 20)), 3, device, sample_clocks=False)
+        rh = run_variant(sth, max(3, min(args.steps, 20)), 3, device, sample_clocks=False, use_graph=not args.no_graph)
         out["mha"] = result_block(sth, rh, max(3, min(args.steps, 20)))
         out["mha"]["roofline_frac"] = sth.bytes / rh["kernel_s"] / 1e9 / peak
         out["mqa_speedup_over_mha"] = out["mha"]["us_per_step"] / blk["us_per_step"]
@@ -390,7 +411,7 @@ def run_sweep(mqa, args, device, rank):
                 continue
             st = StepState(mqa, variant, w, device, 0, min_rotate_bytes=4 * L2_BYTES)
             steps = 20 if cache < 8 * 2 ** 30 else 5
-            r = run_variant(st, steps, 3, device, sample_clocks=False)
+            r = run_variant(st, steps, 3, device, sample_clocks=False, use_graph=not args.no_graph)
             blk = result_block(st, r, steps)
             blk.update({"workload": name, "variant": variant, "b": w.b, "h": w.h, "m": w.m_max,
                         "frac_of_measured_copy": blk["gbs"] / peak})

@@ -94,9 +94,9 @@ int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new,
  *          on return are unspecified.  Two calls that may overlap on the GPU need two
  *          workspaces.  May be NULL when mqa_workspace_bytes(...) is 0.
  *   status optional; LEN_CLAMPED, PIPELINE_TIMEOUT.
- * The memory axis is cut into splits that run in parallel, each keeping a running maximum
+ * The memory axis is cut into pieces that run in parallel, each keeping a running maximum
  * and sum (an exact re-association of the same softmax), and a second kernel combines the
- * splits; shared K/V rows are read from HBM once and used for all h heads.
+ * pieces; shared K/V rows are read from HBM once and used for all h heads.
  */
 int mqa_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                     void* workspace, size_t workspace_bytes, int32_t* status,
@@ -138,10 +138,12 @@ int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace
 size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v);
 
 /*
- * mqa_plan_splits -- how many splits of the memory axis the step will use for these sizes on
- * the current device (`multi_query` non-zero: mqa_decode_step, zero: mha_decode_step), and,
- * through *chunk_rows (optional), the rows per split.  Returns 0 for invalid arguments.
- * Informational: lets a caller see the launch plan; host-only.
+ * mqa_plan_splits -- the launch plan for these sizes on the current device (`multi_query`
+ * non-zero: mqa_decode_step, zero: mha_decode_step).  Returns the number of pieces one
+ * sequence's memory axis may be cut into (1 = no second pass), and through *chunk_rows
+ * (optional) the rows of one piece: the fixed split length, or, when the persistent kernel is
+ * used (every SM takes an equal share of the valid rows of the whole batch), the rows one SM
+ * streams when every cache is full.  Returns 0 for invalid arguments.  Informational; host-only.
  */
 int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int* chunk_rows);
 

@@ -36,13 +36,17 @@ int sm_count() {
     return n;
 }
 
-enum class Kernel { kSimt, kMma1, kMma2 };
+enum class Kernel { kSimt, kMma1, kMma2, kStream1, kStream2 };
 
 struct Plan {
-    int n_splits = 0;     // 0 = invalid
-    int chunk_rows = 0;   // rows of the memory axis per split (multiple of 64)
+    int n_splits = 0;     // 0 = invalid.  Fixed-split kernels: splits per sequence.  Persistent kernel: the
+                          // most CTAs that can hold pieces of one sequence.
+    int chunk_rows = 0;   // rows of the memory axis per split (persistent kernel: per CTA for full caches)
     size_t units = 0;     // b * h
+    int b = 0, h = 0;
+    int grid = 0;         // persistent kernel: number of CTAs
     Kernel kernel = Kernel::kSimt;
+    bool stream() const { return kernel == Kernel::kStream1 || kernel == Kernel::kStream2; }
 };
 
 bool dims_ok(int b, int h, int m_max) { return b > 0 && h > 0 && m_max > 0; }
@@ -53,6 +57,7 @@ bool dims_ok(int b, int h, int m_max) { return b > 0 && h > 0 && m_max > 0; }
 Plan plan_simt(int b, int h, int m_max) {
     Plan p;
     p.units = (size_t)b * h;
+    p.b = b; p.h = h;
     const long target_ctas = (long)sm_count() * 16;
     long want = (target_ctas + (long)p.units - 1) / (long)p.units;
     const long cap = m_max / 256 > 1 ? m_max / 256 : 1;
@@ -72,6 +77,7 @@ Plan plan_simt(int b, int h, int m_max) {
 Plan plan_mma(int b, int h, int m_max) {
     Plan p;
     p.units = (size_t)b * h;
+    p.b = b; p.h = h;
     p.kernel = h <= 16 ? Kernel::kMma1 : Kernel::kMma2;
     const int ctas_per_sm = h <= 16 ? MmaCfg<1>::kMinBlocks : MmaCfg<2>::kMinBlocks;
     const long slots = (long)sm_count() * ctas_per_sm;
@@ -97,16 +103,52 @@ Plan plan_mma(int b, int h, int m_max) {
     return p;
 }
 
+// Persistent tensor-core kernel: one CTA per SM, equal shares of the line of valid tiles.
+Plan plan_stream(int b, int h, int m_max) {
+    Plan p;
+    p.units = (size_t)b * h;
+    p.b = b; p.h = h;
+    p.kernel = h <= 16 ? Kernel::kStream1 : Kernel::kStream2;
+    p.grid = sm_count();
+    const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
+    p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
+    int parts = (p.grid + b - 1) / b + 1;
+    p.n_splits = parts < p.grid ? parts : p.grid;
+    return p;
+}
+
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // heads beyond two 16-row tensor-core tiles, or a row space too large for the 32-bit TMA
     // coordinates, go to the general CUDA-core kernel
-    if (multi_query && h <= 32 && (long long)b * m_max < 0x7fffffffLL) return plan_mma(b, h, m_max);
-    return plan_simt(b, h, m_max);
+    if (!(multi_query && h <= 32 && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
+    // enough tiles to give every SM a real share: the persistent kernel; otherwise fixed splits
+    const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
+    if (b <= kStreamMaxSeqs && tiles >= 8LL * sm_count()) return plan_stream(b, h, m_max);
+    return plan_mma(b, h, m_max);
 }
 
 size_t plan_workspace_bytes(const Plan& p) {
+    if (p.stream()) {
+        const int slots = p.grid + p.b;
+        return stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) + stream_acc_bytes(slots, p.h);
+    }
     if (p.n_splits <= 1) return 0;
     return partial_ml_bytes(p.units, p.n_splits) + partial_acc_bytes(p.units, p.n_splits);
+}
+
+struct StreamWorkspace {
+    int2* span;
+    float2* ml;
+    float* acc;
+};
+StreamWorkspace stream_workspace(const Plan& p, const void* workspace) {
+    char* base = static_cast<char*>(const_cast<void*>(workspace));
+    const int slots = p.grid + p.b;
+    StreamWorkspace w;
+    w.span = reinterpret_cast<int2*>(base);
+    w.ml = reinterpret_cast<float2*>(base + stream_span_bytes(p.b));
+    w.acc = reinterpret_cast<float*>(base + stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h));
+    return w;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -191,6 +233,31 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
+std::atomic<int> g_stream_opt_in[kMaxDevices][2];
+
+template <int M_TILES>
+int launch_stream(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                  void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
+    using Cfg = StreamCfg<M_TILES>;
+    auto kernel = mqa_decode_stream_mma_kernel<M_TILES>;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!g_stream_opt_in[dev][M_TILES - 1].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+        g_stream_opt_in[dev][M_TILES - 1].store(1, std::memory_order_release);
+    }
+    alignas(64) CUtensorMap map_k, map_v;
+    if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
+        return MQA_ERR_CUDA;
+    const StreamWorkspace w = stream_workspace(p, workspace);
+    kernel<<<(unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(
+        map_k, map_v, static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
+    return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
+}
+
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
 
 int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
@@ -202,6 +269,10 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
+    if (p.kernel == Kernel::kStream1)
+        return launch_stream<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+    if (p.kernel == Kernel::kStream2)
+        return launch_stream<2>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     float2* part_ml = reinterpret_cast<float2*>(workspace);
     float* part_acc = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits))
@@ -225,6 +296,11 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     if (p.units > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     int rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
+    if (p.stream()) {
+        const StreamWorkspace w = stream_workspace(p, workspace);
+        stream_combine_kernel<<<(unsigned)((size_t)b * h), kHeadDim, 0, stream>>>(w.span, w.ml, w.acc, o, b, h);
+        return launch_status();
+    }
     if (p.n_splits <= 1) return MQA_OK;
     const float2* part_ml = reinterpret_cast<const float2*>(workspace);
     const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +

@@ -1,18 +1,26 @@
-// Split-m multi-query decode kernel (Section 3: logits = einsum(bhk,bmk->bhm), softmax over m,
-// o = einsum(bhm,bmv->bhv)) for sm_100a.
+// Multi-query decode kernels on the tensor cores (Section 3: logits = einsum(bhk,bmk->bhm),
+// softmax over m, o = einsum(bhm,bmv->bhv)) for sm_100a.
 //
-// One CTA owns one split of one sequence's memory axis.  A producer warp streams that split's
-// K and V rows HBM -> shared memory with TMA (cp.async.bulk.tensor, 128-byte swizzle) through
-// a ring of stages guarded by full/empty mbarriers; every K/V byte is fetched from HBM once
-// and is then used for ALL h heads, which is the whole point of the multi-query layout
-// (h flops per byte instead of 1).  At h flops per byte the CUDA cores cannot keep up with
-// HBM, so the two contractions run on the tensor cores with the heads as the M rows:
+// A producer warp streams K and V rows HBM -> shared memory with TMA (cp.async.bulk.tensor,
+// 128-byte swizzle) through a ring of stages guarded by full/empty mbarriers; every K/V byte is
+// fetched from HBM once and is then used for ALL h heads, which is the whole point of the
+// multi-query layout (h flops per byte instead of 1).  At h flops per byte the CUDA cores
+// cannot keep up with HBM, so the two contractions run on the tensor cores with the heads as
+// the M rows:
 //     S[h x rows]   = Q[h x k] * K_tile^T          (bf16 mma, fp32 accumulate)
 //     O[h x v]     += P[h x rows] * V_tile         (P = exp2(S - max), split into bf16 hi + lo
 //                                                  parts so that the weights keep ~16 bits)
 // Each consumer warp takes whole 32-row tiles round-robin and keeps its own online-softmax
-// state (running max, running sum, fp32 accumulators) in registers; warps are merged through
-// shared memory at the end and the CTA writes its partial (or the final o for a single split).
+// state (running max, running sum, fp32 accumulators) in registers.
+//
+// Two kernels share that inner loop:
+//   * mqa_decode_split_mma_kernel   -- one CTA per (sequence, fixed-size split); used when the
+//                                      whole problem is small (short caches, few sequences);
+//   * mqa_decode_stream_mma_kernel  -- a persistent grid of one CTA per SM; the 32-row tiles of
+//                                      all sequences (valid rows only, from lens) form one
+//                                      line that is cut into equal contiguous shares, so every
+//                                      SM streams the same number of bytes whatever the batch
+//                                      size, context length or raggedness.
 //
 // Rows at or beyond lens[b] are never used: their logits are replaced by -inf by index and
 // their V fragments are zeroed by index (a NaN times a zero weight would still be a NaN).
@@ -29,21 +37,37 @@ constexpr int kBoxCols = 64;                           // 64 bf16 = 128 bytes = 
 constexpr int kBoxBytes = kTileRows * kBoxCols * 2;    // 4 KiB
 constexpr int kStageBytes = 4 * kBoxBytes;             // K lo, K hi, V lo, V hi = 16 KiB
 constexpr int kRowWarps = 4;                           // consumer warps that share the tiles
-constexpr long long kWaitLimitCycles = 2000000000ll;    // every mbarrier wait gives up after ~1 s of SM clock ...
+constexpr long long kWaitLimitCycles = 2000000000ll;   // every mbarrier wait gives up after ~1 s of SM clock ...
 constexpr uint32_t kWaitRounds = 1u << 24;             // ... or after this many polling rounds
+constexpr int kStreamMaxSeqs = 1024;                   // sequences the persistent kernel can index in shared memory
 
+// Ring depth must be a multiple of kRowWarps: tile i lives in stage i % kStages and belongs to
+// row-warp i % kRowWarps, so with this rule every use of a stage is waited on by the same warp.
+// A parity wait can only tell the current phase from the one before it; a warp that skipped a
+// use of a stage could mistake an old phase for the one it needs.
 template <int M_TILES>
-struct MmaCfg {
+struct MmaCfg {                                        // fixed-split kernel
     static constexpr int kConsumerWarps = M_TILES * kRowWarps;
     static constexpr int kThreads = (kConsumerWarps + 1) * 32;
-    // Ring depth.  It must be a multiple of kRowWarps: tile i lives in stage i % kStages and belongs
-    // to row-warp i % kRowWarps, so with this rule every use of a stage is waited on by the same warp.
-    // A parity wait can only tell the current phase from the one before it; a warp that skipped a use
-    // of a stage could mistake an old phase for the one it needs.
     static constexpr int kStages = (M_TILES == 1) ? 4 : 12;
     static_assert(kStages % kRowWarps == 0, "a stage must always be consumed by the same warp");
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
     static constexpr int kMinBlocks = (M_TILES == 1) ? 2 : 1;
+};
+
+template <int M_TILES>
+struct StreamCfg {                                     // persistent kernel, one CTA per SM
+    static constexpr int kConsumerWarps = M_TILES * kRowWarps;
+    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    static constexpr int kStages = 12;
+    static_assert(kStages % kRowWarps == 0, "a stage must always be consumed by the same warp");
+    static constexpr int kStateFloats = 16 * 4 + 4;    // acc + (m, l) x 2 rows, per thread
+    static constexpr int kMergeBytes = M_TILES * kStateFloats * 32 * 4;
+    static constexpr int kPrefixBytes = (kStreamMaxSeqs + 1) * 4 + 12;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kMergeBytes + kPrefixBytes + 256 /* barriers */ +
+                                      1024 /* alignment slack */;
+    static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
+    static constexpr int kCtasPerSm = 1;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -106,13 +130,186 @@ __device__ __forceinline__ uint32_t pack_bf16(float x_lo, float x_hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x_hi), "f"(x_lo));
     return r;
 }
-
-// Byte offset of (row, 16-byte chunk 0..15 along the 128 columns) inside one K or V tile as
-// TMA lays it out: two 64-column boxes, each 128-byte-swizzled (chunk index XOR row mod 8).
-__device__ __forceinline__ uint32_t tile_offset(int row, int chunk) {
-    return (uint32_t)((chunk >> 3) * kBoxBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// ---- the consumer warp's state and inner loop ------------------------------------------------
+// Layout of a K or V tile in shared memory as TMA writes it: two 64-column boxes of 32 rows x
+// 128 bytes; inside a box the 16-byte chunk index (0..7) is XORed with (row mod 8).
+// An ldmatrix lane addresses row (8*j + lane%8) of its matrix, so (row mod 8) == lane%8 for every
+// access and the swizzle folds into four per-lane offsets (one per chunk pair).
+struct LaneOffsets {
+    uint32_t k[4];   // K: [(lane/16)*8 + lane%8] row, chunk pair c -> byte offset (without box/tile-row parts)
+    uint32_t v[4];   // V: [((lane/8)&1)*8 + lane%8] row, chunk pair c
+    __device__ __forceinline__ void init(int lane) {
+        const int lm = lane >> 3, lr = lane & 7;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            k[c] = (uint32_t)((((lm >> 1) * 8 + lr) * 128) + ((((c * 2) | (lm & 1)) ^ lr) << 4));
+            v[c] = (uint32_t)((((lm & 1) * 8 + lr) * 128) + ((((c * 2) | (lm >> 1)) ^ lr) << 4));
+        }
+    }
+};
+
+struct WarpState {
+    float acc[16][4];     // O fragments: [8-column tile][c0 c1 (head g) | c2 c3 (head g+8)]
+    float m[2];           // running maxima (log2 units) of heads g and g+8
+    float l[2];           // this thread's share of the running sums
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+        m[0] = m[1] = -INFINITY;
+        l[0] = l[1] = 0.f;
+    }
+};
+
+// Q fragments (A operand, 16 heads x 128 columns) of head tile mt of sequence seq, straight from
+// global memory; heads >= h are zero.
+__device__ __forceinline__ void load_q_fragments(uint32_t (&qa)[8][4], const uint32_t* __restrict__ q, size_t seq,
+                                                 int h, int mt, int lane) {
+    const int g = lane >> 2, t4 = lane & 3;
+    const int head0 = mt * 16 + g, head1 = head0 + 8;
+    const uint32_t* q0 = q + (seq * h + head0) * (kHeadDim / 2);
+    const uint32_t* q1 = q + (seq * h + head1) * (kHeadDim / 2);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        const int w0 = ks * 8 + t4;                    // 32-bit word: columns ks*16 + t4*2 + {0,1}
+        qa[ks][0] = head0 < h ? __ldg(q0 + w0) : 0u;
+        qa[ks][1] = head1 < h ? __ldg(q1 + w0) : 0u;
+        qa[ks][2] = head0 < h ? __ldg(q0 + w0 + 4) : 0u;   // columns + 8
+        qa[ks][3] = head1 < h ? __ldg(q1 + w0 + 4) : 0u;
+    }
+}
+
+// One 32-row tile (cache rows row0 .. row0+31 of the sequence, of which rows < r1 are valid) for
+// 16 heads: S = Q K^T, online softmax update, O += P V.
+__device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)[8][4], const LaneOffsets& off,
+                                             uint32_t k_s, uint32_t v_s, int row0, int r1, int lane) {
+    const int t4 = lane & 3;
+    const bool ragged = row0 + kTileRows > r1;
+
+    // S = Q K^T: 4 n-tiles of 8 rows, 8 k-steps of 16 columns
+    float sc[4][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t a = k_s + off.k[ks & 3] + (ks >> 2) * kBoxBytes;
+#pragma unroll
+        for (int np = 0; np < 2; ++np) {               // n-tile pairs (0,1) and (2,3): 16 rows = 2 KiB apart
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(a + np * 2048, b0, b1, b2, b3);
+            mma_bf16(sc[np * 2], qa[ks], b0, b1);
+            mma_bf16(sc[np * 2 + 1], qa[ks], b2, b3);
+        }
+    }
+    // scale to log2 units, mask by index, row maxima
+    float top[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float x = sc[nt][j] * kLog2e;
+            sc[nt][j] = (!ragged || row0 + nt * 8 + t4 * 2 + (j & 1) < r1) ? x : -INFINITY;   // select, never multiply
+            top[j >> 1] = fmaxf(top[j >> 1], sc[nt][j]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        top[r] = fmaxf(top[r], __shfl_xor_sync(0xffffffffu, top[r], 1));
+        top[r] = fmaxf(top[r], __shfl_xor_sync(0xffffffffu, top[r], 2));
+    }
+    // a new maximum rescales what has been accumulated; most tiles do not bring one
+    if (__any_sync(0xffffffffu, top[0] > st.m[0] || top[1] > st.m[1])) {
+        float rescale[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const float m_new = fmaxf(st.m[r], top[r]);     // the tile's first row is valid: finite
+            rescale[r] = fast_exp2(st.m[r] - m_new);        // 0 on the first tile, 1 if unchanged
+            st.m[r] = m_new;
+            st.l[r] *= rescale[r];
+        }
+#pragma unroll
+        for (int vt = 0; vt < 16; ++vt) {
+            st.acc[vt][0] *= rescale[0]; st.acc[vt][1] *= rescale[0];
+            st.acc[vt][2] *= rescale[1]; st.acc[vt][3] *= rescale[1];
+        }
+    }
+    // P = exp2(S - max) as bf16 hi + lo A-fragments for the two 16-row k-steps
+    uint32_t p_hi[2][4], p_lo[2][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        float p[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            p[j] = fast_exp2(sc[nt][j] - st.m[j >> 1]);     // exactly 1 at the maximum, 0 when masked
+            st.l[j >> 1] += p[j];
+        }
+        const uint32_t hi01 = pack_bf16(p[0], p[1]), hi23 = pack_bf16(p[2], p[3]);
+        const uint32_t lo01 = pack_bf16(p[0] - bf16_lo(hi01), p[1] - bf16_hi(hi01));
+        const uint32_t lo23 = pack_bf16(p[2] - bf16_lo(hi23), p[3] - bf16_hi(hi23));
+        const int kk = nt >> 1, hf = (nt & 1) * 2;          // A regs: {g,k}, {g+8,k}, {g,k+8}, {g+8,k+8}
+        p_hi[kk][hf] = hi01; p_hi[kk][hf + 1] = hi23;
+        p_lo[kk][hf] = lo01; p_lo[kk][hf + 1] = lo23;
+    }
+    // O += P V : 2 k-steps of 16 rows x 16 n-tiles of 8 columns
+#pragma unroll
+    for (int kk = 0; kk < 2; ++kk) {
+        uint32_t keep_lo = 0xffffffffu, keep_hi = 0xffffffffu;   // per-register row masks (ragged tile)
+        if (ragged) {
+            const int ra = row0 + kk * 16 + t4 * 2;              // rows held by b0/b2: ra, ra+1; b1/b3: +8
+            keep_lo = (ra < r1 ? 0x0000ffffu : 0u) | (ra + 1 < r1 ? 0xffff0000u : 0u);
+            keep_hi = (ra + 8 < r1 ? 0x0000ffffu : 0u) | (ra + 9 < r1 ? 0xffff0000u : 0u);
+        }
+#pragma unroll
+        for (int vp = 0; vp < 8; ++vp) {                         // pairs of 8-column n-tiles
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(v_s + off.v[vp & 3] + (vp >> 2) * kBoxBytes + kk * 2048, b0, b1, b2, b3);
+            if (ragged) { b0 &= keep_lo; b1 &= keep_hi; b2 &= keep_lo; b3 &= keep_hi; }
+            mma_bf16(st.acc[vp * 2], p_hi[kk], b0, b1);
+            mma_bf16(st.acc[vp * 2 + 1], p_hi[kk], b2, b3);
+            mma_bf16(st.acc[vp * 2], p_lo[kk], b0, b1);
+            mma_bf16(st.acc[vp * 2 + 1], p_lo[kk], b2, b3);
+        }
+    }
+}
+
+// Merge `other` (the same heads over other rows) into `st`.  Either side may be empty (m = -inf).
+__device__ __forceinline__ void merge_state(WarpState& st, const float* __restrict__ other, int lane) {
+    // `other` is thread-private storage: float index r * 32 + lane, r = 0..63 acc, 64..65 m, 66..67 l
+    float wa[2], wb[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const float mb = other[(64 + r) * 32 + lane];
+        const float lb = other[(66 + r) * 32 + lane];
+        const float m_new = fmaxf(st.m[r], mb);
+        wa[r] = st.m[r] == -INFINITY ? 0.f : fast_exp2(st.m[r] - m_new);
+        wb[r] = mb == -INFINITY ? 0.f : fast_exp2(mb - m_new);
+        st.m[r] = m_new;
+        st.l[r] = st.l[r] * wa[r] + lb * wb[r];
+    }
+#pragma unroll
+    for (int vt = 0; vt < 16; ++vt) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            st.acc[vt][j] = st.acc[vt][j] * wa[j >> 1] + other[(vt * 4 + j) * 32 + lane] * wb[j >> 1];
+    }
+}
+
+__device__ __forceinline__ void store_state(const WarpState& st, float* __restrict__ dst, int lane) {
+#pragma unroll
+    for (int vt = 0; vt < 16; ++vt) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[(vt * 4 + j) * 32 + lane] = st.acc[vt][j];
+    }
+    dst[64 * 32 + lane] = st.m[0]; dst[65 * 32 + lane] = st.m[1];
+    dst[66 * 32 + lane] = st.l[0]; dst[67 * 32 + lane] = st.l[1];
+}
+
+// =============================================================================================
+// Fixed-split kernel: one CTA per (sequence, split of chunk_rows rows).
+// =============================================================================================
 template <int M_TILES>
 __global__ void __launch_bounds__(MmaCfg<M_TILES>::kThreads, MmaCfg<M_TILES>::kMinBlocks)
 mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -155,6 +352,10 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     }
     __syncthreads();
 
+    const int mt = warp % M_TILES;                         // which 16-head tile this warp serves
+    const int rw = warp / M_TILES;                         // which tiles (round-robin over kRowWarps)
+    WarpState st;
+
     if (warp == Cfg::kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
         if (lane == 0) {
@@ -176,134 +377,20 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
-    }
-
-    // Per-thread state of a consumer warp (declared for all warps; the producer leaves it unused).
-    const int cw = warp;                                   // consumer warp index
-    const int mt = cw % M_TILES;                           // which 16-head tile this warp serves
-    const int rw = cw / M_TILES;                           // which tiles (round-robin over kRowWarps)
-    const int g = lane >> 2, t4 = lane & 3;
-    float acc[16][4];
-    float m_run[2] = {-INFINITY, -INFINITY};               // heads mt*16+g and mt*16+g+8
-    float l_run[2] = {0.f, 0.f};                           // this thread's share of the row sums
-
-    if (warp < Cfg::kConsumerWarps) {
+    } else {
         // --------------------------------------------------------------- consumer warps
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
-
-        // Q fragments (A operand, 16 heads x 128), straight from global memory; heads >= h are zero.
+        st.reset();
         uint32_t qa[8][4];
-        {
-            const int head0 = mt * 16 + g, head1 = head0 + 8;
-            const uint32_t* q0 = q + ((size_t)seq * h + head0) * (kHeadDim / 2);
-            const uint32_t* q1 = q + ((size_t)seq * h + head1) * (kHeadDim / 2);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const int w0 = ks * 8 + t4;                // 32-bit word index: columns ks*16 + t4*2 + {0,1}
-                qa[ks][0] = head0 < h ? q0[w0] : 0u;
-                qa[ks][1] = head1 < h ? q1[w0] : 0u;
-                qa[ks][2] = head0 < h ? q0[w0 + 4] : 0u;   // columns + 8
-                qa[ks][3] = head1 < h ? q1[w0 + 4] : 0u;
-            }
-        }
-        // ldmatrix lane roles (matrix = lane / 8, row within the matrix = lane % 8)
-        const int lm = lane >> 3, lr = lane & 7;
-
+        load_q_fragments(qa, q, (size_t)seq, h, mt, lane);
+        LaneOffsets off;
+        off.init(lane);
         bool ok = true;
         for (int i = rw; i < n_tiles; i += kRowWarps) {
             const int s = i % kStages;
             ok = mbar_wait(full_s + s * 8, (i / kStages) & 1);
             if (!ok) break;
             const uint32_t k_s = stages_s + s * kStageBytes;
-            const uint32_t v_s = k_s + 2 * kBoxBytes;
-            const int row0 = r0 + i * kTileRows;           // first cache row of this tile
-            const bool ragged = row0 + kTileRows > r1;
-
-            // S = Q K^T for 32 rows: 4 n-tiles of 8 rows
-            float sc[4][4];
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-                for (int np = 0; np < 2; ++np) {           // n-tile pairs (0,1) and (2,3)
-                    uint32_t b0, b1, b2, b3;
-                    const int row = (np * 2 + (lm >> 1)) * 8 + lr;
-                    ldmatrix_x4(k_s + tile_offset(row, ks * 2 + (lm & 1)), b0, b1, b2, b3);
-                    mma_bf16(sc[np * 2], qa[ks], b0, b1);
-                    mma_bf16(sc[np * 2 + 1], qa[ks], b2, b3);
-                }
-            }
-            // scale to log2 units, mask by index, row maxima
-            float top[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int row = row0 + nt * 8 + t4 * 2 + (j & 1);
-                    const float x = sc[nt][j] * kLog2e;
-                    sc[nt][j] = (!ragged || row < r1) ? x : -INFINITY;      // select, never multiply
-                    top[j >> 1] = fmaxf(top[j >> 1], sc[nt][j]);
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                top[r] = fmaxf(top[r], __shfl_xor_sync(0xffffffffu, top[r], 1));
-                top[r] = fmaxf(top[r], __shfl_xor_sync(0xffffffffu, top[r], 2));
-            }
-            float rescale[2];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const float m_new = fmaxf(m_run[r], top[r]);    // the tile's first row is valid: finite
-                rescale[r] = fast_exp2(m_run[r] - m_new);       // 0 on this warp's first tile
-                m_run[r] = m_new;
-                l_run[r] *= rescale[r];
-            }
-#pragma unroll
-            for (int vt = 0; vt < 16; ++vt) {
-                acc[vt][0] *= rescale[0]; acc[vt][1] *= rescale[0];
-                acc[vt][2] *= rescale[1]; acc[vt][3] *= rescale[1];
-            }
-            // P = exp2(S - max) as bf16 hi + lo A-fragments for the two 16-row k-steps
-            uint32_t p_hi[2][4], p_lo[2][4];
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                float p[4], ph[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    p[j] = fast_exp2(sc[nt][j] - m_run[j >> 1]);   // exactly 1 at the maximum, 0 when masked
-                    l_run[j >> 1] += p[j];
-                }
-                const uint32_t hi01 = pack_bf16(p[0], p[1]), hi23 = pack_bf16(p[2], p[3]);
-                ph[0] = bf16_lo(hi01); ph[1] = bf16_hi(hi01); ph[2] = bf16_lo(hi23); ph[3] = bf16_hi(hi23);
-                const uint32_t lo01 = pack_bf16(p[0] - ph[0], p[1] - ph[1]);
-                const uint32_t lo23 = pack_bf16(p[2] - ph[2], p[3] - ph[3]);
-                const int kk = nt >> 1, hf = (nt & 1) * 2;          // A regs: {g,k}, {g+8,k}, {g,k+8}, {g+8,k+8}
-                p_hi[kk][hf] = hi01; p_hi[kk][hf + 1] = hi23;
-                p_lo[kk][hf] = lo01; p_lo[kk][hf + 1] = lo23;
-            }
-            // O += P V : 2 k-steps of 16 rows x 16 n-tiles of 8 columns
-#pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {
-                uint32_t keep_lo = 0xffffffffu, keep_hi = 0xffffffffu;   // per-register row masks (ragged tile)
-                if (ragged) {
-                    const int ra = row0 + kk * 16 + t4 * 2;              // rows held by b0/b1: ra, ra+1; b2/b3: +8
-                    keep_lo = (ra < r1 ? 0x0000ffffu : 0u) | (ra + 1 < r1 ? 0xffff0000u : 0u);
-                    keep_hi = (ra + 8 < r1 ? 0x0000ffffu : 0u) | (ra + 9 < r1 ? 0xffff0000u : 0u);
-                }
-#pragma unroll
-                for (int vp = 0; vp < 8; ++vp) {                         // pairs of 8-column n-tiles
-                    uint32_t b0, b1, b2, b3;
-                    const int row = kk * 16 + (lm & 1) * 8 + lr;
-                    ldmatrix_x4_trans(v_s + tile_offset(row, vp * 2 + (lm >> 1)), b0, b1, b2, b3);
-                    if (ragged) { b0 &= keep_lo; b1 &= keep_hi; b2 &= keep_lo; b3 &= keep_hi; }
-                    mma_bf16(acc[vp * 2], p_hi[kk], b0, b1);
-                    mma_bf16(acc[vp * 2], p_lo[kk], b0, b1);
-                    mma_bf16(acc[vp * 2 + 1], p_hi[kk], b2, b3);
-                    mma_bf16(acc[vp * 2 + 1], p_lo[kk], b2, b3);
-                }
-            }
+            consume_tile(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_s + s * 8);                 // this warp is done with the stage
         }
@@ -327,23 +414,24 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     }
 
     // ---- merge the kRowWarps warps of each head tile through shared memory (stages are free now)
+    const int g = lane >> 2, t4 = lane & 3;
     float* sm_acc = reinterpret_cast<float*>(stages);                   // [consumer warp][16][128]
     float2* sm_ml = reinterpret_cast<float2*>(stages + Cfg::kConsumerWarps * 16 * kHeadDim * 4);  // [cw][16]
     if (warp < Cfg::kConsumerWarps) {
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+            st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 1);
+            st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 2);
         }
-        float* mine = sm_acc + (size_t)cw * 16 * kHeadDim;
+        float* mine = sm_acc + (size_t)warp * 16 * kHeadDim;
 #pragma unroll
         for (int vt = 0; vt < 16; ++vt) {
-            *reinterpret_cast<float2*>(mine + g * kHeadDim + vt * 8 + t4 * 2) = make_float2(acc[vt][0], acc[vt][1]);
-            *reinterpret_cast<float2*>(mine + (g + 8) * kHeadDim + vt * 8 + t4 * 2) = make_float2(acc[vt][2], acc[vt][3]);
+            *reinterpret_cast<float2*>(mine + g * kHeadDim + vt * 8 + t4 * 2) = make_float2(st.acc[vt][0], st.acc[vt][1]);
+            *reinterpret_cast<float2*>(mine + (g + 8) * kHeadDim + vt * 8 + t4 * 2) = make_float2(st.acc[vt][2], st.acc[vt][3]);
         }
         if (t4 == 0) {
-            sm_ml[cw * 16 + g] = make_float2(m_run[0], l_run[0]);
-            sm_ml[cw * 16 + g + 8] = make_float2(m_run[1], l_run[1]);
+            sm_ml[warp * 16 + g] = make_float2(st.m[0], st.l[0]);
+            sm_ml[warp * 16 + g + 8] = make_float2(st.m[1], st.l[1]);
         }
     }
     __syncthreads();
@@ -374,6 +462,255 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
             if (c == 0) part_ml[slot] = make_float2(top, den);
         }
     }
+}
+
+// =============================================================================================
+// Persistent kernel: the valid 32-row tiles of all sequences, in sequence order, form one line
+// of T tiles; CTA c of G takes tiles [c*T/G, (c+1)*T/G).  A CTA's share is a run of segments,
+// each a contiguous run of tiles of one sequence.  A segment that covers its whole sequence
+// writes the final o; any other segment writes a partial into slot (c + sequence) -- along the
+// line every step moves to the next CTA, the next sequence, or both, so that sum never repeats
+// -- and the second-pass kernel merges the slots of each sequence that was cut.
+// =============================================================================================
+struct StreamWork {
+    long long total;      // T
+    long long begin, end; // this CTA's tiles
+};
+
+// cta that owns global tile t when T tiles are cut into G shares [c*T/G, (c+1)*T/G)
+__host__ __device__ inline int stream_owner(long long t, long long T, int G) {
+    return (int)(((t + 1) * G + T - 1) / T - 1);
+}
+
+// Workspace layout of the persistent kernel
+__host__ __device__ inline size_t stream_span_bytes(int b) { return (((size_t)(b + 1) * sizeof(int2)) + 255) & ~(size_t)255; }
+__host__ __device__ inline size_t stream_ml_bytes(int slots, int h) {
+    return (((size_t)slots * h * sizeof(float2)) + 255) & ~(size_t)255;
+}
+__host__ __device__ inline size_t stream_acc_bytes(int slots, int h) { return (size_t)slots * h * kHeadDim * sizeof(float); }
+
+template <int M_TILES>
+__global__ void __launch_bounds__(StreamCfg<M_TILES>::kThreads, 1)
+mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
+                             float* __restrict__ o, int2* __restrict__ seq_span, float2* __restrict__ part_ml,
+                             float* __restrict__ part_acc, int32_t* __restrict__ status, int b, int h, int m_max) {
+    using Cfg = StreamCfg<M_TILES>;
+    constexpr int kStages = Cfg::kStages;
+    constexpr int kConsumerThreads = Cfg::kConsumerWarps * 32;
+    const int cta = blockIdx.x, G = gridDim.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* stages = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    float* merge_buf = reinterpret_cast<float*>(stages + kStages * kStageBytes);            // [M_TILES][68][32]
+    int* prefix = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(merge_buf) + Cfg::kMergeBytes);  // [b + 1]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + Cfg::kPrefixBytes / 8 * 8);
+    const uint32_t stages_s = smem_addr(stages);
+    const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
+    __shared__ int timed_out, issued;
+
+    // ---- tiles per sequence and their running sum (every CTA computes the same table) -----------
+    for (int s = threadIdx.x; s < b; s += Cfg::kThreads) {
+        const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
+        prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
+        if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
+            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
+        }
+    }
+    if (threadIdx.x == 0) {
+        prefix[0] = 0;
+        timed_out = 0;
+        issued = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_s + s * 8, 1);
+            mbar_init(empty_s + s * 8, M_TILES);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {                                       // inclusive scan of prefix[1..b] by one warp
+        const int per = (b + 31) / 32;
+        const int lo = 1 + lane * per, hi = min(b, lo + per - 1);
+        int sum = 0;
+        for (int s = lo; s <= hi; ++s) sum += prefix[s];
+        int incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        int run = incl - sum;
+        for (int s = lo; s <= hi; ++s) { run += prefix[s]; prefix[s] = run; }
+    }
+    __syncthreads();
+    const long long T = prefix[b];
+    const long long t_begin = (long long)cta * T / G, t_end = (long long)(cta + 1) * T / G;
+
+    // which CTAs hold pieces of each sequence (read by the second pass); spread over the CTAs
+    for (int s = cta + (int)threadIdx.x * G; s < b; s += G * Cfg::kThreads) {
+        const int t0 = prefix[s], t1 = prefix[s + 1];
+        seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
+    }
+    if (cta == 0 && threadIdx.x == 0) seq_span[b] = make_int2((int)T, G);
+    if (t_begin >= t_end) return;                          // uniform: this CTA has no tiles
+
+    // first sequence of this CTA's share: the s with prefix[s] <= t_begin < prefix[s+1]
+    int s_first;
+    {
+        int lo = 0, hi = b - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (prefix[mid] <= t_begin) lo = mid; else hi = mid - 1;
+        }
+        s_first = lo;
+        while (prefix[s_first + 1] <= t_begin) ++s_first;  // skip sequences without tiles
+    }
+
+    const int mt = warp % M_TILES;
+    const int rw = warp / M_TILES;
+
+    if (warp == Cfg::kConsumerWarps) {
+        // ------------------------------------------------------------------ producer warp
+        if (lane == 0) {
+            bool ok = true;
+            int s = s_first;
+            int j = 0;                                     // tiles issued by this CTA so far
+            for (long long t = t_begin; t < t_end && ok; ++t, ++j) {
+                while (prefix[s + 1] <= t) ++s;
+                const int stg = j % kStages;
+                if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
+                if (!ok) break;
+                const uint32_t bar = full_s + stg * 8;
+                const uint32_t dst = stages_s + stg * kStageBytes;
+                mbar_expect_tx(bar, kStageBytes);
+                const int y = s * m_max + (int)(t - prefix[s]) * kTileRows;
+                tma_load_2d(dst, &map_k, 0, y, bar);
+                tma_load_2d(dst + kBoxBytes, &map_k, kBoxCols, y, bar);
+                tma_load_2d(dst + 2 * kBoxBytes, &map_v, 0, y, bar);
+                tma_load_2d(dst + 3 * kBoxBytes, &map_v, kBoxCols, y, bar);
+                issued = j + 1;
+            }
+            if (!ok) atomicExch(&timed_out, 1);
+        }
+    } else {
+        // --------------------------------------------------------------- consumer warps
+        WarpState st;
+        LaneOffsets off;
+        off.init(lane);
+        const int g = lane >> 2, t4 = lane & 3;
+        float* my_buf = merge_buf + mt * Cfg::kStateFloats * 32;
+        bool ok = true;
+        int j = 0;                                         // index of the segment's first tile in this CTA's stream
+        int s = s_first;
+        for (long long t = t_begin; t < t_end;) {
+            while (prefix[s + 1] <= t) ++s;
+            const long long seg_end = min((long long)prefix[s + 1], t_end);
+            const int n_seg = (int)(seg_end - t);
+            const int first_row = (int)(t - prefix[s]) * kTileRows;
+            const int L = min(max(__ldg(lens + s), 0), m_max);
+            const bool whole = (t == prefix[s]) && (seg_end == prefix[s + 1]);
+
+            st.reset();
+            uint32_t qa[8][4];
+            load_q_fragments(qa, q, (size_t)s, h, mt, lane);
+            // this warp's tiles of the segment: stream positions jj = j .. j+n_seg-1 with jj % kRowWarps == rw
+            for (int jj = j + ((rw - j) & (kRowWarps - 1)); jj < j + n_seg; jj += kRowWarps) {
+                const int stg = jj % kStages;
+                if (ok) ok = mbar_wait(full_s + stg * 8, (jj / kStages) & 1);
+                if (ok) {
+                    const uint32_t k_s = stages_s + stg * kStageBytes;
+                    consume_tile(st, qa, off, k_s, k_s + 2 * kBoxBytes, first_row + (jj - j) * kTileRows, L, lane);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_s + stg * 8);   // released even after a failed wait: nobody may hang
+            }
+            // fold the row-warps of this head tile into row-warp 0: 3 -> 2 -> 1 -> 0
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 1);
+                st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 2);
+            }
+            named_barrier(1, kConsumerThreads);            // the previous segment's last reader is done with the buffer
+#pragma unroll 1
+            for (int r = kRowWarps - 1; r >= 1; --r) {
+                if (rw == r) store_state(st, my_buf, lane);
+                named_barrier(1, kConsumerThreads);
+                if (rw == r - 1) merge_state(st, my_buf, lane);
+            }
+            if (rw == 0) {
+                const int head0 = mt * 16 + g, head1 = head0 + 8;
+                if (whole) {
+                    const float inv0 = 1.f / st.l[0], inv1 = 1.f / st.l[1];
+                    float* o0 = o + ((size_t)s * h + head0) * kHeadDim + t4 * 2;
+                    float* o1 = o + ((size_t)s * h + head1) * kHeadDim + t4 * 2;
+#pragma unroll
+                    for (int vt = 0; vt < 16; ++vt) {
+                        if (head0 < h) *reinterpret_cast<float2*>(o0 + vt * 8) = make_float2(st.acc[vt][0] * inv0, st.acc[vt][1] * inv0);
+                        if (head1 < h) *reinterpret_cast<float2*>(o1 + vt * 8) = make_float2(st.acc[vt][2] * inv1, st.acc[vt][3] * inv1);
+                    }
+                } else {
+                    const size_t slot = (size_t)cta + s;
+                    float* a0 = part_acc + (slot * h + head0) * kHeadDim + t4 * 2;
+                    float* a1 = part_acc + (slot * h + head1) * kHeadDim + t4 * 2;
+#pragma unroll
+                    for (int vt = 0; vt < 16; ++vt) {
+                        if (head0 < h) *reinterpret_cast<float2*>(a0 + vt * 8) = make_float2(st.acc[vt][0], st.acc[vt][1]);
+                        if (head1 < h) *reinterpret_cast<float2*>(a1 + vt * 8) = make_float2(st.acc[vt][2], st.acc[vt][3]);
+                    }
+                    if (t4 == 0) {
+                        if (head0 < h) part_ml[slot * h + head0] = make_float2(st.m[0], st.l[0]);
+                        if (head1 < h) part_ml[slot * h + head1] = make_float2(st.m[1], st.l[1]);
+                    }
+                }
+            }
+            j += n_seg;
+            t = seg_end;
+        }
+        if (!ok) atomicExch(&timed_out, 1);
+    }
+
+    __syncthreads();
+    if (timed_out) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < kStages && s < issued; ++s) {
+                const int last_use = (issued - 1 - s) / kStages;
+                mbar_wait(full_s + s * 8, last_use & 1);
+            }
+            if (status) atomicOr(status, kStatusPipelineTimeout);
+        }
+        __syncthreads();
+    }
+}
+
+// Second pass of the persistent kernel: one CTA per (sequence, head) merges the slots of the
+// CTAs that hold pieces of the sequence (nothing to do when a single CTA had the whole sequence,
+// or it is empty).  seq_span[b] holds (T, G): a CTA whose share of the T tiles is empty wrote no
+// slot and is skipped.
+__global__ void __launch_bounds__(kHeadDim)
+stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restrict__ part_ml,
+                      const float* __restrict__ part_acc, float* __restrict__ o, int b, int h) {
+    const int s = blockIdx.x / h, head = blockIdx.x % h;
+    const int c = threadIdx.x;
+    const int2 span = seq_span[s];
+    if (span.y <= span.x) return;
+    const long long T = seq_span[b].x, G = seq_span[b].y;
+    float top = -INFINITY;
+    for (int cta = span.x; cta <= span.y; ++cta) {
+        if (cta * T / G == (cta + 1) * T / G) continue;
+        top = fmaxf(top, part_ml[((size_t)cta + s) * h + head].x);
+    }
+    float num = 0.f, den = 0.f;
+    for (int cta = span.x; cta <= span.y; ++cta) {
+        if (cta * T / G == (cta + 1) * T / G) continue;
+        const size_t slot = (size_t)cta + s;
+        const float2 ml = part_ml[slot * h + head];
+        const float w = fast_exp2(ml.x - top);
+        den = fmaf(w, ml.y, den);
+        num = fmaf(w, part_acc[(slot * h + head) * kHeadDim + c], num);
+    }
+    o[((size_t)s * h + head) * kHeadDim + c] = num / den;
 }
 
 }  // namespace mqa

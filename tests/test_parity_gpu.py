@@ -95,6 +95,39 @@ def test_small_cases_match_oracle(variant, b, h, m_max, lens):
     run_case(variant, b, h, m_max, lens, seed=b * 1000 + h)
 
 
+def _mixed_lens(b, m_max, seed):
+    r = np.random.default_rng(seed)
+    lens = r.integers(1, m_max + 1, size=b).astype(np.int32)
+    lens[r.integers(0, b, size=max(1, b // 10))] = 0          # some empty sequences
+    lens[r.integers(0, b, size=max(1, b // 10))] = m_max       # some full ones
+    lens[0], lens[-1] = 0, m_max
+    return lens
+
+
+# Batches large enough for the persistent kernel (>= 8 tiles of 32 rows per SM), shaped so that one
+# SM's share spans several sequences, starts and ends mid-sequence, and meets empty sequences.
+STREAM = [
+    (300, 8, 200, 21),      # 7 tiles per sequence, ~14 tiles per SM: every SM crosses sequences
+    (40, 16, 1500, 22),
+    (160, 32, 333, 23),
+    (1024, 4, 64, 24),      # the most sequences the persistent kernel indexes
+    (1100, 8, 64, 25),      # more than that: fixed-split kernel
+    (37, 32, 4000, 26),
+]
+
+
+@pytest.mark.parametrize("b,h,m_max,seed", STREAM)
+def test_persistent_kernel_shapes(b, h, m_max, seed):
+    run_case("mqa", b, h, m_max, _mixed_lens(b, m_max, seed), seed=seed)
+
+
+def test_persistent_kernel_all_empty_but_one():
+    b, h, m_max = 64, 16, 1024
+    lens = np.zeros(b, np.int32)
+    lens[17] = 1000
+    run_case("mqa", b, h, m_max, lens, seed=31)
+
+
 @pytest.mark.parametrize("variant", ["mqa", "mha"])
 @pytest.mark.parametrize("edge", range(60, 70))
 def test_every_length_around_a_tile_edge(variant, edge):
