@@ -151,6 +151,26 @@ StreamWorkspace stream_workspace(const Plan& p, const void* workspace) {
     return w;
 }
 
+// Launch `kernel` so that it may begin while the kernel before it in the stream is still running
+// (programmatic dependent launch).  Every kernel of this library waits (griddepcontrol.wait)
+// before it touches memory an earlier kernel may write, so the only effect is that launch
+// latency and set-up overlap the tail of the previous kernel.
+template <typename... Params, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem,
+                             cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
@@ -227,9 +247,9 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     alignas(64) CUtensorMap map_k, map_v;
     if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
         return MQA_ERR_CUDA;
-    kernel<<<(unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream>>>(
-        map_k, map_v, static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
-        p.n_splits);
+    launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
+                     static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
+                     p.n_splits);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -253,8 +273,8 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
     if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
-    kernel<<<(unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(
-        map_k, map_v, static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
+    launch_dependent(kernel, (unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
+                     static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -282,9 +302,9 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (p.kernel == Kernel::kMma2)
         return launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream);
     const unsigned grid = (unsigned)(p.units * (size_t)p.n_splits);
-    decode_split_simt_kernel<<<grid, kSimtThreads, 0, stream>>>(
-        static_cast<const uint4*>(q), static_cast<const uint4*>(K), static_cast<const uint4*>(V), lens, o,
-        part_ml, part_acc, status, h, multi_query ? h : 1, m_max, p.chunk_rows, p.n_splits);
+    launch_dependent(decode_split_simt_kernel, grid, kSimtThreads, 0, stream, static_cast<const uint4*>(q),
+                     static_cast<const uint4*>(K), static_cast<const uint4*>(V), lens, o, part_ml, part_acc, status, h,
+                     multi_query ? h : 1, m_max, p.chunk_rows, p.n_splits);
     return launch_status();
 }
 
@@ -298,15 +318,15 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     if (rc) return rc;
     if (p.stream()) {
         const StreamWorkspace w = stream_workspace(p, workspace);
-        stream_combine_kernel<<<(unsigned)((size_t)b * h), kHeadDim, 0, stream>>>(w.span, w.ml, w.acc, o, b, h);
+        launch_dependent(stream_combine_kernel, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h);
         return launch_status();
     }
     if (p.n_splits <= 1) return MQA_OK;
     const float2* part_ml = reinterpret_cast<const float2*>(workspace);
     const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits));
-    combine_splits_kernel<<<(unsigned)p.units, kHeadDim, 0, stream>>>(part_ml, part_acc, lens, o, h, m_max,
-                                                                      p.chunk_rows, p.n_splits);
+    launch_dependent(combine_splits_kernel, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens, o, h, m_max,
+                     p.chunk_rows, p.n_splits);
     return launch_status();
 }
 
@@ -333,9 +353,9 @@ int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new, int3
         !aligned4(status))
         return MQA_ERR_INVALID_ARG;
     if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
-    kv_cache_append_kernel<<<(unsigned)b, kAppendThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<uint4*>(K), static_cast<uint4*>(V), static_cast<const uint4*>(k_new),
-        static_cast<const uint4*>(v_new), lens, advance, status, kv_heads, m_max);
+    launch_dependent(kv_cache_append_kernel, (unsigned)b, kAppendThreads, 0, static_cast<cudaStream_t>(stream),
+                     static_cast<uint4*>(K), static_cast<uint4*>(V), static_cast<const uint4*>(k_new),
+                     static_cast<const uint4*>(v_new), lens, advance, status, kv_heads, m_max);
     return launch_status();
 }
 

@@ -26,6 +26,7 @@ combine_splits_kernel(const float2* __restrict__ part_ml, const float* __restric
                       int h, int m_max, int chunk_rows, int n_splits) {
     const size_t u = blockIdx.x;
     const int c = threadIdx.x;
+    grid_dependency_wait();          // the partials come from the kernel before this one
     int L = lens[u / h];
     L = L < 0 ? 0 : (L > m_max ? m_max : L);
     int live = (L + chunk_rows - 1) / chunk_rows;

@@ -32,6 +32,13 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
     return r;
 }
 
+// Programmatic dependent launch.  grid_dependency_wait(): block until the kernels this launch was
+// made dependent on have finished and their writes are visible (a no-op for an ordinary launch).
+// grid_launch_dependents(): allow the next kernel in the stream, if it was launched as a
+// programmatic dependent, to start its prologue while this grid is still running.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 // Clamp a sequence length into [0, m_max]; flag the status word if it had to move.
 __device__ __forceinline__ int clamp_len(int L, int m_max, int32_t* status) {
     if (L < 0 || L > m_max) {

@@ -39,6 +39,7 @@ constexpr int kStageBytes = 4 * kBoxBytes;             // K lo, K hi, V lo, V hi
 constexpr int kRowWarps = 4;                           // consumer warps that share the tiles
 constexpr long long kWaitLimitCycles = 2000000000ll;   // every mbarrier wait gives up after ~1 s of SM clock ...
 constexpr uint32_t kWaitRounds = 1u << 24;             // ... or after this many polling rounds
+constexpr int kSingleRoundingMinRows = 1024;            // prefixes this long feed P to the tensor cores in one bf16 rounding
 constexpr int kStreamMaxSeqs = 1024;                   // sequences the persistent kernel can index in shared memory
 
 // Ring depth must be a multiple of kRowWarps: tile i lives in stage i % kStages and belongs to
@@ -184,6 +185,10 @@ __device__ __forceinline__ void load_q_fragments(uint32_t (&qa)[8][4], const uin
 
 // One 32-row tile (cache rows row0 .. row0+31 of the sequence, of which rows < r1 are valid) for
 // 16 heads: S = Q K^T, online softmax update, O += P V.
+// HILO: feed P to the tensor cores as bf16 hi + lo parts (weights good to ~2^-17) instead of one
+// bf16 rounding (2^-9 per weight).  One rounding is enough once the prefix is long: the output
+// is then an average over many rows, of size ~1/sqrt(rows), and so is the rounding error.
+template <bool HILO>
 __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)[8][4], const LaneOffsets& off,
                                              uint32_t k_s, uint32_t v_s, int row0, int r1, int lane) {
     const int t4 = lane & 3;
@@ -247,11 +252,12 @@ __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)
             st.l[j >> 1] += p[j];
         }
         const uint32_t hi01 = pack_bf16(p[0], p[1]), hi23 = pack_bf16(p[2], p[3]);
-        const uint32_t lo01 = pack_bf16(p[0] - bf16_lo(hi01), p[1] - bf16_hi(hi01));
-        const uint32_t lo23 = pack_bf16(p[2] - bf16_lo(hi23), p[3] - bf16_hi(hi23));
         const int kk = nt >> 1, hf = (nt & 1) * 2;          // A regs: {g,k}, {g+8,k}, {g,k+8}, {g+8,k+8}
         p_hi[kk][hf] = hi01; p_hi[kk][hf + 1] = hi23;
-        p_lo[kk][hf] = lo01; p_lo[kk][hf + 1] = lo23;
+        if (HILO) {
+            p_lo[kk][hf] = pack_bf16(p[0] - bf16_lo(hi01), p[1] - bf16_hi(hi01));
+            p_lo[kk][hf + 1] = pack_bf16(p[2] - bf16_lo(hi23), p[3] - bf16_hi(hi23));
+        }
     }
     // O += P V : 2 k-steps of 16 rows x 16 n-tiles of 8 columns
 #pragma unroll
@@ -269,8 +275,10 @@ __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)
             if (ragged) { b0 &= keep_lo; b1 &= keep_hi; b2 &= keep_lo; b3 &= keep_hi; }
             mma_bf16(st.acc[vp * 2], p_hi[kk], b0, b1);
             mma_bf16(st.acc[vp * 2 + 1], p_hi[kk], b2, b3);
-            mma_bf16(st.acc[vp * 2], p_lo[kk], b0, b1);
-            mma_bf16(st.acc[vp * 2 + 1], p_lo[kk], b2, b3);
+            if (HILO) {
+                mma_bf16(st.acc[vp * 2], p_lo[kk], b0, b1);
+                mma_bf16(st.acc[vp * 2 + 1], p_lo[kk], b2, b3);
+            }
         }
     }
 }
@@ -322,6 +330,8 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const int split = blockIdx.x % n_splits;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
+    grid_launch_dependents();
     const int L = clamp_len(lens[seq], m_max, threadIdx.x == 0 ? status : nullptr);
     const int r0 = split * chunk_rows;
     const int r1 = min(L, r0 + chunk_rows);
@@ -390,7 +400,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
             ok = mbar_wait(full_s + s * 8, (i / kStages) & 1);
             if (!ok) break;
             const uint32_t k_s = stages_s + s * kStageBytes;
-            consume_tile(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
+            consume_tile<true>(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_s + s * 8);                 // this warp is done with the stage
         }
@@ -510,16 +520,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
     __shared__ int timed_out, issued;
 
-    // ---- tiles per sequence and their running sum (every CTA computes the same table) -----------
-    for (int s = threadIdx.x; s < b; s += Cfg::kThreads) {
-        const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
-        prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
-        if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
-            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
-        }
-    }
     if (threadIdx.x == 0) {
-        prefix[0] = 0;
         timed_out = 0;
         issued = 0;
         for (int s = 0; s < kStages; ++s) {
@@ -529,6 +530,18 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
+    grid_launch_dependents();
+
+    // ---- tiles per sequence and their running sum (every CTA computes the same table) -----------
+    for (int s = threadIdx.x; s < b; s += Cfg::kThreads) {
+        const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
+        prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
+        if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
+            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
+        }
+    }
+    if (threadIdx.x == 0) prefix[0] = 0;
     __syncthreads();
     if (warp == 0) {                                       // inclusive scan of prefix[1..b] by one warp
         const int per = (b + 31) / 32;
@@ -621,7 +634,11 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                 if (ok) ok = mbar_wait(full_s + stg * 8, (jj / kStages) & 1);
                 if (ok) {
                     const uint32_t k_s = stages_s + stg * kStageBytes;
-                    consume_tile(st, qa, off, k_s, k_s + 2 * kBoxBytes, first_row + (jj - j) * kTileRows, L, lane);
+                    const int row0 = first_row + (jj - j) * kTileRows;
+                    if (L >= kSingleRoundingMinRows)
+                        consume_tile<false>(st, qa, off, k_s, k_s + 2 * kBoxBytes, row0, L, lane);
+                    else
+                        consume_tile<true>(st, qa, off, k_s, k_s + 2 * kBoxBytes, row0, L, lane);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty_s + stg * 8);   // released even after a failed wait: nobody may hang
@@ -693,6 +710,7 @@ stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restric
                       const float* __restrict__ part_acc, float* __restrict__ o, int b, int h) {
     const int s = blockIdx.x / h, head = blockIdx.x % h;
     const int c = threadIdx.x;
+    grid_dependency_wait();          // the slots come from the kernel before this one
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
     const long long T = seq_span[b].x, G = seq_span[b].y;

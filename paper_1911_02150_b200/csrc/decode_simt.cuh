@@ -33,6 +33,8 @@ decode_split_simt_kernel(const uint4* __restrict__ q, const uint4* __restrict__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, cl = lane & 15;
 
+    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
+    grid_launch_dependents();
     const int L = clamp_len(lens[u / h], m_max, threadIdx.x == 0 ? status : nullptr);
     const int r0 = split * chunk_rows;
     const int r1 = min(L, r0 + chunk_rows);
