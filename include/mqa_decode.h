@@ -52,7 +52,9 @@ enum {
     MQA_ERR_INVALID_ARG = 1,         /* null or misaligned pointer, non-positive dimension   */
     MQA_ERR_UNSUPPORTED = 2,         /* k or v != 128, or a size the launch grid cannot hold */
     MQA_ERR_WORKSPACE_TOO_SMALL = 3, /* workspace_bytes < mqa_workspace_bytes(...)           */
-    MQA_ERR_CUDA = 4                 /* the CUDA runtime reported an error at launch         */
+    MQA_ERR_CUDA = 4,                /* the CUDA runtime reported an error at launch         */
+    MQA_ERR_STATIC_SCRATCH_TOO_SMALL = 5 /* mqa_decode_step_noalloc: these sizes need more scratch
+                                            than the library's built-in MQA_NOALLOC_SCRATCH_BYTES */
 };
 
 enum {
@@ -146,6 +148,36 @@ size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v);
  * streams when every cache is full.  Returns 0 for invalid arguments.  Informational; host-only.
  */
 int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int* chunk_rows);
+
+/*
+ * mqa_decode_step_noalloc -- mqa_decode_step for callers that cannot allocate.  (The paper has
+ * no counterpart to this entry point; it computes exactly what mqa_decode_step computes.)
+ *
+ * Some callers of a decode step cannot give it a workspace: a plugin or custom op that runs
+ * inside a host framework whose device memory was planned and reserved at start-up has no
+ * allocator to ask, and cudaMalloc is either forbidden there (it stalls the whole device while
+ * it runs) or bound to fail (the framework already holds all the memory).  This entry point
+ * takes only inputs and outputs.  Its scratch is a fixed array of MQA_NOALLOC_SCRATCH_BYTES
+ * bytes of device global memory inside the library image, which every GPU that loads the
+ * library keeps reserved until the process exits.
+ *
+ *   Arguments: as mqa_decode_step, without workspace and workspace_bytes.
+ *   Returns MQA_ERR_STATIC_SCRATCH_TOO_SMALL, and launches nothing, when
+ *   mqa_workspace_bytes(b, h, m_max, k, v) exceeds MQA_NOALLOC_SCRATCH_BYTES; otherwise whatever
+ *   mqa_decode_step returns for the same arguments.
+ *   Allocation: none.  The call uses no cudaMalloc, cudaFree or other allocating routine.
+ *   First call on a device: looks up the array's device address (cudaGetSymbolAddress, with
+ *   that device current) and remembers it; make this first call during set-up, before any
+ *   stream capture is begun on that device.
+ *   Sharing: every call on a device uses the same array, which still holds whatever the last
+ *   call left in it.  Nothing has to be cleared -- the second pass reads only slots that the
+ *   first pass of the same call has written -- but two calls whose kernels may overlap on the
+ *   GPU (different streams, no ordering between them) race on it and corrupt each other's
+ *   results.  Calls on one stream are safe.
+ */
+#define MQA_NOALLOC_SCRATCH_BYTES (8u * 1024u * 1024u)
+int mqa_decode_step_noalloc(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                            int32_t* status, int b, int h, int m_max, int k, int v, mqa_stream_t stream);
 
 /* mqa_status_string -- a static, human-readable name for a return code. */
 const char* mqa_status_string(int code);

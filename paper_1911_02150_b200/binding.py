@@ -17,14 +17,15 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmqa_decode.so")
 
 MQA_OK = 0
-ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 1, 2, 3, 4
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_STATIC_SCRATCH_TOO_SMALL = 1, 2, 3, 4, 5
+NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 STATUS_APPEND_CACHE_FULL, STATUS_APPEND_NEGATIVE_LEN, STATUS_LEN_CLAMPED, STATUS_PIPELINE_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = (
     "kv_cache_append", "mqa_decode_step", "mha_decode_step",
     "mqa_decode_step_split", "mqa_decode_step_combine",
     "mha_decode_step_split", "mha_decode_step_combine",
-    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string",
+    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string", "mqa_decode_step_noalloc",
 )
 
 _lib = None
@@ -56,6 +57,8 @@ def lib() -> ctypes.CDLL:
             f = getattr(L, n)
             f.argtypes = [vp, vp, vp, sz, I, I, I, I, I, vp]
             f.restype = I
+        L.mqa_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, I, I, I, I, I, vp]
+        L.mqa_decode_step_noalloc.restype = I
         L.mqa_workspace_bytes.argtypes = [I, I, I, I, I]
         L.mqa_workspace_bytes.restype = sz
         L.mqa_plan_splits.argtypes = [I, I, I, I, I, I, ctypes.POINTER(I)]
@@ -187,3 +190,28 @@ def mqa_decode_step_combine(q, K, V, lens, o, workspace=None, status=None, strea
 
 def mha_decode_step_combine(q, K, V, lens, o, workspace=None, status=None, stream=None):
     return _step("mha_decode_step_combine", False, q, K, V, lens, o, workspace, status, stream, "combine")
+
+
+def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
+    """The multi-query step for callers that cannot allocate a workspace (a plugin inside a host
+    framework that planned and reserved all device memory up front): same arguments as
+    :func:`mqa_decode_step` minus the workspace; the scratch is a fixed array inside the library.
+
+    Make the first call on each device during set-up (it looks up the array's address).  All
+    calls on a device share that one array, so calls whose kernels could overlap on the GPU must
+    not be issued concurrently.  Raises ``MqaError`` with ``ERR_STATIC_SCRATCH_TOO_SMALL`` when the
+    sizes need more than ``NOALLOC_SCRATCH_BYTES`` of scratch."""
+    b, h, k = q.shape
+    m_max, v = K.shape[-2], V.shape[-1]
+    _need(q, torch.bfloat16, (b, h, k), "q")
+    _need(K, torch.bfloat16, (b, m_max, k), "K")
+    _need(V, torch.bfloat16, (b, m_max, v), "V")
+    _need(lens, torch.int32, (b,), "lens")
+    _need(o, torch.float32, (b, h, v), "o")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    with torch.cuda.device(q.device):
+        rc = lib().mqa_decode_step_noalloc(_ptr(q), _ptr(K), _ptr(V), _ptr(lens), _ptr(o), _ptr(status),
+                                           b, h, m_max, k, v, _stream(stream))
+    _check(rc, "mqa_decode_step_noalloc")
+    return o

@@ -420,6 +420,8 @@ const char* mqa_status_string(int code) {
         case MQA_ERR_UNSUPPORTED: return "unsupported configuration (k and v must be 128)";
         case MQA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small (see mqa_workspace_bytes)";
         case MQA_ERR_CUDA: return "CUDA launch error";
+        case MQA_ERR_STATIC_SCRATCH_TOO_SMALL:
+            return "these sizes need more scratch than the built-in array of mqa_decode_step_noalloc";
         default: return "unknown status code";
     }
 }

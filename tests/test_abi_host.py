@@ -21,6 +21,7 @@ def L():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "mqa_decode.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"^\s*#.*$", "", text, flags=re.M)          # preprocessor lines
     return sorted(set(re.findall(r"\b(\w+)\s*\([^;{}]*\)\s*;", text)))
 
 
