@@ -216,12 +216,12 @@ EncodeTiledFn encode_fn() {
 
 // The cache of one tensor (K or V) as a 2-D bf16 tensor [rows = b * m_max][128 columns], fetched in
 // boxes of kTileRows rows x 64 columns (128 bytes, the span of the 128-byte swizzle).
-bool encode_cache_map(CUtensorMap* map, const void* base, long long rows) {
+bool encode_cache_map(CUtensorMap* map, const void* base, long long rows, int box_rows = kTileRows) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
-    const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)kTileRows};
+    const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -269,11 +269,13 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
         }
         g_stream_opt_in[dev][M_TILES - 1].store(1, std::memory_order_release);
     }
-    alignas(64) CUtensorMap map_k, map_v;
-    if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
+    alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub;
+    const long long rows = (long long)b * m_max;
+    if (!encode_cache_map(&map_k, K, rows, kStreamStageRows) || !encode_cache_map(&map_v, V, rows, kStreamStageRows) ||
+        !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
-    launch_dependent(kernel, (unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
+    launch_dependent(kernel, (unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
                      static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }

@@ -20,7 +20,8 @@
 //                                      all sequences (valid rows only, from lens) form one
 //                                      line that is cut into equal contiguous shares, so every
 //                                      SM streams the same number of bytes whatever the batch
-//                                      size, context length or raggedness.
+//                                      size, context length or raggedness.  It stages 128 rows
+//                                      at a time; each of its 4 row-warps takes 32 of them.
 //
 // Rows at or beyond lens[b] are never used: their logits are replaced by -inf by index and
 // their V fragments are zeroed by index (a NaN times a zero weight would still be a NaN).
@@ -37,6 +38,12 @@ constexpr int kBoxCols = 64;                           // 64 bf16 = 128 bytes = 
 constexpr int kBoxBytes = kTileRows * kBoxCols * 2;    // 4 KiB
 constexpr int kStageBytes = 4 * kBoxBytes;             // K lo, K hi, V lo, V hi = 16 KiB
 constexpr int kRowWarps = 4;                           // consumer warps that share the tiles
+// The persistent kernel stages 128 rows at a time (4 sub-tiles of 32 rows, one per row-warp): a full
+// stage is fetched with four 16 KiB TMA boxes, which the copy engine moves measurably faster than
+// sixteen 4 KiB ones; a stage at the end of a segment is fetched sub-tile by sub-tile with 4 KiB boxes.
+constexpr int kStreamStageRows = kRowWarps * kTileRows;        // 128
+constexpr int kStreamBoxBytes = kStreamStageRows * kBoxCols * 2;   // 16 KiB: 128 rows x 128 bytes
+constexpr int kStreamStageBytes = 4 * kStreamBoxBytes;         // 64 KiB
 constexpr long long kWaitLimitCycles = 2000000000ll;   // every mbarrier wait gives up after ~1 s of SM clock ...
 constexpr uint32_t kWaitRounds = 1u << 24;             // ... or after this many polling rounds
 constexpr int kSingleRoundingMinRows = 1024;            // prefixes this long feed P to the tensor cores in one bf16 rounding
@@ -60,12 +67,11 @@ template <int M_TILES>
 struct StreamCfg {                                     // persistent kernel, one CTA per SM
     static constexpr int kConsumerWarps = M_TILES * kRowWarps;
     static constexpr int kThreads = (kConsumerWarps + 1) * 32;
-    static constexpr int kStages = 12;
-    static_assert(kStages % kRowWarps == 0, "a stage must always be consumed by the same warp");
+    static constexpr int kStages = 3;                  // every consumer warp waits on every stage: any depth is safe
     static constexpr int kStateFloats = 16 * 4 + 4;    // acc + (m, l) x 2 rows, per thread
     static constexpr int kMergeBytes = M_TILES * kStateFloats * 32 * 4;
     static constexpr int kPrefixBytes = (kStreamMaxSeqs + 1) * 4 + 12;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kMergeBytes + kPrefixBytes + 256 /* barriers */ +
+    static constexpr int kSmemBytes = kStages * kStreamStageBytes + kMergeBytes + kPrefixBytes + 256 /* barriers */ +
                                       1024 /* alignment slack */;
     static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
     static constexpr int kCtasPerSm = 1;
@@ -188,7 +194,8 @@ __device__ __forceinline__ void load_q_fragments(uint32_t (&qa)[8][4], const uin
 // HILO: feed P to the tensor cores as bf16 hi + lo parts (weights good to ~2^-17) instead of one
 // bf16 rounding (2^-9 per weight).  One rounding is enough once the prefix is long: the output
 // is then an average over many rows, of size ~1/sqrt(rows), and so is the rounding error.
-template <bool HILO>
+// HALF_STRIDE: bytes between the box holding columns 0..63 and the box holding columns 64..127.
+template <bool HILO, int HALF_STRIDE>
 __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)[8][4], const LaneOffsets& off,
                                              uint32_t k_s, uint32_t v_s, int row0, int r1, int lane) {
     const int t4 = lane & 3;
@@ -200,7 +207,7 @@ __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)
     for (int nt = 0; nt < 4; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-        const uint32_t a = k_s + off.k[ks & 3] + (ks >> 2) * kBoxBytes;
+        const uint32_t a = k_s + off.k[ks & 3] + (ks >> 2) * HALF_STRIDE;
 #pragma unroll
         for (int np = 0; np < 2; ++np) {               // n-tile pairs (0,1) and (2,3): 16 rows = 2 KiB apart
             uint32_t b0, b1, b2, b3;
@@ -271,7 +278,7 @@ __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)
 #pragma unroll
         for (int vp = 0; vp < 8; ++vp) {                         // pairs of 8-column n-tiles
             uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(v_s + off.v[vp & 3] + (vp >> 2) * kBoxBytes + kk * 2048, b0, b1, b2, b3);
+            ldmatrix_x4_trans(v_s + off.v[vp & 3] + (vp >> 2) * HALF_STRIDE + kk * 2048, b0, b1, b2, b3);
             if (ragged) { b0 &= keep_lo; b1 &= keep_hi; b2 &= keep_lo; b3 &= keep_hi; }
             mma_bf16(st.acc[vp * 2], p_hi[kk], b0, b1);
             mma_bf16(st.acc[vp * 2 + 1], p_hi[kk], b2, b3);
@@ -400,7 +407,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
             ok = mbar_wait(full_s + s * 8, (i / kStages) & 1);
             if (!ok) break;
             const uint32_t k_s = stages_s + s * kStageBytes;
-            consume_tile<true>(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
+            consume_tile<true, kBoxBytes>(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_s + s * 8);                 // this warp is done with the stage
         }
@@ -502,6 +509,7 @@ __host__ __device__ inline size_t stream_acc_bytes(int slots, int h) { return (s
 template <int M_TILES>
 __global__ void __launch_bounds__(StreamCfg<M_TILES>::kThreads, 1)
 mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                             const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
                              const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                              float* __restrict__ o, int2* __restrict__ seq_span, float2* __restrict__ part_ml,
                              float* __restrict__ part_acc, int32_t* __restrict__ status, int b, int h, int m_max) {
@@ -513,7 +521,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* stages = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-    float* merge_buf = reinterpret_cast<float*>(stages + kStages * kStageBytes);            // [M_TILES][68][32]
+    float* merge_buf = reinterpret_cast<float*>(stages + kStages * kStreamStageBytes);      // [M_TILES][68][32]
     int* prefix = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(merge_buf) + Cfg::kMergeBytes);  // [b + 1]
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + Cfg::kPrefixBytes / 8 * 8);
     const uint32_t stages_s = smem_addr(stages);
@@ -524,8 +532,8 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         timed_out = 0;
         issued = 0;
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_s + s * 8, 1);
-            mbar_init(empty_s + s * 8, M_TILES);
+            mbar_init(full_s + s * 8, 1);                      // the producer's arrive + the TMA bytes
+            mbar_init(empty_s + s * 8, Cfg::kConsumerWarps);   // every consumer warp passes every stage
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -533,7 +541,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
 
-    // ---- tiles per sequence and their running sum (every CTA computes the same table) -----------
+    // ---- 32-row sub-tiles per sequence and their running sum (every CTA computes the same table)
     for (int s = threadIdx.x; s < b; s += Cfg::kThreads) {
         const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
         prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
@@ -561,17 +569,9 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     const long long T = prefix[b];
     const long long t_begin = (long long)cta * T / G, t_end = (long long)(cta + 1) * T / G;
 
-    // which CTAs hold pieces of each sequence (read by the second pass); spread over the CTAs
-    for (int s = cta + (int)threadIdx.x * G; s < b; s += G * Cfg::kThreads) {
-        const int t0 = prefix[s], t1 = prefix[s + 1];
-        seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
-    }
-    if (cta == 0 && threadIdx.x == 0) seq_span[b] = make_int2((int)T, G);
-    if (t_begin >= t_end) return;                          // uniform: this CTA has no tiles
-
     // first sequence of this CTA's share: the s with prefix[s] <= t_begin < prefix[s+1]
-    int s_first;
-    {
+    int s_first = 0;
+    if (t_begin < t_end) {
         int lo = 0, hi = b - 1;
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
@@ -586,41 +586,63 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 
     if (warp == Cfg::kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
-        if (lane == 0) {
+        if (lane == 0 && t_begin < t_end) {
             bool ok = true;
             int s = s_first;
-            int j = 0;                                     // tiles issued by this CTA so far
-            for (long long t = t_begin; t < t_end && ok; ++t, ++j) {
+            int j = 0;                                     // stages issued by this CTA so far
+            for (long long t = t_begin; t < t_end && ok;) {
                 while (prefix[s + 1] <= t) ++s;
-                const int stg = j % kStages;
-                if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
-                if (!ok) break;
-                const uint32_t bar = full_s + stg * 8;
-                const uint32_t dst = stages_s + stg * kStageBytes;
-                mbar_expect_tx(bar, kStageBytes);
-                const int y = s * m_max + (int)(t - prefix[s]) * kTileRows;
-                tma_load_2d(dst, &map_k, 0, y, bar);
-                tma_load_2d(dst + kBoxBytes, &map_k, kBoxCols, y, bar);
-                tma_load_2d(dst + 2 * kBoxBytes, &map_v, 0, y, bar);
-                tma_load_2d(dst + 3 * kBoxBytes, &map_v, kBoxCols, y, bar);
-                issued = j + 1;
+                const long long seg_end = min((long long)prefix[s + 1], t_end);
+                for (long long u = t; u < seg_end && ok; u += kRowWarps, ++j) {
+                    const int nsub = (int)min((long long)kRowWarps, seg_end - u);
+                    const int stg = j % kStages;
+                    if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
+                    if (!ok) break;
+                    const uint32_t bar = full_s + stg * 8;
+                    const uint32_t dst = stages_s + stg * kStreamStageBytes;
+                    mbar_expect_tx(bar, nsub * kStageBytes);
+                    const int y = s * m_max + (int)(u - prefix[s]) * kTileRows;
+                    if (nsub == kRowWarps) {
+                        tma_load_2d(dst, &map_k, 0, y, bar);
+                        tma_load_2d(dst + kStreamBoxBytes, &map_k, kBoxCols, y, bar);
+                        tma_load_2d(dst + 2 * kStreamBoxBytes, &map_v, 0, y, bar);
+                        tma_load_2d(dst + 3 * kStreamBoxBytes, &map_v, kBoxCols, y, bar);
+                    } else {
+                        for (int i = 0; i < nsub; ++i) {
+                            const uint32_t d = dst + i * kBoxBytes;
+                            tma_load_2d(d, &map_k_sub, 0, y + i * kTileRows, bar);
+                            tma_load_2d(d + kStreamBoxBytes, &map_k_sub, kBoxCols, y + i * kTileRows, bar);
+                            tma_load_2d(d + 2 * kStreamBoxBytes, &map_v_sub, 0, y + i * kTileRows, bar);
+                            tma_load_2d(d + 3 * kStreamBoxBytes, &map_v_sub, kBoxCols, y + i * kTileRows, bar);
+                        }
+                    }
+                    issued = j + 1;
+                }
+                t = seg_end;
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
     } else {
         // --------------------------------------------------------------- consumer warps
+        // which CTAs hold pieces of each sequence (read by the second pass); spread over the CTAs
+        if (warp == 0) {
+            for (int s = cta + lane * G; s < b; s += G * 32) {
+                const int t0 = prefix[s], t1 = prefix[s + 1];
+                seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
+            }
+            if (cta == 0 && lane == 0) seq_span[b] = make_int2((int)T, G);
+        }
         WarpState st;
         LaneOffsets off;
         off.init(lane);
         const int g = lane >> 2, t4 = lane & 3;
         float* my_buf = merge_buf + mt * Cfg::kStateFloats * 32;
         bool ok = true;
-        int j = 0;                                         // index of the segment's first tile in this CTA's stream
+        int j = 0;                                         // stages consumed by this CTA so far
         int s = s_first;
         for (long long t = t_begin; t < t_end;) {
             while (prefix[s + 1] <= t) ++s;
             const long long seg_end = min((long long)prefix[s + 1], t_end);
-            const int n_seg = (int)(seg_end - t);
             const int first_row = (int)(t - prefix[s]) * kTileRows;
             const int L = min(max(__ldg(lens + s), 0), m_max);
             const bool whole = (t == prefix[s]) && (seg_end == prefix[s + 1]);
@@ -628,17 +650,17 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
             st.reset();
             uint32_t qa[8][4];
             load_q_fragments(qa, q, (size_t)s, h, mt, lane);
-            // this warp's tiles of the segment: stream positions jj = j .. j+n_seg-1 with jj % kRowWarps == rw
-            for (int jj = j + ((rw - j) & (kRowWarps - 1)); jj < j + n_seg; jj += kRowWarps) {
-                const int stg = jj % kStages;
-                if (ok) ok = mbar_wait(full_s + stg * 8, (jj / kStages) & 1);
-                if (ok) {
-                    const uint32_t k_s = stages_s + stg * kStageBytes;
-                    const int row0 = first_row + (jj - j) * kTileRows;
+            for (long long u = t; u < seg_end; u += kRowWarps, ++j) {
+                const int nsub = (int)min((long long)kRowWarps, seg_end - u);
+                const int stg = j % kStages;
+                if (ok) ok = mbar_wait(full_s + stg * 8, (j / kStages) & 1);
+                if (ok && rw < nsub) {                     // row-warp rw takes sub-tile rw of the stage
+                    const uint32_t k_s = stages_s + stg * kStreamStageBytes + rw * kBoxBytes;
+                    const int row0 = first_row + ((int)(u - t) + rw) * kTileRows;
                     if (L >= kSingleRoundingMinRows)
-                        consume_tile<false>(st, qa, off, k_s, k_s + 2 * kBoxBytes, row0, L, lane);
+                        consume_tile<false, kStreamBoxBytes>(st, qa, off, k_s, k_s + 2 * kStreamBoxBytes, row0, L, lane);
                     else
-                        consume_tile<true>(st, qa, off, k_s, k_s + 2 * kBoxBytes, row0, L, lane);
+                        consume_tile<true, kStreamBoxBytes>(st, qa, off, k_s, k_s + 2 * kStreamBoxBytes, row0, L, lane);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty_s + stg * 8);   // released even after a failed wait: nobody may hang
@@ -682,7 +704,6 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                     }
                 }
             }
-            j += n_seg;
             t = seg_end;
         }
         if (!ok) atomicExch(&timed_out, 1);
