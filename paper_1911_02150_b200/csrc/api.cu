@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <cstdlib>
 
 #include "../../include/mqa_decode.h"
 #include "append.cuh"
@@ -13,6 +14,7 @@
 #include "common.cuh"
 #include "decode_mma.cuh"
 #include "decode_simt.cuh"
+#include "decode_umma.cuh"
 
 namespace mqa {
 namespace {
@@ -36,7 +38,7 @@ int sm_count() {
     return n;
 }
 
-enum class Kernel { kSimt, kMma1, kMma2, kStream1, kStream2 };
+enum class Kernel { kSimt, kMma1, kMma2, kStream1, kStream2, kUmma };
 
 struct Plan {
     int n_splits = 0;     // 0 = invalid.  Fixed-split kernels: splits per sequence.  Persistent kernel: the
@@ -46,7 +48,7 @@ struct Plan {
     int b = 0, h = 0;
     int grid = 0;         // persistent kernel: number of CTAs
     Kernel kernel = Kernel::kSimt;
-    bool stream() const { return kernel == Kernel::kStream1 || kernel == Kernel::kStream2; }
+    bool stream() const { return kernel == Kernel::kStream1 || kernel == Kernel::kStream2 || kernel == Kernel::kUmma; }
 };
 
 bool dims_ok(int b, int h, int m_max) { return b > 0 && h > 0 && m_max > 0; }
@@ -108,7 +110,10 @@ Plan plan_stream(int b, int h, int m_max) {
     Plan p;
     p.units = (size_t)b * h;
     p.b = b; p.h = h;
-    p.kernel = h <= 16 ? Kernel::kStream1 : Kernel::kStream2;
+    // up to 32 heads the register-fragment mma.sync kernel; 33..64 heads the tcgen05 kernel.
+    // MQA_DECODE_UMMA=1 in the environment sends 17..32 heads to the tcgen05 kernel as well (for comparisons).
+    static const bool force_umma = [] { const char* e = getenv("MQA_DECODE_UMMA"); return e && e[0] == '1'; }();
+    p.kernel = h <= 16 ? Kernel::kStream1 : ((h <= 32 && !force_umma) ? Kernel::kStream2 : Kernel::kUmma);
     p.grid = sm_count();
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
@@ -120,11 +125,11 @@ Plan plan_stream(int b, int h, int m_max) {
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // heads beyond two 16-row tensor-core tiles, or a row space too large for the 32-bit TMA
     // coordinates, go to the general CUDA-core kernel
-    if (!(multi_query && h <= 32 && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
-    // enough tiles to give every SM a real share: the persistent kernel; otherwise fixed splits
+    if (!(multi_query && h <= 64 && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
+    // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
-    if (b <= kStreamMaxSeqs && tiles >= 8LL * sm_count()) return plan_stream(b, h, m_max);
-    return plan_mma(b, h, m_max);
+    if (b <= kStreamMaxSeqs && tiles >= 8LL * sm_count() && sm_count() <= 256) return plan_stream(b, h, m_max);
+    return h <= 32 ? plan_mma(b, h, m_max) : plan_simt(b, h, m_max);
 }
 
 size_t plan_workspace_bytes(const Plan& p) {
@@ -280,6 +285,32 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
+std::atomic<int> g_umma_opt_in[kMaxDevices];
+
+int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
+    auto kernel = mqa_decode_stream_umma_kernel;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!g_umma_opt_in[dev].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+        g_umma_opt_in[dev].store(1, std::memory_order_release);
+    }
+    alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub, map_q;
+    const long long rows = (long long)b * m_max;
+    if (!encode_cache_map(&map_k, K, rows, kUmmaStageRows) || !encode_cache_map(&map_v, V, rows, kUmmaStageRows) ||
+        !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows) ||
+        !encode_cache_map(&map_q, q, (long long)b * h, 64))
+        return MQA_ERR_CUDA;
+    const StreamWorkspace w = stream_workspace(p, workspace);
+    launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, kUmmaSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
+                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
+    return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
+}
+
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
 
 int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
@@ -291,6 +322,7 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
+    if (p.kernel == Kernel::kUmma) return launch_umma(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream1)
         return launch_stream<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream2)

@@ -665,42 +665,91 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty_s + stg * 8);   // released even after a failed wait: nobody may hang
             }
-            // fold the row-warps of this head tile into row-warp 0: 3 -> 2 -> 1 -> 0
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 1);
                 st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 2);
             }
-            named_barrier(1, kConsumerThreads);            // the previous segment's last reader is done with the buffer
-#pragma unroll 1
-            for (int r = kRowWarps - 1; r >= 1; --r) {
-                if (rw == r) store_state(st, my_buf, lane);
+            const int head0 = mt * 16 + g, head1 = head0 + 8;
+            const size_t slot = (size_t)cta + s;
+            if (seg_end == t_end) {
+                // Last segment of this CTA: nothing is in flight any more, so the stage memory is
+                // free.  Every row-warp parks its state there and all consumer threads merge in
+                // parallel, each taking a quarter of its own fragment columns.
+                float* park = reinterpret_cast<float*>(stages);                   // [consumer warp][68][32]
+                named_barrier(1, kConsumerThreads);                               // all warps are done reading tiles
+                store_state(st, park + warp * Cfg::kStateFloats * 32, lane);
                 named_barrier(1, kConsumerThreads);
-                if (rw == r - 1) merge_state(st, my_buf, lane);
-            }
-            if (rw == 0) {
-                const int head0 = mt * 16 + g, head1 = head0 + 8;
-                if (whole) {
-                    const float inv0 = 1.f / st.l[0], inv1 = 1.f / st.l[1];
-                    float* o0 = o + ((size_t)s * h + head0) * kHeadDim + t4 * 2;
-                    float* o1 = o + ((size_t)s * h + head1) * kHeadDim + t4 * 2;
+                float wgt[kRowWarps][2], m_new[2] = {-INFINITY, -INFINITY}, l_new[2] = {0.f, 0.f};
 #pragma unroll
-                    for (int vt = 0; vt < 16; ++vt) {
-                        if (head0 < h) *reinterpret_cast<float2*>(o0 + vt * 8) = make_float2(st.acc[vt][0] * inv0, st.acc[vt][1] * inv0);
-                        if (head1 < h) *reinterpret_cast<float2*>(o1 + vt * 8) = make_float2(st.acc[vt][2] * inv1, st.acc[vt][3] * inv1);
-                    }
-                } else {
-                    const size_t slot = (size_t)cta + s;
-                    float* a0 = part_acc + (slot * h + head0) * kHeadDim + t4 * 2;
-                    float* a1 = part_acc + (slot * h + head1) * kHeadDim + t4 * 2;
+                for (int w = 0; w < kRowWarps; ++w) {
+                    const float* src = park + (w * M_TILES + mt) * Cfg::kStateFloats * 32;
+                    wgt[w][0] = src[64 * 32 + lane];
+                    wgt[w][1] = src[65 * 32 + lane];
+                    m_new[0] = fmaxf(m_new[0], wgt[w][0]);
+                    m_new[1] = fmaxf(m_new[1], wgt[w][1]);
+                }
 #pragma unroll
-                    for (int vt = 0; vt < 16; ++vt) {
-                        if (head0 < h) *reinterpret_cast<float2*>(a0 + vt * 8) = make_float2(st.acc[vt][0], st.acc[vt][1]);
-                        if (head1 < h) *reinterpret_cast<float2*>(a1 + vt * 8) = make_float2(st.acc[vt][2], st.acc[vt][3]);
+                for (int w = 0; w < kRowWarps; ++w) {
+                    const float* src = park + (w * M_TILES + mt) * Cfg::kStateFloats * 32;
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        wgt[w][r] = wgt[w][r] == -INFINITY ? 0.f : fast_exp2(wgt[w][r] - m_new[r]);
+                        l_new[r] = fmaf(wgt[w][r], src[(66 + r) * 32 + lane], l_new[r]);
                     }
-                    if (t4 == 0) {
-                        if (head0 < h) part_ml[slot * h + head0] = make_float2(st.m[0], st.l[0]);
-                        if (head1 < h) part_ml[slot * h + head1] = make_float2(st.m[1], st.l[1]);
+                }
+                const float inv0 = whole ? 1.f / l_new[0] : 1.f, inv1 = whole ? 1.f / l_new[1] : 1.f;
+                float* d0 = (whole ? o + ((size_t)s * h + head0) * kHeadDim : part_acc + (slot * h + head0) * kHeadDim) + t4 * 2;
+                float* d1 = (whole ? o + ((size_t)s * h + head1) * kHeadDim : part_acc + (slot * h + head1) * kHeadDim) + t4 * 2;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int vt = rw * 4 + q4;                                    // this thread's quarter
+                    float v[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int w = 0; w < kRowWarps; ++w) {
+                        const float* src = park + (w * M_TILES + mt) * Cfg::kStateFloats * 32;
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj) v[jj] = fmaf(wgt[w][jj >> 1], src[(vt * 4 + jj) * 32 + lane], v[jj]);
+                    }
+                    if (head0 < h) *reinterpret_cast<float2*>(d0 + vt * 8) = make_float2(v[0] * inv0, v[1] * inv0);
+                    if (head1 < h) *reinterpret_cast<float2*>(d1 + vt * 8) = make_float2(v[2] * inv1, v[3] * inv1);
+                }
+                if (!whole && rw == 0 && t4 == 0) {
+                    if (head0 < h) part_ml[slot * h + head0] = make_float2(m_new[0], l_new[0]);
+                    if (head1 < h) part_ml[slot * h + head1] = make_float2(m_new[1], l_new[1]);
+                }
+            } else {
+                // A segment in the middle of the share: tiles of the next one are already streaming
+                // into the stages, so fold the row-warps 3 -> 2 -> 1 -> 0 through the small buffer.
+                named_barrier(1, kConsumerThreads);        // the previous segment's last reader is done with the buffer
+#pragma unroll 1
+                for (int r = kRowWarps - 1; r >= 1; --r) {
+                    if (rw == r) store_state(st, my_buf, lane);
+                    named_barrier(1, kConsumerThreads);
+                    if (rw == r - 1) merge_state(st, my_buf, lane);
+                }
+                if (rw == 0) {
+                    if (whole) {
+                        const float inv0 = 1.f / st.l[0], inv1 = 1.f / st.l[1];
+                        float* o0 = o + ((size_t)s * h + head0) * kHeadDim + t4 * 2;
+                        float* o1 = o + ((size_t)s * h + head1) * kHeadDim + t4 * 2;
+#pragma unroll
+                        for (int vt = 0; vt < 16; ++vt) {
+                            if (head0 < h) *reinterpret_cast<float2*>(o0 + vt * 8) = make_float2(st.acc[vt][0] * inv0, st.acc[vt][1] * inv0);
+                            if (head1 < h) *reinterpret_cast<float2*>(o1 + vt * 8) = make_float2(st.acc[vt][2] * inv1, st.acc[vt][3] * inv1);
+                        }
+                    } else {
+                        float* a0 = part_acc + (slot * h + head0) * kHeadDim + t4 * 2;
+                        float* a1 = part_acc + (slot * h + head1) * kHeadDim + t4 * 2;
+#pragma unroll
+                        for (int vt = 0; vt < 16; ++vt) {
+                            if (head0 < h) *reinterpret_cast<float2*>(a0 + vt * 8) = make_float2(st.acc[vt][0], st.acc[vt][1]);
+                            if (head1 < h) *reinterpret_cast<float2*>(a1 + vt * 8) = make_float2(st.acc[vt][2], st.acc[vt][3]);
+                        }
+                        if (t4 == 0) {
+                            if (head0 < h) part_ml[slot * h + head0] = make_float2(st.m[0], st.l[0]);
+                            if (head1 < h) part_ml[slot * h + head1] = make_float2(st.m[1], st.l[1]);
+                        }
                     }
                 }
             }
@@ -734,20 +783,41 @@ stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restric
     grid_dependency_wait();          // the slots come from the kernel before this one
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
+    __shared__ float w_s[256], l_s[256];
+    __shared__ int slot_s[256], n_s;
+    const int n_cta = span.y - span.x + 1;              // at most the grid of the first pass (<= 256 SMs)
     const long long T = seq_span[b].x, G = seq_span[b].y;
-    float top = -INFINITY;
-    for (int cta = span.x; cta <= span.y; ++cta) {
-        if (cta * T / G == (cta + 1) * T / G) continue;
-        top = fmaxf(top, part_ml[((size_t)cta + s) * h + head].x);
+    // every candidate CTA's (max, sum) is fetched by its own thread: one round trip for all of them
+    for (int i = c; i < n_cta; i += kHeadDim) {
+        const long long cta = span.x + i;
+        const bool live = cta * T / G != (cta + 1) * T / G;
+        const float2 ml = live ? part_ml[((size_t)cta + s) * h + head] : make_float2(-INFINITY, 0.f);
+        w_s[i] = ml.x;
+        l_s[i] = ml.y;
     }
+    __syncthreads();
+    float top = -INFINITY;
+    for (int i = 0; i < n_cta; ++i) top = fmaxf(top, w_s[i]);
+    __syncthreads();
+    if (c == 0) {                                       // compact the live pieces, in order
+        int n = 0;
+        for (int i = 0; i < n_cta; ++i) {
+            if (w_s[i] == -INFINITY) continue;
+            w_s[n] = fast_exp2(w_s[i] - top);
+            l_s[n] = l_s[i];
+            slot_s[n] = span.x + i + s;
+            ++n;
+        }
+        n_s = n;
+    }
+    __syncthreads();
+    const int n = n_s;
     float num = 0.f, den = 0.f;
-    for (int cta = span.x; cta <= span.y; ++cta) {
-        if (cta * T / G == (cta + 1) * T / G) continue;
-        const size_t slot = (size_t)cta + s;
-        const float2 ml = part_ml[slot * h + head];
-        const float w = fast_exp2(ml.x - top);
-        den = fmaf(w, ml.y, den);
-        num = fmaf(w, part_acc[(slot * h + head) * kHeadDim + c], num);
+    const float* col = part_acc + (size_t)head * kHeadDim + c;
+#pragma unroll 4
+    for (int i = 0; i < n; ++i) {
+        den = fmaf(w_s[i], l_s[i], den);
+        num = fmaf(w_s[i], col[(size_t)slot_s[i] * h * kHeadDim], num);
     }
     o[((size_t)s * h + head) * kHeadDim + c] = num / den;
 }

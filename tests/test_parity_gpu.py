@@ -113,6 +113,10 @@ STREAM = [
     (1024, 4, 64, 24),      # the most sequences the persistent kernel indexes
     (1100, 8, 64, 25),      # more than that: fixed-split kernel
     (37, 32, 4000, 26),
+    (64, 24, 700, 27),      # 17..64 heads: the tcgen05 kernel; 24 heads leave half of the second head group empty
+    (40, 48, 1500, 28),
+    (33, 64, 2100, 29),
+    (300, 17, 200, 30),
 ]
 
 
