@@ -111,9 +111,9 @@ Plan plan_stream(int b, int h, int m_max) {
     p.units = (size_t)b * h;
     p.b = b; p.h = h;
     // up to 32 heads the register-fragment mma.sync kernel; 33..64 heads the tcgen05 kernel.
-    // MQA_DECODE_UMMA=1 in the environment sends 17..32 heads to the tcgen05 kernel as well (for comparisons).
+    // MQA_DECODE_UMMA=1 in the environment sends every head count to the tcgen05 kernel (for comparisons).
     static const bool force_umma = [] { const char* e = getenv("MQA_DECODE_UMMA"); return e && e[0] == '1'; }();
-    p.kernel = h <= 16 ? Kernel::kStream1 : ((h <= 32 && !force_umma) ? Kernel::kStream2 : Kernel::kUmma);
+    p.kernel = force_umma ? Kernel::kUmma : (h <= 16 ? Kernel::kStream1 : (h <= 32 ? Kernel::kStream2 : Kernel::kUmma));
     p.grid = sm_count();
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
@@ -285,25 +285,27 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
-std::atomic<int> g_umma_opt_in[kMaxDevices];
+std::atomic<int> g_umma_opt_in[kMaxDevices][3];
 
+template <int R>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
-    auto kernel = mqa_decode_stream_umma_kernel;
+    auto kernel = mqa_decode_stream_umma_kernel<R>;
+    constexpr int kSlot = R == 4 ? 0 : (R == 2 ? 1 : 2);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
-    if (!g_umma_opt_in[dev].load(std::memory_order_acquire)) {
+    if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes) != cudaSuccess) {
             cudaGetLastError();
             return MQA_ERR_CUDA;
         }
-        g_umma_opt_in[dev].store(1, std::memory_order_release);
+        g_umma_opt_in[dev][kSlot].store(1, std::memory_order_release);
     }
     alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub, map_q;
     const long long rows = (long long)b * m_max;
     if (!encode_cache_map(&map_k, K, rows, kUmmaStageRows) || !encode_cache_map(&map_v, V, rows, kUmmaStageRows) ||
         !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows) ||
-        !encode_cache_map(&map_q, q, (long long)b * h, 64))
+        !encode_cache_map(&map_q, q, (long long)b * h, R == 4 ? 16 : (R == 2 ? 32 : ((h + 15) & ~15))))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, kUmmaSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
@@ -322,7 +324,11 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
-    if (p.kernel == Kernel::kUmma) return launch_umma(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+    if (p.kernel == Kernel::kUmma) {
+        if (h <= 16) return launch_umma<4>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+        if (h <= 32) return launch_umma<2>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+        return launch_umma<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+    }
     if (p.kernel == Kernel::kStream1)
         return launch_stream<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream2)

@@ -117,6 +117,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+// Bring a tensor map into the descriptor cache ahead of its first use by a copy.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -357,6 +361,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
     __shared__ int timed_out, issued;   // a wait ran out; tiles whose copies were started
 
+    if (warp == Cfg::kConsumerWarps && lane == 0) { prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); }
     if (threadIdx.x == 0) {
         timed_out = 0;
         issued = 0;
@@ -528,6 +533,10 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
     __shared__ int timed_out, issued;
 
+    if (warp == Cfg::kConsumerWarps && lane == 0) {
+        prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
+        prefetch_tensormap(&map_k_sub); prefetch_tensormap(&map_v_sub);
+    }
     if (threadIdx.x == 0) {
         timed_out = 0;
         issued = 0;
