@@ -370,7 +370,7 @@ def main():
         "gpu_launches": st.launches_per_step * args.steps,
         "clocks": r["clocks"],
     }
-    traffic = os.path.join(ROOT, "profiles", "traffic.json")
+    traffic = os.path.join(ROOT, "profiles", "traffic.txt")
     if os.path.exists(traffic):
         try:
             out["roofline"]["traffic"] = json.load(open(traffic)).get(w.name, {}).get("mqa_split_dram_bytes")
