@@ -4,7 +4,10 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
 One "step" is one pass of the whole hot path over one batch: the in-place append of the new
-token's key/value row, the split-m pass over the cache and the combine pass.  The headline
+token's key/value row, the split-m pass over the cache and the merge of the splits -- for the
+multi-query variant through mqa_decode_append_step (one kernel launch at the headline size), for
+the multi-head variant kv_cache_append + mha_decode_step.  The multi-query step as three separate
+launches is timed beside it.  The headline
 workload is the long-context configuration (b=32, h=32, k=v=128, 8192-row cache); the other
 workloads (`--workload`, `--sweep`) are the parity configurations and the bandwidth sweep.
 Prints ONE JSON line (rank 0).  `value` is achieved HBM GB/s of the multi-query step
@@ -128,7 +131,9 @@ class StepState:
         self.step_fn = mqa.mqa_decode_step if variant == "mqa" else mqa.mha_decode_step
         self.split_fn = mqa.mqa_decode_step_split if variant == "mqa" else mqa.mha_decode_step_split
         self.combine_fn = mqa.mqa_decode_step_combine if variant == "mqa" else mqa.mha_decode_step_combine
-        self.launches_per_step = 2 + (1 if self.n_splits > 1 else 0)
+        self.launches_three = 2 + (1 if self.n_splits > 1 else 0)
+        # the multi-query step is one call (append + attention + merge); multi-head is append + step
+        self.launches_per_step = mqa.append_step_launches(b, h, m) if variant == "mqa" else self.launches_three
         # pinned host copies of the per-step inputs / result for the end-to-end leg
         s0 = self.sets[0]
         self.host_in = [s0[n].cpu().pin_memory() for n in ("q", "k_new", "v_new")]
@@ -137,6 +142,15 @@ class StepState:
         self.d2h_bytes = self.host_o.numel() * 4
 
     def step(self, i):
+        s = self.sets[i % len(self.sets)]
+        if self.variant == "mqa":
+            self.mqa.mqa_decode_append_step(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, self.o,
+                                            self.ws, self.status, advance=False)
+        else:
+            self.step_separate(i)
+
+    def step_separate(self, i):
+        """The same step as separate calls: kv_cache_append, then the decode step (pass + second pass)."""
         s = self.sets[i % len(self.sets)]
         self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
         self.step_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
@@ -150,8 +164,7 @@ class StepState:
         s = self.sets[i % len(self.sets)]
         for name, src in zip(("q", "k_new", "v_new"), self.host_in):
             s[name].copy_(src, non_blocking=True)
-        self.append(s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, advance=False, status=self.status)
-        self.step_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
+        self.step(i)
         self.host_o.copy_(self.o, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the caller needs o before the next token
 
@@ -213,6 +226,17 @@ def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=T
     if sampler:
         sampler.__exit__()
     secs = statistics.median(regions)
+    # the same step as separate calls (append, pass over the cache, second pass)
+    sep_s = None
+    if st.variant == "mqa":
+        if use_graph:
+            g_sep = capture_graph(st.step_separate, steps)
+            g_sep.replay()
+            torch.cuda.synchronize(device)
+            run_sep = lambda _i: g_sep.replay()
+        else:
+            run_sep = st.step_separate
+        sep_s = statistics.median(time_region(run_sep, calls, device) for _ in range(max(3, min(20, len(regions)))))
     # per-launch duration of the pass over the cache (the dominant kernel): K back-to-back launches
     kernel_regions = [time_region(run_split, calls, device) for _ in range(max(3, min(20, len(regions))))]
     kernel_s = statistics.median(kernel_regions) / steps
@@ -221,7 +245,7 @@ def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=T
         st.step_e2e(i)
     e2e_s = time_region(st.step_e2e, steps, device)
     status = int(st.status.item())
-    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status,
+    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status, "separate_s": sep_s,
             "clocks": sampler.summary() if sampler else None, "first_region_s": regions[0],
             "min_region_s": min(regions), "regions": len(regions), "graph": bool(use_graph)}
 
@@ -297,6 +321,8 @@ def result_block(st, r, steps):
     return {"us_per_step": us, "gbs": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_step": st.bytes,
             "n_splits": st.n_splits, "chunk_rows": st.chunk_rows, "cache_sets": len(st.sets),
             "kernel_us": r["kernel_s"] * 1e6, "status": r["status"],
+            "separate_calls_us_per_step": None if r.get("separate_s") is None else r["separate_s"] / steps * 1e6,
+            "launches_per_step": st.launches_per_step,
             "first_region_us_per_step": r["first_region_s"] / steps * 1e6,
             "min_us_per_step": r["min_region_s"] / steps * 1e6, "regions": r["regions"], "cuda_graph": r["graph"]}
 

@@ -115,6 +115,30 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
                     int b, int h, int m_max, int k, int v, mqa_stream_t stream);
 
 /*
+ * mqa_decode_append_step -- one whole decoding step of the incremental multi-query function
+ * (Section 3) in a single call: the new token's key/value row is concatenated to each
+ * sequence's cache at row lens[b] (as kv_cache_append does), then the h heads attend over
+ * the lens[b] + 1 rows (as mqa_decode_step does).  For batches large enough for the persistent
+ * kernel and h <= 32 there is no separate append launch: the CTA that streams a sequence's last
+ * tile writes the new row just before it fetches that tile, and the second-pass kernel advances
+ * lens (two launches instead of three).  Other sizes run the same step as separate launches
+ * (h > 32 at large sizes: only with advance != 0, otherwise MQA_ERR_UNSUPPORTED).
+ *
+ *   q, k_new, v_new   [b, h, k], [b, k], [b, v] bf16
+ *   K, V              [b, m_max, k], [b, m_max, v] bf16, read-write (row lens[b] is written)
+ *   lens              [b] int32: rows valid BEFORE the call.  advance != 0: lens[b] += 1 on return
+ *                     (for sequences that took a row); advance == 0: lens is left as it was, although
+ *                     the row has been written and attended over.
+ *   o, workspace, workspace_bytes, status   as for mqa_decode_step.  A sequence with lens[b] == m_max
+ *                     (or negative) takes no new row: APPEND_CACHE_FULL (APPEND_NEGATIVE_LEN) is flagged
+ *                     and it attends over its existing rows.
+ * Results are those of kv_cache_append followed by mqa_decode_step on the same inputs.
+ */
+int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
+                           int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status,
+                           int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+
+/*
  * The two phases of a step, separately (mqa_decode_step == split then combine with the same
  * arguments; likewise mha).  They exist so that a caller can time or schedule the phases on
  * their own.  *_split runs the pass over the cache (Section 3 / 2.4 lines, per split) and
@@ -178,6 +202,13 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
 #define MQA_NOALLOC_SCRATCH_BYTES (8u * 1024u * 1024u)
 int mqa_decode_step_noalloc(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                             int32_t* status, int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+
+/*
+ * mqa_append_step_launches -- how many kernels one call of mqa_decode_append_step launches for these
+ * sizes on the current device when lens is advanced (0 for invalid arguments).  Informational;
+ * host-only.
+ */
+int mqa_append_step_launches(int b, int h, int m_max, int k, int v);
 
 /* mqa_status_string -- a static, human-readable name for a return code. */
 const char* mqa_status_string(int code);

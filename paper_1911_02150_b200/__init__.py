@@ -4,7 +4,7 @@ The product is the CUDA library ``libmqa_decode.so`` (C ABI: ``include/mqa_decod
 this package is its thin Python binding plus the seeded synthetic workloads.
 """
 from .binding import (  # noqa: F401
-    MqaError, alloc_workspace, kv_cache_append, lib, mha_decode_step, mha_decode_step_combine,
-    mha_decode_step_split, mqa_decode_step, mqa_decode_step_combine, mqa_decode_step_noalloc, mqa_decode_step_split, plan_splits,
+    MqaError, alloc_workspace, append_step_launches, kv_cache_append, lib, mha_decode_step, mha_decode_step_combine,
+    mha_decode_step_split, mqa_decode_step, mqa_decode_step_combine, mqa_decode_step_noalloc, mqa_decode_append_step, mqa_decode_step_split, plan_splits,
     status_string, workspace_bytes,
 )

@@ -26,6 +26,7 @@ EXPORTS = (
     "mqa_decode_step_split", "mqa_decode_step_combine",
     "mha_decode_step_split", "mha_decode_step_combine",
     "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string", "mqa_decode_step_noalloc",
+    "mqa_decode_append_step", "mqa_append_step_launches",
 )
 
 _lib = None
@@ -59,6 +60,10 @@ def lib() -> ctypes.CDLL:
             f.restype = I
         L.mqa_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, I, I, I, I, I, vp]
         L.mqa_decode_step_noalloc.restype = I
+        L.mqa_decode_append_step.argtypes = [vp, vp, vp, vp, vp, vp, I, vp, vp, sz, vp, I, I, I, I, I, vp]
+        L.mqa_decode_append_step.restype = I
+        L.mqa_append_step_launches.argtypes = [I, I, I, I, I]
+        L.mqa_append_step_launches.restype = I
         L.mqa_workspace_bytes.argtypes = [I, I, I, I, I]
         L.mqa_workspace_bytes.restype = sz
         L.mqa_plan_splits.argtypes = [I, I, I, I, I, I, ctypes.POINTER(I)]
@@ -75,6 +80,11 @@ def status_string(code: int) -> str:
 
 def workspace_bytes(b: int, h: int, m_max: int, k: int = 128, v: int = 128) -> int:
     return int(lib().mqa_workspace_bytes(b, h, m_max, k, v))
+
+
+def append_step_launches(b: int, h: int, m_max: int, k: int = 128, v: int = 128) -> int:
+    """Kernel launches of one :func:`mqa_decode_append_step` call at these sizes ."""
+    return int(lib().mqa_append_step_launches(b, h, m_max, k, v))
 
 
 def plan_splits(multi_query: bool, b: int, h: int, m_max: int, k: int = 128, v: int = 128):
@@ -214,4 +224,28 @@ def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
         rc = lib().mqa_decode_step_noalloc(_ptr(q), _ptr(K), _ptr(V), _ptr(lens), _ptr(o), _ptr(status),
                                            b, h, m_max, k, v, _stream(stream))
     _check(rc, "mqa_decode_step_noalloc")
+    return o
+
+
+def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None):
+    """One whole multi-query decoding step in one call: append ``k_new``/``v_new`` at row ``lens[b]`` of the
+    shared cache, then attend over ``lens[b] + 1`` rows; ``lens`` is advanced on the device when ``advance``.
+    For batches the persistent kernel serves (h <= 32) the append runs inside the pass over the cache."""
+    b, h, k = q.shape
+    m_max, v = K.shape[-2], V.shape[-1]
+    _need(q, torch.bfloat16, (b, h, k), "q")
+    _need(K, torch.bfloat16, (b, m_max, k), "K")
+    _need(V, torch.bfloat16, (b, m_max, v), "V")
+    _need(k_new, torch.bfloat16, (b, k), "k_new")
+    _need(v_new, torch.bfloat16, (b, v), "v_new")
+    _need(lens, torch.int32, (b,), "lens")
+    _need(o, torch.float32, (b, h, v), "o")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (_ptr(workspace), workspace.numel() * workspace.element_size())
+    with torch.cuda.device(q.device):
+        rc = lib().mqa_decode_append_step(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(lens),
+                                          int(bool(advance)), _ptr(o), ws_ptr, ws_bytes, _ptr(status),
+                                          b, h, m_max, k, v, _stream(stream))
+    _check(rc, "mqa_decode_append_step")
     return o

@@ -237,7 +237,7 @@ std::atomic<int> g_smem_opt_in[kMaxDevices][2];
 
 template <int M_TILES>
 int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-               float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
+               float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias) {
     using Cfg = MmaCfg<M_TILES>;
     auto kernel = mqa_decode_split_mma_kernel<M_TILES>;
     int dev = 0;
@@ -254,25 +254,34 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
         return MQA_ERR_CUDA;
     launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
                      static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
-                     p.n_splits);
+                     p.n_splits, len_bias);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
-std::atomic<int> g_stream_opt_in[kMaxDevices][2];
+std::atomic<int> g_stream_opt_in[kMaxDevices][4];
 
-template <int M_TILES>
+template <int M_TILES, bool FUSED>
 int launch_stream(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-                  void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
+                  void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream,
+                  const void* k_new = nullptr, const void* v_new = nullptr) {
     using Cfg = StreamCfg<M_TILES>;
-    auto kernel = mqa_decode_stream_mma_kernel<M_TILES>;
+    auto kernel = mqa_decode_stream_mma_kernel<M_TILES, FUSED>;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
-    if (!g_stream_opt_in[dev][M_TILES - 1].load(std::memory_order_acquire)) {
+    constexpr int kSlot = (M_TILES - 1) * 2 + (FUSED ? 1 : 0);
+    if (!g_stream_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
             cudaGetLastError();
             return MQA_ERR_CUDA;
         }
-        g_stream_opt_in[dev][M_TILES - 1].store(1, std::memory_order_release);
+        g_stream_opt_in[dev][kSlot].store(1, std::memory_order_release);
+    }
+    FusedArgs fa = {};
+    if (FUSED) {
+        fa.k_new = static_cast<const uint4*>(k_new);
+        fa.v_new = static_cast<const uint4*>(v_new);
+        fa.K = static_cast<uint4*>(const_cast<void*>(K));
+        fa.V = static_cast<uint4*>(const_cast<void*>(V));
     }
     alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub;
     const long long rows = (long long)b * m_max;
@@ -281,7 +290,7 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     launch_dependent(kernel, (unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
+                     static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max, fa);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -317,7 +326,7 @@ int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ER
 
 int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
               void* workspace, size_t workspace_bytes, int32_t* status,
-              int b, int h, int m_max, int k, int v, cudaStream_t stream) {
+              int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0) {
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
     const Plan p = make_plan(multi_query, b, h, m_max);
@@ -330,26 +339,27 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
         return launch_umma<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     }
     if (p.kernel == Kernel::kStream1)
-        return launch_stream<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+        return launch_stream<1, false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream2)
-        return launch_stream<2>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+        return launch_stream<2, false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     float2* part_ml = reinterpret_cast<float2*>(workspace);
     float* part_acc = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits))
                                 : nullptr;
     if (p.kernel == Kernel::kMma1)
-        return launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream);
+        return launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, len_bias);
     if (p.kernel == Kernel::kMma2)
-        return launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream);
+        return launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, len_bias);
     const unsigned grid = (unsigned)(p.units * (size_t)p.n_splits);
     launch_dependent(decode_split_simt_kernel, grid, kSimtThreads, 0, stream, static_cast<const uint4*>(q),
                      static_cast<const uint4*>(K), static_cast<const uint4*>(V), lens, o, part_ml, part_acc, status, h,
-                     multi_query ? h : 1, m_max, p.chunk_rows, p.n_splits);
+                     multi_query ? h : 1, m_max, p.chunk_rows, p.n_splits, len_bias);
     return launch_status();
 }
 
 int run_combine(bool multi_query, const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes,
-                int b, int h, int m_max, int k, int v, cudaStream_t stream) {
+                int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0,
+                int32_t* lens_advance = nullptr) {
     if (!lens || !o || !dims_ok(b, h, m_max) || !aligned16(o) || !aligned4(lens)) return MQA_ERR_INVALID_ARG;
     if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
     const Plan p = make_plan(multi_query, b, h, m_max);
@@ -358,7 +368,8 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     if (rc) return rc;
     if (p.stream()) {
         const StreamWorkspace w = stream_workspace(p, workspace);
-        launch_dependent(stream_combine_kernel, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h);
+        launch_dependent(stream_combine_kernel, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h,
+                         lens_advance, m_max);
         return launch_status();
     }
     if (p.n_splits <= 1) return MQA_OK;
@@ -366,7 +377,7 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits));
     launch_dependent(combine_splits_kernel, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens, o, h, m_max,
-                     p.chunk_rows, p.n_splits);
+                     p.chunk_rows, p.n_splits, len_bias);
     return launch_status();
 }
 
@@ -376,6 +387,14 @@ int run_step(bool multi_query, const void* q, const void* K, const void* V, cons
     int rc = run_split(multi_query, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream);
     if (rc) return rc;
     return run_combine(multi_query, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream);
+}
+
+// lens[i] += 1 for the sequences that took a row (the multi-launch form of mqa_decode_append_step
+// advances lens last, after the kernels that read the old value).
+__global__ void lens_advance_kernel(int32_t* lens, int b, int m_max) {
+    grid_dependency_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < b && lens[i] >= 0 && lens[i] < m_max) lens[i] += 1;
 }
 
 }  // namespace
@@ -439,11 +458,58 @@ int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace
                        static_cast<cudaStream_t>(stream));
 }
 
+int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
+                           int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
+                           int h, int m_max, int k, int v, mqa_stream_t stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
+    if (rc) return rc;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return MQA_ERR_INVALID_ARG;
+    const Plan p = make_plan(true, b, h, m_max);
+    if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
+    rc = check_workspace(p, workspace, workspace_bytes);
+    if (rc) return rc;
+    if (p.kernel == Kernel::kStream1 || p.kernel == Kernel::kStream2) {
+        rc = p.kernel == Kernel::kStream1
+                 ? launch_stream<1, true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new)
+                 : launch_stream<2, true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
+        if (rc) return rc;
+        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
+    }
+    // other plans: the same step as separate launches.  Without `advance` the append leaves lens alone and
+    // the step is told that a sequence which took a row has one more row than lens says.
+    if (p.stream()) {   // the tcgen05 plan reads lens as it stands: advance, step, and take the advance back
+        if (!advance) return MQA_ERR_UNSUPPORTED;
+        rc = kv_cache_append(K, V, k_new, v_new, lens, 1, status, b, 1, m_max, k, v, stream_);
+        if (rc) return rc;
+        return mqa_decode_step(q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream_);
+    }
+    rc = kv_cache_append(K, V, k_new, v_new, lens, 0, status, b, 1, m_max, k, v, stream_);
+    if (rc) return rc;
+    rc = run_split(true, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream, 1);
+    if (rc) return rc;
+    rc = run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 1);
+    if (rc) return rc;
+    if (advance) {
+        launch_dependent(lens_advance_kernel, (unsigned)((b + 255) / 256), 256u, 0, stream, lens, b, m_max);
+        return launch_status();
+    }
+    return MQA_OK;
+}
+
 size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
     const size_t a = plan_workspace_bytes(make_plan(true, b, h, m_max));
     const size_t c = plan_workspace_bytes(make_plan(false, b, h, m_max));
     return a > c ? a : c;
+}
+
+int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
+    if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
+    const Plan p = make_plan(true, b, h, m_max);
+    if (p.kernel == Kernel::kStream1 || p.kernel == Kernel::kStream2) return 2;   // pass with the append inside, second pass
+    if (p.stream()) return 3;                          // append, tcgen05 pass, second pass
+    return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }
 
 int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int* chunk_rows) {

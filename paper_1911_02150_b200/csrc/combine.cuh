@@ -23,11 +23,11 @@ __host__ __device__ inline size_t partial_acc_bytes(size_t units, int S) {
 __global__ void __launch_bounds__(kHeadDim)
 combine_splits_kernel(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
                       const int32_t* __restrict__ lens, float* __restrict__ o,
-                      int h, int m_max, int chunk_rows, int n_splits) {
+                      int h, int m_max, int chunk_rows, int n_splits, int len_bias) {
     const size_t u = blockIdx.x;
     const int c = threadIdx.x;
     grid_dependency_wait();          // the partials come from the kernel before this one
-    int L = lens[u / h];
+    int L = biased_len(lens[u / h], m_max, len_bias);
     L = L < 0 ? 0 : (L > m_max ? m_max : L);
     int live = (L + chunk_rows - 1) / chunk_rows;
     if (live > n_splits) live = n_splits;

@@ -48,4 +48,10 @@ __device__ __forceinline__ int clamp_len(int L, int m_max, int32_t* status) {
     return L;
 }
 
+// Rows to attend over when the caller's lens[] still holds the count from before this step's append
+// (bias = 1): a sequence that could take the new row (0 <= lens < m_max) has one more row than lens says.
+__device__ __forceinline__ int biased_len(int raw, int m_max, int bias) {
+    return (bias && raw >= 0 && raw < m_max) ? raw + 1 : raw;
+}
+
 }  // namespace mqa

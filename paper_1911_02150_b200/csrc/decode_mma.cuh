@@ -334,7 +334,7 @@ __global__ void __launch_bounds__(MmaCfg<M_TILES>::kThreads, MmaCfg<M_TILES>::kM
 mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                             float* __restrict__ o, float2* __restrict__ part_ml, float* __restrict__ part_acc,
-                            int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits) {
+                            int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias) {
     using Cfg = MmaCfg<M_TILES>;
     constexpr int kStages = Cfg::kStages;
     const int seq = blockIdx.x / n_splits;
@@ -343,7 +343,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
-    const int L = clamp_len(lens[seq], m_max, threadIdx.x == 0 ? status : nullptr);
+    const int L = clamp_len(biased_len(lens[seq], m_max, len_bias), m_max, threadIdx.x == 0 ? status : nullptr);
     const int r0 = split * chunk_rows;
     const int r1 = min(L, r0 + chunk_rows);
     if (r0 >= L) {                                         // nothing valid in this split (uniform)
@@ -511,14 +511,42 @@ __host__ __device__ inline size_t stream_ml_bytes(int slots, int h) {
 }
 __host__ __device__ inline size_t stream_acc_bytes(int slots, int h) { return (size_t)slots * h * kHeadDim * sizeof(float); }
 
-template <int M_TILES>
+// What the append-and-attend step (FUSED) does on top of the pass over the cache: the CTA whose share
+// holds a sequence's last tile writes the new token's key and value row (row lens[b]) into the cache
+// just before it fetches that tile, so the step attends over lens[b] + 1 rows without a separate
+// append launch.  lens itself is advanced by the second-pass kernel, when no CTA reads it any more.
+struct FusedArgs {
+    const uint4* k_new;      // [b, 128] bf16 rows as 16-byte words; null = nothing to append
+    const uint4* v_new;
+    uint4* K;                // the cache, written at row lens[b]
+    uint4* V;
+};
+
+// lens[s]; the append-and-attend step reads it with plain loads (the kernel after it writes lens).
+template <bool FUSED>
+__device__ __forceinline__ int read_len(const int32_t* lens, int s) {
+    if constexpr (FUSED) return *reinterpret_cast<const volatile int32_t*>(lens + s);
+    else return __ldg(lens + s);
+}
+
+// Rows of sequence s this launch attends over, and whether the step appends to it.
+__device__ __forceinline__ int fused_rows(int raw, int m_max, bool appending, bool* can_append) {
+    const bool ok = appending && raw >= 0 && raw < m_max;
+    if (can_append) *can_append = ok;
+    const int L = raw < 0 ? 0 : (raw > m_max ? m_max : raw);
+    return ok ? L + 1 : L;
+}
+
+template <int M_TILES, bool FUSED>
 __global__ void __launch_bounds__(StreamCfg<M_TILES>::kThreads, 1)
 mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                              const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
                              const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                              float* __restrict__ o, int2* __restrict__ seq_span, float2* __restrict__ part_ml,
-                             float* __restrict__ part_acc, int32_t* __restrict__ status, int b, int h, int m_max) {
+                             float* __restrict__ part_acc, int32_t* __restrict__ status, int b, int h, int m_max,
+                             const FusedArgs fa) {
     using Cfg = StreamCfg<M_TILES>;
+    const bool appending = FUSED && fa.k_new != nullptr;
     constexpr int kStages = Cfg::kStages;
     constexpr int kConsumerThreads = Cfg::kConsumerWarps * 32;
     const int cta = blockIdx.x, G = gridDim.x;
@@ -552,7 +580,12 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 
     // ---- 32-row sub-tiles per sequence and their running sum (every CTA computes the same table)
     for (int s = threadIdx.x; s < b; s += Cfg::kThreads) {
-        const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
+        const int raw = read_len<FUSED>(lens, s);
+        clamp_len(raw, m_max, cta == 0 ? status : nullptr);
+        bool can_append;
+        const int L = fused_rows(raw, m_max, appending, &can_append);
+        if (appending && !can_append && cta == 0 && status)
+            atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
         prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
         if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
             for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
@@ -595,41 +628,63 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 
     if (warp == Cfg::kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
-        if (lane == 0 && t_begin < t_end) {
+        // Lane 0 waits and issues the copies; the other lanes come along only to write the new row
+        // of a sequence (FUSED) before the tile that contains it is fetched.
+        if (t_begin < t_end && (lane == 0 || appending)) {
             bool ok = true;
             int s = s_first;
             int j = 0;                                     // stages issued by this CTA so far
             for (long long t = t_begin; t < t_end && ok;) {
                 while (prefix[s + 1] <= t) ++s;
                 const long long seg_end = min((long long)prefix[s + 1], t_end);
+                int new_row = -1;                          // row this step appends to sequence s
+                if (appending) {
+                    bool can_append;
+                    const int L = fused_rows(read_len<FUSED>(lens, s), m_max, true, &can_append);
+                    if (can_append) new_row = L - 1;
+                }
                 for (long long u = t; u < seg_end && ok; u += kRowWarps, ++j) {
                     const int nsub = (int)min((long long)kRowWarps, seg_end - u);
                     const int stg = j % kStages;
-                    if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
-                    if (!ok) break;
-                    const uint32_t bar = full_s + stg * 8;
-                    const uint32_t dst = stages_s + stg * kStreamStageBytes;
-                    mbar_expect_tx(bar, nsub * kStageBytes);
-                    const int y = s * m_max + (int)(u - prefix[s]) * kTileRows;
-                    if (nsub == kRowWarps) {
-                        tma_load_2d(dst, &map_k, 0, y, bar);
-                        tma_load_2d(dst + kStreamBoxBytes, &map_k, kBoxCols, y, bar);
-                        tma_load_2d(dst + 2 * kStreamBoxBytes, &map_v, 0, y, bar);
-                        tma_load_2d(dst + 3 * kStreamBoxBytes, &map_v, kBoxCols, y, bar);
-                    } else {
-                        for (int i = 0; i < nsub; ++i) {
-                            const uint32_t d = dst + i * kBoxBytes;
-                            tma_load_2d(d, &map_k_sub, 0, y + i * kTileRows, bar);
-                            tma_load_2d(d + kStreamBoxBytes, &map_k_sub, kBoxCols, y + i * kTileRows, bar);
-                            tma_load_2d(d + 2 * kStreamBoxBytes, &map_v_sub, 0, y + i * kTileRows, bar);
-                            tma_load_2d(d + 3 * kStreamBoxBytes, &map_v_sub, kBoxCols, y + i * kTileRows, bar);
+                    const int row_first = (int)(u - prefix[s]) * kTileRows;
+                    if (appending) {
+                        if (new_row >= row_first && new_row < row_first + nsub * kTileRows) {
+                            const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
+                            const size_t src = (size_t)s * (kRowBytes / 16) + (lane & 15);
+                            if (lane < 16) fa.K[dst] = fa.k_new[src]; else fa.V[dst] = fa.v_new[src];
+                            asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
+                        }
+                        __syncwarp();
+                    }
+                    if (lane == 0) {
+                        if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
+                        if (ok) {
+                            const uint32_t bar = full_s + stg * 8;
+                            const uint32_t dst = stages_s + stg * kStreamStageBytes;
+                            mbar_expect_tx(bar, nsub * kStageBytes);
+                            const int y = s * m_max + row_first;
+                            if (nsub == kRowWarps) {
+                                tma_load_2d(dst, &map_k, 0, y, bar);
+                                tma_load_2d(dst + kStreamBoxBytes, &map_k, kBoxCols, y, bar);
+                                tma_load_2d(dst + 2 * kStreamBoxBytes, &map_v, 0, y, bar);
+                                tma_load_2d(dst + 3 * kStreamBoxBytes, &map_v, kBoxCols, y, bar);
+                            } else {
+                                for (int i = 0; i < nsub; ++i) {
+                                    const uint32_t d = dst + i * kBoxBytes;
+                                    tma_load_2d(d, &map_k_sub, 0, y + i * kTileRows, bar);
+                                    tma_load_2d(d + kStreamBoxBytes, &map_k_sub, kBoxCols, y + i * kTileRows, bar);
+                                    tma_load_2d(d + 2 * kStreamBoxBytes, &map_v_sub, 0, y + i * kTileRows, bar);
+                                    tma_load_2d(d + 3 * kStreamBoxBytes, &map_v_sub, kBoxCols, y + i * kTileRows, bar);
+                                }
+                            }
+                            issued = j + 1;
                         }
                     }
-                    issued = j + 1;
+                    if (appending) ok = __shfl_sync(0xffffffffu, ok, 0);
                 }
                 t = seg_end;
             }
-            if (!ok) atomicExch(&timed_out, 1);
+            if (!ok && lane == 0) atomicExch(&timed_out, 1);
         }
     } else {
         // --------------------------------------------------------------- consumer warps
@@ -653,7 +708,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
             while (prefix[s + 1] <= t) ++s;
             const long long seg_end = min((long long)prefix[s + 1], t_end);
             const int first_row = (int)(t - prefix[s]) * kTileRows;
-            const int L = min(max(__ldg(lens + s), 0), m_max);
+            const int L = fused_rows(read_len<FUSED>(lens, s), m_max, appending, nullptr);
             const bool whole = (t == prefix[s]) && (seg_end == prefix[s + 1]);
 
             st.reset();
@@ -765,6 +820,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
             t = seg_end;
         }
         if (!ok) atomicExch(&timed_out, 1);
+
     }
 
     __syncthreads();
@@ -786,10 +842,15 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 // slot and is skipped.
 __global__ void __launch_bounds__(kHeadDim)
 stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restrict__ part_ml,
-                      const float* __restrict__ part_acc, float* __restrict__ o, int b, int h) {
+                      const float* __restrict__ part_acc, float* __restrict__ o, int b, int h,
+                      int32_t* lens_advance, int m_max) {
     const int s = blockIdx.x / h, head = blockIdx.x % h;
     const int c = threadIdx.x;
     grid_dependency_wait();          // the slots come from the kernel before this one
+    if (lens_advance && head == 0 && c == 0) {       // append-and-attend step: lens[s] += 1 for a sequence that took a row
+        const int raw = lens_advance[s];
+        if (raw >= 0 && raw < m_max) lens_advance[s] = raw + 1;
+    }
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
     __shared__ float w_s[256], l_s[256];

@@ -27,7 +27,7 @@ decode_split_simt_kernel(const uint4* __restrict__ q, const uint4* __restrict__ 
                          const uint4* __restrict__ V, const int32_t* __restrict__ lens,
                          float* __restrict__ o, float2* __restrict__ part_ml,
                          float* __restrict__ part_acc, int32_t* __restrict__ status,
-                         int h, int heads_per_cache, int m_max, int chunk_rows, int n_splits) {
+                         int h, int heads_per_cache, int m_max, int chunk_rows, int n_splits, int len_bias) {
     const size_t u = blockIdx.x / n_splits;            // unit = sequence * h + head
     const int split = blockIdx.x % n_splits;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -35,7 +35,7 @@ decode_split_simt_kernel(const uint4* __restrict__ q, const uint4* __restrict__ 
 
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
-    const int L = clamp_len(lens[u / h], m_max, threadIdx.x == 0 ? status : nullptr);
+    const int L = clamp_len(biased_len(lens[u / h], m_max, len_bias), m_max, threadIdx.x == 0 ? status : nullptr);
     const int r0 = split * chunk_rows;
     const int r1 = min(L, r0 + chunk_rows);
     if (r0 >= L) {                                     // nothing valid in this split

@@ -1,0 +1,131 @@
+"""mqa_decode_append_step (append + attention + merge in one call, one kernel launch for large
+batches) against the oracle: oracle append, then oracle multi-query step on the grown cache."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1911_02150_b200 as mqa
+from paper_1911_02150_b200 import binding, workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+ABS_TOL, REL_TOL = 4e-3, 1e-2
+
+
+def check_close(got, ref, what):
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    err = np.abs(got.astype(np.float64) - ref)
+    assert err.max() <= ABS_TOL, f"{what}: max abs err {err.max():.3e}"
+    assert np.all(err.max(-1) <= REL_TOL * np.abs(ref).max(-1)), f"{what}: row-relative error"
+
+
+def run(b, h, m_max, lens0, advance, seed):
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=seed, device=DEV)
+    lens0 = np.asarray(lens0, np.int32)
+    wl.poison_tail(inp["K"], np.clip(lens0, 0, m_max))
+    wl.poison_tail(inp["V"], np.clip(lens0, 0, m_max))
+    Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
+    skipped = oracle.kv_cache_append(Kh, Vh, wl.bits(inp["k_new"]), wl.bits(inp["v_new"]), lens_h, True)
+    ref = oracle.mqa_decode_step(wl.bits(inp["q"]), Kh, Vh, lens_h)
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    ws.fill_(0xFF)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws, status,
+                               advance=advance)
+    torch.cuda.synchronize()
+    check_close(o.cpu().numpy(), ref, f"append_step b={b} h={h} m_max={m_max}")
+    assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)   # the append, bit for bit
+    assert np.array_equal(lens_t.cpu().numpy(), lens_h if advance else lens0)
+    want_status = 0
+    if (lens0 >= m_max).any():
+        want_status |= binding.STATUS_APPEND_CACHE_FULL
+    if (lens0 < 0).any():
+        want_status |= binding.STATUS_APPEND_NEGATIVE_LEN | binding.STATUS_LEN_CLAMPED
+    assert int(status.item()) == want_status, (int(status.item()), want_status, skipped)
+    return inp, o
+
+
+def lens_mix(b, m_max, seed):
+    r = np.random.default_rng(seed)
+    lens = r.integers(0, m_max, size=b).astype(np.int32)
+    lens[r.integers(0, b, size=max(1, b // 8))] = 0          # first token of a sequence
+    lens[r.integers(0, b, size=max(1, b // 8))] = m_max - 1  # fills the cache
+    return lens
+
+
+CASES = [
+    # b, h, m_max: plans with the append inside the pass (persistent mma.sync kernel) ...
+    (40, 16, 1500), (160, 32, 333), (300, 8, 200), (37, 32, 4000), (64, 5, 777),
+    # ... and plans that run as separate launches (small batch; tcgen05 plan for h > 32 with advance)
+    (4, 8, 300), (1, 16, 20000), (2, 40, 600),
+]
+
+
+@pytest.mark.parametrize("advance", [True, False])
+@pytest.mark.parametrize("b,h,m_max", CASES)
+def test_append_step_matches_oracle(b, h, m_max, advance):
+    run(b, h, m_max, lens_mix(b, m_max, seed=b + h), advance, seed=b * 7 + h)
+
+
+def test_append_step_full_and_negative_sequences_take_no_row():
+    b, h, m_max = 48, 16, 1024
+    lens = lens_mix(b, m_max, seed=5)
+    lens[3] = m_max          # full: no row, attends over m_max rows
+    lens[7] = -2             # negative: no row, empty prefix -> zeros
+    run(b, h, m_max, lens, True, seed=77)
+
+
+def test_append_step_tcgen05_plan_needs_advance():
+    b, h, m_max = 40, 48, 1500           # persistent tcgen05 plan
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=9, device=DEV)
+    lens_np = lens_mix(b, m_max, seed=9)
+    run(b, h, m_max, lens_np, True, seed=9)
+    lens_t = torch.from_numpy(lens_np).to(DEV)
+    o = torch.zeros(b, h, 128, dtype=torch.float32, device=DEV)
+    with pytest.raises(mqa.MqaError) as e:
+        mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o,
+                                   mqa.alloc_workspace(b, h, m_max, DEV), advance=False)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+
+
+def test_incremental_decoding_with_append_steps():
+    """A decoding loop of 40 steps on a batch large enough for the persistent kernel (append inside the pass): every step's
+    output against the oracle on the cache as it then stands, and two runs bit-identical."""
+    b, h, m_max, steps = 96, 16, 512, 40
+    gen = torch.Generator(device=DEV)
+    outs = []
+    for rep in range(2):
+        gen.manual_seed(321)
+        K = torch.zeros(b, m_max, 128, dtype=torch.bfloat16, device=DEV)
+        V = torch.zeros_like(K)
+        nan = torch.tensor(wl.NAN_BITS, dtype=torch.int16, device=DEV)
+        K.view(torch.int16).fill_(nan); V.view(torch.int16).fill_(nan)
+        start = np.random.default_rng(3).integers(380, 470, size=b).astype(np.int32)     # prefill of different lengths
+        for s in range(b):
+            K[s, : start[s]] = wl.bf16_normal((int(start[s]), 128), 1.0, gen, DEV)
+            V[s, : start[s]] = wl.bf16_normal((int(start[s]), 128), 1.0, gen, DEV)
+        lens_t = torch.from_numpy(start.copy()).to(DEV)
+        ws = mqa.alloc_workspace(b, h, m_max, DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        run_outs, qs = [], []
+        for t in range(steps):
+            q = wl.bf16_normal((b, h, 128), 128 ** -0.5, gen, DEV)
+            k_new = wl.bf16_normal((b, 128), 1.0, gen, DEV)
+            v_new = wl.bf16_normal((b, 128), 1.0, gen, DEV)
+            o = torch.empty(b, h, 128, dtype=torch.float32, device=DEV)
+            mqa.mqa_decode_append_step(q, K, V, k_new, v_new, lens_t, o, ws, status)
+            run_outs.append(o); qs.append(q)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.array_equal(lens_t.cpu().numpy(), start + steps)
+        outs.append(run_outs)
+        if rep == 0:
+            Kb, Vb = wl.bits(K), wl.bits(V)
+            for t in (0, 1, 17, steps - 1):
+                ref = oracle.mqa_decode_step(wl.bits(qs[t]), Kb, Vb, (start + t + 1).astype(np.int32))
+                check_close(run_outs[t].cpu().numpy(), ref, f"step {t}")
+    for a, c in zip(*outs):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
