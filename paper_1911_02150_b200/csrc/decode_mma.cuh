@@ -494,9 +494,40 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 // line every step moves to the next CTA, the next sequence, or both, so that sum never repeats
 // -- and the second-pass kernel merges the slots of each sequence that was cut.
 // =============================================================================================
-struct StreamWork {
-    long long total;      // T
-    long long begin, end; // this CTA's tiles
+// Crossing from one sequence to the next inside a share is not free (the row-warps are merged, a
+// partial or the result is written, the next sequence's Q is fetched), so the line carries, in front
+// of each sequence's tiles, kBoundaryPenalty virtual tiles that cost nothing to "process": a CTA
+// whose share contains a crossing gets that many fewer real tiles, and all CTAs finish together.
+constexpr int kBoundaryPenalty = 8;
+
+// A run of 32-row tiles [lo, hi) of sequence s inside one CTA's share.
+struct Segment {
+    int s, lo, hi;
+    bool whole;           // the share holds every tile of the sequence: it writes the final o
+};
+
+// Walks one CTA's share [t, t_end) of the line.  prefix[s] = position of sequence s's block (its penalty
+// tiles, then its real tiles); sequences without rows have no block.
+struct ShareWalker {
+    const int* prefix;
+    long long t, t_end;
+    int s;
+    __device__ __forceinline__ bool next(Segment& g) {
+        while (t < t_end) {
+            while (prefix[s + 1] <= t) ++s;
+            const long long v0 = prefix[s], v1 = prefix[s + 1];
+            const int n = (int)(v1 - v0) - kBoundaryPenalty;                    // real tiles, >= 1
+            const long long end = v1 < t_end ? v1 : t_end;
+            const long long lo = t - v0 - kBoundaryPenalty, hi = end - v0 - kBoundaryPenalty;
+            t = end;
+            g.s = s;
+            g.lo = lo > 0 ? (int)lo : 0;
+            g.hi = hi < n ? (int)hi : n;
+            g.whole = g.lo == 0 && g.hi == n;
+            if (g.hi > g.lo) return true;
+        }
+        return false;
+    }
 };
 
 // cta that owns global tile t when T tiles are cut into G shares [c*T/G, (c+1)*T/G)
@@ -586,7 +617,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         const int L = fused_rows(raw, m_max, appending, &can_append);
         if (appending && !can_append && cta == 0 && status)
             atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
-        prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
+        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
         if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
             for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
         }
@@ -632,21 +663,21 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         // of a sequence (FUSED) before the tile that contains it is fetched.
         if (t_begin < t_end && (lane == 0 || appending)) {
             bool ok = true;
-            int s = s_first;
             int j = 0;                                     // stages issued by this CTA so far
-            for (long long t = t_begin; t < t_end && ok;) {
-                while (prefix[s + 1] <= t) ++s;
-                const long long seg_end = min((long long)prefix[s + 1], t_end);
+            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            Segment g;
+            while (ok && walk.next(g)) {
+                const int s = g.s;
                 int new_row = -1;                          // row this step appends to sequence s
                 if (appending) {
                     bool can_append;
                     const int L = fused_rows(read_len<FUSED>(lens, s), m_max, true, &can_append);
                     if (can_append) new_row = L - 1;
                 }
-                for (long long u = t; u < seg_end && ok; u += kRowWarps, ++j) {
-                    const int nsub = (int)min((long long)kRowWarps, seg_end - u);
+                for (int u = g.lo; u < g.hi && ok; u += kRowWarps, ++j) {
+                    const int nsub = min(kRowWarps, g.hi - u);
                     const int stg = j % kStages;
-                    const int row_first = (int)(u - prefix[s]) * kTileRows;
+                    const int row_first = u * kTileRows;
                     if (appending) {
                         if (new_row >= row_first && new_row < row_first + nsub * kTileRows) {
                             const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
@@ -682,7 +713,6 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                     }
                     if (appending) ok = __shfl_sync(0xffffffffu, ok, 0);
                 }
-                t = seg_end;
             }
             if (!ok && lane == 0) atomicExch(&timed_out, 1);
         }
@@ -691,7 +721,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         // which CTAs hold pieces of each sequence (read by the second pass); spread over the CTAs
         if (warp == 0) {
             for (int s = cta + lane * G; s < b; s += G * 32) {
-                const int t0 = prefix[s], t1 = prefix[s + 1];
+                const int t0 = prefix[s] + kBoundaryPenalty, t1 = prefix[s + 1];     // its real tiles on the line
                 seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
             }
             if (cta == 0 && lane == 0) seq_span[b] = make_int2((int)T, G);
@@ -703,24 +733,24 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         float* my_buf = merge_buf + mt * Cfg::kStateFloats * 32;
         bool ok = true;
         int j = 0;                                         // stages consumed by this CTA so far
-        int s = s_first;
-        for (long long t = t_begin; t < t_end;) {
-            while (prefix[s + 1] <= t) ++s;
-            const long long seg_end = min((long long)prefix[s + 1], t_end);
-            const int first_row = (int)(t - prefix[s]) * kTileRows;
+        ShareWalker walk{prefix, t_begin, t_end, s_first};
+        Segment g_;
+        while (walk.next(g_)) {
+            const int s = g_.s;
             const int L = fused_rows(read_len<FUSED>(lens, s), m_max, appending, nullptr);
-            const bool whole = (t == prefix[s]) && (seg_end == prefix[s + 1]);
+            const bool whole = g_.whole;
+            const bool last_segment = walk.t >= t_end;     // (a later block could only add penalty tiles)
 
             st.reset();
             uint32_t qa[8][4];
             load_q_fragments(qa, q, (size_t)s, h, mt, lane);
-            for (long long u = t; u < seg_end; u += kRowWarps, ++j) {
-                const int nsub = (int)min((long long)kRowWarps, seg_end - u);
+            for (int u = g_.lo; u < g_.hi; u += kRowWarps, ++j) {
+                const int nsub = min(kRowWarps, g_.hi - u);
                 const int stg = j % kStages;
                 if (ok) ok = mbar_wait(full_s + stg * 8, (j / kStages) & 1);
                 if (ok && rw < nsub) {                     // row-warp rw takes sub-tile rw of the stage
                     const uint32_t k_s = stages_s + stg * kStreamStageBytes + rw * kBoxBytes;
-                    const int row0 = first_row + ((int)(u - t) + rw) * kTileRows;
+                    const int row0 = (u + rw) * kTileRows;
                     if (L >= kSingleRoundingMinRows)
                         consume_tile<false, kStreamBoxBytes>(st, qa, off, k_s, k_s + 2 * kStreamBoxBytes, row0, L, lane);
                     else
@@ -736,7 +766,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
             }
             const int head0 = mt * 16 + g, head1 = head0 + 8;
             const size_t slot = (size_t)cta + s;
-            if (seg_end == t_end) {
+            if (last_segment) {
                 // Last segment of this CTA: nothing is in flight any more, so the stage memory is
                 // free.  Every row-warp parks its state there and all consumer threads merge in
                 // parallel, each taking a quarter of its own fragment columns.
@@ -817,10 +847,8 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                     }
                 }
             }
-            t = seg_end;
         }
         if (!ok) atomicExch(&timed_out, 1);
-
     }
 
     __syncthreads();

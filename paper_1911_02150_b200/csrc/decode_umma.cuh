@@ -202,7 +202,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     // ---- 32-row sub-tiles per sequence and their running sum (as in the mma.sync persistent kernel)
     for (int s = threadIdx.x; s < b; s += kUmmaThreads) {
         const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
-        prefix[s + 1] = (L + kTileRows - 1) / kTileRows;
+        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
         if (L == 0 && s % G == cta)
             for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
     }
@@ -254,10 +254,11 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // =============================================================== TMA producer
         if (lane == 0 && t_begin < t_end) {
             bool ok = true;
-            int s = s_first, j = 0, seg = 0;
-            for (long long t = t_begin; t < t_end && ok; ++seg) {
-                while (prefix[s + 1] <= t) ++s;
-                const long long seg_end = min((long long)prefix[s + 1], t_end);
+            int j = 0, seg = 0;
+            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            Segment g;
+            for (; ok && walk.next(g); ++seg) {
+                const int s = g.s;
                 const int qi = seg & 1;
                 if (seg >= 2) ok = mbar_wait(q_empty + qi * 8, ((seg >> 1) - 1) & 1);
                 if (!ok) break;
@@ -268,15 +269,15 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     tma_load_2d(d, &map_q, 0, s * h, q_full + qi * 8);
                     tma_load_2d(d + kUmmaQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
                 }
-                for (long long u = t; u < seg_end && ok; u += kSubs, ++j) {
-                    const int nsub = (int)min((long long)kSubs, seg_end - u);
+                for (int u = g.lo; u < g.hi && ok; u += kSubs, ++j) {
+                    const int nsub = min(kSubs, g.hi - u);
                     const int stg = j % kUmmaStages;
                     if (j >= kUmmaStages) ok = mbar_wait(kv_empty + stg * 8, ((j / kUmmaStages) - 1) & 1);
                     if (!ok) break;
                     const uint32_t bar = kv_full + stg * 8;
                     const uint32_t dst = stages_s + stg * kUmmaStageBytes;
                     mbar_expect_tx(bar, nsub * kStageBytes);
-                    const int y = s * m_max + (int)(u - prefix[s]) * kTileRows;
+                    const int y = s * m_max + u * kTileRows;
                     if (nsub == kSubs) {
                         tma_load_2d(dst, &map_k, 0, y, bar);
                         tma_load_2d(dst + kUmmaBoxBytes, &map_k, kBoxCols, y, bar);
@@ -290,7 +291,6 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     }
                     issued = j + 1;
                 }
-                t = seg_end;
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
@@ -321,15 +321,15 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 tc_commit(kv_empty + (jj % kUmmaStages) * 8);       // the stage's K and V are free again
                 tc_commit(pv_done + pb * 8);                        // this P buffer is free, O is up to date
             };
-            int s = s_first, j = 0, seg = 0;
+            int j = 0, seg = 0;
             bool prev_first = false;
             int prev_seg = 0;
-            for (long long t = t_begin; t < t_end; ++seg) {
-                while (prefix[s + 1] <= t) ++s;
-                const long long seg_end = min((long long)prefix[s + 1], t_end);
+            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            Segment g;
+            for (; walk.next(g); ++seg) {
                 const int qi = seg & 1;
                 if (ok) ok = mbar_wait(q_full + qi * 8, (seg >> 1) & 1);
-                for (long long u = t; u < seg_end; u += kSubs, ++j) {
+                for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
                     const int stg = j % kUmmaStages, sb = j & 1;
                     if (ok) ok = mbar_wait(kv_full + stg * 8, (j / kUmmaStages) & 1);
                     if (ok && j >= 2) ok = mbar_wait(s_free + sb * 8, ((j >> 1) - 1) & 1);
@@ -344,12 +344,11 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         }
                     }
                     tc_commit(s_ready + sb * 8);
-                    if (u + kSubs >= seg_end) tc_commit(q_empty + qi * 8);   // last use of this segment's Q
+                    if (u + kSubs >= g.hi) tc_commit(q_empty + qi * 8);   // last use of this segment's Q
                     if (j > 0) issue_pv(j - 1, prev_first, prev_seg);
-                    prev_first = (u == t);
+                    prev_first = (u == g.lo);
                     prev_seg = seg;
                 }
-                t = seg_end;
             }
             if (j > 0) issue_pv(j - 1, prev_first, prev_seg);
             if (!ok) atomicExch(&timed_out, 1);
@@ -358,7 +357,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // =============================================================== softmax warps
         if (warp == 0) {                                    // second-pass bookkeeping, spread over the CTAs
             for (int s = cta + lane * G; s < b; s += G * 32) {
-                const int t0 = prefix[s], t1 = prefix[s + 1];
+                const int t0 = prefix[s] + kBoundaryPenalty, t1 = prefix[s + 1];     // its real tiles on the line
                 seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
             }
             if (cta == 0 && lane == 0) seq_span[b] = make_int2((int)T, G);
@@ -371,20 +370,20 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
             const int sm_threads = n_sm_warps * 32, sm_tid = warp * 32 + lane;
                         bool ok = true;
-            int s = s_first, j = 0, seg = 0;
-            for (long long t = t_begin; t < t_end; ++seg) {
-                while (prefix[s + 1] <= t) ++s;
-                const long long seg_end = min((long long)prefix[s + 1], t_end);
-                const int first_row = (int)(t - prefix[s]) * kTileRows;
+            int j = 0, seg = 0;
+            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            Segment g;
+            for (; walk.next(g); ++seg) {
+                const int s = g.s;
                 const int L = min(max(__ldg(lens + s), 0), m_max);
-                const bool whole = (t == prefix[s]) && (seg_end == prefix[s + 1]);
+                const bool whole = g.whole;
                 float m_run = -INFINITY, l_run = 0.f;
-                for (long long u = t; u < seg_end; u += kSubs, ++j) {
+                for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
                     const int sb = j & 1, stg = j % kUmmaStages;
                     // rows of this stage that count: what was fetched (the share may end mid-stage) and
                     // lies inside the prefix; always >= 1
-                    const int fetched = (int)min((long long)kSubs, seg_end - u) * kTileRows;
-                    const int valid = min(fetched, L - (first_row + (int)(u - t) * kTileRows));
+                    const int fetched = min(kSubs, g.hi - u) * kTileRows;
+                    const int valid = min(fetched, L - u * kTileRows);
                     if (ok) ok = mbar_wait(s_ready + sb * 8, (j >> 1) & 1);
                     tc_fence_after();
                     uint32_t r[kCpr];
@@ -402,7 +401,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     // are all beyond the prefix keeps its state.
                     const float m_new = fmaxf(m_run, __fmul_rn(top, kLog2e));
                     const float rescale = m_new == -INFINITY ? 1.f : fast_exp2(m_run - m_new);   // 0 on a copy's first columns
-                    const bool moved = live && m_new > m_run && u != t;      // O holds something to rescale
+                    const bool moved = live && m_new > m_run && u != g.lo;   // O holds something to rescale
                     l_run *= rescale;
                     m_run = m_new;
                     // ---- P = exp2(S - max) as bf16 hi + lo pairs (two cache rows per 32-bit TMEM column)
@@ -518,7 +517,6 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(o_free);         // the next segment may overwrite O
-                t = seg_end;
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
