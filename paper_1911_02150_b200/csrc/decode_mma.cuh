@@ -498,7 +498,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 // partial or the result is written, the next sequence's Q is fetched), so the line carries, in front
 // of each sequence's tiles, kBoundaryPenalty virtual tiles that cost nothing to "process": a CTA
 // whose share contains a crossing gets that many fewer real tiles, and all CTAs finish together.
-constexpr int kBoundaryPenalty = 8;
+constexpr int kBoundaryPenalty = 12;
 
 // A run of 32-row tiles [lo, hi) of sequence s inside one CTA's share.
 struct Segment {
