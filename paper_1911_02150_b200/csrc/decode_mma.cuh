@@ -659,9 +659,9 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 
     if (warp == Cfg::kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
-        // Lane 0 waits and issues the copies; the other lanes come along only to write the new row
-        // of a sequence (FUSED) before the tile that contains it is fetched.
-        if (t_begin < t_end && (lane == 0 || appending)) {
+        // One thread waits and issues the copies; in the append-and-attend step it also writes the new
+        // row of a sequence (512 bytes) before the tile that contains it is fetched.
+        if (t_begin < t_end && lane == 0) {
             bool ok = true;
             int j = 0;                                     // stages issued by this CTA so far
             ShareWalker walk{prefix, t_begin, t_end, s_first};
@@ -678,16 +678,17 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                     const int nsub = min(kRowWarps, g.hi - u);
                     const int stg = j % kStages;
                     const int row_first = u * kTileRows;
-                    if (appending) {
-                        if (new_row >= row_first && new_row < row_first + nsub * kTileRows) {
-                            const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
-                            const size_t src = (size_t)s * (kRowBytes / 16) + (lane & 15);
-                            if (lane < 16) fa.K[dst] = fa.k_new[src]; else fa.V[dst] = fa.v_new[src];
-                            asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
-                        }
-                        __syncwarp();
+                    if (appending && new_row >= row_first && new_row < row_first + nsub * kTileRows) {
+                        const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16);
+                        const size_t src = (size_t)s * (kRowBytes / 16);
+                        uint4 kr[16], vr[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { kr[i] = fa.k_new[src + i]; vr[i] = fa.v_new[src + i]; }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { fa.K[dst + i] = kr[i]; fa.V[dst + i] = vr[i]; }
+                        asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
                     }
-                    if (lane == 0) {
+                    {
                         if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
                         if (ok) {
                             const uint32_t bar = full_s + stg * 8;
@@ -711,10 +712,9 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                             issued = j + 1;
                         }
                     }
-                    if (appending) ok = __shfl_sync(0xffffffffu, ok, 0);
                 }
             }
-            if (!ok && lane == 0) atomicExch(&timed_out, 1);
+            if (!ok) atomicExch(&timed_out, 1);
         }
     } else {
         // --------------------------------------------------------------- consumer warps
