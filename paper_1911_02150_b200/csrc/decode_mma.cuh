@@ -881,41 +881,45 @@ stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restric
     }
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
-    __shared__ float w_s[256], l_s[256];
-    __shared__ int slot_s[256], n_s;
+    __shared__ float m_s[256], l_s[256];
     const int n_cta = span.y - span.x + 1;              // at most the grid of the first pass (<= 256 SMs)
     const long long T = seq_span[b].x, G = seq_span[b].y;
-    // every candidate CTA's (max, sum) is fetched by its own thread: one round trip for all of them
+    // One round trip for everything this CTA needs: each candidate piece's (max, sum) is fetched by its own
+    // thread, and every thread fetches its column of the first pieces' accumulators at the same time (their
+    // addresses do not depend on the weights).  A CTA whose share of the line is empty wrote no slot: its
+    // max is taken as -inf, which makes its weight exactly zero and its (unwritten) slot is never used.
+    constexpr int kEager = 8;
+    float a[kEager];
+    const float* col = part_acc + ((size_t)span.x + s) * h * kHeadDim + (size_t)head * kHeadDim + c;
+#pragma unroll
+    for (int i = 0; i < kEager; ++i) a[i] = i < n_cta ? __ldcg(col + (size_t)i * h * kHeadDim) : 0.f;
     for (int i = c; i < n_cta; i += kHeadDim) {
         const long long cta = span.x + i;
         const bool live = cta * T / G != (cta + 1) * T / G;
-        const float2 ml = live ? part_ml[((size_t)cta + s) * h + head] : make_float2(-INFINITY, 0.f);
-        w_s[i] = ml.x;
+        const float2 ml = live ? __ldcg(part_ml + ((size_t)cta + s) * h + head) : make_float2(-INFINITY, 0.f);
+        m_s[i] = ml.x;
         l_s[i] = ml.y;
     }
     __syncthreads();
     float top = -INFINITY;
-    for (int i = 0; i < n_cta; ++i) top = fmaxf(top, w_s[i]);
-    __syncthreads();
-    if (c == 0) {                                       // compact the live pieces, in order
-        int n = 0;
-        for (int i = 0; i < n_cta; ++i) {
-            if (w_s[i] == -INFINITY) continue;
-            w_s[n] = fast_exp2(w_s[i] - top);
-            l_s[n] = l_s[i];
-            slot_s[n] = span.x + i + s;
-            ++n;
-        }
-        n_s = n;
-    }
-    __syncthreads();
-    const int n = n_s;
+    for (int i = 0; i < n_cta; ++i) top = fmaxf(top, m_s[i]);
     float num = 0.f, den = 0.f;
-    const float* col = part_acc + (size_t)head * kHeadDim + c;
-#pragma unroll 4
-    for (int i = 0; i < n; ++i) {
-        den = fmaf(w_s[i], l_s[i], den);
-        num = fmaf(w_s[i], col[(size_t)slot_s[i] * h * kHeadDim], num);
+#pragma unroll
+    for (int i = 0; i < kEager; ++i) {
+        if (i < n_cta) {
+            const float w = fast_exp2(m_s[i] - top);
+            if (w != 0.f) {                                  // never multiply an unwritten slot
+                den = fmaf(w, l_s[i], den);
+                num = fmaf(w, a[i], num);
+            }
+        }
+    }
+    for (int i = kEager; i < n_cta; ++i) {
+        const float w = fast_exp2(m_s[i] - top);
+        if (w != 0.f) {
+            den = fmaf(w, l_s[i], den);
+            num = fmaf(w, __ldcg(col + (size_t)i * h * kHeadDim), num);
+        }
     }
     o[((size_t)s * h + head) * kHeadDim + c] = num / den;
 }
