@@ -64,6 +64,7 @@ Plan plan_simt(int b, int h, int m_max) {
     long want = (target_ctas + (long)p.units - 1) / (long)p.units;
     const long cap = m_max / 256 > 1 ? m_max / 256 : 1;
     if (want > cap) want = cap;
+    if (want > 1024) want = 1024;                 // the second pass keeps one (max, sum) per split in shared memory
     if (want < 1) want = 1;
     int chunk = (int)((m_max + want - 1) / want);
     chunk = (chunk + 63) / 64 * 64;
@@ -368,16 +369,24 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     if (rc) return rc;
     if (p.stream()) {
         const StreamWorkspace w = stream_workspace(p, workspace);
-        launch_dependent(stream_combine_kernel, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h,
-                         lens_advance, m_max);
+        if (p.n_splits <= kCombineEager)
+            launch_dependent(stream_combine_kernel<1>, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
+                             b, h, lens_advance, m_max);
+        else
+            launch_dependent(stream_combine_kernel<4>, (unsigned)((size_t)b * h), 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc,
+                             o, b, h, lens_advance, m_max);
         return launch_status();
     }
     if (p.n_splits <= 1) return MQA_OK;
     const float2* part_ml = reinterpret_cast<const float2*>(workspace);
     const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits));
-    launch_dependent(combine_splits_kernel, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens, o, h, m_max,
-                     p.chunk_rows, p.n_splits, len_bias);
+    if (p.n_splits <= kCombineEager)
+        launch_dependent(combine_splits_kernel<1>, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens, o, h,
+                         m_max, p.chunk_rows, p.n_splits, len_bias);
+    else
+        launch_dependent(combine_splits_kernel<4>, (unsigned)p.units, 4 * kHeadDim, 0, stream, part_ml, part_acc, lens, o, h,
+                         m_max, p.chunk_rows, p.n_splits, len_bias);
     return launch_status();
 }
 

@@ -3,7 +3,7 @@
 //     o = sum_s e^{M_s - M} acc_s / sum_s e^{M_s - M} l_s,
 // (maxima are stored multiplied by log2(e), so each weight is one exp2 of a difference)
 // the same softmax re-associated; splits that start at or beyond lens[b] hold nothing and are
-// skipped.  One CTA of 128 threads per (sequence, head): thread c owns output column c.
+// skipped.  One CTA per (sequence, head).
 #pragma once
 #include "common.cuh"
 
@@ -20,33 +20,88 @@ __host__ __device__ inline size_t partial_acc_bytes(size_t units, int S) {
     return units * (size_t)S * kHeadDim * sizeof(float);
 }
 
-__global__ void __launch_bounds__(kHeadDim)
+// Threads: 128 columns x GROUPS piece groups.  Group g takes pieces g, g + GROUPS, ...;
+// a thread fetches its column of up to kCombineEager of them in one go (the addresses do not depend
+// on the weights), so merging a few dozen pieces costs one round trip to L2, not one per piece.
+// The host picks GROUPS = 1 (128 threads) when no sequence can have more than kCombineEager pieces,
+// else 4 (512 threads).
+constexpr int kCombineEager = 8;
+
+// Merge `n` pieces of one (sequence, head).  ml_of(i) / acc_of(i) give piece i's (max, sum) and the address of
+// its 128 accumulators; a piece whose max is -inf is skipped entirely (it may never have been written).
+template <int kCombineGroups, typename MlOf, typename AccOf>
+__device__ __forceinline__ void merge_pieces(int n, MlOf ml_of, AccOf acc_of, float* __restrict__ out) {
+    constexpr int kCombineThreads = kHeadDim * kCombineGroups;
+    __shared__ float m_s[1024], l_s[1024];
+    __shared__ float num_s[kCombineGroups][kHeadDim], den_s[kCombineGroups];
+    const int c = threadIdx.x & (kHeadDim - 1), g = threadIdx.x >> 7;
+    float a[kCombineEager];
+#pragma unroll
+    for (int e = 0; e < kCombineEager; ++e) {
+        const int i = g + e * kCombineGroups;
+        a[e] = i < n ? __ldcg(acc_of(i) + c) : 0.f;
+    }
+    for (int i = threadIdx.x; i < n; i += kCombineThreads) {
+        const float2 ml = ml_of(i);
+        m_s[i] = ml.x;
+        l_s[i] = ml.y;
+    }
+    __syncthreads();
+    float top = -INFINITY;
+    for (int i = 0; i < n; ++i) top = fmaxf(top, m_s[i]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int e = 0; e < kCombineEager; ++e) {
+        const int i = g + e * kCombineGroups;
+        if (i < n) {
+            const float w = fast_exp2(m_s[i] - top);
+            if (w != 0.f) { den = fmaf(w, l_s[i], den); num = fmaf(w, a[e], num); }   // never multiply an unwritten slot
+        }
+    }
+    for (int i0 = g + kCombineEager * kCombineGroups; i0 < n; i0 += kCombineEager * kCombineGroups) {
+#pragma unroll
+        for (int e = 0; e < kCombineEager; ++e) {
+            const int i = i0 + e * kCombineGroups;
+            a[e] = i < n ? __ldcg(acc_of(i) + c) : 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < kCombineEager; ++e) {
+            const int i = i0 + e * kCombineGroups;
+            if (i < n) {
+                const float w = fast_exp2(m_s[i] - top);
+                if (w != 0.f) { den = fmaf(w, l_s[i], den); num = fmaf(w, a[e], num); }
+            }
+        }
+    }
+    num_s[g][c] = num;
+    if (c == 0) den_s[g] = den;
+    __syncthreads();
+    if (g == 0) {
+#pragma unroll
+        for (int k = 1; k < kCombineGroups; ++k) { num += num_s[k][c]; den += den_s[k]; }
+        out[c] = num / den;
+    }
+}
+
+template <int GROUPS>
+__global__ void __launch_bounds__(kHeadDim * GROUPS)
 combine_splits_kernel(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
                       const int32_t* __restrict__ lens, float* __restrict__ o,
                       int h, int m_max, int chunk_rows, int n_splits, int len_bias) {
     const size_t u = blockIdx.x;
-    const int c = threadIdx.x;
     grid_dependency_wait();          // the partials come from the kernel before this one
     int L = biased_len(lens[u / h], m_max, len_bias);
     L = L < 0 ? 0 : (L > m_max ? m_max : L);
     int live = (L + chunk_rows - 1) / chunk_rows;
     if (live > n_splits) live = n_splits;
     if (live == 0) {
-        o[u * kHeadDim + c] = 0.f;
+        if (threadIdx.x < kHeadDim) o[u * kHeadDim + threadIdx.x] = 0.f;
         return;
     }
     const float2* ml = part_ml + u * n_splits;
     const float* acc = part_acc + u * (size_t)n_splits * kHeadDim;
-    float top = -INFINITY;
-    for (int s = 0; s < live; ++s) top = fmaxf(top, ml[s].x);
-    float num = 0.f, den = 0.f;
-    for (int s = 0; s < live; ++s) {
-        const float2 p = ml[s];
-        const float w = fast_exp2(p.x - top);
-        den = fmaf(w, p.y, den);
-        num = fmaf(w, acc[(size_t)s * kHeadDim + c], num);
-    }
-    o[u * kHeadDim + c] = num / den;
+    merge_pieces<GROUPS>(live, [&](int i) { return __ldcg(ml + i); }, [&](int i) { return acc + (size_t)i * kHeadDim; },
+                 o + u * kHeadDim);
 }
 
 }  // namespace mqa

@@ -868,60 +868,31 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
 // CTAs that hold pieces of the sequence (nothing to do when a single CTA had the whole sequence,
 // or it is empty).  seq_span[b] holds (T, G): a CTA whose share of the T tiles is empty wrote no
 // slot and is skipped.
-__global__ void __launch_bounds__(kHeadDim)
+template <int GROUPS>
+__global__ void __launch_bounds__(kHeadDim * GROUPS)
 stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restrict__ part_ml,
                       const float* __restrict__ part_acc, float* __restrict__ o, int b, int h,
                       int32_t* lens_advance, int m_max) {
     const int s = blockIdx.x / h, head = blockIdx.x % h;
-    const int c = threadIdx.x;
     grid_dependency_wait();          // the slots come from the kernel before this one
-    if (lens_advance && head == 0 && c == 0) {       // append-and-attend step: lens[s] += 1 for a sequence that took a row
+    if (lens_advance && head == 0 && threadIdx.x == 0) {   // append-and-attend step: lens[s] += 1 for a sequence that took a row
         const int raw = lens_advance[s];
         if (raw >= 0 && raw < m_max) lens_advance[s] = raw + 1;
     }
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
-    __shared__ float m_s[256], l_s[256];
-    const int n_cta = span.y - span.x + 1;              // at most the grid of the first pass (<= 256 SMs)
     const long long T = seq_span[b].x, G = seq_span[b].y;
-    // One round trip for everything this CTA needs: each candidate piece's (max, sum) is fetched by its own
-    // thread, and every thread fetches its column of the first pieces' accumulators at the same time (their
-    // addresses do not depend on the weights).  A CTA whose share of the line is empty wrote no slot: its
-    // max is taken as -inf, which makes its weight exactly zero and its (unwritten) slot is never used.
-    constexpr int kEager = 8;
-    float a[kEager];
-    const float* col = part_acc + ((size_t)span.x + s) * h * kHeadDim + (size_t)head * kHeadDim + c;
-#pragma unroll
-    for (int i = 0; i < kEager; ++i) a[i] = i < n_cta ? __ldcg(col + (size_t)i * h * kHeadDim) : 0.f;
-    for (int i = c; i < n_cta; i += kHeadDim) {
-        const long long cta = span.x + i;
-        const bool live = cta * T / G != (cta + 1) * T / G;
-        const float2 ml = live ? __ldcg(part_ml + ((size_t)cta + s) * h + head) : make_float2(-INFINITY, 0.f);
-        m_s[i] = ml.x;
-        l_s[i] = ml.y;
-    }
-    __syncthreads();
-    float top = -INFINITY;
-    for (int i = 0; i < n_cta; ++i) top = fmaxf(top, m_s[i]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int i = 0; i < kEager; ++i) {
-        if (i < n_cta) {
-            const float w = fast_exp2(m_s[i] - top);
-            if (w != 0.f) {                                  // never multiply an unwritten slot
-                den = fmaf(w, l_s[i], den);
-                num = fmaf(w, a[i], num);
-            }
-        }
-    }
-    for (int i = kEager; i < n_cta; ++i) {
-        const float w = fast_exp2(m_s[i] - top);
-        if (w != 0.f) {
-            den = fmaf(w, l_s[i], den);
-            num = fmaf(w, __ldcg(col + (size_t)i * h * kHeadDim), num);
-        }
-    }
-    o[((size_t)s * h + head) * kHeadDim + c] = num / den;
+    const int n_cta = span.y - span.x + 1;              // at most the grid of the first pass (<= 256 SMs)
+    // piece i is the slot of CTA span.x + i; a CTA whose share of the line is empty wrote none (max = -inf)
+    merge_pieces<GROUPS>(
+        n_cta,
+        [&](int i) {
+            const long long cta = span.x + i;
+            const bool live = cta * T / G != (cta + 1) * T / G;
+            return live ? __ldcg(part_ml + ((size_t)cta + s) * h + head) : make_float2(-INFINITY, 0.f);
+        },
+        [&](int i) { return part_acc + (((size_t)span.x + i + s) * h + head) * kHeadDim; },
+        o + ((size_t)s * h + head) * kHeadDim);
 }
 
 }  // namespace mqa
