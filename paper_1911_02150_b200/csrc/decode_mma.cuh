@@ -70,7 +70,7 @@ struct StreamCfg {                                     // persistent kernel, one
     static constexpr int kStages = 3;                  // every consumer warp waits on every stage: any depth is safe
     static constexpr int kStateFloats = 16 * 4 + 4;    // acc + (m, l) x 2 rows, per thread
     static constexpr int kMergeBytes = M_TILES * kStateFloats * 32 * 4;
-    static constexpr int kPrefixBytes = (kStreamMaxSeqs + 1) * 4 + 12;
+    static constexpr int kPrefixBytes = 2 * (kStreamMaxSeqs + 1) * 4 + 16;   // line positions + rows per sequence
     static constexpr int kSmemBytes = kStages * kStreamStageBytes + kMergeBytes + kPrefixBytes + 256 /* barriers */ +
                                       1024 /* alignment slack */;
     static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
@@ -500,6 +500,19 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 // whose share contains a crossing gets that many fewer real tiles, and all CTAs finish together.
 constexpr int kBoundaryPenalty = 12;
 
+// Share c of G of a line of T positions: [c*T/G, (c+1)*T/G).  32-bit arithmetic when the products fit
+// (a 64-bit division by a run-time divisor is a long dependent sequence at the head of every CTA).
+__device__ __forceinline__ void share_bounds(int c, long long T, int G, long long* begin, long long* end) {
+    if (T <= 0x7fffffff / G) {
+        const unsigned int t = (unsigned int)T, g = (unsigned int)G;
+        *begin = ((unsigned int)c * t) / g;
+        *end = ((unsigned int)(c + 1) * t) / g;
+    } else {
+        *begin = (long long)c * T / G;
+        *end = (long long)(c + 1) * T / G;
+    }
+}
+
 // A run of 32-row tiles [lo, hi) of sequence s inside one CTA's share.
 struct Segment {
     int s, lo, hi;
@@ -587,10 +600,12 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     uint8_t* stages = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
     float* merge_buf = reinterpret_cast<float*>(stages + kStages * kStreamStageBytes);      // [M_TILES][68][32]
     int* prefix = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(merge_buf) + Cfg::kMergeBytes);  // [b + 1]
+    int* rows_of = prefix + kStreamMaxSeqs + 1;         // [b] rows to attend over; bit 30: this step appends a row
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + Cfg::kPrefixBytes / 8 * 8);
     const uint32_t stages_s = smem_addr(stages);
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
-    __shared__ int timed_out, issued;
+    __shared__ int timed_out, issued, s_first_sm;
+    constexpr int kAppendBit = 1 << 30;
 
     if (warp == Cfg::kConsumerWarps && lane == 0) {
         prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
@@ -618,13 +633,16 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         if (appending && !can_append && cta == 0 && status)
             atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
         prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
+        rows_of[s] = L | (appending && can_append ? kAppendBit : 0);
         if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
             for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
         }
     }
-    if (threadIdx.x == 0) prefix[0] = 0;
+    if (threadIdx.x == 0) { prefix[0] = 0; s_first_sm = 0; }
     __syncthreads();
-    if (warp == 0) {                                       // inclusive scan of prefix[1..b] by one warp
+    if (warp == 0) {
+        // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
+        // also notes which sequence that is
         const int per = (b + 31) / 32;
         const int lo = 1 + lane * per, hi = min(b, lo + per - 1);
         int sum = 0;
@@ -635,24 +653,21 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
             const int up = __shfl_up_sync(0xffffffffu, incl, d);
             if (lane >= d) incl += up;
         }
+        long long tb, te;
+        share_bounds(cta, __shfl_sync(0xffffffffu, incl, 31), G, &tb, &te);
         int run = incl - sum;
-        for (int s = lo; s <= hi; ++s) { run += prefix[s]; prefix[s] = run; }
+        for (int s = lo; s <= hi; ++s) {
+            const int before = run;
+            run += prefix[s];
+            prefix[s] = run;
+            if (before <= tb && tb < run) s_first_sm = s - 1;      // sequence s-1 occupies [before, run)
+        }
     }
     __syncthreads();
     const long long T = prefix[b];
-    const long long t_begin = (long long)cta * T / G, t_end = (long long)(cta + 1) * T / G;
-
-    // first sequence of this CTA's share: the s with prefix[s] <= t_begin < prefix[s+1]
-    int s_first = 0;
-    if (t_begin < t_end) {
-        int lo = 0, hi = b - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (prefix[mid] <= t_begin) lo = mid; else hi = mid - 1;
-        }
-        s_first = lo;
-        while (prefix[s_first + 1] <= t_begin) ++s_first;  // skip sequences without tiles
-    }
+    long long t_begin, t_end;
+    share_bounds(cta, T, G, &t_begin, &t_end);
+    const int s_first = s_first_sm;                        // the s with prefix[s] <= t_begin < prefix[s+1]
 
     const int mt = warp % M_TILES;
     const int rw = warp / M_TILES;
@@ -668,12 +683,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
             Segment g;
             while (ok && walk.next(g)) {
                 const int s = g.s;
-                int new_row = -1;                          // row this step appends to sequence s
-                if (appending) {
-                    bool can_append;
-                    const int L = fused_rows(read_len<FUSED>(lens, s), m_max, true, &can_append);
-                    if (can_append) new_row = L - 1;
-                }
+                const int new_row = (rows_of[s] & kAppendBit) ? (rows_of[s] & (kAppendBit - 1)) - 1 : -1;   // row this step appends
                 for (int u = g.lo; u < g.hi && ok; u += kRowWarps, ++j) {
                     const int nsub = min(kRowWarps, g.hi - u);
                     const int stg = j % kStages;
@@ -737,7 +747,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         Segment g_;
         while (walk.next(g_)) {
             const int s = g_.s;
-            const int L = fused_rows(read_len<FUSED>(lens, s), m_max, appending, nullptr);
+            const int L = rows_of[s] & (kAppendBit - 1);
             const bool whole = g_.whole;
             const bool last_segment = walk.t >= t_end;     // (a later block could only add penalty tiles)
 
