@@ -5,7 +5,7 @@
 // as mqa_decode_stream_mma_kernel; what changes is who does the two contractions:
 //
 //   producer warp   TMA: the segment's Q (64 head rows x 128) once, then K and V in 64-row stages
-//   MMA warp        one thread issues tcgen05.mma:   S[64 heads x 64 rows] = Q K_stage^T   (TMEM)
+//   MMA warps       one thread each issues the tcgen05.mma of   S[64 heads x 64 rows] = Q K_stage^T   (TMEM)
 //                                                    O[64 heads x 128]    += P V_stage     (TMEM)
 //                   operands are read by the tensor core straight from the TMA-written shared
 //                   memory (K row-major = K-major B; V row-major = MN-major B), so K and V are
@@ -33,8 +33,8 @@ constexpr int kUmmaStageBytes = 4 * kUmmaBoxBytes;               // K lo, K hi, 
 constexpr int kUmmaStages = 5;
 constexpr int kUmmaQBytes = 2 * 64 * 128;                        // 64 head rows x 128 columns bf16 = 16 KiB
 constexpr int kUmmaSoftmaxWarps = 4;                             // heads 0..63
-constexpr int kUmmaProducerWarp = 4, kUmmaMmaWarp = 5;
-constexpr int kUmmaThreads = 6 * 32;
+constexpr int kUmmaProducerWarp = 4, kUmmaMmaWarp = 5, kUmmaPvWarp = 6;   // two issuing threads: S = Q K^T, and O += P V
+constexpr int kUmmaThreads = 7 * 32;
 // TMEM columns: S0 [0,64) S1 [64,128) O [128,256); P as bf16 pairs, two buffers of hi [32 cols] + lo [32 cols]
 constexpr int kUmmaTmemCols = 512;
 constexpr int kTmemO = 128, kTmemP = 256;
@@ -295,35 +295,13 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             if (!ok) atomicExch(&timed_out, 1);
         }
     } else if (warp == kUmmaMmaWarp) {
-        // =============================================================== MMA issuer
+        // =============================================================== issuer of S = Q K^T
+        // (one tcgen05.mma or commit costs this thread ~45 ns, measured; the two contractions of a stage are
+        // therefore issued by two threads)
         if (lane == 0 && t_begin < t_end) {
             constexpr uint32_t kIdescS = umma_idesc(64, kUmmaStageRows, false);
-            constexpr uint32_t kIdescO = umma_idesc(64, kHeadDim, true);
             bool ok = true;
-            // P V for stage jj (its P is in shared memory once p_ready completes phase jj)
-            auto issue_pv = [&](int jj, bool first_of_segment, int seg_of_jj) {
-                const int pb = jj & 1;
-                if (ok) ok = mbar_wait(p_ready + pb * 8, (jj >> 1) & 1);
-                if (ok && first_of_segment && seg_of_jj >= 1) ok = mbar_wait(o_free, (seg_of_jj - 1) & 1);
-                tc_fence_after();
-                const uint32_t v_s = stages_s + (jj % kUmmaStages) * kUmmaStageBytes + 2 * kUmmaBoxBytes;
-                if (ok) {
-#pragma unroll
-                    for (int part = 0; part < 2; ++part) {          // P hi, then P lo
-#pragma unroll
-                        for (int kk = 0; kk < kUmmaStageRows / 16; ++kk) {
-                            const uint32_t a = tmem_base + kTmemP + pb * 64 + part * 32 + kk * 8;   // 16 bf16 = 8 columns
-                            const uint64_t bd = umma_desc(v_s + kk * 2048, kUmmaBoxBytes, 1024);
-                            umma_ts(tmem_base + kTmemO, a, bd, kIdescO, (first_of_segment && part == 0 && kk == 0) ? 0u : 1u);
-                        }
-                    }
-                }
-                tc_commit(kv_empty + (jj % kUmmaStages) * 8);       // the stage's K and V are free again
-                tc_commit(pv_done + pb * 8);                        // this P buffer is free, O is up to date
-            };
             int j = 0, seg = 0;
-            bool prev_first = false;
-            int prev_seg = 0;
             ShareWalker walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
@@ -345,12 +323,42 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     }
                     tc_commit(s_ready + sb * 8);
                     if (u + kSubs >= g.hi) tc_commit(q_empty + qi * 8);   // last use of this segment's Q
-                    if (j > 0) issue_pv(j - 1, prev_first, prev_seg);
-                    prev_first = (u == g.lo);
-                    prev_seg = seg;
                 }
             }
-            if (j > 0) issue_pv(j - 1, prev_first, prev_seg);
+            if (!ok) atomicExch(&timed_out, 1);
+        }
+    } else if (warp == kUmmaPvWarp) {
+        // =============================================================== issuer of O += P V
+        if (lane == 0 && t_begin < t_end) {
+            constexpr uint32_t kIdescO = umma_idesc(64, kHeadDim, true);
+            bool ok = true;
+            int j = 0, seg = 0;
+            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            Segment g;
+            for (; walk.next(g); ++seg) {
+                const int L = min(max(__ldg(lens + g.s), 0), m_max);
+                const int parts = L >= kSingleRoundingMinRows ? 1 : 2;   // P hi only, or hi then lo (as the softmax warps wrote it)
+                for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
+                    const int pb = j & 1;
+                    if (ok) ok = mbar_wait(p_ready + pb * 8, (j >> 1) & 1);
+                    if (ok && u == g.lo && seg >= 1) ok = mbar_wait(o_free, (seg - 1) & 1);   // the segment before has read O out
+                    tc_fence_after();
+                    const uint32_t v_s = stages_s + (j % kUmmaStages) * kUmmaStageBytes + 2 * kUmmaBoxBytes;
+                    if (ok) {
+                        for (int part = 0; part < parts; ++part) {
+#pragma unroll
+                            for (int kk = 0; kk < kUmmaStageRows / 16; ++kk) {
+                                const uint32_t a = tmem_base + kTmemP + pb * 64 + part * 32 + kk * 8;   // 16 bf16 = 8 columns
+                                const uint64_t bd = umma_desc(v_s + kk * 2048, kUmmaBoxBytes, 1024);
+                                umma_ts(tmem_base + kTmemO, a, bd, kIdescO, (u == g.lo && part == 0 && kk == 0) ? 0u : 1u);
+                            }
+                        }
+                    }
+                    // S = Q K^T of this stage finished before its softmax began, so both K and V are free now
+                    tc_commit(kv_empty + (j % kUmmaStages) * 8);
+                    tc_commit(pv_done + pb * 8);                        // this P buffer is free, O is up to date
+                }
+            }
             if (!ok) atomicExch(&timed_out, 1);
         }
     } else {
@@ -377,6 +385,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 const int s = g.s;
                 const int L = min(max(__ldg(lens + s), 0), m_max);
                 const bool whole = g.whole;
+                const bool hilo = L < kSingleRoundingMinRows;    // long prefixes: one bf16 rounding of P is enough
                 float m_run = -INFINITY, l_run = 0.f;
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
                     const int sb = j & 1, stg = j % kUmmaStages;
@@ -412,7 +421,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         const float p1 = col0 + i + 1 < valid ? fast_exp2(__fmul_rn(__uint_as_float(r[i + 1]), kLog2e) - m_new) : 0.f;
                         l_run += p0 + p1;
                         p_hi[i / 2] = pack_bf16(p0, p1);
-                        p_lo[i / 2] = pack_bf16(p0 - bf16_lo(p_hi[i / 2]), p1 - bf16_hi(p_hi[i / 2]));
+                        if (hilo) p_lo[i / 2] = pack_bf16(p0 - bf16_lo(p_hi[i / 2]), p1 - bf16_hi(p_hi[i / 2]));
                     }
                     // this P buffer was last read by the P V of stage j-2
                     const int pb = j & 1;
@@ -434,7 +443,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     }
                     tc_fence_after();
                     tmem_st_words<kCpr / 2>(lane_base + kTmemP + pb * 64 + (col0 >> 1), p_hi);
-                    tmem_st_words<kCpr / 2>(lane_base + kTmemP + pb * 64 + 32 + (col0 >> 1), p_lo);
+                    if (hilo) tmem_st_words<kCpr / 2>(lane_base + kTmemP + pb * 64 + 32 + (col0 >> 1), p_lo);
                     // a stage that runs past the prefix: the tensor core would multiply the zero weights
                     // with whatever lies there (NaN * 0 = NaN), so those V rows are cleared first
                     if (valid < kUmmaStageRows) {
