@@ -119,10 +119,9 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
  * (Section 3) in a single call: the new token's key/value row is concatenated to each
  * sequence's cache at row lens[b] (as kv_cache_append does), then the h heads attend over
  * the lens[b] + 1 rows (as mqa_decode_step does).  For batches large enough for the persistent
- * kernel and h <= 32 there is no separate append launch: the CTA that streams a sequence's last
+ * kernels (h <= 64) there is no separate append launch: the CTA that streams a sequence's last
  * tile writes the new row just before it fetches that tile, and the second-pass kernel advances
- * lens (two launches instead of three).  Other sizes run the same step as separate launches
- * (h > 32 at large sizes: only with advance != 0, otherwise MQA_ERR_UNSUPPORTED).
+ * lens (two launches instead of three).  Other sizes run the same step as separate launches.
  *
  *   q, k_new, v_new   [b, h, k], [b, k], [b, v] bf16
  *   K, V              [b, m_max, k], [b, m_max, v] bf16, read-write (row lens[b] is written)

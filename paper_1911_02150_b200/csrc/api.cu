@@ -295,32 +295,50 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
-std::atomic<int> g_umma_opt_in[kMaxDevices][3];
+std::atomic<int> g_umma_opt_in[kMaxDevices][6];
 
-template <int R>
+template <int HP, bool FUSED>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-                void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream) {
-    auto kernel = mqa_decode_stream_umma_kernel<R>;
-    constexpr int kSlot = R == 4 ? 0 : (R == 2 ? 1 : 2);
+                void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream,
+                const void* k_new = nullptr, const void* v_new = nullptr) {
+    using Cfg = UmmaCfg<HP>;
+    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED>;
+    constexpr int kSlot = (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 2 + (FUSED ? 1 : 0);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
             cudaGetLastError();
             return MQA_ERR_CUDA;
         }
         g_umma_opt_in[dev][kSlot].store(1, std::memory_order_release);
     }
+    FusedArgs fa = {};
+    if (FUSED) {
+        fa.k_new = static_cast<const uint4*>(k_new);
+        fa.v_new = static_cast<const uint4*>(v_new);
+        fa.K = static_cast<uint4*>(const_cast<void*>(K));
+        fa.V = static_cast<uint4*>(const_cast<void*>(V));
+    }
     alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub, map_q;
     const long long rows = (long long)b * m_max;
     if (!encode_cache_map(&map_k, K, rows, kUmmaStageRows) || !encode_cache_map(&map_v, V, rows, kUmmaStageRows) ||
         !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows) ||
-        !encode_cache_map(&map_q, q, (long long)b * h, R == 4 ? 16 : (R == 2 ? 32 : ((h + 15) & ~15))))
+        !encode_cache_map(&map_q, q, (long long)b * h, HP))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
-    launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, kUmmaSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max);
+    launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
+                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, fa);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
+}
+
+template <bool FUSED>
+int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
+                    void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream,
+                    const void* k_new = nullptr, const void* v_new = nullptr) {
+    if (h <= 16) return launch_umma<16, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
+    if (h <= 32) return launch_umma<32, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
+    return launch_umma<64, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
 }
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
@@ -334,11 +352,7 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
-    if (p.kernel == Kernel::kUmma) {
-        if (h <= 16) return launch_umma<4>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
-        if (h <= 32) return launch_umma<2>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
-        return launch_umma<1>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
-    }
+    if (p.kernel == Kernel::kUmma) return launch_umma_for<false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream1)
         return launch_stream<1, false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream2)
@@ -485,14 +499,13 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
         if (rc) return rc;
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
     }
+    if (p.kernel == Kernel::kUmma) {
+        rc = launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
+        if (rc) return rc;
+        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
+    }
     // other plans: the same step as separate launches.  Without `advance` the append leaves lens alone and
     // the step is told that a sequence which took a row has one more row than lens says.
-    if (p.stream()) {   // the tcgen05 plan reads lens as it stands: advance, step, and take the advance back
-        if (!advance) return MQA_ERR_UNSUPPORTED;
-        rc = kv_cache_append(K, V, k_new, v_new, lens, 1, status, b, 1, m_max, k, v, stream_);
-        if (rc) return rc;
-        return mqa_decode_step(q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream_);
-    }
     rc = kv_cache_append(K, V, k_new, v_new, lens, 0, status, b, 1, m_max, k, v, stream_);
     if (rc) return rc;
     rc = run_split(true, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream, 1);
@@ -516,8 +529,7 @@ size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v) {
 int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
     const Plan p = make_plan(true, b, h, m_max);
-    if (p.kernel == Kernel::kStream1 || p.kernel == Kernel::kStream2) return 2;   // pass with the append inside, second pass
-    if (p.stream()) return 3;                          // append, tcgen05 pass, second pass
+    if (p.stream()) return 2;                          // pass with the append inside, second pass
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }
 

@@ -581,6 +581,64 @@ __device__ __forceinline__ int fused_rows(int raw, int m_max, bool appending, bo
     return ok ? L + 1 : L;
 }
 
+constexpr int kAppendBit = 1 << 30;                    // in rows_of[]: this step appends a row to the sequence
+
+// The schedule of a persistent kernel, computed by every CTA for itself (all THREADS threads call this):
+// prefix[s] = position on the line of sequence s's block (kBoundaryPenalty virtual tiles, then its 32-row
+// tiles; no block for an empty prefix, whose output is zeroed here), rows_of[s] = rows to attend over
+// (kAppendBit set when this step appends one), T = length of the line, [t_begin, t_end) = this CTA's share,
+// s_first = the sequence that holds position t_begin.
+template <bool FUSED, int THREADS>
+__device__ __forceinline__ void stream_plan(const int32_t* __restrict__ lens, float* __restrict__ o,
+                                            int32_t* __restrict__ status, int b, int h, int m_max, bool appending,
+                                            int* prefix, int* rows_of, int* s_first_sm, long long* T_out,
+                                            long long* t_begin_out, long long* t_end_out, int* s_first_out) {
+    const int cta = blockIdx.x, G = gridDim.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int s = threadIdx.x; s < b; s += THREADS) {
+        const int raw = read_len<FUSED>(lens, s);
+        clamp_len(raw, m_max, cta == 0 ? status : nullptr);
+        bool can_append;
+        const int L = fused_rows(raw, m_max, appending, &can_append);
+        if (appending && !can_append && cta == 0 && status)
+            atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
+        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
+        rows_of[s] = L | (appending && can_append ? kAppendBit : 0);
+        if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
+            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
+        }
+    }
+    if (threadIdx.x == 0) { prefix[0] = 0; *s_first_sm = 0; }
+    __syncthreads();
+    if (warp == 0) {
+        // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
+        // also notes which sequence that is
+        const int per = (b + 31) / 32;
+        const int lo = 1 + lane * per, hi = min(b, lo + per - 1);
+        int sum = 0;
+        for (int s = lo; s <= hi; ++s) sum += prefix[s];
+        int incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        long long tb, te;
+        share_bounds(cta, __shfl_sync(0xffffffffu, incl, 31), G, &tb, &te);
+        int run = incl - sum;
+        for (int s = lo; s <= hi; ++s) {
+            const int before = run;
+            run += prefix[s];
+            prefix[s] = run;
+            if (before <= tb && tb < run) *s_first_sm = s - 1;     // sequence s-1 occupies [before, run)
+        }
+    }
+    __syncthreads();
+    *T_out = prefix[b];
+    share_bounds(cta, *T_out, G, t_begin_out, t_end_out);
+    *s_first_out = *s_first_sm;                            // the s with prefix[s] <= t_begin < prefix[s+1]
+}
+
 template <int M_TILES, bool FUSED>
 __global__ void __launch_bounds__(StreamCfg<M_TILES>::kThreads, 1)
 mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -605,7 +663,6 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     const uint32_t stages_s = smem_addr(stages);
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
     __shared__ int timed_out, issued, s_first_sm;
-    constexpr int kAppendBit = 1 << 30;
 
     if (warp == Cfg::kConsumerWarps && lane == 0) {
         prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
@@ -624,50 +681,10 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
 
-    // ---- 32-row sub-tiles per sequence and their running sum (every CTA computes the same table)
-    for (int s = threadIdx.x; s < b; s += Cfg::kThreads) {
-        const int raw = read_len<FUSED>(lens, s);
-        clamp_len(raw, m_max, cta == 0 ? status : nullptr);
-        bool can_append;
-        const int L = fused_rows(raw, m_max, appending, &can_append);
-        if (appending && !can_append && cta == 0 && status)
-            atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
-        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
-        rows_of[s] = L | (appending && can_append ? kAppendBit : 0);
-        if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
-            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
-        }
-    }
-    if (threadIdx.x == 0) { prefix[0] = 0; s_first_sm = 0; }
-    __syncthreads();
-    if (warp == 0) {
-        // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
-        // also notes which sequence that is
-        const int per = (b + 31) / 32;
-        const int lo = 1 + lane * per, hi = min(b, lo + per - 1);
-        int sum = 0;
-        for (int s = lo; s <= hi; ++s) sum += prefix[s];
-        int incl = sum;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += up;
-        }
-        long long tb, te;
-        share_bounds(cta, __shfl_sync(0xffffffffu, incl, 31), G, &tb, &te);
-        int run = incl - sum;
-        for (int s = lo; s <= hi; ++s) {
-            const int before = run;
-            run += prefix[s];
-            prefix[s] = run;
-            if (before <= tb && tb < run) s_first_sm = s - 1;      // sequence s-1 occupies [before, run)
-        }
-    }
-    __syncthreads();
-    const long long T = prefix[b];
-    long long t_begin, t_end;
-    share_bounds(cta, T, G, &t_begin, &t_end);
-    const int s_first = s_first_sm;                        // the s with prefix[s] <= t_begin < prefix[s+1]
+    long long T, t_begin, t_end;
+    int s_first;
+    stream_plan<FUSED, Cfg::kThreads>(lens, o, status, b, h, m_max, appending, prefix, rows_of, &s_first_sm, &T, &t_begin,
+                                      &t_end, &s_first);
 
     const int mt = warp % M_TILES;
     const int rw = warp / M_TILES;

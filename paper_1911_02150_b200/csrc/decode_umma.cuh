@@ -1,23 +1,30 @@
-// Persistent multi-query decode kernel on the 5th-generation tensor cores (tcgen05 + TMEM) for
-// head counts where the register-fragment mma.sync path runs out of issue slots and shared-memory
-// bandwidth (h > 16).  Same step as the other kernels (Section 3: logits = einsum(bhk,bmk->bhm),
-// softmax over m, o = einsum(bhm,bmv->bhv)), same equal-share scheduling, slots and second pass
-// as mqa_decode_stream_mma_kernel; what changes is who does the two contractions:
+// Persistent multi-query decode kernel on the 5th-generation tensor cores (tcgen05 + TMEM).
+// Same step as the other kernels (Section 3: logits = einsum(bhk,bmk->bhm), softmax over m,
+// o = einsum(bhm,bmv->bhv)), same equal-share scheduling, slots and second pass as
+// mqa_decode_stream_mma_kernel; what changes is who does the two contractions and which way round
+// they are laid out.  The cache rows are the M dimension of both products and the heads are N:
 //
-//   producer warp   TMA: the segment's Q (64 head rows x 128) once, then K and V in 64-row stages
-//   MMA warps       one thread each issues the tcgen05.mma of   S[64 heads x 64 rows] = Q K_stage^T   (TMEM)
-//                                                    O[64 heads x 128]    += P V_stage     (TMEM)
-//                   operands are read by the tensor core straight from the TMA-written shared
-//                   memory (K row-major = K-major B; V row-major = MN-major B), so K and V are
-//                   read from shared memory once for all heads and no fragment ever enters a register
-//   softmax warps   the M=64 accumulator puts row r in TMEM lane 32*(r/16) + r%16, one row per thread
-//                   of warp r/16: tcgen05.ld the logits, exact online softmax in fp32 registers, P
-//                   written to shared memory as bf16 hi + lo (K-major A operand), O rescaled in TMEM
-//                   on the rare stages where a row's maximum moves.  With 32 heads or fewer the 64
-//                   rows hold R = 2 or 4 copies of the heads (Q is loaded R times); copy c takes the
-//                   c-th part of each stage's 64 cache rows, so every softmax warp has work and a
-//                   thread handles 64/R logits per stage.  The R partial results of a head are
-//                   merged when the segment ends.
+//     S^T[128 cache rows x HP heads]  = K_stage[128 x 128] * Q^T          A = the TMA-written K rows (K-major),
+//                                                                          B = the sequence's Q rows (K-major)
+//     O^T[128 columns x HP heads]    += V_stage^T[128 x 128 rows] * P^T   A = the TMA-written V rows (MN-major),
+//                                                                          B = P^T, written by the softmax warps
+//
+// so K and V are read from shared memory by the tensor core itself, once for all heads; the work
+// per stage grows with the padded head count HP (16, 32 or 64) and nothing is replicated.  In TMEM
+// a cache row of S^T is a lane, so a softmax thread owns one cache row of the stage and all its
+// heads: masking by index is a per-thread decision and the weights need no exchange between
+// threads.  The reference maximum of a head is shared by all rows and moves only when some logit
+// exceeds it by more than 2^kMaxLead (always on a segment's first stage): then the warps find the
+// stage's maxima together, rescale their sums and the O^T accumulator, and go on.  Softmax is shift
+// invariant, so a reference that lags the true maximum by a bounded amount changes nothing but the
+// common scale of numerator and denominator.
+//
+//   producer warp      TMA: a segment's Q rows once, then K and V rows in 128-row stages (separate
+//                      rings: a K slot is free again as soon as S^T is done)
+//   two MMA warps      one thread each issues the tcgen05.mma of S^T, and of O^T
+//   4 softmax warps    tcgen05.ld the logits of their row, P = exp2(S - reference) as bf16 (hi, and lo
+//                      for short prefixes) into shared memory, per-thread partial sums; at the end
+//                      of a segment the sums are added up and O^T is read out of TMEM
 //
 // Everything between the roles is an mbarrier; every wait is bounded (see mbar_wait).
 #pragma once
@@ -27,22 +34,34 @@
 
 namespace mqa {
 
-constexpr int kUmmaStageRows = 64;                               // cache rows per stage
-constexpr int kUmmaBoxBytes = kUmmaStageRows * 128;              // 8 KiB: 64 rows x 128 bytes
-constexpr int kUmmaStageBytes = 4 * kUmmaBoxBytes;               // K lo, K hi, V lo, V hi = 32 KiB
-constexpr int kUmmaStages = 5;
-constexpr int kUmmaQBytes = 2 * 64 * 128;                        // 64 head rows x 128 columns bf16 = 16 KiB
-constexpr int kUmmaSoftmaxWarps = 4;                             // heads 0..63
-constexpr int kUmmaProducerWarp = 4, kUmmaMmaWarp = 5, kUmmaPvWarp = 6;   // two issuing threads: S = Q K^T, and O += P V
+constexpr int kUmmaStageRows = 128;                              // cache rows per stage
+constexpr int kUmmaHalfBytes = kUmmaStageRows * 128;             // 16 KiB: one 64-column box of 128 rows
+constexpr int kUmmaSlotBytes = 2 * kUmmaHalfBytes;               // 32 KiB: the K (or the V) rows of a stage
+constexpr int kUmmaSoftmaxWarps = 4;
+constexpr int kUmmaProducerWarp = 4, kUmmaSWarp = 5, kUmmaPvWarp = 6;
 constexpr int kUmmaThreads = 7 * 32;
-// TMEM columns: S0 [0,64) S1 [64,128) O [128,256); P as bf16 pairs, two buffers of hi [32 cols] + lo [32 cols]
-constexpr int kUmmaTmemCols = 512;
-constexpr int kTmemO = 128, kTmemP = 256;
-constexpr int kUmmaPrefixBytes = (kStreamMaxSeqs + 1) * 4 + 12;
-constexpr int kUmmaXchgBytes = 48 * 32 * 4 + 48 * 8;              // merge of the head copies: 48 rows x (32 columns + (m, l))
-constexpr int kUmmaSmemBytes = kUmmaStages * kUmmaStageBytes + 2 * kUmmaQBytes + kUmmaPrefixBytes +
-                               kUmmaXchgBytes + 512 /* barriers */ + 1024 /* alignment slack */;
-static_assert(kUmmaSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
+constexpr float kMaxLead = 16.f;                                 // log2 units a logit may exceed the reference maximum by
+
+template <int HP>
+struct UmmaCfg {
+    static_assert(HP == 16 || HP == 32 || HP == 64, "padded head count");
+    static constexpr int kKSlots = 2, kVSlots = 3;
+    static constexpr int kQBytes = HP * 256;                     // HP head rows x 128 columns bf16, two 64-column boxes
+    // P^T tile: 128 cache rows x 128 bytes (64 bf16 head slots, HP used), 128-byte swizzle: an MN-major B
+    // operand, so that a softmax thread writes the weights of its cache row with 16-byte stores.  Two tiles:
+    // the hi parts of two buffers (one rounding of P), or hi and lo of a single buffer (short prefixes).
+    static constexpr int kPBytes = kUmmaStageRows * 128;
+    static constexpr int kPTiles = 2;
+    static constexpr int kQBufs = HP <= 32 ? 2 : 1;             // 64 head rows: one Q buffer (shared memory)
+    static constexpr int kChunk = HP < 32 ? HP : 32;             // heads handled per TMEM load
+    static constexpr int kRedBytes = (2 * kUmmaSoftmaxWarps + 2) * HP * 4;   // per-warp maxima and sums, reference maxima, factors
+    static constexpr int kPlanBytes = (2 * kStreamMaxSeqs + 1) * 4 + 12;   // line positions + rows per sequence
+    static constexpr int kBarriers = 2 * kKSlots + 2 * kVSlots + 13;
+    static constexpr int kSmemBytes = (kKSlots + kVSlots) * kUmmaSlotBytes + kQBufs * kQBytes + kPTiles * kPBytes + kRedBytes +
+                                      kPlanBytes + kBarriers * 8 + 1024 /* alignment slack */;
+    static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
+    static constexpr int kTmemCols = 3 * HP <= 64 ? 64 : (3 * HP <= 128 ? 128 : 256);   // S^T twice, O^T once
+};
 
 // ---- tcgen05 wrappers ----------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
@@ -138,41 +157,82 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_byte_addr, uint32_t 
     const uint64_t hi = (uint64_t)((sbo >> 4) & 0x3FFFu) | (1ull << 14) | (2ull << 29);
     return lo | (hi << 32);
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, M x N tile, B optionally MN-major.
-__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
+// Instruction descriptor: fp32 accumulator, bf16 A and B, M x N tile, A and B K-major unless said otherwise.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// R = copies of the heads among the 64 accumulator rows: 4 (h <= 16), 2 (h <= 32) or 1 (h <= 64).
-template <int R>
+// Barrier over `threads` threads that also ORs a predicate over them.
+__device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"((uint32_t)pred), "r"(id), "r"(threads) : "memory");
+    return out != 0;
+}
+
+// Reduces N (16 or 32) values per lane over the 32 lanes of a warp, all at once: afterwards lane l holds
+// the total (sum, or maximum) of value number l % N.  v is used up.
+template <int N, bool MAX>
+__device__ __forceinline__ float warp_reduce_scatter(float (&v)[N], int lane) {
+#pragma unroll
+    for (int d = N / 2; d >= 1; d >>= 1) {
+        const bool up = (lane & d) != 0;
+#pragma unroll
+        for (int i = 0; i < d; ++i) {
+            const float send = up ? v[i] : v[i + d];
+            const float keep = up ? v[i + d] : v[i];
+            const float got = __shfl_xor_sync(0xffffffffu, send, d);
+            v[i] = MAX ? fmaxf(keep, got) : keep + got;
+        }
+    }
+    if (N == 16) {
+        const float got = __shfl_xor_sync(0xffffffffu, v[0], 16);
+        v[0] = MAX ? fmaxf(v[0], got) : v[0] + got;
+    }
+    return v[0];
+}
+
+// HP = head rows of the Q tile (h rounded up to 16, 32 or 64).
+template <int HP, bool FUSED>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                               const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
                               const __grid_constant__ CUtensorMap map_q,
                               const int32_t* __restrict__ lens, float* __restrict__ o, int2* __restrict__ seq_span,
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
-                              int b, int h, int m_max) {
+                              int b, int h, int m_max, const FusedArgs fa) {
+    using Cfg = UmmaCfg<HP>;
+    constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = HP / CH;
+    constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
+    const bool appending = FUSED && fa.k_new != nullptr;
     const int cta = blockIdx.x, G = gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int H16 = R == 4 ? 16 : (R == 2 ? 32 : ((h + 15) & ~15));   // rows one copy of the heads takes
-    const int n_sm_warps = R > 1 ? 4 : (H16 >> 4);          // softmax warps whose rows hold real heads
-    constexpr int kCpr = kUmmaStageRows / R;                // stage columns (cache rows) per copy
 
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* stages = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-    uint8_t* q_buf = stages + kUmmaStages * kUmmaStageBytes;            // 2 x 16 KiB
-    int* prefix = reinterpret_cast<int*>(q_buf + 2 * kUmmaQBytes);      // [b + 1]
-    float* xchg_o = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(prefix) + kUmmaPrefixBytes / 8 * 8);   // [48][32]
-    float2* xchg_ml = reinterpret_cast<float2*>(xchg_o + 48 * 32);                                              // [48]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(xchg_ml + 48);
-    const uint32_t stages_s = smem_addr(stages), q_s = smem_addr(q_buf);
+    uint8_t* ring = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);   // K slots, then V slots
+    uint8_t* q_buf = ring + (NK + NV) * kUmmaSlotBytes;                 // 2 x Q
+    uint8_t* p_buf = q_buf + Cfg::kQBufs * Cfg::kQBytes;                // P^T tiles
+    float* red_m = reinterpret_cast<float*>(p_buf + Cfg::kPTiles * Cfg::kPBytes);   // [4 warps][HP]
+    float* red_l = red_m + kUmmaSoftmaxWarps * HP;                                  // [4 warps][HP]
+    float* m_sm = red_l + kUmmaSoftmaxWarps * HP;                                   // [HP] reference maxima (log2 units) of the segment
+    float* f_sm = m_sm + HP;                                                        // [HP] factor of the last move
+    int* prefix = reinterpret_cast<int*>(f_sm + HP);                                // [b + 1]
+    int* rows_of = prefix + kStreamMaxSeqs + 1;                                     // [b]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + (Cfg::kPlanBytes + 7) / 8 * 8);
+    const uint32_t k_ring = smem_addr(ring), v_ring = k_ring + NK * kUmmaSlotBytes;
+    const uint32_t q_s = smem_addr(q_buf), p_s = smem_addr(p_buf);
     // barrier table
-    const uint32_t kv_full = smem_addr(bars), kv_empty = kv_full + kUmmaStages * 8;
-    const uint32_t q_full = kv_empty + kUmmaStages * 8, q_empty = q_full + 16;
+    const uint32_t k_full = smem_addr(bars), k_empty = k_full + NK * 8;
+    const uint32_t v_full = k_empty + NK * 8, v_empty = v_full + NV * 8;
+    const uint32_t q_full = v_empty + NV * 8, q_empty = q_full + 16;
     const uint32_t s_ready = q_empty + 16, s_free = s_ready + 16;
     const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;
-    __shared__ int timed_out, issued;
+    __shared__ int timed_out, issued, s_first_sm;
     __shared__ uint32_t tmem_base_slot;
 
     if (warp == kUmmaProducerWarp && lane == 0) {
@@ -182,73 +242,32 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     if (threadIdx.x == 0) {
         timed_out = 0;
         issued = 0;
-        for (int s = 0; s < kUmmaStages; ++s) { mbar_init(kv_full + s * 8, 1); mbar_init(kv_empty + s * 8, 1); }
+        for (int s = 0; s < NK; ++s) { mbar_init(k_full + s * 8, 1); mbar_init(k_empty + s * 8, 1); }
+        for (int s = 0; s < NV; ++s) { mbar_init(v_full + s * 8, 1); mbar_init(v_empty + s * 8, 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(q_full + s * 8, 1); mbar_init(q_empty + s * 8, 1);
-            mbar_init(s_ready + s * 8, 1); mbar_init(s_free + s * 8, n_sm_warps);
-            mbar_init(p_ready + s * 8, n_sm_warps); mbar_init(pv_done + s * 8, 1);
+            mbar_init(s_ready + s * 8, 1); mbar_init(s_free + s * 8, kUmmaSoftmaxWarps);
+            mbar_init(p_ready + s * 8, kUmmaSoftmaxWarps); mbar_init(pv_done + s * 8, 1);
         }
-        mbar_init(o_free, n_sm_warps);
+        mbar_init(o_free, kUmmaSoftmaxWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == kUmmaMmaWarp) {                             // one warp owns the TMEM allocation
-        tmem_alloc(smem_addr(&tmem_base_slot), kUmmaTmemCols);
+    if (warp == kUmmaSWarp) {                               // one warp owns the TMEM allocation
+        tmem_alloc(smem_addr(&tmem_base_slot), Cfg::kTmemCols);
         tmem_relinquish();
     }
-    grid_dependency_wait();
+    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
 
-    // ---- 32-row sub-tiles per sequence and their running sum (as in the mma.sync persistent kernel)
-    for (int s = threadIdx.x; s < b; s += kUmmaThreads) {
-        const int L = clamp_len(lens[s], m_max, cta == 0 ? status : nullptr);
-        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
-        if (L == 0 && s % G == cta)
-            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
-    }
-    if (threadIdx.x == 0) prefix[0] = 0;
     tc_fence_before();
-    __syncthreads();
+    long long T, t_begin, t_end;
+    int s_first;
+    stream_plan<FUSED, kUmmaThreads>(lens, o, status, b, h, m_max, appending, prefix, rows_of, &s_first_sm, &T, &t_begin,
+                                     &t_end, &s_first);
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    if (warp < 4) {
-        // a row of P is written only in the columns of its own copy; the rest stays zero for the whole kernel
-        uint32_t z[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) z[i] = 0u;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_st32(tmem_base + ((uint32_t)(warp * 32) << 16) + kTmemP + c * 32, z);
-        tmem_wait_st();
-        tc_fence_before();
-    }
-    if (warp == 0) {
-        const int per = (b + 31) / 32;
-        const int lo = 1 + lane * per, hi = min(b, lo + per - 1);
-        int sum = 0;
-        for (int s = lo; s <= hi; ++s) sum += prefix[s];
-        int incl = sum;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += up;
-        }
-        int run = incl - sum;
-        for (int s = lo; s <= hi; ++s) { run += prefix[s]; prefix[s] = run; }
-    }
-    __syncthreads();
-    const long long T = prefix[b];
-    const long long t_begin = (long long)cta * T / G, t_end = (long long)(cta + 1) * T / G;
-    int s_first = 0;
-    if (t_begin < t_end) {
-        int lo = 0, hi = b - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (prefix[mid] <= t_begin) lo = mid; else hi = mid - 1;
-        }
-        s_first = lo;
-        while (prefix[s_first + 1] <= t_begin) ++s_first;
-    }
-    constexpr int kSubs = kUmmaStageRows / kTileRows;       // 2 sub-tiles of 32 rows per stage
+    const uint32_t tmem_o = tmem_base + 2 * HP;             // S^T buffers at columns 0 and HP, O^T after them
 
     if (warp == kUmmaProducerWarp) {
         // =============================================================== TMA producer
@@ -259,104 +278,117 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             Segment g;
             for (; ok && walk.next(g); ++seg) {
                 const int s = g.s;
-                const int qi = seg & 1;
-                if (seg >= 2) ok = mbar_wait(q_empty + qi * 8, ((seg >> 1) - 1) & 1);
+                const int qi = seg % NQ;
+                if (seg >= NQ) ok = mbar_wait(q_empty + qi * 8, ((seg / NQ) - 1) & 1);
                 if (!ok) break;
-                mbar_expect_tx(q_full + qi * 8, R * H16 * kRowBytes);
-#pragma unroll
-                for (int c = 0; c < R; ++c) {               // R copies of the sequence's head rows (box = H16 rows x 64 columns)
-                    const uint32_t d = q_s + qi * kUmmaQBytes + c * H16 * 128;
-                    tma_load_2d(d, &map_q, 0, s * h, q_full + qi * 8);
-                    tma_load_2d(d + kUmmaQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
-                }
+                // the sequence's head rows (rows past h belong to the next sequence or read as zero: their
+                // columns of S^T and O^T are never stored)
+                mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
+                tma_load_2d(q_s + qi * Cfg::kQBytes, &map_q, 0, s * h, q_full + qi * 8);
+                tma_load_2d(q_s + qi * Cfg::kQBytes + Cfg::kQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
+                const int new_row = (rows_of[s] & kAppendBit) ? (rows_of[s] & (kAppendBit - 1)) - 1 : -1;   // row this step appends
                 for (int u = g.lo; u < g.hi && ok; u += kSubs, ++j) {
                     const int nsub = min(kSubs, g.hi - u);
-                    const int stg = j % kUmmaStages;
-                    if (j >= kUmmaStages) ok = mbar_wait(kv_empty + stg * 8, ((j / kUmmaStages) - 1) & 1);
-                    if (!ok) break;
-                    const uint32_t bar = kv_full + stg * 8;
-                    const uint32_t dst = stages_s + stg * kUmmaStageBytes;
-                    mbar_expect_tx(bar, nsub * kStageBytes);
-                    const int y = s * m_max + u * kTileRows;
-                    if (nsub == kSubs) {
-                        tma_load_2d(dst, &map_k, 0, y, bar);
-                        tma_load_2d(dst + kUmmaBoxBytes, &map_k, kBoxCols, y, bar);
-                        tma_load_2d(dst + 2 * kUmmaBoxBytes, &map_v, 0, y, bar);
-                        tma_load_2d(dst + 3 * kUmmaBoxBytes, &map_v, kBoxCols, y, bar);
-                    } else {
-                        tma_load_2d(dst, &map_k_sub, 0, y, bar);
-                        tma_load_2d(dst + kUmmaBoxBytes, &map_k_sub, kBoxCols, y, bar);
-                        tma_load_2d(dst + 2 * kUmmaBoxBytes, &map_v_sub, 0, y, bar);
-                        tma_load_2d(dst + 3 * kUmmaBoxBytes, &map_v_sub, kBoxCols, y, bar);
+                    const int row_first = u * kTileRows;
+                    if (appending && new_row >= row_first && new_row < row_first + nsub * kTileRows) {
+                        const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16);
+                        const size_t src = (size_t)s * (kRowBytes / 16);
+                        uint4 kr[16], vr[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { kr[i] = fa.k_new[src + i]; vr[i] = fa.v_new[src + i]; }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { fa.K[dst + i] = kr[i]; fa.V[dst + i] = vr[i]; }
+                        asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
                     }
-                    issued = j + 1;
+                    const int y = s * m_max + row_first;
+#pragma unroll
+                    for (int kv = 0; kv < 2; ++kv) {        // the K rows, then the V rows, each into its own ring
+                        const int n_slots = kv ? NV : NK;
+                        const int slot = j % n_slots;
+                        const uint32_t full = (kv ? v_full : k_full) + slot * 8;
+                        if (j >= n_slots) ok = ok && mbar_wait((kv ? v_empty : k_empty) + slot * 8, ((j / n_slots) - 1) & 1);
+                        if (!ok) break;
+                        const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes;
+                        mbar_expect_tx(full, nsub * 2 * kBoxBytes);
+                        if (nsub == kSubs) {
+                            tma_load_2d(dst, kv ? &map_v : &map_k, 0, y, full);
+                            tma_load_2d(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full);
+                        } else {
+                            for (int i = 0; i < nsub; ++i) {
+                                const uint32_t d = dst + i * kBoxBytes;
+                                tma_load_2d(d, kv ? &map_v_sub : &map_k_sub, 0, y + i * kTileRows, full);
+                                tma_load_2d(d + kUmmaHalfBytes, kv ? &map_v_sub : &map_k_sub, kBoxCols, y + i * kTileRows, full);
+                            }
+                        }
+                        issued = 2 * j + kv + 1;            // copies started: K of stage j, then V of stage j
+                    }
                 }
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
-    } else if (warp == kUmmaMmaWarp) {
-        // =============================================================== issuer of S = Q K^T
-        // (one tcgen05.mma or commit costs this thread ~45 ns, measured; the two contractions of a stage are
-        // therefore issued by two threads)
+    } else if (warp == kUmmaSWarp) {
+        // =============================================================== issuer of S^T = K Q^T
         if (lane == 0 && t_begin < t_end) {
-            constexpr uint32_t kIdescS = umma_idesc(64, kUmmaStageRows, false);
+            constexpr uint32_t kIdescS = umma_idesc(128, HP, false, false);
             bool ok = true;
             int j = 0, seg = 0;
             ShareWalker walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
-                const int qi = seg & 1;
-                if (ok) ok = mbar_wait(q_full + qi * 8, (seg >> 1) & 1);
+                const int qi = seg % NQ;
+                if (ok) ok = mbar_wait(q_full + qi * 8, (seg / NQ) & 1);
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
-                    const int stg = j % kUmmaStages, sb = j & 1;
-                    if (ok) ok = mbar_wait(kv_full + stg * 8, (j / kUmmaStages) & 1);
+                    const int slot = j % NK, sb = j & 1;
+                    if (ok) ok = mbar_wait(k_full + slot * 8, (j / NK) & 1);
                     if (ok && j >= 2) ok = mbar_wait(s_free + sb * 8, ((j >> 1) - 1) & 1);
                     tc_fence_after();
                     if (ok) {
-                        const uint32_t k_s = stages_s + stg * kUmmaStageBytes;
+                        const uint32_t k_s = k_ring + slot * kUmmaSlotBytes;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {             // 8 k-steps of 16 columns; 4 per 64-column box
-                            const uint64_t a = umma_desc(q_s + qi * kUmmaQBytes + (ks >> 2) * (kUmmaQBytes / 2) + (ks & 3) * 32, 16, 1024);
-                            const uint64_t bd = umma_desc(k_s + (ks >> 2) * kUmmaBoxBytes + (ks & 3) * 32, 16, 1024);
-                            umma_ss(tmem_base + sb * 64, a, bd, kIdescS, ks ? 1u : 0u);
+                            const uint64_t a = umma_desc(k_s + (ks >> 2) * kUmmaHalfBytes + (ks & 3) * 32, 16, 1024);
+                            const uint64_t bd = umma_desc(q_s + qi * Cfg::kQBytes + (ks >> 2) * (Cfg::kQBytes / 2) + (ks & 3) * 32, 16, 1024);
+                            umma_ss(tmem_base + sb * HP, a, bd, kIdescS, ks ? 1u : 0u);
                         }
                     }
                     tc_commit(s_ready + sb * 8);
+                    tc_commit(k_empty + slot * 8);                   // the K rows are not needed again
                     if (u + kSubs >= g.hi) tc_commit(q_empty + qi * 8);   // last use of this segment's Q
                 }
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
     } else if (warp == kUmmaPvWarp) {
-        // =============================================================== issuer of O += P V
+        // =============================================================== issuer of O^T += V^T P^T
         if (lane == 0 && t_begin < t_end) {
-            constexpr uint32_t kIdescO = umma_idesc(64, kHeadDim, true);
+            constexpr uint32_t kIdescO = umma_idesc(128, HP, true, true);
             bool ok = true;
             int j = 0, seg = 0;
             ShareWalker walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
-                const int L = min(max(__ldg(lens + g.s), 0), m_max);
+                const int L = rows_of[g.s] & (kAppendBit - 1);
                 const int parts = L >= kSingleRoundingMinRows ? 1 : 2;   // P hi only, or hi then lo (as the softmax warps wrote it)
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
-                    const int pb = j & 1;
+                    const int pb = j & 1, slot = j % NV;
+                    if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
                     if (ok) ok = mbar_wait(p_ready + pb * 8, (j >> 1) & 1);
-                    if (ok && u == g.lo && seg >= 1) ok = mbar_wait(o_free, (seg - 1) & 1);   // the segment before has read O out
+                    if (ok && u == g.lo && seg >= 1) ok = mbar_wait(o_free, (seg - 1) & 1);   // the segment before has read O^T out
                     tc_fence_after();
-                    const uint32_t v_s = stages_s + (j % kUmmaStages) * kUmmaStageBytes + 2 * kUmmaBoxBytes;
                     if (ok) {
+                        const uint32_t v_s = v_ring + slot * kUmmaSlotBytes;
                         for (int part = 0; part < parts; ++part) {
+                            const uint32_t pt = p_s + (parts == 2 ? part : pb) * Cfg::kPBytes;
 #pragma unroll
-                            for (int kk = 0; kk < kUmmaStageRows / 16; ++kk) {
-                                const uint32_t a = tmem_base + kTmemP + pb * 64 + part * 32 + kk * 8;   // 16 bf16 = 8 columns
-                                const uint64_t bd = umma_desc(v_s + kk * 2048, kUmmaBoxBytes, 1024);
-                                umma_ts(tmem_base + kTmemO, a, bd, kIdescO, (u == g.lo && part == 0 && kk == 0) ? 0u : 1u);
+                            for (int kk = 0; kk < 8; ++kk) {         // 8 k-steps of 16 cache rows
+                                const uint64_t a = umma_desc(v_s + kk * 2048, kUmmaHalfBytes, 1024);
+                                const uint64_t bd = umma_desc(pt + kk * 2048, Cfg::kPBytes, 1024);
+                                umma_ss(tmem_o, a, bd, kIdescO, (u == g.lo && part == 0 && kk == 0) ? 0u : 1u);
                             }
                         }
                     }
-                    // S = Q K^T of this stage finished before its softmax began, so both K and V are free now
-                    tc_commit(kv_empty + (j % kUmmaStages) * 8);
-                    tc_commit(pv_done + pb * 8);                        // this P buffer is free, O is up to date
+                    tc_commit(v_empty + slot * 8);
+                    tc_commit(pv_done + pb * 8);                     // this P^T buffer is free, O^T is up to date
                 }
             }
             if (!ok) atomicExch(&timed_out, 1);
@@ -370,162 +402,201 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             }
             if (cta == 0 && lane == 0) seq_span[b] = make_int2((int)T, G);
         }
-        if (warp < n_sm_warps && t_begin < t_end) {
-            const int row = warp * 16 + (lane & 15);        // accumulator row of this thread (lanes 16..31 hold none)
-            const int head = row % H16, copy = row / H16;   // the copy is the same for a whole warp
-            const bool live = lane < 16 && head < h;
-            const int col0 = copy * kCpr;                   // this copy's columns of every stage
+        if (t_begin < t_end) {
+            const int t = warp * 32 + lane;                 // this thread's cache row of every stage = its TMEM lane;
+                                                            // at the end of a segment, its column of O^T
             const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-            const int sm_threads = n_sm_warps * 32, sm_tid = warp * 32 + lane;
-                        bool ok = true;
+            // where this row's weights go in a P^T tile (128 cache rows x 128 bytes, 128-byte swizzle): the 16
+            // bytes of heads 8c .. 8c+7 at row * 128 + ((c ^ (row & 7)) << 4)
+            const uint32_t p_row = (uint32_t)(t * 128), p_xor = (uint32_t)((t & 7) << 4);
+            bool ok = true;
             int j = 0, seg = 0;
             ShareWalker walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
                 const int s = g.s;
-                const int L = min(max(__ldg(lens + s), 0), m_max);
+                const int L = rows_of[s] & (kAppendBit - 1);
                 const bool whole = g.whole;
                 const bool hilo = L < kSingleRoundingMinRows;    // long prefixes: one bf16 rounding of P is enough
-                float m_run = -INFINITY, l_run = 0.f;
+                float l_sum[HP];                            // this row's share of every head's sum of weights
+#pragma unroll
+                for (int i = 0; i < HP; ++i) l_sum[i] = 0.f;
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
-                    const int sb = j & 1, stg = j % kUmmaStages;
+                    const int sb = j & 1, pb = j & 1;
+                    const bool first = u == g.lo;           // nothing accumulated yet: no reference maxima, O^T not started
                     // rows of this stage that count: what was fetched (the share may end mid-stage) and
                     // lies inside the prefix; always >= 1
                     const int fetched = min(kSubs, g.hi - u) * kTileRows;
                     const int valid = min(fetched, L - u * kTileRows);
+                    const bool row_ok = t < valid;
                     if (ok) ok = mbar_wait(s_ready + sb * 8, (j >> 1) & 1);
                     tc_fence_after();
-                    uint32_t r[kCpr];
-                    tmem_ld_cols<kCpr>(lane_base + sb * 64 + col0, r);
+                    uint32_t xr[HP];
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        uint32_t part[CH];
+                        tmem_ld_cols<CH>(lane_base + sb * HP + c * CH, part);
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) xr[c * CH + i] = part[i];
+                    }
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(s_free + sb * 8);             // S is in registers now
-                    // ---- the stage's maximum for this row (its own columns only)
-                    float top = -INFINITY;
+                    if (lane == 0) mbar_arrive(s_free + sb * 8);             // S^T is in registers now
+                    // ---- logits in log2 units, masked by index; how far the largest leads its reference
+                    float x[HP];
+                    float lead = -INFINITY;
 #pragma unroll
-                    for (int i = 0; i < kCpr; ++i)
-                        if (col0 + i < valid) top = fmaxf(top, __uint_as_float(r[i]));   // select by index
-                    // same rounding as below: the maximum's weight is exactly 1.  A copy whose columns
-                    // are all beyond the prefix keeps its state.
-                    const float m_new = fmaxf(m_run, __fmul_rn(top, kLog2e));
-                    const float rescale = m_new == -INFINITY ? 1.f : fast_exp2(m_run - m_new);   // 0 on a copy's first columns
-                    const bool moved = live && m_new > m_run && u != g.lo;   // O holds something to rescale
-                    l_run *= rescale;
-                    m_run = m_new;
-                    // ---- P = exp2(S - max) as bf16 hi + lo pairs (two cache rows per 32-bit TMEM column)
-                    uint32_t p_hi[kCpr / 2], p_lo[kCpr / 2];
+                    for (int i = 0; i < HP; i += 4) {
+                        const float4 m4 = first ? make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY)
+                                                : *reinterpret_cast<const float4*>(m_sm + i);
+                        const float mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
-                    for (int i = 0; i < kCpr; i += 2) {
-                        const float p0 = col0 + i < valid ? fast_exp2(__fmul_rn(__uint_as_float(r[i]), kLog2e) - m_new) : 0.f;
-                        const float p1 = col0 + i + 1 < valid ? fast_exp2(__fmul_rn(__uint_as_float(r[i + 1]), kLog2e) - m_new) : 0.f;
-                        l_run += p0 + p1;
-                        p_hi[i / 2] = pack_bf16(p0, p1);
-                        if (hilo) p_lo[i / 2] = pack_bf16(p0 - bf16_lo(p_hi[i / 2]), p1 - bf16_hi(p_hi[i / 2]));
-                    }
-                    // this P buffer was last read by the P V of stage j-2
-                    const int pb = j & 1;
-                    if (j >= 2 && ok) ok = mbar_wait(pv_done + pb * 8, ((j >> 1) - 1) & 1);
-                    if (__any_sync(0xffffffffu, moved)) {
-                        // rare after the first stages: rescale this row of O in TMEM, between the P V of the
-                        // stage before (waited for here) and the P V of this stage (not yet released)
-                        if (ok) ok = mbar_wait(pv_done + (pb ^ 1) * 8, ((j - 1) >> 1) & 1);
-                        tc_fence_after();
-                        uint32_t x[32];
-#pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
-                            tmem_ld32(lane_base + kTmemO + c * 32, x);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) x[i] = __float_as_uint(__uint_as_float(x[i]) * (moved ? rescale : 1.f));
-                            tmem_st32(lane_base + kTmemO + c * 32, x);
+                        for (int e = 0; e < 4; ++e) {
+                            x[i + e] = row_ok ? __fmul_rn(__uint_as_float(xr[i + e]), kLog2e) : -INFINITY;   // select, never multiply
+                            lead = fmaxf(lead, x[i + e] - mv[e]);           // (-inf) - (-inf) = NaN is ignored by fmaxf
                         }
                     }
-                    tc_fence_after();
-                    tmem_st_words<kCpr / 2>(lane_base + kTmemP + pb * 64 + (col0 >> 1), p_hi);
-                    if (hilo) tmem_st_words<kCpr / 2>(lane_base + kTmemP + pb * 64 + 32 + (col0 >> 1), p_lo);
+                    if (named_barrier_or(1, kUmmaSoftmaxWarps * 32, lead > kMaxLead)) {
+                        // ---- some logit leads by too much (always on a segment's first stage): every head's
+                        // reference moves to the largest logit seen so far; sums and O^T are rescaled
+#pragma unroll
+                        for (int c = 0; c < NCH; ++c) {
+                            float r[CH];
+#pragma unroll
+                            for (int i = 0; i < CH; ++i) r[i] = x[c * CH + i];
+                            const float top = warp_reduce_scatter<CH, true>(r, lane);
+                            if (lane < CH) red_m[warp * HP + c * CH + lane] = top;
+                        }
+                        named_barrier(2, kUmmaSoftmaxWarps * 32);
+                        if (t < HP) {
+                            const float m_old = first ? -INFINITY : m_sm[t];
+                            float m_new = m_old;
+#pragma unroll
+                            for (int w = 0; w < kUmmaSoftmaxWarps; ++w) m_new = fmaxf(m_new, red_m[w * HP + t]);   // finite: the stage has a valid row
+                            f_sm[t] = fast_exp2(m_old - m_new);              // 0 on the first stage, 1 if unchanged
+                            m_sm[t] = m_new;
+                        }
+                        named_barrier(2, kUmmaSoftmaxWarps * 32);
+                        if (!first) {
+#pragma unroll
+                            for (int i = 0; i < HP; i += 4) {
+                                const float4 f4 = *reinterpret_cast<const float4*>(f_sm + i);
+                                l_sum[i] *= f4.x; l_sum[i + 1] *= f4.y; l_sum[i + 2] *= f4.z; l_sum[i + 3] *= f4.w;
+                            }
+                            // O^T holds the stages before this one: wait for the last of their products, scale
+                            // column (head) i of this thread's lane by f[i]
+                            if (ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
+                            tc_fence_after();
+#pragma unroll
+                            for (int c = 0; c < NCH; ++c) {
+                                uint32_t y[CH];
+                                tmem_ld_cols<CH>(lane_base + 2 * HP + c * CH, y);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < CH; i += 4) {
+                                    const float4 f4 = *reinterpret_cast<const float4*>(f_sm + c * CH + i);
+                                    y[i] = __float_as_uint(__uint_as_float(y[i]) * f4.x);
+                                    y[i + 1] = __float_as_uint(__uint_as_float(y[i + 1]) * f4.y);
+                                    y[i + 2] = __float_as_uint(__uint_as_float(y[i + 2]) * f4.z);
+                                    y[i + 3] = __float_as_uint(__uint_as_float(y[i + 3]) * f4.w);
+                                }
+                                tmem_st_words<CH>(lane_base + 2 * HP + c * CH, y);
+                            }
+                            tmem_wait_st();
+                            tc_fence_before();
+                        }
+                    }
+                    // this P^T tile was last read by the product of stage j-2 (of stage j-1 when hi and lo take
+                    // both tiles)
+                    if (j >= 2 && ok) ok = mbar_wait(pv_done + pb * 8, ((j >> 1) - 1) & 1);
+                    if (hilo && j >= 1 && ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
+                    // ---- P = exp2(S - reference): 0 for a masked row; bf16 hi (and lo) into the P^T tiles
+                    const uint32_t p_hi = p_s + (hilo ? 0 : pb) * Cfg::kPBytes + p_row, p_lo = p_s + Cfg::kPBytes + p_row;
+#pragma unroll
+                    for (int c = 0; c < HP / 8; ++c) {
+                        const float4 ma = *reinterpret_cast<const float4*>(m_sm + c * 8);
+                        const float4 mb = *reinterpret_cast<const float4*>(m_sm + c * 8 + 4);
+                        const float mv[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+                        float pw[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            pw[e] = fast_exp2(x[c * 8 + e] - mv[e]);
+                            l_sum[c * 8 + e] += pw[e];
+                        }
+                        uint32_t hi[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) hi[e] = pack_bf16(pw[2 * e], pw[2 * e + 1]);
+                        const uint32_t at = ((uint32_t)(c << 4)) ^ p_xor;
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(p_hi + at), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]));
+                        if (hilo) {
+                            uint32_t lo[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                lo[e] = pack_bf16(pw[2 * e] - bf16_lo(hi[e]), pw[2 * e + 1] - bf16_hi(hi[e]));
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(p_lo + at), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]));
+                        }
+                    }
                     // a stage that runs past the prefix: the tensor core would multiply the zero weights
                     // with whatever lies there (NaN * 0 = NaN), so those V rows are cleared first
                     if (valid < kUmmaStageRows) {
-                        const uint32_t v_s = stages_s + stg * kUmmaStageBytes + 2 * kUmmaBoxBytes;
-                        for (int i = sm_tid; i < (kUmmaStageRows - valid) * 16; i += sm_threads) {
+                        const int slot = j % NV;
+                        if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
+                        const uint32_t v_s = v_ring + slot * kUmmaSlotBytes;
+                        for (int i = t; i < (kUmmaStageRows - valid) * 16; i += kUmmaSoftmaxWarps * 32) {
                             const int vrow = valid + (i >> 4), ch = i & 15;  // 16 chunks of 16 bytes per row
-                            const uint32_t a = v_s + (ch >> 3) * kUmmaBoxBytes + vrow * 128 + ((ch & 7) << 4);
+                            const uint32_t a = v_s + (ch >> 3) * kUmmaHalfBytes + vrow * 128 + ((ch & 7) << 4);
                             asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
                         }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // cleared V visible to the tensor core
                     }
-                    tmem_wait_st();
-                    tc_fence_before();
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P^T (and cleared V) visible to the tensor core
                     __syncwarp();
                     if (lane == 0) mbar_arrive(p_ready + pb * 8);
                 }
-                // ---- segment done: wait for its last P V, merge the copies of each head, read O out of TMEM
-                if (j >= 2 && ok) ok = mbar_wait(pv_done + (j & 1) * 8, ((j - 2) >> 1) & 1);        // P V of stage j-2 ...
-                if (ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);           // ... and of the last stage
+                // ---- segment done: add up the rows' sums, wait for the last product, read O^T out of TMEM
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    float r[CH];
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) r[i] = l_sum[c * CH + i];
+                    const float tot = warp_reduce_scatter<CH, false>(r, lane);
+                    if (lane < CH) red_l[warp * HP + c * CH + lane] = tot;
+                }
+                named_barrier(2, kUmmaSoftmaxWarps * 32);
+                if (ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
                 tc_fence_after();
                 const size_t slot = (size_t)cta + s;
-                float w_own = 1.f, m_tot = m_run, l_tot = l_run;
-                float w_other[R > 1 ? R - 1 : 1];
-                if constexpr (R > 1) {
-                    if (lane < 16 && copy > 0) xchg_ml[(copy - 1) * H16 + head] = make_float2(m_run, l_run);
-                    named_barrier(2, 128);
-                    if (copy == 0) {
+                float* dst = (whole ? o + (size_t)s * h * kHeadDim : part_acc + slot * h * kHeadDim) + t;
 #pragma unroll
-                        for (int c = 1; c < R; ++c) m_tot = fmaxf(m_tot, xchg_ml[(c - 1) * H16 + head].x);
-                        w_own = m_run == -INFINITY ? 0.f : fast_exp2(m_run - m_tot);   // copy 0 always holds the first row: finite
-                        l_tot = l_run * w_own;
+                for (int c = 0; c < NCH; ++c) {
+                    uint32_t y[CH];
+                    tmem_ld_cols<CH>(lane_base + 2 * HP + c * CH, y);
+                    float inv[CH];
 #pragma unroll
-                        for (int c = 1; c < R; ++c) {
-                            const float2 ml = xchg_ml[(c - 1) * H16 + head];
-                            w_other[c - 1] = ml.x == -INFINITY ? 0.f : fast_exp2(ml.x - m_tot);
-                            l_tot = fmaf(w_other[c - 1], ml.y, l_tot);
+                    for (int i = 0; i < CH; i += 4) {
+                        float4 tot = *reinterpret_cast<const float4*>(red_l + c * CH + i);
+#pragma unroll
+                        for (int w = 1; w < kUmmaSoftmaxWarps; ++w) {
+                            const float4 o4 = *reinterpret_cast<const float4*>(red_l + w * HP + c * CH + i);
+                            tot.x += o4.x; tot.y += o4.y; tot.z += o4.z; tot.w += o4.w;
                         }
+                        inv[i] = whole ? 1.f / tot.x : 1.f; inv[i + 1] = whole ? 1.f / tot.y : 1.f;
+                        inv[i + 2] = whole ? 1.f / tot.z : 1.f; inv[i + 3] = whole ? 1.f / tot.w : 1.f;
                     }
-                }
-                float* dst = whole ? o + ((size_t)s * h + head) * kHeadDim : part_acc + (slot * h + head) * kHeadDim;
-                const float inv = whole ? 1.f / l_tot : 1.f;
-                uint32_t x[32];
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(lane_base + kTmemO + c * 32, x);
                     tmem_wait_ld();
-                    if constexpr (R > 1) {
-                        if (lane < 16 && copy > 0) {
-                            float4* put = reinterpret_cast<float4*>(xchg_o + ((copy - 1) * H16 + head) * 32);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) put[i] = make_float4(__uint_as_float(x[4 * i]), __uint_as_float(x[4 * i + 1]), __uint_as_float(x[4 * i + 2]), __uint_as_float(x[4 * i + 3]));
-                        }
-                        named_barrier(2, 128);
-                        if (copy == 0) {
-#pragma unroll
-                            for (int cc = 1; cc < R; ++cc) {
-                                const float4* get = reinterpret_cast<const float4*>(xchg_o + ((cc - 1) * H16 + head) * 32);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const float4 v4 = get[i];
-                                    const float wgt = w_other[cc - 1];
-                                    x[4 * i] = __float_as_uint(fmaf(wgt, v4.x, __uint_as_float(x[4 * i]) * (cc == 1 ? w_own : 1.f)));
-                                    x[4 * i + 1] = __float_as_uint(fmaf(wgt, v4.y, __uint_as_float(x[4 * i + 1]) * (cc == 1 ? w_own : 1.f)));
-                                    x[4 * i + 2] = __float_as_uint(fmaf(wgt, v4.z, __uint_as_float(x[4 * i + 2]) * (cc == 1 ? w_own : 1.f)));
-                                    x[4 * i + 3] = __float_as_uint(fmaf(wgt, v4.w, __uint_as_float(x[4 * i + 3]) * (cc == 1 ? w_own : 1.f)));
-                                }
-                            }
-                        }
-                    }
-                    if (live && copy == 0) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<float4*>(dst + c * 32 + i) =
-                                make_float4(__uint_as_float(x[i]) * inv, __uint_as_float(x[i + 1]) * inv,
-                                            __uint_as_float(x[i + 2]) * inv, __uint_as_float(x[i + 3]) * inv);
-                    }
-                    if constexpr (R > 1) named_barrier(2, 128);              // the exchange buffer is free again
+                    for (int i = 0; i < CH; ++i)
+                        if (c * CH + i < h) dst[(size_t)(c * CH + i) * kHeadDim] = __uint_as_float(y[i]) * inv[i];
                 }
-                if (live && copy == 0 && !whole) part_ml[slot * h + head] = make_float2(m_tot, l_tot);
+                if (!whole && t < h) {
+                    float tot = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kUmmaSoftmaxWarps; ++w) tot += red_l[w * HP + t];
+                    part_ml[slot * h + t] = make_float2(m_sm[t], tot);
+                }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);         // the next segment may overwrite O
+                if (lane == 0) mbar_arrive(o_free);         // the next segment may overwrite O^T
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
@@ -534,16 +605,16 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     tc_fence_before();
     __syncthreads();
     if (timed_out && threadIdx.x == 0) {
-        for (int s = 0; s < kUmmaStages && s < issued; ++s) {
-            const int last_use = (issued - 1 - s) / kUmmaStages;
-            mbar_wait(kv_full + s * 8, last_use & 1);
-        }
+        // before the CTA leaves: the last copy started into each ring slot has to land
+        const int n_k = (issued + 1) / 2, n_v = issued / 2;
+        for (int s = 0; s < NK && s < n_k; ++s) mbar_wait(k_full + s * 8, ((n_k - 1 - s) / NK) & 1);
+        for (int s = 0; s < NV && s < n_v; ++s) mbar_wait(v_full + s * 8, ((n_v - 1 - s) / NV) & 1);
         if (status) atomicOr(status, kStatusPipelineTimeout);
     }
     __syncthreads();
-    if (warp == kUmmaMmaWarp) {
+    if (warp == kUmmaSWarp) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kUmmaTmemCols);
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
 }
 

@@ -57,9 +57,11 @@ def lens_mix(b, m_max, seed):
 
 
 CASES = [
-    # b, h, m_max: plans with the append inside the pass (persistent mma.sync kernel) ...
+    # b, h, m_max: plans with the append inside the pass (persistent kernels) ...
     (40, 16, 1500), (160, 32, 333), (300, 8, 200), (37, 32, 4000), (64, 5, 777),
-    # ... and plans that run as separate launches (small batch; tcgen05 plan for h > 32 with advance)
+    # ... the persistent tcgen05 kernel (h > 32) ...
+    (40, 48, 1500), (33, 64, 2100),
+    # ... and plans that run as separate launches (small batches)
     (4, 8, 300), (1, 16, 20000), (2, 40, 600),
 ]
 
@@ -76,19 +78,6 @@ def test_append_step_full_and_negative_sequences_take_no_row():
     lens[3] = m_max          # full: no row, attends over m_max rows
     lens[7] = -2             # negative: no row, empty prefix -> zeros
     run(b, h, m_max, lens, True, seed=77)
-
-
-def test_append_step_tcgen05_plan_needs_advance():
-    b, h, m_max = 40, 48, 1500           # persistent tcgen05 plan
-    inp = wl.make_inputs(b, h, m_max, "mqa", seed=9, device=DEV)
-    lens_np = lens_mix(b, m_max, seed=9)
-    run(b, h, m_max, lens_np, True, seed=9)
-    lens_t = torch.from_numpy(lens_np).to(DEV)
-    o = torch.zeros(b, h, 128, dtype=torch.float32, device=DEV)
-    with pytest.raises(mqa.MqaError) as e:
-        mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o,
-                                   mqa.alloc_workspace(b, h, m_max, DEV), advance=False)
-    assert e.value.code == binding.ERR_UNSUPPORTED
 
 
 def test_incremental_decoding_with_append_steps():
