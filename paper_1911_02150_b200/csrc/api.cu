@@ -111,10 +111,10 @@ Plan plan_stream(int b, int h, int m_max) {
     Plan p;
     p.units = (size_t)b * h;
     p.b = b; p.h = h;
-    // up to 32 heads the register-fragment mma.sync kernel; 33..64 heads the tcgen05 kernel.
-    // MQA_DECODE_UMMA=1 in the environment sends every head count to the tcgen05 kernel (for comparisons).
-    static const bool force_umma = [] { const char* e = getenv("MQA_DECODE_UMMA"); return e && e[0] == '1'; }();
-    p.kernel = force_umma ? Kernel::kUmma : (h <= 16 ? Kernel::kStream1 : (h <= 32 ? Kernel::kStream2 : Kernel::kUmma));
+    // the tcgen05 kernel for every head count up to 64.  MQA_DECODE_MMA=1 in the environment sends h <= 32 to the
+    // register-fragment mma.sync kernel instead (for comparisons).
+    static const bool force_mma = [] { const char* e = getenv("MQA_DECODE_MMA"); return e && e[0] == '1'; }();
+    p.kernel = (force_mma && h <= 32) ? (h <= 16 ? Kernel::kStream1 : Kernel::kStream2) : Kernel::kUmma;
     p.grid = sm_count();
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
@@ -291,7 +291,7 @@ int launch_stream(const Plan& p, const void* q, const void* K, const void* V, co
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     launch_dependent(kernel, (unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max, fa);
+                     static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -328,7 +328,7 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, fa);
+                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 

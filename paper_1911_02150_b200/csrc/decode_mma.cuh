@@ -498,19 +498,15 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 // partial or the result is written, the next sequence's Q is fetched), so the line carries, in front
 // of each sequence's tiles, kBoundaryPenalty virtual tiles that cost nothing to "process": a CTA
 // whose share contains a crossing gets that many fewer real tiles, and all CTAs finish together.
-constexpr int kBoundaryPenalty = 12;
+constexpr int kBoundaryPenalty = 12;         // mma.sync kernel (the tcgen05 kernel has its own)
 
-// Share c of G of a line of T positions: [c*T/G, (c+1)*T/G).  32-bit arithmetic when the products fit
-// (a 64-bit division by a run-time divisor is a long dependent sequence at the head of every CTA).
-__device__ __forceinline__ void share_bounds(int c, long long T, int G, long long* begin, long long* end) {
-    if (T <= 0x7fffffff / G) {
-        const unsigned int t = (unsigned int)T, g = (unsigned int)G;
-        *begin = ((unsigned int)c * t) / g;
-        *end = ((unsigned int)(c + 1) * t) / g;
-    } else {
-        *begin = (long long)c * T / G;
-        *end = (long long)(c + 1) * T / G;
-    }
+// Share c of G of a line of T positions: [c*T/G, (c+1)*T/G).  The division by the run-time grid size is
+// a multiplication by magic = ceil(2^64 / G), computed on the host (exact for c*T < 2^48, G <= 256; a
+// division in the kernel would be a long dependent sequence at the head of every CTA).  magic = 0: G = 1.
+__host__ __device__ inline unsigned long long share_magic(int G) { return G <= 1 ? 0ull : ~0ull / (unsigned long long)G + 1ull; }
+__device__ __forceinline__ int share_begin(int c, int T, unsigned long long magic) {
+    const unsigned long long n = (unsigned long long)(unsigned int)c * (unsigned int)T;
+    return magic ? (int)__umul64hi(n, magic) : (int)n;
 }
 
 // A run of 32-row tiles [lo, hi) of sequence s inside one CTA's share.
@@ -521,21 +517,22 @@ struct Segment {
 
 // Walks one CTA's share [t, t_end) of the line.  prefix[s] = position of sequence s's block (its penalty
 // tiles, then its real tiles); sequences without rows have no block.
+template <int PENALTY>
 struct ShareWalker {
     const int* prefix;
-    long long t, t_end;
+    int t, t_end;
     int s;
     __device__ __forceinline__ bool next(Segment& g) {
         while (t < t_end) {
             while (prefix[s + 1] <= t) ++s;
-            const long long v0 = prefix[s], v1 = prefix[s + 1];
-            const int n = (int)(v1 - v0) - kBoundaryPenalty;                    // real tiles, >= 1
-            const long long end = v1 < t_end ? v1 : t_end;
-            const long long lo = t - v0 - kBoundaryPenalty, hi = end - v0 - kBoundaryPenalty;
+            const int v0 = prefix[s], v1 = prefix[s + 1];
+            const int n = v1 - v0 - PENALTY;                                    // real tiles, >= 1
+            const int end = v1 < t_end ? v1 : t_end;
+            const int lo = t - v0 - PENALTY, hi = end - v0 - PENALTY;
             t = end;
             g.s = s;
-            g.lo = lo > 0 ? (int)lo : 0;
-            g.hi = hi < n ? (int)hi : n;
+            g.lo = lo > 0 ? lo : 0;
+            g.hi = hi < n ? hi : n;
             g.whole = g.lo == 0 && g.hi == n;
             if (g.hi > g.lo) return true;
         }
@@ -566,11 +563,10 @@ struct FusedArgs {
     uint4* V;
 };
 
-// lens[s]; the append-and-attend step reads it with plain loads (the kernel after it writes lens).
+// lens[s], read from L2 (the kernels before and after this one may write lens).
 template <bool FUSED>
 __device__ __forceinline__ int read_len(const int32_t* lens, int s) {
-    if constexpr (FUSED) return *reinterpret_cast<const volatile int32_t*>(lens + s);
-    else return __ldg(lens + s);
+    return __ldcg(lens + s);
 }
 
 // Rows of sequence s this launch attends over, and whether the step appends to it.
@@ -586,13 +582,14 @@ constexpr int kAppendBit = 1 << 30;                    // in rows_of[]: this ste
 // The schedule of a persistent kernel, computed by every CTA for itself (all THREADS threads call this):
 // prefix[s] = position on the line of sequence s's block (kBoundaryPenalty virtual tiles, then its 32-row
 // tiles; no block for an empty prefix, whose output is zeroed here), rows_of[s] = rows to attend over
-// (kAppendBit set when this step appends one), T = length of the line, [t_begin, t_end) = this CTA's share,
-// s_first = the sequence that holds position t_begin.
-template <bool FUSED, int THREADS>
-__device__ __forceinline__ void stream_plan(const int32_t* __restrict__ lens, float* __restrict__ o,
-                                            int32_t* __restrict__ status, int b, int h, int m_max, bool appending,
-                                            int* prefix, int* rows_of, int* s_first_sm, long long* T_out,
-                                            long long* t_begin_out, long long* t_end_out, int* s_first_out) {
+// (kAppendBit set when this step appends one).  Returns T = length of the line, [t_begin, t_end) = this
+// CTA's share, s_first = the sequence that holds position t_begin.  plan_sm: 4 ints of shared memory.
+struct SharePlan { int T, t_begin, t_end, s_first; };
+
+template <bool FUSED, int THREADS, int PENALTY>
+__device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ lens, float* __restrict__ o,
+                                                 int32_t* __restrict__ status, int b, int h, int m_max, bool appending,
+                                                 unsigned long long magic, int* prefix, int* rows_of, int* plan_sm) {
     const int cta = blockIdx.x, G = gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int s = threadIdx.x; s < b; s += THREADS) {
@@ -602,18 +599,18 @@ __device__ __forceinline__ void stream_plan(const int32_t* __restrict__ lens, fl
         const int L = fused_rows(raw, m_max, appending, &can_append);
         if (appending && !can_append && cta == 0 && status)
             atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
-        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + kBoundaryPenalty : 0;
+        prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + PENALTY : 0;
         rows_of[s] = L | (appending && can_append ? kAppendBit : 0);
         if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
             for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
         }
     }
-    if (threadIdx.x == 0) { prefix[0] = 0; *s_first_sm = 0; }
+    if (threadIdx.x == 0) { prefix[0] = 0; plan_sm[3] = 0; }
     __syncthreads();
     if (warp == 0) {
         // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
         // also notes which sequence that is
-        const int per = (b + 31) / 32;
+        const int per = (b + 31) >> 5;
         const int lo = 1 + lane * per, hi = min(b, lo + per - 1);
         int sum = 0;
         for (int s = lo; s <= hi; ++s) sum += prefix[s];
@@ -623,20 +620,78 @@ __device__ __forceinline__ void stream_plan(const int32_t* __restrict__ lens, fl
             const int up = __shfl_up_sync(0xffffffffu, incl, d);
             if (lane >= d) incl += up;
         }
-        long long tb, te;
-        share_bounds(cta, __shfl_sync(0xffffffffu, incl, 31), G, &tb, &te);
+        const int T = __shfl_sync(0xffffffffu, incl, 31);
+        const int tb = share_begin(cta, T, magic), te = share_begin(cta + 1, T, magic);
+        if (lane == 0) { plan_sm[0] = T; plan_sm[1] = tb; plan_sm[2] = te; }
         int run = incl - sum;
         for (int s = lo; s <= hi; ++s) {
             const int before = run;
             run += prefix[s];
             prefix[s] = run;
-            if (before <= tb && tb < run) *s_first_sm = s - 1;     // sequence s-1 occupies [before, run)
+            if (before <= tb && tb < run) plan_sm[3] = s - 1;     // sequence s-1 occupies [before, run)
         }
     }
     __syncthreads();
-    *T_out = prefix[b];
-    share_bounds(cta, *T_out, G, t_begin_out, t_end_out);
-    *s_first_out = *s_first_sm;                            // the s with prefix[s] <= t_begin < prefix[s+1]
+    SharePlan p;
+    p.T = plan_sm[0]; p.t_begin = plan_sm[1]; p.t_end = plan_sm[2]; p.s_first = plan_sm[3];
+    return p;
+}
+
+// The producer warp's short cut to its first copies (all 32 lanes call this): for up to kFastSeqs sequences
+// the warp reads lens itself, scans the tile counts in registers and finds the first segment of this
+// CTA's share, so that the first copies start one L2 round trip after the wait for the kernel before,
+// while the other warps build the shared tables (stream_plan, which gives the same segment again).
+// Returns false when there is nothing to start early (more sequences, an empty share, or a share that
+// begins between two sequences); *rows = rows_of[] entry of the segment's sequence.
+constexpr int kFastSeqs = 256;
+template <bool FUSED, int PENALTY>
+__device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, int b, int m_max, bool appending,
+                                              unsigned long long magic, Segment* g, int* rows) {
+    if (b > kFastSeqs) return false;
+    const int cta = blockIdx.x, lane = threadIdx.x & 31;
+    const int per = (b + 31) >> 5, base = lane * per;
+    int tl[kFastSeqs / 32], rw[kFastSeqs / 32];
+    int sum = 0;
+#pragma unroll
+    for (int i = 0; i < kFastSeqs / 32; ++i) {
+        tl[i] = 0; rw[i] = 0;
+        if (i < per && base + i < b) {
+            bool can_append;
+            const int L = fused_rows(read_len<FUSED>(lens, base + i), m_max, appending, &can_append);
+            tl[i] = L > 0 ? (L + kTileRows - 1) / kTileRows + PENALTY : 0;
+            rw[i] = L | (appending && can_append ? kAppendBit : 0);
+        }
+        sum += tl[i];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+    }
+    const int T = __shfl_sync(0xffffffffu, incl, 31);
+    const int tb = share_begin(cta, T, magic), te = share_begin(cta + 1, T, magic);
+    int run = incl - sum, fs = -1, v0 = 0, v1 = 0, fr = 0;
+#pragma unroll
+    for (int i = 0; i < kFastSeqs / 32; ++i) {
+        const int before = run;
+        run += tl[i];
+        if (before <= tb && tb < run) { fs = base + i; v0 = before; v1 = run; fr = rw[i]; }
+    }
+    const unsigned found = __ballot_sync(0xffffffffu, fs >= 0);
+    if (tb >= te || found == 0) return false;
+    const int src = __ffs(found) - 1;
+    fs = __shfl_sync(0xffffffffu, fs, src); v0 = __shfl_sync(0xffffffffu, v0, src);
+    v1 = __shfl_sync(0xffffffffu, v1, src); fr = __shfl_sync(0xffffffffu, fr, src);
+    const int n = v1 - v0 - PENALTY;
+    const int end = v1 < te ? v1 : te;
+    const int lo = tb - v0 - PENALTY, hi = end - v0 - PENALTY;
+    g->s = fs;
+    g->lo = lo > 0 ? lo : 0;
+    g->hi = hi < n ? hi : n;
+    g->whole = g->lo == 0 && g->hi == n;
+    *rows = fr;
+    return g->hi > g->lo;
 }
 
 template <int M_TILES, bool FUSED>
@@ -646,7 +701,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
                              const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                              float* __restrict__ o, int2* __restrict__ seq_span, float2* __restrict__ part_ml,
                              float* __restrict__ part_acc, int32_t* __restrict__ status, int b, int h, int m_max,
-                             const FusedArgs fa) {
+                             unsigned long long magic, const FusedArgs fa) {
     using Cfg = StreamCfg<M_TILES>;
     const bool appending = FUSED && fa.k_new != nullptr;
     constexpr int kStages = Cfg::kStages;
@@ -662,7 +717,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + Cfg::kPrefixBytes / 8 * 8);
     const uint32_t stages_s = smem_addr(stages);
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
-    __shared__ int timed_out, issued, s_first_sm;
+    __shared__ int timed_out, issued, plan_sm[4];
 
     if (warp == Cfg::kConsumerWarps && lane == 0) {
         prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
@@ -681,10 +736,9 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
 
-    long long T, t_begin, t_end;
-    int s_first;
-    stream_plan<FUSED, Cfg::kThreads>(lens, o, status, b, h, m_max, appending, prefix, rows_of, &s_first_sm, &T, &t_begin,
-                                      &t_end, &s_first);
+    const SharePlan plan = stream_plan<FUSED, Cfg::kThreads, kBoundaryPenalty>(lens, o, status, b, h, m_max, appending, magic, prefix,
+                                                             rows_of, plan_sm);
+    const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
 
     const int mt = warp % M_TILES;
     const int rw = warp / M_TILES;
@@ -696,7 +750,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         if (t_begin < t_end && lane == 0) {
             bool ok = true;
             int j = 0;                                     // stages issued by this CTA so far
-            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            ShareWalker<kBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             while (ok && walk.next(g)) {
                 const int s = g.s;
@@ -760,7 +814,7 @@ mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __
         float* my_buf = merge_buf + mt * Cfg::kStateFloats * 32;
         bool ok = true;
         int j = 0;                                         // stages consumed by this CTA so far
-        ShareWalker walk{prefix, t_begin, t_end, s_first};
+        ShareWalker<kBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
         Segment g_;
         while (walk.next(g_)) {
             const int s = g_.s;

@@ -37,9 +37,12 @@ namespace mqa {
 constexpr int kUmmaStageRows = 128;                              // cache rows per stage
 constexpr int kUmmaHalfBytes = kUmmaStageRows * 128;             // 16 KiB: one 64-column box of 128 rows
 constexpr int kUmmaSlotBytes = 2 * kUmmaHalfBytes;               // 32 KiB: the K (or the V) rows of a stage
-constexpr int kUmmaSoftmaxWarps = 4;
-constexpr int kUmmaProducerWarp = 4, kUmmaSWarp = 5, kUmmaPvWarp = 6;
-constexpr int kUmmaThreads = 7 * 32;
+constexpr int kUmmaSoftmaxWarps = 8;                             // warp w: TMEM lanes 32 * (w % 4) .., heads of half w / 4
+constexpr int kUmmaSoftmaxThreads = kUmmaSoftmaxWarps * 32;
+constexpr int kUmmaProducerWarp = 8, kUmmaSWarp = 9, kUmmaPvWarp = 10;
+constexpr int kUmmaThreads = 11 * 32;
+// virtual tiles in front of each sequence on the line (see kBoundaryPenalty): what a crossing costs this kernel
+constexpr int kUmmaBoundaryPenalty = 12;
 constexpr float kMaxLead = 16.f;                                 // log2 units a logit may exceed the reference maximum by
 
 template <int HP>
@@ -53,14 +56,16 @@ struct UmmaCfg {
     static constexpr int kPBytes = kUmmaStageRows * 128;
     static constexpr int kPTiles = 2;
     static constexpr int kQBufs = HP <= 32 ? 2 : 1;             // 64 head rows: one Q buffer (shared memory)
-    static constexpr int kChunk = HP < 32 ? HP : 32;             // heads handled per TMEM load
-    static constexpr int kRedBytes = (2 * kUmmaSoftmaxWarps + 2) * HP * 4;   // per-warp maxima and sums, reference maxima, factors
+    static constexpr int kHeadsPerThread = HP / 2;               // a cache row's heads are split over two warps
+    static constexpr int kChunk = kHeadsPerThread < 32 ? kHeadsPerThread : 32;   // heads handled per TMEM load
+    // per-quarter maxima and sums [4][HP] each, reference maxima, factors of the last move, 1/sum of two segments
+    static constexpr int kRedBytes = (2 * 4 + 4) * HP * 4;
     static constexpr int kPlanBytes = (2 * kStreamMaxSeqs + 1) * 4 + 12;   // line positions + rows per sequence
-    static constexpr int kBarriers = 2 * kKSlots + 2 * kVSlots + 13;
+    static constexpr int kBarriers = 2 * kKSlots + 2 * kVSlots + 14;
     static constexpr int kSmemBytes = (kKSlots + kVSlots) * kUmmaSlotBytes + kQBufs * kQBytes + kPTiles * kPBytes + kRedBytes +
                                       kPlanBytes + kBarriers * 8 + 1024 /* alignment slack */;
     static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
-    static constexpr int kTmemCols = 3 * HP <= 64 ? 64 : (3 * HP <= 128 ? 128 : 256);   // S^T twice, O^T once
+    static constexpr int kTmemCols = 4 * HP;                     // S^T twice, O^T twice (64, 128 or 256 columns)
 };
 
 // ---- tcgen05 wrappers ----------------------------------------------------------------------
@@ -130,10 +135,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
 }
-// COLS (16, 32 or 64) consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+// COLS (8, 16, 32 or 64) consecutive fp32 columns of this thread's TMEM lane
 template <int COLS>
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[COLS]) {
-    if constexpr (COLS == 16) {
+    if constexpr (COLS == 8) {
+        tmem_ld8(taddr, r);
+    } else if constexpr (COLS == 16) {
         tmem_ld16(taddr, r);
     } else {
 #pragma unroll
@@ -175,7 +187,7 @@ __device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred)
     return out != 0;
 }
 
-// Reduces N (16 or 32) values per lane over the 32 lanes of a warp, all at once: afterwards lane l holds
+// Reduces N (8, 16 or 32) values per lane over the 32 lanes of a warp, all at once: afterwards lane l holds
 // the total (sum, or maximum) of value number l % N.  v is used up.
 template <int N, bool MAX>
 __device__ __forceinline__ float warp_reduce_scatter(float (&v)[N], int lane) {
@@ -190,8 +202,9 @@ __device__ __forceinline__ float warp_reduce_scatter(float (&v)[N], int lane) {
             v[i] = MAX ? fmaxf(keep, got) : keep + got;
         }
     }
-    if (N == 16) {
-        const float got = __shfl_xor_sync(0xffffffffu, v[0], 16);
+#pragma unroll
+    for (int d = N; d < 32; d <<= 1) {
+        const float got = __shfl_xor_sync(0xffffffffu, v[0], d);
         v[0] = MAX ? fmaxf(v[0], got) : v[0] + got;
     }
     return v[0];
@@ -205,9 +218,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               const __grid_constant__ CUtensorMap map_q,
                               const int32_t* __restrict__ lens, float* __restrict__ o, int2* __restrict__ seq_span,
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
-                              int b, int h, int m_max, const FusedArgs fa) {
+                              int b, int h, int m_max, unsigned long long magic, const FusedArgs fa) {
     using Cfg = UmmaCfg<HP>;
-    constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = HP / CH;
+    constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
     const bool appending = FUSED && fa.k_new != nullptr;
     const int cta = blockIdx.x, G = gridDim.x;
@@ -217,11 +230,12 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     uint8_t* ring = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);   // K slots, then V slots
     uint8_t* q_buf = ring + (NK + NV) * kUmmaSlotBytes;                 // 2 x Q
     uint8_t* p_buf = q_buf + Cfg::kQBufs * Cfg::kQBytes;                // P^T tiles
-    float* red_m = reinterpret_cast<float*>(p_buf + Cfg::kPTiles * Cfg::kPBytes);   // [4 warps][HP]
-    float* red_l = red_m + kUmmaSoftmaxWarps * HP;                                  // [4 warps][HP]
-    float* m_sm = red_l + kUmmaSoftmaxWarps * HP;                                   // [HP] reference maxima (log2 units) of the segment
+    float* red_m = reinterpret_cast<float*>(p_buf + Cfg::kPTiles * Cfg::kPBytes);   // [4 lane quarters][HP]
+    float* red_l = red_m + 4 * HP;                                                  // [4 lane quarters][HP]
+    float* m_sm = red_l + 4 * HP;                                   // [HP] reference maxima (log2 units) of the segment
     float* f_sm = m_sm + HP;                                                        // [HP] factor of the last move
-    int* prefix = reinterpret_cast<int*>(f_sm + HP);                                // [b + 1]
+    float* inv_sm = f_sm + HP;                                                      // [2][HP] 1 / sum of weights (1 for a partial), by segment parity
+    int* prefix = reinterpret_cast<int*>(inv_sm + 2 * HP);                          // [b + 1]
     int* rows_of = prefix + kStreamMaxSeqs + 1;                                     // [b]
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + (Cfg::kPlanBytes + 7) / 8 * 8);
     const uint32_t k_ring = smem_addr(ring), v_ring = k_ring + NK * kUmmaSlotBytes;
@@ -231,8 +245,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     const uint32_t v_full = k_empty + NK * 8, v_empty = v_full + NV * 8;
     const uint32_t q_full = v_empty + NV * 8, q_empty = q_full + 16;
     const uint32_t s_ready = q_empty + 16, s_free = s_ready + 16;
-    const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;
-    __shared__ int timed_out, issued, s_first_sm;
+    const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;   // o_free: one per O^T buffer
+    __shared__ int timed_out, issued, plan_sm[4];
     __shared__ uint32_t tmem_base_slot;
 
     if (warp == kUmmaProducerWarp && lane == 0) {
@@ -248,8 +262,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             mbar_init(q_full + s * 8, 1); mbar_init(q_empty + s * 8, 1);
             mbar_init(s_ready + s * 8, 1); mbar_init(s_free + s * 8, kUmmaSoftmaxWarps);
             mbar_init(p_ready + s * 8, kUmmaSoftmaxWarps); mbar_init(pv_done + s * 8, 1);
+            mbar_init(o_free + s * 8, kUmmaSoftmaxWarps);
         }
-        mbar_init(o_free, kUmmaSoftmaxWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -257,74 +271,95 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         tmem_alloc(smem_addr(&tmem_base_slot), Cfg::kTmemCols);
         tmem_relinquish();
     }
+    // ---- what the producer thread does for a segment and for a stage
+    bool p_ok = true;                                       // no producer wait has run out
+    auto issue_q = [&](int s, int seg) {
+        const int qi = seg % NQ;
+        if (seg >= NQ) p_ok = p_ok && mbar_wait(q_empty + qi * 8, ((seg / NQ) - 1) & 1);
+        if (!p_ok) return;
+        // the sequence's head rows (rows past h belong to the next sequence or read as zero: their
+        // columns of S^T and O^T are never stored)
+        mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
+        tma_load_2d(q_s + qi * Cfg::kQBytes, &map_q, 0, s * h, q_full + qi * 8);
+        tma_load_2d(q_s + qi * Cfg::kQBytes + Cfg::kQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
+    };
+    auto issue_stage = [&](int s, int u, int hi, int j, int rows_entry) {
+        const int nsub = min(kSubs, hi - u);
+        const int row_first = u * kTileRows;
+        const int new_row = (rows_entry & kAppendBit) ? (rows_entry & (kAppendBit - 1)) - 1 : -1;   // row this step appends
+        if (appending && new_row >= row_first && new_row < row_first + nsub * kTileRows) {
+            const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16);
+            const size_t src = (size_t)s * (kRowBytes / 16);
+#pragma unroll 1
+            for (int i = 0; i < 16; i += 4) {
+                uint4 kr[4], vr[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { kr[e] = fa.k_new[src + i + e]; vr[e] = fa.v_new[src + i + e]; }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { fa.K[dst + i + e] = kr[e]; fa.V[dst + i + e] = vr[e]; }
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
+        }
+        const int y = s * m_max + row_first;
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {                    // the K rows, then the V rows, each into its own ring
+            const int n_slots = kv ? NV : NK;
+            const int slot = j % n_slots;
+            const uint32_t full = (kv ? v_full : k_full) + slot * 8;
+            if (j >= n_slots) p_ok = p_ok && mbar_wait((kv ? v_empty : k_empty) + slot * 8, ((j / n_slots) - 1) & 1);
+            if (!p_ok) return;
+            const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes;
+            mbar_expect_tx(full, nsub * 2 * kBoxBytes);
+            if (nsub == kSubs) {
+                tma_load_2d(dst, kv ? &map_v : &map_k, 0, y, full);
+                tma_load_2d(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full);
+            } else {
+                for (int i = 0; i < nsub; ++i) {
+                    const uint32_t d = dst + i * kBoxBytes;
+                    tma_load_2d(d, kv ? &map_v_sub : &map_k_sub, 0, y + i * kTileRows, full);
+                    tma_load_2d(d + kUmmaHalfBytes, kv ? &map_v_sub : &map_k_sub, kBoxCols, y + i * kTileRows, full);
+                }
+            }
+            issued = 2 * j + kv + 1;                        // copies started: K of stage j, then V of stage j
+        }
+    };
+
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
 
+    // the producer warp starts its first stages (at most what the rings hold without a wait) before the tables exist
+    int pre_issued = 0;
+    if (warp == kUmmaProducerWarp) {
+        Segment g0;
+        int r0;
+        if (first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g0, &r0) && lane == 0) {
+            issue_q(g0.s, 0);
+            for (int u = g0.lo; u < g0.hi && pre_issued < (NK < NV ? NK : NV); u += kSubs, ++pre_issued)
+                issue_stage(g0.s, u, g0.hi, pre_issued, r0);
+        }
+    }
+
     tc_fence_before();
-    long long T, t_begin, t_end;
-    int s_first;
-    stream_plan<FUSED, kUmmaThreads>(lens, o, status, b, h, m_max, appending, prefix, rows_of, &s_first_sm, &T, &t_begin,
-                                     &t_end, &s_first);
+    const SharePlan plan = stream_plan<FUSED, kUmmaThreads, kUmmaBoundaryPenalty>(lens, o, status, b, h, m_max, appending, magic, prefix,
+                                                            rows_of, plan_sm);
+    const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    const uint32_t tmem_o = tmem_base + 2 * HP;             // S^T buffers at columns 0 and HP, O^T after them
+    const uint32_t tmem_o = tmem_base + 2 * HP;             // S^T buffers at columns 0 and HP, two O^T buffers after them
 
     if (warp == kUmmaProducerWarp) {
         // =============================================================== TMA producer
         if (lane == 0 && t_begin < t_end) {
-            bool ok = true;
             int j = 0, seg = 0;
-            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
-            for (; ok && walk.next(g); ++seg) {
-                const int s = g.s;
-                const int qi = seg % NQ;
-                if (seg >= NQ) ok = mbar_wait(q_empty + qi * 8, ((seg / NQ) - 1) & 1);
-                if (!ok) break;
-                // the sequence's head rows (rows past h belong to the next sequence or read as zero: their
-                // columns of S^T and O^T are never stored)
-                mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
-                tma_load_2d(q_s + qi * Cfg::kQBytes, &map_q, 0, s * h, q_full + qi * 8);
-                tma_load_2d(q_s + qi * Cfg::kQBytes + Cfg::kQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
-                const int new_row = (rows_of[s] & kAppendBit) ? (rows_of[s] & (kAppendBit - 1)) - 1 : -1;   // row this step appends
-                for (int u = g.lo; u < g.hi && ok; u += kSubs, ++j) {
-                    const int nsub = min(kSubs, g.hi - u);
-                    const int row_first = u * kTileRows;
-                    if (appending && new_row >= row_first && new_row < row_first + nsub * kTileRows) {
-                        const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16);
-                        const size_t src = (size_t)s * (kRowBytes / 16);
-                        uint4 kr[16], vr[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) { kr[i] = fa.k_new[src + i]; vr[i] = fa.v_new[src + i]; }
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) { fa.K[dst + i] = kr[i]; fa.V[dst + i] = vr[i]; }
-                        asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
-                    }
-                    const int y = s * m_max + row_first;
-#pragma unroll
-                    for (int kv = 0; kv < 2; ++kv) {        // the K rows, then the V rows, each into its own ring
-                        const int n_slots = kv ? NV : NK;
-                        const int slot = j % n_slots;
-                        const uint32_t full = (kv ? v_full : k_full) + slot * 8;
-                        if (j >= n_slots) ok = ok && mbar_wait((kv ? v_empty : k_empty) + slot * 8, ((j / n_slots) - 1) & 1);
-                        if (!ok) break;
-                        const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes;
-                        mbar_expect_tx(full, nsub * 2 * kBoxBytes);
-                        if (nsub == kSubs) {
-                            tma_load_2d(dst, kv ? &map_v : &map_k, 0, y, full);
-                            tma_load_2d(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full);
-                        } else {
-                            for (int i = 0; i < nsub; ++i) {
-                                const uint32_t d = dst + i * kBoxBytes;
-                                tma_load_2d(d, kv ? &map_v_sub : &map_k_sub, 0, y + i * kTileRows, full);
-                                tma_load_2d(d + kUmmaHalfBytes, kv ? &map_v_sub : &map_k_sub, kBoxCols, y + i * kTileRows, full);
-                            }
-                        }
-                        issued = 2 * j + kv + 1;            // copies started: K of stage j, then V of stage j
-                    }
-                }
+            for (; p_ok && walk.next(g); ++seg) {
+                if (!(seg == 0 && pre_issued > 0)) issue_q(g.s, seg);
+                const int rows_entry = rows_of[g.s];
+                for (int u = g.lo; u < g.hi && p_ok; u += kSubs, ++j)
+                    if (j >= pre_issued) issue_stage(g.s, u, g.hi, j, rows_entry);
             }
-            if (!ok) atomicExch(&timed_out, 1);
+            if (!p_ok) atomicExch(&timed_out, 1);
         }
     } else if (warp == kUmmaSWarp) {
         // =============================================================== issuer of S^T = K Q^T
@@ -332,7 +367,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             constexpr uint32_t kIdescS = umma_idesc(128, HP, false, false);
             bool ok = true;
             int j = 0, seg = 0;
-            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
                 const int qi = seg % NQ;
@@ -364,7 +399,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             constexpr uint32_t kIdescO = umma_idesc(128, HP, true, true);
             bool ok = true;
             int j = 0, seg = 0;
-            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
                 const int L = rows_of[g.s] & (kAppendBit - 1);
@@ -373,7 +408,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     const int pb = j & 1, slot = j % NV;
                     if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
                     if (ok) ok = mbar_wait(p_ready + pb * 8, (j >> 1) & 1);
-                    if (ok && u == g.lo && seg >= 1) ok = mbar_wait(o_free, (seg - 1) & 1);   // the segment before has read O^T out
+                    // segments alternate between the two O^T buffers; the segment before the last has read this one out
+                    if (ok && u == g.lo && seg >= 2) ok = mbar_wait(o_free + (seg & 1) * 8, ((seg >> 1) - 1) & 1);
                     tc_fence_after();
                     if (ok) {
                         const uint32_t v_s = v_ring + slot * kUmmaSlotBytes;
@@ -383,7 +419,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                             for (int kk = 0; kk < 8; ++kk) {         // 8 k-steps of 16 cache rows
                                 const uint64_t a = umma_desc(v_s + kk * 2048, kUmmaHalfBytes, 1024);
                                 const uint64_t bd = umma_desc(pt + kk * 2048, Cfg::kPBytes, 1024);
-                                umma_ss(tmem_o, a, bd, kIdescO, (u == g.lo && part == 0 && kk == 0) ? 0u : 1u);
+                                umma_ss(tmem_o + (seg & 1) * HP, a, bd, kIdescO, (u == g.lo && part == 0 && kk == 0) ? 0u : 1u);
                             }
                         }
                     }
@@ -397,30 +433,64 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // =============================================================== softmax warps
         if (warp == 0) {                                    // second-pass bookkeeping, spread over the CTAs
             for (int s = cta + lane * G; s < b; s += G * 32) {
-                const int t0 = prefix[s] + kBoundaryPenalty, t1 = prefix[s + 1];     // its real tiles on the line
+                const int t0 = prefix[s] + kUmmaBoundaryPenalty, t1 = prefix[s + 1];     // its real tiles on the line
                 seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
             }
             if (cta == 0 && lane == 0) seq_span[b] = make_int2((int)T, G);
         }
         if (t_begin < t_end) {
-            const int t = warp * 32 + lane;                 // this thread's cache row of every stage = its TMEM lane;
-                                                            // at the end of a segment, its column of O^T
-            const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+            constexpr int HH = Cfg::kHeadsPerThread;
+            const int quarter = warp & 3, half = warp >> 2;
+            const int t = quarter * 32 + lane;              // this thread's cache row of every stage = its TMEM lane;
+                                                            // when a segment is read out, its column of O^T
+            const int tid = warp * 32 + lane;               // 0 .. 255 among the softmax threads
+            const int head0 = half * HH;                    // this thread's heads: head0 .. head0 + HH - 1
+            const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
             // where this row's weights go in a P^T tile (128 cache rows x 128 bytes, 128-byte swizzle): the 16
             // bytes of heads 8c .. 8c+7 at row * 128 + ((c ^ (row & 7)) << 4)
             const uint32_t p_row = (uint32_t)(t * 128), p_xor = (uint32_t)((t & 7) << 4);
             bool ok = true;
             int j = 0, seg = 0;
-            ShareWalker walk{prefix, t_begin, t_end, s_first};
+            // a finished segment whose O^T has not been read out of TMEM yet (done after the next segment's first stage)
+            bool pend = false;
+            bool prev_hilo = false;                         // the stage before wrote hi and lo parts of P
+            float* pend_dst = nullptr;
+            int pend_par = 0, pend_j = 0;
+            auto read_out = [&]() {
+                // O^T[column t][head] of the finished segment -> o (divided by the sum) or its partial slot
+                if (ok) ok = mbar_wait(pv_done + (pend_j & 1) * 8, (pend_j >> 1) & 1);   // the segment's last product
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    uint32_t y[CH];
+                    tmem_ld_cols<CH>(lane_base + 2 * HP + pend_par * HP + head0 + c * CH, y);
+                    float inv[CH];
+#pragma unroll
+                    for (int i = 0; i < CH; i += 4) {
+                        const float4 v4 = *reinterpret_cast<const float4*>(inv_sm + pend_par * HP + head0 + c * CH + i);
+                        inv[i] = v4.x; inv[i + 1] = v4.y; inv[i + 2] = v4.z; inv[i + 3] = v4.w;
+                    }
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < CH; ++i)
+                        if (head0 + c * CH + i < h) pend_dst[(size_t)(head0 + c * CH + i) * kHeadDim] = __uint_as_float(y[i]) * inv[i];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_free + pend_par * 8);   // this O^T buffer may be overwritten
+                pend = false;
+            };
+            ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
                 const int s = g.s;
                 const int L = rows_of[s] & (kAppendBit - 1);
                 const bool whole = g.whole;
                 const bool hilo = L < kSingleRoundingMinRows;    // long prefixes: one bf16 rounding of P is enough
-                float l_sum[HP];                            // this row's share of every head's sum of weights
+                const int par = seg & 1;                    // O^T buffer of this segment
+                float l_sum[HH];                            // this row's share of its heads' sums of weights
 #pragma unroll
-                for (int i = 0; i < HP; ++i) l_sum[i] = 0.f;
+                for (int i = 0; i < HH; ++i) l_sum[i] = 0.f;
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
                     const int sb = j & 1, pb = j & 1;
                     const bool first = u == g.lo;           // nothing accumulated yet: no reference maxima, O^T not started
@@ -431,11 +501,11 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     const bool row_ok = t < valid;
                     if (ok) ok = mbar_wait(s_ready + sb * 8, (j >> 1) & 1);
                     tc_fence_after();
-                    uint32_t xr[HP];
+                    uint32_t xr[HH];
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         uint32_t part[CH];
-                        tmem_ld_cols<CH>(lane_base + sb * HP + c * CH, part);
+                        tmem_ld_cols<CH>(lane_base + sb * HP + head0 + c * CH, part);
 #pragma unroll
                         for (int i = 0; i < CH; ++i) xr[c * CH + i] = part[i];
                     }
@@ -444,12 +514,12 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     __syncwarp();
                     if (lane == 0) mbar_arrive(s_free + sb * 8);             // S^T is in registers now
                     // ---- logits in log2 units, masked by index; how far the largest leads its reference
-                    float x[HP];
+                    float x[HH];
                     float lead = -INFINITY;
 #pragma unroll
-                    for (int i = 0; i < HP; i += 4) {
+                    for (int i = 0; i < HH; i += 4) {
                         const float4 m4 = first ? make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY)
-                                                : *reinterpret_cast<const float4*>(m_sm + i);
+                                                : *reinterpret_cast<const float4*>(m_sm + head0 + i);
                         const float mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
@@ -457,7 +527,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                             lead = fmaxf(lead, x[i + e] - mv[e]);           // (-inf) - (-inf) = NaN is ignored by fmaxf
                         }
                     }
-                    if (named_barrier_or(1, kUmmaSoftmaxWarps * 32, lead > kMaxLead)) {
+                    if (named_barrier_or(1, kUmmaSoftmaxThreads, lead > kMaxLead)) {
                         // ---- some logit leads by too much (always on a segment's first stage): every head's
                         // reference moves to the largest logit seen so far; sums and O^T are rescaled
 #pragma unroll
@@ -466,22 +536,22 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 #pragma unroll
                             for (int i = 0; i < CH; ++i) r[i] = x[c * CH + i];
                             const float top = warp_reduce_scatter<CH, true>(r, lane);
-                            if (lane < CH) red_m[warp * HP + c * CH + lane] = top;
+                            if (lane < CH) red_m[quarter * HP + head0 + c * CH + lane] = top;
                         }
-                        named_barrier(2, kUmmaSoftmaxWarps * 32);
-                        if (t < HP) {
-                            const float m_old = first ? -INFINITY : m_sm[t];
+                        named_barrier(2, kUmmaSoftmaxThreads);
+                        if (tid < HP) {
+                            const float m_old = first ? -INFINITY : m_sm[tid];
                             float m_new = m_old;
 #pragma unroll
-                            for (int w = 0; w < kUmmaSoftmaxWarps; ++w) m_new = fmaxf(m_new, red_m[w * HP + t]);   // finite: the stage has a valid row
-                            f_sm[t] = fast_exp2(m_old - m_new);              // 0 on the first stage, 1 if unchanged
-                            m_sm[t] = m_new;
+                            for (int w = 0; w < 4; ++w) m_new = fmaxf(m_new, red_m[w * HP + tid]);   // finite: the stage has a valid row
+                            f_sm[tid] = fast_exp2(m_old - m_new);            // 0 on the first stage, 1 if unchanged
+                            m_sm[tid] = m_new;
                         }
-                        named_barrier(2, kUmmaSoftmaxWarps * 32);
+                        named_barrier(2, kUmmaSoftmaxThreads);
                         if (!first) {
 #pragma unroll
-                            for (int i = 0; i < HP; i += 4) {
-                                const float4 f4 = *reinterpret_cast<const float4*>(f_sm + i);
+                            for (int i = 0; i < HH; i += 4) {
+                                const float4 f4 = *reinterpret_cast<const float4*>(f_sm + head0 + i);
                                 l_sum[i] *= f4.x; l_sum[i + 1] *= f4.y; l_sum[i + 2] *= f4.z; l_sum[i + 3] *= f4.w;
                             }
                             // O^T holds the stages before this one: wait for the last of their products, scale
@@ -491,32 +561,34 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 #pragma unroll
                             for (int c = 0; c < NCH; ++c) {
                                 uint32_t y[CH];
-                                tmem_ld_cols<CH>(lane_base + 2 * HP + c * CH, y);
+                                const uint32_t at = lane_base + 2 * HP + par * HP + head0 + c * CH;
+                                tmem_ld_cols<CH>(at, y);
                                 tmem_wait_ld();
 #pragma unroll
                                 for (int i = 0; i < CH; i += 4) {
-                                    const float4 f4 = *reinterpret_cast<const float4*>(f_sm + c * CH + i);
+                                    const float4 f4 = *reinterpret_cast<const float4*>(f_sm + head0 + c * CH + i);
                                     y[i] = __float_as_uint(__uint_as_float(y[i]) * f4.x);
                                     y[i + 1] = __float_as_uint(__uint_as_float(y[i + 1]) * f4.y);
                                     y[i + 2] = __float_as_uint(__uint_as_float(y[i + 2]) * f4.z);
                                     y[i + 3] = __float_as_uint(__uint_as_float(y[i + 3]) * f4.w);
                                 }
-                                tmem_st_words<CH>(lane_base + 2 * HP + c * CH, y);
+                                tmem_st_words<CH>(at, y);
                             }
                             tmem_wait_st();
                             tc_fence_before();
                         }
                     }
-                    // this P^T tile was last read by the product of stage j-2 (of stage j-1 when hi and lo take
-                    // both tiles)
+                    // this P^T tile was last read by the product of stage j-2 (of stage j-1 when that stage or
+                    // this one has hi and lo parts, which take both tiles)
                     if (j >= 2 && ok) ok = mbar_wait(pv_done + pb * 8, ((j >> 1) - 1) & 1);
-                    if (hilo && j >= 1 && ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
+                    if ((hilo || prev_hilo) && j >= 1 && ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
+                    prev_hilo = hilo;
                     // ---- P = exp2(S - reference): 0 for a masked row; bf16 hi (and lo) into the P^T tiles
                     const uint32_t p_hi = p_s + (hilo ? 0 : pb) * Cfg::kPBytes + p_row, p_lo = p_s + Cfg::kPBytes + p_row;
 #pragma unroll
-                    for (int c = 0; c < HP / 8; ++c) {
-                        const float4 ma = *reinterpret_cast<const float4*>(m_sm + c * 8);
-                        const float4 mb = *reinterpret_cast<const float4*>(m_sm + c * 8 + 4);
+                    for (int c = 0; c < HH / 8; ++c) {
+                        const float4 ma = *reinterpret_cast<const float4*>(m_sm + head0 + c * 8);
+                        const float4 mb = *reinterpret_cast<const float4*>(m_sm + head0 + c * 8 + 4);
                         const float mv[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
                         float pw[8];
 #pragma unroll
@@ -527,7 +599,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         uint32_t hi[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) hi[e] = pack_bf16(pw[2 * e], pw[2 * e + 1]);
-                        const uint32_t at = ((uint32_t)(c << 4)) ^ p_xor;
+                        const uint32_t at = ((uint32_t)((half * (HH / 8) + c) << 4)) ^ p_xor;
                         asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(p_hi + at), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]));
                         if (hilo) {
                             uint32_t lo[4];
@@ -543,7 +615,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         const int slot = j % NV;
                         if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
                         const uint32_t v_s = v_ring + slot * kUmmaSlotBytes;
-                        for (int i = t; i < (kUmmaStageRows - valid) * 16; i += kUmmaSoftmaxWarps * 32) {
+                        for (int i = tid; i < (kUmmaStageRows - valid) * 16; i += kUmmaSoftmaxThreads) {
                             const int vrow = valid + (i >> 4), ch = i & 15;  // 16 chunks of 16 bytes per row
                             const uint32_t a = v_s + (ch >> 3) * kUmmaHalfBytes + vrow * 128 + ((ch & 7) << 4);
                             asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
@@ -552,51 +624,37 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P^T (and cleared V) visible to the tensor core
                     __syncwarp();
                     if (lane == 0) mbar_arrive(p_ready + pb * 8);
+                    // the segment before this one is read out of its own O^T buffer now, after this
+                    // segment's first stage is on its way (its last product has long finished)
+                    if (pend) read_out();
                 }
-                // ---- segment done: add up the rows' sums, wait for the last product, read O^T out of TMEM
+                // ---- segment done: add up the rows' sums; thread i < HP keeps head i's 1/sum for the read-out
+                // and writes (maximum, sum) of a partial result.  O^T itself is read out later (see above).
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     float r[CH];
 #pragma unroll
                     for (int i = 0; i < CH; ++i) r[i] = l_sum[c * CH + i];
                     const float tot = warp_reduce_scatter<CH, false>(r, lane);
-                    if (lane < CH) red_l[warp * HP + c * CH + lane] = tot;
+                    if (lane < CH) red_l[quarter * HP + head0 + c * CH + lane] = tot;
                 }
-                named_barrier(2, kUmmaSoftmaxWarps * 32);
-                if (ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
-                tc_fence_after();
+                named_barrier(2, kUmmaSoftmaxThreads);
                 const size_t slot = (size_t)cta + s;
-                float* dst = (whole ? o + (size_t)s * h * kHeadDim : part_acc + slot * h * kHeadDim) + t;
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    uint32_t y[CH];
-                    tmem_ld_cols<CH>(lane_base + 2 * HP + c * CH, y);
-                    float inv[CH];
-#pragma unroll
-                    for (int i = 0; i < CH; i += 4) {
-                        float4 tot = *reinterpret_cast<const float4*>(red_l + c * CH + i);
-#pragma unroll
-                        for (int w = 1; w < kUmmaSoftmaxWarps; ++w) {
-                            const float4 o4 = *reinterpret_cast<const float4*>(red_l + w * HP + c * CH + i);
-                            tot.x += o4.x; tot.y += o4.y; tot.z += o4.z; tot.w += o4.w;
-                        }
-                        inv[i] = whole ? 1.f / tot.x : 1.f; inv[i + 1] = whole ? 1.f / tot.y : 1.f;
-                        inv[i + 2] = whole ? 1.f / tot.z : 1.f; inv[i + 3] = whole ? 1.f / tot.w : 1.f;
-                    }
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < CH; ++i)
-                        if (c * CH + i < h) dst[(size_t)(c * CH + i) * kHeadDim] = __uint_as_float(y[i]) * inv[i];
-                }
-                if (!whole && t < h) {
+                if (tid < HP) {
                     float tot = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kUmmaSoftmaxWarps; ++w) tot += red_l[w * HP + t];
-                    part_ml[slot * h + t] = make_float2(m_sm[t], tot);
+                    for (int w = 0; w < 4; ++w) tot += red_l[w * HP + tid];
+                    inv_sm[par * HP + tid] = whole ? 1.f / tot : 1.f;
+                    if (!whole && tid < h) part_ml[slot * h + tid] = make_float2(m_sm[tid], tot);
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);         // the next segment may overwrite O^T
+                pend = true;
+                pend_dst = (whole ? o + (size_t)s * h * kHeadDim : part_acc + slot * h * kHeadDim) + t;
+                pend_par = par;
+                pend_j = j - 1;
+            }
+            if (pend) {
+                named_barrier(2, kUmmaSoftmaxThreads);      // the last segment's 1/sum values are in shared memory
+                read_out();
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
