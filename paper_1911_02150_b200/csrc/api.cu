@@ -136,7 +136,7 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
 size_t plan_workspace_bytes(const Plan& p) {
     if (p.stream()) {
         const int slots = p.grid + p.b;
-        return stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) + stream_acc_bytes(slots, p.h);
+        return stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) + stream_acc_bytes(slots, p.h) + stream_ctrl_bytes(p.b);
     }
     if (p.n_splits <= 1) return 0;
     return partial_ml_bytes(p.units, p.n_splits) + partial_acc_bytes(p.units, p.n_splits);
@@ -146,6 +146,7 @@ struct StreamWorkspace {
     int2* span;
     float2* ml;
     float* acc;
+    unsigned long long* ctrl;     // control block of the single-launch step (tcgen05 kernel)
 };
 StreamWorkspace stream_workspace(const Plan& p, const void* workspace) {
     char* base = static_cast<char*>(const_cast<void*>(workspace));
@@ -154,6 +155,8 @@ StreamWorkspace stream_workspace(const Plan& p, const void* workspace) {
     w.span = reinterpret_cast<int2*>(base);
     w.ml = reinterpret_cast<float2*>(base + stream_span_bytes(p.b));
     w.acc = reinterpret_cast<float*>(base + stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h));
+    w.ctrl = reinterpret_cast<unsigned long long*>(base + stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) +
+                                                   stream_acc_bytes(slots, p.h));
     return w;
 }
 
@@ -299,8 +302,8 @@ std::atomic<int> g_umma_opt_in[kMaxDevices][6];
 
 template <int HP, bool FUSED>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-                void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream,
-                const void* k_new = nullptr, const void* v_new = nullptr) {
+                void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
+                const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
     using Cfg = UmmaCfg<HP>;
     auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED>;
     constexpr int kSlot = (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 2 + (FUSED ? 1 : 0);
@@ -328,31 +331,35 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa);
+                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa,
+                     merge ? w.ctrl : nullptr, lens_advance);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
 template <bool FUSED>
 int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-                    void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream,
-                    const void* k_new = nullptr, const void* v_new = nullptr) {
-    if (h <= 16) return launch_umma<16, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
-    if (h <= 32) return launch_umma<32, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
-    return launch_umma<64, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
+                    void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
+                    const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
+    if (h <= 16)
+        return launch_umma<16, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance);
+    if (h <= 32)
+        return launch_umma<32, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance);
+    return launch_umma<64, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance);
 }
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
 
 int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
               void* workspace, size_t workspace_bytes, int32_t* status,
-              int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0) {
+              int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0, bool merge_in_kernel = false) {
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
     const Plan p = make_plan(multi_query, b, h, m_max);
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
-    if (p.kernel == Kernel::kUmma) return launch_umma_for<false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
+    if (p.kernel == Kernel::kUmma)
+        return launch_umma_for<false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge_in_kernel);
     if (p.kernel == Kernel::kStream1)
         return launch_stream<1, false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     if (p.kernel == Kernel::kStream2)
@@ -407,8 +414,11 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
 int run_step(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
              void* workspace, size_t workspace_bytes, int32_t* status,
              int b, int h, int m_max, int k, int v, cudaStream_t stream) {
-    int rc = run_split(multi_query, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream);
-    if (rc) return rc;
+    // the tcgen05 plan is a single launch: the CTA that delivers the last piece of a sequence merges the pieces
+    const bool one_launch = make_plan(multi_query, b, h, m_max).kernel == Kernel::kUmma;
+    int rc = run_split(multi_query, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream, 0,
+                       one_launch);
+    if (rc || one_launch) return rc;
     return run_combine(multi_query, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream);
 }
 
@@ -500,9 +510,9 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
     }
     if (p.kernel == Kernel::kUmma) {
-        rc = launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
-        if (rc) return rc;
-        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
+        // one launch: append inside the pass, pieces merged by the last CTA to deliver one, lens advanced at the end
+        return launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, true, k_new, v_new,
+                                     advance ? lens : nullptr);
     }
     // other plans: the same step as separate launches.  Without `advance` the append leaves lens alone and
     // the step is told that a sequence which took a row has one more row than lens says.
@@ -529,6 +539,7 @@ size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v) {
 int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
     const Plan p = make_plan(true, b, h, m_max);
+    if (p.kernel == Kernel::kUmma) return 1;           // append, pass, merge and lens advance in one kernel
     if (p.stream()) return 2;                          // pass with the append inside, second pass
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }

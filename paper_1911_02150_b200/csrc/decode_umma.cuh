@@ -175,6 +175,41 @@ __host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool a_mn_major,
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// ---- control block of the single-launch step ---------------------------------------------------
+// When a control block is given, the CTA that is last to deliver a piece of a sequence merges the pieces
+// itself (no second-pass kernel), and one CTA advances lens at the end.  The block lives in the caller's
+// workspace, whose contents are arbitrary the first time, and nothing in it is ever reset: every launch
+// works under a new epoch E, read from the block by every CTA before anything in it is written, and a
+// word counts only if it carries E.
+//   ctrl[0] magic (the block has been used before), ctrl[1] epoch of the last launch
+//   ctrl[8 + c]        = E once CTA c has read the epoch and lens      ("started")
+//   ctrl[8 + 256 + s]  = E << 20 | pieces of sequence s delivered so far
+// The epoch is moved on by the first CTA that finds every CTA started (at least the CTA that started
+// last does: the store of its own mark, a fence.sc and then the reads).  Until then nobody leaves
+// the old epoch behind, so all CTAs of a launch agree on E.
+constexpr unsigned long long kCtrlMagic = 0x6d71615f6374726cull;
+constexpr unsigned long long kCtrlFirstEpoch = 0x9e3779b97f4ull;          // 44 bits
+constexpr unsigned long long kCtrlEpochMask = (1ull << 44) - 1;
+constexpr int kCtrlCountBits = 20;
+constexpr int kCtrlStarted = 8, kCtrlCounters = 8 + 256;
+__host__ __device__ inline size_t stream_ctrl_bytes(int b) { return (((size_t)(kCtrlCounters + b) * 8) + 255) & ~(size_t)255; }
+
+// One more piece of a sequence delivered: returns how many were delivered before it in this launch.
+__device__ __forceinline__ unsigned int ctrl_arrive(unsigned long long* word, unsigned long long E) {
+    const unsigned long long cmask = (1ull << kCtrlCountBits) - 1;
+    unsigned long long old = atomicAdd(word, 1ull);
+    if ((old >> kCtrlCountBits) == E) return (unsigned int)(old & cmask);
+    // the word is from an earlier launch (or was never written): put this launch's tag on it, counting this piece
+    unsigned long long expected = old + 1;
+    for (int tries = 0; tries < 1024; ++tries) {
+        const unsigned long long prev = atomicCAS(word, expected, (E << kCtrlCountBits) | 1ull);
+        if (prev == expected) return 0u;
+        if ((prev >> kCtrlCountBits) == E) return (unsigned int)(atomicAdd(word, 1ull) & cmask);   // another CTA tagged it meanwhile
+        expected = prev;                                   // another CTA's add to the old word came in between
+    }
+    return 0xffffffffu;                                    // never seen; the caller then does not merge
+}
+
 // Barrier over `threads` threads that also ORs a predicate over them.
 __device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred) {
     uint32_t out;
@@ -210,6 +245,62 @@ __device__ __forceinline__ float warp_reduce_scatter(float (&v)[N], int lane) {
     return v[0];
 }
 
+// All the softmax threads of the CTA that delivered the last piece of sequence s: o[s] = the pieces held by
+// the CTAs lo..hi (those with a share of the line), merged in CTA order.  8 threads per head, 16 columns each.
+__device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
+                                                   float* __restrict__ o, int s, int h, int lo, int hi, int T,
+                                                   unsigned long long magic, int tid) {
+    const int g8 = tid & 7;
+    for (int head = tid >> 3; head < h; head += kUmmaSoftmaxThreads / 8) {
+        float top = -INFINITY, den = 0.f;
+        float4 num[4];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) num[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c0 = lo; c0 <= hi; c0 += 6) {
+            float2 ml[6];
+            float4 a[6][4];
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+                const int c = c0 + k;
+                const bool live = c <= hi && share_begin(c, T, magic) != share_begin(c + 1, T, magic);
+                ml[k] = make_float2(-INFINITY, 0.f);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) a[k][q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (live) {
+                    const size_t unit = ((size_t)c + s) * h + head;
+                    ml[k] = __ldcg(part_ml + unit);
+                    const float4* src = reinterpret_cast<const float4*>(part_acc + unit * kHeadDim) + g8;
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) a[k][q4] = __ldcg(src + q4 * 8);
+                }
+            }
+            float top_new = top;
+#pragma unroll
+            for (int k = 0; k < 6; ++k) top_new = fmaxf(top_new, ml[k].x);
+            const float keep = top == -INFINITY ? 0.f : fast_exp2(top - top_new);
+            den *= keep;
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) { num[q4].x *= keep; num[q4].y *= keep; num[q4].z *= keep; num[q4].w *= keep; }
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+                const float w = ml[k].x == -INFINITY ? 0.f : fast_exp2(ml[k].x - top_new);
+                den = fmaf(w, ml[k].y, den);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    num[q4].x = fmaf(w, a[k][q4].x, num[q4].x); num[q4].y = fmaf(w, a[k][q4].y, num[q4].y);
+                    num[q4].z = fmaf(w, a[k][q4].z, num[q4].z); num[q4].w = fmaf(w, a[k][q4].w, num[q4].w);
+                }
+            }
+            top = top_new;
+        }
+        const float inv = 1.f / den;
+        float4* dst = reinterpret_cast<float4*>(o + ((size_t)s * h + head) * kHeadDim) + g8;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4)
+            dst[q4 * 8] = make_float4(num[q4].x * inv, num[q4].y * inv, num[q4].z * inv, num[q4].w * inv);
+    }
+}
+
 // HP = head rows of the Q tile (h rounded up to 16, 32 or 64).
 template <int HP, bool FUSED>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
@@ -218,7 +309,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               const __grid_constant__ CUtensorMap map_q,
                               const int32_t* __restrict__ lens, float* __restrict__ o, int2* __restrict__ seq_span,
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
-                              int b, int h, int m_max, unsigned long long magic, const FusedArgs fa) {
+                              int b, int h, int m_max, unsigned long long magic, const FusedArgs fa,
+                              unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance) {
     using Cfg = UmmaCfg<HP>;
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
@@ -246,7 +338,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     const uint32_t q_full = v_empty + NV * 8, q_empty = q_full + 16;
     const uint32_t s_ready = q_empty + 16, s_free = s_ready + 16;
     const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;   // o_free: one per O^T buffer
-    __shared__ int timed_out, issued, plan_sm[4];
+    __shared__ int timed_out, issued, plan_sm[4], merge_sm[8];   // merge_sm: count, then (sequence, first CTA, last CTA) x 2
+    __shared__ unsigned long long epoch_sm[2];              // this launch's epoch; the epoch word as found
     __shared__ uint32_t tmem_base_slot;
 
     if (warp == kUmmaProducerWarp && lane == 0) {
@@ -256,6 +349,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     if (threadIdx.x == 0) {
         timed_out = 0;
         issued = 0;
+        merge_sm[0] = 0;
         for (int s = 0; s < NK; ++s) { mbar_init(k_full + s * 8, 1); mbar_init(k_empty + s * 8, 1); }
         for (int s = 0; s < NV; ++s) { mbar_init(v_full + s * 8, 1); mbar_init(v_empty + s * 8, 1); }
         for (int s = 0; s < 2; ++s) {
@@ -326,6 +420,13 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
     grid_launch_dependents();
+    if (ctrl && threadIdx.x == 0) {
+        const unsigned long long was = __ldcg(ctrl + 1);
+        unsigned long long E = __ldcg(ctrl) == kCtrlMagic ? ((was + 1) & kCtrlEpochMask) : kCtrlFirstEpoch;
+        if (E == 0) E = 1;
+        epoch_sm[0] = E;
+        epoch_sm[1] = was;
+    }
 
     // the producer warp starts its first stages (at most what the rings hold without a wait) before the tables exist
     int pre_issued = 0;
@@ -349,6 +450,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 
     if (warp == kUmmaProducerWarp) {
         // =============================================================== TMA producer
+        const unsigned long long E = ctrl ? epoch_sm[0] : 0ull;
+        if (ctrl && lane == 0) __stcg(ctrl + kCtrlStarted + cta, E);   // this CTA has read the epoch and lens
         if (lane == 0 && t_begin < t_end) {
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
@@ -360,6 +463,24 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     if (j >= pre_issued) issue_stage(g.s, u, g.hi, j, rows_entry);
             }
             if (!p_ok) atomicExch(&timed_out, 1);
+        }
+        if (ctrl) {
+            // Has every CTA started?  Then nobody will read the epoch word or lens again: the first CTA to
+            // see that moves the epoch on and, in the append-and-attend step, advances lens.
+            __syncwarp();
+            asm volatile("fence.sc.gpu;" ::: "memory");
+            bool all = true;
+            for (int c = lane; c < G; c += 32) all = all && __ldcg(ctrl + kCtrlStarted + c) == E;
+            all = __all_sync(0xffffffffu, all);
+            int won = 0;
+            if (all && lane == 0) won = atomicCAS(ctrl + 1, epoch_sm[1], E) == epoch_sm[1];
+            won = __shfl_sync(0xffffffffu, won, 0);
+            if (won) {
+                if (lane == 0) __stcg(ctrl, kCtrlMagic);
+                if (lens_advance)
+                    for (int s = lane; s < b; s += 32)
+                        if (rows_of[s] & kAppendBit) lens_advance[s] = rows_of[s] & (kAppendBit - 1);
+            }
         }
     } else if (warp == kUmmaSWarp) {
         // =============================================================== issuer of S^T = K Q^T
@@ -455,7 +576,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             bool pend = false;
             bool prev_hilo = false;                         // the stage before wrote hi and lo parts of P
             float* pend_dst = nullptr;
-            int pend_par = 0, pend_j = 0;
+            int pend_par = 0, pend_j = 0, pend_s = 0;
+            bool pend_whole = false;
             auto read_out = [&]() {
                 // O^T[column t][head] of the finished segment -> o (divided by the sum) or its partial slot
                 if (ok) ok = mbar_wait(pv_done + (pend_j & 1) * 8, (pend_j >> 1) & 1);   // the segment's last product
@@ -479,6 +601,30 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 __syncwarp();
                 if (lane == 0) mbar_arrive(o_free + pend_par * 8);   // this O^T buffer may be overwritten
                 pend = false;
+                if (ctrl && !pend_whole) {
+                    // ---- single-launch step: the piece is delivered; the CTA that delivers a sequence's
+                    // last piece merges them all into o (pieces in CTA order whoever merges: deterministic)
+                    const int s = pend_s;
+                    __threadfence();
+                    named_barrier(2, kUmmaSoftmaxThreads);
+                    if (warp == 0) {
+                        const int t0 = prefix[s] + kUmmaBoundaryPenalty, t1 = prefix[s + 1];
+                        const int lo = stream_owner(t0, T, G), hi = stream_owner(t1 - 1, T, G);
+                        int n = 0;
+                        for (int c = lo + lane; c <= hi; c += 32) n += share_begin(c, T, magic) != share_begin(c + 1, T, magic);
+#pragma unroll
+                        for (int d = 16; d >= 1; d >>= 1) n += __shfl_xor_sync(0xffffffffu, n, d);
+                        if (lane == 0) {
+                            const unsigned int before = ctrl_arrive(ctrl + kCtrlCounters + s, epoch_sm[0]);
+                            if (before + 1 == (unsigned int)n) {        // the last piece: note the merge, done when the share is finished
+                                const int k = merge_sm[0]++;
+                                merge_sm[1 + 3 * k] = s;
+                                merge_sm[2 + 3 * k] = lo;
+                                merge_sm[3 + 3 * k] = hi;
+                            }
+                        }
+                    }
+                }
             };
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
@@ -651,10 +797,20 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 pend_dst = (whole ? o + (size_t)s * h * kHeadDim : part_acc + slot * h * kHeadDim) + t;
                 pend_par = par;
                 pend_j = j - 1;
+                pend_s = s;
+                pend_whole = whole;
             }
             if (pend) {
                 named_barrier(2, kUmmaSoftmaxThreads);      // the last segment's 1/sum values are in shared memory
                 read_out();
+            }
+            if (ctrl) {
+                // sequences whose last piece this CTA delivered (a share has at most two cut segments)
+                named_barrier(2, kUmmaSoftmaxThreads);
+                const int n_merge = merge_sm[0];
+                if (n_merge > 0) __threadfence();
+                for (int k = 0; k < n_merge; ++k)
+                    merge_sequence_pieces(part_ml, part_acc, o, merge_sm[1 + 3 * k], h, merge_sm[2 + 3 * k], merge_sm[3 + 3 * k], T, magic, tid);
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
