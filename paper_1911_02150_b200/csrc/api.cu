@@ -39,6 +39,7 @@ int sm_count() {
 }
 
 enum class Kernel { kSimt, kMma1, kMma2, kStream1, kStream2, kUmma };
+constexpr int kMergeInKernelMaxPieces = 8;
 
 struct Plan {
     int n_splits = 0;     // 0 = invalid.  Fixed-split kernels: splits per sequence.  Persistent kernel: the
@@ -48,6 +49,7 @@ struct Plan {
     int b = 0, h = 0;
     int grid = 0;         // persistent kernel: number of CTAs
     Kernel kernel = Kernel::kSimt;
+    bool merge_in_kernel = false;   // tcgen05 plan: pieces merged by the CTA that delivers a sequence's last one (single launch)
     bool stream() const { return kernel == Kernel::kStream1 || kernel == Kernel::kStream2 || kernel == Kernel::kUmma; }
 };
 
@@ -120,6 +122,9 @@ Plan plan_stream(int b, int h, int m_max) {
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
     int parts = (p.grid + b - 1) / b + 1;
     p.n_splits = parts < p.grid ? parts : p.grid;
+    // a sequence cut into a few pieces is merged by one CTA inside the kernel; many pieces (few, long
+    // sequences) are better spread over all SMs by the second-pass kernel
+    p.merge_in_kernel = p.kernel == Kernel::kUmma && p.n_splits <= kMergeInKernelMaxPieces;
     return p;
 }
 
@@ -129,7 +134,7 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
     if (!(multi_query && h <= 64 && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
     // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
-    if (b <= kStreamMaxSeqs && tiles >= 8LL * sm_count() && sm_count() <= 256) return plan_stream(b, h, m_max);
+    if (b <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256) return plan_stream(b, h, m_max);
     return h <= 32 ? plan_mma(b, h, m_max) : plan_simt(b, h, m_max);
 }
 
@@ -415,7 +420,7 @@ int run_step(bool multi_query, const void* q, const void* K, const void* V, cons
              void* workspace, size_t workspace_bytes, int32_t* status,
              int b, int h, int m_max, int k, int v, cudaStream_t stream) {
     // the tcgen05 plan is a single launch: the CTA that delivers the last piece of a sequence merges the pieces
-    const bool one_launch = make_plan(multi_query, b, h, m_max).kernel == Kernel::kUmma;
+    const bool one_launch = dims_ok(b, h, m_max) && make_plan(multi_query, b, h, m_max).merge_in_kernel;
     int rc = run_split(multi_query, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream, 0,
                        one_launch);
     if (rc || one_launch) return rc;
@@ -511,8 +516,12 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
     }
     if (p.kernel == Kernel::kUmma) {
         // one launch: append inside the pass, pieces merged by the last CTA to deliver one, lens advanced at the end
-        return launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, true, k_new, v_new,
-                                     advance ? lens : nullptr);
+        if (p.merge_in_kernel)
+            return launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, true, k_new, v_new,
+                                         advance ? lens : nullptr);
+        rc = launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, false, k_new, v_new);
+        if (rc) return rc;
+        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
     }
     // other plans: the same step as separate launches.  Without `advance` the append leaves lens alone and
     // the step is told that a sequence which took a row has one more row than lens says.
@@ -539,7 +548,7 @@ size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v) {
 int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
     const Plan p = make_plan(true, b, h, m_max);
-    if (p.kernel == Kernel::kUmma) return 1;           // append, pass, merge and lens advance in one kernel
+    if (p.merge_in_kernel) return 1;                   // append, pass, merge and lens advance in one kernel
     if (p.stream()) return 2;                          // pass with the append inside, second pass
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }

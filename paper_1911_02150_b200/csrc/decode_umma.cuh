@@ -365,6 +365,20 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         tmem_alloc(smem_addr(&tmem_base_slot), Cfg::kTmemCols);
         tmem_relinquish();
     }
+    // ---- the append inside the pass, by the 32 lanes of the producer warp: lane l < 16 moves 16 bytes of the
+    // new key row, lane l >= 16 of the new value row.  The row is loaded when its segment begins and stored (and
+    // made visible to the copy engine) before the stage that contains it is fetched.
+    auto row_load = [&](int s) -> uint4 {
+        const uint4* src = (lane < 16 ? fa.k_new : fa.v_new) + (size_t)s * (kRowBytes / 16) + (lane & 15);
+        return __ldg(src);
+    };
+    auto row_store = [&](int s, int new_row, uint4 value) {
+        uint4* dst = (lane < 16 ? fa.K : fa.V) + ((size_t)s * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
+        *dst = value;
+        asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
+        __syncwarp();
+        asm volatile("fence.proxy.async;" ::: "memory");
+    };
     // ---- what the producer thread does for a segment and for a stage
     bool p_ok = true;                                       // no producer wait has run out
     auto issue_q = [&](int s, int seg) {
@@ -377,23 +391,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         tma_load_2d(q_s + qi * Cfg::kQBytes, &map_q, 0, s * h, q_full + qi * 8);
         tma_load_2d(q_s + qi * Cfg::kQBytes + Cfg::kQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
     };
-    auto issue_stage = [&](int s, int u, int hi, int j, int rows_entry) {
+    auto issue_stage = [&](int s, int u, int hi, int j) {
         const int nsub = min(kSubs, hi - u);
         const int row_first = u * kTileRows;
-        const int new_row = (rows_entry & kAppendBit) ? (rows_entry & (kAppendBit - 1)) - 1 : -1;   // row this step appends
-        if (appending && new_row >= row_first && new_row < row_first + nsub * kTileRows) {
-            const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16);
-            const size_t src = (size_t)s * (kRowBytes / 16);
-#pragma unroll 1
-            for (int i = 0; i < 16; i += 4) {
-                uint4 kr[4], vr[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) { kr[e] = fa.k_new[src + i + e]; vr[e] = fa.v_new[src + i + e]; }
-#pragma unroll
-                for (int e = 0; e < 4; ++e) { fa.K[dst + i + e] = kr[e]; fa.V[dst + i + e] = vr[e]; }
-            }
-            asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
-        }
         const int y = s * m_max + row_first;
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {                    // the K rows, then the V rows, each into its own ring
@@ -433,10 +433,16 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     if (warp == kUmmaProducerWarp) {
         Segment g0;
         int r0;
-        if (first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g0, &r0) && lane == 0) {
-            issue_q(g0.s, 0);
-            for (int u = g0.lo; u < g0.hi && pre_issued < (NK < NV ? NK : NV); u += kSubs, ++pre_issued)
-                issue_stage(g0.s, u, g0.hi, pre_issued, r0);
+        if (first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g0, &r0)) {
+            const int new_row = (r0 & kAppendBit) ? (r0 & (kAppendBit - 1)) - 1 : -1;   // row this step appends
+            const int n_pre = min((g0.hi - g0.lo + kSubs - 1) / kSubs, NK < NV ? NK : NV);
+            if (appending && new_row >= g0.lo * kTileRows && new_row < min(g0.hi, g0.lo + n_pre * kSubs) * kTileRows)
+                row_store(g0.s, new_row, row_load(g0.s));   // the new row lies in the stages started here
+            if (lane == 0) {
+                issue_q(g0.s, 0);
+                for (int u = g0.lo; pre_issued < n_pre; u += kSubs, ++pre_issued) issue_stage(g0.s, u, g0.hi, pre_issued);
+            }
+            pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
         }
     }
 
@@ -452,17 +458,30 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // =============================================================== TMA producer
         const unsigned long long E = ctrl ? epoch_sm[0] : 0ull;
         if (ctrl && lane == 0) __stcg(ctrl + kCtrlStarted + cta, E);   // this CTA has read the epoch and lens
-        if (lane == 0 && t_begin < t_end) {
+        if (t_begin < t_end) {                              // all lanes walk the share; lane 0 waits and issues the copies
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; p_ok && walk.next(g); ++seg) {
-                if (!(seg == 0 && pre_issued > 0)) issue_q(g.s, seg);
+                if (lane == 0 && !(seg == 0 && pre_issued > 0)) issue_q(g.s, seg);
                 const int rows_entry = rows_of[g.s];
-                for (int u = g.lo; u < g.hi && p_ok; u += kSubs, ++j)
-                    if (j >= pre_issued) issue_stage(g.s, u, g.hi, j, rows_entry);
+                const int new_row = (rows_entry & kAppendBit) ? (rows_entry & (kAppendBit - 1)) - 1 : -1;   // row this step appends
+                // the new row is in this segment and was not written on the way to the first stages
+                bool row_due = appending && new_row >= g.lo * kTileRows && new_row < g.hi * kTileRows &&
+                               !(seg == 0 && new_row < (g.lo + pre_issued * kSubs) * kTileRows);
+                uint4 row = make_uint4(0u, 0u, 0u, 0u);
+                if (row_due) row = row_load(g.s);
+                for (int u = g.lo; u < g.hi && p_ok; u += kSubs, ++j) {
+                    // stored once the segment's first stage is on its way, or earlier if that stage holds the row
+                    if (row_due && (u > g.lo || new_row < (u + kSubs) * kTileRows)) {
+                        row_store(g.s, new_row, row);
+                        row_due = false;
+                    }
+                    if (lane == 0 && j >= pre_issued) issue_stage(g.s, u, g.hi, j);
+                    p_ok = __shfl_sync(0xffffffffu, (int)p_ok, 0) != 0;
+                }
             }
-            if (!p_ok) atomicExch(&timed_out, 1);
+            if (lane == 0 && !p_ok) atomicExch(&timed_out, 1);
         }
         if (ctrl) {
             // Has every CTA started?  Then nobody will read the epoch word or lens again: the first CTA to
