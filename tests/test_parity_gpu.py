@@ -104,19 +104,23 @@ def _mixed_lens(b, m_max, seed):
     return lens
 
 
-# Batches large enough for the persistent kernel (>= 8 tiles of 32 rows per SM), shaped so that one
-# SM's share spans several sequences, starts and ends mid-sequence, and meets empty sequences.
+# Batches large enough for the persistent kernel (caches of 1024 rows or more, two 32-row tiles per SM or more),
+# shaped so that one SM's share spans several sequences, starts and ends mid-sequence and meets empty sequences;
+# and batches just outside it (short caches, too many sequences), which take the fixed-split kernels.
 STREAM = [
-    (300, 8, 200, 21),      # 7 tiles per sequence, ~14 tiles per SM: every SM crosses sequences
+    (200, 8, 1100, 21),     # ~50 tiles per SM over 1.4 sequences: every SM crosses a sequence
     (40, 16, 1500, 22),
-    (160, 32, 333, 23),
-    (1024, 4, 64, 24),      # the most sequences the persistent kernel indexes
+    (150, 17, 1030, 23),    # 17..32 heads: two 16-head groups, the second nearly empty
+    (1024, 4, 1024, 24),    # the most sequences the persistent kernel indexes
     (1100, 8, 64, 25),      # more than that: fixed-split kernel
     (37, 32, 4000, 26),
-    (64, 24, 700, 27),      # 17..64 heads: the tcgen05 kernel; 24 heads leave half of the second head group empty
-    (40, 48, 1500, 28),
+    (60, 24, 1300, 27),
+    (40, 48, 1500, 28),     # 33..64 heads
     (33, 64, 2100, 29),
-    (300, 17, 200, 30),
+    (300, 17, 200, 30),     # short caches: fixed-split kernel
+    (160, 32, 333, 31),
+    (3, 16, 9000, 32),      # few long sequences: cut into many pieces, merged by the second-pass kernel
+    (1, 8, 20000, 33),
 ]
 
 

@@ -1,0 +1,126 @@
+"""The single-launch decoding step of the persistent tcgen05 kernel: the pieces of a sequence that was cut over
+several CTAs are merged inside the kernel, under an epoch kept in the caller's workspace.  What is checked here is
+what that adds: the workspace may hold anything (other shapes' leftovers included), every call works under a new
+epoch (CUDA-graph replays too), lens is advanced exactly once, and the shared reference maximum of the softmax
+moves when a large logit turns up late in a long cache."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1911_02150_b200 as mqa
+from paper_1911_02150_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+ABS_TOL, REL_TOL = 4e-3, 1e-2
+
+
+def check_close(got, ref, what):
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    err = np.abs(got.astype(np.float64) - ref)
+    assert err.max() <= ABS_TOL, f"{what}: max abs err {err.max():.3e}"
+    assert np.all(err.max(-1) <= REL_TOL * np.abs(ref).max(-1)), f"{what}: row-relative error"
+
+
+def lens_for(b, m_max, seed):
+    r = np.random.default_rng(seed)
+    lens = r.integers(1, m_max + 1, size=b).astype(np.int32)
+    lens[0], lens[-1] = m_max, 1
+    return lens
+
+
+def test_launch_counts():
+    assert mqa.append_step_launches(32, 32, 8192) == 1        # cut into a few pieces per sequence: merged in the kernel
+    assert mqa.append_step_launches(256, 16, 2048) == 1
+    assert mqa.append_step_launches(1, 16, 32768) == 2        # one sequence over every SM: second-pass kernel
+    assert mqa.append_step_launches(4, 8, 300) >= 3           # small: separate launches
+
+
+def test_workspace_contents_do_not_matter():
+    shapes = [(40, 32, 2048, 1), (64, 16, 1500, 2), (33, 64, 2100, 3), (40, 32, 2048, 4)]
+    nbytes = max(mqa.workspace_bytes(b, h, m) for b, h, m, _ in shapes)
+    gen = torch.Generator(device=DEV).manual_seed(0)
+    ws = torch.randint(0, 256, (nbytes,), dtype=torch.uint8, device=DEV, generator=gen)   # garbage to begin with
+    for rnd in range(2):
+        for b, h, m_max, seed in shapes:                      # each shape finds what the shape before left behind
+            inp = wl.make_inputs(b, h, m_max, "mqa", seed=seed, device=DEV)
+            lens = lens_for(b, m_max, seed)
+            wl.poison_tail(inp["K"], lens); wl.poison_tail(inp["V"], lens)
+            o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
+            status = torch.zeros(1, dtype=torch.int32, device=DEV)
+            mqa.mqa_decode_step(inp["q"], inp["K"], inp["V"], torch.from_numpy(lens).to(DEV), o, ws, status)
+            torch.cuda.synchronize()
+            ref = oracle.mqa_decode_step(wl.bits(inp["q"]), wl.bits(inp["K"]), wl.bits(inp["V"]), lens)
+            check_close(o.cpu().numpy(), ref, f"round {rnd} b={b} h={h} m_max={m_max}")
+            assert int(status.item()) == 0
+        ws[: nbytes // 2].fill_(0xFF)                         # and a partly overwritten workspace
+
+
+def test_many_calls_on_one_workspace_are_bit_identical():
+    b, h, m_max = 48, 32, 3000
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=11, device=DEV)
+    lens_t = torch.from_numpy(lens_for(b, m_max, 11)).to(DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    outs = []
+    for _ in range(6):
+        o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
+        mqa.mqa_decode_step(inp["q"], inp["K"], inp["V"], lens_t, o, ws)
+        outs.append(o)
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0])                        # whichever CTA merged: pieces in a fixed order
+
+
+def test_graph_replays_of_append_steps_advance_lens_once_each():
+    b, h, m_max, per_graph, replays = 40, 16, 2048, 3, 2
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=12, device=DEV)
+    lens0 = np.random.default_rng(12).integers(900, 2000, size=b).astype(np.int32)
+    lens0[3] = m_max - 2                                      # fills up on the way: later steps take no row
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    o = torch.zeros(b, h, 128, dtype=torch.float32, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    side = torch.cuda.Stream(device=DEV)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws, status,
+                                   advance=True)              # set-up call outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    steps = 1
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(per_graph):
+            mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws, status,
+                                       advance=True)
+    for _ in range(replays):
+        graph.replay()
+        steps += per_graph
+    torch.cuda.synchronize()
+    k_new, v_new = wl.bits(inp["k_new"]), wl.bits(inp["v_new"])
+    for _ in range(steps):
+        oracle.kv_cache_append(Kh, Vh, k_new, v_new, lens_h, True)
+    ref = oracle.mqa_decode_step(wl.bits(inp["q"]), Kh, Vh, lens_h)
+    assert np.array_equal(lens_t.cpu().numpy(), lens_h)
+    assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)
+    check_close(o.cpu().numpy(), ref, "last step of the replayed graph")
+
+
+def test_reference_maximum_moves_late_in_a_long_cache():
+    b, h, m_max = 40, 32, 4096
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=13, device=DEV)
+    q = torch.zeros_like(inp["q"]); q[..., 0] = 1.0
+    K = torch.zeros_like(inp["K"])
+    K[:, 700, 0] = 30.0                                       # a first jump of the maximum, in a later stage ...
+    K[:, 3001, 0] = 200.0                                     # ... and a dominant logit still later
+    K[5, 3001, 0] = 0.0; K[5, 40, 0] = 200.0                  # one sequence has it in its very first stage
+    lens_t = torch.full((b,), m_max, dtype=torch.int32, device=DEV)
+    o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
+    mqa.mqa_decode_step(q, K, inp["V"], lens_t, o, mqa.alloc_workspace(b, h, m_max, DEV))
+    torch.cuda.synchronize()
+    star = torch.full((b,), 3001, device=DEV); star[5] = 40
+    want = inp["V"][torch.arange(b, device=DEV), star].float()[:, None, :].expand(b, h, 128)
+    assert torch.equal(o, want.contiguous())                  # weight exactly 1 on that row, 0 elsewhere
