@@ -91,14 +91,20 @@ int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new,
  *   q      [b, h, k] bf16          K, V   [b, m_max, k], [b, m_max, v] bf16 (read only)
  *   lens   [b] int32: rows to attend over (i.e. AFTER the append)
  *   o      [b, h, v] fp32, written
- *   workspace, workspace_bytes   scratch for the per-split partial results; at least
- *          mqa_workspace_bytes(b, h, m_max, k, v) bytes.  Contents on entry are ignored and
- *          on return are unspecified.  Two calls that may overlap on the GPU need two
- *          workspaces.  May be NULL when mqa_workspace_bytes(...) is 0.
+ *   workspace, workspace_bytes   scratch for the per-piece partial results; at least
+ *          mqa_workspace_bytes(b, h, m_max, k, v) bytes.  It may hold anything on entry (never
+ *          cleared, never assumed clear) and its contents on return are unspecified.  Two calls
+ *          that may overlap on the GPU need two workspaces.  May be NULL when
+ *          mqa_workspace_bytes(...) is 0.
  *   status optional; LEN_CLAMPED, PIPELINE_TIMEOUT.
- * The memory axis is cut into pieces that run in parallel, each keeping a running maximum
- * and sum (an exact re-association of the same softmax), and a second kernel combines the
- * pieces; shared K/V rows are read from HBM once and used for all h heads.
+ * The memory axis is cut into pieces that run in parallel, each keeping a maximum and a sum
+ * (an exact re-association of the same softmax); shared K/V rows are read from HBM once and
+ * used for all h heads.  For large batches (every SM takes an equal share of all valid rows)
+ * the pieces of a sequence are merged inside the same kernel by the CTA that finishes the
+ * sequence's last piece: one launch.  The bookkeeping for that lives in the workspace under a
+ * per-call epoch that the kernel itself moves on, so nothing has to be initialised and CUDA-graph
+ * replays are safe; after a call that reported PIPELINE_TIMEOUT, clear the workspace (any
+ * constant) before using it again.  Other sizes use a second kernel to combine the pieces.
  */
 int mqa_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                     void* workspace, size_t workspace_bytes, int32_t* status,
@@ -119,9 +125,10 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
  * (Section 3) in a single call: the new token's key/value row is concatenated to each
  * sequence's cache at row lens[b] (as kv_cache_append does), then the h heads attend over
  * the lens[b] + 1 rows (as mqa_decode_step does).  For batches large enough for the persistent
- * kernels (h <= 64) there is no separate append launch: the CTA that streams a sequence's last
- * tile writes the new row just before it fetches that tile, and the second-pass kernel advances
- * lens (two launches instead of three).  Other sizes run the same step as separate launches.
+ * kernel (h <= 64) the whole step is one launch: the CTA that streams a sequence's last tile
+ * writes the new row before it fetches that tile, the pieces of a sequence are merged by the
+ * CTA that finishes the last one, and lens is advanced once every CTA has read it.  Other
+ * sizes run the same step as separate launches (mqa_append_step_launches tells how many).
  *
  *   q, k_new, v_new   [b, h, k], [b, k], [b, v] bf16
  *   K, V              [b, m_max, k], [b, m_max, v] bf16, read-write (row lens[b] is written)
@@ -138,11 +145,13 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
                            int b, int h, int m_max, int k, int v, mqa_stream_t stream);
 
 /*
- * The two phases of a step, separately (mqa_decode_step == split then combine with the same
- * arguments; likewise mha).  They exist so that a caller can time or schedule the phases on
- * their own.  *_split runs the pass over the cache (Section 3 / 2.4 lines, per split) and
- * leaves partial results in the workspace -- or final results in o when the plan has a single
- * split; *_combine merges the splits into o and is a no-op (no launch) for a single split.
+ * The two phases of a step, separately (split then combine with the same arguments gives what
+ * mqa_decode_step gives; likewise mha).  They exist so that a caller can time or schedule the
+ * phases on their own.  *_split runs the pass over the cache (Section 3 / 2.4 lines, per piece)
+ * and leaves partial results in the workspace -- or final results in o when the plan has a
+ * single piece; *_combine merges the pieces into o with a second kernel (also where
+ * mqa_decode_step itself would merge them inside its one launch) and is a no-op (no launch)
+ * for a single piece.
  */
 int mqa_decode_step_split(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                           void* workspace, size_t workspace_bytes, int32_t* status,
@@ -193,8 +202,8 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
  *   that device current) and remembers it; make this first call during set-up, before any
  *   stream capture is begun on that device.
  *   Sharing: every call on a device uses the same array, which still holds whatever the last
- *   call left in it.  Nothing has to be cleared -- the second pass reads only slots that the
- *   first pass of the same call has written -- but two calls whose kernels may overlap on the
+ *   call left in it.  Nothing has to be cleared -- a call reads only what the same call has
+ *   written, or what carries its own epoch -- but two calls whose kernels may overlap on the
  *   GPU (different streams, no ordering between them) race on it and corrupt each other's
  *   results.  Calls on one stream are safe.
  */

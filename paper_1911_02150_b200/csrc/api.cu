@@ -38,7 +38,7 @@ int sm_count() {
     return n;
 }
 
-enum class Kernel { kSimt, kMma1, kMma2, kStream1, kStream2, kUmma };
+enum class Kernel { kSimt, kMma1, kMma2, kUmma };
 constexpr int kMergeInKernelMaxPieces = 8;
 
 struct Plan {
@@ -50,7 +50,7 @@ struct Plan {
     int grid = 0;         // persistent kernel: number of CTAs
     Kernel kernel = Kernel::kSimt;
     bool merge_in_kernel = false;   // tcgen05 plan: pieces merged by the CTA that delivers a sequence's last one (single launch)
-    bool stream() const { return kernel == Kernel::kStream1 || kernel == Kernel::kStream2 || kernel == Kernel::kUmma; }
+    bool stream() const { return kernel == Kernel::kUmma; }
 };
 
 bool dims_ok(int b, int h, int m_max) { return b > 0 && h > 0 && m_max > 0; }
@@ -113,10 +113,7 @@ Plan plan_stream(int b, int h, int m_max) {
     Plan p;
     p.units = (size_t)b * h;
     p.b = b; p.h = h;
-    // the tcgen05 kernel for every head count up to 64.  MQA_DECODE_MMA=1 in the environment sends h <= 32 to the
-    // register-fragment mma.sync kernel instead (for comparisons).
-    static const bool force_mma = [] { const char* e = getenv("MQA_DECODE_MMA"); return e && e[0] == '1'; }();
-    p.kernel = (force_mma && h <= 32) ? (h <= 16 ? Kernel::kStream1 : Kernel::kStream2) : Kernel::kUmma;
+    p.kernel = Kernel::kUmma;
     p.grid = sm_count();
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
@@ -267,42 +264,6 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
-std::atomic<int> g_stream_opt_in[kMaxDevices][4];
-
-template <int M_TILES, bool FUSED>
-int launch_stream(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-                  void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream,
-                  const void* k_new = nullptr, const void* v_new = nullptr) {
-    using Cfg = StreamCfg<M_TILES>;
-    auto kernel = mqa_decode_stream_mma_kernel<M_TILES, FUSED>;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
-    constexpr int kSlot = (M_TILES - 1) * 2 + (FUSED ? 1 : 0);
-    if (!g_stream_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
-            cudaGetLastError();
-            return MQA_ERR_CUDA;
-        }
-        g_stream_opt_in[dev][kSlot].store(1, std::memory_order_release);
-    }
-    FusedArgs fa = {};
-    if (FUSED) {
-        fa.k_new = static_cast<const uint4*>(k_new);
-        fa.v_new = static_cast<const uint4*>(v_new);
-        fa.K = static_cast<uint4*>(const_cast<void*>(K));
-        fa.V = static_cast<uint4*>(const_cast<void*>(V));
-    }
-    alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub;
-    const long long rows = (long long)b * m_max;
-    if (!encode_cache_map(&map_k, K, rows, kStreamStageRows) || !encode_cache_map(&map_v, V, rows, kStreamStageRows) ||
-        !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows))
-        return MQA_ERR_CUDA;
-    const StreamWorkspace w = stream_workspace(p, workspace);
-    launch_dependent(kernel, (unsigned)p.grid, Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     static_cast<const uint32_t*>(q), lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa);
-    return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
-}
-
 std::atomic<int> g_umma_opt_in[kMaxDevices][6];
 
 template <int HP, bool FUSED>
@@ -365,10 +326,6 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (rc) return rc;
     if (p.kernel == Kernel::kUmma)
         return launch_umma_for<false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge_in_kernel);
-    if (p.kernel == Kernel::kStream1)
-        return launch_stream<1, false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
-    if (p.kernel == Kernel::kStream2)
-        return launch_stream<2, false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream);
     float2* part_ml = reinterpret_cast<float2*>(workspace);
     float* part_acc = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits))
@@ -507,13 +464,6 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
     rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
-    if (p.kernel == Kernel::kStream1 || p.kernel == Kernel::kStream2) {
-        rc = p.kernel == Kernel::kStream1
-                 ? launch_stream<1, true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new)
-                 : launch_stream<2, true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, k_new, v_new);
-        if (rc) return rc;
-        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
-    }
     if (p.kernel == Kernel::kUmma) {
         // one launch: append inside the pass, pieces merged by the last CTA to deliver one, lens advanced at the end
         if (p.merge_in_kernel)

@@ -13,15 +13,11 @@
 // Each consumer warp takes whole 32-row tiles round-robin and keeps its own online-softmax
 // state (running max, running sum, fp32 accumulators) in registers.
 //
-// Two kernels share that inner loop:
-//   * mqa_decode_split_mma_kernel   -- one CTA per (sequence, fixed-size split); used when the
-//                                      whole problem is small (short caches, few sequences);
-//   * mqa_decode_stream_mma_kernel  -- a persistent grid of one CTA per SM; the 32-row tiles of
-//                                      all sequences (valid rows only, from lens) form one
-//                                      line that is cut into equal contiguous shares, so every
-//                                      SM streams the same number of bytes whatever the batch
-//                                      size, context length or raggedness.  It stages 128 rows
-//                                      at a time; each of its 4 row-warps takes 32 of them.
+// mqa_decode_split_mma_kernel runs one CTA per (sequence, fixed-size split) and is used when the
+// whole problem is small (short caches, few sequences); large batches go to the persistent
+// tcgen05 kernel (decode_umma.cuh).  The second half of this file is what the persistent kernel's
+// schedule is made of: the line of 32-row tiles, its equal shares, segments, slots and the
+// second-pass kernel that merges the slots of a sequence cut into many pieces.
 //
 // Rows at or beyond lens[b] are never used: their logits are replaced by -inf by index and
 // their V fragments are zeroed by index (a NaN times a zero weight would still be a NaN).
@@ -38,12 +34,6 @@ constexpr int kBoxCols = 64;                           // 64 bf16 = 128 bytes = 
 constexpr int kBoxBytes = kTileRows * kBoxCols * 2;    // 4 KiB
 constexpr int kStageBytes = 4 * kBoxBytes;             // K lo, K hi, V lo, V hi = 16 KiB
 constexpr int kRowWarps = 4;                           // consumer warps that share the tiles
-// The persistent kernel stages 128 rows at a time (4 sub-tiles of 32 rows, one per row-warp): a full
-// stage is fetched with four 16 KiB TMA boxes, which the copy engine moves measurably faster than
-// sixteen 4 KiB ones; a stage at the end of a segment is fetched sub-tile by sub-tile with 4 KiB boxes.
-constexpr int kStreamStageRows = kRowWarps * kTileRows;        // 128
-constexpr int kStreamBoxBytes = kStreamStageRows * kBoxCols * 2;   // 16 KiB: 128 rows x 128 bytes
-constexpr int kStreamStageBytes = 4 * kStreamBoxBytes;         // 64 KiB
 constexpr long long kWaitLimitCycles = 2000000000ll;   // every mbarrier wait gives up after ~1 s of SM clock ...
 constexpr uint32_t kWaitRounds = 1u << 24;             // ... or after this many polling rounds
 constexpr int kSingleRoundingMinRows = 1024;            // prefixes this long feed P to the tensor cores in one bf16 rounding
@@ -61,20 +51,6 @@ struct MmaCfg {                                        // fixed-split kernel
     static_assert(kStages % kRowWarps == 0, "a stage must always be consumed by the same warp");
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
     static constexpr int kMinBlocks = (M_TILES == 1) ? 2 : 1;
-};
-
-template <int M_TILES>
-struct StreamCfg {                                     // persistent kernel, one CTA per SM
-    static constexpr int kConsumerWarps = M_TILES * kRowWarps;
-    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
-    static constexpr int kStages = 3;                  // every consumer warp waits on every stage: any depth is safe
-    static constexpr int kStateFloats = 16 * 4 + 4;    // acc + (m, l) x 2 rows, per thread
-    static constexpr int kMergeBytes = M_TILES * kStateFloats * 32 * 4;
-    static constexpr int kPrefixBytes = 2 * (kStreamMaxSeqs + 1) * 4 + 16;   // line positions + rows per sequence
-    static constexpr int kSmemBytes = kStages * kStreamStageBytes + kMergeBytes + kPrefixBytes + 256 /* barriers */ +
-                                      1024 /* alignment slack */;
-    static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
-    static constexpr int kCtasPerSm = 1;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -492,13 +468,13 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 // each a contiguous run of tiles of one sequence.  A segment that covers its whole sequence
 // writes the final o; any other segment writes a partial into slot (c + sequence) -- along the
 // line every step moves to the next CTA, the next sequence, or both, so that sum never repeats
-// -- and the second-pass kernel merges the slots of each sequence that was cut.
+// -- and the slots of each sequence that was cut are merged, inside the kernel by the CTA that
+// delivers the last one or by the second-pass kernel below.
 // =============================================================================================
-// Crossing from one sequence to the next inside a share is not free (the row-warps are merged, a
-// partial or the result is written, the next sequence's Q is fetched), so the line carries, in front
-// of each sequence's tiles, kBoundaryPenalty virtual tiles that cost nothing to "process": a CTA
-// whose share contains a crossing gets that many fewer real tiles, and all CTAs finish together.
-constexpr int kBoundaryPenalty = 12;         // mma.sync kernel (the tcgen05 kernel has its own)
+// Crossing from one sequence to the next inside a share is not free (sums are added up, a partial or
+// the result is written, the next sequence's Q is fetched), so the line carries, in front of each
+// sequence's tiles, PENALTY virtual tiles that cost nothing to "process": a CTA whose share contains a
+// crossing gets that many fewer real tiles, and all CTAs finish together.
 
 // Share c of G of a line of T positions: [c*T/G, (c+1)*T/G).  The division by the run-time grid size is
 // a multiplication by magic = ceil(2^64 / G), computed on the host (exact for c*T < 2^48, G <= 256; a
@@ -580,7 +556,7 @@ __device__ __forceinline__ int fused_rows(int raw, int m_max, bool appending, bo
 constexpr int kAppendBit = 1 << 30;                    // in rows_of[]: this step appends a row to the sequence
 
 // The schedule of a persistent kernel, computed by every CTA for itself (all THREADS threads call this):
-// prefix[s] = position on the line of sequence s's block (kBoundaryPenalty virtual tiles, then its 32-row
+// prefix[s] = position on the line of sequence s's block (PENALTY virtual tiles, then its 32-row
 // tiles; no block for an empty prefix, whose output is zeroed here), rows_of[s] = rows to attend over
 // (kAppendBit set when this step appends one).  Returns T = length of the line, [t_begin, t_end) = this
 // CTA's share, s_first = the sequence that holds position t_begin.  plan_sm: 4 ints of shared memory.
@@ -692,257 +668,6 @@ __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, 
     g->whole = g->lo == 0 && g->hi == n;
     *rows = fr;
     return g->hi > g->lo;
-}
-
-template <int M_TILES, bool FUSED>
-__global__ void __launch_bounds__(StreamCfg<M_TILES>::kThreads, 1)
-mqa_decode_stream_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                             const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
-                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
-                             float* __restrict__ o, int2* __restrict__ seq_span, float2* __restrict__ part_ml,
-                             float* __restrict__ part_acc, int32_t* __restrict__ status, int b, int h, int m_max,
-                             unsigned long long magic, const FusedArgs fa) {
-    using Cfg = StreamCfg<M_TILES>;
-    const bool appending = FUSED && fa.k_new != nullptr;
-    constexpr int kStages = Cfg::kStages;
-    constexpr int kConsumerThreads = Cfg::kConsumerWarps * 32;
-    const int cta = blockIdx.x, G = gridDim.x;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* stages = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-    float* merge_buf = reinterpret_cast<float*>(stages + kStages * kStreamStageBytes);      // [M_TILES][68][32]
-    int* prefix = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(merge_buf) + Cfg::kMergeBytes);  // [b + 1]
-    int* rows_of = prefix + kStreamMaxSeqs + 1;         // [b] rows to attend over; bit 30: this step appends a row
-    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(prefix) + Cfg::kPrefixBytes / 8 * 8);
-    const uint32_t stages_s = smem_addr(stages);
-    const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
-    __shared__ int timed_out, issued, plan_sm[4];
-
-    if (warp == Cfg::kConsumerWarps && lane == 0) {
-        prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-        prefetch_tensormap(&map_k_sub); prefetch_tensormap(&map_v_sub);
-    }
-    if (threadIdx.x == 0) {
-        timed_out = 0;
-        issued = 0;
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_s + s * 8, 1);                      // the producer's arrive + the TMA bytes
-            mbar_init(empty_s + s * 8, Cfg::kConsumerWarps);   // every consumer warp passes every stage
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
-    grid_launch_dependents();
-
-    const SharePlan plan = stream_plan<FUSED, Cfg::kThreads, kBoundaryPenalty>(lens, o, status, b, h, m_max, appending, magic, prefix,
-                                                             rows_of, plan_sm);
-    const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
-
-    const int mt = warp % M_TILES;
-    const int rw = warp / M_TILES;
-
-    if (warp == Cfg::kConsumerWarps) {
-        // ------------------------------------------------------------------ producer warp
-        // One thread waits and issues the copies; in the append-and-attend step it also writes the new
-        // row of a sequence (512 bytes) before the tile that contains it is fetched.
-        if (t_begin < t_end && lane == 0) {
-            bool ok = true;
-            int j = 0;                                     // stages issued by this CTA so far
-            ShareWalker<kBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
-            Segment g;
-            while (ok && walk.next(g)) {
-                const int s = g.s;
-                const int new_row = (rows_of[s] & kAppendBit) ? (rows_of[s] & (kAppendBit - 1)) - 1 : -1;   // row this step appends
-                for (int u = g.lo; u < g.hi && ok; u += kRowWarps, ++j) {
-                    const int nsub = min(kRowWarps, g.hi - u);
-                    const int stg = j % kStages;
-                    const int row_first = u * kTileRows;
-                    if (appending && new_row >= row_first && new_row < row_first + nsub * kTileRows) {
-                        const size_t dst = ((size_t)s * m_max + new_row) * (kRowBytes / 16);
-                        const size_t src = (size_t)s * (kRowBytes / 16);
-                        uint4 kr[16], vr[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) { kr[i] = fa.k_new[src + i]; vr[i] = fa.v_new[src + i]; }
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) { fa.K[dst + i] = kr[i]; fa.V[dst + i] = vr[i]; }
-                        asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
-                    }
-                    {
-                        if (j >= kStages) ok = mbar_wait(empty_s + stg * 8, ((j / kStages) - 1) & 1);
-                        if (ok) {
-                            const uint32_t bar = full_s + stg * 8;
-                            const uint32_t dst = stages_s + stg * kStreamStageBytes;
-                            mbar_expect_tx(bar, nsub * kStageBytes);
-                            const int y = s * m_max + row_first;
-                            if (nsub == kRowWarps) {
-                                tma_load_2d(dst, &map_k, 0, y, bar);
-                                tma_load_2d(dst + kStreamBoxBytes, &map_k, kBoxCols, y, bar);
-                                tma_load_2d(dst + 2 * kStreamBoxBytes, &map_v, 0, y, bar);
-                                tma_load_2d(dst + 3 * kStreamBoxBytes, &map_v, kBoxCols, y, bar);
-                            } else {
-                                for (int i = 0; i < nsub; ++i) {
-                                    const uint32_t d = dst + i * kBoxBytes;
-                                    tma_load_2d(d, &map_k_sub, 0, y + i * kTileRows, bar);
-                                    tma_load_2d(d + kStreamBoxBytes, &map_k_sub, kBoxCols, y + i * kTileRows, bar);
-                                    tma_load_2d(d + 2 * kStreamBoxBytes, &map_v_sub, 0, y + i * kTileRows, bar);
-                                    tma_load_2d(d + 3 * kStreamBoxBytes, &map_v_sub, kBoxCols, y + i * kTileRows, bar);
-                                }
-                            }
-                            issued = j + 1;
-                        }
-                    }
-                }
-            }
-            if (!ok) atomicExch(&timed_out, 1);
-        }
-    } else {
-        // --------------------------------------------------------------- consumer warps
-        // which CTAs hold pieces of each sequence (read by the second pass); spread over the CTAs
-        if (warp == 0) {
-            for (int s = cta + lane * G; s < b; s += G * 32) {
-                const int t0 = prefix[s] + kBoundaryPenalty, t1 = prefix[s + 1];     // its real tiles on the line
-                seq_span[s] = t1 > t0 ? make_int2(stream_owner(t0, T, G), stream_owner(t1 - 1, T, G)) : make_int2(0, 0);
-            }
-            if (cta == 0 && lane == 0) seq_span[b] = make_int2((int)T, G);
-        }
-        WarpState st;
-        LaneOffsets off;
-        off.init(lane);
-        const int g = lane >> 2, t4 = lane & 3;
-        float* my_buf = merge_buf + mt * Cfg::kStateFloats * 32;
-        bool ok = true;
-        int j = 0;                                         // stages consumed by this CTA so far
-        ShareWalker<kBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
-        Segment g_;
-        while (walk.next(g_)) {
-            const int s = g_.s;
-            const int L = rows_of[s] & (kAppendBit - 1);
-            const bool whole = g_.whole;
-            const bool last_segment = walk.t >= t_end;     // (a later block could only add penalty tiles)
-
-            st.reset();
-            uint32_t qa[8][4];
-            load_q_fragments(qa, q, (size_t)s, h, mt, lane);
-            for (int u = g_.lo; u < g_.hi; u += kRowWarps, ++j) {
-                const int nsub = min(kRowWarps, g_.hi - u);
-                const int stg = j % kStages;
-                if (ok) ok = mbar_wait(full_s + stg * 8, (j / kStages) & 1);
-                if (ok && rw < nsub) {                     // row-warp rw takes sub-tile rw of the stage
-                    const uint32_t k_s = stages_s + stg * kStreamStageBytes + rw * kBoxBytes;
-                    const int row0 = (u + rw) * kTileRows;
-                    if (L >= kSingleRoundingMinRows)
-                        consume_tile<false, kStreamBoxBytes>(st, qa, off, k_s, k_s + 2 * kStreamBoxBytes, row0, L, lane);
-                    else
-                        consume_tile<true, kStreamBoxBytes>(st, qa, off, k_s, k_s + 2 * kStreamBoxBytes, row0, L, lane);
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_s + stg * 8);   // released even after a failed wait: nobody may hang
-            }
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 1);
-                st.l[r] += __shfl_xor_sync(0xffffffffu, st.l[r], 2);
-            }
-            const int head0 = mt * 16 + g, head1 = head0 + 8;
-            const size_t slot = (size_t)cta + s;
-            if (last_segment) {
-                // Last segment of this CTA: nothing is in flight any more, so the stage memory is
-                // free.  Every row-warp parks its state there and all consumer threads merge in
-                // parallel, each taking a quarter of its own fragment columns.
-                float* park = reinterpret_cast<float*>(stages);                   // [consumer warp][68][32]
-                named_barrier(1, kConsumerThreads);                               // all warps are done reading tiles
-                store_state(st, park + warp * Cfg::kStateFloats * 32, lane);
-                named_barrier(1, kConsumerThreads);
-                float wgt[kRowWarps][2], m_new[2] = {-INFINITY, -INFINITY}, l_new[2] = {0.f, 0.f};
-#pragma unroll
-                for (int w = 0; w < kRowWarps; ++w) {
-                    const float* src = park + (w * M_TILES + mt) * Cfg::kStateFloats * 32;
-                    wgt[w][0] = src[64 * 32 + lane];
-                    wgt[w][1] = src[65 * 32 + lane];
-                    m_new[0] = fmaxf(m_new[0], wgt[w][0]);
-                    m_new[1] = fmaxf(m_new[1], wgt[w][1]);
-                }
-#pragma unroll
-                for (int w = 0; w < kRowWarps; ++w) {
-                    const float* src = park + (w * M_TILES + mt) * Cfg::kStateFloats * 32;
-#pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        wgt[w][r] = wgt[w][r] == -INFINITY ? 0.f : fast_exp2(wgt[w][r] - m_new[r]);
-                        l_new[r] = fmaf(wgt[w][r], src[(66 + r) * 32 + lane], l_new[r]);
-                    }
-                }
-                const float inv0 = whole ? 1.f / l_new[0] : 1.f, inv1 = whole ? 1.f / l_new[1] : 1.f;
-                float* d0 = (whole ? o + ((size_t)s * h + head0) * kHeadDim : part_acc + (slot * h + head0) * kHeadDim) + t4 * 2;
-                float* d1 = (whole ? o + ((size_t)s * h + head1) * kHeadDim : part_acc + (slot * h + head1) * kHeadDim) + t4 * 2;
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int vt = rw * 4 + q4;                                    // this thread's quarter
-                    float v[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int w = 0; w < kRowWarps; ++w) {
-                        const float* src = park + (w * M_TILES + mt) * Cfg::kStateFloats * 32;
-#pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) v[jj] = fmaf(wgt[w][jj >> 1], src[(vt * 4 + jj) * 32 + lane], v[jj]);
-                    }
-                    if (head0 < h) *reinterpret_cast<float2*>(d0 + vt * 8) = make_float2(v[0] * inv0, v[1] * inv0);
-                    if (head1 < h) *reinterpret_cast<float2*>(d1 + vt * 8) = make_float2(v[2] * inv1, v[3] * inv1);
-                }
-                if (!whole && rw == 0 && t4 == 0) {
-                    if (head0 < h) part_ml[slot * h + head0] = make_float2(m_new[0], l_new[0]);
-                    if (head1 < h) part_ml[slot * h + head1] = make_float2(m_new[1], l_new[1]);
-                }
-            } else {
-                // A segment in the middle of the share: tiles of the next one are already streaming
-                // into the stages, so fold the row-warps 3 -> 2 -> 1 -> 0 through the small buffer.
-                named_barrier(1, kConsumerThreads);        // the previous segment's last reader is done with the buffer
-#pragma unroll 1
-                for (int r = kRowWarps - 1; r >= 1; --r) {
-                    if (rw == r) store_state(st, my_buf, lane);
-                    named_barrier(1, kConsumerThreads);
-                    if (rw == r - 1) merge_state(st, my_buf, lane);
-                }
-                if (rw == 0) {
-                    if (whole) {
-                        const float inv0 = 1.f / st.l[0], inv1 = 1.f / st.l[1];
-                        float* o0 = o + ((size_t)s * h + head0) * kHeadDim + t4 * 2;
-                        float* o1 = o + ((size_t)s * h + head1) * kHeadDim + t4 * 2;
-#pragma unroll
-                        for (int vt = 0; vt < 16; ++vt) {
-                            if (head0 < h) *reinterpret_cast<float2*>(o0 + vt * 8) = make_float2(st.acc[vt][0] * inv0, st.acc[vt][1] * inv0);
-                            if (head1 < h) *reinterpret_cast<float2*>(o1 + vt * 8) = make_float2(st.acc[vt][2] * inv1, st.acc[vt][3] * inv1);
-                        }
-                    } else {
-                        float* a0 = part_acc + (slot * h + head0) * kHeadDim + t4 * 2;
-                        float* a1 = part_acc + (slot * h + head1) * kHeadDim + t4 * 2;
-#pragma unroll
-                        for (int vt = 0; vt < 16; ++vt) {
-                            if (head0 < h) *reinterpret_cast<float2*>(a0 + vt * 8) = make_float2(st.acc[vt][0], st.acc[vt][1]);
-                            if (head1 < h) *reinterpret_cast<float2*>(a1 + vt * 8) = make_float2(st.acc[vt][2], st.acc[vt][3]);
-                        }
-                        if (t4 == 0) {
-                            if (head0 < h) part_ml[slot * h + head0] = make_float2(st.m[0], st.l[0]);
-                            if (head1 < h) part_ml[slot * h + head1] = make_float2(st.m[1], st.l[1]);
-                        }
-                    }
-                }
-            }
-        }
-        if (!ok) atomicExch(&timed_out, 1);
-    }
-
-    __syncthreads();
-    if (timed_out) {
-        if (threadIdx.x == 0) {
-            for (int s = 0; s < kStages && s < issued; ++s) {
-                const int last_use = (issued - 1 - s) / kStages;
-                mbar_wait(full_s + s * 8, last_use & 1);
-            }
-            if (status) atomicOr(status, kStatusPipelineTimeout);
-        }
-        __syncthreads();
-    }
 }
 
 // Second pass of the persistent kernel: one CTA per (sequence, head) merges the slots of the

@@ -1,8 +1,8 @@
-// Persistent multi-query decode kernel on the 5th-generation tensor cores (tcgen05 + TMEM).
-// Same step as the other kernels (Section 3: logits = einsum(bhk,bmk->bhm), softmax over m,
-// o = einsum(bhm,bmv->bhv)), same equal-share scheduling, slots and second pass as
-// mqa_decode_stream_mma_kernel; what changes is who does the two contractions and which way round
-// they are laid out.  The cache rows are the M dimension of both products and the heads are N:
+// Persistent multi-query decode kernel on the 5th-generation tensor cores (tcgen05 + TMEM): one CTA
+// per SM, every CTA an equal share of the line of valid 32-row tiles of the whole batch (see the
+// second half of decode_mma.cuh).  The step is the three lines of Section 3: logits =
+// einsum(bhk,bmk->bhm), softmax over m, o = einsum(bhm,bmv->bhv).  The cache rows are the M dimension
+// of both products and the heads are N:
 //
 //     S^T[128 cache rows x HP heads]  = K_stage[128 x 128] * Q^T          A = the TMA-written K rows (K-major),
 //                                                                          B = the sequence's Q rows (K-major)
@@ -11,22 +11,27 @@
 //
 // so K and V are read from shared memory by the tensor core itself, once for all heads; the work
 // per stage grows with the padded head count HP (16, 32 or 64) and nothing is replicated.  In TMEM
-// a cache row of S^T is a lane, so a softmax thread owns one cache row of the stage and all its
-// heads: masking by index is a per-thread decision and the weights need no exchange between
-// threads.  The reference maximum of a head is shared by all rows and moves only when some logit
-// exceeds it by more than 2^kMaxLead (always on a segment's first stage): then the warps find the
-// stage's maxima together, rescale their sums and the O^T accumulator, and go on.  Softmax is shift
-// invariant, so a reference that lags the true maximum by a bounded amount changes nothing but the
-// common scale of numerator and denominator.
+// a cache row of S^T is a lane, so a softmax thread owns one cache row of the stage (two threads
+// share a row's heads): masking by index is a per-thread decision and the weights need no exchange
+// between threads.  The reference maximum of a head is shared by all rows and moves only when some
+// logit exceeds it by more than 2^kMaxLead (always on a segment's first stage): then the warps find
+// the stage's maxima together, rescale their sums and the O^T accumulator, and go on.  Softmax is
+// shift invariant, so a reference that lags the true maximum by a bounded amount changes nothing but
+// the common scale of numerator and denominator.
 //
 //   producer warp      TMA: a segment's Q rows once, then K and V rows in 128-row stages (separate
-//                      rings: a K slot is free again as soon as S^T is done)
+//                      rings: a K slot is free again as soon as S^T is done).  It finds its first
+//                      copies from its own scan of lens, before the shared tables exist, and in the
+//                      append-and-attend step moves the new key/value row into the cache.
 //   two MMA warps      one thread each issues the tcgen05.mma of S^T, and of O^T
-//   4 softmax warps    tcgen05.ld the logits of their row, P = exp2(S - reference) as bf16 (hi, and lo
-//                      for short prefixes) into shared memory, per-thread partial sums; at the end
-//                      of a segment the sums are added up and O^T is read out of TMEM
+//   8 softmax warps    tcgen05.ld the logits of their row, P = exp2(S - reference) as bf16 (hi, and lo
+//                      for short prefixes) into shared memory, per-thread partial sums.  Two O^T
+//                      buffers: a finished segment is read out of TMEM after the next one's first stage.
 //
-// Everything between the roles is an mbarrier; every wait is bounded (see mbar_wait).
+// A sequence cut over several CTAs leaves one piece per CTA in the workspace.  With a control block
+// (see below) the CTA that delivers the last piece merges them inside this kernel; without one the
+// second-pass kernel does.  Everything between the roles is an mbarrier; every wait is bounded (see
+// mbar_wait); no CTA ever waits for another CTA.
 #pragma once
 #include <cuda.h>
 
@@ -41,8 +46,8 @@ constexpr int kUmmaSoftmaxWarps = 8;                             // warp w: TMEM
 constexpr int kUmmaSoftmaxThreads = kUmmaSoftmaxWarps * 32;
 constexpr int kUmmaProducerWarp = 8, kUmmaSWarp = 9, kUmmaPvWarp = 10;
 constexpr int kUmmaThreads = 11 * 32;
-// virtual tiles in front of each sequence on the line (see kBoundaryPenalty): what a crossing costs this kernel
-constexpr int kUmmaBoundaryPenalty = 12;
+// virtual tiles in front of each sequence on the line: what crossing from one sequence to the next costs this kernel
+constexpr int kUmmaBoundaryPenalty = 8;
 constexpr float kMaxLead = 16.f;                                 // log2 units a logit may exceed the reference maximum by
 
 template <int HP>
