@@ -243,7 +243,8 @@ std::atomic<int> g_smem_opt_in[kMaxDevices][2];
 
 template <int M_TILES>
 int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
-               float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias) {
+               float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias,
+               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
     using Cfg = MmaCfg<M_TILES>;
     auto kernel = mqa_decode_split_mma_kernel<M_TILES>;
     int dev = 0;
@@ -258,9 +259,16 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     alignas(64) CUtensorMap map_k, map_v;
     if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
         return MQA_ERR_CUDA;
+    FusedArgs fa = {};
+    if (k_new) {                                       // the whole decoding step in this launch (one CTA per sequence)
+        fa.k_new = static_cast<const uint4*>(k_new);
+        fa.v_new = static_cast<const uint4*>(v_new);
+        fa.K = static_cast<uint4*>(const_cast<void*>(K));
+        fa.V = static_cast<uint4*>(const_cast<void*>(V));
+    }
     launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
                      static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
-                     p.n_splits, len_bias);
+                     p.n_splits, len_bias, fa, lens_advance);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -354,10 +362,10 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
         const StreamWorkspace w = stream_workspace(p, workspace);
         if (p.n_splits <= kCombineEager)
             launch_dependent(stream_combine_kernel<1>, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
-                             b, h, lens_advance, m_max);
+                             b, h, lens_advance, m_max, share_magic(p.grid));
         else
             launch_dependent(stream_combine_kernel<4>, (unsigned)((size_t)b * h), 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc,
-                             o, b, h, lens_advance, m_max);
+                             o, b, h, lens_advance, m_max, share_magic(p.grid));
         return launch_status();
     }
     if (p.n_splits <= 1) return MQA_OK;
@@ -387,6 +395,7 @@ int run_step(bool multi_query, const void* q, const void* K, const void* V, cons
 // lens[i] += 1 for the sequences that took a row (the multi-launch form of mqa_decode_append_step
 // advances lens last, after the kernels that read the old value).
 __global__ void lens_advance_kernel(int32_t* lens, int b, int m_max) {
+    grid_launch_dependents();
     grid_dependency_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < b && lens[i] >= 0 && lens[i] < m_max) lens[i] += 1;
@@ -475,6 +484,14 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
     }
     // other plans: the same step as separate launches.  Without `advance` the append leaves lens alone and
     // the step is told that a sequence which took a row has one more row than lens says.
+    if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits == 1) {
+        // one CTA per sequence: it writes the row, attends and moves lens on, all in one launch
+        return p.kernel == Kernel::kMma1
+                   ? launch_mma<1>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
+                                   advance ? lens : nullptr)
+                   : launch_mma<2>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
+                                   advance ? lens : nullptr);
+    }
     rc = kv_cache_append(K, V, k_new, v_new, lens, 0, status, b, 1, m_max, k, v, stream_);
     if (rc) return rc;
     rc = run_split(true, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream, 1);
@@ -499,6 +516,7 @@ int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return 0;
     const Plan p = make_plan(true, b, h, m_max);
     if (p.merge_in_kernel) return 1;                   // append, pass, merge and lens advance in one kernel
+    if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits == 1) return 1;   // one CTA per sequence does it all
     if (p.stream()) return 2;                          // pass with the append inside, second pass
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }

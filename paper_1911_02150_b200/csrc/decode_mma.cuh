@@ -121,6 +121,16 @@ __device__ __forceinline__ void named_barrier(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// The append-and-attend step: the kernel that owns a sequence's last tile also writes the new token's key
+// and value row (row lens[b]) into the cache before it fetches that tile, so the step attends over
+// lens[b] + 1 rows without a separate append launch.
+struct FusedArgs {
+    const uint4* k_new;      // [b, 128] bf16 rows as 16-byte words; null = nothing to append
+    const uint4* v_new;
+    uint4* K;                // the cache, written at row lens[b]
+    uint4* V;
+};
+
 // ---- the consumer warp's state and inner loop ------------------------------------------------
 // Layout of a K or V tile in shared memory as TMA writes it: two 64-column boxes of 32 rows x
 // 128 bytes; inside a box the 16-byte chunk index (0..7) is XORed with (row mod 8).
@@ -310,24 +320,13 @@ __global__ void __launch_bounds__(MmaCfg<M_TILES>::kThreads, MmaCfg<M_TILES>::kM
 mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                             float* __restrict__ o, float2* __restrict__ part_ml, float* __restrict__ part_acc,
-                            int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias) {
+                            int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias,
+                            const FusedArgs fa, int32_t* __restrict__ lens_advance) {
     using Cfg = MmaCfg<M_TILES>;
     constexpr int kStages = Cfg::kStages;
     const int seq = blockIdx.x / n_splits;
     const int split = blockIdx.x % n_splits;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
-    grid_launch_dependents();
-    const int L = clamp_len(biased_len(lens[seq], m_max, len_bias), m_max, threadIdx.x == 0 ? status : nullptr);
-    const int r0 = split * chunk_rows;
-    const int r1 = min(L, r0 + chunk_rows);
-    if (r0 >= L) {                                         // nothing valid in this split (uniform)
-        if (n_splits == 1)                                 // L == 0: the empty prefix gives zeros
-            for (int i = threadIdx.x; i < h * kHeadDim; i += Cfg::kThreads) o[(size_t)seq * h * kHeadDim + i] = 0.f;
-        return;
-    }
-    const int n_tiles = (r1 - r0 + kTileRows - 1) / kTileRows;
 
     extern __shared__ uint8_t smem_raw[];
     // 1 KiB alignment in the shared window: the 128-byte swizzle repeats every 8 rows x 128 bytes
@@ -348,6 +347,33 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // everything above overlaps the tail of the kernel before this one
+    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
+    grid_launch_dependents();
+    // With one CTA per sequence (n_splits == 1) the CTA may do the whole decoding step: write the new row
+    // (fa.k_new given), attend over one row more, and move lens[seq] on at the end (lens_advance given) --
+    // nobody else reads this sequence's length.
+    const int raw = lens[seq];
+    const bool appended = fa.k_new != nullptr && raw >= 0 && raw < m_max;
+    if (fa.k_new != nullptr) {
+        if (!appended && threadIdx.x == 0 && status) atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
+        if (appended && warp == 0) {                       // lanes 0-15 move the key row, 16-31 the value row
+            const size_t src = (size_t)seq * (kRowBytes / 16) + (lane & 15);
+            const size_t dst = ((size_t)seq * m_max + raw) * (kRowBytes / 16) + (lane & 15);
+            if (lane < 16) fa.K[dst] = fa.k_new[src]; else fa.V[dst] = fa.v_new[src];
+            asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row (a barrier follows)
+        }
+    }
+    const int L = clamp_len(appended ? raw + 1 : biased_len(raw, m_max, len_bias), m_max, threadIdx.x == 0 ? status : nullptr);
+    const int r0 = split * chunk_rows;
+    const int r1 = min(L, r0 + chunk_rows);
+    if (r0 >= L) {                                         // nothing valid in this split (uniform)
+        if (n_splits == 1)                                 // L == 0: the empty prefix gives zeros
+            for (int i = threadIdx.x; i < h * kHeadDim; i += Cfg::kThreads) o[(size_t)seq * h * kHeadDim + i] = 0.f;
+        return;
+    }
+    const int n_tiles = (r1 - r0 + kTileRows - 1) / kTileRows;
+
     __syncthreads();
 
     const int mt = warp % M_TILES;                         // which 16-head tile this warp serves
@@ -460,6 +486,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
             if (c == 0) part_ml[slot] = make_float2(top, den);
         }
     }
+    if (lens_advance && appended && threadIdx.x == 0) lens_advance[seq] = raw + 1;   // every thread read lens[seq] barriers ago
 }
 
 // =============================================================================================
@@ -527,17 +554,6 @@ __host__ __device__ inline size_t stream_ml_bytes(int slots, int h) {
     return (((size_t)slots * h * sizeof(float2)) + 255) & ~(size_t)255;
 }
 __host__ __device__ inline size_t stream_acc_bytes(int slots, int h) { return (size_t)slots * h * kHeadDim * sizeof(float); }
-
-// What the append-and-attend step (FUSED) does on top of the pass over the cache: the CTA whose share
-// holds a sequence's last tile writes the new token's key and value row (row lens[b]) into the cache
-// just before it fetches that tile, so the step attends over lens[b] + 1 rows without a separate
-// append launch.  lens itself is advanced by the second-pass kernel, when no CTA reads it any more.
-struct FusedArgs {
-    const uint4* k_new;      // [b, 128] bf16 rows as 16-byte words; null = nothing to append
-    const uint4* v_new;
-    uint4* K;                // the cache, written at row lens[b]
-    uint4* V;
-};
 
 // lens[s], read from L2 (the kernels before and after this one may write lens).
 template <bool FUSED>
@@ -678,8 +694,9 @@ template <int GROUPS>
 __global__ void __launch_bounds__(kHeadDim * GROUPS)
 stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restrict__ part_ml,
                       const float* __restrict__ part_acc, float* __restrict__ o, int b, int h,
-                      int32_t* lens_advance, int m_max) {
+                      int32_t* lens_advance, int m_max, unsigned long long magic) {
     const int s = blockIdx.x / h, head = blockIdx.x % h;
+    grid_launch_dependents();        // the kernel after this one may set itself up; it waits before it reads
     grid_dependency_wait();          // the slots come from the kernel before this one
     if (lens_advance && head == 0 && threadIdx.x == 0) {   // append-and-attend step: lens[s] += 1 for a sequence that took a row
         const int raw = lens_advance[s];
@@ -687,14 +704,14 @@ stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restric
     }
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
-    const long long T = seq_span[b].x, G = seq_span[b].y;
+    const int T = seq_span[b].x;                        // length of the line (magic: the first pass's grid size, see share_begin)
     const int n_cta = span.y - span.x + 1;              // at most the grid of the first pass (<= 256 SMs)
     // piece i is the slot of CTA span.x + i; a CTA whose share of the line is empty wrote none (max = -inf)
     merge_pieces<GROUPS>(
         n_cta,
         [&](int i) {
-            const long long cta = span.x + i;
-            const bool live = cta * T / G != (cta + 1) * T / G;
+            const int cta = span.x + i;
+            const bool live = share_begin(cta, T, magic) != share_begin(cta + 1, T, magic);
             return live ? __ldcg(part_ml + ((size_t)cta + s) * h + head) : make_float2(-INFINITY, 0.f);
         },
         [&](int i) { return part_acc + (((size_t)span.x + i + s) * h + head) * kHeadDim; },
