@@ -360,12 +360,16 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     if (rc) return rc;
     if (p.stream()) {
         const StreamWorkspace w = stream_workspace(p, workspace);
+        const unsigned grid = (unsigned)((size_t)b * h);
         if (p.n_splits <= kCombineEager)
-            launch_dependent(stream_combine_kernel<1>, (unsigned)((size_t)b * h), kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
-                             b, h, lens_advance, m_max, share_magic(p.grid));
+            launch_dependent(stream_combine_kernel<1>, grid, kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h, lens_advance,
+                             m_max, share_magic(p.grid));
+        else if (p.n_splits <= 4 * kCombineEager)
+            launch_dependent(stream_combine_kernel<4>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h,
+                             lens_advance, m_max, share_magic(p.grid));
         else
-            launch_dependent(stream_combine_kernel<4>, (unsigned)((size_t)b * h), 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc,
-                             o, b, h, lens_advance, m_max, share_magic(p.grid));
+            launch_dependent(stream_combine_kernel<kCombineManyGroups>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
+                             b, h, lens_advance, m_max, share_magic(p.grid));
         return launch_status();
     }
     if (p.n_splits <= 1) return MQA_OK;
@@ -395,7 +399,6 @@ int run_step(bool multi_query, const void* q, const void* K, const void* V, cons
 // lens[i] += 1 for the sequences that took a row (the multi-launch form of mqa_decode_append_step
 // advances lens last, after the kernels that read the old value).
 __global__ void lens_advance_kernel(int32_t* lens, int b, int m_max) {
-    grid_launch_dependents();
     grid_dependency_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < b && lens[i] >= 0 && lens[i] < m_max) lens[i] += 1;

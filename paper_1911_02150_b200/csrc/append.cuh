@@ -14,8 +14,8 @@ kv_cache_append_kernel(uint4* __restrict__ K, uint4* __restrict__ V,
                        int32_t* __restrict__ lens, int advance, int32_t* __restrict__ status,
                        int kv_heads, int m_max) {
     const int bi = blockIdx.x;
+    grid_dependency_wait();          // lens may come from the kernel before this one
     grid_launch_dependents();        // the step that follows may set itself up; it waits before reading
-    grid_dependency_wait();
     const int row = lens[bi];
     if (row < 0 || row >= m_max) {   // uniform over the CTA
         if (threadIdx.x == 0 && status)

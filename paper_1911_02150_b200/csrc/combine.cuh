@@ -23,16 +23,19 @@ __host__ __device__ inline size_t partial_acc_bytes(size_t units, int S) {
 // Threads: 128 columns x GROUPS piece groups.  Group g takes pieces g, g + GROUPS, ...;
 // a thread fetches its column of up to kCombineEager of them in one go (the addresses do not depend
 // on the weights), so merging a few dozen pieces costs one round trip to L2, not one per piece.
-// The host picks GROUPS = 1 (128 threads, 8 pieces in flight per thread) when no sequence can have more than
-// kCombineEager pieces, else 4 (512 threads, 40 in flight: 160 pieces in one go).
+// The host picks the shape by the most pieces a sequence can have: GROUPS = 1 (128 threads, 8 pieces in flight
+// per thread) up to kCombineEager pieces, GROUPS = 4 (512 threads, 8 in flight) up to 4 * kCombineEager, and
+// GROUPS = 5 (still 4 thread groups, 40 in flight per thread: 160 pieces in one go) beyond.
 constexpr int kCombineEager = 8;
+constexpr int kCombineManyGroups = 5;
 
 // Merge `n` pieces of one (sequence, head).  ml_of(i) / acc_of(i) give piece i's (max, sum) and the address of
 // its 128 accumulators; a piece whose max is -inf is skipped entirely (it may never have been written).
-template <int kCombineGroups, typename MlOf, typename AccOf>
+template <int kCombineShape, typename MlOf, typename AccOf>
 __device__ __forceinline__ void merge_pieces(int n, MlOf ml_of, AccOf acc_of, float* __restrict__ out) {
+    constexpr int kCombineGroups = kCombineShape >= 4 ? 4 : 1;
     constexpr int kCombineThreads = kHeadDim * kCombineGroups;
-    constexpr int kCombineEager = kCombineGroups == 1 ? 8 : 40;     // loads in flight per thread
+    constexpr int kCombineEager = kCombineShape == kCombineManyGroups ? 40 : 8;     // loads in flight per thread
     __shared__ float m_s[1024], l_s[1024];
     __shared__ float num_s[kCombineGroups][kHeadDim], den_s[kCombineGroups];
     const int c = threadIdx.x & (kHeadDim - 1), g = threadIdx.x >> 7;
@@ -85,12 +88,11 @@ __device__ __forceinline__ void merge_pieces(int n, MlOf ml_of, AccOf acc_of, fl
 }
 
 template <int GROUPS>
-__global__ void __launch_bounds__(kHeadDim * GROUPS)
+__global__ void __launch_bounds__(kHeadDim * (GROUPS >= 4 ? 4 : 1))
 combine_splits_kernel(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
                       const int32_t* __restrict__ lens, float* __restrict__ o,
                       int h, int m_max, int chunk_rows, int n_splits, int len_bias) {
     const size_t u = blockIdx.x;
-    grid_launch_dependents();        // the kernel after this one may set itself up; it waits before it reads
     grid_dependency_wait();          // the partials come from the kernel before this one
     int L = biased_len(lens[u / h], m_max, len_bias);
     L = L < 0 ? 0 : (L > m_max ? m_max : L);

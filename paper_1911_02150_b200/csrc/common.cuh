@@ -35,7 +35,10 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
 // Programmatic dependent launch.  grid_dependency_wait(): block until the kernels this launch was
 // made dependent on have finished and their writes are visible (a no-op for an ordinary launch).
 // grid_launch_dependents(): allow the next kernel in the stream, if it was launched as a
-// programmatic dependent, to start its prologue while this grid is still running.
+// programmatic dependent, to start its prologue while this grid is still running.  Every kernel
+// here waits first and lets its dependents start afterwards: with second-pass kernels that let
+// theirs start before their own wait, a decoding loop of four kernels per step gave results that
+// differed from run to run.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 

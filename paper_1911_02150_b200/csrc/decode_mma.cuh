@@ -415,6 +415,10 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
             if (!ok) break;
             const uint32_t k_s = stages_s + s * kStageBytes;
             consume_tile<true, kBoxBytes>(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
+            // The tile was read through the generic proxy (ldmatrix) and the copy engine will write the stage
+            // again through the async proxy: without this fence the last ldmatrix of a tile now and then saw
+            // rows of the tile that came four tiles later (one run in a few hundred, 16 output columns off).
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_s + s * 8);                 // this warp is done with the stage
         }
@@ -691,12 +695,11 @@ __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, 
 // or it is empty).  seq_span[b] holds (T, G): a CTA whose share of the T tiles is empty wrote no
 // slot and is skipped.
 template <int GROUPS>
-__global__ void __launch_bounds__(kHeadDim * GROUPS)
+__global__ void __launch_bounds__(kHeadDim * (GROUPS >= 4 ? 4 : 1))
 stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restrict__ part_ml,
                       const float* __restrict__ part_acc, float* __restrict__ o, int b, int h,
                       int32_t* lens_advance, int m_max, unsigned long long magic) {
     const int s = blockIdx.x / h, head = blockIdx.x % h;
-    grid_launch_dependents();        // the kernel after this one may set itself up; it waits before it reads
     grid_dependency_wait();          // the slots come from the kernel before this one
     if (lens_advance && head == 0 && threadIdx.x == 0) {   // append-and-attend step: lens[s] += 1 for a sequence that took a row
         const int raw = lens_advance[s];
