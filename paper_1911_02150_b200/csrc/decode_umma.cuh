@@ -753,6 +753,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     if (j >= 2 && ok) ok = mbar_wait(pv_done + pb * 8, ((j >> 1) - 1) & 1);
                     if ((hilo || prev_hilo) && j >= 1 && ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
                     prev_hilo = hilo;
+                    tc_fence_after();                       // the tensor core's reads of the tile come before the stores below
                     // ---- P = exp2(S - reference): 0 for a masked row; bf16 hi (and lo) into the P^T tiles
                     const uint32_t p_hi = p_s + (hilo ? 0 : pb) * Cfg::kPBytes + p_row, p_lo = p_s + Cfg::kPBytes + p_row;
 #pragma unroll
