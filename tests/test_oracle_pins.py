@@ -490,3 +490,68 @@ def test_threads_are_reported_and_do_not_change_results():
     c = oracle.mqa_decode_step(qb, Kb, Vb, lens)
     oracle.set_num_threads(n)
     assert np.array_equal(a, c)
+
+
+# ---------------------------------------------------------------------------------------------
+# The whole-layer oracle (projections either side of the step), Section 3
+# ---------------------------------------------------------------------------------------------
+def _layer_case(seed, b=3, h=4, d=24, k=8, v=8, m=5):
+    from oracle import layer_step as ls
+    r = np.random.default_rng(seed)
+    def bf(shape, std):
+        return ls.f64_to_bf16_bits(r.normal(0.0, std, size=shape))
+    x, Pq, Pk, Pv, Po = bf((b, d), 1.0), bf((h, d, k), d ** -0.5), bf((d, k), d ** -0.5), bf((d, v), d ** -0.5), bf((h, d, v), (h * v) ** -0.5)
+    K, V = bf((b, m + 1, k), 1.0), bf((b, m + 1, v), 1.0)
+    return ls, x, Pq, Pk, Pv, Po, K, V, m
+
+
+def test_layer_oracle_without_interface_roundings_is_the_papers_incremental_function():
+    ls, x, Pq, Pk, Pv, Po, K, V, m = _layer_case(11)
+    b = x.shape[0]
+    lens = np.full(b, m, np.int32)
+    Kc, Vc = K.copy(), V.copy()
+    y, qb, kb, vb = ls.multiquery_layer_decode_step(x, Pq, Pk, Pv, Po, Kc, Vc, lens, round_interfaces=False)
+    f = ls.bf16_to_f64
+    # the paper's function keeps the new row unrounded; give it the row as the bf16 cache holds it by projecting
+    # with the same inputs and checking the two agree to bf16 precision on the row, exactly on everything else
+    y_ref, K_ref, V_ref = pf.multiquery_self_attention_incremental(f(x), f(K[:, :m]), f(V[:, :m]), f(Pq), f(Pk), f(Pv), f(Po))
+    assert np.array_equal(lens, np.full(b, m + 1))
+    assert np.array_equal(Kc[:, :m], K[:, :m]) and np.array_equal(Vc[:, :m], V[:, :m])
+    np.testing.assert_allclose(f(Kc[:, m]), K_ref[:, m], rtol=2 ** -8, atol=1e-30)       # one bf16 rounding of the new row
+    np.testing.assert_allclose(f(Vc[:, m]), V_ref[:, m], rtol=2 ** -8, atol=1e-30)
+    # attending, head by head with the paper's single-query function, over the cache as stored (rounded row): y to fp64
+    Kf, Vf = f(Kc), f(Vc)
+    y_chk = np.zeros_like(y)
+    for s in range(b):
+        for i in range(Pq.shape[0]):
+            y_chk[s] += f(Po)[i] @ pf.attend(f(x)[s] @ f(Pq)[i], Kf[s], Vf[s])
+    np.testing.assert_allclose(y, y_chk, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(y, y_ref, rtol=0, atol=2e-2)                             # the row's rounding moves y only slightly
+
+
+def test_layer_oracle_interface_roundings_are_small_and_where_stated():
+    ls, x, Pq, Pk, Pv, Po, K, V, m = _layer_case(12)
+    b = x.shape[0]
+    y0, qb0, kb0, vb0 = ls.multiquery_layer_decode_step(x, Pq, Pk, Pv, Po, K.copy(), V.copy(), np.full(b, m, np.int32), round_interfaces=False)
+    y1, qb1, kb1, vb1 = ls.multiquery_layer_decode_step(x, Pq, Pk, Pv, Po, K.copy(), V.copy(), np.full(b, m, np.int32), round_interfaces=True)
+    assert np.array_equal(qb0, qb1) and np.array_equal(kb0, kb1) and np.array_equal(vb0, vb1)
+    assert 0 < np.abs(y0 - y1).max() < 2e-2
+    f = ls.bf16_to_f64
+    assert np.array_equal(ls.f64_to_bf16_bits(f(qb1)), qb1)                              # rounding is idempotent
+    # ties to even, and exactness of the widening
+    assert ls.f64_to_bf16_bits(np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8]))[0] == 0x3F80 and ls.f64_to_bf16_bits(np.array([1.0 + 3 * 2 ** -8]))[0] == 0x3F82
+    assert f(np.array([0x3F80, 0xC000], np.uint16)).tolist() == [1.0, -2.0]
+
+
+def test_layer_oracle_empty_and_full_sequences():
+    ls, x, Pq, Pk, Pv, Po, K, V, m = _layer_case(13)
+    b = x.shape[0]
+    lens = np.array([0, m, m + 1], np.int32)                                            # first token; normal; cache full
+    Kc, Vc = K.copy(), V.copy()
+    y, _, kb, vb = ls.multiquery_layer_decode_step(x, Pq, Pk, Pv, Po, Kc, Vc, lens)
+    assert lens.tolist() == [1, m + 1, m + 1]
+    assert np.array_equal(Kc[0, 0], kb[0]) and np.array_equal(Kc[2], K[2])              # row 0 written; full cache untouched
+    f = ls.bf16_to_f64
+    # a single row: the output is that value row, whatever the query
+    o_single = f(ls.f64_to_bf16_bits(f(vb[0])))
+    np.testing.assert_allclose(y[0], np.einsum("hv,hdv->d", np.tile(o_single, (Pq.shape[0], 1)), f(Po)), rtol=1e-12, atol=1e-13)
