@@ -218,6 +218,33 @@ int mqa_decode_step_noalloc(const void* q, const void* K, const void* V, const i
  */
 int mqa_append_step_launches(int b, int h, int m_max, int k, int v);
 
+/*
+ * mqa_layer_decode_step -- the whole incremental multi-query layer of Section 3
+ * (MultiquerySelfAttentionIncremental) for one new token per sequence: the projections
+ * q = einsum(bd,hdk->bhk)(x, P_q), k_new = einsum(bd,dk->bk)(x, P_k), v_new = einsum(bd,dv->bv)(x, P_v),
+ * then what mqa_decode_append_step does with them (the new row is concatenated to the cache at row
+ * lens[b], the h heads attend over lens[b] + 1 rows), then y = einsum(bhv,hdv->bd)(o, P_o).
+ *
+ *   x                [b, d] bf16                 P_q  [h, d, k] bf16        P_k, P_v  [d, k], [d, v] bf16
+ *   P_o              [h, d, v] bf16              K, V, lens, advance, status   as for mqa_decode_append_step
+ *   y                [b, d] fp32, written
+ *   workspace        at least mqa_layer_workspace_bytes(b, h, d, m_max, k, v) bytes; may hold anything on entry.
+ *                    It carries q, k_new, v_new (bf16), o (fp32), the per-head-group partial sums of y and the
+ *                    attention step's own workspace.
+ * d must be a multiple of 128 (MQA_ERR_UNSUPPORTED otherwise), k = v = 128.  The products run on the tensor
+ * cores in bf16 with fp32 accumulation; q, k_new and v_new are rounded to bf16 where the step and the cache
+ * take them, o is rounded to bf16 as an operand of the output product; y is summed over head groups in a fixed
+ * order (no float atomics: results are reproducible bit for bit).  Kernels: projections in, the step (one
+ * launch for large batches), projection out, the sum over head groups.
+ */
+int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const void* P_v, const void* P_o,
+                          void* K, void* V, int32_t* lens, int advance, float* y,
+                          void* workspace, size_t workspace_bytes, int32_t* status,
+                          int b, int h, int d, int m_max, int k, int v, mqa_stream_t stream);
+
+/* mqa_layer_workspace_bytes -- scratch mqa_layer_decode_step needs (0 for invalid or unsupported sizes). Host-only. */
+size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v);
+
 /* mqa_status_string -- a static, human-readable name for a return code. */
 const char* mqa_status_string(int code);
 

@@ -27,6 +27,7 @@ EXPORTS = (
     "mha_decode_step_split", "mha_decode_step_combine",
     "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
+    "mqa_layer_decode_step", "mqa_layer_workspace_bytes",
 )
 
 _lib = None
@@ -64,6 +65,10 @@ def lib() -> ctypes.CDLL:
         L.mqa_decode_append_step.restype = I
         L.mqa_append_step_launches.argtypes = [I, I, I, I, I]
         L.mqa_append_step_launches.restype = I
+        L.mqa_layer_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, I, vp, vp, sz, vp, I, I, I, I, I, I, vp]
+        L.mqa_layer_decode_step.restype = I
+        L.mqa_layer_workspace_bytes.argtypes = [I, I, I, I, I, I]
+        L.mqa_layer_workspace_bytes.restype = sz
         L.mqa_workspace_bytes.argtypes = [I, I, I, I, I]
         L.mqa_workspace_bytes.restype = sz
         L.mqa_plan_splits.argtypes = [I, I, I, I, I, I, ctypes.POINTER(I)]
@@ -249,3 +254,37 @@ def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, statu
                                           b, h, m_max, k, v, _stream(stream))
     _check(rc, "mqa_decode_append_step")
     return o
+
+
+def layer_workspace_bytes(b: int, h: int, d: int, m_max: int, k: int = 128, v: int = 128) -> int:
+    return int(lib().mqa_layer_workspace_bytes(b, h, d, m_max, k, v))
+
+
+def alloc_layer_workspace(b: int, h: int, d: int, m_max: int, device) -> torch.Tensor:
+    return torch.empty(max(16, layer_workspace_bytes(b, h, d, m_max)), dtype=torch.uint8, device=device)
+
+
+def mqa_layer_decode_step(x, P_q, P_k, P_v, P_o, K, V, lens, y, workspace, status=None, advance: bool = True, stream=None):
+    """The whole incremental multi-query layer step: projections of ``x[b,d]`` to q, k_new, v_new, append +
+    attention over the shared cache, output projection to ``y[b,d]`` (fp32)."""
+    b, d = x.shape
+    h, _, k = P_q.shape
+    m_max, v = K.shape[-2], V.shape[-1]
+    _need(x, torch.bfloat16, (b, d), "x")
+    _need(P_q, torch.bfloat16, (h, d, k), "P_q")
+    _need(P_k, torch.bfloat16, (d, k), "P_k")
+    _need(P_v, torch.bfloat16, (d, v), "P_v")
+    _need(P_o, torch.bfloat16, (h, d, v), "P_o")
+    _need(K, torch.bfloat16, (b, m_max, k), "K")
+    _need(V, torch.bfloat16, (b, m_max, v), "V")
+    _need(lens, torch.int32, (b,), "lens")
+    _need(y, torch.float32, (b, d), "y")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    with torch.cuda.device(x.device):
+        rc = lib().mqa_layer_decode_step(_ptr(x), _ptr(P_q), _ptr(P_k), _ptr(P_v), _ptr(P_o), _ptr(K), _ptr(V), _ptr(lens),
+                                         int(bool(advance)), _ptr(y), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _ptr(status),
+                                         b, h, d, m_max, k, v, _stream(stream))
+    _check(rc, "mqa_layer_decode_step")
+    return y

@@ -13,6 +13,7 @@
 #include "combine.cuh"
 #include "common.cuh"
 #include "decode_mma.cuh"
+#include "project.cuh"
 #include "decode_simt.cuh"
 #include "decode_umma.cuh"
 
@@ -239,6 +240,19 @@ bool encode_cache_map(CUtensorMap* map, const void* base, long long rows, int bo
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A row-major bf16 matrix [rows][cols] fetched in boxes of box_rows rows x 64 columns (128-byte swizzle).
+bool encode_matrix_map(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 std::atomic<int> g_smem_opt_in[kMaxDevices][2];
 
 template <int M_TILES>
@@ -404,6 +418,99 @@ __global__ void lens_advance_kernel(int32_t* lens, int b, int m_max) {
     if (i < b && lens[i] >= 0 && lens[i] < m_max) lens[i] += 1;
 }
 
+// ---- the whole layer step: projections, append + attention, output projection ---------------------
+size_t align256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+struct LayerWorkspace {
+    size_t q, k_new, v_new, o, part_y, step, total;     // byte offsets
+    int groups;                                         // head groups of the output projection
+};
+LayerWorkspace layer_workspace(int b, int h, int d, int m_max) {
+    LayerWorkspace w;
+    w.groups = (h + kProjHeadsPerCta - 1) / kProjHeadsPerCta;
+    size_t at = 0;
+    w.q = at;      at += align256((size_t)b * h * kHeadDim * 2);
+    w.k_new = at;  at += align256((size_t)b * kHeadDim * 2);
+    w.v_new = at;  at += align256((size_t)b * kHeadDim * 2);
+    w.o = at;      at += align256((size_t)b * h * kHeadDim * 4);
+    w.part_y = at; at += align256((size_t)w.groups * b * d * 4);
+    w.step = at;   at += align256(plan_workspace_bytes(make_plan(true, b, h, m_max)));
+    w.total = at;
+    return w;
+}
+
+std::atomic<int> g_proj_opt_in[kMaxDevices][8];
+
+template <int NB>
+int launch_projections_in(const void* x, const void* P_q, const void* P_k, const void* P_v, void* q, void* k_new, void* v_new,
+                          int32_t* status, int b, int h, int d, cudaStream_t stream) {
+    using Cfg = ProjCfg<NB>;
+    auto kernel = project_in_kernel<NB>;
+    constexpr int kSlot = NB == 16 ? 0 : (NB == 32 ? 1 : (NB == 64 ? 2 : 3));
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!g_proj_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+        g_proj_opt_in[dev][kSlot].store(1, std::memory_order_release);
+    }
+    alignas(64) CUtensorMap map_pq, map_pk, map_pv, map_x;
+    if (!encode_matrix_map(&map_pq, P_q, (long long)h * d, kHeadDim, 128) || !encode_matrix_map(&map_pk, P_k, d, kHeadDim, 128) ||
+        !encode_matrix_map(&map_pv, P_v, d, kHeadDim, 128) || !encode_matrix_map(&map_x, x, b, d, NB))
+        return MQA_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(h + 2), (unsigned)((b + 127) / 128));
+    cfg.blockDim = dim3(kProjThreads);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, map_pq, map_pk, map_pv, map_x, static_cast<__nv_bfloat16*>(q),
+                       static_cast<__nv_bfloat16*>(k_new), static_cast<__nv_bfloat16*>(v_new), status, b, h, d);
+    return launch_status();
+}
+
+template <int NB>
+int launch_projection_out(const void* P_o, const float* o, float* part_y, float* y, int groups, int32_t* status, int b, int h,
+                          int d, cudaStream_t stream) {
+    using Cfg = ProjCfg<NB>;
+    auto kernel = project_out_kernel<NB>;
+    constexpr int kSlot = 4 + (NB == 16 ? 0 : (NB == 32 ? 1 : (NB == 64 ? 2 : 3)));
+    constexpr int kSmem = 2 * Cfg::kStageBytes + 256 + 1024;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!g_proj_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+        g_proj_opt_in[dev][kSlot].store(1, std::memory_order_release);
+    }
+    alignas(64) CUtensorMap map_po;
+    if (!encode_matrix_map(&map_po, P_o, (long long)h * d, kHeadDim, 128)) return MQA_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(d / 128), (unsigned)groups, (unsigned)((b + 127) / 128));
+    cfg.blockDim = dim3(kProjThreads);
+    cfg.dynamicSmemBytes = kSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, map_po, o, part_y, status, b, h, d);
+    if (launch_status()) return MQA_ERR_CUDA;
+    const int n = b * d;
+    launch_dependent(reduce_y_kernel, (unsigned)((n / 4 + 255) / 256), 256u, 0, stream, static_cast<const float*>(part_y), y, n,
+                     groups);
+    return launch_status();
+}
+
 }  // namespace
 }  // namespace mqa
 
@@ -506,6 +613,49 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
         return launch_status();
     }
     return MQA_OK;
+}
+
+size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v) {
+    if (!dims_ok(b, h, m_max) || d <= 0 || d % 128 != 0 || k != kHeadDim || v != kHeadDim) return 0;
+    return layer_workspace(b, h, d, m_max).total;
+}
+
+int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const void* P_v, const void* P_o, void* K, void* V,
+                          int32_t* lens, int advance, float* y, void* workspace, size_t workspace_bytes, int32_t* status,
+                          int b, int h, int d, int m_max, int k, int v, mqa_stream_t stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!x || !P_q || !P_k || !P_v || !P_o || !K || !V || !lens || !y || !workspace) return MQA_ERR_INVALID_ARG;
+    if (!dims_ok(b, h, m_max) || d <= 0 || k <= 0 || v <= 0) return MQA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(P_q) || !aligned16(P_k) || !aligned16(P_v) || !aligned16(P_o) || !aligned16(K) ||
+        !aligned16(V) || !aligned16(y) || !aligned16(workspace) || !aligned4(lens) || !aligned4(status))
+        return MQA_ERR_INVALID_ARG;
+    if (k != kHeadDim || v != kHeadDim || d % 128 != 0 || (long long)h * d >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
+    const LayerWorkspace w = layer_workspace(b, h, d, m_max);
+    if (workspace_bytes < w.total) return MQA_ERR_WORKSPACE_TOO_SMALL;
+    char* base = static_cast<char*>(workspace);
+    void* q = base + w.q;
+    void* k_new = base + w.k_new;
+    void* v_new = base + w.v_new;
+    float* o = reinterpret_cast<float*>(base + w.o);
+    float* part_y = reinterpret_cast<float*>(base + w.part_y);
+    const int nb = b >= 128 ? 128 : (b > 64 ? 128 : (b > 32 ? 64 : (b > 16 ? 32 : 16)));
+    int rc;
+    switch (nb) {
+        case 16: rc = launch_projections_in<16>(x, P_q, P_k, P_v, q, k_new, v_new, status, b, h, d, stream); break;
+        case 32: rc = launch_projections_in<32>(x, P_q, P_k, P_v, q, k_new, v_new, status, b, h, d, stream); break;
+        case 64: rc = launch_projections_in<64>(x, P_q, P_k, P_v, q, k_new, v_new, status, b, h, d, stream); break;
+        default: rc = launch_projections_in<128>(x, P_q, P_k, P_v, q, k_new, v_new, status, b, h, d, stream); break;
+    }
+    if (rc) return rc;
+    rc = mqa_decode_append_step(q, K, V, k_new, v_new, lens, advance, o, base + w.step, w.total - w.step, status, b, h, m_max, k,
+                                v, stream_);
+    if (rc) return rc;
+    switch (nb) {
+        case 16: return launch_projection_out<16>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
+        case 32: return launch_projection_out<32>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
+        case 64: return launch_projection_out<64>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
+        default: return launch_projection_out<128>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
+    }
 }
 
 size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v) {
