@@ -250,6 +250,37 @@ def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=T
             "min_region_s": min(regions), "regions": len(regions), "graph": bool(use_graph)}
 
 
+def layer_block(mqa, w, device, seed, steps, d_model=1024):
+    """The whole incremental multi-query layer step (projections of x[b,d] to q, k_new, v_new; append + attention;
+    output projection) on the same workload, d = 1024 as in the paper's models: µs per step, K steps as one CUDA graph,
+    cache sets rotated past L2.  The weights (2 h d 128 + 2 d 128 bf16 elements) are read every step as well."""
+    gen = torch.Generator(device=device).manual_seed(seed + 17)
+    n = lambda shape, std: wl.bf16_normal(shape, std, gen, device)
+    b, h, m, d = w.b, w.h, w.m_max, d_model
+    W = [n((h, d, 128), (d * 128) ** -0.5), n((d, 128), d ** -0.5), n((d, 128), d ** -0.5), n((h, d, 128), (h * 128) ** -0.5)]
+    nset = max(1, min(8, (8 * L2_BYTES + b * m * 512 - 1) // (b * m * 512)))
+    sets = [(n((b, d), 1.0), n((b, m, 128), 1.0), n((b, m, 128), 1.0)) for _ in range(nset)]
+    lens = torch.from_numpy(wl.initial_lens(w, seed)).to(device)
+    y = torch.empty(b, d, dtype=torch.float32, device=device)
+    ws = mqa.alloc_layer_workspace(b, h, d, m, device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def step(i):
+        x, K, V = sets[i % nset]
+        mqa.mqa_layer_decode_step(x, W[0], W[1], W[2], W[3], K, V, lens, y, ws, status, advance=False)
+
+    for i in range(3):
+        step(i)
+    torch.cuda.synchronize(device)
+    g = capture_graph(step, steps)
+    g.replay()
+    torch.cuda.synchronize(device)
+    secs = statistics.median(time_region(lambda _i: g.replay(), 1, device) for _ in range(20))
+    weight_bytes = sum(t.numel() * 2 for t in W)
+    return {"us_per_step": secs / steps * 1e6, "d_model": d, "weight_bytes": weight_bytes, "status": int(status.item()),
+            "launches_per_step": 3 + mqa.append_step_launches(b, h, m), "cache_sets": nset}
+
+
 def cpu_baseline(w, seed, budget_s=20.0):
     """The oracle, as it stands, on the host cores: one multi-query step of the same workload on
     as many whole sequences as fit the time budget."""
@@ -336,6 +367,7 @@ def main():
     ap.add_argument("--workload", default="long_context")
     ap.add_argument("--no-mha", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-layer", action="store_true", help="skip the timing of the whole layer step (projections either side)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true", help="run every workload and write gpurun_out/sweep.json")
     args = ap.parse_args()
@@ -412,6 +444,9 @@ def main():
         out["mqa_speedup_over_mha"] = out["mha"]["us_per_step"] / blk["us_per_step"]
         del sth
         torch.cuda.empty_cache()
+    if not args.no_layer:
+        out["layer_step"] = layer_block(mqa, w, device, seed, max(3, min(args.steps, 20)))
+        out["layer_step"]["projections_us"] = out["layer_step"]["us_per_step"] - blk["us_per_step"]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, seed)
     if rank == 0:

@@ -506,8 +506,7 @@ int launch_projection_out(const void* P_o, const float* o, float* part_y, float*
     cudaLaunchKernelEx(&cfg, kernel, map_po, o, part_y, status, b, h, d);
     if (launch_status()) return MQA_ERR_CUDA;
     const int n = b * d;
-    launch_dependent(reduce_y_kernel, (unsigned)((n / 4 + 255) / 256), 256u, 0, stream, static_cast<const float*>(part_y), y, n,
-                     groups);
+    launch_dependent(reduce_y_kernel, (unsigned)((n + 255) / 256), 256u, 0, stream, static_cast<const float*>(part_y), y, n, groups);
     return launch_status();
 }
 

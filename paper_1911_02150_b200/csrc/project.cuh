@@ -274,19 +274,22 @@ project_out_kernel(const __grid_constant__ CUtensorMap map_po, const float* __re
     if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem, Cfg::kTmemCols); }
 }
 
-// y[b, d] = sum over the head groups of project_out_kernel, in group order
+// y[b, d] = sum over the head groups of project_out_kernel, in group order (8 loads in flight per thread)
 __global__ void __launch_bounds__(256)
 reduce_y_kernel(const float* __restrict__ part_y, float* __restrict__ y, int n, int groups) {
     grid_dependency_wait();
     grid_launch_dependents();
-    const int i = blockIdx.x * 256 + threadIdx.x;      // one float4 of y
-    if (i * 4 >= n) return;
-    float4 acc = __ldcg(reinterpret_cast<const float4*>(part_y) + i);
-    for (int g = 1; g < groups; ++g) {
-        const float4 p = __ldcg(reinterpret_cast<const float4*>(part_y + (size_t)g * n) + i);
-        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+    const int i = blockIdx.x * 256 + threadIdx.x;      // one element of y
+    if (i >= n) return;
+    float acc = 0.f;
+    for (int g0 = 0; g0 < groups; g0 += 8) {
+        float p[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) p[e] = g0 + e < groups ? __ldcg(part_y + (size_t)(g0 + e) * n + i) : 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc += p[e];
     }
-    reinterpret_cast<float4*>(y)[i] = acc;
+    y[i] = acc;
 }
 
 }  // namespace mqa
