@@ -297,7 +297,8 @@ std::atomic<int> g_umma_opt_in[kMaxDevices][6];
 template <int HP, bool FUSED>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
-                const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
+                const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
+                bool late_wait = false) {
     using Cfg = UmmaCfg<HP>;
     auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED>;
     constexpr int kSlot = (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 2 + (FUSED ? 1 : 0);
@@ -326,19 +327,20 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     const StreamWorkspace w = stream_workspace(p, workspace);
     launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
                      map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa,
-                     merge ? w.ctrl : nullptr, lens_advance);
+                     merge ? w.ctrl : nullptr, lens_advance, late_wait ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
 template <bool FUSED>
 int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                     void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
-                    const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
+                    const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
+                    bool late_wait = false) {
     if (h <= 16)
-        return launch_umma<16, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance);
+        return launch_umma<16, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, late_wait);
     if (h <= 32)
-        return launch_umma<32, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance);
-    return launch_umma<64, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance);
+        return launch_umma<32, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, late_wait);
+    return launch_umma<64, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, late_wait);
 }
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
@@ -577,9 +579,11 @@ int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace
                        static_cast<cudaStream_t>(stream));
 }
 
-int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
-                           int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
-                           int h, int m_max, int k, int v, mqa_stream_t stream_) {
+// after_projection: the kernel before this step in the stream is the layer step's input projection (see late_wait in
+// mqa_decode_stream_umma_kernel)
+static int append_step_impl(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
+                            int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
+                            int h, int m_max, int k, int v, mqa_stream_t stream_, bool after_projection) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
@@ -592,8 +596,9 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
         // one launch: append inside the pass, pieces merged by the last CTA to deliver one, lens advanced at the end
         if (p.merge_in_kernel)
             return launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, true, k_new, v_new,
-                                         advance ? lens : nullptr);
-        rc = launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, false, k_new, v_new);
+                                         advance ? lens : nullptr, after_projection);
+        rc = launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, false, k_new, v_new, nullptr,
+                                   after_projection);
         if (rc) return rc;
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
     }
@@ -618,6 +623,13 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
         return launch_status();
     }
     return MQA_OK;
+}
+
+int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
+                           int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
+                           int h, int m_max, int k, int v, mqa_stream_t stream) {
+    return append_step_impl(q, K, V, k_new, v_new, lens, advance, o, workspace, workspace_bytes, status, b, h, m_max, k, v,
+                            stream, false);
 }
 
 size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v) {
@@ -652,8 +664,8 @@ int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const
         default: rc = launch_projections_in<128>(x, P_q, P_k, P_v, q, k_new, v_new, status, b, h, d, stream); break;
     }
     if (rc) return rc;
-    rc = mqa_decode_append_step(q, K, V, k_new, v_new, lens, advance, o, base + w.step, w.total - w.step, status, b, h, m_max, k,
-                                v, stream_);
+    rc = append_step_impl(q, K, V, k_new, v_new, lens, advance, o, base + w.step, w.total - w.step, status, b, h, m_max, k, v,
+                          stream_, true);
     if (rc) return rc;
     switch (nb) {
         case 16: return launch_projection_out<16>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);

@@ -315,7 +315,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               const int32_t* __restrict__ lens, float* __restrict__ o, int2* __restrict__ seq_span,
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
                               int b, int h, int m_max, unsigned long long magic, const FusedArgs fa,
-                              unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance) {
+                              unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int late_wait) {
     using Cfg = UmmaCfg<HP>;
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
@@ -423,8 +423,13 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         }
     };
 
-    grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
-    grid_launch_dependents();
+    // late_wait: the kernel before this one writes nothing but q and the new key/value row (the input projection
+    // of the layer step) and, like every kernel here, lets this one start only after its own wait -- so everything
+    // older is complete, and only the producer warp has to wait, before it touches q or the new row.
+    if (!late_wait) {
+        grid_dependency_wait();      // lens and the newest cache row may come from the kernel before
+        grid_launch_dependents();
+    }
     if (ctrl && threadIdx.x == 0) {
         const unsigned long long was = __ldcg(ctrl + 1);
         unsigned long long E = __ldcg(ctrl) == kCtrlMagic ? ((was + 1) & kCtrlEpochMask) : kCtrlFirstEpoch;
@@ -437,15 +442,27 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     int pre_issued = 0;
     if (warp == kUmmaProducerWarp) {
         Segment g0;
-        int r0;
-        if (first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g0, &r0)) {
-            const int new_row = (r0 & kAppendBit) ? (r0 & (kAppendBit - 1)) - 1 : -1;   // row this step appends
-            const int n_pre = min((g0.hi - g0.lo + kSubs - 1) / kSubs, NK < NV ? NK : NV);
-            if (appending && new_row >= g0.lo * kTileRows && new_row < min(g0.hi, g0.lo + n_pre * kSubs) * kTileRows)
+        int r0 = 0;
+        const bool fast = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g0, &r0);
+        const int new_row = (fast && (r0 & kAppendBit)) ? (r0 & (kAppendBit - 1)) - 1 : -1;   // row this step appends
+        const int n_pre = fast ? min((g0.hi - g0.lo + kSubs - 1) / kSubs, NK < NV ? NK : NV) : 0;
+        if (late_wait) {
+            // stages that do not hold the new row start while the kernel before this one is still running
+            if (lane == 0)
+                for (int u = g0.lo; pre_issued < n_pre && !(appending && new_row >= u * kTileRows && new_row < (u + kSubs) * kTileRows);
+                     u += kSubs, ++pre_issued)
+                    issue_stage(g0.s, u, g0.hi, pre_issued);
+            pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
+            grid_dependency_wait();      // q and the new row are there now
+            grid_launch_dependents();
+        }
+        if (fast) {
+            const int u0 = g0.lo + pre_issued * kSubs;
+            if (appending && new_row >= u0 * kTileRows && new_row < min(g0.hi, g0.lo + n_pre * kSubs) * kTileRows)
                 row_store(g0.s, new_row, row_load(g0.s));   // the new row lies in the stages started here
             if (lane == 0) {
                 issue_q(g0.s, 0);
-                for (int u = g0.lo; pre_issued < n_pre; u += kSubs, ++pre_issued) issue_stage(g0.s, u, g0.hi, pre_issued);
+                for (int u = u0; pre_issued < n_pre; u += kSubs, ++pre_issued) issue_stage(g0.s, u, g0.hi, pre_issued);
             }
             pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
         }
