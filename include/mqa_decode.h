@@ -219,6 +219,24 @@ int mqa_decode_step_noalloc(const void* q, const void* K, const void* V, const i
 int mqa_append_step_launches(int b, int h, int m_max, int k, int v);
 
 /*
+ * mqa_decode_local_step -- one decoding step of multi-query attention restricted to a local neighbourhood
+ * (Section 4.1: the current position and the previous window - 1 positions; Section 4.3: the memory tensors
+ * padded to the window size).  The cache is a ring of `window` rows per sequence: the new token's key/value row
+ * is written to row pos[b] % window and the h heads attend over the min(pos[b] + 1, window) rows that hold tokens
+ * (the order of the rows in the ring does not matter to a softmax).
+ *
+ *   q, k_new, v_new   [b, h, k], [b, k], [b, v] bf16
+ *   K, V              [b, window, k], [b, window, v] bf16, read-write
+ *   pos               [b] int32: tokens of the sequence before this step (0 for the first); advance != 0: pos[b] += 1
+ *   o                 [b, h, v] fp32, written;  status optional (APPEND_NEGATIVE_LEN for pos[b] < 0: no row, zeros)
+ * One launch (one CTA per sequence); no workspace.  Supported for h <= 32 and windows that one CTA covers (the
+ * plan for these sizes has a single split: windows of up to a few hundred rows; MQA_ERR_UNSUPPORTED otherwise).
+ */
+int mqa_decode_local_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* pos,
+                          int advance, float* o, int32_t* status, int b, int h, int window, int k, int v,
+                          mqa_stream_t stream);
+
+/*
  * mqa_layer_decode_step -- the whole incremental multi-query layer of Section 3
  * (MultiquerySelfAttentionIncremental) for one new token per sequence: the projections
  * q = einsum(bd,hdk->bhk)(x, P_q), k_new = einsum(bd,dk->bk)(x, P_k), v_new = einsum(bd,dv->bv)(x, P_v),

@@ -27,7 +27,7 @@ EXPORTS = (
     "mha_decode_step_split", "mha_decode_step_combine",
     "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
-    "mqa_layer_decode_step", "mqa_layer_workspace_bytes",
+    "mqa_layer_decode_step", "mqa_layer_workspace_bytes", "mqa_decode_local_step",
 )
 
 _lib = None
@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.mqa_append_step_launches.restype = I
         L.mqa_layer_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, I, vp, vp, sz, vp, I, I, I, I, I, I, vp]
         L.mqa_layer_decode_step.restype = I
+        L.mqa_decode_local_step.argtypes = [vp, vp, vp, vp, vp, vp, I, vp, vp, I, I, I, I, I, vp]
+        L.mqa_decode_local_step.restype = I
         L.mqa_layer_workspace_bytes.argtypes = [I, I, I, I, I, I]
         L.mqa_layer_workspace_bytes.restype = sz
         L.mqa_workspace_bytes.argtypes = [I, I, I, I, I]
@@ -288,3 +290,24 @@ def mqa_layer_decode_step(x, P_q, P_k, P_v, P_o, K, V, lens, y, workspace, statu
                                          b, h, d, m_max, k, v, _stream(stream))
     _check(rc, "mqa_layer_decode_step")
     return y
+
+
+def mqa_decode_local_step(q, K, V, k_new, v_new, pos, o, status=None, advance: bool = True, stream=None):
+    """One decoding step of local multi-query attention: ``K``/``V`` ``[b, window, 128]`` are rings of the last
+    ``window`` positions, ``pos[b]`` counts the tokens so far; the new row goes to row ``pos % window``."""
+    b, h, k = q.shape
+    window, v = K.shape[-2], V.shape[-1]
+    _need(q, torch.bfloat16, (b, h, k), "q")
+    _need(K, torch.bfloat16, (b, window, k), "K")
+    _need(V, torch.bfloat16, (b, window, v), "V")
+    _need(k_new, torch.bfloat16, (b, k), "k_new")
+    _need(v_new, torch.bfloat16, (b, v), "v_new")
+    _need(pos, torch.int32, (b,), "pos")
+    _need(o, torch.float32, (b, h, v), "o")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    with torch.cuda.device(q.device):
+        rc = lib().mqa_decode_local_step(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(pos), int(bool(advance)),
+                                         _ptr(o), _ptr(status), b, h, window, k, v, _stream(stream))
+    _check(rc, "mqa_decode_local_step")
+    return o

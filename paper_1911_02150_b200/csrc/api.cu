@@ -264,7 +264,7 @@ std::atomic<int> g_smem_opt_in[kMaxDevices][2];
 template <int M_TILES>
 int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias,
-               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
+               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr, bool ring = false) {
     using Cfg = MmaCfg<M_TILES>;
     auto kernel = mqa_decode_split_mma_kernel<M_TILES>;
     int dev = 0;
@@ -288,7 +288,7 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     }
     launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
                      static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
-                     p.n_splits, len_bias, fa, lens_advance);
+                     p.n_splits, len_bias, fa, lens_advance, ring ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -630,6 +630,22 @@ int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, c
                            int h, int m_max, int k, int v, mqa_stream_t stream) {
     return append_step_impl(q, K, V, k_new, v_new, lens, advance, o, workspace, workspace_bytes, status, b, h, m_max, k, v,
                             stream, false);
+}
+
+int mqa_decode_local_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* pos, int advance,
+                          float* o, int32_t* status, int b, int h, int window, int k, int v, mqa_stream_t stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_step_args(q, K, V, pos, o, status, b, h, window, k, v);
+    if (rc) return rc;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return MQA_ERR_INVALID_ARG;
+    const Plan p = plan_mma(b, h > 32 ? 32 : h, window);
+    // one CTA per sequence over the whole window: windows of up to a few hundred rows, at most 32 heads
+    if (h > 32 || p.n_splits != 1 || (long long)b * window >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
+    return p.kernel == Kernel::kMma1
+               ? launch_mma<1>(p, q, K, V, pos, o, nullptr, nullptr, status, b, h, window, stream, 0, k_new, v_new,
+                               advance ? pos : nullptr, true)
+               : launch_mma<2>(p, q, K, V, pos, o, nullptr, nullptr, status, b, h, window, stream, 0, k_new, v_new,
+                               advance ? pos : nullptr, true);
 }
 
 size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v) {

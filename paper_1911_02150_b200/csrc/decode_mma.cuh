@@ -321,7 +321,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                             float* __restrict__ o, float2* __restrict__ part_ml, float* __restrict__ part_acc,
                             int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias,
-                            const FusedArgs fa, int32_t* __restrict__ lens_advance) {
+                            const FusedArgs fa, int32_t* __restrict__ lens_advance, int ring) {
     using Cfg = MmaCfg<M_TILES>;
     constexpr int kStages = Cfg::kStages;
     const int seq = blockIdx.x / n_splits;
@@ -353,18 +353,21 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // With one CTA per sequence (n_splits == 1) the CTA may do the whole decoding step: write the new row
     // (fa.k_new given), attend over one row more, and move lens[seq] on at the end (lens_advance given) --
     // nobody else reads this sequence's length.
+    // ring: the cache is a window of the last m_max positions (local attention, Section 4.1): lens[seq] counts
+    // the tokens so far, the new row goes to row lens[seq] % m_max and min(lens[seq] + 1, m_max) rows are attended.
     const int raw = lens[seq];
-    const bool appended = fa.k_new != nullptr && raw >= 0 && raw < m_max;
+    const bool appended = fa.k_new != nullptr && raw >= 0 && (ring || raw < m_max);
     if (fa.k_new != nullptr) {
         if (!appended && threadIdx.x == 0 && status) atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
         if (appended && warp == 0) {                       // lanes 0-15 move the key row, 16-31 the value row
             const size_t src = (size_t)seq * (kRowBytes / 16) + (lane & 15);
-            const size_t dst = ((size_t)seq * m_max + raw) * (kRowBytes / 16) + (lane & 15);
+            const size_t dst = ((size_t)seq * m_max + (ring ? raw % m_max : raw)) * (kRowBytes / 16) + (lane & 15);
             if (lane < 16) fa.K[dst] = fa.k_new[src]; else fa.V[dst] = fa.v_new[src];
             asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row (a barrier follows)
         }
     }
-    const int L = clamp_len(appended ? raw + 1 : biased_len(raw, m_max, len_bias), m_max, threadIdx.x == 0 ? status : nullptr);
+    const int L = clamp_len(appended ? (ring ? min(raw + 1, m_max) : raw + 1) : biased_len(raw, m_max, len_bias), m_max,
+                            threadIdx.x == 0 ? status : nullptr);
     const int r0 = split * chunk_rows;
     const int r1 = min(L, r0 + chunk_rows);
     if (r0 >= L) {                                         // nothing valid in this split (uniform)
