@@ -219,6 +219,29 @@ int mqa_decode_step_noalloc(const void* q, const void* K, const void* V, const i
 int mqa_append_step_launches(int b, int h, int m_max, int k, int v);
 
 /*
+ * mqa_decode_append_step_host -- mqa_decode_append_step for a caller whose per-token inputs and result live in
+ * HOST memory (the decoder's other layers, a sampler): q, k_new, v_new are copied to the device, the step runs,
+ * o is copied back, all enqueued on `stream` (nothing is synchronised: wait on the stream before reading o_host).
+ * The cache, lens, workspace and status stay on the device as in mqa_decode_append_step.
+ *
+ *   q_host, k_new_host, v_new_host   HOST pointers, [b, h, k], [b, k], [b, v] bf16; pinned memory makes the copies
+ *                     asynchronous.  When the three are packed back to back with each part padded to a multiple of
+ *                     256 bytes they travel as one copy.
+ *   o_host            HOST pointer, [b, h, v] fp32.  Pinned memory that the device can address (cudaHostAlloc,
+ *                     cudaHostRegister) is written by the step's kernels themselves, with no copy after them;
+ *                     any other host memory is filled by a copy from the staging buffer.  Either way it is
+ *                     complete once the stream has passed this call's work.
+ *   staging           DEVICE scratch of at least mqa_host_staging_bytes(b, h, k, v) bytes (the device copies of the
+ *                     above); owned by the caller, one per call that may be in flight
+ * Other arguments and errors as for mqa_decode_append_step; MQA_ERR_WORKSPACE_TOO_SMALL also for a small staging.
+ */
+int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, const void* v_new_host, float* o_host,
+                                void* K, void* V, int32_t* lens, int advance, void* staging, size_t staging_bytes,
+                                void* workspace, size_t workspace_bytes, int32_t* status,
+                                int b, int h, int m_max, int k, int v, mqa_stream_t stream);
+size_t mqa_host_staging_bytes(int b, int h, int k, int v);
+
+/*
  * mqa_decode_local_step -- one decoding step of multi-query attention restricted to a local neighbourhood
  * (Section 4.1: the current position and the previous window - 1 positions; Section 4.3: the memory tensors
  * padded to the window size).  The cache is a ring of `window` rows per sequence: the new token's key/value row

@@ -28,6 +28,7 @@ EXPORTS = (
     "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
     "mqa_layer_decode_step", "mqa_layer_workspace_bytes", "mqa_decode_local_step",
+    "mqa_decode_append_step_host", "mqa_host_staging_bytes",
 )
 
 _lib = None
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.mqa_layer_decode_step.restype = I
         L.mqa_decode_local_step.argtypes = [vp, vp, vp, vp, vp, vp, I, vp, vp, I, I, I, I, I, vp]
         L.mqa_decode_local_step.restype = I
+        L.mqa_decode_append_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, I, vp, sz, vp, sz, vp, I, I, I, I, I, vp]
+        L.mqa_decode_append_step_host.restype = I
+        L.mqa_host_staging_bytes.argtypes = [I, I, I, I]
+        L.mqa_host_staging_bytes.restype = sz
         L.mqa_layer_workspace_bytes.argtypes = [I, I, I, I, I, I]
         L.mqa_layer_workspace_bytes.restype = sz
         L.mqa_workspace_bytes.argtypes = [I, I, I, I, I]
@@ -106,6 +111,23 @@ def alloc_workspace(b: int, h: int, m_max: int, device, k: int = 128, v: int = 1
     with torch.cuda.device(device):
         n = workspace_bytes(b, h, m_max, k, v)
     return torch.empty(max(n, 16), dtype=torch.uint8, device=device)
+
+
+class _OnDevice:
+    """`with` block that makes a tensor's device current only when it is not already (the common case costs nothing)."""
+    __slots__ = ("ctx",)
+
+    def __init__(self, device):
+        idx = device.index if device.index is not None else torch.cuda.current_device()
+        self.ctx = None if idx == torch.cuda.current_device() else torch.cuda.device(idx)
+
+    def __enter__(self):
+        if self.ctx is not None:
+            self.ctx.__enter__()
+
+    def __exit__(self, *exc):
+        if self.ctx is not None:
+            self.ctx.__exit__(*exc)
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -154,7 +176,7 @@ def kv_cache_append(K, V, k_new, v_new, lens, advance: bool = True, status=None,
     _need(lens, torch.int32, (b,), "lens")
     if status is not None:
         _need(status, torch.int32, (1,), "status")
-    with torch.cuda.device(K.device):
+    with _OnDevice(K.device):
         rc = lib().kv_cache_append(_ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(lens), int(bool(advance)),
                                    _ptr(status), b, kvh, m_max, k, v, _stream(stream))
     _check(rc, "kv_cache_append")
@@ -172,7 +194,7 @@ def _step(name: str, multi_query: bool, q, K, V, lens, o, workspace, status, str
     if status is not None:
         _need(status, torch.int32, (1,), "status")
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (_ptr(workspace), workspace.numel() * workspace.element_size())
-    with torch.cuda.device(q.device):
+    with _OnDevice(q.device):
         if phase == "combine":
             rc = getattr(lib(), name)(_ptr(lens), _ptr(o), ws_ptr, ws_bytes, b, h, m_max, k, v, _stream(stream))
         else:
@@ -227,7 +249,7 @@ def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
     _need(o, torch.float32, (b, h, v), "o")
     if status is not None:
         _need(status, torch.int32, (1,), "status")
-    with torch.cuda.device(q.device):
+    with _OnDevice(q.device):
         rc = lib().mqa_decode_step_noalloc(_ptr(q), _ptr(K), _ptr(V), _ptr(lens), _ptr(o), _ptr(status),
                                            b, h, m_max, k, v, _stream(stream))
     _check(rc, "mqa_decode_step_noalloc")
@@ -237,7 +259,7 @@ def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
 def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None):
     """One whole multi-query decoding step in one call: append ``k_new``/``v_new`` at row ``lens[b]`` of the
     shared cache, then attend over ``lens[b] + 1`` rows; ``lens`` is advanced on the device when ``advance``.
-    For batches the persistent kernel serves (h <= 32) the append runs inside the pass over the cache."""
+    For batches the persistent kernel serves (h <= 64) the whole step is one kernel launch."""
     b, h, k = q.shape
     m_max, v = K.shape[-2], V.shape[-1]
     _need(q, torch.bfloat16, (b, h, k), "q")
@@ -250,7 +272,7 @@ def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, statu
     if status is not None:
         _need(status, torch.int32, (1,), "status")
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (_ptr(workspace), workspace.numel() * workspace.element_size())
-    with torch.cuda.device(q.device):
+    with _OnDevice(q.device):
         rc = lib().mqa_decode_append_step(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(lens),
                                           int(bool(advance)), _ptr(o), ws_ptr, ws_bytes, _ptr(status),
                                           b, h, m_max, k, v, _stream(stream))
@@ -283,7 +305,7 @@ def mqa_layer_decode_step(x, P_q, P_k, P_v, P_o, K, V, lens, y, workspace, statu
     _need(y, torch.float32, (b, d), "y")
     if status is not None:
         _need(status, torch.int32, (1,), "status")
-    with torch.cuda.device(x.device):
+    with _OnDevice(x.device):
         rc = lib().mqa_layer_decode_step(_ptr(x), _ptr(P_q), _ptr(P_k), _ptr(P_v), _ptr(P_o), _ptr(K), _ptr(V), _ptr(lens),
                                          int(bool(advance)), _ptr(y), _ptr(workspace),
                                          workspace.numel() * workspace.element_size(), _ptr(status),
@@ -306,8 +328,65 @@ def mqa_decode_local_step(q, K, V, k_new, v_new, pos, o, status=None, advance: b
     _need(o, torch.float32, (b, h, v), "o")
     if status is not None:
         _need(status, torch.int32, (1,), "status")
-    with torch.cuda.device(q.device):
+    with _OnDevice(q.device):
         rc = lib().mqa_decode_local_step(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(pos), int(bool(advance)),
                                          _ptr(o), _ptr(status), b, h, window, k, v, _stream(stream))
     _check(rc, "mqa_decode_local_step")
     return o
+
+
+def host_staging_bytes(b: int, h: int, k: int = 128, v: int = 128) -> int:
+    return int(lib().mqa_host_staging_bytes(b, h, k, v))
+
+
+def _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream):
+    """Checks the tensors of the host-buffer step and returns the C call's argument tuple (plain integers)."""
+    b, h, k = q_host.shape
+    m_max, v = K.shape[-2], V.shape[-1]
+    for t, dt, shape, name in ((q_host, torch.bfloat16, (b, h, k), "q_host"), (k_new_host, torch.bfloat16, (b, k), "k_new_host"),
+                               (v_new_host, torch.bfloat16, (b, v), "v_new_host"), (o_host, torch.float32, (b, h, v), "o_host")):
+        if t.is_cuda or t.dtype != dt or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError(f"{name}: want a contiguous CPU tensor {dt} {shape}")
+    _need(K, torch.bfloat16, (b, m_max, k), "K")
+    _need(V, torch.bfloat16, (b, m_max, v), "V")
+    _need(lens, torch.int32, (b,), "lens")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    s = torch.cuda.current_stream(K.device) if stream is None else stream
+    return (q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(), o_host.data_ptr(), K.data_ptr(), V.data_ptr(),
+            lens.data_ptr(), int(bool(advance)), staging.data_ptr(), staging.numel() * staging.element_size(),
+            None if workspace is None else workspace.data_ptr(), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+            None if status is None else status.data_ptr(), b, h, m_max, k, v, s.cuda_stream)
+
+
+def mqa_decode_append_step_host(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace=None, status=None,
+                                advance: bool = True, stream=None):
+    """:func:`mqa_decode_append_step` with the per-token inputs and the result in host memory (CPU tensors, pinned for
+    asynchronous copies); ``staging`` is a device uint8 tensor of ``host_staging_bytes(b, h)`` bytes.  Nothing is
+    synchronised: wait on the stream before reading ``o_host``."""
+    args = _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream)
+    with _OnDevice(K.device):
+        rc = lib().mqa_decode_append_step_host(*args)
+    _check(rc, "mqa_decode_append_step_host")
+    return o_host
+
+
+class HostStep:
+    """The host-buffer decoding step bound once to its buffers: a decoding loop refills the same pinned tensors for
+    every token, so the checks and the pointer marshalling are done here and each call is the C call alone.  The
+    tensors are kept alive by this object; the stream is the one current (or given) at construction, and the cache's
+    device must be current when the step is called."""
+    __slots__ = ("fn", "args", "keep", "o_host")
+
+    def __init__(self, q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace=None, status=None,
+                 advance: bool = True, stream=None):
+        self.args = _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream)
+        self.keep = (q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, stream)
+        self.fn = lib().mqa_decode_append_step_host
+        self.o_host = o_host
+
+    def __call__(self):
+        rc = self.fn(*self.args)
+        if rc != MQA_OK:
+            raise MqaError(rc, "mqa_decode_append_step_host")
+        return self.o_host

@@ -648,6 +648,62 @@ int mqa_decode_local_step(const void* q, void* K, void* V, const void* k_new, co
                                advance ? pos : nullptr, true);
 }
 
+size_t mqa_host_staging_bytes(int b, int h, int k, int v) {
+    if (b <= 0 || h <= 0 || k != kHeadDim || v != kHeadDim) return 0;
+    return align256((size_t)b * h * k * 2) + 2 * align256((size_t)b * kHeadDim * 2) + align256((size_t)b * h * v * 4);
+}
+
+int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, const void* v_new_host, float* o_host,
+                                void* K, void* V, int32_t* lens, int advance, void* staging, size_t staging_bytes,
+                                void* workspace, size_t workspace_bytes, int32_t* status, int b, int h, int m_max, int k,
+                                int v, mqa_stream_t stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!q_host || !k_new_host || !v_new_host || !o_host || !staging) return MQA_ERR_INVALID_ARG;
+    if (!dims_ok(b, h, m_max) || k <= 0 || v <= 0 || !aligned16(staging)) return MQA_ERR_INVALID_ARG;
+    if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
+    if (staging_bytes < mqa_host_staging_bytes(b, h, k, v)) return MQA_ERR_WORKSPACE_TOO_SMALL;
+    const size_t q_bytes = (size_t)b * h * k * 2, row_bytes = (size_t)b * kHeadDim * 2, o_bytes = (size_t)b * h * v * 4;
+    char* base = static_cast<char*>(staging);
+    char* q_dev = base;
+    char* k_dev = q_dev + align256(q_bytes);
+    char* v_dev = k_dev + align256(row_bytes);
+    float* o_dev = reinterpret_cast<float*>(v_dev + align256(row_bytes));
+    // the step's inputs: one copy when the caller packed them back to back (256-byte aligned parts), else three
+    const char* qh = static_cast<const char*>(q_host);
+    const bool packed = static_cast<const char*>(k_new_host) == qh + align256(q_bytes) &&
+                        static_cast<const char*>(v_new_host) == qh + align256(q_bytes) + align256(row_bytes);
+    if (packed) {
+        if (cudaMemcpyAsync(q_dev, qh, align256(q_bytes) + align256(row_bytes) + row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+    } else {
+        if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaMemcpyAsync(k_dev, k_new_host, row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaMemcpyAsync(v_dev, v_new_host, row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+    }
+    // the result: where o_host is pinned memory that this device can address, the kernels store o there themselves
+    // (posted writes that overlap the end of the step); otherwise it goes through the staging buffer and a copy
+    float* o_direct = nullptr;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, o_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+        aligned16(attr.devicePointer))
+        o_direct = static_cast<float*>(attr.devicePointer);
+    else
+        cudaGetLastError();
+    const int rc = append_step_impl(q_dev, K, V, k_dev, v_dev, lens, advance, o_direct ? o_direct : o_dev, workspace,
+                                    workspace_bytes, status, b, h, m_max, k, v, stream_, false);
+    if (rc || o_direct) return rc;
+    if (cudaMemcpyAsync(o_host, o_dev, o_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return MQA_ERR_CUDA;
+    }
+    return MQA_OK;
+}
+
 size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || d <= 0 || d % 128 != 0 || k != kHeadDim || v != kHeadDim) return 0;
     return layer_workspace(b, h, d, m_max).total;

@@ -118,3 +118,39 @@ def test_incremental_decoding_with_append_steps():
                 check_close(run_outs[t].cpu().numpy(), ref, f"step {t}")
     for a, c in zip(*outs):
         assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+
+
+def test_host_buffer_entry_point_matches_the_device_one():
+    b, h, m_max = 40, 16, 1500
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=21, device=DEV)
+    lens0 = lens_mix(b, m_max, seed=21)
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    K2, V2 = inp["K"].clone(), inp["V"].clone()
+    lens_a, lens_b = torch.from_numpy(lens0).to(DEV), torch.from_numpy(lens0.copy()).to(DEV)
+    o_dev = torch.empty(b, h, 128, dtype=torch.float32, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_a, o_dev, ws)
+    # host side: once as three separate pinned tensors, once packed back to back (one copy)
+    for packed in (False, True):
+        Kc, Vc, lens_c = K2.clone(), V2.clone(), lens_b.clone()
+        if packed:
+            parts = [inp[n].cpu().contiguous() for n in ("q", "k_new", "v_new")]
+            buf = torch.empty(sum(t.numel() * 2 for t in parts), dtype=torch.uint8).pin_memory()
+            views, at = [], 0
+            for t in parts:
+                n = t.numel() * 2
+                buf[at : at + n].copy_(t.view(torch.uint8).view(-1))
+                views.append(buf[at : at + n].view(torch.bfloat16).view(t.shape))
+                at += n
+            qh, kh, vh = views
+        else:
+            qh, kh, vh = (inp[n].cpu().pin_memory() for n in ("q", "k_new", "v_new"))
+        o_host = torch.full((b, h, 128), float("nan"), dtype=torch.float32).pin_memory()
+        staging = torch.empty(mqa.host_staging_bytes(b, h), dtype=torch.uint8, device=DEV)
+        if packed:
+            mqa.HostStep(qh, kh, vh, o_host, Kc, Vc, lens_c, staging, ws)()      # bound once, then the bare C call
+        else:
+            mqa.mqa_decode_append_step_host(qh, kh, vh, o_host, Kc, Vc, lens_c, staging, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(o_host, o_dev.cpu())
+        assert torch.equal(Kc.view(torch.int16), inp["K"].view(torch.int16)) and torch.equal(lens_c, lens_a)
