@@ -161,8 +161,9 @@ class StepState:
     def step(self, i):
         s = self.sets[i % len(self.sets)]
         if self.variant == "mqa":
+            # a decoding loop: between two steps nothing else writes the cache, lens or the workspace
             self.mqa.mqa_decode_append_step(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, self.o,
-                                            self.ws, self.status, advance=False)
+                                            self.ws, self.status, advance=False, chained=True)
         else:
             self.step_separate(i)
 
@@ -438,6 +439,7 @@ def main():
         "config": {"workload": workload_name(w), "parallelism": f"batch shards x{world}, no collective",
                    "l2": f"rotating {len(st.sets)} cache sets of {st.cache_bytes >> 20} MiB (> L2) between steps",
                    "launch": "K steps replayed as one CUDA graph" if r["graph"] else "K steps launched from the host",
+                   "step": "mqa_decode_append_step, MQA_STEP_CHAINED (a decoding loop: only steps write the cache)",
                    "n_splits": st.n_splits, "chunk_rows": st.chunk_rows},
         "us_per_step": blk["us_per_step"], "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
         "mqa": blk,

@@ -132,14 +132,30 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
  *
  *   q, k_new, v_new   [b, h, k], [b, k], [b, v] bf16
  *   K, V              [b, m_max, k], [b, m_max, v] bf16, read-write (row lens[b] is written)
- *   lens              [b] int32: rows valid BEFORE the call.  advance != 0: lens[b] += 1 on return
- *                     (for sequences that took a row); advance == 0: lens is left as it was, although
- *                     the row has been written and attended over.
+ *   lens              [b] int32: rows valid BEFORE the call.
+ *   advance           bit flags.  MQA_STEP_ADVANCE (1): lens[b] += 1 on return for sequences that took a
+ *                     row; without it lens is left as it was, although the row has been written and
+ *                     attended over.  MQA_STEP_CHAINED (2): a promise by the caller about the work that
+ *                     precedes this call on `stream` -- since the most recent step of this library on this
+ *                     cache (that step excepted), or since the stream was last idle, nothing enqueued on
+ *                     it writes K, V, lens or the workspace.  A decoding loop keeps it: between two steps
+ *                     run projections, a sampler, copies of q.  The first step after something else filled
+ *                     the cache (a prefill kernel) must not carry it.  With the promise the persistent
+ *                     kernel starts fetching the cache, except each prefix's last rows, while the kernel
+ *                     before it is still finishing, and reads q, the new rows and lens only after that
+ *                     kernel has completed.  What it fetches early goes by lens as it reads then; should
+ *                     lens have moved by the time it may rely on it, it fetches again.
+ *                     MQA_STEP_TEST_WRONG_GUESS (4), for tests, with MQA_STEP_CHAINED: the early fetch is
+ *                     deliberately the wrong one, so that this recovery runs; results are unchanged.
+ *                     Any other bit: MQA_ERR_INVALID_ARG.
  *   o, workspace, workspace_bytes, status   as for mqa_decode_step.  A sequence with lens[b] == m_max
  *                     (or negative) takes no new row: APPEND_CACHE_FULL (APPEND_NEGATIVE_LEN) is flagged
  *                     and it attends over its existing rows.
  * Results are those of kv_cache_append followed by mqa_decode_step on the same inputs.
  */
+#define MQA_STEP_ADVANCE 1
+#define MQA_STEP_CHAINED 2
+#define MQA_STEP_TEST_WRONG_GUESS 4
 int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
                            int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status,
                            int b, int h, int m_max, int k, int v, mqa_stream_t stream);

@@ -150,6 +150,14 @@ def _need(t: torch.Tensor, dtype, shape, name: str):
         raise ValueError(f"{name} must be contiguous")
 
 
+STEP_ADVANCE, STEP_CHAINED, STEP_TEST_WRONG_GUESS = 1, 2, 4
+
+
+def _step_flags(advance, chained) -> int:
+    """``chained``: False, True, or "wrong-guess" (the testing form of True)."""
+    return (STEP_ADVANCE if advance else 0) | (STEP_CHAINED if chained else 0) | (STEP_TEST_WRONG_GUESS if chained == "wrong-guess" else 0)
+
+
 def _check(rc: int, where: str):
     if rc != MQA_OK:
         raise MqaError(rc, where)
@@ -256,10 +264,14 @@ def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
     return o
 
 
-def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None):
+def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None,
+                           chained: bool = False):
     """One whole multi-query decoding step in one call: append ``k_new``/``v_new`` at row ``lens[b]`` of the
     shared cache, then attend over ``lens[b] + 1`` rows; ``lens`` is advanced on the device when ``advance``.
-    For batches the persistent kernel serves (h <= 64) the whole step is one kernel launch."""
+    For batches the persistent kernel serves (h <= 64) the whole step is one kernel launch.  ``chained``: the
+    caller's promise that nothing enqueued on the stream since this library's last step on this cache writes
+    the cache, ``lens`` or the workspace (a decoding loop); the kernel then starts on the cache before the
+    kernel ahead of it has finished."""
     b, h, k = q.shape
     m_max, v = K.shape[-2], V.shape[-1]
     _need(q, torch.bfloat16, (b, h, k), "q")
@@ -274,7 +286,7 @@ def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, statu
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (_ptr(workspace), workspace.numel() * workspace.element_size())
     with _OnDevice(q.device):
         rc = lib().mqa_decode_append_step(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(lens),
-                                          int(bool(advance)), _ptr(o), ws_ptr, ws_bytes, _ptr(status),
+                                          _step_flags(advance, chained), _ptr(o), ws_ptr, ws_bytes, _ptr(status),
                                           b, h, m_max, k, v, _stream(stream))
     _check(rc, "mqa_decode_append_step")
     return o
@@ -339,7 +351,7 @@ def host_staging_bytes(b: int, h: int, k: int = 128, v: int = 128) -> int:
     return int(lib().mqa_host_staging_bytes(b, h, k, v))
 
 
-def _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream):
+def _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream, chained=False):
     """Checks the tensors of the host-buffer step and returns the C call's argument tuple (plain integers)."""
     b, h, k = q_host.shape
     m_max, v = K.shape[-2], V.shape[-1]
@@ -354,17 +366,17 @@ def _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging,
         _need(status, torch.int32, (1,), "status")
     s = torch.cuda.current_stream(K.device) if stream is None else stream
     return (q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(), o_host.data_ptr(), K.data_ptr(), V.data_ptr(),
-            lens.data_ptr(), int(bool(advance)), staging.data_ptr(), staging.numel() * staging.element_size(),
+            lens.data_ptr(), _step_flags(advance, chained), staging.data_ptr(), staging.numel() * staging.element_size(),
             None if workspace is None else workspace.data_ptr(), 0 if workspace is None else workspace.numel() * workspace.element_size(),
             None if status is None else status.data_ptr(), b, h, m_max, k, v, s.cuda_stream)
 
 
 def mqa_decode_append_step_host(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace=None, status=None,
-                                advance: bool = True, stream=None):
+                                advance: bool = True, stream=None, chained: bool = False):
     """:func:`mqa_decode_append_step` with the per-token inputs and the result in host memory (CPU tensors, pinned for
     asynchronous copies); ``staging`` is a device uint8 tensor of ``host_staging_bytes(b, h)`` bytes.  Nothing is
     synchronised: wait on the stream before reading ``o_host``."""
-    args = _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream)
+    args = _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream, chained)
     with _OnDevice(K.device):
         rc = lib().mqa_decode_append_step_host(*args)
     _check(rc, "mqa_decode_append_step_host")
@@ -379,8 +391,9 @@ class HostStep:
     __slots__ = ("fn", "args", "keep", "o_host")
 
     def __init__(self, q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace=None, status=None,
-                 advance: bool = True, stream=None):
-        self.args = _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream)
+                 advance: bool = True, stream=None, chained: bool = False):
+        self.args = _host_step_args(q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, advance, stream,
+                                    chained)
         self.keep = (q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, stream)
         self.fn = lib().mqa_decode_append_step_host
         self.o_host = o_host

@@ -292,16 +292,17 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
-std::atomic<int> g_umma_opt_in[kMaxDevices][6];
+constexpr size_t kL2KeepBytes = 64u << 20;   // K and V together: half of the 126 MB L2
+std::atomic<int> g_umma_opt_in[kMaxDevices][9];
 
-template <int HP, bool FUSED>
+template <int HP, bool FUSED, bool GUESS = false>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
                 const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
-                bool late_wait = false) {
+                int early = 0) {
     using Cfg = UmmaCfg<HP>;
-    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED>;
-    constexpr int kSlot = (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 2 + (FUSED ? 1 : 0);
+    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS>;
+    constexpr int kSlot = (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
@@ -325,9 +326,11 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
         !encode_cache_map(&map_q, q, (long long)b * h, HP))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
+    // a cache that cannot stay in L2 from one step to the next is streamed through it with the evict-first policy
+    const int read_once = (size_t)b * m_max * 2 * kRowBytes > kL2KeepBytes ? 1 : 0;
     launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
                      map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa,
-                     merge ? w.ctrl : nullptr, lens_advance, late_wait ? 1 : 0);
+                     merge ? w.ctrl : nullptr, lens_advance, early, read_once);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -335,12 +338,19 @@ template <bool FUSED>
 int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                     void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
                     const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
-                    bool late_wait = false) {
-    if (h <= 16)
-        return launch_umma<16, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, late_wait);
-    if (h <= 32)
-        return launch_umma<32, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, late_wait);
-    return launch_umma<64, FUSED>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, late_wait);
+                    int early = 0) {
+#define MQA_UMMA_ARGS p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, early
+    if constexpr (FUSED) {
+        if (early >= 2) {                                   // the kernels that carry the code for copies started on a guess
+            if (h <= 16) return launch_umma<16, true, true>(MQA_UMMA_ARGS);
+            if (h <= 32) return launch_umma<32, true, true>(MQA_UMMA_ARGS);
+            return launch_umma<64, true, true>(MQA_UMMA_ARGS);
+        }
+    }
+    if (h <= 16) return launch_umma<16, FUSED>(MQA_UMMA_ARGS);
+    if (h <= 32) return launch_umma<32, FUSED>(MQA_UMMA_ARGS);
+    return launch_umma<64, FUSED>(MQA_UMMA_ARGS);
+#undef MQA_UMMA_ARGS
 }
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
@@ -579,11 +589,18 @@ int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace
                        static_cast<cudaStream_t>(stream));
 }
 
-// after_projection: the kernel before this step in the stream is the layer step's input projection (see late_wait in
-// mqa_decode_stream_umma_kernel)
+// early: what the persistent kernel may do before it waits for the kernel before it (see early in
+// mqa_decode_stream_umma_kernel): kEarlyAfterProjection inside the layer step, kEarlyChained when the caller set
+// MQA_STEP_CHAINED.  flags: MQA_STEP_ADVANCE | MQA_STEP_CHAINED.
+constexpr int kEarlyNone = 0, kEarlyAfterProjection = 1, kEarlyChained = 2, kEarlyChainedWrongGuess = 3;
 static int append_step_impl(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
-                            int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
+                            int flags, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
                             int h, int m_max, int k, int v, mqa_stream_t stream_, bool after_projection) {
+    if (flags & ~(MQA_STEP_ADVANCE | MQA_STEP_CHAINED | MQA_STEP_TEST_WRONG_GUESS)) return MQA_ERR_INVALID_ARG;
+    const int advance = flags & MQA_STEP_ADVANCE;
+    const int early = after_projection ? kEarlyAfterProjection
+                      : !(flags & MQA_STEP_CHAINED) ? kEarlyNone
+                      : (flags & MQA_STEP_TEST_WRONG_GUESS) ? kEarlyChainedWrongGuess : kEarlyChained;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
@@ -596,9 +613,9 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
         // one launch: append inside the pass, pieces merged by the last CTA to deliver one, lens advanced at the end
         if (p.merge_in_kernel)
             return launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, true, k_new, v_new,
-                                         advance ? lens : nullptr, after_projection);
+                                         advance ? lens : nullptr, early);
         rc = launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, false, k_new, v_new, nullptr,
-                                   after_projection);
+                                   early);
         if (rc) return rc;
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr);
     }
@@ -736,8 +753,8 @@ int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const
         default: rc = launch_projections_in<128>(x, P_q, P_k, P_v, q, k_new, v_new, status, b, h, d, stream); break;
     }
     if (rc) return rc;
-    rc = append_step_impl(q, K, V, k_new, v_new, lens, advance, o, base + w.step, w.total - w.step, status, b, h, m_max, k, v,
-                          stream_, true);
+    rc = append_step_impl(q, K, V, k_new, v_new, lens, advance ? MQA_STEP_ADVANCE : 0, o, base + w.step, w.total - w.step, status,
+                          b, h, m_max, k, v, stream_, true);
     if (rc) return rc;
     switch (nb) {
         case 16: return launch_projection_out<16>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);

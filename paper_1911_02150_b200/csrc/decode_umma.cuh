@@ -66,7 +66,7 @@ struct UmmaCfg {
     // per-quarter maxima and sums [4][HP] each, reference maxima, factors of the last move, 1/sum of two segments
     static constexpr int kRedBytes = (2 * 4 + 4) * HP * 4;
     static constexpr int kPlanBytes = (2 * kStreamMaxSeqs + 1) * 4 + 12;   // line positions + rows per sequence
-    static constexpr int kBarriers = 2 * kKSlots + 2 * kVSlots + 14;
+    static constexpr int kBarriers = 2 * kKSlots + 2 * kVSlots + 15;
     static constexpr int kSmemBytes = (kKSlots + kVSlots) * kUmmaSlotBytes + kQBufs * kQBytes + kPTiles * kPBytes + kRedBytes +
                                       kPlanBytes + kBarriers * 8 + 1024 /* alignment slack */;
     static_assert(kSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
@@ -306,8 +306,9 @@ __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__
     }
 }
 
-// HP = head rows of the Q tile (h rounded up to 16, 32 or 64).
-template <int HP, bool FUSED>
+// HP = head rows of the Q tile (h rounded up to 16, 32 or 64).  GUESS: built with the code that starts copies on a
+// guess before the wait (GUESS && early >= 2 below); kernels without it take early 0 or 1 only.
+template <int HP, bool FUSED, bool GUESS = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                               const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
@@ -315,8 +316,10 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               const int32_t* __restrict__ lens, float* __restrict__ o, int2* __restrict__ seq_span,
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
                               int b, int h, int m_max, unsigned long long magic, const FusedArgs fa,
-                              unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int late_wait) {
+                              unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int early_arg,
+                              int read_once) {
     using Cfg = UmmaCfg<HP>;
+    const int early = GUESS ? early_arg : (early_arg == 1 ? 1 : 0);
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
     const bool appending = FUSED && fa.k_new != nullptr;
@@ -343,15 +346,16 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     const uint32_t q_full = v_empty + NV * 8, q_empty = q_full + 16;
     const uint32_t s_ready = q_empty + 16, s_free = s_ready + 16;
     const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;   // o_free: one per O^T buffer
+    const uint32_t go = o_free + 16;                        // the share's first segment is settled (see early below)
     __shared__ int timed_out, issued, plan_sm[4], merge_sm[8];   // merge_sm: count, then (sequence, first CTA, last CTA) x 2
     __shared__ unsigned long long epoch_sm[2];              // this launch's epoch; the epoch word as found
     __shared__ uint32_t tmem_base_slot;
 
+    // set up by the thread that issues the copies: it may start some before the first CTA-wide barrier, and
+    // program order is what puts the initialisation before them; every other thread first passes that barrier
     if (warp == kUmmaProducerWarp && lane == 0) {
         prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); prefetch_tensormap(&map_k_sub);
         prefetch_tensormap(&map_v_sub); prefetch_tensormap(&map_q);
-    }
-    if (threadIdx.x == 0) {
         timed_out = 0;
         issued = 0;
         merge_sm[0] = 0;
@@ -363,6 +367,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             mbar_init(p_ready + s * 8, kUmmaSoftmaxWarps); mbar_init(pv_done + s * 8, 1);
             mbar_init(o_free + s * 8, kUmmaSoftmaxWarps);
         }
+        mbar_init(go, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -396,6 +401,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         tma_load_2d(q_s + qi * Cfg::kQBytes, &map_q, 0, s * h, q_full + qi * 8);
         tma_load_2d(q_s + qi * Cfg::kQBytes + Cfg::kQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
     };
+    const uint64_t stream_policy = l2_stream_policy(read_once != 0);
     auto issue_stage = [&](int s, int u, int hi, int j) {
         const int nsub = min(kSubs, hi - u);
         const int row_first = u * kTileRows;
@@ -410,23 +416,99 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes;
             mbar_expect_tx(full, nsub * 2 * kBoxBytes);
             if (nsub == kSubs) {
-                tma_load_2d(dst, kv ? &map_v : &map_k, 0, y, full);
-                tma_load_2d(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full);
+                tma_load_2d_hint(dst, kv ? &map_v : &map_k, 0, y, full, stream_policy);
+                tma_load_2d_hint(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full, stream_policy);
             } else {
                 for (int i = 0; i < nsub; ++i) {
                     const uint32_t d = dst + i * kBoxBytes;
-                    tma_load_2d(d, kv ? &map_v_sub : &map_k_sub, 0, y + i * kTileRows, full);
-                    tma_load_2d(d + kUmmaHalfBytes, kv ? &map_v_sub : &map_k_sub, kBoxCols, y + i * kTileRows, full);
+                    tma_load_2d_hint(d, kv ? &map_v_sub : &map_k_sub, 0, y + i * kTileRows, full, stream_policy);
+                    tma_load_2d_hint(d + kUmmaHalfBytes, kv ? &map_v_sub : &map_k_sub, kBoxCols, y + i * kTileRows, full, stream_policy);
                 }
             }
             issued = 2 * j + kv + 1;                        // copies started: K of stage j, then V of stage j
         }
     };
 
-    // late_wait: the kernel before this one writes nothing but q and the new key/value row (the input projection
-    // of the layer step) and, like every kernel here, lets this one start only after its own wait -- so everything
-    // older is complete, and only the producer warp has to wait, before it touches q or the new row.
-    if (!late_wait) {
+    // ---- what may start before the wait on the kernel before this one (early):
+    // 0  nothing.
+    // 1  that kernel writes nothing but q and the new key/value row (the input projection of the layer step) and,
+    //    like every kernel here, lets this one start only after its own wait -- so everything older is complete,
+    //    lens included, and only the producer warp has to wait, before it touches q or the new row.
+    // 2  that kernel may be a step of this library on the same cache (a decoding loop): it writes one row per
+    //    sequence, at or just below the end of the prefix, and moves lens on by one.  The producer warp works out
+    //    its first segment from lens as it reads now and starts the copies of the stages that lie wholly below the
+    //    last two rows of that prefix; right after the wait it asks for that sequence's q, then works the segment
+    //    out again, and if the first stages are no longer the same (lens moved under it and a tile boundary was
+    //    crossed) the copies are left to land and everything is started again.  The warp that issues S^T = K Q^T,
+    //    whose results everything else waits for, starts only when told that the segment is settled (go).
+    // 3  as 2 with a guess that is wrong on purpose, so that tests reach the recovery.
+    int pre_issued = 0;                                     // stages whose copies were started here
+    if (warp == kUmmaProducerWarp) {
+        // One loop body serves both sides of the wait (with a guess it runs twice, and the second time its
+        // instructions are already on the SM): work out the share's first segment, start what may be started.
+        Segment g0 = {};
+        int r0 = 0;
+        bool have = false, q_started = false;
+        const int passes = early >= 1 ? 2 : 1;
+        for (int pass = 0; pass < passes; ++pass) {
+            const bool before = pass + 1 < passes;          // this pass runs ahead of the wait
+            if (!before) {
+                grid_dependency_wait();                     // q, the new row, lens: all there now
+                grid_launch_dependents();
+                if (GUESS && early >= 2 && have) {                   // q of the guessed sequence, while the guess is checked
+                    if (lane == 0) issue_q(g0.s, 0);
+                    q_started = true;
+                }
+            }
+            if (before || early != 1) {                     // (early == 1: lens cannot have moved)
+                Segment g = {};
+                int r = 0;
+                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r);
+                if (GUESS && before && early == 3) g.lo += kSubs;    // for tests: a guess that is one stage off
+                if (!before && GUESS && early >= 2) {
+                    if (have && !(found && g.s == g0.s && g.lo == g0.lo && g.lo + pre_issued * kSubs <= g.hi)) {
+                        // what was started on the guess is not how this share begins: each of those barriers has
+                        // completed one phase when its copy has landed; one more arrival completes a second,
+                        // empty one, and the slot is as new (no consumer has looked: the first of them waits for go)
+                        if (lane == 0) {
+                            p_ok = p_ok && mbar_wait(q_full, 0);
+                            if (p_ok) mbar_arrive(q_full);
+                            for (int i = 0; i < pre_issued; ++i) {
+                                p_ok = p_ok && mbar_wait(k_full + i * 8, 0) && mbar_wait(v_full + i * 8, 0);
+                                if (p_ok) { mbar_arrive(k_full + i * 8); mbar_arrive(v_full + i * 8); }
+                            }
+                        }
+                        p_ok = __shfl_sync(0xffffffffu, (int)p_ok, 0) != 0;
+                        pre_issued = 0;
+                        q_started = false;
+                    }
+                    if (lane == 0) mbar_arrive(go);
+                }
+                have = found;
+                g0 = g;
+                r0 = r;
+            }
+            if (have) {
+                const int L = r0 & (kAppendBit - 1);
+                const int new_row = (r0 & kAppendBit) ? L - 1 : -1;          // row this step appends
+                // rows that may be fetched now lie below stop_row: ahead of the wait not this step's new row
+                // (early == 1) or, on a guess, the prefix's last two rows, and then whole stages only
+                const int stop_row = !before ? 0x7fffffff : early == 1 ? (new_row >= 0 ? new_row : 0x7fffffff) : L - 2;
+                const int n_pre = min((g0.hi - g0.lo + kSubs - 1) / kSubs, NK < NV ? NK : NV);   // what the rings hold without a wait
+                const int u0 = g0.lo + pre_issued * kSubs;
+                if (!before && appending && new_row >= u0 * kTileRows && new_row < min(g0.hi, g0.lo + n_pre * kSubs) * kTileRows)
+                    row_store(g0.s, new_row, row_load(g0.s));   // the new row lies in the stages started now
+                if (lane == 0) {
+                    if (!before && !q_started) issue_q(g0.s, 0);
+                    for (int u = u0; pre_issued < n_pre && (u + kSubs) * kTileRows <= stop_row &&
+                                     !(before && GUESS && early >= 2 && u + kSubs > g0.hi);
+                         u += kSubs, ++pre_issued)
+                        issue_stage(g0.s, u, g0.hi, pre_issued);
+                }
+                pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
+            }
+        }
+    } else if (early != 1) {
         grid_dependency_wait();      // lens and the newest cache row may come from the kernel before
         grid_launch_dependents();
     }
@@ -436,36 +518,6 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         if (E == 0) E = 1;
         epoch_sm[0] = E;
         epoch_sm[1] = was;
-    }
-
-    // the producer warp starts its first stages (at most what the rings hold without a wait) before the tables exist
-    int pre_issued = 0;
-    if (warp == kUmmaProducerWarp) {
-        Segment g0;
-        int r0 = 0;
-        const bool fast = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g0, &r0);
-        const int new_row = (fast && (r0 & kAppendBit)) ? (r0 & (kAppendBit - 1)) - 1 : -1;   // row this step appends
-        const int n_pre = fast ? min((g0.hi - g0.lo + kSubs - 1) / kSubs, NK < NV ? NK : NV) : 0;
-        if (late_wait) {
-            // stages that do not hold the new row start while the kernel before this one is still running
-            if (lane == 0)
-                for (int u = g0.lo; pre_issued < n_pre && !(appending && new_row >= u * kTileRows && new_row < (u + kSubs) * kTileRows);
-                     u += kSubs, ++pre_issued)
-                    issue_stage(g0.s, u, g0.hi, pre_issued);
-            pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
-            grid_dependency_wait();      // q and the new row are there now
-            grid_launch_dependents();
-        }
-        if (fast) {
-            const int u0 = g0.lo + pre_issued * kSubs;
-            if (appending && new_row >= u0 * kTileRows && new_row < min(g0.hi, g0.lo + n_pre * kSubs) * kTileRows)
-                row_store(g0.s, new_row, row_load(g0.s));   // the new row lies in the stages started here
-            if (lane == 0) {
-                issue_q(g0.s, 0);
-                for (int u = u0; pre_issued < n_pre; u += kSubs, ++pre_issued) issue_stage(g0.s, u, g0.hi, pre_issued);
-            }
-            pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
-        }
     }
 
     tc_fence_before();
@@ -527,7 +579,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // =============================================================== issuer of S^T = K Q^T
         if (lane == 0 && t_begin < t_end) {
             constexpr uint32_t kIdescS = umma_idesc(128, HP, false, false);
-            bool ok = true;
+            bool ok = !(GUESS && early >= 2) || mbar_wait(go, 0);
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
@@ -568,8 +620,10 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 const int parts = L >= kSingleRoundingMinRows ? 1 : 2;   // P hi only, or hi then lo (as the softmax warps wrote it)
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
                     const int pb = j & 1, slot = j % NV;
-                    if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
+                    // the weights first: they exist only once q has arrived, and before that a slot's barrier may
+                    // still be on its way back from copies started on a guess (see early above)
                     if (ok) ok = mbar_wait(p_ready + pb * 8, (j >> 1) & 1);
+                    if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
                     // segments alternate between the two O^T buffers; the segment before the last has read this one out
                     if (ok && u == g.lo && seg >= 2) ok = mbar_wait(o_free + (seg & 1) * 8, ((seg >> 1) - 1) & 1);
                     tc_fence_after();

@@ -124,3 +124,100 @@ def test_reference_maximum_moves_late_in_a_long_cache():
     star = torch.full((b,), 3001, device=DEV); star[5] = 40
     want = inp["V"][torch.arange(b, device=DEV), star].float()[:, None, :].expand(b, h, 128)
     assert torch.equal(o, want.contiguous())                  # weight exactly 1 on that row, 0 elsewhere
+
+
+@pytest.mark.parametrize("chained", [True, "wrong-guess"])
+@pytest.mark.parametrize("b,h,m_max", [(40, 16, 2048), (32, 32, 4096), (33, 64, 2100), (256, 8, 1100)])
+def test_chained_steps_in_a_loop_match_unchained_ones_and_the_oracle(b, h, m_max, chained):
+    """A decoding loop whose steps carry the promise that lets the kernel fetch the cache before the step ahead of it
+    has finished.  lens moves under every early guess (each step advances it), prefixes cross tile and stage
+    boundaries on the way, one sequence fills up; with "wrong-guess" every early fetch is the wrong one and is redone."""
+    steps = 70
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=31, device=DEV)
+    r = np.random.default_rng(31)
+    lens0 = r.integers(m_max // 2, m_max - steps - 1, size=b).astype(np.int32)
+    lens0[0] = 4 * 128 - 3                                    # crosses a stage boundary after three steps
+    lens0[1] = m_max - 5                                      # fills up
+    lens0[2] = 1                                              # a short prefix: nothing to fetch early
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    gen = torch.Generator(device=DEV).manual_seed(32)
+    qs = [wl.bf16_normal((b, h, 128), 128 ** -0.5, gen, DEV) for _ in range(steps)]
+    ks = [wl.bf16_normal((b, 128), 1.0, gen, DEV) for _ in range(steps)]
+    vs = [wl.bf16_normal((b, 128), 1.0, gen, DEV) for _ in range(steps)]
+    results = {}
+    for mode in (False, chained):
+        K, V = inp["K"].clone(), inp["V"].clone()
+        lens_t = torch.from_numpy(lens0.copy()).to(DEV)
+        ws = mqa.alloc_workspace(b, h, m_max, DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        outs = [torch.empty(b, h, 128, dtype=torch.float32, device=DEV) for _ in range(steps)]
+        torch.cuda.synchronize()
+        for t in range(steps):                                # back to back: each kernel starts under the one before
+            mqa.mqa_decode_append_step(qs[t], K, V, ks[t], vs[t], lens_t, outs[t], ws, status, advance=True,
+                                       chained=mode if t > 0 else False)    # the first step follows the set-up copies
+        torch.cuda.synchronize()
+        results[mode] = (K, V, lens_t, outs, int(status.item()))
+    Ka, Va, la, oa, sa = results[False]
+    Kc, Vc, lc, oc, sc = results[chained]
+    assert sa == sc and torch.equal(la, lc)
+    assert torch.equal(Ka.view(torch.int16), Kc.view(torch.int16)) and torch.equal(Va.view(torch.int16), Vc.view(torch.int16))
+    for t in range(steps):
+        assert torch.equal(oa[t].view(torch.int32), oc[t].view(torch.int32)), f"step {t}"
+    # and the loop itself against the oracle, at a few steps
+    Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
+    for t in range(steps):
+        oracle.kv_cache_append(Kh, Vh, wl.bits(ks[t]), wl.bits(vs[t]), lens_h, True)
+        if t in (0, 3, 4, steps - 1):
+            ref = oracle.mqa_decode_step(wl.bits(qs[t]), Kh, Vh, lens_h)
+            check_close(oc[t].cpu().numpy(), ref, f"chained step {t}")
+    assert np.array_equal(lc.cpu().numpy(), lens_h)
+    assert np.array_equal(wl.bits(Kc), Kh) and np.array_equal(wl.bits(Vc), Vh)
+
+
+def test_chained_steps_replayed_from_a_graph():
+    b, h, m_max, per_graph, replays = 32, 32, 4096, 4, 3
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=41, device=DEV)
+    lens0 = np.full(b, 3 * 128 - 5, np.int32)                 # every sequence crosses a stage boundary together
+    lens0[5] = m_max - 3
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    o = torch.zeros(b, h, 128, dtype=torch.float32, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    step = lambda chained: mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws,
+                                                      status, advance=True, chained=chained)
+    side = torch.cuda.Stream(device=DEV)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(False)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(per_graph):
+            step(True)                                        # in a replay the step before is the previous replay's last
+    for _ in range(replays):
+        graph.replay()
+    torch.cuda.synchronize()
+    k_new, v_new = wl.bits(inp["k_new"]), wl.bits(inp["v_new"])
+    for _ in range(1 + per_graph * replays):
+        oracle.kv_cache_append(Kh, Vh, k_new, v_new, lens_h, True)
+    assert np.array_equal(lens_t.cpu().numpy(), lens_h)
+    assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)
+    check_close(o.cpu().numpy(), oracle.mqa_decode_step(wl.bits(inp["q"]), Kh, Vh, lens_h), "last chained step of the replayed graph")
+
+
+def test_unknown_step_flags_are_refused():
+    b, h, m_max = 8, 8, 256
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=1, device=DEV)
+    lens_t = torch.full((b,), 7, dtype=torch.int32, device=DEV)
+    o = torch.zeros(b, h, 128, dtype=torch.float32, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    from paper_1911_02150_b200 import binding
+    rc = binding.lib().mqa_decode_append_step(inp["q"].data_ptr(), inp["K"].data_ptr(), inp["V"].data_ptr(), inp["k_new"].data_ptr(),
+                                              inp["v_new"].data_ptr(), lens_t.data_ptr(), 8, o.data_ptr(), ws.data_ptr(), ws.numel(),
+                                              None, b, h, m_max, 128, 128, None)
+    assert rc == binding.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert int(lens_t[0]) == 7 and float(o.abs().max()) == 0.0
