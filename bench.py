@@ -306,6 +306,49 @@ def layer_block(mqa, w, device, seed, steps, d_model=1024):
             "launches_per_step": 3 + mqa.append_step_launches(b, h, m), "cache_sets": nset}
 
 
+def paper_loop_block(mqa, device, seed):
+    """The paper's timed decoding shape (Section 4.1: 128 sequences, h = 8, 128 target positions): 128 successive steps,
+    each appending one row and attending over the prefix, the cache growing from 1 to 128 rows; the loop is one CUDA
+    graph, lens lives on the device and is advanced by the steps.  Multi-query: one mqa_decode_append_step per step;
+    multi-head (per-head cache): kv_cache_append + mha_decode_step."""
+    w = wl.WORKLOADS["paper_incremental"]
+    b, h, m, steps = w.b, w.h, w.m_max, w.steps
+    out = {"b": b, "h": h, "steps": steps, "cache_rows": f"1..{m}"}
+    for variant in ("mqa", "mha"):
+        inp = wl.make_inputs(b, h, m, variant, seed=seed, device=device)
+        lens0 = torch.zeros(b, dtype=torch.int32, device=device)
+        lens = lens0.clone()
+        o = torch.empty(b, h, 128, dtype=torch.float32, device=device)
+        ws = mqa.alloc_workspace(b, h, m, device)
+        status = torch.zeros(1, dtype=torch.int32, device=device)
+        if variant == "mqa":
+            step = lambda i: mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens, o, ws,
+                                                        status, advance=True, chained=i > 0)
+            launches = mqa.append_step_launches(b, h, m)
+        else:
+            def step(i):
+                mqa.kv_cache_append(inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens, advance=True, status=status)
+                mqa.mha_decode_step(inp["q"], inp["K"], inp["V"], lens, o, ws, status)
+            launches = 2 + (1 if mqa.plan_splits(False, b, h, m)[0] > 1 else 0)
+        for i in range(3):
+            step(i)
+        lens.copy_(lens0)
+        torch.cuda.synchronize(device)
+        g = capture_graph(step, steps)
+        times = []
+        for _ in range(20):
+            lens.copy_(lens0)                               # every replay decodes from an empty cache
+            times.append(time_region(lambda _i: g.replay(), 1, device))
+        assert int(lens[0]) == steps
+        secs = statistics.median(times)
+        total_bytes = sum(wl.algorithmic_bytes(b * t, b, h, 1 if variant == "mqa" else h) for t in range(1, steps + 1))
+        out[variant] = {"us_per_step": secs / steps * 1e6, "us_per_loop": secs * 1e6, "gbs": total_bytes / secs / 1e9,
+                        "us_per_token": secs / steps / b * 1e6, "launches_per_step": launches, "status": int(status.item())}
+        del inp
+    out["mqa_speedup_over_mha"] = out["mha"]["us_per_step"] / out["mqa"]["us_per_step"]
+    return out
+
+
 def cpu_baseline(w, seed, budget_s=20.0):
     """The oracle, as it stands, on the host cores: one multi-query step of the same workload on
     as many whole sequences as fit the time budget."""
@@ -472,6 +515,7 @@ def main():
         torch.cuda.empty_cache()
     if not args.no_layer:
         out["layer_step"] = layer_block(mqa, w, device, seed, max(3, min(args.steps, 20)))
+        out["paper_incremental"] = paper_loop_block(mqa, device, seed)
         out["layer_step"]["projections_us"] = out["layer_step"]["us_per_step"] - blk["us_per_step"]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, seed)

@@ -332,7 +332,7 @@ __device__ __forceinline__ void store_state(const WarpState& st, float* __restri
 // =============================================================================================
 // Fixed-split kernel: one CTA per (sequence, split of chunk_rows rows).
 // =============================================================================================
-template <int M_TILES>
+template <int M_TILES, bool EARLY = false>
 __global__ void __launch_bounds__(MmaCfg<M_TILES>::kThreads, MmaCfg<M_TILES>::kMinBlocks)
 mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
@@ -353,8 +353,9 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const uint32_t full_s = smem_addr(bars), empty_s = full_s + kStages * 8;
     __shared__ int timed_out, issued;   // a wait ran out; tiles whose copies were started
 
-    if (warp == Cfg::kConsumerWarps && lane == 0) { prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); }
-    if (threadIdx.x == 0) {
+    // set up by the thread that issues the copies (it may issue some before the first CTA-wide barrier)
+    if (warp == Cfg::kConsumerWarps && lane == 0) {
+        prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
         timed_out = 0;
         issued = 0;
         for (int s = 0; s < kStages; ++s) {
@@ -363,6 +364,32 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    const int row_base = seq * m_max + split * chunk_rows; // row coordinate in the [b*m_max, 128] view
+    auto issue_tile = [&](int i) {
+        const int s = i % kStages;
+        const uint32_t bar = full_s + s * 8;
+        const uint32_t dst = stages_s + s * kStageBytes;
+        mbar_expect_tx(bar, kStageBytes);
+        const int y = row_base + i * kTileRows;
+        tma_load_2d(dst, &map_k, 0, y, bar);
+        tma_load_2d(dst + kBoxBytes, &map_k, kBoxCols, y, bar);
+        tma_load_2d(dst + 2 * kBoxBytes, &map_v, 0, y, bar);
+        tma_load_2d(dst + 3 * kBoxBytes, &map_v, kBoxCols, y, bar);
+        issued = i + 1;
+    };
+    // EARLY (the caller's promise that only this library's steps have written the cache and lens since its last step
+    // on them): one CTA owns the sequence, its tiles are tiles 0, 1, ... whatever lens says, so those that lie wholly
+    // below the prefix's last two rows -- by lens as it reads now, which the step ahead may be about to advance -- are
+    // fetched while that step is still finishing.  Only their number is a guess: should fewer tiles count in the end,
+    // the surplus is left to land and ignored.
+    int pre = 0;
+    if (EARLY && n_splits == 1 && !ring && warp == Cfg::kConsumerWarps && lane == 0) {
+        const int raw_guess = __ldcg(lens + seq);
+        const int rows_guess = min(max(raw_guess, 0) + (fa.k_new != nullptr ? 1 : 0), m_max);
+        pre = min((rows_guess - 2) / kTileRows, kStages);
+        if (pre < 0) pre = 0;
+        for (int i = 0; i < pre; ++i) issue_tile(i);
     }
     // everything above overlaps the tail of the kernel before this one
     grid_dependency_wait();          // lens and the newest cache row may come from the kernel before
@@ -390,6 +417,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     if (r0 >= L) {                                         // nothing valid in this split (uniform)
         if (n_splits == 1)                                 // L == 0: the empty prefix gives zeros
             for (int i = threadIdx.x; i < h * kHeadDim; i += Cfg::kThreads) o[(size_t)seq * h * kHeadDim + i] = 0.f;
+        for (int i = 0; i < pre; ++i) mbar_wait(full_s + i * 8, 0);   // copies started on a guess land before the CTA leaves
         return;
     }
     const int n_tiles = (r1 - r0 + kTileRows - 1) / kTileRows;
@@ -403,22 +431,14 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     if (warp == Cfg::kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
         if (lane == 0) {
-            const int row_base = seq * m_max + r0;         // row coordinate in the [b*m_max, 128] view
             bool ok = true;
-            for (int i = 0; i < n_tiles && ok; ++i) {
+            for (int i = pre; i < n_tiles && ok; ++i) {
                 const int s = i % kStages;
                 if (i >= kStages) ok = mbar_wait(empty_s + s * 8, ((i / kStages) - 1) & 1);
                 if (!ok) break;
-                const uint32_t bar = full_s + s * 8;
-                const uint32_t dst = stages_s + s * kStageBytes;
-                mbar_expect_tx(bar, kStageBytes);
-                const int y = row_base + i * kTileRows;
-                tma_load_2d(dst, &map_k, 0, y, bar);
-                tma_load_2d(dst + kBoxBytes, &map_k, kBoxCols, y, bar);
-                tma_load_2d(dst + 2 * kBoxBytes, &map_v, 0, y, bar);
-                tma_load_2d(dst + 3 * kBoxBytes, &map_v, kBoxCols, y, bar);
-                issued = i + 1;
+                issue_tile(i);
             }
+            for (int i = n_tiles; i < pre; ++i) ok = mbar_wait(full_s + i * 8, 0) && ok;   // a surplus of the guess
             if (!ok) atomicExch(&timed_out, 1);
         }
     } else {

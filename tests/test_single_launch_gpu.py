@@ -221,3 +221,47 @@ def test_unknown_step_flags_are_refused():
     assert rc == binding.ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert int(lens_t[0]) == 7 and float(o.abs().max()) == 0.0
+
+
+def test_chained_steps_of_the_paper_shaped_loop():
+    """128 sequences, 8 heads, a cache growing from nothing to 128 rows (Section 4.1), every step after the first
+    carrying the promise: the one-CTA-per-sequence kernel fetches its lower tiles ahead of the wait."""
+    b, h, m_max, steps = 128, 8, 128, 128
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=51, device=DEV)
+    gen = torch.Generator(device=DEV).manual_seed(52)
+    qs = [wl.bf16_normal((b, h, 128), 128 ** -0.5, gen, DEV) for _ in range(steps)]
+    ks = [wl.bf16_normal((b, 128), 1.0, gen, DEV) for _ in range(steps)]
+    vs = [wl.bf16_normal((b, 128), 1.0, gen, DEV) for _ in range(steps)]
+    nan = torch.tensor(wl.NAN_BITS, dtype=torch.int16, device=DEV)
+    runs = {}
+    for chained in (False, True):
+        K, V = torch.empty_like(inp["K"]), torch.empty_like(inp["V"])
+        K.view(torch.int16).fill_(nan); V.view(torch.int16).fill_(nan)
+        lens_t = torch.zeros(b, dtype=torch.int32, device=DEV)
+        lens_t[3] = 100                                       # one sequence starts with a prefix (of NaN rows it never reads: replaced below)
+        K[3, :100] = wl.bf16_normal((100, 128), 1.0, gen, DEV) if not runs else runs[False][3][3, :100]
+        V[3, :100] = wl.bf16_normal((100, 128), 1.0, gen, DEV) if not runs else runs[False][4][3, :100]
+        K0, V0 = K.clone(), V.clone()
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        ws = mqa.alloc_workspace(b, h, m_max, DEV)
+        outs = [torch.empty(b, h, 128, dtype=torch.float32, device=DEV) for _ in range(steps)]
+        torch.cuda.synchronize()
+        for t in range(steps):
+            mqa.mqa_decode_append_step(qs[t], K, V, ks[t], vs[t], lens_t, outs[t], ws, status, advance=True,
+                                       chained=chained and t > 0)
+        torch.cuda.synchronize()
+        runs[chained] = (outs, K, lens_t, K0, V0, V, int(status.item()))
+    for t in range(steps):
+        assert torch.equal(runs[False][0][t].view(torch.int32), runs[True][0][t].view(torch.int32)), f"step {t}"
+    assert torch.equal(runs[False][1].view(torch.int16), runs[True][1].view(torch.int16))
+    assert torch.equal(runs[False][2], runs[True][2]) and runs[False][6] == runs[True][6]
+    # the chained loop against the oracle at a few steps (sequence 3 fills up after 28 steps and takes no more rows)
+    Kh, Vh = wl.bits(runs[True][3]), wl.bits(runs[True][4])
+    lens_h = np.zeros(b, np.int32); lens_h[3] = 100
+    for t in range(steps):
+        oracle.kv_cache_append(Kh, Vh, wl.bits(ks[t]), wl.bits(vs[t]), lens_h, True)
+        if t in (0, 1, 31, 32, 33, 64, steps - 1):
+            ref = oracle.mqa_decode_step(wl.bits(qs[t]), Kh, Vh, lens_h)
+            check_close(runs[True][0][t].cpu().numpy(), ref, f"paper-shaped chained step {t}")
+    assert np.array_equal(runs[True][2].cpu().numpy(), lens_h)
+    assert runs[True][6] == mqa.binding.STATUS_APPEND_CACHE_FULL
