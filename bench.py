@@ -303,7 +303,7 @@ def layer_block(mqa, w, device, seed, steps, d_model=1024):
     secs = statistics.median(time_region(lambda _i: g.replay(), 1, device) for _ in range(20))
     weight_bytes = sum(t.numel() * 2 for t in W)
     return {"us_per_step": secs / steps * 1e6, "d_model": d, "weight_bytes": weight_bytes, "status": int(status.item()),
-            "launches_per_step": 3 + mqa.append_step_launches(b, h, m), "cache_sets": nset}
+            "launches_per_step": 2 + mqa.append_step_launches(b, h, m), "cache_sets": nset}
 
 
 def paper_loop_block(mqa, device, seed):

@@ -286,13 +286,13 @@ int mqa_decode_local_step(const void* q, void* K, void* V, const void* k_new, co
  *   P_o              [h, d, v] bf16              K, V, lens, advance, status   as for mqa_decode_append_step
  *   y                [b, d] fp32, written
  *   workspace        at least mqa_layer_workspace_bytes(b, h, d, m_max, k, v) bytes; may hold anything on entry.
- *                    It carries q, k_new, v_new (bf16), o (fp32), the per-head-group partial sums of y and the
- *                    attention step's own workspace.
+ *                    It carries q, k_new, v_new (bf16), o (fp32) and the attention step's own workspace.
  * d must be a multiple of 128 (MQA_ERR_UNSUPPORTED otherwise), k = v = 128.  The products run on the tensor
  * cores in bf16 with fp32 accumulation; q, k_new and v_new are rounded to bf16 where the step and the cache
  * take them, o is rounded to bf16 as an operand of the output product; y is summed over head groups in a fixed
  * order (no float atomics: results are reproducible bit for bit).  Kernels: projections in, the step (one
- * launch for large batches), projection out, the sum over head groups.
+ * launch for large batches), projection out (its head groups are one thread-block cluster of up to 16 CTAs, which
+ * sum y through distributed shared memory).
  */
 int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const void* P_v, const void* P_o,
                           void* K, void* V, int32_t* lens, int advance, float* y,

@@ -441,18 +441,15 @@ __global__ void lens_advance_kernel(int32_t* lens, int b, int m_max) {
 size_t align256(size_t n) { return (n + 255) & ~(size_t)255; }
 
 struct LayerWorkspace {
-    size_t q, k_new, v_new, o, part_y, step, total;     // byte offsets
-    int groups;                                         // head groups of the output projection
+    size_t q, k_new, v_new, o, step, total;             // byte offsets
 };
 LayerWorkspace layer_workspace(int b, int h, int d, int m_max) {
     LayerWorkspace w;
-    w.groups = (h + kProjHeadsPerCta - 1) / kProjHeadsPerCta;
     size_t at = 0;
     w.q = at;      at += align256((size_t)b * h * kHeadDim * 2);
     w.k_new = at;  at += align256((size_t)b * kHeadDim * 2);
     w.v_new = at;  at += align256((size_t)b * kHeadDim * 2);
     w.o = at;      at += align256((size_t)b * h * kHeadDim * 4);
-    w.part_y = at; at += align256((size_t)w.groups * b * d * 4);
     w.step = at;   at += align256(plan_workspace_bytes(make_plan(true, b, h, m_max)));
     w.total = at;
     return w;
@@ -494,9 +491,10 @@ int launch_projections_in(const void* x, const void* P_q, const void* P_k, const
     return launch_status();
 }
 
+// The output projection: the head groups of a (d tile, batch tile) are the CTAs of one thread-block cluster (see
+// project_out_kernel), so there are at most kProjMaxGroups of them, each with ceil(h / groups) heads.
 template <int NB>
-int launch_projection_out(const void* P_o, const float* o, float* part_y, float* y, int groups, int32_t* status, int b, int h,
-                          int d, cudaStream_t stream) {
+int launch_projection_out(const void* P_o, const float* o, float* y, int32_t* status, int b, int h, int d, cudaStream_t stream) {
     using Cfg = ProjCfg<NB>;
     auto kernel = project_out_kernel<NB>;
     constexpr int kSlot = 4 + (NB == 16 ? 0 : (NB == 32 ? 1 : (NB == 64 ? 2 : 3)));
@@ -504,7 +502,8 @@ int launch_projection_out(const void* P_o, const float* o, float* part_y, float*
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_proj_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess ||
+            (kProjMaxGroups > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
             cudaGetLastError();
             return MQA_ERR_CUDA;
         }
@@ -512,20 +511,23 @@ int launch_projection_out(const void* P_o, const float* o, float* part_y, float*
     }
     alignas(64) CUtensorMap map_po;
     if (!encode_matrix_map(&map_po, P_o, (long long)h * d, kHeadDim, 128)) return MQA_ERR_CUDA;
+    const int heads_per_cta = (h + kProjMaxGroups - 1) / kProjMaxGroups;
+    const int groups = (h + heads_per_cta - 1) / heads_per_cta;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(d / 128), (unsigned)groups, (unsigned)((b + 127) / 128));
     cfg.blockDim = dim3(kProjThreads);
     cfg.dynamicSmemBytes = kSmem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = (unsigned)groups;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, kernel, map_po, o, part_y, status, b, h, d);
-    if (launch_status()) return MQA_ERR_CUDA;
-    const int n = b * d;
-    launch_dependent(reduce_y_kernel, (unsigned)((n + 255) / 256), 256u, 0, stream, static_cast<const float*>(part_y), y, n, groups);
+    cfg.numAttrs = 2;
+    cudaLaunchKernelEx(&cfg, kernel, map_po, o, y, status, b, h, d, heads_per_cta);
     return launch_status();
 }
 
@@ -757,7 +759,6 @@ int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const
     void* k_new = base + w.k_new;
     void* v_new = base + w.v_new;
     float* o = reinterpret_cast<float*>(base + w.o);
-    float* part_y = reinterpret_cast<float*>(base + w.part_y);
     const int nb = b >= 128 ? 128 : (b > 64 ? 128 : (b > 32 ? 64 : (b > 16 ? 32 : 16)));
     int rc;
     switch (nb) {
@@ -771,10 +772,10 @@ int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const
                           b, h, m_max, k, v, stream_, true);
     if (rc) return rc;
     switch (nb) {
-        case 16: return launch_projection_out<16>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
-        case 32: return launch_projection_out<32>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
-        case 64: return launch_projection_out<64>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
-        default: return launch_projection_out<128>(P_o, o, part_y, y, w.groups, status, b, h, d, stream);
+        case 16: return launch_projection_out<16>(P_o, o, y, status, b, h, d, stream);
+        case 32: return launch_projection_out<32>(P_o, o, y, status, b, h, d, stream);
+        case 64: return launch_projection_out<64>(P_o, o, y, status, b, h, d, stream);
+        default: return launch_projection_out<128>(P_o, o, y, status, b, h, d, stream);
     }
 }
 

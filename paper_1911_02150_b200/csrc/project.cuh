@@ -13,8 +13,8 @@
 //                        Out^T[128 features x NB] = sum over d in chunks of 128:  W_chunk^T (MN-major A) * x_chunk^T (K-major B)
 //   project_out_kernel   CTA (d tile j, head group g): Y^T[128 x NB] = sum over the group's heads:
 //                        P_o[head][128 d-rows of tile j x 128] (K-major A) * o[:, head, :]^T (K-major B, converted
-//                        from fp32 to bf16 by the CTA); partial sums per head group go to the workspace
-//   reduce_y_kernel      y[b, d] = sum over head groups, in a fixed order (no float atomics)
+//                        from fp32 to bf16 by the CTA); the head groups of a tile are one thread-block cluster and
+//                        add their sums up through distributed shared memory, in a fixed order (no float atomics)
 //
 // NB = batch columns of a tile (the batch rounded up to 16, 32, 64 or 128; larger batches take
 // several tiles of 128).  Every wait is bounded (mbar_wait); TMEM is freed on every path.
@@ -27,7 +27,8 @@ namespace mqa {
 
 constexpr int kProjThreads = 6 * 32;           // warps 0-3: convert / read out, warp 4: TMA, warp 5: MMA issue
 constexpr int kProjChunkBytes = 128 * 256;     // 128 rows x 128 bf16 of a weight matrix: 32 KiB, two 64-column boxes
-constexpr int kProjHeadsPerCta = 2;            // project_out: heads summed by one CTA
+constexpr int kProjMaxGroups = 16;             // project_out: head groups of a tile = CTAs of one cluster (16: the
+                                               // non-portable cluster size, which the B200 offers; two heads per CTA at h = 32)
 
 template <int NB>
 struct ProjCfg {
@@ -161,61 +162,101 @@ project_in_kernel(const __grid_constant__ CUtensorMap map_pq, const __grid_const
     if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem, Cfg::kTmemCols); }
 }
 
+// ---- thread-block cluster helpers (the output projection sums its head groups through distributed shared memory)
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
+    return n;
+}
+// every thread of every CTA of the cluster, the same number of times on every path
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+// The head groups of one (d tile, batch tile) form one thread-block cluster (gridDim.y CTAs, at most 16): each CTA
+// accumulates Y^T over its heads in TMEM, leaves it in its shared memory, and after a cluster barrier every CTA adds up,
+// in group order, the batch rows that fall to it (row n to CTA n mod cluster size) out of all the CTAs' shared memory
+// and stores them to y.  No partial sums pass through global memory and no float atomics are used.
 template <int NB>
 __global__ void __launch_bounds__(kProjThreads, 1)
-project_out_kernel(const __grid_constant__ CUtensorMap map_po, const float* __restrict__ o, float* __restrict__ part_y,
-                   int32_t* __restrict__ status, int b, int h, int d) {
+project_out_kernel(const __grid_constant__ CUtensorMap map_po, const float* __restrict__ o, float* __restrict__ y,
+                   int32_t* __restrict__ status, int b, int h, int d, int heads_per_cta) {
     using Cfg = ProjCfg<NB>;
-    constexpr int S = 2;                                           // one stage per head of the group
+    constexpr int S = 2;                                           // ring of two stages: a head's weights and its o tile
     const int tile = blockIdx.x, group = blockIdx.y, row0 = blockIdx.z * 128;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int head0 = group * kProjHeadsPerCta;
-    const int n_heads = min(kProjHeadsPerCta, h - head0);
+    const int head0 = group * heads_per_cta;
+    const int n_heads = max(0, min(heads_per_cta, h - head0));
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* stages = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
     const uint32_t stages_s = smem_addr(stages);
-    const uint32_t w_full = stages_s + S * Cfg::kStageBytes, o_full = w_full + S * 8, done_s = o_full + S * 8;
+    const uint32_t w_full = stages_s + S * Cfg::kStageBytes, o_full = w_full + S * 8, empty_s = o_full + S * 8, done_s = empty_s + S * 8;
     __shared__ uint32_t tmem_slot;
-    __shared__ int timed_out;
+    __shared__ int timed_out, issued;
 
-    if (threadIdx.x == 0) {
+    if (warp == 4 && lane == 0) {                                  // by the thread that issues the copies
+        prefetch_tensormap(&map_po);
         timed_out = 0;
-        for (int s = 0; s < S; ++s) { mbar_init(w_full + s * 8, 1); mbar_init(o_full + s * 8, 4); }
+        issued = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(w_full + s * 8, 1); mbar_init(o_full + s * 8, 4); mbar_init(empty_s + s * 8, 1); }
         mbar_init(done_s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 4 && lane == 0) prefetch_tensormap(&map_po);
     if (warp == 5) { tmem_alloc(smem_addr(&tmem_slot), Cfg::kTmemCols); tmem_relinquish(); }
+    auto issue_weights = [&](int i) {
+        const int st = i % S;
+        const uint32_t bar = w_full + st * 8, w_s = stages_s + st * Cfg::kStageBytes;
+        mbar_expect_tx(bar, kProjChunkBytes);
+        const int yrow = (head0 + i) * d + tile * 128;
+        tma_load_2d(w_s, &map_po, 0, yrow, bar);
+        tma_load_2d(w_s + kProjChunkBytes / 2, &map_po, kBoxCols, yrow, bar);
+        issued = i + 1;
+    };
+    // the weights do not depend on the kernel before this one: the first copies start at once
+    if (warp == 4 && lane == 0)
+        for (int i = 0; i < n_heads && i < S; ++i) issue_weights(i);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-
-    if (warp == 4 && lane == 0) {
-        // the weights do not depend on the kernel before this one: their copies start at once
-        for (int i = 0; i < n_heads; ++i) {
-            const uint32_t bar = w_full + i * 8, w_s = stages_s + i * Cfg::kStageBytes;
-            mbar_expect_tx(bar, kProjChunkBytes);
-            const int y = (head0 + i) * d + tile * 128;
-            tma_load_2d(w_s, &map_po, 0, y, bar);
-            tma_load_2d(w_s + kProjChunkBytes / 2, &map_po, kBoxCols, y, bar);
-        }
-    }
     grid_dependency_wait();          // o comes from the kernel before this one
     grid_launch_dependents();
 
-    if (warp == 5) {
+    if (warp == 4) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int i = S; i < n_heads && ok; ++i) {
+                ok = mbar_wait(empty_s + (i % S) * 8, ((i / S) - 1) & 1);
+                if (ok) issue_weights(i);
+            }
+            if (!ok) atomicExch(&timed_out, 1);
+        }
+    } else if (warp == 5) {
         if (lane == 0) {
             constexpr uint32_t kIdesc = umma_idesc(128, NB, false, false);
             bool ok = true;
             for (int i = 0; i < n_heads; ++i) {
-                if (ok) ok = mbar_wait(w_full + i * 8, 0);
-                if (ok) ok = mbar_wait(o_full + i * 8, 0);
+                const int st = i % S;
+                if (ok) ok = mbar_wait(w_full + st * 8, (i / S) & 1);
+                if (ok) ok = mbar_wait(o_full + st * 8, (i / S) & 1);
                 tc_fence_after();
                 if (ok) {
-                    const uint32_t w_s = stages_s + i * Cfg::kStageBytes, o_s = w_s + kProjChunkBytes;
+                    const uint32_t w_s = stages_s + st * Cfg::kStageBytes, o_s = w_s + kProjChunkBytes;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {                         // 8 k-steps of 16 columns; 4 per 64-column box
                         const uint64_t a = umma_desc(w_s + (ks >> 2) * (kProjChunkBytes / 2) + (ks & 3) * 32, 16, 1024);
@@ -223,16 +264,20 @@ project_out_kernel(const __grid_constant__ CUtensorMap map_po, const float* __re
                         umma_ss(tmem, a, bd, kIdesc, (i > 0 || ks > 0) ? 1u : 0u);
                     }
                 }
+                tc_commit(empty_s + st * 8);                                 // the stage may be filled again
             }
             tc_commit(done_s);
             if (!ok) atomicExch(&timed_out, 1);
         }
-    } else if (warp < 4) {
+    } else {
         // ---- o[:, head, :] (fp32) -> bf16 tile [NB rows x 128 columns], K-major with the 128-byte swizzle:
         // row n, 16-byte chunk c of its 64-column half at n * 128 + ((c ^ (n & 7)) << 4)
         const int tid = warp * 32 + lane;
+        bool ok = true;
         for (int i = 0; i < n_heads; ++i) {
-            const uint32_t o_s = stages_s + i * Cfg::kStageBytes + kProjChunkBytes;
+            const int st = i % S;
+            if (i >= S && ok) ok = mbar_wait(empty_s + st * 8, ((i / S) - 1) & 1);   // the product that read this tile is done
+            const uint32_t o_s = stages_s + st * Cfg::kStageBytes + kProjChunkBytes;
             for (int item = tid; item < NB * 16; item += 128) {
                 const int n = item >> 4, ch = item & 15;                     // batch row of the tile, 8-column chunk
                 uint32_t w[4] = {0u, 0u, 0u, 0u};
@@ -247,49 +292,46 @@ project_out_kernel(const __grid_constant__ CUtensorMap map_po, const float* __re
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the tile is read by the tensor core
             __syncwarp();
-            if (lane == 0) mbar_arrive(o_full + i * 8);
+            if (lane == 0) mbar_arrive(o_full + st * 8);
         }
-        // ---- read-out: thread t = column tile * 128 + t of y, one TMEM lane; a TMEM column is a batch row
+        // ---- this CTA's Y^T (thread t = row t of the d tile, one TMEM lane; a TMEM column is a batch row) into its
+        // shared memory as [NB batch rows][128]: the stages are free once the last product has completed
         const int t = warp * 32 + lane;
-        const bool ok = mbar_wait(done_s, 0);
+        if (ok) ok = mbar_wait(done_s, 0);
         tc_fence_after();
-        if (ok) {
+        if (ok && n_heads > 0) {
             uint32_t acc[NB];
             tmem_ld_row<NB>(tmem + ((uint32_t)(warp * 32) << 16), acc);
-            float* out = part_y + ((size_t)group * b) * d + (size_t)tile * 128 + t;
 #pragma unroll
             for (int i = 0; i < NB; ++i)
-                if (row0 + i < b) out[(size_t)(row0 + i) * d] = __uint_as_float(acc[i]);
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(stages_s + (uint32_t)(i * 128 + t) * 4), "r"(acc[i]) : "memory");
         } else {
-            atomicExch(&timed_out, 1);
+#pragma unroll
+            for (int i = 0; i < NB; ++i)
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(stages_s + (uint32_t)(i * 128 + t) * 4), "r"(0u) : "memory");
         }
+        if (!ok) atomicExch(&timed_out, 1);
     }
     tc_fence_before();
     __syncthreads();
     if (timed_out && threadIdx.x == 0) {
-        for (int i = 0; i < n_heads; ++i) mbar_wait(w_full + i * 8, 0);       // the weight copies have to land before the CTA leaves
+        // before anything else: the last copy started into each stage has to land
+        for (int s = 0; s < S && s < issued; ++s) mbar_wait(w_full + s * 8, ((issued - 1 - s) / S) & 1);
         if (status) atomicOr(status, kStatusPipelineTimeout);
     }
     __syncthreads();
-    if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem, Cfg::kTmemCols); }
-}
-
-// y[b, d] = sum over the head groups of project_out_kernel, in group order (8 loads in flight per thread)
-__global__ void __launch_bounds__(256)
-reduce_y_kernel(const float* __restrict__ part_y, float* __restrict__ y, int n, int groups) {
-    grid_dependency_wait();
-    grid_launch_dependents();
-    const int i = blockIdx.x * 256 + threadIdx.x;      // one element of y
-    if (i >= n) return;
-    float acc = 0.f;
-    for (int g0 = 0; g0 < groups; g0 += 8) {
-        float p[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) p[e] = g0 + e < groups ? __ldcg(part_y + (size_t)(g0 + e) * n + i) : 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc += p[e];
+    cluster_sync();                  // every group's Y^T is in its shared memory
+    if (warp < 4) {
+        const int t = warp * 32 + lane;
+        const uint32_t rank = cluster_cta_rank(), n_groups = cluster_size();
+        for (int n = (int)rank; n < NB && row0 + n < b; n += (int)n_groups) {
+            float sum = 0.f;
+            for (uint32_t g = 0; g < n_groups; ++g) sum += ld_cluster_f32(stages_s + (uint32_t)(n * 128 + t) * 4, g);
+            y[(size_t)(row0 + n) * d + (size_t)tile * 128 + t] = sum;
+        }
     }
-    y[i] = acc;
+    cluster_sync();                  // nobody leaves while its shared memory is being read
+    if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem, Cfg::kTmemCols); }
 }
 
 }  // namespace mqa
