@@ -175,6 +175,7 @@ __device__ __forceinline__ uint32_t cluster_size() {
 }
 // every thread of every CTA of the cluster, the same number of times on every path
 __device__ __forceinline__ void cluster_sync() {
+    __syncwarp();                    // the aligned forms want the whole warp at the same instruction
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }

@@ -33,6 +33,24 @@ def test_header_and_binding_agree(L):
         assert hasattr(L, n), f"{n} is declared in include/mqa_decode.h but not exported"
 
 
+def test_header_constants_and_binding_agree():
+    text = open(os.path.join(ROOT, "include", "mqa_decode.h")).read()
+    defines = {m.group(1): int(m.group(2), 0) for m in re.finditer(r"^#define\s+(MQA_\w+)\s+\(?(\d+|0x[0-9a-fA-F]+)u?\)?\s*$", text, flags=re.M)}
+    assert defines["MQA_STEP_ADVANCE"] == binding.STEP_ADVANCE == 1
+    assert defines["MQA_STEP_CHAINED"] == binding.STEP_CHAINED == 2
+    assert defines["MQA_STEP_TEST_WRONG_GUESS"] == binding.STEP_TEST_WRONG_GUESS == 4
+    assert binding._step_flags(True, False) == 1 and binding._step_flags(False, True) == 2
+    assert binding._step_flags(True, "wrong-guess") == 7
+
+
+def test_step_flags_are_checked_before_any_launch(L):
+    vp = ctypes.c_void_p
+    a = vp(0x1000)
+    # an unknown flag bit: refused on the host, nothing dereferenced
+    rc = L.mqa_decode_append_step(a, a, a, a, a, a, 8, a, a, 1 << 30, None, 4, 8, 256, 128, 128, None)
+    assert rc == binding.ERR_INVALID_ARG
+
+
 def test_status_strings(L):
     seen = {binding.status_string(c) for c in range(0, 5)}
     assert len(seen) == 5
