@@ -384,7 +384,7 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
 
 int run_combine(bool multi_query, const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes,
                 int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0,
-                int32_t* lens_advance = nullptr) {
+                int32_t* lens_advance = nullptr, bool fused = false) {
     if (!lens || !o || !dims_ok(b, h, m_max) || !aligned16(o) || !aligned4(lens)) return MQA_ERR_INVALID_ARG;
     if (k != kHeadDim || v != kHeadDim) return MQA_ERR_UNSUPPORTED;
     const Plan p = make_plan(multi_query, b, h, m_max);
@@ -409,12 +409,15 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     const float2* part_ml = reinterpret_cast<const float2*>(workspace);
     const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +
                                                            partial_ml_bytes(p.units, p.n_splits));
+    // fused (the append-and-attend step of a sequence cut into fixed splits): the pass wrote a piece for every split,
+    // the second pass does not look at lens and moves it on when asked to
+    const int32_t* lens_read = fused ? nullptr : lens;
     if (p.n_splits <= kCombineEager)
-        launch_dependent(combine_splits_kernel<1>, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens, o, h,
-                         m_max, p.chunk_rows, p.n_splits, len_bias);
+        launch_dependent(combine_splits_kernel<1>, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens_read, o, h,
+                         m_max, p.chunk_rows, p.n_splits, len_bias, fused ? lens_advance : static_cast<int32_t*>(nullptr));
     else
-        launch_dependent(combine_splits_kernel<4>, (unsigned)p.units, 4 * kHeadDim, 0, stream, part_ml, part_acc, lens, o, h,
-                         m_max, p.chunk_rows, p.n_splits, len_bias);
+        launch_dependent(combine_splits_kernel<4>, (unsigned)p.units, 4 * kHeadDim, 0, stream, part_ml, part_acc, lens_read, o, h,
+                         m_max, p.chunk_rows, p.n_splits, len_bias, fused ? lens_advance : static_cast<int32_t*>(nullptr));
     return launch_status();
 }
 
@@ -645,6 +648,16 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
                    : launch_mma<2>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
                                    advance ? lens : nullptr);
     }
+    if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits > 1) {
+        // fixed splits: the CTA whose rows hold the new one writes it; the second pass moves lens on.  Two launches.
+        float2* part_ml = reinterpret_cast<float2*>(workspace);
+        float* part_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + partial_ml_bytes(p.units, p.n_splits));
+        rc = p.kernel == Kernel::kMma1
+                 ? launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr)
+                 : launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr);
+        if (rc) return rc;
+        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr, true);
+    }
     rc = kv_cache_append(K, V, k_new, v_new, lens, 0, status, b, 1, m_max, k, v, stream_);
     if (rc) return rc;
     rc = run_split(true, q, K, V, lens, o, workspace, workspace_bytes, status, b, h, m_max, k, v, stream, 1);
@@ -792,6 +805,7 @@ int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if (p.merge_in_kernel) return 1;                   // append, pass, merge and lens advance in one kernel
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits == 1) return 1;   // one CTA per sequence does it all
     if (p.stream()) return 2;                          // pass with the append inside, second pass
+    if (p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) return 2;   // fixed splits: the same two
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }
 

@@ -53,6 +53,10 @@ __device__ __forceinline__ void merge_pieces(int n, MlOf ml_of, AccOf acc_of, fl
     __syncthreads();
     float top = -INFINITY;
     for (int i = 0; i < n; ++i) top = fmaxf(top, m_s[i]);
+    if (top == -INFINITY) {                                // nothing but empty pieces: the empty prefix gives zeros
+        if (g == 0) out[c] = 0.f;
+        return;
+    }
     float num = 0.f, den = 0.f;
 #pragma unroll
     for (int e = 0; e < kCombineEager; ++e) {
@@ -91,13 +95,21 @@ template <int GROUPS>
 __global__ void __launch_bounds__(kHeadDim * (GROUPS >= 4 ? 4 : 1))
 combine_splits_kernel(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
                       const int32_t* __restrict__ lens, float* __restrict__ o,
-                      int h, int m_max, int chunk_rows, int n_splits, int len_bias) {
+                      int h, int m_max, int chunk_rows, int n_splits, int len_bias, int32_t* __restrict__ lens_advance) {
     const size_t u = blockIdx.x;
     grid_dependency_wait();          // the partials come from the kernel before this one
-    int L = biased_len(lens[u / h], m_max, len_bias);
-    L = L < 0 ? 0 : (L > m_max ? m_max : L);
-    int live = (L + chunk_rows - 1) / chunk_rows;
-    if (live > n_splits) live = n_splits;
+    // lens == nullptr: every split wrote its piece (an empty one has max = -inf) and nobody here looks at lens, so
+    // the CTA of a sequence's first head may move it on (lens_advance: the append-and-attend step)
+    int live = n_splits;
+    if (lens != nullptr) {
+        int L = biased_len(lens[u / h], m_max, len_bias);
+        L = L < 0 ? 0 : (L > m_max ? m_max : L);
+        live = (L + chunk_rows - 1) / chunk_rows;
+        if (live > n_splits) live = n_splits;
+    } else if (lens_advance != nullptr && u % h == 0 && threadIdx.x == 0) {
+        const int raw = lens_advance[u / h];
+        if (raw >= 0 && raw < m_max) lens_advance[u / h] = raw + 1;
+    }
     if (live == 0) {
         if (threadIdx.x < kHeadDim) o[u * kHeadDim + threadIdx.x] = 0.f;
         return;

@@ -399,11 +399,13 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // nobody else reads this sequence's length.
     // ring: the cache is a window of the last m_max positions (local attention, Section 4.1): lens[seq] counts
     // the tokens so far, the new row goes to row lens[seq] % m_max and min(lens[seq] + 1, m_max) rows are attended.
+    // A sequence cut into several splits (n_splits > 1) may take its new row too: the CTA whose rows hold it writes
+    // it, every split attends over one row more, and lens is left to the second-pass kernel.
     const int raw = lens[seq];
     const bool appended = fa.k_new != nullptr && raw >= 0 && (ring || raw < m_max);
     if (fa.k_new != nullptr) {
         if (!appended && threadIdx.x == 0 && status) atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
-        if (appended && warp == 0) {                       // lanes 0-15 move the key row, 16-31 the value row
+        if (appended && warp == 0 && (n_splits == 1 || raw / chunk_rows == split)) {   // lanes 0-15 move the key row, 16-31 the value row
             const size_t src = (size_t)seq * (kRowBytes / 16) + (lane & 15);
             const size_t dst = ((size_t)seq * m_max + (ring ? raw % m_max : raw)) * (kRowBytes / 16) + (lane & 15);
             if (lane < 16) fa.K[dst] = fa.k_new[src]; else fa.V[dst] = fa.v_new[src];
@@ -417,6 +419,9 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     if (r0 >= L) {                                         // nothing valid in this split (uniform)
         if (n_splits == 1)                                 // L == 0: the empty prefix gives zeros
             for (int i = threadIdx.x; i < h * kHeadDim; i += Cfg::kThreads) o[(size_t)seq * h * kHeadDim + i] = 0.f;
+        else                                               // an empty piece, for a second pass that does not look at lens
+            for (int i = threadIdx.x; i < h; i += Cfg::kThreads)
+                part_ml[((size_t)seq * h + i) * n_splits + split] = make_float2(-INFINITY, 0.f);
         for (int i = 0; i < pre; ++i) mbar_wait(full_s + i * 8, 0);   // copies started on a guess land before the CTA leaves
         return;
     }
