@@ -20,7 +20,7 @@ def check_close(got, ref, what):
     assert np.all(err.max(-1) <= REL_TOL * np.abs(ref).max(-1)), f"{what}: row-relative error"
 
 
-def run(b, h, m_max, lens0, advance, seed):
+def run(b, h, m_max, lens0, advance, seed, chained=False):
     inp = wl.make_inputs(b, h, m_max, "mqa", seed=seed, device=DEV)
     lens0 = np.asarray(lens0, np.int32)
     wl.poison_tail(inp["K"], np.clip(lens0, 0, m_max))
@@ -34,7 +34,7 @@ def run(b, h, m_max, lens0, advance, seed):
     ws.fill_(0xFF)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws, status,
-                               advance=advance)
+                               advance=advance, chained=chained)
     torch.cuda.synchronize()
     check_close(o.cpu().numpy(), ref, f"append_step b={b} h={h} m_max={m_max}")
     assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)   # the append, bit for bit
@@ -70,6 +70,13 @@ CASES = [
 @pytest.mark.parametrize("b,h,m_max", CASES)
 def test_append_step_matches_oracle(b, h, m_max, advance):
     run(b, h, m_max, lens_mix(b, m_max, seed=b + h), advance, seed=b * 7 + h)
+
+
+@pytest.mark.parametrize("chained", [True, "wrong-guess"])
+@pytest.mark.parametrize("b,h,m_max", CASES + [(300, 16, 1500), (1024, 8, 1024)])
+def test_append_step_with_the_chained_promise_matches_oracle(b, h, m_max, chained):
+    """Every plan accepts the promise (most ignore it); nothing but the set-up copies precedes the step here, so it holds."""
+    run(b, h, m_max, lens_mix(b, m_max, seed=b + h + 1), True, seed=b * 5 + h, chained=chained)
 
 
 def test_append_step_full_and_negative_sequences_take_no_row():
