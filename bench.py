@@ -151,19 +151,20 @@ class StepState:
         self.host_o = torch.empty(b, h, 128, dtype=torch.float32).pin_memory()
         self.d2h_bytes = self.host_o.numel() * 4
         self.h2d_bytes = sum(sizes)
-        self.host_steps = None
+        self.host_steps = self.bound_steps = None
         if variant == "mqa":
+            # the step bound once per cache set.  A decoding loop: between two steps nothing else writes the cache,
+            # lens or the workspace, hence chained
+            self.bound_steps = [mqa.AppendStep(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, self.o, self.ws,
+                                               self.status, advance=False, chained=True) for s in self.sets]
             # the library's host-buffer call, bound once per cache set (what a decoding loop over fixed pinned buffers does)
             qh, kh, vh = self.host_views
             self.host_steps = [mqa.HostStep(qh, kh, vh, self.host_o, s["K"], s["V"], self.lens_before, self.staging, self.ws,
                                             self.status, advance=False) for s in self.sets]
 
     def step(self, i):
-        s = self.sets[i % len(self.sets)]
-        if self.variant == "mqa":
-            # a decoding loop: between two steps nothing else writes the cache, lens or the workspace
-            self.mqa.mqa_decode_append_step(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, self.o,
-                                            self.ws, self.status, advance=False, chained=True)
+        if self.bound_steps is not None:
+            self.bound_steps[i % len(self.bound_steps)](torch.cuda.current_stream())   # (a capturing stream, in a graph)
         else:
             self.step_separate(i)
 
@@ -182,7 +183,7 @@ class StepState:
         stream = torch.cuda.current_stream()
         if self.host_steps is not None:
             # copies in, step, copy out: all enqueued by one C call on pinned host buffers
-            self.host_steps[i % len(self.host_steps)]()
+            self.host_steps[i % len(self.host_steps)](stream)
             stream.synchronize()                       # the caller needs o before the next token
             return
         s = self.sets[i % len(self.sets)]

@@ -264,14 +264,8 @@ def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
     return o
 
 
-def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None,
-                           chained: bool = False):
-    """One whole multi-query decoding step in one call: append ``k_new``/``v_new`` at row ``lens[b]`` of the
-    shared cache, then attend over ``lens[b] + 1`` rows; ``lens`` is advanced on the device when ``advance``.
-    For batches the persistent kernel serves (h <= 64) the whole step is one kernel launch.  ``chained``: the
-    caller's promise that nothing enqueued on the stream since this library's last step on this cache writes
-    the cache, ``lens`` or the workspace (a decoding loop); the kernel then starts on the cache before the
-    kernel ahead of it has finished."""
+def _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained):
+    """Checks the tensors of the append-and-attend step and returns the C call's argument tuple (plain integers)."""
     b, h, k = q.shape
     m_max, v = K.shape[-2], V.shape[-1]
     _need(q, torch.bfloat16, (b, h, k), "q")
@@ -283,13 +277,48 @@ def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, statu
     _need(o, torch.float32, (b, h, v), "o")
     if status is not None:
         _need(status, torch.int32, (1,), "status")
-    ws_ptr, ws_bytes = (None, 0) if workspace is None else (_ptr(workspace), workspace.numel() * workspace.element_size())
+    s = torch.cuda.current_stream(q.device) if stream is None else stream
+    return (q.data_ptr(), K.data_ptr(), V.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), lens.data_ptr(),
+            _step_flags(advance, chained), o.data_ptr(), None if workspace is None else workspace.data_ptr(),
+            0 if workspace is None else workspace.numel() * workspace.element_size(),
+            None if status is None else status.data_ptr(), b, h, m_max, k, v, s.cuda_stream)
+
+
+def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None,
+                           chained: bool = False):
+    """One whole multi-query decoding step in one call: append ``k_new``/``v_new`` at row ``lens[b]`` of the
+    shared cache, then attend over ``lens[b] + 1`` rows; ``lens`` is advanced on the device when ``advance``.
+    For batches the persistent kernel serves (h <= 64) the whole step is one kernel launch.  ``chained``: the
+    caller's promise that nothing enqueued on the stream since this library's last step on this cache writes
+    the cache, ``lens`` or the workspace (a decoding loop); the kernel then starts on the cache before the
+    kernel ahead of it has finished."""
+    args = _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained)
     with _OnDevice(q.device):
-        rc = lib().mqa_decode_append_step(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(lens),
-                                          _step_flags(advance, chained), _ptr(o), ws_ptr, ws_bytes, _ptr(status),
-                                          b, h, m_max, k, v, _stream(stream))
+        rc = lib().mqa_decode_append_step(*args)
     _check(rc, "mqa_decode_append_step")
     return o
+
+
+class AppendStep:
+    """:func:`mqa_decode_append_step` bound once to its tensors: a decoding loop refills the same q, k_new and v_new
+    buffers for every token, so the checks and the pointer marshalling (about 20 us of Python per call, several times
+    a short step) are done here and each call is the C call alone.  The tensors are kept alive by this object; the
+    stream is the one current (or given) at construction, and the cache's device must be current when it is called."""
+    __slots__ = ("fn", "args", "keep", "o")
+
+    def __init__(self, q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None,
+                 chained: bool = False):
+        self.args = _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained)
+        self.keep = (q, K, V, k_new, v_new, lens, o, workspace, status, stream)
+        self.fn = lib().mqa_decode_append_step
+        self.o = o
+
+    def __call__(self, stream=None):
+        """``stream``: another stream than the bound one for this call (a stream that is capturing a graph, say)."""
+        rc = self.fn(*self.args) if stream is None else self.fn(*self.args[:-1], stream.cuda_stream)
+        if rc != MQA_OK:
+            raise MqaError(rc, "mqa_decode_append_step")
+        return self.o
 
 
 def layer_workspace_bytes(b: int, h: int, d: int, m_max: int, k: int = 128, v: int = 128) -> int:
@@ -398,8 +427,9 @@ class HostStep:
         self.fn = lib().mqa_decode_append_step_host
         self.o_host = o_host
 
-    def __call__(self):
-        rc = self.fn(*self.args)
+    def __call__(self, stream=None):
+        """``stream``: another stream than the bound one for this call."""
+        rc = self.fn(*self.args) if stream is None else self.fn(*self.args[:-1], stream.cuda_stream)
         if rc != MQA_OK:
             raise MqaError(rc, "mqa_decode_append_step_host")
         return self.o_host

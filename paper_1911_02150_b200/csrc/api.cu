@@ -232,31 +232,39 @@ EncodeTiledFn encode_fn() {
     return f;
 }
 
-// The cache of one tensor (K or V) as a 2-D bf16 tensor [rows = b * m_max][128 columns], fetched in
-// boxes of kTileRows rows x 64 columns (128 bytes, the span of the 128-byte swizzle).
-bool encode_cache_map(CUtensorMap* map, const void* base, long long rows, int box_rows = kTileRows) {
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
-    const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)box_rows};
-    const cuuint32_t elem[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // A row-major bf16 matrix [rows][cols] fetched in boxes of box_rows rows x 64 columns (128-byte swizzle).
+// A decoding loop asks for the same few maps at every step (the cache, the weights) and encoding one costs about a
+// microsecond of host time, so every thread keeps the maps it encoded last, by (address, shape, box): a map describes
+// nothing but those, so it stays valid whatever the memory holds.
 bool encode_matrix_map(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+    struct Entry { const void* base; long long rows, cols; int box_rows; bool used; CUtensorMap map; };
+    constexpr int kEntries = 32;
+    thread_local Entry kept[kEntries] = {};
+    size_t hash = reinterpret_cast<size_t>(base) >> 8;
+    hash = (hash ^ (hash >> 7) ^ (size_t)rows * 31u ^ (size_t)cols * 131u ^ (size_t)box_rows * 7u) % kEntries;
+    Entry& e = kept[hash];
+    if (e.used && e.base == base && e.rows == rows && e.cols == cols && e.box_rows == box_rows) {
+        *map = e.map;
+        return true;
+    }
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    e.base = base; e.rows = rows; e.cols = cols; e.box_rows = box_rows; e.map = *map; e.used = true;
+    return true;
+}
+
+// The cache of one tensor (K or V) as a 2-D bf16 tensor [rows = b * m_max][128 columns], fetched in
+// boxes of kTileRows rows x 64 columns (128 bytes, the span of the 128-byte swizzle).
+bool encode_cache_map(CUtensorMap* map, const void* base, long long rows, int box_rows = kTileRows) {
+    return encode_matrix_map(map, base, rows, kHeadDim, box_rows);
 }
 
 std::atomic<int> g_smem_opt_in[kMaxDevices][4];

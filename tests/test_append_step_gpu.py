@@ -161,3 +161,24 @@ def test_host_buffer_entry_point_matches_the_device_one():
         torch.cuda.synchronize()
         assert torch.equal(o_host, o_dev.cpu())
         assert torch.equal(Kc.view(torch.int16), inp["K"].view(torch.int16)) and torch.equal(lens_c, lens_a)
+
+
+def test_bound_step_gives_what_the_call_gives():
+    b, h, m_max = 40, 16, 1500
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=22, device=DEV)
+    lens0 = lens_mix(b, m_max, seed=22)
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    K2, V2 = inp["K"].clone(), inp["V"].clone()
+    lens_a, lens_b = torch.from_numpy(lens0).to(DEV), torch.from_numpy(lens0.copy()).to(DEV)
+    o_a, o_b = (torch.empty(b, h, 128, dtype=torch.float32, device=DEV) for _ in range(2))
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    for _ in range(3):                                        # three tokens each way (the same q and rows: only lens moves)
+        mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_a, o_a, ws)
+    step = mqa.AppendStep(inp["q"], K2, V2, inp["k_new"], inp["v_new"], lens_b, o_b, ws)
+    for _ in range(3):
+        assert step() is o_b
+    torch.cuda.synchronize()
+    assert torch.equal(o_a.view(torch.int32), o_b.view(torch.int32)) and torch.equal(lens_a, lens_b)
+    assert torch.equal(inp["K"].view(torch.int16), K2.view(torch.int16)) and torch.equal(inp["V"].view(torch.int16), V2.view(torch.int16))
+    with pytest.raises(TypeError):
+        mqa.AppendStep(inp["q"].float(), K2, V2, inp["k_new"], inp["v_new"], lens_b, o_b, ws)
