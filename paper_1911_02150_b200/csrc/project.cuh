@@ -74,16 +74,32 @@ project_in_kernel(const __grid_constant__ CUtensorMap map_pq, const __grid_const
     __shared__ uint32_t tmem_slot;
     __shared__ int timed_out, issued;
 
-    if (threadIdx.x == 0) {
+    // The weights do not depend on the kernel before this one, x does: a stage's barrier takes two arrivals, one with
+    // the weight chunk's bytes and one with the x chunk's, and the weight copies of the first stages start before the wait.
+    const CUtensorMap* wmap = slab < h ? &map_pq : (slab == h ? &map_pk : &map_pv);
+    const int wrow0 = slab < h ? slab * d : 0;
+    auto issue_weights = [&](int c) {
+        const uint32_t bar = full_s + (c % S) * 8, w_s = stages_s + (c % S) * Cfg::kStageBytes;
+        mbar_expect_tx(bar, kProjChunkBytes);
+        tma_load_2d(w_s, wmap, 0, wrow0 + c * 128, bar);
+        tma_load_2d(w_s + kProjChunkBytes / 2, wmap, kBoxCols, wrow0 + c * 128, bar);
+    };
+    auto issue_x = [&](int c) {
+        const uint32_t bar = full_s + (c % S) * 8, x_s = stages_s + (c % S) * Cfg::kStageBytes + kProjChunkBytes;
+        mbar_expect_tx(bar, Cfg::kActBytes);
+        tma_load_2d(x_s, &map_x, c * 128, row0, bar);                         // rows past b read as zero
+        tma_load_2d(x_s + Cfg::kActBytes / 2, &map_x, c * 128 + kBoxCols, row0, bar);
+        issued = c + 1;
+    };
+    if (warp == 4 && lane == 0) {                                  // by the thread that issues the copies
+        prefetch_tensormap(&map_pq); prefetch_tensormap(&map_pk); prefetch_tensormap(&map_pv); prefetch_tensormap(&map_x);
         timed_out = 0;
         issued = 0;
-        for (int s = 0; s < S; ++s) { mbar_init(full_s + s * 8, 1); mbar_init(empty_s + s * 8, 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(full_s + s * 8, 2); mbar_init(empty_s + s * 8, 1); }
         mbar_init(done_s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 4 && lane == 0) {
-        prefetch_tensormap(&map_pq); prefetch_tensormap(&map_pk); prefetch_tensormap(&map_pv); prefetch_tensormap(&map_x);
+        for (int c = 0; c < n_chunks && c < S; ++c) issue_weights(c);
     }
     if (warp == 5) { tmem_alloc(smem_addr(&tmem_slot), Cfg::kTmemCols); tmem_relinquish(); }
     grid_dependency_wait();          // x may come from the kernel before this one
@@ -95,20 +111,14 @@ project_in_kernel(const __grid_constant__ CUtensorMap map_pq, const __grid_const
 
     if (warp == 4) {
         if (lane == 0) {
-            const CUtensorMap* wmap = slab < h ? &map_pq : (slab == h ? &map_pk : &map_pv);
-            const int wrow0 = slab < h ? slab * d : 0;
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
-                const int st = c % S;
-                if (c >= S) ok = mbar_wait(empty_s + st * 8, ((c / S) - 1) & 1);
-                if (!ok) break;
-                const uint32_t bar = full_s + st * 8, w_s = stages_s + st * Cfg::kStageBytes, x_s = w_s + kProjChunkBytes;
-                mbar_expect_tx(bar, Cfg::kStageBytes);
-                tma_load_2d(w_s, wmap, 0, wrow0 + c * 128, bar);
-                tma_load_2d(w_s + kProjChunkBytes / 2, wmap, kBoxCols, wrow0 + c * 128, bar);
-                tma_load_2d(x_s, &map_x, c * 128, row0, bar);                 // rows past b read as zero
-                tma_load_2d(x_s + Cfg::kActBytes / 2, &map_x, c * 128 + kBoxCols, row0, bar);
-                issued = c + 1;
+                if (c >= S) {
+                    ok = mbar_wait(empty_s + (c % S) * 8, ((c / S) - 1) & 1);
+                    if (!ok) break;
+                    issue_weights(c);
+                }
+                issue_x(c);
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
