@@ -401,14 +401,17 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // the tokens so far, the new row goes to row lens[seq] % m_max and min(lens[seq] + 1, m_max) rows are attended.
     // A sequence cut into several splits (n_splits > 1) may take its new row too: the CTA whose rows hold it writes
     // it, every split attends over one row more, and lens is left to the second-pass kernel.
+    // (the new row's pieces do not depend on lens: asked for first, so that the two loads are in flight together)
+    uint4 row_piece = make_uint4(0u, 0u, 0u, 0u);
+    if (fa.k_new != nullptr && warp == 0)                 // lanes 0-15 move the key row, 16-31 the value row
+        row_piece = (lane < 16 ? fa.k_new : fa.v_new)[(size_t)seq * (kRowBytes / 16) + (lane & 15)];
     const int raw = lens[seq];
     const bool appended = fa.k_new != nullptr && raw >= 0 && (ring || raw < m_max);
     if (fa.k_new != nullptr) {
         if (!appended && threadIdx.x == 0 && status) atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
-        if (appended && warp == 0 && (n_splits == 1 || raw / chunk_rows == split)) {   // lanes 0-15 move the key row, 16-31 the value row
-            const size_t src = (size_t)seq * (kRowBytes / 16) + (lane & 15);
+        if (appended && warp == 0 && (n_splits == 1 || raw / chunk_rows == split)) {
             const size_t dst = ((size_t)seq * m_max + (ring ? raw % m_max : raw)) * (kRowBytes / 16) + (lane & 15);
-            if (lane < 16) fa.K[dst] = fa.k_new[src]; else fa.V[dst] = fa.v_new[src];
+            if (lane < 16) fa.K[dst] = row_piece; else fa.V[dst] = row_piece;
             asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row (a barrier follows)
         }
     }
@@ -508,31 +511,48 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         }
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < M_TILES * 16 * kHeadDim; idx += Cfg::kThreads) {
-        const int c = idx & (kHeadDim - 1);
-        const int hr = (idx >> 7) & 15;
-        const int tile = idx >> 11;
-        const int head = tile * 16 + hr;
-        if (head >= h) continue;
+    // per head, once: the largest of the row-warps' maxima, each warp's weight, the sum
+    float* sm_w = reinterpret_cast<float*>(sm_ml + Cfg::kConsumerWarps * 16);   // [M_TILES * 16][8]: kRowWarps weights, max, sum
+    if (threadIdx.x < M_TILES * 16) {
+        const int tile = threadIdx.x >> 4, hr = threadIdx.x & 15;
+        float2 ml[kRowWarps];
         float top = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kRowWarps; ++w) top = fmaxf(top, sm_ml[(w * M_TILES + tile) * 16 + hr].x);
-        float num = 0.f, den = 0.f;
+        for (int w = 0; w < kRowWarps; ++w) {
+            ml[w] = sm_ml[(w * M_TILES + tile) * 16 + hr];              // consumer warp (rw = w, mt = tile)
+            top = fmaxf(top, ml[w].x);
+        }
+        float den = 0.f;
 #pragma unroll
         for (int w = 0; w < kRowWarps; ++w) {
-            const int src = w * M_TILES + tile;                          // consumer warp (rw = w, mt = tile)
-            const float2 ml = sm_ml[src * 16 + hr];
-            const float wt = fast_exp2(ml.x - top);                      // a warp without tiles: exp2(-inf) = 0
-            den = fmaf(wt, ml.y, den);
-            num = fmaf(wt, sm_acc[((size_t)src * 16 + hr) * kHeadDim + c], num);
+            const float wt = ml[w].x == -INFINITY ? 0.f : fast_exp2(ml[w].x - top);   // a warp without tiles counts for nothing
+            den = fmaf(wt, ml[w].y, den);
+            sm_w[threadIdx.x * 8 + w] = wt;
+        }
+        sm_w[threadIdx.x * 8 + kRowWarps] = top;
+        sm_w[threadIdx.x * 8 + kRowWarps + 1] = den;
+    }
+    __syncthreads();
+    // then 16 bytes of a head's 128 outputs per thread and round
+    for (int idx = threadIdx.x; idx < h * (kHeadDim / 4); idx += Cfg::kThreads) {
+        const int head = idx >> 5, c4 = idx & 31;
+        const int tile = head >> 4, hr = head & 15;
+        const float* wts = sm_w + head * 8;
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < kRowWarps; ++w) {
+            const float4 a = *reinterpret_cast<const float4*>(sm_acc + ((size_t)(w * M_TILES + tile) * 16 + hr) * kHeadDim + c4 * 4);
+            const float wt = wts[w];
+            num.x = fmaf(wt, a.x, num.x); num.y = fmaf(wt, a.y, num.y); num.z = fmaf(wt, a.z, num.z); num.w = fmaf(wt, a.w, num.w);
         }
         const size_t unit = (size_t)seq * h + head;
         if (n_splits == 1) {
-            o[unit * kHeadDim + c] = num / den;
+            const float inv = 1.f / wts[kRowWarps + 1];
+            *reinterpret_cast<float4*>(o + unit * kHeadDim + c4 * 4) = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
         } else {
             const size_t slot = unit * n_splits + split;
-            part_acc[slot * kHeadDim + c] = num;
-            if (c == 0) part_ml[slot] = make_float2(top, den);
+            *reinterpret_cast<float4*>(part_acc + slot * kHeadDim + c4 * 4) = num;
+            if (c4 == 0) part_ml[slot] = make_float2(wts[kRowWarps], wts[kRowWarps + 1]);
         }
     }
     if (lens_advance && appended && threadIdx.x == 0) lens_advance[seq] = raw + 1;   // every thread read lens[seq] barriers ago
