@@ -285,8 +285,10 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
         }
         g_smem_opt_in[dev][kSlot].store(1, std::memory_order_release);
     }
-    alignas(64) CUtensorMap map_k, map_v;
-    if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max))
+    alignas(64) CUtensorMap map_k, map_v, map_k_big, map_v_big;
+    if (!encode_cache_map(&map_k, K, (long long)b * m_max) || !encode_cache_map(&map_v, V, (long long)b * m_max) ||
+        !encode_cache_map(&map_k_big, K, (long long)b * m_max, 4 * kTileRows) ||
+        !encode_cache_map(&map_v_big, V, (long long)b * m_max, 4 * kTileRows))
         return MQA_ERR_CUDA;
     FusedArgs fa = {};
     if (k_new) {                                       // the whole decoding step in this launch (one CTA per sequence)
@@ -296,7 +298,7 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
         fa.V = static_cast<uint4*>(const_cast<void*>(V));
     }
     launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
-                     static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
+                     map_k_big, map_v_big, static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
                      p.n_splits, len_bias, fa, lens_advance, ring ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }

@@ -201,10 +201,10 @@ __device__ __forceinline__ void load_q_fragments(uint32_t (&qa)[8][4], const uin
 // HILO: feed P to the tensor cores as bf16 hi + lo parts (weights good to ~2^-17) instead of one
 // bf16 rounding (2^-9 per weight).  One rounding is enough once the prefix is long: the output
 // is then an average over many rows, of size ~1/sqrt(rows), and so is the rounding error.
-// HALF_STRIDE: bytes between the box holding columns 0..63 and the box holding columns 64..127.
-template <bool HILO, int HALF_STRIDE>
+// half_stride: bytes between the box holding columns 0..63 and the box holding columns 64..127.
+template <bool HILO>
 __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)[8][4], const LaneOffsets& off,
-                                             uint32_t k_s, uint32_t v_s, int row0, int r1, int lane) {
+                                             uint32_t k_s, uint32_t v_s, uint32_t half_stride, int row0, int r1, int lane) {
     const int t4 = lane & 3;
     const bool ragged = row0 + kTileRows > r1;
 
@@ -214,7 +214,7 @@ __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)
     for (int nt = 0; nt < 4; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-        const uint32_t a = k_s + off.k[ks & 3] + (ks >> 2) * HALF_STRIDE;
+        const uint32_t a = k_s + off.k[ks & 3] + (ks >> 2) * half_stride;
 #pragma unroll
         for (int np = 0; np < 2; ++np) {               // n-tile pairs (0,1) and (2,3): 16 rows = 2 KiB apart
             uint32_t b0, b1, b2, b3;
@@ -285,7 +285,7 @@ __device__ __forceinline__ void consume_tile(WarpState& st, const uint32_t (&qa)
 #pragma unroll
         for (int vp = 0; vp < 8; ++vp) {                         // pairs of 8-column n-tiles
             uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(v_s + off.v[vp & 3] + (vp >> 2) * HALF_STRIDE + kk * 2048, b0, b1, b2, b3);
+            ldmatrix_x4_trans(v_s + off.v[vp & 3] + (vp >> 2) * half_stride + kk * 2048, b0, b1, b2, b3);
             if (ragged) { b0 &= keep_lo; b1 &= keep_hi; b2 &= keep_lo; b3 &= keep_hi; }
             mma_bf16(st.acc[vp * 2], p_hi[kk], b0, b1);
             mma_bf16(st.acc[vp * 2 + 1], p_hi[kk], b2, b3);
@@ -335,6 +335,7 @@ __device__ __forceinline__ void store_state(const WarpState& st, float* __restri
 template <int M_TILES, bool EARLY = false>
 __global__ void __launch_bounds__(MmaCfg<M_TILES>::kThreads, MmaCfg<M_TILES>::kMinBlocks)
 mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                            const __grid_constant__ CUtensorMap map_k_big, const __grid_constant__ CUtensorMap map_v_big,
                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                             float* __restrict__ o, float2* __restrict__ part_ml, float* __restrict__ part_acc,
                             int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias,
@@ -429,6 +430,9 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         return;
     }
     const int n_tiles = (r1 - r0 + kTileRows - 1) / kTileRows;
+    // a few tiles (each has a stage of its own), beginning at a multiple of 128 rows: fetched four tiles per copy
+    // (from three tiles on: a copy moves all 128 rows of its box, and one or two tiles are quicker on their own)
+    const bool big = !EARLY && n_tiles >= 3 && n_tiles <= kStages && (r0 & (4 * kTileRows - 1)) == 0;
 
     __syncthreads();
 
@@ -438,7 +442,19 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 
     if (warp == Cfg::kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
-        if (lane == 0) {
+        if (lane == 0 && big) {
+            // four tiles per copy: boxes of 128 rows (K columns 0-63, 64-127, V likewise), a quarter of the copies
+            for (int grp = 0; grp * 4 < n_tiles; ++grp) {
+                const uint32_t bar = full_s + grp * 8, dst = stages_s + grp * 4 * kStageBytes;
+                mbar_expect_tx(bar, 4 * kStageBytes);
+                const int y = row_base + grp * 4 * kTileRows;
+                tma_load_2d(dst, &map_k_big, 0, y, bar);
+                tma_load_2d(dst + 4 * kBoxBytes, &map_k_big, kBoxCols, y, bar);
+                tma_load_2d(dst + 8 * kBoxBytes, &map_v_big, 0, y, bar);
+                tma_load_2d(dst + 12 * kBoxBytes, &map_v_big, kBoxCols, y, bar);
+                issued = grp + 1;
+            }
+        } else if (lane == 0) {
             bool ok = true;
             for (int i = pre; i < n_tiles && ok; ++i) {
                 const int s = i % kStages;
@@ -459,10 +475,12 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         bool ok = true;
         for (int i = rw; i < n_tiles; i += kRowWarps) {
             const int s = i % kStages;
-            ok = mbar_wait(full_s + s * 8, (i / kStages) & 1);
+            ok = big ? mbar_wait(full_s + (i >> 2) * 8, 0) : mbar_wait(full_s + s * 8, (i / kStages) & 1);
             if (!ok) break;
-            const uint32_t k_s = stages_s + s * kStageBytes;
-            consume_tile<true, kBoxBytes>(st, qa, off, k_s, k_s + 2 * kBoxBytes, r0 + i * kTileRows, r1, lane);
+            // a tile's K boxes, then its V boxes; in a copy of four tiles the tile is 32 of a box's 128 rows
+            const uint32_t k_s = big ? stages_s + (i >> 2) * 4 * kStageBytes + (i & 3) * kBoxBytes : stages_s + s * kStageBytes;
+            const uint32_t half = big ? 4 * kBoxBytes : kBoxBytes;
+            consume_tile<true>(st, qa, off, k_s, k_s + 2 * half, half, r0 + i * kTileRows, r1, lane);
             // The tile was read through the generic proxy (ldmatrix) and the copy engine will write the stage
             // again through the async proxy: without this fence the last ldmatrix of a tile now and then saw
             // rows of the tile that came four tiles later (one run in a few hundred, 16 output columns off).
