@@ -438,7 +438,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-layer", action="store_true", help="skip the timing of the whole layer step (projections either side)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
-    ap.add_argument("--sweep", action="store_true", help="run every workload and write gpurun_out/sweep.json")
+    ap.add_argument("--sweep", action="store_true", help="run every workload, both variants, and write the table to --sweep-out")
+    ap.add_argument("--sweep-out", default="sweep.json", help="where --sweep writes its table (JSON)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = wl.WORKLOADS[args.workload]
@@ -525,7 +526,7 @@ def main():
 
 
 def run_sweep(mqa, args, device, rank):
-    """Every workload, both variants: us per step and GB/s per point -> gpurun_out/sweep.json."""
+    """Every workload, both variants: us per step and GB/s per point, written to args.sweep_out."""
     peak, peak_kind = measured_peak()
     rows = []
     for name, w in wl.WORKLOADS.items():
@@ -551,11 +552,12 @@ def run_sweep(mqa, args, device, rank):
             print(json.dumps(blk), file=sys.stderr)
             del st
             torch.cuda.empty_cache()
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
+    out_dir = os.path.dirname(os.path.abspath(args.sweep_out))
+    os.makedirs(out_dir, exist_ok=True)
+    with open(args.sweep_out, "w") as f:
         json.dump({"peak_gbs": peak, "peak_kind": peak_kind, "rows": rows}, f, indent=1)
     if rank == 0:
-        print(json.dumps({"sweep_points": len(rows), "written": "gpurun_out/sweep.json"}))
+        print(json.dumps({"sweep_points": len(rows), "written": args.sweep_out}))
 
 
 if __name__ == "__main__":
