@@ -105,7 +105,7 @@ class StepState:
     """Device-resident state of one variant: rotating cache sets (to keep reads out of L2), the
     step's inputs and outputs, and the launch plan."""
 
-    def __init__(self, mqa, variant, w, device, seed, min_rotate_bytes):
+    def __init__(self, mqa, variant, w, device, seed, min_rotate_bytes, host_legs=True):
         self.mqa, self.variant, self.w, self.device = mqa, variant, w, device
         b, h, m = w.b, w.h, w.m_max
         self.kvh = 1 if variant == "mqa" else h
@@ -134,6 +134,14 @@ class StepState:
         self.launches_three = 2 + (1 if self.n_splits > 1 else 0)
         # the multi-query step is one call (append + attention + merge); multi-head is append + step
         self.launches_per_step = mqa.append_step_launches(b, h, m) if variant == "mqa" else self.launches_three
+        self.host_steps = self.bound_steps = None
+        if variant == "mqa":
+            # the step bound once per cache set.  A decoding loop: apart from the steps themselves nothing writes lens or
+            # the caches' rows, hence chained (the sets share one workspace and one o, which the promise leaves free)
+            self.bound_steps = [mqa.AppendStep(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, self.o, self.ws,
+                                               self.status, advance=False, chained=True) for s in self.sets]
+        if not host_legs:
+            return
         # pinned host copies of the per-step inputs / result for the end-to-end leg
         # (q, k_new, v_new packed in one pinned buffer and one device buffer: one host-to-device copy per step)
         s0 = self.sets[0]
@@ -151,12 +159,7 @@ class StepState:
         self.host_o = torch.empty(b, h, 128, dtype=torch.float32).pin_memory()
         self.d2h_bytes = self.host_o.numel() * 4
         self.h2d_bytes = sum(sizes)
-        self.host_steps = self.bound_steps = None
         if variant == "mqa":
-            # the step bound once per cache set.  A decoding loop: between two steps nothing else writes the cache,
-            # lens or the workspace, hence chained
-            self.bound_steps = [mqa.AppendStep(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], self.lens_before, self.o, self.ws,
-                                               self.status, advance=False, chained=True) for s in self.sets]
             # the library's host-buffer call, bound once per cache set (what a decoding loop over fixed pinned buffers does)
             qh, kh, vh = self.host_views
             self.host_steps = [mqa.HostStep(qh, kh, vh, self.host_o, s["K"], s["V"], self.lens_before, self.staging, self.ws,
@@ -219,6 +222,59 @@ def capture_graph(fn, steps):
     return g
 
 
+def time_isolated(st: StepState, steps, device):
+    """Seconds per step when the step does NOT follow a step: every timed launch comes after an unrelated kernel that
+    has nothing to do with the cache (a 4 MiB fill by torch, ~2 us), has its own CUDA-event pair around it, and is
+    launched from the host.  What a back-to-back loop hides -- launch latency, the set-up that programmatic dependent
+    launch overlaps with the previous step, copies started early on the chained promise -- is all inside this figure,
+    and so is the resolution of an event pair (about half a microsecond)."""
+    spacer = torch.empty(1 << 20, dtype=torch.float32, device=device)
+    n = max(steps, 20)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for i in range(3):
+        spacer.fill_(float(i)); st.step(i)
+    torch.cuda.synchronize(device)
+    for i, (e0, e1) in enumerate(ev):
+        spacer.fill_(float(i))
+        e0.record(); st.step(i); e1.record()
+    torch.cuda.synchronize(device)
+    return statistics.median(e0.elapsed_time(e1) for e0, e1 in ev) * 1e-3
+
+
+def quick_point(mqa, variant, w, device, steps=20, min_rotate_bytes=4 * L2_BYTES):
+    """One sweep point for the default bench line: us per step (K steps as one CUDA graph, caches rotated past L2),
+    GB/s, launches.  None for the fields of a point that was skipped, with the reason."""
+    kvh = 1 if variant == "mqa" else w.h
+    cache = 2 * w.b * kvh * w.m_max * 256
+    row = {"workload": w.name, "variant": variant, "b": w.b, "h": w.h, "m": w.m_max}
+    free, _ = torch.cuda.mem_get_info(device)
+    if cache > 16 * 2 ** 30:
+        row["skipped"] = f"a {cache >> 30} GiB cache takes longer to fill than the default run allows (bench.py --sweep runs it)"
+        return row
+    if cache + 6 * 2 ** 30 > free:
+        row["skipped"] = f"cache of {cache >> 30} GiB does not fit"
+        return row
+    st = StepState(mqa, variant, w, device, 0, min_rotate_bytes=min_rotate_bytes, host_legs=False)
+    for i in range(3):
+        st.step(i)
+    torch.cuda.synchronize(device)
+    g = capture_graph(st.step, steps)
+    g.replay()
+    torch.cuda.synchronize(device)
+    secs = statistics.median(time_region(lambda _i: g.replay(), 1, device) for _ in range(10)) / steps
+    gbs = st.bytes / secs / 1e9
+    row.update({"us_per_step": secs * 1e6, "gbs": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_step": st.bytes,
+                "launches_per_step": st.launches_per_step, "cache_sets": len(st.sets), "status": int(st.status.item())})
+    del st, g
+    torch.cuda.empty_cache()
+    return row
+
+
+# The points the >= 70 % target names (long-context configurations) and the ragged batch, for the default bench line.
+LINE_SWEEP = ("sweep_b1_m32768", "sweep_b8_m32768", "sweep_b64_m32768", "sweep_b256_m32768", "sweep_b64_m4096",
+              "sweep_b256_m4096", "ragged")
+
+
 def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=True, min_warm_s=0.2):
     t0 = time.time()
     i = 0
@@ -266,12 +322,13 @@ def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=T
     # per-launch duration of the pass over the cache (the dominant kernel): K back-to-back launches
     kernel_regions = [time_region(run_split, calls, device) for _ in range(max(3, min(20, len(regions))))]
     kernel_s = statistics.median(kernel_regions) / steps
+    isolated_s = time_isolated(st, steps, device)
     # end to end with host buffers (eager: every step waits for its result)
     for i in range(3):
         st.step_e2e(i)
     e2e_s = time_region(st.step_e2e, steps, device)
     status = int(st.status.item())
-    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status, "separate_s": sep_s,
+    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status, "separate_s": sep_s, "isolated_s": isolated_s,
             "clocks": sampler.summary() if sampler else None, "first_region_s": regions[0],
             "min_region_s": min(regions), "regions": len(regions), "graph": bool(use_graph)}
 
@@ -420,7 +477,7 @@ def result_block(st, r, steps):
     gbs = st.bytes / (r["secs"] / steps) / 1e9
     return {"us_per_step": us, "gbs": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_step": st.bytes,
             "n_splits": st.n_splits, "chunk_rows": st.chunk_rows, "cache_sets": len(st.sets),
-            "kernel_us": r["kernel_s"] * 1e6, "status": r["status"],
+            "pass_only_us": r["kernel_s"] * 1e6, "isolated_us": r["isolated_s"] * 1e6, "status": r["status"],
             "separate_calls_us_per_step": None if r.get("separate_s") is None else r["separate_s"] / steps * 1e6,
             "launches_per_step": st.launches_per_step,
             "first_region_us_per_step": r["first_region_s"] / steps * 1e6,
@@ -437,6 +494,7 @@ def main():
     ap.add_argument("--no-mha", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-layer", action="store_true", help="skip the timing of the whole layer step (projections either side)")
+    ap.add_argument("--no-line-sweep", action="store_true", help="skip the long-context sweep points of the default line")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true", help="run every workload, both variants, and write the table to --sweep-out")
     ap.add_argument("--sweep-out", default="sweep.json", help="where --sweep writes its table (JSON)")
@@ -476,7 +534,16 @@ def main():
     total_bytes = sharding.sum_over_ranks(st.bytes, device)
     value = total_bytes / (secs_max / args.steps) / 1e9
     e2e_value = total_bytes / (e2e_max / args.steps) / 1e9
-    kernel_gbs = st.bytes / r["kernel_s"] / 1e9
+    step_s = r["secs"] / args.steps
+    one_launch = st.launches_per_step == 1
+    # the dominant kernel: with one launch per step it IS the step, and its duration is the step's (K back-to-back
+    # launches of that call, CUDA events); otherwise it is the pass over the cache, timed on its own below
+    dom_s = step_s if one_launch else r["kernel_s"]
+    dom_gbs = st.bytes / dom_s / 1e9
+    pass_gbs = st.bytes / r["kernel_s"] / 1e9
+    iso_gbs = st.bytes / r["isolated_s"] / 1e9
+    step_kernel = mqa.plan_kernel_name(True, True, w.b, w.h, w.m_max)
+    pass_kernel = mqa.plan_kernel_name(True, False, w.b, w.h, w.m_max)
     out = {
         "metric": "mqa_decode_step_hbm_gbs", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": secs_max / args.steps * 1e3, "higher_is_better": True,
@@ -485,13 +552,24 @@ def main():
                    "l2": f"rotating {len(st.sets)} cache sets of {st.cache_bytes >> 20} MiB (> L2) between steps",
                    "launch": "K steps replayed as one CUDA graph" if r["graph"] else "K steps launched from the host",
                    "step": "mqa_decode_append_step, MQA_STEP_CHAINED (a decoding loop: only steps write the cache)",
+                   "value_is": "the back-to-back loop (each step's set-up overlaps the step before); roofline.isolated "
+                               "is the same step after an unrelated kernel",
                    "n_splits": st.n_splits, "chunk_rows": st.chunk_rows},
         "us_per_step": blk["us_per_step"], "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
         "mqa": blk,
-        "roofline": {"bound": "hbm", "achieved": kernel_gbs, "peak": peak, "unit": "GB/s", "frac": kernel_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "traffic": None,
-                     "kernel": "split pass of mqa_decode_step", "kernel_us": r["kernel_s"] * 1e6,
-                     "algorithmic_bytes": st.bytes},
+        "roofline": {"bound": "hbm", "achieved": dom_gbs, "peak": peak, "unit": "GB/s", "frac": dom_gbs / peak,
+                     "frac_of_8TBs": dom_gbs / NOMINAL_HBM_GBS, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "kernel": step_kernel if one_launch else pass_kernel,
+                     "kernel_is": ("the step's one launch (append + pass over the cache + merge), back to back"
+                                   if one_launch else "the pass over the cache, back to back (the step adds a second-pass kernel)"),
+                     "kernel_us": dom_s * 1e6, "algorithmic_bytes": st.bytes,
+                     "pass_only": {"kernel": pass_kernel, "kernel_us": r["kernel_s"] * 1e6, "achieved": pass_gbs,
+                                   "frac": pass_gbs / peak, "frac_of_8TBs": pass_gbs / NOMINAL_HBM_GBS,
+                                   "what": "mqa_decode_step_split back to back: no append, no merge"},
+                     "isolated": {"kernel_us": r["isolated_s"] * 1e6, "achieved": iso_gbs, "frac": iso_gbs / peak,
+                                  "frac_of_8TBs": iso_gbs / NOMINAL_HBM_GBS,
+                                  "what": "the whole step launched from the host after an unrelated kernel, one CUDA-event "
+                                          "pair per launch: nothing of it overlaps a step before"}},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": st.h2d_bytes,
                 "d2h_bytes_per_step": st.d2h_bytes, "us_per_step": e2e_max / args.steps * 1e6,
                 "note": "per-step inputs q,k_new,v_new from pinned host memory, o read back; the KV cache is "
@@ -502,7 +580,10 @@ def main():
     traffic = os.path.join(ROOT, "profiles", "traffic.txt")
     if os.path.exists(traffic):
         try:
-            out["roofline"]["traffic"] = json.load(open(traffic)).get(w.name, {}).get("mqa_split_dram_bytes")
+            entry = json.load(open(traffic)).get(w.name, {})
+            key = "mqa_step_dram_bytes" if one_launch else "mqa_split_dram_bytes"
+            out["roofline"]["traffic"] = entry.get(key)
+            out["roofline"]["traffic_source"] = entry.get(key.replace("_dram_bytes", "_source"), entry.get("source"))
         except Exception:
             pass
     del st
@@ -519,6 +600,10 @@ def main():
         out["layer_step"] = layer_block(mqa, w, device, seed, max(3, min(args.steps, 20)))
         out["paper_incremental"] = paper_loop_block(mqa, device, seed)
         out["layer_step"]["projections_us"] = out["layer_step"]["us_per_step"] - blk["us_per_step"]
+    if not args.no_line_sweep and world == 1:
+        # the other long-context points and the ragged batch: us, GB/s, fraction of 8 TB/s, launches, both variants
+        out["sweep"] = [quick_point(mqa, variant, wl.WORKLOADS[name], device)
+                        for name in LINE_SWEEP for variant in ("mqa", "mha")]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, seed)
     if rank == 0:

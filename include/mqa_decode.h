@@ -24,8 +24,11 @@
  *     Calls only enqueue work on it: they never synchronise, never allocate device memory and
  *     never free anything.  The launch configuration is chosen from the integer arguments and
  *     the current device alone, never from device data.
- *   - Return value: MQA_OK (0) or one of the positive codes below.  On any error NO kernel has
- *     been launched and no buffer has been touched.
+ *   - Return value: MQA_OK (0) or one of the positive codes below.  Arguments, sizes and the
+ *     workspace are checked before anything is enqueued: with every code except MQA_ERR_CUDA no
+ *     kernel or copy has been launched and no buffer has been touched.  MQA_ERR_CUDA reports a
+ *     failed launch or copy; in a call that enqueues several, the earlier ones are then already
+ *     on the stream.
  *   - Cache rows at or beyond lens[b] are don't-care: they may hold anything (NaN, Inf) and
  *     do not influence o.  lens[b] outside [0, m_max] is clamped into it for the attention
  *     and reported through `status`; nothing is read or written out of bounds.
@@ -101,10 +104,13 @@ int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new,
  * (an exact re-association of the same softmax); shared K/V rows are read from HBM once and
  * used for all h heads.  For large batches (every SM takes an equal share of all valid rows)
  * the pieces of a sequence are merged inside the same kernel by the CTA that finishes the
- * sequence's last piece: one launch.  The bookkeeping for that lives in the workspace under a
- * per-call epoch that the kernel itself moves on, so nothing has to be initialised and CUDA-graph
- * replays are safe; after a call that reported PIPELINE_TIMEOUT, clear the workspace (any
- * constant) before using it again.  Other sizes use a second kernel to combine the pieces.
+ * sequence's last piece: one launch.  The bookkeeping for that lives at the head of the workspace
+ * under a per-call epoch that the kernel itself moves on -- one epoch per workspace, whatever the
+ * sizes of the calls that share it -- so nothing has to be initialised, CUDA-graph replays are
+ * safe, and a workspace may serve calls of different shapes one after the other.  A call that
+ * reported PIPELINE_TIMEOUT moves the epoch on as well: the workspace needs no repair afterwards.
+ * Between two calls the caller may overwrite the whole workspace or leave it alone, but must not
+ * restore an older copy of it.  Other sizes use a second kernel to combine the pieces.
  */
 int mqa_decode_step(const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                     void* workspace, size_t workspace_bytes, int32_t* status,
@@ -136,15 +142,20 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
  *   advance           bit flags.  MQA_STEP_ADVANCE (1): lens[b] += 1 on return for sequences that took a
  *                     row; without it lens is left as it was, although the row has been written and
  *                     attended over.  MQA_STEP_CHAINED (2): a promise by the caller about the work that
- *                     precedes this call on `stream` -- since the most recent step of this library on this
- *                     cache (that step excepted), or since the stream was last idle, nothing enqueued on
- *                     it writes K, V, lens or the workspace.  A decoding loop keeps it: between two steps
- *                     run projections, a sampler, copies of q.  The first step after something else filled
- *                     the cache (a prefill kernel) must not carry it.  With the promise the persistent
- *                     kernel starts fetching the cache, except each prefix's last rows, while the kernel
- *                     before it is still finishing, and reads q, the new rows and lens only after that
- *                     kernel has completed.  What it fetches early goes by lens as it reads then; should
- *                     lens have moved by the time it may rely on it, it fetches again.
+ *                     precedes this call on `stream` and may still be running when this call's kernel
+ *                     starts (everything enqueued since the stream was last idle, or since the kernel
+ *                     before the most recent kernel completed): apart from steps of this library, none
+ *                     of it writes lens, and none of it writes rows of THIS cache below the last two
+ *                     rows of each prefix.  Steps of this library on this or on other caches keep the
+ *                     promise (a step writes one row per sequence at the end of its prefix and moves
+ *                     lens on by one), and so do projections, a sampler, copies of q; other caches, o
+ *                     and the workspace may be written freely.  The first step after something else
+ *                     filled the cache (a prefill kernel) must not carry the flag.  With the promise
+ *                     the persistent kernel starts fetching the cache, except each prefix's last rows,
+ *                     while the kernel before it is still finishing, and reads q, the new rows, lens
+ *                     and the workspace only after that kernel has completed.  What it fetches early
+ *                     goes by lens as it reads then; should lens have moved by the time it may rely on
+ *                     it, it fetches again.
  *                     MQA_STEP_TEST_WRONG_GUESS (4), for tests, with MQA_STEP_CHAINED: the early fetch is
  *                     deliberately the wrong one, so that this recovery runs; results are unchanged.
  *                     Any other bit: MQA_ERR_INVALID_ARG.
@@ -198,6 +209,14 @@ size_t mqa_workspace_bytes(int b, int h, int m_max, int k, int v);
 int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int* chunk_rows);
 
 /*
+ * mqa_plan_kernel_name -- the name of the kernel that does the pass over the cache for these sizes on
+ * the current device (`multi_query` as for mqa_plan_splits; `whole_step` non-zero: as launched by
+ * mqa_decode_append_step with MQA_STEP_CHAINED, zero: as launched by mqa_decode_step).  A static string,
+ * "" for invalid arguments.  Informational (benchmarks and profiles name what they timed); host-only.
+ */
+const char* mqa_plan_kernel_name(int multi_query, int whole_step, int b, int h, int m_max, int k, int v);
+
+/*
  * mqa_decode_step_noalloc -- mqa_decode_step for callers that cannot allocate.  (The paper has
  * no counterpart to this entry point; it computes exactly what mqa_decode_step computes.)
  *
@@ -218,7 +237,8 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
  *   that device current) and remembers it; make this first call during set-up, before any
  *   stream capture is begun on that device.
  *   Sharing: every call on a device uses the same array, which still holds whatever the last
- *   call left in it.  Nothing has to be cleared -- a call reads only what the same call has
+ *   call left in it, of whatever shape that call was.  Nothing has to be cleared, not even
+ *   after a call that reported PIPELINE_TIMEOUT -- a call reads only what the same call has
  *   written, or what carries its own epoch -- but two calls whose kernels may overlap on the
  *   GPU (different streams, no ordering between them) race on it and corrupt each other's
  *   results.  Calls on one stream are safe.

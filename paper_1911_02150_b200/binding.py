@@ -25,7 +25,7 @@ EXPORTS = (
     "kv_cache_append", "mqa_decode_step", "mha_decode_step",
     "mqa_decode_step_split", "mqa_decode_step_combine",
     "mha_decode_step_split", "mha_decode_step_combine",
-    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_status_string", "mqa_decode_step_noalloc",
+    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
     "mqa_layer_decode_step", "mqa_layer_workspace_bytes", "mqa_decode_local_step",
     "mqa_decode_append_step_host", "mqa_host_staging_bytes",
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.mqa_workspace_bytes.restype = sz
         L.mqa_plan_splits.argtypes = [I, I, I, I, I, I, ctypes.POINTER(I)]
         L.mqa_plan_splits.restype = I
+        L.mqa_plan_kernel_name.argtypes = [I, I, I, I, I, I, I]
+        L.mqa_plan_kernel_name.restype = ctypes.c_char_p
         L.mqa_status_string.argtypes = [I]
         L.mqa_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -104,6 +106,11 @@ def plan_splits(multi_query: bool, b: int, h: int, m_max: int, k: int = 128, v: 
     chunk = ctypes.c_int(0)
     n = lib().mqa_plan_splits(int(bool(multi_query)), b, h, m_max, k, v, ctypes.byref(chunk))
     return int(n), int(chunk.value)
+
+
+def plan_kernel_name(multi_query: bool, whole_step: bool, b: int, h: int, m_max: int, k: int = 128, v: int = 128) -> str:
+    """Name of the kernel that passes over the cache for these sizes (informational)."""
+    return lib().mqa_plan_kernel_name(int(bool(multi_query)), int(bool(whole_step)), b, h, m_max, k, v).decode()
 
 
 def alloc_workspace(b: int, h: int, m_max: int, device, k: int = 128, v: int = 128) -> torch.Tensor:

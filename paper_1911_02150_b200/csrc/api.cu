@@ -142,13 +142,26 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
     return h <= 32 ? plan_mma(b, h, m_max) : plan_simt(b, h, m_max);
 }
 
+// Every workspace begins with the control block of the single-launch step (kStreamCtrlBytes: see decode_umma.cuh),
+// whatever the plan: a workspace that serves several shapes then keeps one epoch for all of them, and the kernels of
+// the other plans never write over it.  The plan's own scratch follows.
 size_t plan_workspace_bytes(const Plan& p) {
     if (p.stream()) {
         const int slots = p.grid + p.b;
-        return stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) + stream_acc_bytes(slots, p.h) + stream_ctrl_bytes(p.b);
+        return kStreamCtrlBytes + stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) + stream_acc_bytes(slots, p.h);
     }
     if (p.n_splits <= 1) return 0;
-    return partial_ml_bytes(p.units, p.n_splits) + partial_acc_bytes(p.units, p.n_splits);
+    return kStreamCtrlBytes + partial_ml_bytes(p.units, p.n_splits) + partial_acc_bytes(p.units, p.n_splits);
+}
+
+// Fixed-split plans: (max, sum) pairs, then the accumulators, after the control block.
+float2* partials_ml(const void* workspace) {
+    return workspace ? reinterpret_cast<float2*>(static_cast<char*>(const_cast<void*>(workspace)) + kStreamCtrlBytes) : nullptr;
+}
+float* partials_acc(const Plan& p, const void* workspace) {
+    return workspace ? reinterpret_cast<float*>(static_cast<char*>(const_cast<void*>(workspace)) + kStreamCtrlBytes +
+                                                partial_ml_bytes(p.units, p.n_splits))
+                     : nullptr;
 }
 
 struct StreamWorkspace {
@@ -161,11 +174,11 @@ StreamWorkspace stream_workspace(const Plan& p, const void* workspace) {
     char* base = static_cast<char*>(const_cast<void*>(workspace));
     const int slots = p.grid + p.b;
     StreamWorkspace w;
+    w.ctrl = reinterpret_cast<unsigned long long*>(base);
+    base += kStreamCtrlBytes;
     w.span = reinterpret_cast<int2*>(base);
     w.ml = reinterpret_cast<float2*>(base + stream_span_bytes(p.b));
     w.acc = reinterpret_cast<float*>(base + stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h));
-    w.ctrl = reinterpret_cast<unsigned long long*>(base + stream_span_bytes(p.b) + stream_ml_bytes(slots, p.h) +
-                                                   stream_acc_bytes(slots, p.h));
     return w;
 }
 
@@ -377,10 +390,8 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     if (rc) return rc;
     if (p.kernel == Kernel::kUmma)
         return launch_umma_for<false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge_in_kernel);
-    float2* part_ml = reinterpret_cast<float2*>(workspace);
-    float* part_acc = workspace ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
-                                                           partial_ml_bytes(p.units, p.n_splits))
-                                : nullptr;
+    float2* part_ml = partials_ml(workspace);
+    float* part_acc = partials_acc(p, workspace);
     if (p.kernel == Kernel::kMma1)
         return launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, len_bias);
     if (p.kernel == Kernel::kMma2)
@@ -416,9 +427,8 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
         return launch_status();
     }
     if (p.n_splits <= 1) return MQA_OK;
-    const float2* part_ml = reinterpret_cast<const float2*>(workspace);
-    const float* part_acc = reinterpret_cast<const float*>(static_cast<const char*>(workspace) +
-                                                           partial_ml_bytes(p.units, p.n_splits));
+    const float2* part_ml = partials_ml(workspace);
+    const float* part_acc = partials_acc(p, workspace);
     // fused (the append-and-attend step of a sequence cut into fixed splits): the pass wrote a piece for every split,
     // the second pass does not look at lens and moves it on when asked to
     const int32_t* lens_read = fused ? nullptr : lens;
@@ -610,22 +620,30 @@ int mha_decode_step_combine(const int32_t* lens, float* o, const void* workspace
 // MQA_STEP_CHAINED.  flags: MQA_STEP_ADVANCE | MQA_STEP_CHAINED.
 constexpr int kEarlyNone = 0, kEarlyAfterProjection = 1, kEarlyChained = 2, kEarlyChainedWrongGuess = 3;
 constexpr int kGuessMaxPieces = 6, kGuessMinShareRows = 8 * kUmmaStageRows;
-static int append_step_impl(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
-                            int flags, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
-                            int h, int m_max, int k, int v, mqa_stream_t stream_, bool after_projection) {
+// Every check of mqa_decode_append_step that needs no launch: flags, pointers, sizes, the plan, the workspace.
+static int check_append_step(const void* q, const void* K, const void* V, const void* k_new, const void* v_new,
+                             const int32_t* lens, int flags, const float* o, const void* workspace, size_t workspace_bytes,
+                             const int32_t* status, int b, int h, int m_max, int k, int v) {
     if (flags & ~(MQA_STEP_ADVANCE | MQA_STEP_CHAINED | MQA_STEP_TEST_WRONG_GUESS)) return MQA_ERR_INVALID_ARG;
-    const int advance = flags & MQA_STEP_ADVANCE;
-    int early = after_projection ? kEarlyAfterProjection
-                : !(flags & MQA_STEP_CHAINED) ? kEarlyNone
-                : (flags & MQA_STEP_TEST_WRONG_GUESS) ? kEarlyChainedWrongGuess : kEarlyChained;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
     if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return MQA_ERR_INVALID_ARG;
     const Plan p = make_plan(true, b, h, m_max);
     if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
-    rc = check_workspace(p, workspace, workspace_bytes);
+    return check_workspace(p, workspace, workspace_bytes);
+}
+
+static int append_step_impl(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
+                            int flags, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
+                            int h, int m_max, int k, int v, mqa_stream_t stream_, bool after_projection) {
+    int rc = check_append_step(q, K, V, k_new, v_new, lens, flags, o, workspace, workspace_bytes, status, b, h, m_max, k, v);
     if (rc) return rc;
+    const int advance = flags & MQA_STEP_ADVANCE;
+    int early = after_projection ? kEarlyAfterProjection
+                : !(flags & MQA_STEP_CHAINED) ? kEarlyNone
+                : (flags & MQA_STEP_TEST_WRONG_GUESS) ? kEarlyChainedWrongGuess : kEarlyChained;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const Plan p = make_plan(true, b, h, m_max);
     if (p.kernel == Kernel::kUmma) {
         // copies started on a guess pay where the step is one launch over long shares (measured: 0.4-0.7 us gained with
         // up to 6 pieces per sequence, 0.3-2.5 us lost with more pieces, short shares or a second-pass kernel)
@@ -660,8 +678,8 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
     }
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits > 1) {
         // fixed splits: the CTA whose rows hold the new one writes it; the second pass moves lens on.  Two launches.
-        float2* part_ml = reinterpret_cast<float2*>(workspace);
-        float* part_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + partial_ml_bytes(p.units, p.n_splits));
+        float2* part_ml = partials_ml(workspace);
+        float* part_acc = partials_acc(p, workspace);
         rc = p.kernel == Kernel::kMma1
                  ? launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr)
                  : launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr);
@@ -724,6 +742,10 @@ int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, cons
     char* k_dev = q_dev + align256(q_bytes);
     char* v_dev = k_dev + align256(row_bytes);
     float* o_dev = reinterpret_cast<float*>(v_dev + align256(row_bytes));
+    // everything that can be refused is refused before the first copy is enqueued
+    const int bad = check_append_step(q_dev, K, V, k_dev, v_dev, lens, advance, o_dev, workspace, workspace_bytes, status, b, h,
+                                      m_max, k, v);
+    if (bad) return bad;
     // the step's inputs: one copy when the caller packed them back to back (256-byte aligned parts), else three
     const char* qh = static_cast<const char*>(q_host);
     const bool packed = static_cast<const char*>(k_new_host) == qh + align256(q_bytes) &&
@@ -824,6 +846,22 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
     const Plan p = make_plan(multi_query != 0, b, h, m_max);
     if (chunk_rows) *chunk_rows = p.chunk_rows;
     return p.n_splits;
+}
+
+const char* mqa_plan_kernel_name(int multi_query, int whole_step, int b, int h, int m_max, int k, int v) {
+    if (!dims_ok(b, h, m_max) || k != kHeadDim || v != kHeadDim) return "";
+    const Plan p = make_plan(multi_query != 0, b, h, m_max);
+    switch (p.kernel) {
+        case Kernel::kUmma: {
+            const bool guess = whole_step && p.merge_in_kernel && p.n_splits <= kGuessMaxPieces && p.chunk_rows >= kGuessMinShareRows;
+            if (h <= 16) return !whole_step ? "mqa_decode_stream_umma_kernel<16>" : guess ? "mqa_decode_stream_umma_kernel<16, fused, guess>" : "mqa_decode_stream_umma_kernel<16, fused>";
+            if (h <= 32) return !whole_step ? "mqa_decode_stream_umma_kernel<32>" : guess ? "mqa_decode_stream_umma_kernel<32, fused, guess>" : "mqa_decode_stream_umma_kernel<32, fused>";
+            return !whole_step ? "mqa_decode_stream_umma_kernel<64>" : guess ? "mqa_decode_stream_umma_kernel<64, fused, guess>" : "mqa_decode_stream_umma_kernel<64, fused>";
+        }
+        case Kernel::kMma1: return "mqa_decode_split_mma_kernel<1>";
+        case Kernel::kMma2: return "mqa_decode_split_mma_kernel<2>";
+        default: return "decode_split_simt_kernel";
+    }
 }
 
 const char* mqa_status_string(int code) {

@@ -680,12 +680,14 @@ __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ len
             atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
         prefix[s + 1] = L > 0 ? (L + kTileRows - 1) / kTileRows + PENALTY : 0;
         rows_of[s] = L | (appending && can_append ? kAppendBit : 0);
-        if (L == 0 && s % G == cta) {                      // the empty prefix gives zeros
-            for (int i = 0; i < h * kHeadDim; ++i) o[(size_t)s * h * kHeadDim + i] = 0.f;
-        }
     }
     if (threadIdx.x == 0) { prefix[0] = 0; plan_sm[3] = 0; }
     __syncthreads();
+    for (int s = cta; s < b; s += G) {                     // the empty prefix gives zeros: all threads, 16 bytes each
+        if ((rows_of[s] & (kAppendBit - 1)) != 0) continue;
+        float4* dst = reinterpret_cast<float4*>(o + (size_t)s * h * kHeadDim);
+        for (int i = threadIdx.x; i < h * (kHeadDim / 4); i += THREADS) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     if (warp == 0) {
         // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
         // also notes which sequence that is

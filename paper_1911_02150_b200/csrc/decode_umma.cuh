@@ -182,22 +182,24 @@ __host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool a_mn_major,
 
 // ---- control block of the single-launch step ---------------------------------------------------
 // When a control block is given, the CTA that is last to deliver a piece of a sequence merges the pieces
-// itself (no second-pass kernel), and one CTA advances lens at the end.  The block lives in the caller's
-// workspace, whose contents are arbitrary the first time, and nothing in it is ever reset: every launch
-// works under a new epoch E, read from the block by every CTA before anything in it is written, and a
-// word counts only if it carries E.
-//   ctrl[0] magic (the block has been used before), ctrl[1] epoch of the last launch
+// itself (no second-pass kernel), and one CTA advances lens at the end.  The block is the first
+// kStreamCtrlBytes of the caller's workspace -- the same place and size whatever the batch, the head count
+// and the grid, and no other kernel of the library writes there -- so every launch that uses a workspace
+// finds the epoch word of the launch before it, of whatever shape that was.  Its contents are arbitrary
+// the first time and nothing in it is ever reset: every launch works under a new epoch E = the epoch word
+// as found + 1 (44 bits), read by every CTA before anything in the block is written, and a word counts only
+// if it carries E.
+//   ctrl[1]            epoch of the last launch (whatever the memory held, the first time)
 //   ctrl[8 + c]        = E once CTA c has read the epoch and lens      ("started")
 //   ctrl[8 + 256 + s]  = E << 20 | pieces of sequence s delivered so far
 // The epoch is moved on by the first CTA that finds every CTA started (at least the CTA that started
 // last does: the store of its own mark, a fence.sc and then the reads).  Until then nobody leaves
-// the old epoch behind, so all CTAs of a launch agree on E.
-constexpr unsigned long long kCtrlMagic = 0x6d71615f6374726cull;
-constexpr unsigned long long kCtrlFirstEpoch = 0x9e3779b97f4ull;          // 44 bits
+// the old epoch behind, so all CTAs of a launch agree on E.  A launch whose waits ran out still moves the
+// epoch on (every CTA marks itself before its loop), so the block needs no repair afterwards.
 constexpr unsigned long long kCtrlEpochMask = (1ull << 44) - 1;
 constexpr int kCtrlCountBits = 20;
 constexpr int kCtrlStarted = 8, kCtrlCounters = 8 + 256;
-__host__ __device__ inline size_t stream_ctrl_bytes(int b) { return (((size_t)(kCtrlCounters + b) * 8) + 255) & ~(size_t)255; }
+constexpr size_t kStreamCtrlBytes = (((size_t)(kCtrlCounters + kStreamMaxSeqs) * 8) + 255) & ~(size_t)255;
 
 // One more piece of a sequence delivered: returns how many were delivered before it in this launch.
 __device__ __forceinline__ unsigned int ctrl_arrive(unsigned long long* word, unsigned long long E) {
@@ -514,7 +516,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     }
     if (ctrl && threadIdx.x == 0) {
         const unsigned long long was = __ldcg(ctrl + 1);
-        unsigned long long E = __ldcg(ctrl) == kCtrlMagic ? ((was + 1) & kCtrlEpochMask) : kCtrlFirstEpoch;
+        unsigned long long E = (was + 1) & kCtrlEpochMask;
         if (E == 0) E = 1;
         epoch_sm[0] = E;
         epoch_sm[1] = was;
@@ -569,7 +571,6 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             if (all && lane == 0) won = atomicCAS(ctrl + 1, epoch_sm[1], E) == epoch_sm[1];
             won = __shfl_sync(0xffffffffu, won, 0);
             if (won) {
-                if (lane == 0) __stcg(ctrl, kCtrlMagic);
                 if (lens_advance)
                     for (int s = lane; s < b; s += 32)
                         if (rows_of[s] & kAppendBit) lens_advance[s] = rows_of[s] & (kAppendBit - 1);

@@ -43,6 +43,19 @@ def oracle_step(variant, q, K, V, lens_np, idx=None):
     return fn(wl.bits(q), wl.bits(K), wl.bits(V), lens_np.astype(np.int32))
 
 
+def check_against_oracle(variant, q, K, V, lens_np, o, what, idx=None, chunk_bytes=1 << 30):
+    """Every sequence (or those in idx) against the oracle, read back a slice of sequences at a time so that the host
+    never holds more than about chunk_bytes of one cache tensor (the largest caches here are tens of GiB)."""
+    b = q.shape[0]
+    seqs = list(range(b)) if idx is None else list(idx)
+    per_seq = K[0].numel() * 2
+    step = max(1, chunk_bytes // per_seq)
+    for at in range(0, len(seqs), step):
+        part = seqs[at:at + step]
+        ref = oracle_step(variant, q, K, V, lens_np, part)
+        check_close(o[torch.as_tensor(part, device=o.device)].cpu().numpy(), ref, f"{what} sequences {part[0]}..{part[-1]}")
+
+
 def gpu_step(variant, q, K, V, lens_t, expect_status=0):
     b, h, _ = q.shape
     o = torch.full((b, h, V.shape[-1]), float("nan"), dtype=torch.float32, device=q.device)
@@ -63,13 +76,7 @@ def run_case(variant, b, h, m_max, lens_np, seed=0, sample=None):
     wl.poison_tail(inp["V"], lens_np)
     lens_t = torch.from_numpy(lens_np).to(DEV)
     o = gpu_step(variant, inp["q"], inp["K"], inp["V"], lens_t)
-    got = o.cpu().numpy()
-    if sample is None:
-        ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], lens_np)
-    else:
-        ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], lens_np, sample)
-        got = got[sample]
-    check_close(got, ref, f"{variant} b={b} h={h} m_max={m_max}")
+    check_against_oracle(variant, inp["q"], inp["K"], inp["V"], lens_np, o, f"{variant} b={b} h={h} m_max={m_max}", sample)
     return inp, o
 
 
@@ -158,11 +165,8 @@ def test_long_context_configuration(variant):
         same = (Kbefore.view(torch.int16) == inp["K"].view(torch.int16)).all(dim=-1)
         assert bool(same[:, : w.m_max - 1].all())
         assert torch.equal(inp["K"][:, w.m_max - 1].view(torch.int16), inp["k_new"].view(torch.int16))
-    sample = None if variant == "mqa" else [0, 7, 31]  # 3 of 32 sequences (all heads) for the 4 GiB cache
-    lens_np = lens0 + 1
-    ref = oracle_step(variant, inp["q"], inp["K"], inp["V"], lens_np, sample)
-    got = o.cpu().numpy() if sample is None else o.cpu().numpy()[sample]
-    check_close(got, ref, f"long_context {variant}")
+    # every sequence and head, also of the 4 GiB multi-head cache
+    check_against_oracle(variant, inp["q"], inp["K"], inp["V"], lens0 + 1, o, f"long_context {variant}")
 
 
 @pytest.mark.parametrize("variant", ["mqa", "mha"])
@@ -171,8 +175,7 @@ def test_ragged_configuration(variant):
     w = wl.WORKLOADS["ragged"]
     lens = wl.ragged_lens(w.b, w.m_max, seed=0)
     assert lens.min() >= 1 and lens.max() <= w.m_max
-    sample = None if variant == "mqa" else list(range(0, 256, 16))
-    run_case(variant, w.b, w.h, w.m_max, lens, seed=0, sample=sample)
+    run_case(variant, w.b, w.h, w.m_max, lens, seed=0)
 
 
 @pytest.mark.parametrize("variant", ["mqa", "mha"])
@@ -213,27 +216,25 @@ def test_paper_incremental_decoding(variant):
         check_close(outs[t].cpu().numpy(), ref, f"{variant} step {t + 1}")
 
 
-SWEEP = [("mqa", 1, 512), ("mha", 1, 512), ("mqa", 8, 4096), ("mha", 8, 4096), ("mqa", 64, 32768),
-         ("mha", 8, 32768), ("mqa", 256, 32768), ("mha", 64, 4096)]
-
-
-@pytest.mark.parametrize("variant,b,m", SWEEP)
+@pytest.mark.parametrize("variant", ["mqa", "mha"])
+@pytest.mark.parametrize("m", wl.SWEEP_M)
+@pytest.mark.parametrize("b", wl.SWEEP_B)
 def test_sweep_points(variant, b, m):
-    """h=16 sweep points, full-length caches; large points are checked on sampled sequences."""
-    rng = np.random.default_rng(b * 7 + m)
-    n_s = 8 if m < 32768 else 3
-    sample = None if b <= n_s else sorted({0, b - 1, *rng.integers(0, b, size=n_s - 2).tolist()})
-    run_case(variant, b, 16, m, np.full(b, m, np.int32), seed=m + b, sample=sample)
-
-
-def test_largest_multihead_sweep_point_if_it_fits():
-    """b=256, m=32768, h=16 in multi-head form is a 64 GiB cache: 2^35 elements per tensor pair,
-    beyond 32-bit indexing.  Checked on three sampled sequences."""
+    """All 24 points of the bandwidth sweep (h = 16, full-length caches, both variants).  Every sequence is compared
+    with the oracle; only the two multi-head caches of 16 GiB and more (b=64 and b=256 at 32768 rows: the latter is
+    2^35 elements per tensor pair, beyond 32-bit indexing) are compared on the first, the last and six seeded
+    sequences, all heads."""
+    h = 16
+    cache = 2 * b * (h if variant == "mha" else 1) * m * 256
     free, _ = torch.cuda.mem_get_info()
-    if free < 80 * 2 ** 30:
-        pytest.skip("less than 80 GiB free on this GPU")
-    b, h, m = 256, 16, 32768
-    run_case("mha", b, h, m, np.full(b, m, np.int32), seed=5, sample=[0, 129, 255])
+    if cache + 8 * 2 ** 30 > free:
+        pytest.skip(f"a cache of {cache >> 30} GiB does not fit this GPU")
+    sample = None
+    if cache >= 16 * 2 ** 30:
+        rng = np.random.default_rng(b * 7 + m)
+        sample = sorted({0, b - 1, *rng.integers(0, b, size=6).tolist()})
+    run_case(variant, b, h, m, np.full(b, m, np.int32), seed=m + b, sample=sample)
+    torch.cuda.empty_cache()
 
 
 # ----------------------------------------------------------------------------- properties

@@ -57,6 +57,33 @@ def test_workspace_contents_do_not_matter():
         ws[: nbytes // 2].fill_(0xFF)                         # and a partly overwritten workspace
 
 
+@pytest.mark.parametrize("noalloc", [False, True])
+def test_two_shapes_whose_counters_overlap_share_one_epoch(noalloc):
+    """Batches of 601 and 602 sequences (h = 8, 1024 rows) take the same grid, cut most sequences in two and count the
+    delivered pieces in the same words of the control block.  The second shape's first call must not take the first
+    shape's counts for its own: the epoch is one per workspace, not one per shape.  Also through the entry point that
+    brings its own scratch."""
+    h, m_max = 8, 1024
+    sizes = (601, 602, 601)
+    ws = None if noalloc else mqa.alloc_workspace(max(sizes), h, m_max, DEV)
+    for rnd, b in enumerate(sizes):
+        assert mqa.append_step_launches(b, h, m_max) == 1
+        inp = wl.make_inputs(b, h, m_max, "mqa", seed=50 + rnd, device=DEV)
+        lens = np.full(b, m_max, np.int32)
+        lens[::7] = np.random.default_rng(rnd).integers(1, m_max, size=len(lens[::7]))
+        wl.poison_tail(inp["K"], lens); wl.poison_tail(inp["V"], lens)
+        o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        if noalloc:
+            mqa.mqa_decode_step_noalloc(inp["q"], inp["K"], inp["V"], torch.from_numpy(lens).to(DEV), o, status)
+        else:
+            mqa.mqa_decode_step(inp["q"], inp["K"], inp["V"], torch.from_numpy(lens).to(DEV), o, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref = oracle.mqa_decode_step(wl.bits(inp["q"]), wl.bits(inp["K"]), wl.bits(inp["V"]), lens)
+        check_close(o.cpu().numpy(), ref, f"call {rnd}: b={b}")
+
+
 def test_many_calls_on_one_workspace_are_bit_identical():
     b, h, m_max = 48, 32, 3000
     inp = wl.make_inputs(b, h, m_max, "mqa", seed=11, device=DEV)

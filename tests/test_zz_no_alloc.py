@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_1911_02150_b200 as mqa
 from paper_1911_02150_b200 import binding, workloads as wl
 from paper_1911_02150_b200.build import build_library
@@ -18,8 +19,9 @@ ABS_TOL = 4e-3          # the tolerances of tests/test_parity_gpu.py
 REL_TOL = 1e-2
 
 
-def _close(a: torch.Tensor, ref: torch.Tensor):
-    a, ref = a.double().cpu().numpy(), ref.double().cpu().numpy()
+def _close(a: torch.Tensor, ref):
+    a = a.double().cpu().numpy()
+    ref = ref if isinstance(ref, np.ndarray) else ref.double().cpu().numpy()
     err = np.abs(a - ref)
     assert np.all(np.isfinite(a))
     assert err.max() <= ABS_TOL
@@ -51,6 +53,8 @@ def test_noalloc_matches_the_workspace_entry_point_on_two_calls_in_a_row():
         _close(got, want)
         # same kernels, same plan: in fact the very same bits
         assert torch.equal(got.view(torch.int32), want.view(torch.int32))
+        # and, directly, what the paper's step defines (the fp64 oracle on the same bits)
+        _close(got, oracle.mqa_decode_step(wl.bits(inp["q"]), wl.bits(inp["K"]), wl.bits(inp["V"]), lens_np))
 
 
 def test_noalloc_refuses_sizes_beyond_its_scratch_without_launching():
