@@ -187,19 +187,30 @@ StreamWorkspace stream_workspace(const Plan& p, const void* workspace) {
 // before it touches memory an earlier kernel may write, so the only effect is that launch
 // latency and set-up overlap the tail of the previous kernel.
 template <typename... Params, typename... Args>
-cudaError_t launch_dependent(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem,
-                             cudaStream_t stream, Args... args) {
+cudaError_t launch_dependent_clusters(unsigned cluster, void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem,
+                                      cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (cluster > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
+template <typename... Params, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem,
+                             cudaStream_t stream, Args... args) {
+    return launch_dependent_clusters(1u, kernel, grid, block, smem, stream, args...);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -352,9 +363,14 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     const StreamWorkspace w = stream_workspace(p, workspace);
     // a cache that cannot stay in L2 from one step to the next is streamed through it with the evict-first policy
     const int read_once = (size_t)b * m_max * 2 * kRowBytes > kL2KeepBytes ? 1 : 0;
-    launch_dependent(kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub, map_v_sub,
-                     map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa,
-                     merge ? w.ctrl : nullptr, lens_advance, early, read_once);
+    // The single-launch step of a batch that divides the grid runs as clusters of grid / b CTAs (2 to 8, the
+    // portable sizes): with sequences of equal length a cluster then holds exactly one sequence's pieces and merges
+    // them through its shared memory (the kernel decides from lens; otherwise the clusters change nothing).
+    unsigned cluster = 1;
+    if (merge && p.grid % b == 0 && p.grid / b >= 2 && p.grid / b <= 8) cluster = (unsigned)(p.grid / b);
+    launch_dependent_clusters(cluster, kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub,
+                              map_v_sub, map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa,
+                              merge ? w.ctrl : nullptr, lens_advance, early, read_once);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -560,6 +576,10 @@ int launch_projection_out(const void* P_o, const float* o, float* y, int32_t* st
 using namespace mqa;
 
 extern "C" {
+#ifdef MQA_DEBUG_TS
+void mqa_debug_ts(unsigned long long* t) { cudaMemcpyFromSymbol(t, mqa::g_ts, sizeof(mqa::g_ts)); }
+void mqa_debug_st(unsigned long long* t) { cudaMemcpyFromSymbol(t, mqa::g_st, sizeof(mqa::g_st)); }
+#endif
 
 int kv_cache_append(void* K, void* V, const void* k_new, const void* v_new, int32_t* lens, int advance,
                     int32_t* status, int b, int kv_heads, int m_max, int k, int v, mqa_stream_t stream) {

@@ -99,6 +99,10 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
 }
+// Ask for a box of a tensor to be brought into L2 (nothing lands in shared memory, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
 // Policy for data that is read once (read_once): its lines are the first to go, so that a pass over a cache larger
 // than L2 does not push out what every launch needs again (q, lens, the workspace, the kernel's own code and
 // parameters).  Otherwise the ordinary policy: a cache that fits in L2 is found there by the next step.
@@ -136,6 +140,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float x_lo, float x_hi) {
 }
 __device__ __forceinline__ void named_barrier(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// Counts towards a named barrier of `threads` threads without waiting for it.
+__device__ __forceinline__ void named_barrier_arrive(int id, int threads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // The append-and-attend step: the kernel that owns a sequence's last tile also writes the new token's key
@@ -662,16 +670,28 @@ constexpr int kAppendBit = 1 << 30;                    // in rows_of[]: this ste
 // prefix[s] = position on the line of sequence s's block (PENALTY virtual tiles, then its 32-row
 // tiles; no block for an empty prefix, whose output is zeroed here), rows_of[s] = rows to attend over
 // (kAppendBit set when this step appends one).  Returns T = length of the line, [t_begin, t_end) = this
-// CTA's share, s_first = the sequence that holds position t_begin.  plan_sm: 4 ints of shared memory.
-struct SharePlan { int T, t_begin, t_end, s_first; };
+// CTA's share, s_first = the sequence that holds position t_begin, equal = every sequence has the same, non-zero
+// number of tiles (then G shares of a batch that divides G fall on sequence boundaries).  plan_sm: 8 ints of
+// shared memory.
+struct SharePlan { int T, t_begin, t_end, s_first; bool equal; };
 
+// solo_warp: a warp (the one that issues the copies) that takes no part in building the tables, so that the other
+// warps do not wait for it: it must have arrived on barrier kPlanBarInit (named_barrier_arrive over THREADS) once what it
+// initialises in shared memory is in place, and it returns from here when the tables are complete.  -1: none.
+constexpr int kPlanBarInit = 3, kPlanBarScan = 4, kPlanBarDone = 5;
 template <bool FUSED, int THREADS, int PENALTY>
 __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ lens, float* __restrict__ o,
                                                  int32_t* __restrict__ status, int b, int h, int m_max, bool appending,
-                                                 unsigned long long magic, int* prefix, int* rows_of, int* plan_sm) {
+                                                 unsigned long long magic, int* prefix, int* rows_of, int* plan_sm,
+                                                 int solo_warp = -1) {
     const int cta = blockIdx.x, G = gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int s = threadIdx.x; s < b; s += THREADS) {
+    const int planners = solo_warp >= 0 ? THREADS - 32 : THREADS;
+    const int tix = (solo_warp >= 0 && warp > solo_warp) ? (int)threadIdx.x - 32 : (int)threadIdx.x;
+    if (warp == solo_warp) {
+        named_barrier(kPlanBarDone, THREADS);
+    } else {
+    for (int s = tix; s < b; s += planners) {
         const int raw = read_len<FUSED>(lens, s);
         clamp_len(raw, m_max, cta == 0 ? status : nullptr);
         bool can_append;
@@ -682,11 +702,11 @@ __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ len
         rows_of[s] = L | (appending && can_append ? kAppendBit : 0);
     }
     if (threadIdx.x == 0) { prefix[0] = 0; plan_sm[3] = 0; }
-    __syncthreads();
+    if (solo_warp >= 0) named_barrier(kPlanBarInit, THREADS); else __syncthreads();
     for (int s = cta; s < b; s += G) {                     // the empty prefix gives zeros: all threads, 16 bytes each
         if ((rows_of[s] & (kAppendBit - 1)) != 0) continue;
         float4* dst = reinterpret_cast<float4*>(o + (size_t)s * h * kHeadDim);
-        for (int i = threadIdx.x; i < h * (kHeadDim / 4); i += THREADS) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = tix; i < h * (kHeadDim / 4); i += planners) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (warp == 0) {
         // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
@@ -703,18 +723,28 @@ __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ len
         }
         const int T = __shfl_sync(0xffffffffu, incl, 31);
         const int tb = share_begin(cta, T, magic), te = share_begin(cta + 1, T, magic);
-        if (lane == 0) { plan_sm[0] = T; plan_sm[1] = tb; plan_sm[2] = te; }
+        const int first_count = prefix[1];
         int run = incl - sum;
+        bool same = true;
         for (int s = lo; s <= hi; ++s) {
             const int before = run;
+            same = same && prefix[s] == first_count;
             run += prefix[s];
             prefix[s] = run;
             if (before <= tb && tb < run) plan_sm[3] = s - 1;     // sequence s-1 occupies [before, run)
         }
+        same = __all_sync(0xffffffffu, same) && first_count > 0;
+        if (lane == 0) { plan_sm[0] = T; plan_sm[1] = tb; plan_sm[2] = te; plan_sm[4] = same ? 1 : 0; }
     }
-    __syncthreads();
+    if (solo_warp >= 0) {
+        named_barrier(kPlanBarScan, planners);
+        named_barrier_arrive(kPlanBarDone, THREADS);
+    } else {
+        __syncthreads();
+    }
+    }
     SharePlan p;
-    p.T = plan_sm[0]; p.t_begin = plan_sm[1]; p.t_end = plan_sm[2]; p.s_first = plan_sm[3];
+    p.T = plan_sm[0]; p.t_begin = plan_sm[1]; p.t_end = plan_sm[2]; p.s_first = plan_sm[3]; p.equal = plan_sm[4] != 0;
     return p;
 }
 

@@ -39,6 +39,17 @@
 
 namespace mqa {
 
+#ifdef MQA_DEBUG_TS
+__device__ unsigned long long g_ts[256 * 32];
+__device__ __forceinline__ unsigned long long dbg_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TS(k) do { g_ts[blockIdx.x * 32 + (k)] = dbg_ns(); } while (0)
+__device__ unsigned long long g_st[64 * 8];
+#define ST(j, k) do { if (blockIdx.x == MQA_DEBUG_CTA && (j) < 64) g_st[(j) * 8 + (k)] = dbg_ns(); } while (0)
+#else
+#define TS(k) do { } while (0)
+#define ST(j, k) do { } while (0)
+#endif
+
 constexpr int kUmmaStageRows = 128;                              // cache rows per stage
 constexpr int kUmmaHalfBytes = kUmmaStageRows * 128;             // 16 KiB: one 64-column box of 128 rows
 constexpr int kUmmaSlotBytes = 2 * kUmmaHalfBytes;               // 32 KiB: the K (or the V) rows of a stage
@@ -217,6 +228,49 @@ __device__ __forceinline__ unsigned int ctrl_arrive(unsigned long long* word, un
     return 0xffffffffu;                                    // never seen; the caller then does not merge
 }
 
+// ---- thread-block cluster helpers (the pieces of a sequence, and the head groups of the output projection, are summed
+// through distributed shared memory)
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
+    return n;
+}
+// every thread of every CTA of the cluster, the same number of times on every path: what a CTA wrote to its shared
+// memory before is visible to the others after
+__device__ __forceinline__ void cluster_sync() {
+    __syncwarp();                    // the aligned forms want the whole warp at the same instruction
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+// The address, in the cluster's shared window, of this CTA's shared address `local` in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    return remote;
+}
+__device__ __forceinline__ float4 cluster_ld_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 cluster_ld_f2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+
 // Barrier over `threads` threads that also ORs a predicate over them.
 __device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred) {
     uint32_t out;
@@ -349,13 +403,16 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     const uint32_t s_ready = q_empty + 16, s_free = s_ready + 16;
     const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;   // o_free: one per O^T buffer
     const uint32_t go = o_free + 16;                        // the share's first segment is settled (see early below)
-    __shared__ int timed_out, issued, plan_sm[4], merge_sm[8];   // merge_sm: count, then (sequence, first CTA, last CTA) x 2
+    __shared__ int timed_out, issued, plan_sm[8], merge_sm[8];   // merge_sm: count, then (sequence, first CTA, last CTA) x 2
     __shared__ unsigned long long epoch_sm[2];              // this launch's epoch; the epoch word as found
     __shared__ uint32_t tmem_base_slot;
+    __shared__ int waited_sm;                                // 1 once a warp of this CTA has come back from the wait on the kernel before
 
     // set up by the thread that issues the copies: it may start some before the first CTA-wide barrier, and
     // program order is what puts the initialisation before them; every other thread first passes that barrier
     if (warp == kUmmaProducerWarp && lane == 0) {
+        if (GUESS) asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_addr(&waited_sm)), "r"(0) : "memory");
+        TS(0);
         prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); prefetch_tensormap(&map_k_sub);
         prefetch_tensormap(&map_v_sub); prefetch_tensormap(&map_q);
         timed_out = 0;
@@ -372,7 +429,11 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         mbar_init(go, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        TS(10);
     }
+    // what the producer thread set up is in place: the other warps pass this barrier inside stream_plan, before
+    // they touch any of it, and do not wait for this warp again until the tables are built
+    if (warp == kUmmaProducerWarp) { __syncwarp(); named_barrier_arrive(kPlanBarInit, kUmmaThreads); }
     if (warp == kUmmaSWarp) {                               // one warp owns the TMEM allocation
         tmem_alloc(smem_addr(&tmem_base_slot), Cfg::kTmemCols);
         tmem_relinquish();
@@ -416,9 +477,12 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             if (j >= n_slots) p_ok = p_ok && mbar_wait((kv ? v_empty : k_empty) + slot * 8, ((j / n_slots) - 1) & 1);
             if (!p_ok) return;
             const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes;
+            if (j < 2) TS(16 + j * 6 + kv * 3);
             mbar_expect_tx(full, nsub * 2 * kBoxBytes);
+            if (j < 2) TS(16 + j * 6 + kv * 3 + 1);
             if (nsub == kSubs) {
                 tma_load_2d_hint(dst, kv ? &map_v : &map_k, 0, y, full, stream_policy);
+                if (j < 2) TS(16 + j * 6 + kv * 3 + 2);
                 tma_load_2d_hint(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full, stream_policy);
             } else {
                 for (int i = 0; i < nsub; ++i) {
@@ -428,6 +492,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 }
             }
             issued = 2 * j + kv + 1;                        // copies started: K of stage j, then V of stage j
+            if (kv == 0) ST(j, 7);
         }
     };
 
@@ -451,21 +516,34 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         Segment g0 = {};
         int r0 = 0;
         bool have = false, q_started = false;
-        const int passes = early >= 1 ? 2 : 1;
+        // A CTA that starts only when the kernel before has already completed (its SM was that kernel's last to become
+        // free) gains nothing from a guess: by then a warp that went straight to the wait has come back and said so
+        // (waited_sm, zeroed by this thread first, so that a 1 can only be that warp's), lens as it reads now is final,
+        // and one pass does.
+        int late = 0;
+        if (GUESS && early >= 2) {
+            if (lane == 0) asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(late) : "r"(smem_addr(&waited_sm)) : "memory");
+            late = __shfl_sync(0xffffffffu, late, 0);
+        }
+        const int passes = (early >= 1 && !late) ? 2 : 1;
         for (int pass = 0; pass < passes; ++pass) {
             const bool before = pass + 1 < passes;          // this pass runs ahead of the wait
             if (!before) {
+                if (lane == 0) TS(11);
                 grid_dependency_wait();                     // q, the new row, lens: all there now
                 grid_launch_dependents();
+                if (lane == 0) TS(1);
                 if (GUESS && early >= 2 && have) {                   // q of the guessed sequence, while the guess is checked
                     if (lane == 0) issue_q(g0.s, 0);
                     q_started = true;
                 }
+                if (lane == 0) TS(12);
             }
             if (before || early != 1) {                     // (early == 1: lens cannot have moved)
                 Segment g = {};
                 int r = 0;
                 const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r);
+                if (before && lane == 0) TS(8);
                 if (GUESS && before && early == 3) g.lo += kSubs;    // for tests: a guess that is one stage off
                 if (!before && GUESS && early >= 2) {
                     if (have && !(found && g.s == g0.s && g.lo == g0.lo && g.lo + pre_issued * kSubs <= g.hi)) {
@@ -485,6 +563,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         q_started = false;
                     }
                     if (lane == 0) mbar_arrive(go);
+                    if (lane == 0) TS(13);
                 }
                 have = found;
                 g0 = g;
@@ -513,8 +592,10 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     } else if (early != 1) {
         grid_dependency_wait();      // lens and the newest cache row may come from the kernel before
         grid_launch_dependents();
+        if (GUESS && threadIdx.x == kUmmaSWarp * 32)
+            asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_addr(&waited_sm)), "r"(1) : "memory");
     }
-    if (ctrl && threadIdx.x == 0) {
+    if (ctrl && threadIdx.x == kUmmaPvWarp * 32) {          // (a thread with nothing else to do at this point)
         const unsigned long long was = __ldcg(ctrl + 1);
         unsigned long long E = (was + 1) & kCtrlEpochMask;
         if (E == 0) E = 1;
@@ -524,9 +605,18 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 
     tc_fence_before();
     const SharePlan plan = stream_plan<FUSED, kUmmaThreads, kUmmaBoundaryPenalty>(lens, o, status, b, h, m_max, appending, magic, prefix,
-                                                            rows_of, plan_sm);
+                                                            rows_of, plan_sm, kUmmaProducerWarp);
     const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
     tc_fence_after();
+    // The launch is made of clusters of C CTAs when the batch divides the grid (C = G / b).  With sequences of equal
+    // tile counts the C CTAs of cluster r then hold exactly the pieces of sequence r, one piece each: they leave them
+    // in their own shared memory and merge them through the cluster's shared window (every CTA a part of the heads),
+    // with no partial result, fence or counter in global memory.  Decided here, by every CTA alike, from lens.
+    const uint32_t C = cluster_size();
+    const bool via_cluster = ctrl != nullptr && C > 1 && plan.equal && (long long)C * b == G;
+    float* piece_acc = reinterpret_cast<float*>(ring);                        // [h][128] in the first K slot (free by then)
+    float2* piece_ml = reinterpret_cast<float2*>(ring + kUmmaSlotBytes);      // [h] (reference maximum, sum) in the second
+    bool piece_left = false;                                // (softmax warps) this CTA has left a piece there
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_o = tmem_base + 2 * HP;             // S^T buffers at columns 0 and HP, two O^T buffers after them
 
@@ -581,16 +671,22 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         if (lane == 0 && t_begin < t_end) {
             constexpr uint32_t kIdescS = umma_idesc(128, HP, false, false);
             bool ok = !(GUESS && early >= 2) || mbar_wait(go, 0);
+            TS(14);
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; walk.next(g); ++seg) {
                 const int qi = seg % NQ;
                 if (ok) ok = mbar_wait(q_full + qi * 8, (seg / NQ) & 1);
+                if (seg == 0) TS(15);
                 for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
                     const int slot = j % NK, sb = j & 1;
                     if (ok) ok = mbar_wait(k_full + slot * 8, (j / NK) & 1);
+                    if (j == 0) TS(2);
+                    TS(3);
+                    ST(j, 0);
                     if (ok && j >= 2) ok = mbar_wait(s_free + sb * 8, ((j >> 1) - 1) & 1);
+                    ST(j, 1);
                     tc_fence_after();
                     if (ok) {
                         const uint32_t k_s = k_ring + slot * kUmmaSlotBytes;
@@ -624,7 +720,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     // the weights first: they exist only once q has arrived, and before that a slot's barrier may
                     // still be on its way back from copies started on a guess (see early above)
                     if (ok) ok = mbar_wait(p_ready + pb * 8, (j >> 1) & 1);
+                    ST(j, 5);
                     if (ok) ok = mbar_wait(v_full + slot * 8, (j / NV) & 1);
+                    ST(j, 6);
                     // segments alternate between the two O^T buffers; the segment before the last has read this one out
                     if (ok && u == g.lo && seg >= 2) ok = mbar_wait(o_free + (seg & 1) * 8, ((seg >> 1) - 1) & 1);
                     tc_fence_after();
@@ -697,7 +795,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 __syncwarp();
                 if (lane == 0) mbar_arrive(o_free + pend_par * 8);   // this O^T buffer may be overwritten
                 pend = false;
-                if (ctrl && !pend_whole) {
+                if (ctrl && !pend_whole && !via_cluster) {
                     // ---- single-launch step: the piece is delivered; the CTA that delivers a sequence's
                     // last piece merges them all into o (pieces in CTA order whoever merges: deterministic)
                     const int s = pend_s;
@@ -742,6 +840,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     const int valid = min(fetched, L - u * kTileRows);
                     const bool row_ok = t < valid;
                     if (ok) ok = mbar_wait(s_ready + sb * 8, (j >> 1) & 1);
+                    if (tid == 0) ST(j, 2);
                     tc_fence_after();
                     uint32_t xr[HH];
 #pragma unroll
@@ -822,6 +921,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     }
                     // this P^T tile was last read by the product of stage j-2 (of stage j-1 when that stage or
                     // this one has hi and lo parts, which take both tiles)
+                    if (tid == 0) ST(j, 3);
                     if (j >= 2 && ok) ok = mbar_wait(pv_done + pb * 8, ((j >> 1) - 1) & 1);
                     if ((hilo || prev_hilo) && j >= 1 && ok) ok = mbar_wait(pv_done + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
                     prev_hilo = hilo;
@@ -867,6 +967,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P^T (and cleared V) visible to the tensor core
                     __syncwarp();
                     if (lane == 0) mbar_arrive(p_ready + pb * 8);
+                    if (tid == 0) ST(j, 4);
                     // the segment before this one is read out of its own O^T buffer now, after this
                     // segment's first stage is on its way (its last product has long finished)
                     if (pend) read_out();
@@ -888,20 +989,26 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 #pragma unroll
                     for (int w = 0; w < 4; ++w) tot += red_l[w * HP + tid];
                     inv_sm[par * HP + tid] = whole ? 1.f / tot : 1.f;
-                    if (!whole && tid < h) part_ml[slot * h + tid] = make_float2(m_sm[tid], tot);
+                    if (!whole && tid < h) {
+                        if (via_cluster) piece_ml[tid] = make_float2(m_sm[tid], tot);
+                        else part_ml[slot * h + tid] = make_float2(m_sm[tid], tot);
+                    }
                 }
+                piece_left = true;
                 pend = true;
-                pend_dst = (whole ? o + (size_t)s * h * kHeadDim : part_acc + slot * h * kHeadDim) + t;
+                pend_dst = (whole ? o + (size_t)s * h * kHeadDim : via_cluster ? piece_acc : part_acc + slot * h * kHeadDim) + t;
                 pend_par = par;
                 pend_j = j - 1;
                 pend_s = s;
                 pend_whole = whole;
             }
+            if (tid == 0) TS(4);
             if (pend) {
                 named_barrier(2, kUmmaSoftmaxThreads);      // the last segment's 1/sum values are in shared memory
                 read_out();
             }
-            if (ctrl) {
+            if (tid == 0) TS(5);
+            if (ctrl && !via_cluster) {
                 // sequences whose last piece this CTA delivered (a share has at most two cut segments)
                 named_barrier(2, kUmmaSoftmaxThreads);
                 const int n_merge = merge_sm[0];
@@ -913,6 +1020,54 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         }
     }
 
+    if (via_cluster) {
+        // a CTA whose share holds none of the sequence's rows (short sequences: nothing but the virtual tiles in
+        // front of them) leaves an empty piece
+        if (warp < kUmmaSoftmaxWarps && !piece_left && threadIdx.x < h) piece_ml[threadIdx.x] = make_float2(-INFINITY, 0.f);
+        // every thread of the cluster: the C pieces lie in their CTAs' shared memory
+        cluster_sync();
+        if (threadIdx.x == 0) TS(6);
+        if (warp < kUmmaSoftmaxWarps) {
+            // CTA of rank r merges the heads [r * per, (r + 1) * per) of its sequence, pieces in rank (= row) order:
+            // a thread takes 16 bytes of a head's 128 outputs
+            const uint32_t rank = cluster_cta_rank();
+            const int per = (h + (int)C - 1) / (int)C;
+            const int s = cta / (int)C;
+            const int tid = threadIdx.x;
+            const uint32_t acc_s = smem_addr(piece_acc), ml_s = smem_addr(piece_ml);
+            for (int item = tid; item < per * (kHeadDim / 4); item += kUmmaSoftmaxThreads) {
+                const int head = (int)rank * per + (item >> 5), c4 = item & 31;
+                if (head >= h) break;
+                float top = -INFINITY;
+                float2 ml[8];
+                float4 a[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    ml[c] = make_float2(-INFINITY, 0.f);
+                    a[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (c < (int)C) {
+                        ml[c] = cluster_ld_f2(cluster_map(ml_s + head * 8, c));
+                        a[c] = cluster_ld_f4(cluster_map(acc_s + (head * kHeadDim + c4 * 4) * 4, c));
+                    }
+                    top = fmaxf(top, ml[c].x);
+                }
+                float den = 0.f;
+                float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float w = ml[c].x == -INFINITY ? 0.f : fast_exp2(ml[c].x - top);
+                    den = fmaf(w, ml[c].y, den);
+                    num.x = fmaf(w, a[c].x, num.x); num.y = fmaf(w, a[c].y, num.y);
+                    num.z = fmaf(w, a[c].z, num.z); num.w = fmaf(w, a[c].w, num.w);
+                }
+                const float inv = 1.f / den;
+                *reinterpret_cast<float4*>(o + ((size_t)s * h + head) * kHeadDim + c4 * 4) =
+                    make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+            }
+        }
+        if (threadIdx.x == 0) TS(7);
+        cluster_sync();                                 // nobody leaves while its shared memory is being read
+    }
     tc_fence_before();
     __syncthreads();
     if (timed_out && threadIdx.x == 0) {
@@ -927,6 +1082,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         tc_fence_after();
         tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
+    if (threadIdx.x == 0) TS(9);
 }
 
 }  // namespace mqa

@@ -172,31 +172,6 @@ project_in_kernel(const __grid_constant__ CUtensorMap map_pq, const __grid_const
     if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem, Cfg::kTmemCols); }
 }
 
-// ---- thread-block cluster helpers (the output projection sums its head groups through distributed shared memory)
-__device__ __forceinline__ uint32_t cluster_cta_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t cluster_size() {
-    uint32_t n;
-    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
-    return n;
-}
-// every thread of every CTA of the cluster, the same number of times on every path
-__device__ __forceinline__ void cluster_sync() {
-    __syncwarp();                    // the aligned forms want the whole warp at the same instruction
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
-    uint32_t remote;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-    return v;
-}
-
 // The head groups of one (d tile, batch tile) form one thread-block cluster (gridDim.y CTAs, at most 16): each CTA
 // accumulates Y^T over its heads in TMEM, leaves it in its shared memory, and after a cluster barrier every CTA adds up,
 // in group order, the batch rows that fall to it (row n to CTA n mod cluster size) out of all the CTAs' shared memory
