@@ -29,6 +29,17 @@
 
 namespace mqa {
 
+#ifdef MQA_DEBUG_TS
+__device__ unsigned long long g_ts[256 * 32];
+__device__ __forceinline__ unsigned long long dbg_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TS(k) do { g_ts[blockIdx.x * 32 + (k)] = dbg_ns(); } while (0)
+__device__ unsigned long long g_st[64 * 8];
+#define ST(j, k) do { if (blockIdx.x == MQA_DEBUG_CTA && (j) < 64) g_st[(j) * 8 + (k)] = dbg_ns(); } while (0)
+#else
+#define TS(k) do { } while (0)
+#define ST(j, k) do { } while (0)
+#endif
+
 constexpr int kTileRows = 32;                          // cache rows per pipeline stage
 constexpr int kBoxCols = 64;                           // 64 bf16 = 128 bytes = one swizzle span
 constexpr int kBoxBytes = kTileRows * kBoxCols * 2;    // 4 KiB
@@ -755,9 +766,15 @@ __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ len
 // Returns false when there is nothing to start early (more sequences, an empty share, or a share that
 // begins between two sequences); *rows = rows_of[] entry of the segment's sequence.
 constexpr int kFastSeqs = 256;
+// cluster > 1: the grid was launched as clusters of `cluster` CTAs with cluster * b == gridDim.x, this CTA has rank
+// `rank` in its cluster, and a stage is `stage_tiles` tiles.  If every sequence has the same, non-zero number of tiles,
+// cluster c holds sequence c and its CTAs take the sequence's stages in turn (rank r: stages r, r + cluster, ...):
+// then *strided is set and the segment returned is (sequence, first tile of stage r, all tiles of the sequence).
 template <bool FUSED, int PENALTY>
 __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, int b, int m_max, bool appending,
-                                              unsigned long long magic, Segment* g, int* rows) {
+                                              unsigned long long magic, Segment* g, int* rows, int cluster = 1, int rank = 0,
+                                              int stage_tiles = 4, bool* strided = nullptr) {
+    if (strided) *strided = false;
     if (b > kFastSeqs) return false;
     const int cta = blockIdx.x, lane = threadIdx.x & 31;
     const int per = (b + 31) >> 5, base = lane * per;
@@ -773,6 +790,30 @@ __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, 
             rw[i] = L | (appending && can_append ? kAppendBit : 0);
         }
         sum += tl[i];
+    }
+    if (sum >= 0 && lane == 0) TS(28);
+    if (cluster > 1) {
+        const int first = __shfl_sync(0xffffffffu, tl[0], 0);
+        bool same = first > 0;
+#pragma unroll
+        for (int i = 0; i < kFastSeqs / 32; ++i)
+            if (i < per && base + i < b) same = same && tl[i] == first;
+        if (__all_sync(0xffffffffu, same)) {
+            const int s = cta / cluster;
+            int fr = 0;
+#pragma unroll
+            for (int i = 0; i < kFastSeqs / 32; ++i)
+                if (i == s % per) fr = rw[i];
+            fr = __shfl_sync(0xffffffffu, fr, s / per);
+            g->s = s;
+            g->lo = rank * stage_tiles;
+            g->hi = first - PENALTY;
+            g->whole = false;
+            *rows = fr;
+            if (strided) *strided = true;
+            if (lane == 0) TS(29);
+            return g->lo < g->hi;
+        }
     }
     int incl = sum;
 #pragma unroll

@@ -39,17 +39,6 @@
 
 namespace mqa {
 
-#ifdef MQA_DEBUG_TS
-__device__ unsigned long long g_ts[256 * 32];
-__device__ __forceinline__ unsigned long long dbg_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TS(k) do { g_ts[blockIdx.x * 32 + (k)] = dbg_ns(); } while (0)
-__device__ unsigned long long g_st[64 * 8];
-#define ST(j, k) do { if (blockIdx.x == MQA_DEBUG_CTA && (j) < 64) g_st[(j) * 8 + (k)] = dbg_ns(); } while (0)
-#else
-#define TS(k) do { } while (0)
-#define ST(j, k) do { } while (0)
-#endif
-
 constexpr int kUmmaStageRows = 128;                              // cache rows per stage
 constexpr int kUmmaHalfBytes = kUmmaStageRows * 128;             // 16 KiB: one 64-column box of 128 rows
 constexpr int kUmmaSlotBytes = 2 * kUmmaHalfBytes;               // 32 KiB: the K (or the V) rows of a stage
@@ -59,6 +48,7 @@ constexpr int kUmmaProducerWarp = 8, kUmmaSWarp = 9, kUmmaPvWarp = 10;
 constexpr int kUmmaThreads = 11 * 32;
 // virtual tiles in front of each sequence on the line: what crossing from one sequence to the next costs this kernel
 constexpr int kUmmaBoundaryPenalty = 8;
+constexpr int kGuessL2Stages = 2;                                // stages asked into L2 on a guess, beyond those the rings take
 constexpr float kMaxLead = 16.f;                                 // log2 units a logit may exceed the reference maximum by
 
 template <int HP>
@@ -510,12 +500,20 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     //    whose results everything else waits for, starts only when told that the segment is settled (go).
     // 3  as 2 with a guess that is wrong on purpose, so that tests reach the recovery.
     int pre_issued = 0;                                     // stages whose copies were started here
+    // The launch is made of clusters of C CTAs when the batch divides the grid (C = G / b) and the step is a single
+    // launch.  With sequences of equal tile counts cluster c then holds sequence c: its CTAs take the sequence's stages
+    // in turn (rank r: stages r, r + C, ...: "strided"), leave one piece each in their own shared memory and merge the
+    // pieces through the cluster's shared window, with no partial result, fence or counter in global memory.  Whether
+    // the sequences are equal is decided from lens, by every CTA alike (stream_plan); until then it is a guess.
+    const uint32_t C = cluster_size();
+    const int crank = (int)cluster_cta_rank();
+    const int cl = (ctrl != nullptr && C > 1 && (long long)C * b == G) ? (int)C : 1;
     if (warp == kUmmaProducerWarp) {
         // One loop body serves both sides of the wait (with a guess it runs twice, and the second time its
         // instructions are already on the SM): work out the share's first segment, start what may be started.
         Segment g0 = {};
         int r0 = 0;
-        bool have = false, q_started = false;
+        bool have = false, q_started = false, strided0 = false;
         // A CTA that starts only when the kernel before has already completed (its SM was that kernel's last to become
         // free) gains nothing from a guess: by then a warp that went straight to the wait has come back and said so
         // (waited_sm, zeroed by this thread first, so that a 1 can only be that warp's), lens as it reads now is final,
@@ -525,7 +523,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             if (lane == 0) asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(late) : "r"(smem_addr(&waited_sm)) : "memory");
             late = __shfl_sync(0xffffffffu, late, 0);
         }
-        const int passes = (early >= 1 && !late) ? 2 : 1;
+        const bool lensfree = GUESS && early >= 2 && cl > 1;
+        const int passes = late ? 1 : early >= 1 ? 2 : 1;
+#pragma unroll 1
         for (int pass = 0; pass < passes; ++pass) {
             const bool before = pass + 1 < passes;          // this pass runs ahead of the wait
             if (!before) {
@@ -539,14 +539,32 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 }
                 if (lane == 0) TS(12);
             }
-            if (before || early != 1) {                     // (early == 1: lens cannot have moved)
+            if (lensfree && before) {
+                // A guess that needs no look at lens (a round trip to L2 saved on the way to the first copies): the
+                // sequences are equal and long, so this CTA's first stages are stages crank and crank + C of sequence
+                // cta / C.  Checked against lens after the wait like any guess.
+                g0.s = cta / cl;
+                g0.lo = crank * kSubs + (early == 3 ? kSubs : 0);    // (3, for tests: one stage off)
+                g0.hi = m_max / kTileRows;                           // whole tiles of a full cache
+                g0.whole = false;
+                r0 = m_max + 2;                                      // rows below m_max may be asked for
+                have = g0.lo < g0.hi;
+                strided0 = true;
+            } else if (before || early != 1) {              // (early == 1: lens cannot have moved)
                 Segment g = {};
                 int r = 0;
-                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r);
+                bool strided = false;
+                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r, cl, crank, kSubs, &strided);
                 if (before && lane == 0) TS(8);
                 if (GUESS && before && early == 3) g.lo += kSubs;    // for tests: a guess that is one stage off
                 if (!before && GUESS && early >= 2) {
-                    if (have && !(found && g.s == g0.s && g.lo == g0.lo && g.lo + pre_issued * kSubs <= g.hi)) {
+                    // the stages started on the guess stand if this is how the share begins and each of them is a
+                    // whole stage below the prefix's last two rows (which the step before may have been writing)
+                    bool keep = have && found && g.s == g0.s && g.lo == g0.lo && strided == strided0;
+                    const int ust = strided ? kSubs * cl : kSubs;
+                    for (int i = 0; i < pre_issued; ++i)
+                        keep = keep && g.lo + i * ust + kSubs <= g.hi && (g.lo + i * ust + kSubs) * kTileRows <= (r & (kAppendBit - 1)) - 2;
+                    if (have && !keep) {
                         // what was started on the guess is not how this share begins: each of those barriers has
                         // completed one phase when its copy has landed; one more arrival completes a second,
                         // empty one, and the slot is as new (no consumer has looked: the first of them waits for go)
@@ -568,23 +586,40 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 have = found;
                 g0 = g;
                 r0 = r;
+                strided0 = strided;
             }
             if (have) {
                 const int L = r0 & (kAppendBit - 1);
                 const int new_row = (r0 & kAppendBit) ? L - 1 : -1;          // row this step appends
+                const int ust = strided0 ? kSubs * cl : kSubs;               // tiles from one of this CTA's stages to the next
                 // rows that may be fetched now lie below stop_row: ahead of the wait not this step's new row
                 // (early == 1) or, on a guess, the prefix's last two rows, and then whole stages only
                 const int stop_row = !before ? 0x7fffffff : early == 1 ? (new_row >= 0 ? new_row : 0x7fffffff) : L - 2;
-                const int n_pre = min((g0.hi - g0.lo + kSubs - 1) / kSubs, NK < NV ? NK : NV);   // what the rings hold without a wait
-                const int u0 = g0.lo + pre_issued * kSubs;
-                if (!before && appending && new_row >= u0 * kTileRows && new_row < min(g0.hi, g0.lo + n_pre * kSubs) * kTileRows)
+                const int n_pre = min((g0.hi - g0.lo + ust - 1) / ust, NK < NV ? NK : NV);   // what the rings hold without a wait
+                // which of this segment's stages holds the new row (-1: none)
+                int p_row = -1;
+                if (new_row >= 0) {
+                    const int tile = new_row / kTileRows;
+                    if (tile >= g0.lo && tile < g0.hi && (tile - g0.lo) % ust < kSubs) p_row = (tile - g0.lo) / ust;
+                }
+                if (!before && appending && p_row >= pre_issued && p_row < n_pre)
                     row_store(g0.s, new_row, row_load(g0.s));   // the new row lies in the stages started now
                 if (lane == 0) {
                     if (!before && !q_started) issue_q(g0.s, 0);
-                    for (int u = u0; pre_issued < n_pre && (u + kSubs) * kTileRows <= stop_row &&
+                    for (int u = g0.lo + pre_issued * ust; pre_issued < n_pre && (u + kSubs) * kTileRows <= stop_row &&
                                      !(before && GUESS && early >= 2 && u + kSubs > g0.hi);
-                         u += kSubs, ++pre_issued)
+                         u += ust, ++pre_issued)
                         issue_stage(g0.s, u, g0.hi, pre_issued);
+                    if (before && lensfree) {
+                        // and the stages after those are asked into L2 (measured at 32 sequences x 8192 rows on 128
+                        // CTAs: 26.9 us per step without, 26.2 / 26.0 / 26.5 / 27.2 us with 1 / 2 / 3 / 4 stages)
+                        int u = g0.lo + pre_issued * ust;
+                        for (int p = 0; p < kGuessL2Stages && (u + kSubs) * kTileRows <= stop_row && u + kSubs <= g0.hi; ++p, u += ust) {
+                            const int y = g0.s * m_max + u * kTileRows;
+                            tma_prefetch_l2_2d(&map_k, 0, y); tma_prefetch_l2_2d(&map_k, kBoxCols, y);
+                            tma_prefetch_l2_2d(&map_v, 0, y); tma_prefetch_l2_2d(&map_v, kBoxCols, y);
+                        }
+                    }
                 }
                 pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
             }
@@ -608,12 +643,19 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                                                             rows_of, plan_sm, kUmmaProducerWarp);
     const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
     tc_fence_after();
-    // The launch is made of clusters of C CTAs when the batch divides the grid (C = G / b).  With sequences of equal
-    // tile counts the C CTAs of cluster r then hold exactly the pieces of sequence r, one piece each: they leave them
-    // in their own shared memory and merge them through the cluster's shared window (every CTA a part of the heads),
-    // with no partial result, fence or counter in global memory.  Decided here, by every CTA alike, from lens.
-    const uint32_t C = cluster_size();
-    const bool via_cluster = ctrl != nullptr && C > 1 && plan.equal && (long long)C * b == G;
+    // sequences of equal tile counts in a launch made of clusters: strided stages, pieces merged through the cluster
+    const bool via_cluster = cl > 1 && plan.equal;
+    const int ustep = via_cluster ? kSubs * cl : kSubs;     // tiles from one of this CTA's stages to the next
+    // the next segment of this CTA's share: a run of its line share, or the whole sequence of its cluster taken in strides
+    auto next_segment = [&](ShareWalker<kUmmaBoundaryPenalty>& walk, Segment& g, int seg) -> bool {
+        if (!via_cluster) return walk.next(g);
+        if (seg > 0) return false;
+        g.s = cta / cl;
+        g.lo = crank * kSubs;
+        g.hi = prefix[g.s + 1] - prefix[g.s] - kUmmaBoundaryPenalty;
+        g.whole = false;
+        return g.lo < g.hi;
+    };
     float* piece_acc = reinterpret_cast<float*>(ring);                        // [h][128] in the first K slot (free by then)
     float2* piece_ml = reinterpret_cast<float2*>(ring + kUmmaSlotBytes);      // [h] (reference maximum, sum) in the second
     bool piece_left = false;                                // (softmax warps) this CTA has left a piece there
@@ -628,18 +670,23 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
-            for (; p_ok && walk.next(g); ++seg) {
+            for (; p_ok && next_segment(walk, g, seg); ++seg) {
                 if (lane == 0 && !(seg == 0 && pre_issued > 0)) issue_q(g.s, seg);
                 const int rows_entry = rows_of[g.s];
                 const int new_row = (rows_entry & kAppendBit) ? (rows_entry & (kAppendBit - 1)) - 1 : -1;   // row this step appends
+                // which of the segment's stages holds the new row (-1: none, it is not this CTA's to write)
+                int p_row = -1;
+                if (new_row >= 0) {
+                    const int tile = new_row / kTileRows;
+                    if (tile >= g.lo && tile < g.hi && (tile - g.lo) % ustep < kSubs) p_row = (tile - g.lo) / ustep;
+                }
                 // the new row is in this segment and was not written on the way to the first stages
-                bool row_due = appending && new_row >= g.lo * kTileRows && new_row < g.hi * kTileRows &&
-                               !(seg == 0 && new_row < (g.lo + pre_issued * kSubs) * kTileRows);
+                bool row_due = appending && p_row >= 0 && !(seg == 0 && p_row < pre_issued);
                 uint4 row = make_uint4(0u, 0u, 0u, 0u);
                 if (row_due) row = row_load(g.s);
-                for (int u = g.lo; u < g.hi && p_ok; u += kSubs, ++j) {
+                for (int u = g.lo; u < g.hi && p_ok; u += ustep, ++j) {
                     // stored once the segment's first stage is on its way, or earlier if that stage holds the row
-                    if (row_due && (u > g.lo || new_row < (u + kSubs) * kTileRows)) {
+                    if (row_due && (u > g.lo || p_row == 0)) {
                         row_store(g.s, new_row, row);
                         row_due = false;
                     }
@@ -675,11 +722,11 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
-            for (; walk.next(g); ++seg) {
+            for (; next_segment(walk, g, seg); ++seg) {
                 const int qi = seg % NQ;
                 if (ok) ok = mbar_wait(q_full + qi * 8, (seg / NQ) & 1);
                 if (seg == 0) TS(15);
-                for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
+                for (int u = g.lo; u < g.hi; u += ustep, ++j) {
                     const int slot = j % NK, sb = j & 1;
                     if (ok) ok = mbar_wait(k_full + slot * 8, (j / NK) & 1);
                     if (j == 0) TS(2);
@@ -699,7 +746,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     }
                     tc_commit(s_ready + sb * 8);
                     tc_commit(k_empty + slot * 8);                   // the K rows are not needed again
-                    if (u + kSubs >= g.hi) tc_commit(q_empty + qi * 8);   // last use of this segment's Q
+                    if (u + ustep >= g.hi) tc_commit(q_empty + qi * 8);   // last use of this segment's Q
                 }
             }
             if (!ok) atomicExch(&timed_out, 1);
@@ -712,10 +759,10 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             int j = 0, seg = 0;
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
-            for (; walk.next(g); ++seg) {
+            for (; next_segment(walk, g, seg); ++seg) {
                 const int L = rows_of[g.s] & (kAppendBit - 1);
                 const int parts = L >= kSingleRoundingMinRows ? 1 : 2;   // P hi only, or hi then lo (as the softmax warps wrote it)
-                for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
+                for (int u = g.lo; u < g.hi; u += ustep, ++j) {
                     const int pb = j & 1, slot = j % NV;
                     // the weights first: they exist only once q has arrived, and before that a slot's barrier may
                     // still be on its way back from copies started on a guess (see early above)
@@ -822,7 +869,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             };
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
-            for (; walk.next(g); ++seg) {
+            for (; next_segment(walk, g, seg); ++seg) {
                 const int s = g.s;
                 const int L = rows_of[s] & (kAppendBit - 1);
                 const bool whole = g.whole;
@@ -831,7 +878,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 float l_sum[HH];                            // this row's share of its heads' sums of weights
 #pragma unroll
                 for (int i = 0; i < HH; ++i) l_sum[i] = 0.f;
-                for (int u = g.lo; u < g.hi; u += kSubs, ++j) {
+                for (int u = g.lo; u < g.hi; u += ustep, ++j) {
                     const int sb = j & 1, pb = j & 1;
                     const bool first = u == g.lo;           // nothing accumulated yet: no reference maxima, O^T not started
                     // rows of this stage that count: what was fetched (the share may end mid-stage) and
