@@ -393,7 +393,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     const uint32_t s_ready = q_empty + 16, s_free = s_ready + 16;
     const uint32_t p_ready = s_free + 16, pv_done = p_ready + 16, o_free = pv_done + 16;   // o_free: one per O^T buffer
     const uint32_t go = o_free + 16;                        // the share's first segment is settled (see early below)
-    __shared__ int timed_out, issued, plan_sm[8], merge_sm[8];   // merge_sm: count, then (sequence, first CTA, last CTA) x 2
+    __shared__ int timed_out, issued[2], plan_sm[8], merge_sm[8];   // merge_sm: count, then (sequence, first CTA, last CTA) x 2
     __shared__ unsigned long long epoch_sm[2];              // this launch's epoch; the epoch word as found
     __shared__ uint32_t tmem_base_slot;
     __shared__ int waited_sm;                                // 1 once a warp of this CTA has come back from the wait on the kernel before
@@ -406,7 +406,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         prefetch_tensormap(&map_k); prefetch_tensormap(&map_v); prefetch_tensormap(&map_k_sub);
         prefetch_tensormap(&map_v_sub); prefetch_tensormap(&map_q);
         timed_out = 0;
-        issued = 0;
+        issued[0] = issued[1] = 0;
         merge_sm[0] = 0;
         for (int s = 0; s < NK; ++s) { mbar_init(k_full + s * 8, 1); mbar_init(k_empty + s * 8, 1); }
         for (int s = 0; s < NV; ++s) { mbar_init(v_full + s * 8, 1); mbar_init(v_empty + s * 8, 1); }
@@ -442,48 +442,38 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         __syncwarp();
         asm volatile("fence.proxy.async;" ::: "memory");
     };
-    // ---- what the producer thread does for a segment and for a stage
+    // ---- what the producer warp does for a segment and for a stage.  A copy instruction takes a tenth of a
+    // microsecond to issue, so the boxes of a stage go out in one instruction executed by four lanes: lane =
+    // 2 * (0: the K rows, 1: the V rows) + (which 64-column half); the two boxes of Q by lanes 0 and 1.
     bool p_ok = true;                                       // no producer wait has run out
-    auto issue_q = [&](int s, int seg) {
+    auto issue_q = [&](int s, int seg) {                    // lanes 0 and 1
         const int qi = seg % NQ;
         if (seg >= NQ) p_ok = p_ok && mbar_wait(q_empty + qi * 8, ((seg / NQ) - 1) & 1);
         if (!p_ok) return;
         // the sequence's head rows (rows past h belong to the next sequence or read as zero: their
         // columns of S^T and O^T are never stored)
-        mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
-        tma_load_2d(q_s + qi * Cfg::kQBytes, &map_q, 0, s * h, q_full + qi * 8);
-        tma_load_2d(q_s + qi * Cfg::kQBytes + Cfg::kQBytes / 2, &map_q, kBoxCols, s * h, q_full + qi * 8);
+        if (lane == 0) mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
+        tma_load_2d(q_s + qi * Cfg::kQBytes + lane * (Cfg::kQBytes / 2), &map_q, lane * kBoxCols, s * h, q_full + qi * 8);
     };
     const uint64_t stream_policy = l2_stream_policy(read_once != 0);
-    auto issue_stage = [&](int s, int u, int hi, int j) {
+    auto issue_stage = [&](int s, int u, int hi, int j) {   // lanes 0 to 3
+        const int kv = lane >> 1, half = lane & 1;          // the K rows, then the V rows, each into its own ring
         const int nsub = min(kSubs, hi - u);
-        const int row_first = u * kTileRows;
-        const int y = s * m_max + row_first;
-#pragma unroll
-        for (int kv = 0; kv < 2; ++kv) {                    // the K rows, then the V rows, each into its own ring
-            const int n_slots = kv ? NV : NK;
-            const int slot = j % n_slots;
-            const uint32_t full = (kv ? v_full : k_full) + slot * 8;
-            if (j >= n_slots) p_ok = p_ok && mbar_wait((kv ? v_empty : k_empty) + slot * 8, ((j / n_slots) - 1) & 1);
-            if (!p_ok) return;
-            const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes;
-            if (j < 2) TS(16 + j * 6 + kv * 3);
-            mbar_expect_tx(full, nsub * 2 * kBoxBytes);
-            if (j < 2) TS(16 + j * 6 + kv * 3 + 1);
-            if (nsub == kSubs) {
-                tma_load_2d_hint(dst, kv ? &map_v : &map_k, 0, y, full, stream_policy);
-                if (j < 2) TS(16 + j * 6 + kv * 3 + 2);
-                tma_load_2d_hint(dst + kUmmaHalfBytes, kv ? &map_v : &map_k, kBoxCols, y, full, stream_policy);
-            } else {
-                for (int i = 0; i < nsub; ++i) {
-                    const uint32_t d = dst + i * kBoxBytes;
-                    tma_load_2d_hint(d, kv ? &map_v_sub : &map_k_sub, 0, y + i * kTileRows, full, stream_policy);
-                    tma_load_2d_hint(d + kUmmaHalfBytes, kv ? &map_v_sub : &map_k_sub, kBoxCols, y + i * kTileRows, full, stream_policy);
-                }
-            }
-            issued = 2 * j + kv + 1;                        // copies started: K of stage j, then V of stage j
-            if (kv == 0) ST(j, 7);
+        const int y = s * m_max + u * kTileRows;
+        const int n_slots = kv ? NV : NK;
+        const int slot = j % n_slots;
+        const uint32_t full = (kv ? v_full : k_full) + slot * 8;
+        if (j >= n_slots) p_ok = p_ok && mbar_wait((kv ? v_empty : k_empty) + slot * 8, ((j / n_slots) - 1) & 1);
+        if (!p_ok) return;
+        const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes + half * kUmmaHalfBytes;
+        if (half == 0) mbar_expect_tx(full, nsub * 2 * kBoxBytes);
+        if (nsub == kSubs) {
+            tma_load_2d_hint(dst, kv ? &map_v : &map_k, half * kBoxCols, y, full, stream_policy);
+        } else {
+            for (int i = 0; i < nsub; ++i)
+                tma_load_2d_hint(dst + i * kBoxBytes, kv ? &map_v_sub : &map_k_sub, half * kBoxCols, y + i * kTileRows, full, stream_policy);
         }
+        if (half == 0) issued[kv] = j + 1;                  // stages whose K (V) copies were started
     };
 
     // ---- what may start before the wait on the kernel before this one (early):
@@ -534,7 +524,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 grid_launch_dependents();
                 if (lane == 0) TS(1);
                 if (GUESS && early >= 2 && have) {                   // q of the guessed sequence, while the guess is checked
-                    if (lane == 0) issue_q(g0.s, 0);
+                    if (lane < 2) issue_q(g0.s, 0);
                     q_started = true;
                 }
                 if (lane == 0) TS(12);
@@ -604,8 +594,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 }
                 if (!before && appending && p_row >= pre_issued && p_row < n_pre)
                     row_store(g0.s, new_row, row_load(g0.s));   // the new row lies in the stages started now
-                if (lane == 0) {
-                    if (!before && !q_started) issue_q(g0.s, 0);
+                if (lane < 4) {
+                    if (lane < 2 && !before && !q_started) issue_q(g0.s, 0);
                     for (int u = g0.lo + pre_issued * ust; pre_issued < n_pre && (u + kSubs) * kTileRows <= stop_row &&
                                      !(before && GUESS && early >= 2 && u + kSubs > g0.hi);
                          u += ust, ++pre_issued)
@@ -615,13 +605,12 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         // CTAs: 26.9 us per step without, 26.2 / 26.0 / 26.5 / 27.2 us with 1 / 2 / 3 / 4 stages)
                         int u = g0.lo + pre_issued * ust;
                         for (int p = 0; p < kGuessL2Stages && (u + kSubs) * kTileRows <= stop_row && u + kSubs <= g0.hi; ++p, u += ust) {
-                            const int y = g0.s * m_max + u * kTileRows;
-                            tma_prefetch_l2_2d(&map_k, 0, y); tma_prefetch_l2_2d(&map_k, kBoxCols, y);
-                            tma_prefetch_l2_2d(&map_v, 0, y); tma_prefetch_l2_2d(&map_v, kBoxCols, y);
+                            tma_prefetch_l2_2d((lane >> 1) ? &map_v : &map_k, (lane & 1) * kBoxCols, g0.s * m_max + u * kTileRows);
                         }
                     }
                 }
                 pre_issued = __shfl_sync(0xffffffffu, pre_issued, 0);
+                p_ok = __all_sync(0xffffffffu, p_ok);
             }
         }
     } else if (early != 1) {
@@ -671,7 +660,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             ShareWalker<kUmmaBoundaryPenalty> walk{prefix, t_begin, t_end, s_first};
             Segment g;
             for (; p_ok && next_segment(walk, g, seg); ++seg) {
-                if (lane == 0 && !(seg == 0 && pre_issued > 0)) issue_q(g.s, seg);
+                if (lane < 2 && !(seg == 0 && pre_issued > 0)) issue_q(g.s, seg);
                 const int rows_entry = rows_of[g.s];
                 const int new_row = (rows_entry & kAppendBit) ? (rows_entry & (kAppendBit - 1)) - 1 : -1;   // row this step appends
                 // which of the segment's stages holds the new row (-1: none, it is not this CTA's to write)
@@ -690,8 +679,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         row_store(g.s, new_row, row);
                         row_due = false;
                     }
-                    if (lane == 0 && j >= pre_issued) issue_stage(g.s, u, g.hi, j);
-                    p_ok = __shfl_sync(0xffffffffu, (int)p_ok, 0) != 0;
+                    if (lane < 4 && j >= pre_issued) issue_stage(g.s, u, g.hi, j);
+                    p_ok = __all_sync(0xffffffffu, p_ok);
                 }
             }
             if (lane == 0 && !p_ok) atomicExch(&timed_out, 1);
@@ -1119,7 +1108,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     __syncthreads();
     if (timed_out && threadIdx.x == 0) {
         // before the CTA leaves: the last copy started into each ring slot has to land
-        const int n_k = (issued + 1) / 2, n_v = issued / 2;
+        const int n_k = issued[0], n_v = issued[1];
         for (int s = 0; s < NK && s < n_k; ++s) mbar_wait(k_full + s * 8, ((n_k - 1 - s) / NK) & 1);
         for (int s = 0; s < NV && s < n_v; ++s) mbar_wait(v_full + s * 8, ((n_v - 1 - s) / NV) & 1);
         if (status) atomicOr(status, kStatusPipelineTimeout);
