@@ -158,6 +158,9 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
  *                     it, it fetches again.
  *                     MQA_STEP_TEST_WRONG_GUESS (4), for tests, with MQA_STEP_CHAINED: the early fetch is
  *                     deliberately the wrong one, so that this recovery runs; results are unchanged.
+ *                     MQA_STEP_TEST_WITHHOLD_COPY (8), for tests: one on-chip copy of the first CTA is never
+ *                     started, so that a bounded wait runs out (see mqa_set_wait_limit_cycles): the kernel
+ *                     returns by itself, PIPELINE_TIMEOUT is flagged and o is not valid.
  *                     Any other bit: MQA_ERR_INVALID_ARG.
  *   o, workspace, workspace_bytes, status   as for mqa_decode_step.  A sequence with lens[b] == m_max
  *                     (or negative) takes no new row: APPEND_CACHE_FULL (APPEND_NEGATIVE_LEN) is flagged
@@ -167,6 +170,7 @@ int mha_decode_step(const void* q, const void* K, const void* V, const int32_t* 
 #define MQA_STEP_ADVANCE 1
 #define MQA_STEP_CHAINED 2
 #define MQA_STEP_TEST_WRONG_GUESS 4
+#define MQA_STEP_TEST_WITHHOLD_COPY 8
 int mqa_decode_append_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
                            int advance, float* o, void* workspace, size_t workspace_bytes, int32_t* status,
                            int b, int h, int m_max, int k, int v, mqa_stream_t stream);
@@ -321,6 +325,15 @@ int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const
 
 /* mqa_layer_workspace_bytes -- scratch mqa_layer_decode_step needs (0 for invalid or unsupported sizes). Host-only. */
 size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v);
+
+/*
+ * mqa_set_wait_limit_cycles -- how long, in SM clock cycles, a kernel of this library waits for one of its own
+ * on-chip copies or products before it gives up, flags MQA_STATUS_PIPELINE_TIMEOUT and returns (no kernel here
+ * waits without a bound, and none traps).  The default, restored by cycles <= 0, is about one second; tests
+ * shorten it to see a wait run out within milliseconds.  Sets a variable on the current device, for kernels
+ * launched afterwards; unlike the step calls this one is synchronous (it waits for the device to take the value).
+ */
+int mqa_set_wait_limit_cycles(long long cycles);
 
 /* mqa_status_string -- a static, human-readable name for a return code. */
 const char* mqa_status_string(int code);

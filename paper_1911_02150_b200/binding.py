@@ -25,7 +25,7 @@ EXPORTS = (
     "kv_cache_append", "mqa_decode_step", "mha_decode_step",
     "mqa_decode_step_split", "mqa_decode_step_combine",
     "mha_decode_step_split", "mha_decode_step_combine",
-    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_status_string", "mqa_decode_step_noalloc",
+    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_set_wait_limit_cycles", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
     "mqa_layer_decode_step", "mqa_layer_workspace_bytes", "mqa_decode_local_step",
     "mqa_decode_append_step_host", "mqa_host_staging_bytes",
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.mqa_plan_splits.restype = I
         L.mqa_plan_kernel_name.argtypes = [I, I, I, I, I, I, I]
         L.mqa_plan_kernel_name.restype = ctypes.c_char_p
+        L.mqa_set_wait_limit_cycles.argtypes = [ctypes.c_longlong]
+        L.mqa_set_wait_limit_cycles.restype = I
         L.mqa_status_string.argtypes = [I]
         L.mqa_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -157,12 +159,20 @@ def _need(t: torch.Tensor, dtype, shape, name: str):
         raise ValueError(f"{name} must be contiguous")
 
 
-STEP_ADVANCE, STEP_CHAINED, STEP_TEST_WRONG_GUESS = 1, 2, 4
+STEP_ADVANCE, STEP_CHAINED, STEP_TEST_WRONG_GUESS, STEP_TEST_WITHHOLD_COPY = 1, 2, 4, 8
 
 
-def _step_flags(advance, chained) -> int:
-    """``chained``: False, True, or "wrong-guess" (the testing form of True)."""
-    return (STEP_ADVANCE if advance else 0) | (STEP_CHAINED if chained else 0) | (STEP_TEST_WRONG_GUESS if chained == "wrong-guess" else 0)
+def _step_flags(advance, chained, withhold_copy=False) -> int:
+    """``chained``: False, True, or "wrong-guess" (the testing form of True); ``withhold_copy``: the testing flag that
+    makes one bounded wait run out."""
+    return ((STEP_ADVANCE if advance else 0) | (STEP_CHAINED if chained else 0) |
+            (STEP_TEST_WRONG_GUESS if chained == "wrong-guess" else 0) | (STEP_TEST_WITHHOLD_COPY if withhold_copy else 0))
+
+
+def set_wait_limit_cycles(cycles: int) -> None:
+    """How long a kernel waits for one of its own on-chip copies before it flags PIPELINE_TIMEOUT and returns
+    (SM clock cycles; <= 0 restores the default of about a second).  Synchronous."""
+    _check(lib().mqa_set_wait_limit_cycles(int(cycles)), "mqa_set_wait_limit_cycles")
 
 
 def _check(rc: int, where: str):
@@ -271,7 +281,7 @@ def mqa_decode_step_noalloc(q, K, V, lens, o, status=None, stream=None):
     return o
 
 
-def _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained):
+def _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained, withhold_copy=False):
     """Checks the tensors of the append-and-attend step and returns the C call's argument tuple (plain integers)."""
     b, h, k = q.shape
     m_max, v = K.shape[-2], V.shape[-1]
@@ -286,20 +296,20 @@ def _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance
         _need(status, torch.int32, (1,), "status")
     s = torch.cuda.current_stream(q.device) if stream is None else stream
     return (q.data_ptr(), K.data_ptr(), V.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), lens.data_ptr(),
-            _step_flags(advance, chained), o.data_ptr(), None if workspace is None else workspace.data_ptr(),
+            _step_flags(advance, chained, withhold_copy), o.data_ptr(), None if workspace is None else workspace.data_ptr(),
             0 if workspace is None else workspace.numel() * workspace.element_size(),
             None if status is None else status.data_ptr(), b, h, m_max, k, v, s.cuda_stream)
 
 
 def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, status=None, advance: bool = True, stream=None,
-                           chained: bool = False):
+                           chained: bool = False, withhold_copy: bool = False):
     """One whole multi-query decoding step in one call: append ``k_new``/``v_new`` at row ``lens[b]`` of the
     shared cache, then attend over ``lens[b] + 1`` rows; ``lens`` is advanced on the device when ``advance``.
     For batches the persistent kernel serves (h <= 64) the whole step is one kernel launch.  ``chained``: the
     caller's promise that nothing enqueued on the stream since this library's last step on this cache writes
     the cache, ``lens`` or the workspace (a decoding loop); the kernel then starts on the cache before the
     kernel ahead of it has finished."""
-    args = _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained)
+    args = _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained, withhold_copy)
     with _OnDevice(q.device):
         rc = lib().mqa_decode_append_step(*args)
     _check(rc, "mqa_decode_append_step")

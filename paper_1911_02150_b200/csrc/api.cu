@@ -296,7 +296,8 @@ std::atomic<int> g_smem_opt_in[kMaxDevices][4];
 template <int M_TILES, bool EARLY = false>
 int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias,
-               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr, bool ring = false) {
+               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr, bool ring = false,
+               bool withhold = false) {
     using Cfg = MmaCfg<M_TILES>;
     auto kernel = mqa_decode_split_mma_kernel<M_TILES, EARLY>;
     constexpr int kSlot = (M_TILES - 1) * 2 + (EARLY ? 1 : 0);
@@ -323,11 +324,12 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     }
     launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
                      map_k_big, map_v_big, static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
-                     p.n_splits, len_bias, fa, lens_advance, ring ? 1 : 0);
+                     p.n_splits, len_bias, fa, lens_advance, (ring ? 1 : 0) | (withhold ? 2 : 0));
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
 constexpr size_t kL2KeepBytes = 64u << 20;   // K and V together: half of the 126 MB L2
+constexpr int kEarlyTestWithhold = 1 << 8;    // rides on `early`: MQA_STEP_TEST_WITHHOLD_COPY
 std::atomic<int> g_umma_opt_in[kMaxDevices][9];
 
 template <int HP, bool FUSED, bool GUESS = false>
@@ -362,7 +364,8 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     // a cache that cannot stay in L2 from one step to the next is streamed through it with the evict-first policy
-    const int read_once = (size_t)b * m_max * 2 * kRowBytes > kL2KeepBytes ? 1 : 0;
+    const int read_once = ((size_t)b * m_max * 2 * kRowBytes > kL2KeepBytes ? 1 : 0) | ((early & kEarlyTestWithhold) ? 2 : 0);
+    early &= ~kEarlyTestWithhold;
     // The single-launch step of a batch that divides the grid runs as clusters of grid / b CTAs (2 to 8, the
     // portable sizes): with sequences of equal length a cluster then holds exactly one sequence's pieces and merges
     // them through its shared memory (the kernel decides from lens; otherwise the clusters change nothing).
@@ -381,7 +384,7 @@ int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, 
                     int early = 0) {
 #define MQA_UMMA_ARGS p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, early
     if constexpr (FUSED) {
-        if (early >= 2) {                                   // the kernels that carry the code for copies started on a guess
+        if ((early & ~kEarlyTestWithhold) >= 2) {           // the kernels that carry the code for copies started on a guess
             if (h <= 16) return launch_umma<16, true, true>(MQA_UMMA_ARGS);
             if (h <= 32) return launch_umma<32, true, true>(MQA_UMMA_ARGS);
             return launch_umma<64, true, true>(MQA_UMMA_ARGS);
@@ -644,7 +647,7 @@ constexpr int kGuessMaxPieces = 6, kGuessMinShareRows = 8 * kUmmaStageRows;
 static int check_append_step(const void* q, const void* K, const void* V, const void* k_new, const void* v_new,
                              const int32_t* lens, int flags, const float* o, const void* workspace, size_t workspace_bytes,
                              const int32_t* status, int b, int h, int m_max, int k, int v) {
-    if (flags & ~(MQA_STEP_ADVANCE | MQA_STEP_CHAINED | MQA_STEP_TEST_WRONG_GUESS)) return MQA_ERR_INVALID_ARG;
+    if (flags & ~(MQA_STEP_ADVANCE | MQA_STEP_CHAINED | MQA_STEP_TEST_WRONG_GUESS | MQA_STEP_TEST_WITHHOLD_COPY)) return MQA_ERR_INVALID_ARG;
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
     if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return MQA_ERR_INVALID_ARG;
@@ -663,12 +666,14 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
                 : !(flags & MQA_STEP_CHAINED) ? kEarlyNone
                 : (flags & MQA_STEP_TEST_WRONG_GUESS) ? kEarlyChainedWrongGuess : kEarlyChained;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const bool withhold = (flags & MQA_STEP_TEST_WITHHOLD_COPY) != 0;
     const Plan p = make_plan(true, b, h, m_max);
     if (p.kernel == Kernel::kUmma) {
         // copies started on a guess pay where the step is one launch over long shares (measured: 0.4-0.7 us gained with
         // up to 6 pieces per sequence, 0.3-2.5 us lost with more pieces, short shares or a second-pass kernel)
         if (early == kEarlyChained && !(p.merge_in_kernel && p.n_splits <= kGuessMaxPieces && p.chunk_rows >= kGuessMinShareRows))
             early = kEarlyNone;
+        if (withhold) early |= kEarlyTestWithhold;
         // one launch: append inside the pass, pieces merged by the last CTA to deliver one, lens advanced at the end
         if (p.merge_in_kernel)
             return launch_umma_for<true>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, true, k_new, v_new,
@@ -684,7 +689,7 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
         // one CTA per sequence: it writes the row, attends and moves lens on, all in one launch
         // tiles below the prefix's last rows are fetched ahead of the wait (measured: 5.70 -> 5.45 us per step over the
         // 128 steps of a cache growing to 128 rows; nothing gained, 0.2 us lost, at 512 rows)
-        if (early == kEarlyChained && m_max <= 8 * kTileRows)
+        if (early == kEarlyChained && m_max <= 8 * kTileRows && !withhold)
             return p.kernel == Kernel::kMma1
                        ? launch_mma<1, true>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
                                              advance ? lens : nullptr)
@@ -692,17 +697,17 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
                                              advance ? lens : nullptr);
         return p.kernel == Kernel::kMma1
                    ? launch_mma<1>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
-                                   advance ? lens : nullptr)
+                                   advance ? lens : nullptr, false, withhold)
                    : launch_mma<2>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
-                                   advance ? lens : nullptr);
+                                   advance ? lens : nullptr, false, withhold);
     }
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits > 1) {
         // fixed splits: the CTA whose rows hold the new one writes it; the second pass moves lens on.  Two launches.
         float2* part_ml = partials_ml(workspace);
         float* part_acc = partials_acc(p, workspace);
         rc = p.kernel == Kernel::kMma1
-                 ? launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr)
-                 : launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr);
+                 ? launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr, false, withhold)
+                 : launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr, false, withhold);
         if (rc) return rc;
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr, true);
     }
@@ -866,6 +871,15 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
     const Plan p = make_plan(multi_query != 0, b, h, m_max);
     if (chunk_rows) *chunk_rows = p.chunk_rows;
     return p.n_splits;
+}
+
+int mqa_set_wait_limit_cycles(long long cycles) {
+    const long long value = cycles > 0 ? cycles : kWaitLimitCycles;
+    if (cudaMemcpyToSymbol(g_wait_limit_cycles, &value, sizeof value) != cudaSuccess) {
+        cudaGetLastError();
+        return MQA_ERR_CUDA;
+    }
+    return MQA_OK;
 }
 
 const char* mqa_plan_kernel_name(int multi_query, int whole_step, int b, int h, int m_max, int k, int v) {

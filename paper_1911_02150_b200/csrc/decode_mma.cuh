@@ -47,6 +47,8 @@ constexpr int kStageBytes = 4 * kBoxBytes;             // K lo, K hi, V lo, V hi
 constexpr int kRowWarps = 4;                           // consumer warps that share the tiles
 constexpr long long kWaitLimitCycles = 2000000000ll;   // every mbarrier wait gives up after ~1 s of SM clock ...
 constexpr uint32_t kWaitRounds = 1u << 24;             // ... or after this many polling rounds
+// The limit in force, in SM clock cycles (mqa_set_wait_limit_cycles: a test shortens it to see a wait run out).
+__device__ long long g_wait_limit_cycles = kWaitLimitCycles;
 constexpr int kSingleRoundingMinRows = 1024;            // prefixes this long feed P to the tensor cores in one bf16 rounding
 constexpr int kStreamMaxSeqs = 1024;                   // sequences the persistent kernel can index in shared memory
 
@@ -91,11 +93,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
+    const long long limit = g_wait_limit_cycles;
     for (uint32_t round = 0; round < kWaitRounds; ++round) {
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > kWaitLimitCycles && clock64() - t0 > kWaitLimitCycles) return false;
+        if (clock64() - t0 > limit && clock64() - t0 > limit) return false;
     }
     return false;
 }
@@ -358,8 +361,10 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
                             const uint32_t* __restrict__ q, const int32_t* __restrict__ lens,
                             float* __restrict__ o, float2* __restrict__ part_ml, float* __restrict__ part_acc,
                             int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias,
-                            const FusedArgs fa, int32_t* __restrict__ lens_advance, int ring) {
+                            const FusedArgs fa, int32_t* __restrict__ lens_advance, int mode) {
     using Cfg = MmaCfg<M_TILES>;
+    const int ring = mode & 1;                             // the cache is a window (local attention)
+    const bool withhold = (mode & 2) != 0;                 // for tests: one copy is never started, so that a wait runs out
     constexpr int kStages = Cfg::kStages;
     const int seq = blockIdx.x / n_splits;
     const int split = blockIdx.x % n_splits;
@@ -395,7 +400,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         tma_load_2d(dst, &map_k, 0, y, bar);
         tma_load_2d(dst + kBoxBytes, &map_k, kBoxCols, y, bar);
         tma_load_2d(dst + 2 * kBoxBytes, &map_v, 0, y, bar);
-        tma_load_2d(dst + 3 * kBoxBytes, &map_v, kBoxCols, y, bar);
+        if (!(withhold && blockIdx.x == 0 && i == 1)) tma_load_2d(dst + 3 * kBoxBytes, &map_v, kBoxCols, y, bar);
         issued = i + 1;
     };
     // EARLY (the caller's promise that only this library's steps have written the cache and lens since its last step
@@ -451,7 +456,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const int n_tiles = (r1 - r0 + kTileRows - 1) / kTileRows;
     // a few tiles (each has a stage of its own), beginning at a multiple of 128 rows: fetched four tiles per copy
     // (from three tiles on: a copy moves all 128 rows of its box, and one or two tiles are quicker on their own)
-    const bool big = !EARLY && n_tiles >= 3 && n_tiles <= kStages && (r0 & (4 * kTileRows - 1)) == 0;
+    const bool big = !EARLY && !withhold && n_tiles >= 3 && n_tiles <= kStages && (r0 & (4 * kTileRows - 1)) == 0;
 
     __syncthreads();
 

@@ -455,7 +455,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         if (lane == 0) mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
         tma_load_2d(q_s + qi * Cfg::kQBytes + lane * (Cfg::kQBytes / 2), &map_q, lane * kBoxCols, s * h, q_full + qi * 8);
     };
-    const uint64_t stream_policy = l2_stream_policy(read_once != 0);
+    const uint64_t stream_policy = l2_stream_policy((read_once & 1) != 0);
+    const bool withhold = (read_once & 2) != 0;             // for tests: one copy is never started, so that a wait runs out
     auto issue_stage = [&](int s, int u, int hi, int j) {   // lanes 0 to 3
         const int kv = lane >> 1, half = lane & 1;          // the K rows, then the V rows, each into its own ring
         const int nsub = min(kSubs, hi - u);
@@ -467,7 +468,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         if (!p_ok) return;
         const uint32_t dst = (kv ? v_ring : k_ring) + slot * kUmmaSlotBytes + half * kUmmaHalfBytes;
         if (half == 0) mbar_expect_tx(full, nsub * 2 * kBoxBytes);
-        if (nsub == kSubs) {
+        if (withhold && cta == 0 && j == 1 && lane == 3) {
+            // (the V rows' second half of this CTA's second stage stays away)
+        } else if (nsub == kSubs) {
             tma_load_2d_hint(dst, kv ? &map_v : &map_k, half * kBoxCols, y, full, stream_policy);
         } else {
             for (int i = 0; i < nsub; ++i)

@@ -41,13 +41,15 @@ def test_header_constants_and_binding_agree():
     assert defines["MQA_STEP_TEST_WRONG_GUESS"] == binding.STEP_TEST_WRONG_GUESS == 4
     assert binding._step_flags(True, False) == 1 and binding._step_flags(False, True) == 2
     assert binding._step_flags(True, "wrong-guess") == 7
+    assert defines["MQA_STEP_TEST_WITHHOLD_COPY"] == binding.STEP_TEST_WITHHOLD_COPY == 8
+    assert binding._step_flags(False, False, True) == 8
 
 
 def test_step_flags_are_checked_before_any_launch(L):
     vp = ctypes.c_void_p
     a = vp(0x1000)
     # an unknown flag bit: refused on the host, nothing dereferenced
-    rc = L.mqa_decode_append_step(a, a, a, a, a, a, 8, a, a, 1 << 30, None, 4, 8, 256, 128, 128, None)
+    rc = L.mqa_decode_append_step(a, a, a, a, a, a, 16, a, a, 1 << 30, None, 4, 8, 256, 128, 128, None)
     assert rc == binding.ERR_INVALID_ARG
 
 

@@ -6,6 +6,7 @@ import torch
 
 import oracle
 import paper_1911_02150_b200 as mqa
+from guards import Guarded
 from paper_1911_02150_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -28,14 +29,25 @@ def run(b, h, m_max, lens0, advance, seed, chained=False):
     Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
     skipped = oracle.kv_cache_append(Kh, Vh, wl.bits(inp["k_new"]), wl.bits(inp["v_new"]), lens_h, True)
     ref = oracle.mqa_decode_step(wl.bits(inp["q"]), Kh, Vh, lens_h)
-    lens_t = torch.from_numpy(lens0).to(DEV)
-    o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
-    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    # everything small that the step reads or writes sits between guard regions, checked after the kernels have run
+    lens_g = Guarded((b,), torch.int32, DEV, like=torch.from_numpy(lens0).to(DEV))
+    lens_t = lens_g.t
+    o_g = Guarded((b, h, 128), torch.float32, DEV)
+    o = o_g.t
+    o.fill_(float("nan"))
+    ws_g = Guarded((max(16, mqa.workspace_bytes(b, h, m_max)),), torch.uint8, DEV)
+    ws = ws_g.t
     ws.fill_(0xFF)
-    status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws, status,
+    status_g = Guarded((1,), torch.int32, DEV)
+    status = status_g.t
+    status.zero_()
+    q_g, kn_g, vn_g = (Guarded(tuple(inp[n].shape), torch.bfloat16, DEV, like=inp[n]) for n in ("q", "k_new", "v_new"))
+    mqa.mqa_decode_append_step(q_g.t, inp["K"], inp["V"], kn_g.t, vn_g.t, lens_t, o, ws, status,
                                advance=advance, chained=chained)
     torch.cuda.synchronize()
+    for g, name in ((lens_g, "lens"), (o_g, "o"), (ws_g, "workspace"), (status_g, "status"), (q_g, "q"), (kn_g, "k_new"), (vn_g, "v_new")):
+        g.check(f"append_step b={b} h={h} m_max={m_max}: {name}")
+    assert torch.equal(q_g.t, inp["q"]) and torch.equal(kn_g.t, inp["k_new"]) and torch.equal(vn_g.t, inp["v_new"])
     check_close(o.cpu().numpy(), ref, f"append_step b={b} h={h} m_max={m_max}")
     assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)   # the append, bit for bit
     assert np.array_equal(lens_t.cpu().numpy(), lens_h if advance else lens0)

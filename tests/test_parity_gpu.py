@@ -14,6 +14,7 @@ import torch
 
 import oracle
 import paper_1911_02150_b200 as mqa
+from guards import Guarded
 from paper_1911_02150_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -57,16 +58,26 @@ def check_against_oracle(variant, q, K, V, lens_np, o, what, idx=None, chunk_byt
 
 
 def gpu_step(variant, q, K, V, lens_t, expect_status=0):
+    """One step through the C ABI.  The output, the workspace, the queries and lens sit between guard regions (a
+    pattern either side, checked after the kernels have run): a write beyond any of them fails the test even where
+    it would not fault."""
     b, h, _ = q.shape
-    o = torch.full((b, h, V.shape[-1]), float("nan"), dtype=torch.float32, device=q.device)
-    ws = mqa.alloc_workspace(b, h, K.shape[-2], q.device)
-    ws.fill_(0xFF)                                     # stale NaN bit patterns in the scratch
-    status = torch.zeros(1, dtype=torch.int32, device=q.device)
+    og = Guarded((b, h, V.shape[-1]), torch.float32, q.device)
+    og.t.fill_(float("nan"))
+    wsg = Guarded((max(16, mqa.workspace_bytes(b, h, K.shape[-2])),), torch.uint8, q.device)
+    wsg.t.fill_(0xFF)                                  # stale NaN bit patterns in the scratch
+    qg = Guarded(tuple(q.shape), q.dtype, q.device, like=q)
+    lg = Guarded(tuple(lens_t.shape), lens_t.dtype, q.device, like=lens_t)
+    sg = Guarded((1,), torch.int32, q.device)
+    sg.t.zero_()
     fn = mqa.mqa_decode_step if variant == "mqa" else mqa.mha_decode_step
-    fn(q, K, V, lens_t, o, ws, status)
+    fn(qg.t, K, V, lg.t, og.t, wsg.t, sg.t)
     torch.cuda.synchronize()
-    assert int(status.item()) == expect_status
-    return o
+    for g, name in ((og, "o"), (wsg, "workspace"), (qg, "q"), (lg, "lens"), (sg, "status")):
+        g.check(f"{variant} b={b} h={h}: {name}")
+    assert torch.equal(qg.t, q) and torch.equal(lg.t, lens_t)
+    assert int(sg.t.item()) == expect_status
+    return og.t
 
 
 def run_case(variant, b, h, m_max, lens_np, seed=0, sample=None):

@@ -243,7 +243,7 @@ def test_unknown_step_flags_are_refused():
     ws = mqa.alloc_workspace(b, h, m_max, DEV)
     from paper_1911_02150_b200 import binding
     rc = binding.lib().mqa_decode_append_step(inp["q"].data_ptr(), inp["K"].data_ptr(), inp["V"].data_ptr(), inp["k_new"].data_ptr(),
-                                              inp["v_new"].data_ptr(), lens_t.data_ptr(), 8, o.data_ptr(), ws.data_ptr(), ws.numel(),
+                                              inp["v_new"].data_ptr(), lens_t.data_ptr(), 16, o.data_ptr(), ws.data_ptr(), ws.numel(),
                                               None, b, h, m_max, 128, 128, None)
     assert rc == binding.ERR_INVALID_ARG
     torch.cuda.synchronize()
