@@ -4,8 +4,9 @@ Python face of the fp64 CPU oracle for the decode-attention hot path of multi-qu
 attention (arXiv 1911.02150).  Two independent restatements live here:
 
 * ``attention_oracle.c`` -- the bf16-boundary step functions (multi-query step of
-  Section 3, multi-head step of Section 2.4, the cache append, and the single-query
-  attention of Section 2.1), loaded through ``ctypes``;
+  Section 3, multi-head step of Section 2.4, the cache append, the single-query
+  attention of Section 2.1, and the attention lines of the batched multi-query function
+  of Section 3 under the autoregressive mask of Section 2.3), loaded through ``ctypes``;
 * ``paper_functions.py`` -- the paper's five layer functions *with* their projections,
   in numpy fp64, used by the pins that need the projections (incremental == causal).
 
@@ -52,6 +53,8 @@ def _load():
             fn = getattr(lib, name)
             fn.argtypes = [u16p, u16p, u16p, i32p, f64p, I, I, I, I, I]
             fn.restype = I
+        lib.oracle_mqa_batched_attention.argtypes = [u16p, u16p, u16p, i32p, f64p, I, I, I, I, I, I]
+        lib.oracle_mqa_batched_attention.restype = I
         lib.oracle_kv_cache_append.argtypes = [u16p, u16p, u16p, u16p, i32p, I, I, I, I, I, I]
         lib.oracle_kv_cache_append.restype = I
         lib.oracle_num_threads.restype = I
@@ -136,6 +139,34 @@ def mha_decode_step(q, K, V, lens) -> np.ndarray:
     if np.ndim(K) != 4:
         raise ValueError("the multi-head cache is [b, h, m_max, k]")
     return _decode("oracle_mha_decode_step", q, K, V, lens, lambda h: h)
+
+
+def mqa_batched_attention(Q, K, V, start=None) -> np.ndarray:
+    """Section 3, the attention lines of the batched multi-query function under the autoregressive mask of
+    Section 2.3: ``Q[b,h,n,k]``, shared ``K[b,m_max,k]``, ``V[b,m_max,v]`` (uint16 bf16 bits) -> ``O[b,h,n,v]`` fp64.
+    Query position t of sequence b is memory position ``start[b] + t`` and may look at positions up to its own
+    (``start`` None: zeros, the memory is the n positions of the queries themselves)."""
+    Q = np.ascontiguousarray(Q)
+    b, h, n, k = Q.shape
+    K = np.ascontiguousarray(K)
+    V = np.ascontiguousarray(V)
+    m_max, v = K.shape[-2], V.shape[-1]
+    Q = _u16(Q, (b, h, n, k))
+    K = _u16(K, (b, m_max, k))
+    V = _u16(V, (b, m_max, v))
+    st = None
+    if start is not None:
+        st = np.ascontiguousarray(start, dtype=np.int32)
+        assert st.shape == (b,)
+    O = np.empty((b, h, n, v), dtype=np.float64)
+    rc = _load().oracle_mqa_batched_attention(
+        _ptr(Q, ctypes.c_uint16), _ptr(K, ctypes.c_uint16), _ptr(V, ctypes.c_uint16),
+        None if st is None else _ptr(st, ctypes.c_int32), _ptr(O, ctypes.c_double), b, h, n, m_max, k, v)
+    if rc == 2:
+        raise ValueError("start[b] + n must lie within [n, m_max]")
+    if rc:
+        raise MemoryError("oracle scratch allocation failed")
+    return O
 
 
 def kv_cache_append(K, V, k_new, v_new, lens, advance: bool = True) -> int:

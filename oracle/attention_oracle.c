@@ -16,6 +16,11 @@
  *   oracle_mqa_decode_step        Section 3, the same three lines of the incremental
  *                                 multi-query step: all h heads of a sequence attend
  *                                 over the one shared K[b,:,:], V[b,:,:].
+ *   oracle_mqa_batched_attention  Section 3, the three attention lines of the batched multi-query
+ *                                 function (logits = einsum(bhnk,bmk->bhnm), weights =
+ *                                 softmax(logits + mask), O = einsum(bhnm,bmv->bhnv)) with the
+ *                                 mask of Section 2.3 for an autoregressive model: -inf where
+ *                                 a query would look at a later position, 0 elsewhere.
  *   oracle_kv_cache_append        Sections 2.4 / 3, the concatenation of the new
  *                                 token's key and value row on the m axis, done in
  *                                 place in a cache padded to m_max rows.
@@ -186,6 +191,63 @@ int oracle_mha_decode_step(const uint16_t* q, const uint16_t* K, const uint16_t*
                                L, k, v, scratch, o + ((size_t)bi * h + hh) * v);
         }
         free(scratch);
+    }
+    return failed;
+}
+
+/* Section 3 (multi-query, batched), the attention lines only: Q[b,h,n,k], K[b,m_max,k], V[b,m_max,v] as bf16
+ * bit patterns -> O[b,h,n,v] fp64.  Sequence bi has start[bi] + n memory positions (the n query positions are its
+ * last n: position t of the queries is memory position start[bi] + t; start may be NULL = all zero, i.e. m = n,
+ * memory and queries from the same positions).  The mask of Section 2.3 is written out as the paper states it: an
+ * additive term, -inf where memory position j lies after the query's own position, 0 where it does not; the softmax
+ * then runs over all start[bi] + n positions.  Rows beyond that are never read.  Returns 0, 1 on allocation
+ * failure, 2 if some sequence does not fit m_max. */
+int oracle_mqa_batched_attention(const uint16_t* Q, const uint16_t* K, const uint16_t* V, const int32_t* start,
+                                 double* O, int b, int h, int n, int m_max, int k, int v) {
+    for (int bi = 0; bi < b; ++bi) {
+        int st = start ? start[bi] : 0;
+        if (st < 0 || st + n > m_max) return 2;
+    }
+    int failed = 0;
+    long units = (long)b * h * n;
+#pragma omp parallel
+    {
+        double* logits = (double*)malloc((size_t)(m_max > 0 ? m_max : 1) * sizeof(double));
+        if (!logits) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 16)
+        for (long u = 0; u < units; ++u) {
+            if (!logits) continue;
+            long bi = u / ((long)h * n), hh = (u / n) % h, t = u % n;
+            int st = start ? start[bi] : 0;
+            int m = st + n;                                    /* memory positions of this sequence */
+            const uint16_t* q_row = Q + (((size_t)bi * h + hh) * n + t) * k;
+            const uint16_t* Kseq = K + (size_t)bi * m_max * k;
+            const uint16_t* Vseq = V + (size_t)bi * m_max * v;
+            for (int j = 0; j < m; ++j) {
+                double s = 0.0;
+                for (int c = 0; c < k; ++c) s += widen_bf16(q_row[c]) * widen_bf16(Kseq[(size_t)j * k + c]);
+                double mask = (j > st + t) ? -INFINITY : 0.0;  /* a later position is illegal */
+                logits[j] = s + mask;
+            }
+            double top = -INFINITY;
+            for (int j = 0; j < m; ++j)
+                if (logits[j] > top) top = logits[j];
+            double Z = 0.0;
+            for (int j = 0; j < m; ++j) {
+                logits[j] = exp(logits[j] - top);              /* exp(-inf) = 0 for the masked positions */
+                Z += logits[j];
+            }
+            double* out = O + (((size_t)bi * h + hh) * n + t) * v;
+            for (int c = 0; c < v; ++c) {
+                double s = 0.0;
+                for (int j = 0; j < m; ++j) s += logits[j] * widen_bf16(Vseq[(size_t)j * v + c]);
+                out[c] = s / Z;
+            }
+        }
+        free(logits);
     }
     return failed;
 }

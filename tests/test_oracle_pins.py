@@ -555,3 +555,85 @@ def test_layer_oracle_empty_and_full_sequences():
     # a single row: the output is that value row, whatever the query
     o_single = f(ls.f64_to_bf16_bits(f(vb[0])))
     np.testing.assert_allclose(y[0], np.einsum("hv,hdv->d", np.tile(o_single, (Pq.shape[0], 1)), f(Po)), rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------- the batched multi-query attention lines (Section 3) under the causal mask
+def _batched_inputs(b, h, n, m_max, k, v, seed):
+    r = rng(seed)
+    Qb, Qf = bf16_bits(r.normal(size=(b, h, n, k)) * k ** -0.5)
+    Kb, Kf = bf16_bits(r.normal(size=(b, m_max, k)))
+    Vb, Vf = bf16_bits(r.normal(size=(b, m_max, v)))
+    return (Qb, Kb, Vb), (Qf, Kf, Vf)
+
+
+def test_batched_attention_vs_brute_einsum_with_the_additive_mask():
+    """logits = einsum(bhnk,bmk->bhnm), softmax(logits + mask), einsum(bhnm,bmv->bhnv), written out index by
+    index, with the -inf mask of Section 2.3 built here from its definition (a later position is illegal)."""
+    b, h, n, k, v = 2, 3, 4, 3, 2
+    start = np.array([0, 2], np.int32)
+    m_max = 7
+    (Qb, Kb, Vb), (Q, K, V) = _batched_inputs(b, h, n, m_max, k, v, seed=301)
+    got = oracle.mqa_batched_attention(Qb, Kb, Vb, start)
+    for s in range(b):
+        m = int(start[s]) + n
+        mask = np.zeros((1, h, n, m))
+        for t in range(n):
+            for j in range(m):
+                if j > start[s] + t:
+                    mask[0, :, t, j] = -np.inf
+        w = brute_softmax_last(brute_einsum("bhnk,bmk->bhnm", Q[s:s + 1], K[s:s + 1, :m]) + mask)
+        ref = brute_einsum("bhnm,bmv->bhnv", w, V[s:s + 1, :m])
+        np.testing.assert_allclose(got[s:s + 1], ref, rtol=1e-12, atol=1e-14)
+    # start = None means zeros
+    np.testing.assert_array_equal(oracle.mqa_batched_attention(Qb, Kb, Vb), oracle.mqa_batched_attention(Qb, Kb, Vb, np.zeros(b, np.int32)))
+
+
+def test_batched_attention_rows_are_the_incremental_steps():
+    """Section 2.4's reading of autoregressive decoding: query position t attends up to and including its own
+    position, so row t of the batched function under the causal mask is the incremental step over start + t + 1 rows."""
+    b, h, n, m_max, k, v = 3, 4, 9, 40, 128, 128
+    start = np.array([0, 5, 31], np.int32)
+    (Qb, Kb, Vb), _ = _batched_inputs(b, h, n, m_max, k, v, seed=302)
+    got = oracle.mqa_batched_attention(Qb, Kb, Vb, start)
+    for t in range(n):
+        step = oracle.mqa_decode_step(np.ascontiguousarray(Qb[:, :, t]), Kb, Vb, (start + t + 1).astype(np.int32))
+        np.testing.assert_allclose(got[:, :, t], step, rtol=1e-13, atol=1e-15)
+
+
+def test_batched_attention_is_the_papers_function_between_its_projections():
+    """With projections chosen so that they pass their input through (d = k = v, one-hot P_q, P_k, P_v, P_o), the
+    paper's MultiqueryAttentionBatched is the attention lines alone: Y[b,n,:] = sum over heads of O[b,h,n,:]."""
+    b, h, n, d = 2, 3, 5, 4
+    r = rng(303)
+    Xb, X = bf16_bits(r.normal(size=(b, n, d)))
+    eye = np.eye(d)
+    P_q = np.stack([eye * 2.0 ** i for i in range(h)])      # head i scales the queries by 2^i (exact in bf16)
+    P_k, P_v = eye, eye
+    P_o = np.stack([eye for _ in range(h)])
+    Y = pf.multiquery_attention_batched(X, X, _causal_mask(b, h, n), P_q, P_k, P_v, P_o)
+    Qb, _ = bf16_bits(np.einsum("bnd,hdk->bhnk", X, P_q))
+    O = oracle.mqa_batched_attention(Qb, Xb, Xb)
+    np.testing.assert_allclose(O.sum(axis=1), Y, rtol=1e-12, atol=1e-13)
+
+
+def test_batched_attention_library_sdpa_causal_fp64():
+    b, h, n, k, v = 2, 3, 37, 128, 128
+    (Qb, Kb, Vb), (Q, K, V) = _batched_inputs(b, h, n, n, k, v, seed=304)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q), torch.from_numpy(K)[:, None].expand(b, h, n, k), torch.from_numpy(V)[:, None].expand(b, h, n, v),
+        is_causal=True, scale=1.0).numpy()
+    np.testing.assert_allclose(oracle.mqa_batched_attention(Qb, Kb, Vb), ref, rtol=1e-12, atol=1e-14)
+
+
+def test_batched_attention_never_reads_beyond_a_sequences_memory_and_refuses_what_does_not_fit():
+    b, h, n, m_max, k, v = 2, 2, 6, 20, 8, 8
+    start = np.array([3, 14], np.int32)
+    (Qb, Kb, Vb), _ = _batched_inputs(b, h, n, m_max, k, v, seed=305)
+    ref = oracle.mqa_batched_attention(Qb, Kb, Vb, start)
+    Kp, Vp = Kb.copy(), Vb.copy()
+    for s in range(b):
+        Kp[s, start[s] + n:] = 0x7FC0                       # NaN beyond the memory
+        Vp[s, start[s] + n:] = 0x7FC0
+    np.testing.assert_array_equal(oracle.mqa_batched_attention(Qb, Kp, Vp, start), ref)
+    with pytest.raises(ValueError):
+        oracle.mqa_batched_attention(Qb, Kb, Vb, np.array([3, 15], np.int32))
