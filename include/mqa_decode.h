@@ -19,7 +19,9 @@
  *     are dense, row-major, innermost axis last.  q, K, V, k_new, v_new, o and the workspace
  *     must be 16-byte aligned; lens and status 4-byte aligned.
  *   - K, V, q, k_new, v_new hold bf16; o holds fp32; lens holds int32.
- *   - k == v == 128 is the only supported head width; h >= 1.
+ *   - k == v == 128 is the only supported head width; h >= 1.  More than 64 query rows per sequence
+ *     (many heads; or beams x heads over one shared memory, passed as h = beams * heads) run on the
+ *     tensor cores as groups of 64 rows over the same cache.
  *   - `stream` is a cudaStream_t passed as a plain pointer (NULL = the legacy default stream).
  *     Calls only enqueue work on it: they never synchronise, never allocate device memory and
  *     never free anything.  The launch configuration is chosen from the integer arguments and
@@ -325,6 +327,29 @@ int mqa_layer_decode_step(const void* x, const void* P_q, const void* P_k, const
 
 /* mqa_layer_workspace_bytes -- scratch mqa_layer_decode_step needs (0 for invalid or unsupported sizes). Host-only. */
 size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v);
+
+/*
+ * mqa_prefill_attention -- the three attention lines of the batched multi-query function of Section 3
+ * (MultiqueryAttentionBatched: logits = einsum(bhnk,bmk->bhnm), weights = softmax(logits + mask),
+ * O = einsum(bhnm,bmv->bhnv)) for n query positions per sequence at once, under the mask that Section 2.3
+ * gives for an autoregressive model: -inf where a query would look at a position after its own.
+ *
+ *   Q      [b, h, n, k] bf16                    K, V   [b, m_max, k], [b, m_max, v] bf16 (read only)
+ *   start  [b] int32 or NULL (all zero): the memory position of each sequence's first query.  Query t of
+ *          sequence b is memory position start[b] + t and attends over rows 0 .. start[b] + t of that sequence's
+ *          K and V (so start[b] + n <= m_max must hold; with start = 0 and n rows in the cache this is the
+ *          paper's M = X case, the processing of a whole prompt).  A negative start[b] is taken as an empty memory
+ *          for that sequence (zeros) and flagged LEN_CLAMPED, like a bad lens.
+ *   O      [b, h, n, v] fp32, written           status   optional; LEN_CLAMPED, PIPELINE_TIMEOUT
+ *   workspace   at least mqa_prefill_workspace_bytes(b, h, n, m_max, k, v) bytes; as for mqa_decode_step.
+ * Each run of 64 consecutive positions of one head is given to the persistent tensor-core kernel as 64 query rows over
+ * the cache rows up to its last position (rows beyond are not fetched at all; the last 63 are masked per column),
+ * at most 1024 such runs per launch.  Supported: k = v = 128, n a multiple of 64 (MQA_ERR_UNSUPPORTED otherwise).
+ */
+int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int32_t* start, float* O,
+                          void* workspace, size_t workspace_bytes, int32_t* status,
+                          int b, int h, int n, int m_max, int k, int v, mqa_stream_t stream);
+size_t mqa_prefill_workspace_bytes(int b, int h, int n, int m_max, int k, int v);
 
 /*
  * mqa_set_wait_limit_cycles -- how long, in SM clock cycles, a kernel of this library waits for one of its own

@@ -25,7 +25,7 @@ EXPORTS = (
     "kv_cache_append", "mqa_decode_step", "mha_decode_step",
     "mqa_decode_step_split", "mqa_decode_step_combine",
     "mha_decode_step_split", "mha_decode_step_combine",
-    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_set_wait_limit_cycles", "mqa_status_string", "mqa_decode_step_noalloc",
+    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_set_wait_limit_cycles", "mqa_prefill_attention", "mqa_prefill_workspace_bytes", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
     "mqa_layer_decode_step", "mqa_layer_workspace_bytes", "mqa_decode_local_step",
     "mqa_decode_append_step_host", "mqa_host_staging_bytes",
@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.mqa_plan_splits.restype = I
         L.mqa_plan_kernel_name.argtypes = [I, I, I, I, I, I, I]
         L.mqa_plan_kernel_name.restype = ctypes.c_char_p
+        L.mqa_prefill_attention.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, I, I, I, I, I, I, vp]
+        L.mqa_prefill_attention.restype = I
+        L.mqa_prefill_workspace_bytes.argtypes = [I, I, I, I, I, I]
+        L.mqa_prefill_workspace_bytes.restype = sz
         L.mqa_set_wait_limit_cycles.argtypes = [ctypes.c_longlong]
         L.mqa_set_wait_limit_cycles.restype = I
         L.mqa_status_string.argtypes = [I]
@@ -391,6 +395,33 @@ def mqa_decode_local_step(q, K, V, k_new, v_new, pos, o, status=None, advance: b
                                          _ptr(o), _ptr(status), b, h, window, k, v, _stream(stream))
     _check(rc, "mqa_decode_local_step")
     return o
+
+
+def prefill_workspace_bytes(b: int, h: int, n: int, m_max: int, k: int = 128, v: int = 128) -> int:
+    return int(lib().mqa_prefill_workspace_bytes(b, h, n, m_max, k, v))
+
+
+def mqa_prefill_attention(Q, K, V, O, workspace, start=None, status=None, stream=None):
+    """The attention lines of the batched multi-query function under the autoregressive mask: ``Q[b,h,n,k]`` bf16 over
+    the shared ``K[b,m_max,k]``, ``V[b,m_max,v]``; query t of sequence b is memory position ``start[b] + t`` (``start``
+    None: zeros) and attends over the rows up to its own; ``O[b,h,n,v]`` fp32 is written."""
+    b, h, n, k = Q.shape
+    m_max, v = K.shape[-2], V.shape[-1]
+    _need(Q, torch.bfloat16, (b, h, n, k), "Q")
+    _need(K, torch.bfloat16, (b, m_max, k), "K")
+    _need(V, torch.bfloat16, (b, m_max, v), "V")
+    _need(O, torch.float32, (b, h, n, v), "O")
+    if start is not None:
+        _need(start, torch.int32, (b,), "start")
+    if status is not None:
+        _need(status, torch.int32, (1,), "status")
+    s = torch.cuda.current_stream(Q.device) if stream is None else stream
+    with _OnDevice(Q.device):
+        rc = lib().mqa_prefill_attention(Q.data_ptr(), K.data_ptr(), V.data_ptr(), None if start is None else start.data_ptr(),
+                                         O.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                         None if status is None else status.data_ptr(), b, h, n, m_max, k, v, s.cuda_stream)
+    _check(rc, "mqa_prefill_attention")
+    return O
 
 
 def host_staging_bytes(b: int, h: int, k: int = 128, v: int = 128) -> int:

@@ -51,6 +51,9 @@ struct Plan {
     int grid = 0;         // persistent kernel: number of CTAs
     Kernel kernel = Kernel::kSimt;
     bool merge_in_kernel = false;   // tcgen05 plan: pieces merged by the CTA that delivers a sequence's last one (single launch)
+    int groups = 1;       // tcgen05 plan for more than 64 query rows per sequence: groups of 64 rows, each a sequence of the
+                          // schedule over the same cache (then b = sequences x groups and h = 64: see QueryGroups)
+    int h_total = 0;      // query rows per sequence as the caller counts them
     bool stream() const { return kernel == Kernel::kUmma; }
 };
 
@@ -133,9 +136,23 @@ Plan plan_stream(int b, int h, int m_max) {
 }
 
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
-    // heads beyond two 16-row tensor-core tiles, or a row space too large for the 32-bit TMA
-    // coordinates, go to the general CUDA-core kernel
-    if (!(multi_query && h <= 64 && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
+    // a row space too large for the 32-bit TMA coordinates goes to the general CUDA-core kernel
+    if (!(multi_query && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
+    if (h > kGroupRows) {
+        // more query rows than one tile of the tensor-core kernel holds (beams x heads, many heads): groups of 64
+        // rows, each a sequence of the persistent kernel's schedule over the same cache
+        const int groups = (h + kGroupRows - 1) / kGroupRows;
+        const long long seqs = (long long)b * groups;
+        const long long tiles = seqs * ((m_max + kTileRows - 1) / kTileRows);
+        if (seqs <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256 &&
+            (long long)b * h < 0x7fffffffLL) {
+            Plan p = plan_stream((int)seqs, kGroupRows, m_max);
+            p.groups = groups;
+            p.h_total = h;
+            return p;
+        }
+        return plan_simt(b, h, m_max);
+    }
     // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     if (b <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256) return plan_stream(b, h, m_max);
@@ -330,16 +347,19 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
 
 constexpr size_t kL2KeepBytes = 64u << 20;   // K and V together: half of the 126 MB L2
 constexpr int kEarlyTestWithhold = 1 << 8;    // rides on `early`: MQA_STEP_TEST_WITHHOLD_COPY
-std::atomic<int> g_umma_opt_in[kMaxDevices][9];
+std::atomic<int> g_umma_opt_in[kMaxDevices][10];
 
-template <int HP, bool FUSED, bool GUESS = false>
+// b, h: the caller's sequences and query rows per sequence (the kernel is given the plan's: sequences x groups, 64 rows
+// each, where the plan has groups).  grp_in: the groups of a launch of the batched form; otherwise derived from the plan.
+template <int HP, bool FUSED, bool GUESS = false, bool CAUSAL = false>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
                 const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
-                int early = 0) {
+                int early = 0, const QueryGroups* grp_in = nullptr, long long q_rows = 0) {
     using Cfg = UmmaCfg<HP>;
-    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS>;
-    constexpr int kSlot = (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
+    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS, CAUSAL>;
+    constexpr int kSlot = CAUSAL ? 9 : (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
+    const QueryGroups grp = grp_in ? *grp_in : QueryGroups{p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0, 0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
@@ -357,10 +377,10 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
         fa.V = static_cast<uint4*>(const_cast<void*>(V));
     }
     alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub, map_q;
-    const long long rows = (long long)b * m_max;
+    const long long rows = (long long)b * m_max;             // (b caches, however many schedule sequences look at each)
     if (!encode_cache_map(&map_k, K, rows, kUmmaStageRows) || !encode_cache_map(&map_v, V, rows, kUmmaStageRows) ||
         !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows) ||
-        !encode_cache_map(&map_q, q, (long long)b * h, HP))
+        !encode_cache_map(&map_q, q, q_rows > 0 ? q_rows : (long long)b * h, HP))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     // a cache that cannot stay in L2 from one step to the next is streamed through it with the evict-first policy
@@ -370,10 +390,10 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     // portable sizes): with sequences of equal length a cluster then holds exactly one sequence's pieces and merges
     // them through its shared memory (the kernel decides from lens; otherwise the clusters change nothing).
     unsigned cluster = 1;
-    if (merge && p.grid % b == 0 && p.grid / b >= 2 && p.grid / b <= 8) cluster = (unsigned)(p.grid / b);
+    if (merge && p.grid % p.b == 0 && p.grid / p.b >= 2 && p.grid / p.b <= 8) cluster = (unsigned)(p.grid / p.b);
     launch_dependent_clusters(cluster, kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub,
-                              map_v_sub, map_q, lens, o, w.span, w.ml, w.acc, status, b, h, m_max, share_magic(p.grid), fa,
-                              merge ? w.ctrl : nullptr, lens_advance, early, read_once);
+                              map_v_sub, map_q, lens, o, w.span, w.ml, w.acc, status, p.b, p.h, m_max, share_magic(p.grid), fa,
+                              merge ? w.ctrl : nullptr, lens_advance, early, read_once, grp);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -385,13 +405,13 @@ int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, 
 #define MQA_UMMA_ARGS p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, early
     if constexpr (FUSED) {
         if ((early & ~kEarlyTestWithhold) >= 2) {           // the kernels that carry the code for copies started on a guess
-            if (h <= 16) return launch_umma<16, true, true>(MQA_UMMA_ARGS);
-            if (h <= 32) return launch_umma<32, true, true>(MQA_UMMA_ARGS);
+            if (p.h <= 16) return launch_umma<16, true, true>(MQA_UMMA_ARGS);
+            if (p.h <= 32) return launch_umma<32, true, true>(MQA_UMMA_ARGS);
             return launch_umma<64, true, true>(MQA_UMMA_ARGS);
         }
     }
-    if (h <= 16) return launch_umma<16, FUSED>(MQA_UMMA_ARGS);
-    if (h <= 32) return launch_umma<32, FUSED>(MQA_UMMA_ARGS);
+    if (p.h <= 16) return launch_umma<16, FUSED>(MQA_UMMA_ARGS);
+    if (p.h <= 32) return launch_umma<32, FUSED>(MQA_UMMA_ARGS);
     return launch_umma<64, FUSED>(MQA_UMMA_ARGS);
 #undef MQA_UMMA_ARGS
 }
@@ -422,6 +442,23 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
     return launch_status();
 }
 
+// Second pass of the persistent kernel: one CTA per (schedule sequence, query row) merges the sequence's pieces.
+int launch_stream_combine(const Plan& p, const void* workspace, float* o, int32_t* lens_advance, int m_max, cudaStream_t stream,
+                          const QueryGroups& grp) {
+    const StreamWorkspace w = stream_workspace(p, workspace);
+    const unsigned grid = (unsigned)((size_t)p.b * p.h);
+    if (p.n_splits <= kCombineEager)
+        launch_dependent(stream_combine_kernel<1>, grid, kHeadDim, 0, stream, w.span, w.ml, w.acc, o, p.b, p.h, lens_advance,
+                         m_max, share_magic(p.grid), grp);
+    else if (p.n_splits <= 4 * kCombineEager)
+        launch_dependent(stream_combine_kernel<4>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o, p.b, p.h,
+                         lens_advance, m_max, share_magic(p.grid), grp);
+    else
+        launch_dependent(stream_combine_kernel<kCombineManyGroups>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
+                         p.b, p.h, lens_advance, m_max, share_magic(p.grid), grp);
+    return launch_status();
+}
+
 int run_combine(bool multi_query, const int32_t* lens, float* o, const void* workspace, size_t workspace_bytes,
                 int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0,
                 int32_t* lens_advance = nullptr, bool fused = false) {
@@ -432,18 +469,8 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     int rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
     if (p.stream()) {
-        const StreamWorkspace w = stream_workspace(p, workspace);
-        const unsigned grid = (unsigned)((size_t)b * h);
-        if (p.n_splits <= kCombineEager)
-            launch_dependent(stream_combine_kernel<1>, grid, kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h, lens_advance,
-                             m_max, share_magic(p.grid));
-        else if (p.n_splits <= 4 * kCombineEager)
-            launch_dependent(stream_combine_kernel<4>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o, b, h,
-                             lens_advance, m_max, share_magic(p.grid));
-        else
-            launch_dependent(stream_combine_kernel<kCombineManyGroups>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
-                             b, h, lens_advance, m_max, share_magic(p.grid));
-        return launch_status();
+        const QueryGroups grp = {p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0, 0};
+        return launch_stream_combine(p, workspace, o, lens_advance, m_max, stream, grp);
     }
     if (p.n_splits <= 1) return MQA_OK;
     const float2* part_ml = partials_ml(workspace);
@@ -871,6 +898,56 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
     const Plan p = make_plan(multi_query != 0, b, h, m_max);
     if (chunk_rows) *chunk_rows = p.chunk_rows;
     return p.n_splits;
+}
+
+// ---- the batched form (prefill): launches of at most kStreamMaxSeqs groups of 64 query positions --------------
+static Plan prefill_plan(long long groups_in_launch, int m_max) { return plan_stream((int)groups_in_launch, kGroupRows, m_max); }
+
+static int check_prefill_dims(int b, int h, int n, int m_max, int k, int v) {
+    if (!dims_ok(b, h, m_max) || n <= 0 || k <= 0 || v <= 0) return MQA_ERR_INVALID_ARG;
+    if (k != kHeadDim || v != kHeadDim || n % kGroupRows != 0 || n > m_max) return MQA_ERR_UNSUPPORTED;
+    if ((long long)b * m_max >= 0x7fffffffLL || (long long)b * h * n >= 0x7fffffffLL || sm_count() > 256) return MQA_ERR_UNSUPPORTED;
+    return MQA_OK;
+}
+
+size_t mqa_prefill_workspace_bytes(int b, int h, int n, int m_max, int k, int v) {
+    if (check_prefill_dims(b, h, n, m_max, k, v) != MQA_OK) return 0;
+    const long long total = (long long)b * h * (n / kGroupRows);
+    const long long full = total < kStreamMaxSeqs ? total : kStreamMaxSeqs;
+    size_t need = plan_workspace_bytes(prefill_plan(full, m_max));
+    if (total > kStreamMaxSeqs && total % kStreamMaxSeqs != 0) {
+        const size_t last = plan_workspace_bytes(prefill_plan(total % kStreamMaxSeqs, m_max));
+        need = last > need ? last : need;
+    }
+    return need;
+}
+
+int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int32_t* start, float* O, void* workspace,
+                          size_t workspace_bytes, int32_t* status, int b, int h, int n, int m_max, int k, int v,
+                          mqa_stream_t stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!Q || !K || !V || !O || !workspace) return MQA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(workspace) || !aligned4(start) ||
+        !aligned4(status))
+        return MQA_ERR_INVALID_ARG;
+    const int rc = check_prefill_dims(b, h, n, m_max, k, v);
+    if (rc) return rc;
+    if (workspace_bytes < mqa_prefill_workspace_bytes(b, h, n, m_max, k, v)) return MQA_ERR_WORKSPACE_TOO_SMALL;
+    const int per_head = n / kGroupRows;                       // groups of 64 positions per head
+    const long long total = (long long)b * h * per_head;
+    for (long long first = 0; first < total; first += kStreamMaxSeqs) {
+        const long long count = total - first < kStreamMaxSeqs ? total - first : kStreamMaxSeqs;
+        const Plan p = prefill_plan(count, m_max);
+        const QueryGroups grp = {h * per_head, h * n, (int)first, per_head};
+        int err = launch_umma<64, false, false, true>(p, Q, K, V, start, O, workspace, status, b, h, m_max, stream, p.merge_in_kernel,
+                                                      nullptr, nullptr, nullptr, 0, &grp, (long long)b * h * n);
+        if (err) return err;
+        if (!p.merge_in_kernel) {
+            err = launch_stream_combine(p, workspace, O, nullptr, m_max, stream, grp);
+            if (err) return err;
+        }
+    }
+    return MQA_OK;
 }
 
 int mqa_set_wait_limit_cycles(long long cycles) {

@@ -298,11 +298,12 @@ __device__ __forceinline__ float warp_reduce_scatter(float (&v)[N], int lane) {
 
 // All the softmax threads of the CTA that delivered the last piece of sequence s: o[s] = the pieces held by
 // the CTAs lo..hi (those with a share of the line), merged in CTA order.  8 threads per head, 16 columns each.
+// o_rows: the sequence's rows of o (its first query row onwards), n_rows of them (h, or fewer in a last group of rows).
 __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
-                                                   float* __restrict__ o, int s, int h, int lo, int hi, int T,
+                                                   float* __restrict__ o_rows, int n_rows, int s, int h, int lo, int hi, int T,
                                                    unsigned long long magic, int tid) {
     const int g8 = tid & 7;
-    for (int head = tid >> 3; head < h; head += kUmmaSoftmaxThreads / 8) {
+    for (int head = tid >> 3; head < n_rows; head += kUmmaSoftmaxThreads / 8) {
         float top = -INFINITY, den = 0.f;
         float4 num[4];
 #pragma unroll
@@ -345,7 +346,7 @@ __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__
             top = top_new;
         }
         const float inv = 1.f / den;
-        float4* dst = reinterpret_cast<float4*>(o + ((size_t)s * h + head) * kHeadDim) + g8;
+        float4* dst = reinterpret_cast<float4*>(o_rows + (size_t)head * kHeadDim) + g8;
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4)
             dst[q4 * 8] = make_float4(num[q4].x * inv, num[q4].y * inv, num[q4].z * inv, num[q4].w * inv);
@@ -354,7 +355,8 @@ __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__
 
 // HP = head rows of the Q tile (h rounded up to 16, 32 or 64).  GUESS: built with the code that starts copies on a
 // guess before the wait (GUESS && early >= 2 below); kernels without it take early 0 or 1 only.
-template <int HP, bool FUSED, bool GUESS = false>
+// CAUSAL: built with the mask per column of the batched form (QueryGroups::causal_every != 0).
+template <int HP, bool FUSED, bool GUESS = false, bool CAUSAL = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                               const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
@@ -363,7 +365,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
                               int b, int h, int m_max, unsigned long long magic, const FusedArgs fa,
                               unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int early_arg,
-                              int read_once) {
+                              int read_once, const QueryGroups grp) {
     using Cfg = UmmaCfg<HP>;
     const int early = GUESS ? early_arg : (early_arg == 1 ? 1 : 0);
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
@@ -432,11 +434,12 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     // new key row, lane l >= 16 of the new value row.  The row is loaded when its segment begins and stored (and
     // made visible to the copy engine) before the stage that contains it is fetched.
     auto row_load = [&](int s) -> uint4 {
-        const uint4* src = (lane < 16 ? fa.k_new : fa.v_new) + (size_t)s * (kRowBytes / 16) + (lane & 15);
+        const uint4* src = (lane < 16 ? fa.k_new : fa.v_new) + (size_t)group_kv(grp, s) * (kRowBytes / 16) + (lane & 15);
         return __ldg(src);
     };
     auto row_store = [&](int s, int new_row, uint4 value) {
-        uint4* dst = (lane < 16 ? fa.K : fa.V) + ((size_t)s * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
+        // (groups of query rows over one cache each store the row before they fetch it: the same bytes)
+        uint4* dst = (lane < 16 ? fa.K : fa.V) + ((size_t)group_kv(grp, s) * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
         *dst = value;
         asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
         __syncwarp();
@@ -453,14 +456,14 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // the sequence's head rows (rows past h belong to the next sequence or read as zero: their
         // columns of S^T and O^T are never stored)
         if (lane == 0) mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
-        tma_load_2d(q_s + qi * Cfg::kQBytes + lane * (Cfg::kQBytes / 2), &map_q, lane * kBoxCols, s * h, q_full + qi * 8);
+        tma_load_2d(q_s + qi * Cfg::kQBytes + lane * (Cfg::kQBytes / 2), &map_q, lane * kBoxCols, (int)group_row0(grp, s, h), q_full + qi * 8);
     };
     const uint64_t stream_policy = l2_stream_policy((read_once & 1) != 0);
     const bool withhold = (read_once & 2) != 0;             // for tests: one copy is never started, so that a wait runs out
     auto issue_stage = [&](int s, int u, int hi, int j) {   // lanes 0 to 3
         const int kv = lane >> 1, half = lane & 1;          // the K rows, then the V rows, each into its own ring
         const int nsub = min(kSubs, hi - u);
-        const int y = s * m_max + u * kTileRows;
+        const int y = group_kv(grp, s) * m_max + u * kTileRows;
         const int n_slots = kv ? NV : NK;
         const int slot = j % n_slots;
         const uint32_t full = (kv ? v_full : k_full) + slot * 8;
@@ -547,7 +550,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 Segment g = {};
                 int r = 0;
                 bool strided = false;
-                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r, cl, crank, kSubs, &strided);
+                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r, cl, crank, kSubs, &strided, grp);
                 if (before && lane == 0) TS(8);
                 if (GUESS && before && early == 3) g.lo += kSubs;    // for tests: a guess that is one stage off
                 if (!before && GUESS && early >= 2) {
@@ -608,7 +611,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         // CTAs: 26.9 us per step without, 26.2 / 26.0 / 26.5 / 27.2 us with 1 / 2 / 3 / 4 stages)
                         int u = g0.lo + pre_issued * ust;
                         for (int p = 0; p < kGuessL2Stages && (u + kSubs) * kTileRows <= stop_row && u + kSubs <= g0.hi; ++p, u += ust) {
-                            tma_prefetch_l2_2d((lane >> 1) ? &map_v : &map_k, (lane & 1) * kBoxCols, g0.s * m_max + u * kTileRows);
+                            tma_prefetch_l2_2d((lane >> 1) ? &map_v : &map_k, (lane & 1) * kBoxCols, group_kv(grp, g0.s) * m_max + u * kTileRows);
                         }
                     }
                 }
@@ -632,7 +635,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 
     tc_fence_before();
     const SharePlan plan = stream_plan<FUSED, kUmmaThreads, kUmmaBoundaryPenalty>(lens, o, status, b, h, m_max, appending, magic, prefix,
-                                                            rows_of, plan_sm, kUmmaProducerWarp);
+                                                            rows_of, plan_sm, kUmmaProducerWarp, grp);
     const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
     tc_fence_after();
     // sequences of equal tile counts in a launch made of clusters: strided stages, pieces merged through the cluster
@@ -702,7 +705,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             if (won) {
                 if (lens_advance)
                     for (int s = lane; s < b; s += 32)
-                        if (rows_of[s] & kAppendBit) lens_advance[s] = rows_of[s] & (kAppendBit - 1);
+                        if (rows_of[s] & kAppendBit) lens_advance[group_kv(grp, s)] = rows_of[s] & (kAppendBit - 1);
             }
         }
     } else if (warp == kUmmaSWarp) {
@@ -809,7 +812,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             bool pend = false;
             bool prev_hilo = false;                         // the stage before wrote hi and lo parts of P
             float* pend_dst = nullptr;
-            int pend_par = 0, pend_j = 0, pend_s = 0;
+            int pend_par = 0, pend_j = 0, pend_s = 0, pend_rows = 0;
             bool pend_whole = false;
             auto read_out = [&]() {
                 // O^T[column t][head] of the finished segment -> o (divided by the sum) or its partial slot
@@ -828,7 +831,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < CH; ++i)
-                        if (head0 + c * CH + i < h) pend_dst[(size_t)(head0 + c * CH + i) * kHeadDim] = __uint_as_float(y[i]) * inv[i];
+                        if (head0 + c * CH + i < pend_rows) pend_dst[(size_t)(head0 + c * CH + i) * kHeadDim] = __uint_as_float(y[i]) * inv[i];
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -878,6 +881,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     const int fetched = min(kSubs, g.hi - u) * kTileRows;
                     const int valid = min(fetched, L - u * kTileRows);
                     const bool row_ok = t < valid;
+                    // batched form: column c of the group is query position (last position) - 63 + c and looks at the
+                    // rows up to its own, i.e. at this thread's row iff (rows from it to the end) + c >= 64
+                    const int to_end = L - (u * kTileRows + t);
                     if (ok) ok = mbar_wait(s_ready + sb * 8, (j >> 1) & 1);
                     if (tid == 0) ST(j, 2);
                     tc_fence_after();
@@ -903,7 +909,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         const float mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            x[i + e] = row_ok ? __fmul_rn(__uint_as_float(xr[i + e]), kLog2e) : -INFINITY;   // select, never multiply
+                            const bool seen = !CAUSAL || to_end + head0 + i + e >= kGroupRows;
+                            x[i + e] = row_ok && seen ? __fmul_rn(__uint_as_float(xr[i + e]), kLog2e) : -INFINITY;   // select, never multiply
                             lead = fmaxf(lead, x[i + e] - mv[e]);           // (-inf) - (-inf) = NaN is ignored by fmaxf
                         }
                     }
@@ -924,6 +931,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                             float m_new = m_old;
 #pragma unroll
                             for (int w = 0; w < 4; ++w) m_new = fmaxf(m_new, red_m[w * HP + tid]);   // finite: the stage has a valid row
+                            // (batched form: a column may see none of a piece's rows; a finite stand-in gives it weight 0)
+                            if (CAUSAL) m_new = fmaxf(m_new, -1e30f);
                             f_sm[tid] = fast_exp2(m_old - m_new);            // 0 on the first stage, 1 if unchanged
                             m_sm[tid] = m_new;
                         }
@@ -1035,7 +1044,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 }
                 piece_left = true;
                 pend = true;
-                pend_dst = (whole ? o + (size_t)s * h * kHeadDim : via_cluster ? piece_acc : part_acc + slot * h * kHeadDim) + t;
+                pend_dst = (whole ? o + (size_t)group_row0(grp, s, h) * kHeadDim : via_cluster ? piece_acc : part_acc + slot * h * kHeadDim) + t;
+                pend_rows = whole ? group_rows(grp, s, h) : h;
                 pend_par = par;
                 pend_j = j - 1;
                 pend_s = s;
@@ -1053,7 +1063,9 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 const int n_merge = merge_sm[0];
                 if (n_merge > 0) __threadfence();
                 for (int k = 0; k < n_merge; ++k)
-                    merge_sequence_pieces(part_ml, part_acc, o, merge_sm[1 + 3 * k], h, merge_sm[2 + 3 * k], merge_sm[3 + 3 * k], T, magic, tid);
+                    merge_sequence_pieces(part_ml, part_acc, o + (size_t)group_row0(grp, merge_sm[1 + 3 * k], h) * kHeadDim,
+                                          group_rows(grp, merge_sm[1 + 3 * k], h), merge_sm[1 + 3 * k], h, merge_sm[2 + 3 * k],
+                                          merge_sm[3 + 3 * k], T, magic, tid);
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
@@ -1100,7 +1112,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     num.z = fmaf(w, a[c].z, num.z); num.w = fmaf(w, a[c].w, num.w);
                 }
                 const float inv = 1.f / den;
-                *reinterpret_cast<float4*>(o + ((size_t)s * h + head) * kHeadDim + c4 * 4) =
+                if (head >= group_rows(grp, s, h)) break;
+                *reinterpret_cast<float4*>(o + ((size_t)group_row0(grp, s, h) + head) * kHeadDim + c4 * 4) =
                     make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
             }
         }

@@ -73,6 +73,8 @@ CASES = [
     (40, 16, 1500), (160, 32, 333), (300, 8, 200), (37, 32, 4000), (64, 5, 777),
     # ... the persistent tcgen05 kernel (h > 32) ...
     (40, 48, 1500), (33, 64, 2100),
+    # ... more than 64 query rows per sequence: groups of 64 rows over the same cache, each storing the new row ...
+    (24, 128, 2048), (20, 96, 1500),
     # ... and plans that run as separate launches (small batches)
     (4, 8, 300), (1, 16, 20000), (2, 40, 600),
 ]

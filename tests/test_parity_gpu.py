@@ -139,6 +139,11 @@ STREAM = [
     (160, 32, 333, 31),
     (3, 16, 9000, 32),      # few long sequences: cut into many pieces, merged by the second-pass kernel
     (1, 8, 20000, 33),
+    # more than 64 query rows per sequence (beams x heads over one shared memory, or many heads): groups of 64 rows
+    (32, 128, 2048, 34),    # 4 beams x 32 heads: two groups; 64 schedule sequences on 128 CTAs (clusters of two)
+    (40, 96, 1500, 35),     # a last group of 32 rows
+    (3, 200, 9000, 36),     # few long sequences, four groups (the last of 8 rows): second-pass kernel
+    (16, 65, 1100, 37),     # one row more than a group
 ]
 
 
