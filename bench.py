@@ -407,6 +407,56 @@ def paper_loop_block(mqa, device, seed):
     return out
 
 
+def measured_tensor_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+        except Exception:
+            pass
+    return 1590.0, 1400.0, "fallback"
+
+
+def prefill_block(mqa, device, seed, b=32, h=32, n=4096):
+    """The batched form of Section 3 under the autoregressive mask (the processing of a whole prompt: n = m positions,
+    the batch and head count of the headline workload): milliseconds per call and TFLOP/s, counting the method's own
+    4 k flops per (query row, visible key) pair -- not the dense n x m rectangle.  Compute-bound: set against the
+    measured bf16 matmul throughput."""
+    gen = torch.Generator(device=device).manual_seed(seed + 31)
+    Q = wl.bf16_normal((b, h, n, 128), 128 ** -0.5, gen, device)
+    K = wl.bf16_normal((b, n, 128), 1.0, gen, device)
+    V = wl.bf16_normal((b, n, 128), 1.0, gen, device)
+    O = torch.empty(b, h, n, 128, dtype=torch.float32, device=device)
+    ws = torch.empty(max(16, mqa.prefill_workspace_bytes(b, h, n, n)), dtype=torch.uint8, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    call = lambda _i: mqa.mqa_prefill_attention(Q, K, V, O, ws, None, status)
+    for i in range(2):
+        call(i)
+    secs = statistics.median(time_region(call, 1, device) for _ in range(5))
+    flops = 4 * 128 * h * b * n * (n + 1) // 2
+    burst, sustained, kind = measured_tensor_peak()
+    tf = flops / secs / 1e12
+    groups = b * h * (n // 64)
+    return {"b": b, "h": h, "n": n, "ms": secs * 1e3, "tflops": tf, "flops": flops, "bound": "tensor", "peak": sustained,
+            "peak_kind": f"bf16 matmul, sustained, of {kind}", "frac": tf / sustained, "frac_of_burst_peak": tf / burst,
+            "launches": -(-groups // 1024), "kernel": "mqa_decode_stream_umma_kernel<64, causal>",
+            "status": int(status.item())}
+
+
+def many_rows_block(mqa, device, seed, w, rows=128):
+    """Beam search over one shared memory (Section 4.2: beam 4): beams x heads query rows per sequence, here 4 x 32 = 128
+    rows over the headline workload's caches, as groups of 64 rows on the tensor-core kernel.  us per step (attention over
+    the cache, caches rotated past L2), beside the 64-row figure."""
+    out = {}
+    for r in (64, rows):
+        w2 = wl.Workload(f"{w.name}_rows{r}", b=w.b, h=r, m_max=w.m_max, lens="full")
+        row = quick_point(mqa, "mqa", w2, device, steps=10, min_rotate_bytes=4 * L2_BYTES)
+        out[f"rows_{r}"] = {k: row.get(k) for k in ("us_per_step", "gbs", "frac_of_8TBs", "launches_per_step", "status", "skipped")}
+        out[f"rows_{r}"]["kernel"] = mqa.plan_kernel_name(True, True, w.b, r, w.m_max)
+    return out
+
+
 def cpu_baseline(w, seed, budget_s=20.0):
     """The oracle, as it stands, on the host cores: one multi-query step of the same workload on
     as many whole sequences as fit the time budget."""
@@ -600,6 +650,9 @@ def main():
         out["layer_step"] = layer_block(mqa, w, device, seed, max(3, min(args.steps, 20)))
         out["paper_incremental"] = paper_loop_block(mqa, device, seed)
         out["layer_step"]["projections_us"] = out["layer_step"]["us_per_step"] - blk["us_per_step"]
+    if not args.no_layer and world == 1:
+        out["prefill"] = prefill_block(mqa, device, seed)
+        out["beam4_rows"] = many_rows_block(mqa, device, seed, w)
     if not args.no_line_sweep and world == 1:
         # the other long-context points and the ragged batch: us, GB/s, fraction of 8 TB/s, launches, both variants
         out["sweep"] = [quick_point(mqa, variant, wl.WORKLOADS[name], device)

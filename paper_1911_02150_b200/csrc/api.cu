@@ -347,18 +347,20 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
 
 constexpr size_t kL2KeepBytes = 64u << 20;   // K and V together: half of the 126 MB L2
 constexpr int kEarlyTestWithhold = 1 << 8;    // rides on `early`: MQA_STEP_TEST_WITHHOLD_COPY
-std::atomic<int> g_umma_opt_in[kMaxDevices][10];
+std::atomic<int> g_umma_opt_in[kMaxDevices][13];
 
 // b, h: the caller's sequences and query rows per sequence (the kernel is given the plan's: sequences x groups, 64 rows
 // each, where the plan has groups).  grp_in: the groups of a launch of the batched form; otherwise derived from the plan.
-template <int HP, bool FUSED, bool GUESS = false, bool CAUSAL = false>
+template <int HP, bool FUSED, bool GUESS = false, int GROUPED = 0>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
                 const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
                 int early = 0, const QueryGroups* grp_in = nullptr, long long q_rows = 0) {
     using Cfg = UmmaCfg<HP>;
-    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS, CAUSAL>;
-    constexpr int kSlot = CAUSAL ? 9 : (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
+    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS, GROUPED>;
+    static_assert(GROUPED == 0 || HP == 64, "groups hold 64 query rows");
+    constexpr int kSlot = GROUPED == 2 ? 9 : GROUPED == 1 ? 10 + (GUESS ? 2 : FUSED ? 1 : 0)
+                                                          : (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
     const QueryGroups grp = grp_in ? *grp_in : QueryGroups{p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0, 0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
@@ -405,11 +407,13 @@ int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, 
 #define MQA_UMMA_ARGS p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, early
     if constexpr (FUSED) {
         if ((early & ~kEarlyTestWithhold) >= 2) {           // the kernels that carry the code for copies started on a guess
+            if (p.groups > 1) return launch_umma<64, true, true, 1>(MQA_UMMA_ARGS);
             if (p.h <= 16) return launch_umma<16, true, true>(MQA_UMMA_ARGS);
             if (p.h <= 32) return launch_umma<32, true, true>(MQA_UMMA_ARGS);
             return launch_umma<64, true, true>(MQA_UMMA_ARGS);
         }
     }
+    if (p.groups > 1) return launch_umma<64, FUSED, false, 1>(MQA_UMMA_ARGS);
     if (p.h <= 16) return launch_umma<16, FUSED>(MQA_UMMA_ARGS);
     if (p.h <= 32) return launch_umma<32, FUSED>(MQA_UMMA_ARGS);
     return launch_umma<64, FUSED>(MQA_UMMA_ARGS);
@@ -939,7 +943,7 @@ int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int
         const long long count = total - first < kStreamMaxSeqs ? total - first : kStreamMaxSeqs;
         const Plan p = prefill_plan(count, m_max);
         const QueryGroups grp = {h * per_head, h * n, (int)first, per_head};
-        int err = launch_umma<64, false, false, true>(p, Q, K, V, start, O, workspace, status, b, h, m_max, stream, p.merge_in_kernel,
+        int err = launch_umma<64, false, false, 2>(p, Q, K, V, start, O, workspace, status, b, h, m_max, stream, p.merge_in_kernel,
                                                       nullptr, nullptr, nullptr, 0, &grp, (long long)b * h * n);
         if (err) return err;
         if (!p.merge_in_kernel) {

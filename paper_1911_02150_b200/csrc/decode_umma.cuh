@@ -355,8 +355,9 @@ __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__
 
 // HP = head rows of the Q tile (h rounded up to 16, 32 or 64).  GUESS: built with the code that starts copies on a
 // guess before the wait (GUESS && early >= 2 below); kernels without it take early 0 or 1 only.
-// CAUSAL: built with the mask per column of the batched form (QueryGroups::causal_every != 0).
-template <int HP, bool FUSED, bool GUESS = false, bool CAUSAL = false>
+// GROUPED: 0 = every schedule sequence has its own cache (the plain step: nothing of QueryGroups is compiled in);
+// 1 = groups of 64 query rows over shared caches; 2 = the batched form, with its mask per column.
+template <int HP, bool FUSED, bool GUESS = false, int GROUPED = 0>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                               const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
@@ -365,8 +366,10 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
                               int b, int h, int m_max, unsigned long long magic, const FusedArgs fa,
                               unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int early_arg,
-                              int read_once, const QueryGroups grp) {
+                              int read_once, const QueryGroups grp_arg) {
     using Cfg = UmmaCfg<HP>;
+    constexpr bool CAUSAL = GROUPED == 2;
+    const QueryGroups grp = GROUPED ? grp_arg : QueryGroups{0, 0, 0, 0};
     const int early = GUESS ? early_arg : (early_arg == 1 ? 1 : 0);
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
