@@ -1109,7 +1109,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    const float w = ml[c].x == -INFINITY ? 0.f : fast_exp2(ml[c].x - top);
+                    if (ml[c].x == -INFINITY) continue;  // an empty piece (its sums were never written) is skipped, not multiplied
+                    const float w = fast_exp2(ml[c].x - top);
                     den = fmaf(w, ml[c].y, den);
                     num.x = fmaf(w, a[c].x, num.x); num.y = fmaf(w, a[c].y, num.y);
                     num.z = fmaf(w, a[c].z, num.z); num.w = fmaf(w, a[c].w, num.w);

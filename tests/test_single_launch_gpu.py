@@ -84,6 +84,33 @@ def test_two_shapes_whose_counters_overlap_share_one_epoch(noalloc):
         check_close(o.cpu().numpy(), ref, f"call {rnd}: b={b}")
 
 
+@pytest.mark.parametrize("b,h,m_max,rows", [(32, 16, 1024, 300), (64, 8, 1024, 100), (32, 32, 2048, 2048), (16, 32, 4096, 4000)])
+def test_equal_sequences_in_clusters(b, h, m_max, rows):
+    """A batch that divides the grid is launched as clusters, and with sequences of equal length a cluster holds one
+    sequence: its CTAs take the stages in turn and merge through the cluster's shared memory.  Short sequences leave
+    CTAs of a cluster without a stage (300 rows are three stages for four CTAs): their empty pieces must be skipped."""
+    assert mqa.append_step_launches(b, h, m_max) == 1
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=b + rows, device=DEV)
+    lens0 = np.full(b, rows - 1, np.int32)
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
+    oracle.kv_cache_append(Kh, Vh, wl.bits(inp["k_new"]), wl.bits(inp["v_new"]), lens_h, True)
+    ref = oracle.mqa_decode_step(wl.bits(inp["q"]), Kh, Vh, lens_h)
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    ws.fill_(0xFF)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for chained in (False, True):
+        lens_t.copy_(torch.from_numpy(lens0))
+        o = torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV)
+        mqa.mqa_decode_append_step(inp["q"], inp["K"], inp["V"], inp["k_new"], inp["v_new"], lens_t, o, ws, status,
+                                   advance=True, chained=chained)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.array_equal(lens_t.cpu().numpy(), lens_h)
+        check_close(o.cpu().numpy(), ref, f"b={b} rows={rows} chained={chained}")
+
+
 def test_many_calls_on_one_workspace_are_bit_identical():
     b, h, m_max = 48, 32, 3000
     inp = wl.make_inputs(b, h, m_max, "mqa", seed=11, device=DEV)
