@@ -294,8 +294,8 @@ size_t mqa_host_staging_bytes(int b, int h, int k, int v);
  *   K, V              [b, window, k], [b, window, v] bf16, read-write
  *   pos               [b] int32: tokens of the sequence before this step (0 for the first); advance != 0: pos[b] += 1
  *   o                 [b, h, v] fp32, written;  status optional (APPEND_NEGATIVE_LEN for pos[b] < 0: no row, zeros)
- * One launch (one CTA per sequence); no workspace.  Supported for h <= 32 and windows that one CTA covers (the
- * plan for these sizes has a single split: windows of up to a few hundred rows; MQA_ERR_UNSUPPORTED otherwise).
+ * One launch; no workspace.  One warp per sequence, eight sequences per CTA, any number of heads (16 at a time),
+ * windows of up to 4096 rows (the paper's is 32; MQA_ERR_UNSUPPORTED beyond).
  */
 int mqa_decode_local_step(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* pos,
                           int advance, float* o, int32_t* status, int b, int h, int window, int k, int v,

@@ -16,6 +16,7 @@
 #include "project.cuh"
 #include "decode_simt.cuh"
 #include "decode_umma.cuh"
+#include "decode_local.cuh"
 
 namespace mqa {
 namespace {
@@ -313,7 +314,7 @@ std::atomic<int> g_smem_opt_in[kMaxDevices][4];
 template <int M_TILES, bool EARLY = false>
 int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                float2* part_ml, float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias,
-               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr, bool ring = false,
+               const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
                bool withhold = false) {
     using Cfg = MmaCfg<M_TILES>;
     auto kernel = mqa_decode_split_mma_kernel<M_TILES, EARLY>;
@@ -341,10 +342,11 @@ int launch_mma(const Plan& p, const void* q, const void* K, const void* V, const
     }
     launch_dependent(kernel, (unsigned)((size_t)b * p.n_splits), Cfg::kThreads, Cfg::kSmemBytes, stream, map_k, map_v,
                      map_k_big, map_v_big, static_cast<const uint32_t*>(q), lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows,
-                     p.n_splits, len_bias, fa, lens_advance, (ring ? 1 : 0) | (withhold ? 2 : 0));
+                     p.n_splits, len_bias, fa, lens_advance, withhold ? 2 : 0);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
+constexpr int kLocalMaxWindow = 4096;         // the longest window the local step takes (a warp per sequence: decode_local.cuh)
 constexpr size_t kL2KeepBytes = 64u << 20;   // K and V together: half of the 126 MB L2
 constexpr int kEarlyTestWithhold = 1 << 8;    // rides on `early`: MQA_STEP_TEST_WITHHOLD_COPY
 std::atomic<int> g_umma_opt_in[kMaxDevices][13];
@@ -728,17 +730,17 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
                                              advance ? lens : nullptr);
         return p.kernel == Kernel::kMma1
                    ? launch_mma<1>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
-                                   advance ? lens : nullptr, false, withhold)
+                                   advance ? lens : nullptr, withhold)
                    : launch_mma<2>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
-                                   advance ? lens : nullptr, false, withhold);
+                                   advance ? lens : nullptr, withhold);
     }
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits > 1) {
         // fixed splits: the CTA whose rows hold the new one writes it; the second pass moves lens on.  Two launches.
         float2* part_ml = partials_ml(workspace);
         float* part_acc = partials_acc(p, workspace);
         rc = p.kernel == Kernel::kMma1
-                 ? launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr, false, withhold)
-                 : launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr, false, withhold);
+                 ? launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr, withhold)
+                 : launch_mma<2>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new, nullptr, withhold);
         if (rc) return rc;
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr, true);
     }
@@ -768,14 +770,27 @@ int mqa_decode_local_step(const void* q, void* K, void* V, const void* k_new, co
     int rc = check_step_args(q, K, V, pos, o, status, b, h, window, k, v);
     if (rc) return rc;
     if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return MQA_ERR_INVALID_ARG;
-    const Plan p = plan_mma(b, h > 32 ? 32 : h, window);
-    // one CTA per sequence over the whole window: windows of up to a few hundred rows, at most 32 heads
-    if (h > 32 || p.n_splits != 1 || (long long)b * window >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
-    return p.kernel == Kernel::kMma1
-               ? launch_mma<1>(p, q, K, V, pos, o, nullptr, nullptr, status, b, h, window, stream, 0, k_new, v_new,
-                               advance ? pos : nullptr, true)
-               : launch_mma<2>(p, q, K, V, pos, o, nullptr, nullptr, status, b, h, window, stream, 0, k_new, v_new,
-                               advance ? pos : nullptr, true);
+    if ((long long)b * window >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
+    if (window <= kLocalMaxWindow) {
+        // a warp per sequence: windows of a few tiles (the paper's is one), any number of heads
+        static std::atomic<int> opted[kMaxDevices];
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+        if (!opted[dev].load(std::memory_order_acquire)) {
+            if (cudaFuncSetAttribute(mqa_decode_local_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLocalSmemBytes) != cudaSuccess) {
+                cudaGetLastError();
+                return MQA_ERR_CUDA;
+            }
+            opted[dev].store(1, std::memory_order_release);
+        }
+        alignas(64) CUtensorMap map_k, map_v;
+        if (!encode_cache_map(&map_k, K, (long long)b * window) || !encode_cache_map(&map_v, V, (long long)b * window)) return MQA_ERR_CUDA;
+        launch_dependent(mqa_decode_local_kernel, (unsigned)((b + kLocalWarps - 1) / kLocalWarps), kLocalThreads, kLocalSmemBytes, stream,
+                         map_k, map_v, static_cast<const uint32_t*>(q), static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+                         static_cast<uint4*>(K), static_cast<uint4*>(V), pos, o, status, b, h, window, advance ? 1 : 0);
+        return launch_status();
+    }
+    return MQA_ERR_UNSUPPORTED;   // a window that long is the ordinary step's business
 }
 
 size_t mqa_host_staging_bytes(int b, int h, int k, int v) {

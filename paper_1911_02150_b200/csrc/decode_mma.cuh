@@ -363,8 +363,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
                             int32_t* __restrict__ status, int h, int m_max, int chunk_rows, int n_splits, int len_bias,
                             const FusedArgs fa, int32_t* __restrict__ lens_advance, int mode) {
     using Cfg = MmaCfg<M_TILES>;
-    const int ring = mode & 1;                             // the cache is a window (local attention)
-    const bool withhold = (mode & 2) != 0;                 // for tests: one copy is never started, so that a wait runs out
+    const bool withhold = (mode & 2) != 0;                 // for tests: one copy is never started, so that a wait runs out (bit 0: unused)
     constexpr int kStages = Cfg::kStages;
     const int seq = blockIdx.x / n_splits;
     const int split = blockIdx.x % n_splits;
@@ -409,7 +408,7 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // fetched while that step is still finishing.  Only their number is a guess: should fewer tiles count in the end,
     // the surplus is left to land and ignored.
     int pre = 0;
-    if (EARLY && n_splits == 1 && !ring && warp == Cfg::kConsumerWarps && lane == 0) {
+    if (EARLY && n_splits == 1 && warp == Cfg::kConsumerWarps && lane == 0) {
         const int raw_guess = __ldcg(lens + seq);
         const int rows_guess = min(max(raw_guess, 0) + (fa.k_new != nullptr ? 1 : 0), m_max);
         pre = min((rows_guess - 2) / kTileRows, kStages);
@@ -422,8 +421,6 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // With one CTA per sequence (n_splits == 1) the CTA may do the whole decoding step: write the new row
     // (fa.k_new given), attend over one row more, and move lens[seq] on at the end (lens_advance given) --
     // nobody else reads this sequence's length.
-    // ring: the cache is a window of the last m_max positions (local attention, Section 4.1): lens[seq] counts
-    // the tokens so far, the new row goes to row lens[seq] % m_max and min(lens[seq] + 1, m_max) rows are attended.
     // A sequence cut into several splits (n_splits > 1) may take its new row too: the CTA whose rows hold it writes
     // it, every split attends over one row more, and lens is left to the second-pass kernel.
     // (the new row's pieces do not depend on lens: asked for first, so that the two loads are in flight together)
@@ -431,16 +428,16 @@ mqa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     if (fa.k_new != nullptr && warp == 0)                 // lanes 0-15 move the key row, 16-31 the value row
         row_piece = (lane < 16 ? fa.k_new : fa.v_new)[(size_t)seq * (kRowBytes / 16) + (lane & 15)];
     const int raw = lens[seq];
-    const bool appended = fa.k_new != nullptr && raw >= 0 && (ring || raw < m_max);
+    const bool appended = fa.k_new != nullptr && raw >= 0 && raw < m_max;
     if (fa.k_new != nullptr) {
         if (!appended && threadIdx.x == 0 && status) atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
         if (appended && warp == 0 && (n_splits == 1 || raw / chunk_rows == split)) {
-            const size_t dst = ((size_t)seq * m_max + (ring ? raw % m_max : raw)) * (kRowBytes / 16) + (lane & 15);
+            const size_t dst = ((size_t)seq * m_max + raw) * (kRowBytes / 16) + (lane & 15);
             if (lane < 16) fa.K[dst] = row_piece; else fa.V[dst] = row_piece;
             asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row (a barrier follows)
         }
     }
-    const int L = clamp_len(appended ? (ring ? min(raw + 1, m_max) : raw + 1) : biased_len(raw, m_max, len_bias), m_max,
+    const int L = clamp_len(appended ? raw + 1 : biased_len(raw, m_max, len_bias), m_max,
                             threadIdx.x == 0 ? status : nullptr);
     const int r0 = split * chunk_rows;
     const int r1 = min(L, r0 + chunk_rows);

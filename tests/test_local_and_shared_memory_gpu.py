@@ -21,7 +21,13 @@ def check_close(got, ref, what):
     assert np.all(err.max(-1) <= REL_TOL * np.abs(ref).max(-1)), f"{what}: row-relative error"
 
 
-@pytest.mark.parametrize("b,h,window,steps", [(128, 8, 32, 80), (16, 32, 32, 70), (5, 16, 96, 200)])
+@pytest.mark.parametrize("b,h,window,steps", [
+    (128, 8, 32, 80), (16, 32, 32, 70), (5, 16, 96, 200),
+    (1024, 8, 32, 40),        # a thousand sequences: one wave of eight-sequence CTAs
+    (61, 64, 32, 40),         # 64 heads: four passes of 16 over the window; a last CTA with five sequences
+    (20, 40, 96, 120),        # a head count that is no multiple of 16, a window of three tiles
+    (3, 16, 512, 530),        # a window of sixteen tiles
+])
 def test_local_attention_ring_equals_attention_over_the_last_window_rows(b, h, window, steps):
     gen = torch.Generator(device=DEV).manual_seed(window + b)
     K = torch.zeros(b, window, 128, dtype=torch.bfloat16, device=DEV)
