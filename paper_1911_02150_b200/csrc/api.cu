@@ -42,6 +42,9 @@ int sm_count() {
 
 enum class Kernel { kSimt, kMma1, kMma2, kUmma };
 constexpr int kMergeInKernelMaxPieces = 10;
+constexpr int kMaxClusterCtas = 4;            // a sequence's CTAs as one thread-block cluster.  Measured per step: clusters of 8
+                                              // (16 sequences x 16384 rows) 43 us against 29 us without, clusters of 16
+                                              // (8 x 32768) 43 against 30: too few of them fit the GPCs at once
 
 struct Plan {
     int n_splits = 0;     // 0 = invalid.  Fixed-split kernels: splits per sequence.  Persistent kernel: the
@@ -123,16 +126,23 @@ Plan plan_stream(int b, int h, int m_max) {
     // sequences of equal length every share then starts at a sequence's beginning, a sequence has the fewest
     // pieces (none when CTAs take whole sequences) and the CTAs that hold them finish together.  HBM is
     // saturated from about three quarters of the SMs on (measured: same pass time with 112..148 CTAs).
+    // Among the multiples of the batch, first one that makes a sequence's CTAs a thread-block cluster.
     p.grid = sm_count();
-    for (int g = sm_count(); g >= (3 * sm_count() + 3) / 4; --g)
-        if (g % b == 0 || b % g == 0) { p.grid = g; break; }
+    bool found = false;
+    for (int g = sm_count(); g >= (3 * sm_count() + 3) / 4 && !found; --g)
+        if (b % g == 0 || (g % b == 0 && g / b <= kMaxClusterCtas)) { p.grid = g; found = true; }
+    for (int g = sm_count(); g >= (3 * sm_count() + 3) / 4 && !found; --g)
+        if (g % b == 0) { p.grid = g; found = true; }
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
     int parts = (p.grid + b - 1) / b + 1;
     p.n_splits = parts < p.grid ? parts : p.grid;
     // a sequence cut into a few pieces is merged by one CTA inside the kernel; many pieces (few, long
     // sequences) are better spread over all SMs by the second-pass kernel
-    p.merge_in_kernel = p.kernel == Kernel::kUmma && p.n_splits <= kMergeInKernelMaxPieces;
+    // ... unless the batch divides the grid into clusters: then, with sequences
+    // of equal length, a cluster merges its sequence through its shared memory however many pieces that is
+    p.merge_in_kernel = p.kernel == Kernel::kUmma &&
+                        (p.n_splits <= kMergeInKernelMaxPieces || (p.grid % b == 0 && p.grid / b >= 2 && p.grid / b <= kMaxClusterCtas));
     return p;
 }
 
@@ -367,7 +377,8 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
             cudaGetLastError();
             return MQA_ERR_CUDA;
         }
@@ -390,11 +401,10 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     // a cache that cannot stay in L2 from one step to the next is streamed through it with the evict-first policy
     const int read_once = ((size_t)b * m_max * 2 * kRowBytes > kL2KeepBytes ? 1 : 0) | ((early & kEarlyTestWithhold) ? 2 : 0);
     early &= ~kEarlyTestWithhold;
-    // The single-launch step of a batch that divides the grid runs as clusters of grid / b CTAs (2 to 8, the
-    // portable sizes): with sequences of equal length a cluster then holds exactly one sequence's pieces and merges
+    // The single-launch step of a batch that divides the grid runs as clusters of grid / b CTAs (2 to 4): with sequences of equal length a cluster then holds exactly one sequence's pieces and merges
     // them through its shared memory (the kernel decides from lens; otherwise the clusters change nothing).
     unsigned cluster = 1;
-    if (merge && p.grid % p.b == 0 && p.grid / p.b >= 2 && p.grid / p.b <= 8) cluster = (unsigned)(p.grid / p.b);
+    if (merge && p.grid % p.b == 0 && p.grid / p.b >= 2 && p.grid / p.b <= kMaxClusterCtas) cluster = (unsigned)(p.grid / p.b);
     launch_dependent_clusters(cluster, kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub,
                               map_v_sub, map_q, lens, o, w.span, w.ml, w.acc, status, p.b, p.h, m_max, share_magic(p.grid), fa,
                               merge ? w.ctrl : nullptr, lens_advance, early, read_once, grp);

@@ -1092,28 +1092,34 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             for (int item = tid; item < per * (kHeadDim / 4); item += kUmmaSoftmaxThreads) {
                 const int head = (int)rank * per + (item >> 5), c4 = item & 31;
                 if (head >= h) break;
+                // the (maximum, sum) pairs of all pieces first, then the sums eight pieces at a time (a cluster has up to 16)
                 float top = -INFINITY;
-                float2 ml[8];
-                float4 a[8];
+                float2 ml[16];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int c = 0; c < 16; ++c) {
                     ml[c] = make_float2(-INFINITY, 0.f);
-                    a[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (c < (int)C) {
-                        ml[c] = cluster_ld_f2(cluster_map(ml_s + head * 8, c));
-                        a[c] = cluster_ld_f4(cluster_map(acc_s + (head * kHeadDim + c4 * 4) * 4, c));
-                    }
+                    if (c < (int)C) ml[c] = cluster_ld_f2(cluster_map(ml_s + head * 8, c));
                     top = fmaxf(top, ml[c].x);
                 }
                 float den = 0.f;
                 float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    if (ml[c].x == -INFINITY) continue;  // an empty piece (its sums were never written) is skipped, not multiplied
-                    const float w = fast_exp2(ml[c].x - top);
-                    den = fmaf(w, ml[c].y, den);
-                    num.x = fmaf(w, a[c].x, num.x); num.y = fmaf(w, a[c].y, num.y);
-                    num.z = fmaf(w, a[c].z, num.z); num.w = fmaf(w, a[c].w, num.w);
+                for (int c0 = 0; c0 < 16; c0 += 8) {
+                    if (c0 >= (int)C) break;
+                    float4 a[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        a[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (c0 + c < (int)C) a[c] = cluster_ld_f4(cluster_map(acc_s + (head * kHeadDim + c4 * 4) * 4, c0 + c));
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        if (ml[c0 + c].x == -INFINITY) continue;  // an empty piece (its sums were never written) is skipped, not multiplied
+                        const float w = fast_exp2(ml[c0 + c].x - top);
+                        den = fmaf(w, ml[c0 + c].y, den);
+                        num.x = fmaf(w, a[c].x, num.x); num.y = fmaf(w, a[c].y, num.y);
+                        num.z = fmaf(w, a[c].z, num.z); num.w = fmaf(w, a[c].w, num.w);
+                    }
                 }
                 const float inv = 1.f / den;
                 if (head >= group_rows(grp, s, h)) break;

@@ -144,6 +144,10 @@ STREAM = [
     (40, 96, 1500, 35),     # a last group of 32 rows
     (3, 200, 9000, 36),     # few long sequences, four groups (the last of 8 rows): second-pass kernel
     (16, 65, 1100, 37),     # one row more than a group
+    # batches that divide the grid are launched as clusters (16 and 8 CTAs here); with mixed lengths the clusters
+    # change nothing and one CTA merges a sequence's many pieces
+    (8, 16, 20000, 38),
+    (16, 32, 5000, 39),
 ]
 
 
