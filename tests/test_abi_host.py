@@ -106,3 +106,24 @@ def test_binding_type_checks():
     q = torch.zeros(1, 8, 128, dtype=torch.bfloat16)
     with pytest.raises(TypeError):
         binding.mqa_decode_step(q, q, q, torch.zeros(1, dtype=torch.int32), torch.zeros(1, 8, 128))
+
+
+def test_plans_of_many_query_rows_and_of_the_batched_form(L):
+    """More than 64 query rows per sequence are planned as groups of 64 on the tensor-core kernel, and the batched
+    form's workspace and refusals are answered on the host (the plan assumes the 148 SMs of a B200 without a GPU)."""
+    assert binding.plan_kernel_name(True, False, 32, 128, 8192) == "mqa_decode_stream_umma_kernel<64>"
+    assert binding.plan_kernel_name(True, True, 32, 32, 8192) == "mqa_decode_stream_umma_kernel<32, fused, guess>"
+    assert binding.plan_kernel_name(False, False, 32, 32, 8192) == "decode_split_simt_kernel"
+    assert binding.plan_kernel_name(True, False, 0, 32, 8192) == ""
+    assert binding.append_step_launches(32, 128, 8192) == 1
+    assert binding.workspace_bytes(32, 128, 8192) >= binding.workspace_bytes(32, 64, 8192)
+    need = binding.prefill_workspace_bytes(2, 8, 128, 256)
+    assert need > 0
+    assert binding.prefill_workspace_bytes(2, 8, 100, 256) == 0          # n must be a multiple of 64
+    assert binding.prefill_workspace_bytes(2, 8, 512, 256) == 0          # the queries' positions must fit the memory
+    a = ctypes.c_void_p(0x1000)
+    pf = L.mqa_prefill_attention
+    assert pf(a, a, a, None, a, a, need, None, 2, 8, 100, 256, 128, 128, None) == binding.ERR_UNSUPPORTED
+    assert pf(a, a, a, None, a, a, need - 1, None, 2, 8, 128, 256, 128, 128, None) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert pf(None, a, a, None, a, a, need, None, 2, 8, 128, 256, 128, 128, None) == binding.ERR_INVALID_ARG
+    assert pf(a, a, a, ctypes.c_void_p(0x1002), a, a, need, None, 2, 8, 128, 256, 128, 128, None) == binding.ERR_INVALID_ARG
