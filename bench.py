@@ -544,6 +544,8 @@ def main():
     ap.add_argument("--no-mha", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-layer", action="store_true", help="skip the timing of the whole layer step (projections either side)")
+    ap.add_argument("--prefill-only", default=None, metavar="B,H,N",
+                    help="time only the batched (prefill) form at these sizes and print its block (what the ncu capture of that kernel runs)")
     ap.add_argument("--no-line-sweep", action="store_true", help="skip the long-context sweep points of the default line")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true", help="run every workload, both variants, and write the table to --sweep-out")
@@ -572,6 +574,10 @@ def main():
 
     if args.sweep:
         run_sweep(mqa, args, device, rank)
+        return
+    if args.prefill_only:
+        pb, ph, pn = (int(x) for x in args.prefill_only.split(","))
+        print(json.dumps({"prefill": prefill_block(mqa, device, 0, pb, ph, pn)}))
         return
 
     peak, peak_kind = measured_peak()
