@@ -17,6 +17,7 @@
 #include "decode_simt.cuh"
 #include "decode_umma.cuh"
 #include "decode_local.cuh"
+#include "prefill.cuh"
 
 namespace mqa {
 namespace {
@@ -962,6 +963,28 @@ int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int
     const int rc = check_prefill_dims(b, h, n, m_max, k, v);
     if (rc) return rc;
     if (workspace_bytes < mqa_prefill_workspace_bytes(b, h, n, m_max, k, v)) return MQA_ERR_WORKSPACE_TOO_SMALL;
+    if (n % kPfRows == 0) {
+        // whole tiles of 128 positions: the kernel of the batched form proper (two heads per CTA, no workspace used)
+        static std::atomic<int> opt_in[kMaxDevices];
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+        if (!opt_in[dev].load(std::memory_order_acquire)) {
+            if (cudaFuncSetAttribute(mqa_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes) != cudaSuccess) {
+                cudaGetLastError();
+                return MQA_ERR_CUDA;
+            }
+            opt_in[dev].store(1, std::memory_order_release);
+        }
+        const long long ctas = (long long)(n / kPfRows) * b * ((h + 1) / 2);
+        if (ctas >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
+        alignas(64) CUtensorMap map_q, map_k, map_v;
+        if (!encode_cache_map(&map_q, Q, (long long)b * h * n, kPfRows) || !encode_cache_map(&map_k, K, (long long)b * m_max, kPfRows) ||
+            !encode_cache_map(&map_v, V, (long long)b * m_max, kPfRows))
+            return MQA_ERR_CUDA;
+        launch_dependent(mqa_prefill_kernel, (unsigned)ctas, (unsigned)kPfThreads, (size_t)kPfSmemBytes, stream, map_q, map_k, map_v, start, O,
+                         status, b, h, n, m_max);
+        return launch_status();
+    }
     const int per_head = n / kGroupRows;                       // groups of 64 positions per head
     const long long total = (long long)b * h * per_head;
     for (long long first = 0; first < total; first += kStreamMaxSeqs) {

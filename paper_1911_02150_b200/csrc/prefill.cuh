@@ -1,0 +1,301 @@
+// Multi-query attention over many query positions at once (Section 3, the attention lines of the batched function:
+// logits = einsum(bhnk,bmk->bhnm), weights = softmax(logits + mask), O = einsum(bhnm,bmv->bhnv)) under the mask of
+// Section 2.3 for an autoregressive model.  This is the one part of the method whose arithmetic intensity is high:
+// every K/V row is used by all h heads and by every later position, so it runs against the tensor-core roofline.
+//
+// Shape of the work on sm_100a.  A CTA takes 128 consecutive positions of TWO heads of one sequence (multi-query: the
+// heads share K and V, so one staged K/V tile of 128 rows serves 256 query rows) and walks the cache rows up to its
+// last position in stages of 128:
+//     S_w   = Q_w K_j^T       tcgen05.mma, M = 128 query rows (TMEM lanes), N = 128 cache rows, fp32 in TMEM
+//     P_w   = exp2(S_w log2e - m)   one thread per query row: the row's maximum and sum need no other thread
+//     O_w  += P_w V_j         tcgen05.mma with A = P_w read from TMEM (bf16 pairs written over S_w), B = V_j (MN-major)
+// for w = 0, 1.  While the four softmax warps of one head work on S_w, the tensor core computes the other head's
+// products: the issue order is S_0 S_1 | PV_0 S_0' | PV_1 S_1' | ...  TMEM: S_0, S_1, O_0, O_1 of 128 columns each
+// (all 512).  The reference maximum of a row moves only when the row's largest logit leads it by more than
+// kPfMaxLead (then O_w's row is rescaled in TMEM by the row's own thread); P is bounded by 2^kPfMaxLead.
+// Rows of a tile whose memory is shorter than 1024 rows feed P as bf16 hi + lo parts (two products), like the
+// decoding kernels, so that the rounding of few large weights stays inside the tolerance.
+//
+// Roles: warps 0-3 softmax of head 0, warps 4-7 softmax of head 1, warp 8 TMA producer, warp 9 MMA issuer.
+// Every wait is bounded; a wait that runs out flags PIPELINE_TIMEOUT and the CTA drains and leaves.
+#pragma once
+#include "decode_umma.cuh"
+
+namespace mqa {
+
+constexpr int kPfRows = 128;                                   // query positions per tile = cache rows per stage
+constexpr int kPfTileBytes = kPfRows * kRowBytes;              // 32 KiB: 128 rows x 128 bf16, two 64-column boxes
+constexpr int kPfHalfBytes = kPfTileBytes / 2;
+constexpr int kPfKSlots = 2, kPfVSlots = 2;
+constexpr int kPfThreads = 10 * 32;
+constexpr int kPfProducerWarp = 8, kPfMmaWarp = 9;
+constexpr float kPfMaxLead = 8.f;                              // log2 units a logit may exceed its row's reference by
+// barriers: q_full, k_full/k_empty[2], v_full/v_empty[2], s_ready[2], p_ready[2], pv_done[2]
+constexpr int kPfBarriers = 1 + 2 * kPfKSlots + 2 * kPfVSlots + 6;
+constexpr int kPfSmemBytes = (2 + kPfKSlots + kPfVSlots) * kPfTileBytes + kPfBarriers * 8 + 16 + 1024 /* alignment slack */;
+static_assert(kPfSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
+
+// grid: x = ((n_tiles - 1 - position tile) * b + sequence) * head pairs + pair: the longest rows of work first.
+__global__ void __launch_bounds__(kPfThreads, 1)
+mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ start, float* __restrict__ O,
+                   int32_t* __restrict__ status, int b, int h, int n, int m_max) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pairs = (h + 1) >> 1, n_tiles = n / kPfRows;
+    const int pair = blockIdx.x % pairs;
+    const int seq = (blockIdx.x / pairs) % b;
+    const int pt = n_tiles - 1 - blockIdx.x / (pairs * b);
+    const int p0 = pt * kPfRows;                                // first query position of the tile
+    const int head0 = 2 * pair;
+    const int n_act = head0 + 1 < h ? 2 : 1;                    // heads of this CTA (an odd head count leaves one alone)
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);     // the 128-byte swizzle repeats every 1 KiB
+    const uint32_t q_s = smem_addr(base);
+    const uint32_t k_ring = q_s + 2 * kPfTileBytes, v_ring = k_ring + kPfKSlots * kPfTileBytes;
+    const uint32_t bars = v_ring + kPfVSlots * kPfTileBytes;
+    const uint32_t q_full = bars, k_full = bars + 8, k_empty = k_full + 8 * kPfKSlots, v_full = k_empty + 8 * kPfKSlots,
+                   v_empty = v_full + 8 * kPfVSlots, s_ready = v_empty + 8 * kPfVSlots, p_ready = s_ready + 16,
+                   pv_done = p_ready + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + (2 + kPfKSlots + kPfVSlots) * kPfTileBytes + kPfBarriers * 8);
+    __shared__ int timed_out;
+
+    if (threadIdx.x == 0) {
+        prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
+        mbar_init(q_full, 1);
+        for (int i = 0; i < kPfKSlots; ++i) { mbar_init(k_full + 8 * i, 1); mbar_init(k_empty + 8 * i, 1); }
+        for (int i = 0; i < kPfVSlots; ++i) { mbar_init(v_full + 8 * i, 1); mbar_init(v_empty + 8 * i, 1); }
+        for (int w = 0; w < 2; ++w) { mbar_init(s_ready + 8 * w, 1); mbar_init(p_ready + 8 * w, 4); mbar_init(pv_done + 8 * w, 1); }
+        timed_out = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == kPfMmaWarp) {
+        tmem_alloc(smem_addr(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    grid_dependency_wait();              // Q, K, V and start may come from the kernel before
+    grid_launch_dependents();
+    const int raw = start ? __ldg(start + seq) : 0;
+    // rows of the memory this tile's last position sees; a memory that would pass m_max is cut there (flagged)
+    int L = raw + p0 + kPfRows;
+    if (raw < 0 || raw + n > m_max) {
+        if (threadIdx.x == 0 && status) atomicOr(status, kStatusLenClamped);
+        if (L > m_max) L = m_max;
+    }
+    const bool empty = raw < 0 || L <= 0;                      // nothing to look at: zeros (like a bad lens)
+    const int n_kv = empty ? 0 : (L + kPfRows - 1) / kPfRows;   // stages
+    const bool hilo = L < kSingleRoundingMinRows;
+    const long long q_row0 = ((long long)seq * h + head0) * n + p0;     // row of head 0's first query in [b h n, 128]
+
+    if (warp == kPfProducerWarp) {
+        // =============================================================== TMA producer
+        if (lane == 0 && n_kv > 0) {
+            bool ok = true;
+            mbar_expect_tx(q_full, n_act * kPfTileBytes);
+            for (int w = 0; w < n_act; ++w)
+                for (int half = 0; half < 2; ++half)
+                    tma_load_2d(q_s + w * kPfTileBytes + half * kPfHalfBytes, &map_q, half * kBoxCols, (int)(q_row0 + (long long)w * n), q_full);
+            int issued_k = 0, issued_v = 0;
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int y = seq * m_max + j * kPfRows;
+                const int ks = j % kPfKSlots, vs = j % kPfVSlots;
+                if (j >= kPfKSlots) ok = mbar_wait(k_empty + 8 * ks, ((j / kPfKSlots) - 1) & 1);
+                if (!ok) break;
+                mbar_expect_tx(k_full + 8 * ks, kPfTileBytes);
+                tma_load_2d(k_ring + ks * kPfTileBytes, &map_k, 0, y, k_full + 8 * ks);
+                tma_load_2d(k_ring + ks * kPfTileBytes + kPfHalfBytes, &map_k, kBoxCols, y, k_full + 8 * ks);
+                issued_k = j + 1;
+                if (j >= kPfVSlots) ok = mbar_wait(v_empty + 8 * vs, ((j / kPfVSlots) - 1) & 1);
+                if (!ok) break;
+                mbar_expect_tx(v_full + 8 * vs, kPfTileBytes);
+                tma_load_2d(v_ring + vs * kPfTileBytes, &map_v, 0, y, v_full + 8 * vs);
+                tma_load_2d(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs);
+                issued_v = j + 1;
+            }
+            if (!ok) {
+                // a wait ran out: the copies already started are given a bounded wait each before the CTA may leave
+                atomicExch(&timed_out, 1);
+                mbar_wait(q_full, 0);
+                for (int j = max(0, issued_k - kPfKSlots); j < issued_k; ++j) mbar_wait(k_full + 8 * (j % kPfKSlots), (j / kPfKSlots) & 1);
+                for (int j = max(0, issued_v - kPfVSlots); j < issued_v; ++j) mbar_wait(v_full + 8 * (j % kPfVSlots), (j / kPfVSlots) & 1);
+            }
+        }
+    } else if (warp == kPfMmaWarp) {
+        // =============================================================== issuer of both products
+        if (lane == 0 && n_kv > 0) {
+            constexpr uint32_t kIdescS = umma_idesc(128, 128, false, false);
+            constexpr uint32_t kIdescO = umma_idesc(128, 128, false, true);
+            bool ok = mbar_wait(q_full, 0);
+            auto issue_s = [&](int w, int j) {                  // S_w = Q_w K_j^T into its 128 columns
+                const uint32_t k_s = k_ring + (j % kPfKSlots) * kPfTileBytes, qw = q_s + w * kPfTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {                // 8 k-steps of 16 columns; 4 per 64-column box
+                    const uint32_t off = (ks >> 2) * kPfHalfBytes + (ks & 3) * 32;
+                    umma_ss(tmem_base + w * 128, umma_desc(qw + off, 16, 1024), umma_desc(k_s + off, 16, 1024), kIdescS, ks ? 1u : 0u);
+                }
+                tc_commit(s_ready + 8 * w);
+            };
+            auto issue_pv = [&](int w, int j) {                 // O_w += P_w V_j: P from TMEM (bf16 pairs: 8 columns per 16 rows of V)
+                const uint32_t v_s = v_ring + (j % kPfVSlots) * kPfTileBytes;
+                for (int part = 0; part < (hilo ? 2 : 1); ++part) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + part * 64 + kk * 8,
+                                umma_desc(v_s + kk * 2048, kPfHalfBytes, 1024), kIdescO, (j == 0 && part == 0 && kk == 0) ? 0u : 1u);
+                }
+                tc_commit(pv_done + 8 * w);
+            };
+            if (ok) ok = mbar_wait(k_full, 0);
+            tc_fence_after();
+            if (ok) {
+                for (int w = 0; w < n_act; ++w) issue_s(w, 0);
+                tc_commit(k_empty);
+            }
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const bool more = j + 1 < n_kv;
+                for (int w = 0; w < n_act && ok; ++w) {
+                    ok = mbar_wait(p_ready + 8 * w, j & 1);
+                    if (ok && w == 0) ok = mbar_wait(v_full + 8 * (j % kPfVSlots), (j / kPfVSlots) & 1);
+                    if (ok && w == 0 && more) ok = mbar_wait(k_full + 8 * ((j + 1) % kPfKSlots), ((j + 1) / kPfKSlots) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(w, j);
+                    if (w == n_act - 1) tc_commit(v_empty + 8 * (j % kPfVSlots));
+                    if (more) {
+                        issue_s(w, j + 1);
+                        if (w == n_act - 1) tc_commit(k_empty + 8 * ((j + 1) % kPfKSlots));
+                    }
+                }
+            }
+            if (!ok) atomicExch(&timed_out, 1);
+        }
+    } else {
+        // =============================================================== softmax warps: one thread per query row
+        const int w = warp >> 2, quarter = warp & 3, r = quarter * 32 + lane;
+        if (w < n_act) {
+            float* dst = O + (size_t)(q_row0 + (long long)w * n + r) * kHeadDim;
+            if (n_kv == 0) {
+                for (int i = 0; i < kHeadDim; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+                const uint32_t s_t = lane_base + w * 128, o_t = lane_base + 256 + w * 128;
+                const int lim_first = min(raw + p0 + 1, m_max);           // rows the tile's first position sees
+                const int lim = min(raw + p0 + r + 1, m_max);             // rows this thread's position sees: >= 1
+                float m = -INFINITY, l = 0.f;                             // reference maximum (log2 units), sum of weights
+                bool ok = true;
+                for (int j = 0; j < n_kv; ++j) {
+                    const int k0 = j * kPfRows;
+                    if (ok) ok = mbar_wait(s_ready + 8 * w, j & 1);
+                    tc_fence_after();
+                    uint32_t x[128];
+                    tmem_ld_cols<128>(s_t, x);
+                    tmem_wait_ld();
+                    // the mask of Section 2.3, by index (a select: what lies behind a masked logit is never used)
+                    if (k0 + kPfRows > lim_first) {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i)
+                            if (k0 + i >= lim) x[i] = 0xff800000u;        // -inf
+                    }
+                    float mx = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(x[i]));
+                    mx *= kLog2e;
+                    if (__any_sync(0xffffffffu, mx > m + kPfMaxLead)) {
+                        // ---- a row of this warp leads its reference by too much: every row of the warp moves its
+                        // reference to its largest logit so far and rescales its sum and its row of O
+                        const float m_new = fmaxf(m, mx);
+                        if (j > 0) {
+                            const float f = fast_exp2(m - m_new);         // (m is finite from the first stage on)
+                            l *= f;
+                            if (ok) ok = mbar_wait(pv_done + 8 * w, (j - 1) & 1);    // O holds the stages before this one
+                            tc_fence_after();
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t y[32];
+                                tmem_ld32(o_t + c * 32, y);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * f);
+                                tmem_st32(o_t + c * 32, y);
+                            }
+                        }
+                        m = m_new;
+                    }
+                    // ---- P = exp2(S log2e - m) as bf16 pairs over the first columns of S (hi), and their remainders
+                    // over the columns after them (lo) for a short memory
+                    const float neg_m = -m;
+                    float sum = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t hi[8];
+                        float pw[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            pw[i] = fast_exp2(fmaf(__uint_as_float(x[c * 16 + i]), kLog2e, neg_m));
+                            sum += pw[i];
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) hi[i] = pack_bf16(pw[2 * i], pw[2 * i + 1]);
+                        tmem_st8(s_t + c * 8, hi);
+                        if (hilo) {
+                            uint32_t lo[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) lo[i] = pack_bf16(pw[2 * i] - bf16_lo(hi[i]), pw[2 * i + 1] - bf16_hi(hi[i]));
+                            tmem_st8(s_t + 64 + c * 8, lo);
+                        }
+                    }
+                    l += sum;
+                    tmem_wait_st();
+                    tc_fence_before();
+                    if (w == 0 && j == n_kv - 1 && L < k0 + kPfRows) {
+                        // the last stage runs past the memory: the tensor core would multiply the zero weights with
+                        // whatever lies there (NaN * 0 = NaN), so those V rows are cleared first
+                        const int vs = j % kPfVSlots;
+                        if (ok) ok = mbar_wait(v_full + 8 * vs, (j / kPfVSlots) & 1);
+                        const uint32_t v_s = v_ring + vs * kPfTileBytes;
+                        const int first = L - k0;
+                        for (int i = r; i < (kPfRows - first) * 16; i += 128) {
+                            const int vrow = first + (i >> 4), ch = i & 15;
+                            const uint32_t a = v_s + (ch >> 3) * kPfHalfBytes + vrow * 128 + ((ch & 7) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(p_ready + 8 * w);
+                }
+                // ---- the row of O, divided by the sum of its weights
+                if (ok) ok = mbar_wait(pv_done + 8 * w, (n_kv - 1) & 1);
+                tc_fence_after();
+                const float inv = 1.f / l;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t y[32];
+                    tmem_ld32(o_t + c * 32, y);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4*>(dst + c * 32 + i) =
+                            make_float4(__uint_as_float(y[i]) * inv, __uint_as_float(y[i + 1]) * inv, __uint_as_float(y[i + 2]) * inv,
+                                        __uint_as_float(y[i + 3]) * inv);
+                }
+                if (!ok) atomicExch(&timed_out, 1);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kPfMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && timed_out && status) atomicOr(status, kStatusPipelineTimeout);
+}
+
+}  // namespace mqa
