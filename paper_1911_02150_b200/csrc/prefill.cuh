@@ -35,6 +35,29 @@ constexpr int kPfBarriers = 1 + 2 * kPfKSlots + 2 * kPfVSlots + 6;
 constexpr int kPfSmemBytes = (2 + kPfKSlots + kPfVSlots) * kPfTileBytes + kPfBarriers * 8 + 16 + 1024 /* alignment slack */;
 static_assert(kPfSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
 
+// two fp32 values in one 64-bit register: packed multiply-add and add (one instruction for two elements)
+__device__ __forceinline__ unsigned long long f2_pack(float lo, float hi) {
+    unsigned long long d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void f2_unpack(unsigned long long v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ unsigned long long f2_fma(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long f2_add(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // grid: x = ((n_tiles - 1 - position tile) * b + sequence) * head pairs + pair: the longest rows of work first.
 __global__ void __launch_bounds__(kPfThreads, 1)
 mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -146,7 +169,7 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 for (int part = 0; part < (hilo ? 2 : 1); ++part) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + part * 64 + kk * 8,
+                        umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + (kk >> 1) * 32 + part * 16 + (kk & 1) * 8,
                                 umma_desc(v_s + kk * 2048, kPfHalfBytes, 1024), kIdescO, (j == 0 && part == 0 && kk == 0) ? 0u : 1u);
                 }
                 tc_commit(pv_done + 8 * w);
@@ -193,19 +216,31 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int k0 = j * kPfRows;
                     if (ok) ok = mbar_wait(s_ready + 8 * w, j & 1);
                     tc_fence_after();
-                    uint32_t x[128];
-                    tmem_ld_cols<128>(s_t, x);
-                    tmem_wait_ld();
-                    // the mask of Section 2.3, by index (a select: what lies behind a masked logit is never used)
-                    if (k0 + kPfRows > lim_first) {
+                    const bool diag = k0 + kPfRows > lim_first;           // some position of the tile cannot see all of this stage
+                    // ---- first pass over the row's 128 logits, 32 columns at a time (the next load under way while
+                    // one is looked at): the largest.  The mask of Section 2.3 is applied by index, as a select: what
+                    // lies behind a masked logit is never used.
+                    float mx8[8];
 #pragma unroll
-                        for (int i = 0; i < 128; ++i)
-                            if (k0 + i >= lim) x[i] = 0xff800000u;        // -inf
+                    for (int i = 0; i < 8; ++i) mx8[i] = -INFINITY;
+                    {
+                        uint32_t xa[32], xb[32];
+                        tmem_ld32(s_t, xa);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t(&cur)[32] = (c & 1) ? xb : xa;
+                            tmem_wait_ld();
+                            if (c < 3) tmem_ld32(s_t + (c + 1) * 32, (c & 1) ? xa : xb);
+                            if (diag) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (k0 + c * 32 + i >= lim) cur[i] = 0xff800000u;        // -inf
+                            }
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) mx8[i & 7] = max3(mx8[i & 7], __uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+                        }
                     }
-                    float mx = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(x[i]));
-                    mx *= kLog2e;
+                    const float mx = max3(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * kLog2e;
                     if (__any_sync(0xffffffffu, mx > m + kPfMaxLead)) {
                         // ---- a row of this warp leads its reference by too much: every row of the warp moves its
                         // reference to its largest logit so far and rescales its sum and its row of O
@@ -227,30 +262,42 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                         m = m_new;
                     }
-                    // ---- P = exp2(S log2e - m) as bf16 pairs over the first columns of S (hi), and their remainders
-                    // over the columns after them (lo) for a short memory
-                    const float neg_m = -m;
-                    float sum = 0.f;
+                    // ---- second pass: P = exp2(S log2e - m) as bf16 pairs, written over the 32 columns just read: the
+                    // hi parts into the first 16 of them and, for a short memory, their remainders (lo) into the other 16
+                    const unsigned long long neg_m2 = f2_pack(-m, -m), log2e2 = f2_pack(kLog2e, kLog2e);
+                    unsigned long long sum2[2] = {0ull, 0ull};           // (two chains of packed sums)
+                    {
+                        uint32_t xa[32], xb[32];
+                        tmem_ld32(s_t, xa);
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint32_t hi[8];
-                        float pw[16];
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t(&cur)[32] = (c & 1) ? xb : xa;
+                            tmem_wait_ld();
+                            if (c < 3) tmem_ld32(s_t + (c + 1) * 32, (c & 1) ? xa : xb);
+                            if (diag) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            pw[i] = fast_exp2(fmaf(__uint_as_float(x[c * 16 + i]), kLog2e, neg_m));
-                            sum += pw[i];
-                        }
+                                for (int i = 0; i < 32; ++i)
+                                    if (k0 + c * 32 + i >= lim) cur[i] = 0xff800000u;
+                            }
+                            uint32_t hi[16], lo[16];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) hi[i] = pack_bf16(pw[2 * i], pw[2 * i + 1]);
-                        tmem_st8(s_t + c * 8, hi);
-                        if (hilo) {
-                            uint32_t lo[8];
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) lo[i] = pack_bf16(pw[2 * i] - bf16_lo(hi[i]), pw[2 * i + 1] - bf16_hi(hi[i]));
-                            tmem_st8(s_t + 64 + c * 8, lo);
+                            for (int i = 0; i < 16; ++i) {
+                                float a0, a1;
+                                f2_unpack(f2_fma(f2_pack(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), log2e2, neg_m2), a0, a1);
+                                const float pa = fast_exp2(a0), pb = fast_exp2(a1);
+                                sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
+                                hi[i] = pack_bf16(pa, pb);
+                                if (hilo) lo[i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
+                            }
+                            tmem_st16(s_t + c * 32, hi);
+                            if (hilo) tmem_st16(s_t + c * 32 + 16, lo);
                         }
                     }
-                    l += sum;
+                    {
+                        float s0, s1;
+                        f2_unpack(f2_add(sum2[0], sum2[1]), s0, s1);
+                        l += s0 + s1;
+                    }
                     tmem_wait_st();
                     tc_fence_before();
                     if (w == 0 && j == n_kv - 1 && L < k0 + kPfRows) {
