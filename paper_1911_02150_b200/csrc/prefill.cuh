@@ -27,8 +27,9 @@ constexpr int kPfRows = 128;                                   // query position
 constexpr int kPfTileBytes = kPfRows * kRowBytes;              // 32 KiB: 128 rows x 128 bf16, two 64-column boxes
 constexpr int kPfHalfBytes = kPfTileBytes / 2;
 constexpr int kPfKSlots = 2, kPfVSlots = 2;
-constexpr int kPfThreads = 10 * 32;
+constexpr int kPfThreads = 12 * 32;                            // (warps 10 and 11 only complete the third warpgroup)
 constexpr int kPfProducerWarp = 8, kPfMmaWarp = 9;
+constexpr int kPfRegsSoftmax = 216, kPfRegsOther = 72;
 constexpr float kPfMaxLead = 8.f;                              // log2 units a logit may exceed its row's reference by
 // barriers: q_full, k_full/k_empty[2], v_full/v_empty[2], s_ready[2], p_ready[2], pv_done[2]
 constexpr int kPfBarriers = 1 + 2 * kPfKSlots + 2 * kPfVSlots + 6;
@@ -101,7 +102,6 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-
     grid_dependency_wait();              // Q, K, V and start may come from the kernel before
     grid_launch_dependents();
     const int raw = start ? __ldg(start + seq) : 0;
@@ -116,6 +116,8 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const bool hilo = L < kSingleRoundingMinRows;
     const long long q_row0 = ((long long)seq * h + head0) * n + p0;     // row of head 0's first query in [b h n, 128]
 
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPfRegsOther));
     if (warp == kPfProducerWarp) {
         // =============================================================== TMA producer
         if (lane == 0 && n_kv > 0) {
@@ -188,17 +190,24 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (ok && w == 0 && more) ok = mbar_wait(k_full + 8 * ((j + 1) % kPfKSlots), ((j + 1) / kPfKSlots) & 1);
                     if (!ok) break;
                     tc_fence_after();
+                    ST(j, 6 + w);
                     issue_pv(w, j);
                     if (w == n_act - 1) tc_commit(v_empty + 8 * (j % kPfVSlots));
                     if (more) {
                         issue_s(w, j + 1);
                         if (w == n_act - 1) tc_commit(k_empty + 8 * ((j + 1) % kPfKSlots));
+#ifdef PF_EXP_MMATIME
+                        mbar_wait(s_ready + 8 * w, (j + 1) & 1);
+                        ST(j, 1 + 3 * w);
+#endif
                     }
                 }
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPfRegsSoftmax));
         // =============================================================== softmax warps: one thread per query row
         const int w = warp >> 2, quarter = warp & 3, r = quarter * 32 + lane;
         if (w < n_act) {
@@ -215,89 +224,61 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 for (int j = 0; j < n_kv; ++j) {
                     const int k0 = j * kPfRows;
                     if (ok) ok = mbar_wait(s_ready + 8 * w, j & 1);
+                    if (r == 0) ST(j, w * 3);
                     tc_fence_after();
                     const bool diag = k0 + kPfRows > lim_first;           // some position of the tile cannot see all of this stage
-                    // ---- first pass over the row's 128 logits, 32 columns at a time (the next load under way while
-                    // one is looked at): the largest.  The mask of Section 2.3 is applied by index, as a select: what
-                    // lies behind a masked logit is never used.
+                    // ---- the row's 128 logits, read once and kept in registers.  The mask of Section 2.3 is applied
+                    // by index, as a select: what lies behind a masked logit is never used.
+                    uint32_t x[128];
+                    tmem_ld_cols<128>(s_t, x);
+                    tmem_wait_ld();
+                    if (diag) {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i)
+                            if (k0 + i >= lim) x[i] = 0xff800000u;        // -inf
+                    }
                     float mx8[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) mx8[i] = -INFINITY;
-                    {
-                        uint32_t xa[32], xb[32];
-                        tmem_ld32(s_t, xa);
+                    for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1]));
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t(&cur)[32] = (c & 1) ? xb : xa;
-                            tmem_wait_ld();
-                            if (c < 3) tmem_ld32(s_t + (c + 1) * 32, (c & 1) ? xa : xb);
-                            if (diag) {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i)
-                                    if (k0 + c * 32 + i >= lim) cur[i] = 0xff800000u;        // -inf
-                            }
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) mx8[i & 7] = max3(mx8[i & 7], __uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
-                        }
-                    }
+                    for (int i = 8; i < 64; ++i) mx8[i & 7] = max3(mx8[i & 7], __uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1]));
                     const float mx = max3(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * kLog2e;
                     if (__any_sync(0xffffffffu, mx > m + kPfMaxLead)) {
-                        // ---- a row of this warp leads its reference by too much: every row of the warp moves its
-                        // reference to its largest logit so far and rescales its sum and its row of O
                         const float m_new = fmaxf(m, mx);
                         if (j > 0) {
                             const float f = fast_exp2(m - m_new);         // (m is finite from the first stage on)
                             l *= f;
                             if (ok) ok = mbar_wait(pv_done + 8 * w, (j - 1) & 1);    // O holds the stages before this one
                             tc_fence_after();
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                uint32_t y[32];
-                                tmem_ld32(o_t + c * 32, y);
+#pragma unroll 1
+                            for (int c = 0; c < 16; ++c) {
+                                uint32_t y[8];
+                                tmem_ld8(o_t + c * 8, y);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * f);
-                                tmem_st32(o_t + c * 32, y);
+                                for (int i = 0; i < 8; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * f);
+                                tmem_st8(o_t + c * 8, y);
                             }
                         }
                         m = m_new;
                     }
-                    // ---- second pass: P = exp2(S log2e - m) as bf16 pairs, written over the 32 columns just read: the
-                    // hi parts into the first 16 of them and, for a short memory, their remainders (lo) into the other 16
-                    const unsigned long long neg_m2 = f2_pack(-m, -m), log2e2 = f2_pack(kLog2e, kLog2e);
-                    unsigned long long sum2[2] = {0ull, 0ull};           // (two chains of packed sums)
-                    {
-                        uint32_t xa[32], xb[32];
-                        tmem_ld32(s_t, xa);
+                    const float neg_m = -m;
+                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t(&cur)[32] = (c & 1) ? xb : xa;
-                            tmem_wait_ld();
-                            if (c < 3) tmem_ld32(s_t + (c + 1) * 32, (c & 1) ? xa : xb);
-                            if (diag) {
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t hi[16];
 #pragma unroll
-                                for (int i = 0; i < 32; ++i)
-                                    if (k0 + c * 32 + i >= lim) cur[i] = 0xff800000u;
-                            }
-                            uint32_t hi[16], lo[16];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                float a0, a1;
-                                f2_unpack(f2_fma(f2_pack(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), log2e2, neg_m2), a0, a1);
-                                const float pa = fast_exp2(a0), pb = fast_exp2(a1);
-                                sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
-                                hi[i] = pack_bf16(pa, pb);
-                                if (hilo) lo[i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
-                            }
-                            tmem_st16(s_t + c * 32, hi);
-                            if (hilo) tmem_st16(s_t + c * 32 + 16, lo);
+                        for (int i = 0; i < 16; ++i) {
+                            const float pa = fast_exp2(fmaf(__uint_as_float(x[c * 32 + 2 * i]), kLog2e, neg_m));
+                            const float pb = fast_exp2(fmaf(__uint_as_float(x[c * 32 + 2 * i + 1]), kLog2e, neg_m));
+                            sum4[i & 3] += pa + pb;
+                            hi[i] = pack_bf16(pa, pb);
+                            if (hilo) x[c * 32 + i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
                         }
+                        tmem_st16(s_t + c * 32, hi);
+                        if (hilo) tmem_st16(s_t + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 32]));
                     }
-                    {
-                        float s0, s1;
-                        f2_unpack(f2_add(sum2[0], sum2[1]), s0, s1);
-                        l += s0 + s1;
-                    }
+                    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                     tmem_wait_st();
                     tc_fence_before();
                     if (w == 0 && j == n_kv - 1 && L < k0 + kPfRows) {
@@ -316,6 +297,7 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(p_ready + 8 * w);
+                    if (r == 0) ST(j, w * 3 + 2);
                 }
                 // ---- the row of O, divided by the sum of its weights
                 if (ok) ok = mbar_wait(pv_done + 8 * w, (n_kv - 1) & 1);
