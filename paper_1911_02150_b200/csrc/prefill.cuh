@@ -262,23 +262,28 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                         m = m_new;
                     }
-                    const float neg_m = -m;
-                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                    const unsigned long long neg_m2 = f2_pack(-m, -m), log2e2 = f2_pack(kLog2e, kLog2e);
+                    unsigned long long sum2[2] = {0ull, 0ull};
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t hi[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            const float pa = fast_exp2(fmaf(__uint_as_float(x[c * 32 + 2 * i]), kLog2e, neg_m));
-                            const float pb = fast_exp2(fmaf(__uint_as_float(x[c * 32 + 2 * i + 1]), kLog2e, neg_m));
-                            sum4[i & 3] += pa + pb;
+                            float a0, a1;
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
+                            const float pa = fast_exp2(a0), pb = fast_exp2(a1);
+                            sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
                             hi[i] = pack_bf16(pa, pb);
                             if (hilo) x[c * 32 + i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
                         }
                         tmem_st16(s_t + c * 32, hi);
                         if (hilo) tmem_st16(s_t + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 32]));
                     }
-                    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    {
+                        float s0, s1;
+                        f2_unpack(f2_add(sum2[0], sum2[1]), s0, s1);
+                        l += s0 + s1;
+                    }
                     tmem_wait_st();
                     tc_fence_before();
                     if (w == 0 && j == n_kv - 1 && L < k0 + kPfRows) {
