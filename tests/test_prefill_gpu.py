@@ -104,6 +104,41 @@ def test_rows_are_the_decode_steps():
         assert float((o - O[:, :, t]).abs().max()) <= 2e-3
 
 
+WHOLE_TILES = [
+    # b, h, n, m_max, start: n a multiple of 128 (the kernel of the batched form: two heads per CTA)
+    (2, 5, 384, 700, [300, 17]),                # an odd head count: the last CTA of a position tile holds one head
+    (1, 2, 1152, 1300, [100]),                  # memories on both sides of 1024 rows (two roundings of the weights below it)
+    (3, 7, 256, 1000, [744, 0, 511]),           # start + n = m_max exactly; a stage that ends inside the next sequence's rows
+    (2, 1, 128, 128, None),                     # a single head
+    (1, 4, 512, 2049, [1537]),                  # one row of the memory in a stage of its own
+]
+
+
+@pytest.mark.parametrize("b,h,n,m_max,start", WHOLE_TILES)
+def test_whole_tiles_match_oracle(b, h, n, m_max, start):
+    run(b, h, n, m_max, start, seed=7 * b + h)
+
+
+def test_a_negative_start_gives_zeros_and_a_flag():
+    """start[b] < 0 is an empty memory for that sequence (zeros, LEN_CLAMPED); the other sequences are not affected."""
+    b, h, n, m_max = 3, 4, 256, 512
+    gen = torch.Generator(device=DEV).manual_seed(11)
+    Q = wl.bf16_normal((b, h, n, 128), 128 ** -0.5, gen, DEV)
+    K = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    V = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    st = np.array([5, -1, 100], np.int32)
+    O = torch.full((b, h, n, 128), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(16, mqa.prefill_workspace_bytes(b, h, n, m_max)), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mqa.mqa_prefill_attention(Q, K, V, O, ws, torch.from_numpy(st).to(DEV), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == binding.STATUS_LEN_CLAMPED
+    assert bool((O[1] == 0).all())
+    keep = [0, 2]
+    ref = oracle.mqa_batched_attention(wl.bits(Q[keep]), wl.bits(K[keep]), wl.bits(V[keep]), st[keep])
+    check_close(O[keep].cpu().numpy(), ref, "sequences beside a bad start")
+
+
 def test_two_runs_are_bit_identical():
     a = run(4, 8, 256, 700, [0, 400, 444, 13], seed=9)
     c = run(4, 8, 256, 700, [0, 400, 444, 13], seed=9)
