@@ -196,10 +196,6 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (more) {
                         issue_s(w, j + 1);
                         if (w == n_act - 1) tc_commit(k_empty + 8 * ((j + 1) % kPfKSlots));
-#ifdef PF_EXP_MMATIME
-                        mbar_wait(s_ready + 8 * w, (j + 1) & 1);
-                        ST(j, 1 + 3 * w);
-#endif
                     }
                 }
             }
@@ -264,20 +260,36 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                     const unsigned long long neg_m2 = f2_pack(-m, -m), log2e2 = f2_pack(kLog2e, kLog2e);
                     unsigned long long sum2[2] = {0ull, 0ull};
+                    if (hilo) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t hi[16];
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t hi[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            float a0, a1;
-                            f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
-                            const float pa = fast_exp2(a0), pb = fast_exp2(a1);
-                            sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
-                            hi[i] = pack_bf16(pa, pb);
-                            if (hilo) x[c * 32 + i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
+                            for (int i = 0; i < 16; ++i) {
+                                float a0, a1;
+                                f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
+                                const float pa = fast_exp2(a0), pb = fast_exp2(a1);
+                                sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
+                                hi[i] = pack_bf16(pa, pb);
+                                x[c * 32 + i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
+                            }
+                            tmem_st16(s_t + c * 32, hi);
+                            tmem_st16(s_t + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 32]));
                         }
-                        tmem_st16(s_t + c * 32, hi);
-                        if (hilo) tmem_st16(s_t + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 32]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t hi[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                float a0, a1;
+                                f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
+                                const float pa = fast_exp2(a0), pb = fast_exp2(a1);
+                                sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
+                                hi[i] = pack_bf16(pa, pb);
+                            }
+                            tmem_st16(s_t + c * 32, hi);
+                        }
                     }
                     {
                         float s0, s1;
