@@ -119,6 +119,29 @@ def test_whole_tiles_match_oracle(b, h, n, m_max, start):
     run(b, h, n, m_max, start, seed=7 * b + h)
 
 
+def test_a_logit_far_above_every_earlier_one_in_a_long_memory():
+    """Memories of 1024 rows and more form the weights of a stage against the reference as it stands and look at the
+    logits only if the stage's sum is out of range: a key row 300 times larger than the others, deep in the memory, makes
+    logits hundreds of units above (and below) everything before it -- the stage is then done again from the logits."""
+    b, h, n, m_max = 2, 3, 256, 1536
+    gen = torch.Generator(device=DEV).manual_seed(21)
+    Q = wl.bf16_normal((b, h, n, 128), 128 ** -0.5, gen, DEV)
+    K = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    V = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    st = np.array([1280, 1100], np.int32)
+    K[0, 1400] *= 300
+    K[1, 1290] *= 300
+    K[1, 5] *= 40                                           # (and one in the first stage, for comparison)
+    O = torch.full((b, h, n, 128), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(16, mqa.prefill_workspace_bytes(b, h, n, m_max)), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mqa.mqa_prefill_attention(Q, K, V, O, ws, torch.from_numpy(st).to(DEV), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = oracle.mqa_batched_attention(wl.bits(Q), wl.bits(K), wl.bits(V), st)
+    check_close(O.cpu().numpy(), ref, "a dominant key row late in the memory")
+
+
 def test_a_negative_start_gives_zeros_and_a_flag():
     """start[b] < 0 is an empty memory for that sequence (zeros, LEN_CLAMPED); the other sequences are not affected."""
     b, h, n, m_max = 3, 4, 256, 512
