@@ -120,9 +120,9 @@ def test_whole_tiles_match_oracle(b, h, n, m_max, start):
 
 
 def test_a_logit_far_above_every_earlier_one_in_a_long_memory():
-    """Memories of 1024 rows and more form the weights of a stage against the reference as it stands and look at the
-    logits only if the stage's sum is out of range: a key row 300 times larger than the others, deep in the memory, makes
-    logits hundreds of units above (and below) everything before it -- the stage is then done again from the logits."""
+    """A key row 300 times larger than the others, deep in a memory of more than 1024 rows, makes logits hundreds of
+    units above (and below) everything before it: the rows' reference maxima move late and by a lot, and their
+    accumulated outputs are rescaled by factors that underflow."""
     b, h, n, m_max = 2, 3, 256, 1536
     gen = torch.Generator(device=DEV).manual_seed(21)
     Q = wl.bf16_normal((b, h, n, 128), 128 ** -0.5, gen, DEV)
