@@ -930,26 +930,17 @@ int mqa_plan_splits(int multi_query, int b, int h, int m_max, int k, int v, int*
     return p.n_splits;
 }
 
-// ---- the batched form (prefill): launches of at most kStreamMaxSeqs groups of 64 query positions --------------
-static Plan prefill_plan(long long groups_in_launch, int m_max) { return plan_stream((int)groups_in_launch, kGroupRows, m_max); }
-
+// ---- the batched form (prefill) ---------------------------------------------------------------------------------
 static int check_prefill_dims(int b, int h, int n, int m_max, int k, int v) {
     if (!dims_ok(b, h, m_max) || n <= 0 || k <= 0 || v <= 0) return MQA_ERR_INVALID_ARG;
-    if (k != kHeadDim || v != kHeadDim || n % kGroupRows != 0 || n > m_max) return MQA_ERR_UNSUPPORTED;
-    if ((long long)b * m_max >= 0x7fffffffLL || (long long)b * h * n >= 0x7fffffffLL || sm_count() > 256) return MQA_ERR_UNSUPPORTED;
+    if (k != kHeadDim || v != kHeadDim || n > m_max) return MQA_ERR_UNSUPPORTED;
+    const long long ctas = (long long)((n + kPfRows - 1) / kPfRows) * b * ((h + 1) / 2);
+    if ((long long)b * m_max >= 0x7fffffffLL || (long long)b * h * n >= 0x7fffffffLL - kPfRows || ctas >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
     return MQA_OK;
 }
 
 size_t mqa_prefill_workspace_bytes(int b, int h, int n, int m_max, int k, int v) {
-    if (check_prefill_dims(b, h, n, m_max, k, v) != MQA_OK) return 0;
-    const long long total = (long long)b * h * (n / kGroupRows);
-    const long long full = total < kStreamMaxSeqs ? total : kStreamMaxSeqs;
-    size_t need = plan_workspace_bytes(prefill_plan(full, m_max));
-    if (total > kStreamMaxSeqs && total % kStreamMaxSeqs != 0) {
-        const size_t last = plan_workspace_bytes(prefill_plan(total % kStreamMaxSeqs, m_max));
-        need = last > need ? last : need;
-    }
-    return need;
+    return check_prefill_dims(b, h, n, m_max, k, v) == MQA_OK ? 16 : 0;     // (the kernel keeps everything on chip)
 }
 
 int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int32_t* start, float* O, void* workspace,
@@ -963,43 +954,25 @@ int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int
     const int rc = check_prefill_dims(b, h, n, m_max, k, v);
     if (rc) return rc;
     if (workspace_bytes < mqa_prefill_workspace_bytes(b, h, n, m_max, k, v)) return MQA_ERR_WORKSPACE_TOO_SMALL;
-    if (n % kPfRows == 0) {
-        // whole tiles of 128 positions: the kernel of the batched form proper (two heads per CTA, no workspace used)
-        static std::atomic<int> opt_in[kMaxDevices];
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
-        if (!opt_in[dev].load(std::memory_order_acquire)) {
-            if (cudaFuncSetAttribute(mqa_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes) != cudaSuccess) {
-                cudaGetLastError();
-                return MQA_ERR_CUDA;
-            }
-            opt_in[dev].store(1, std::memory_order_release);
-        }
-        const long long ctas = (long long)(n / kPfRows) * b * ((h + 1) / 2);
-        if (ctas >= 0x7fffffffLL) return MQA_ERR_UNSUPPORTED;
-        alignas(64) CUtensorMap map_q, map_k, map_v;
-        if (!encode_cache_map(&map_q, Q, (long long)b * h * n, kPfRows) || !encode_cache_map(&map_k, K, (long long)b * m_max, kPfRows) ||
-            !encode_cache_map(&map_v, V, (long long)b * m_max, kPfRows))
+    static std::atomic<int> opt_in[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!opt_in[dev].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(mqa_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
             return MQA_ERR_CUDA;
-        launch_dependent(mqa_prefill_kernel, (unsigned)ctas, (unsigned)kPfThreads, (size_t)kPfSmemBytes, stream, map_q, map_k, map_v, start, O,
-                         status, b, h, n, m_max);
-        return launch_status();
-    }
-    const int per_head = n / kGroupRows;                       // groups of 64 positions per head
-    const long long total = (long long)b * h * per_head;
-    for (long long first = 0; first < total; first += kStreamMaxSeqs) {
-        const long long count = total - first < kStreamMaxSeqs ? total - first : kStreamMaxSeqs;
-        const Plan p = prefill_plan(count, m_max);
-        const QueryGroups grp = {h * per_head, h * n, (int)first, per_head};
-        int err = launch_umma<64, false, false, 2>(p, Q, K, V, start, O, workspace, status, b, h, m_max, stream, p.merge_in_kernel,
-                                                      nullptr, nullptr, nullptr, 0, &grp, (long long)b * h * n);
-        if (err) return err;
-        if (!p.merge_in_kernel) {
-            err = launch_stream_combine(p, workspace, O, nullptr, m_max, stream, grp);
-            if (err) return err;
         }
+        opt_in[dev].store(1, std::memory_order_release);
     }
-    return MQA_OK;
+    // a CTA per (tile of 128 positions, pair of heads, sequence); the last tile of a head may be partly filled
+    const long long ctas = (long long)((n + kPfRows - 1) / kPfRows) * b * ((h + 1) / 2);
+    alignas(64) CUtensorMap map_q, map_k, map_v;
+    if (!encode_cache_map(&map_q, Q, (long long)b * h * n, kPfRows) || !encode_cache_map(&map_k, K, (long long)b * m_max, kPfRows) ||
+        !encode_cache_map(&map_v, V, (long long)b * m_max, kPfRows))
+        return MQA_ERR_CUDA;
+    launch_dependent(mqa_prefill_kernel, (unsigned)ctas, (unsigned)kPfThreads, (size_t)kPfSmemBytes, stream, map_q, map_k, map_v, start, O,
+                     status, b, h, n, m_max);
+    return launch_status();
 }
 
 int mqa_set_wait_limit_cycles(long long cycles) {

@@ -65,7 +65,7 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                    const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ start, float* __restrict__ O,
                    int32_t* __restrict__ status, int b, int h, int n, int m_max) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pairs = (h + 1) >> 1, n_tiles = n / kPfRows;
+    const int pairs = (h + 1) >> 1, n_tiles = (n + kPfRows - 1) / kPfRows;
     const int pair = blockIdx.x % pairs;
     const int seq = (blockIdx.x / pairs) % b;
     const int pt = n_tiles - 1 - blockIdx.x / (pairs * b);
@@ -105,8 +105,10 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     grid_dependency_wait();              // Q, K, V and start may come from the kernel before
     grid_launch_dependents();
     const int raw = start ? __ldg(start + seq) : 0;
-    // rows of the memory this tile's last position sees; a memory that would pass m_max is cut there (flagged)
-    int L = raw + p0 + kPfRows;
+    // rows of the memory this tile's last position sees (the last tile of a head may hold fewer than 128 positions: the
+    // rows after them are computed on whatever the Q tile holds there and never stored); a memory that would pass m_max
+    // is cut there (flagged)
+    int L = raw + min(p0 + kPfRows, n);
     if (raw < 0 || raw + n > m_max) {
         if (threadIdx.x == 0 && status) atomicOr(status, kStatusLenClamped);
         if (L > m_max) L = m_max;
@@ -209,12 +211,14 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (w < n_act) {
             float* dst = O + (size_t)(q_row0 + (long long)w * n + r) * kHeadDim;
             if (n_kv == 0) {
-                for (int i = 0; i < kHeadDim; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (p0 + r < n)
+                    for (int i = 0; i < kHeadDim; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
             } else {
                 const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
                 const uint32_t s_t = lane_base + w * 128, o_t = lane_base + 256 + w * 128;
-                const int lim_first = min(raw + p0 + 1, m_max);           // rows the tile's first position sees
-                const int lim = min(raw + p0 + r + 1, m_max);             // rows this thread's position sees: >= 1
+                const int lim_first = min(raw + p0 + 1, L);               // rows the tile's first position sees
+                const int lim = min(raw + p0 + r + 1, L);                 // rows this thread's position sees: >= 1
+                const bool stored = p0 + r < n;                           // (a position of this head)
                 float m = -INFINITY, l = 0.f;                             // reference maximum (log2 units), sum of weights
                 bool ok = true;
                 for (int j = 0; j < n_kv; ++j) {
@@ -325,11 +329,13 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     uint32_t y[32];
                     tmem_ld32(o_t + c * 32, y);
                     tmem_wait_ld();
+                    if (stored) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<float4*>(dst + c * 32 + i) =
-                            make_float4(__uint_as_float(y[i]) * inv, __uint_as_float(y[i + 1]) * inv, __uint_as_float(y[i + 2]) * inv,
-                                        __uint_as_float(y[i + 3]) * inv);
+                        for (int i = 0; i < 32; i += 4)
+                            *reinterpret_cast<float4*>(dst + c * 32 + i) =
+                                make_float4(__uint_as_float(y[i]) * inv, __uint_as_float(y[i + 1]) * inv, __uint_as_float(y[i + 2]) * inv,
+                                            __uint_as_float(y[i + 3]) * inv);
+                    }
                 }
                 if (!ok) atomicExch(&timed_out, 1);
             }

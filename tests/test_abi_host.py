@@ -119,11 +119,12 @@ def test_plans_of_many_query_rows_and_of_the_batched_form(L):
     assert binding.workspace_bytes(32, 128, 8192) >= binding.workspace_bytes(32, 64, 8192)
     need = binding.prefill_workspace_bytes(2, 8, 128, 256)
     assert need > 0
-    assert binding.prefill_workspace_bytes(2, 8, 100, 256) == 0          # n must be a multiple of 64
+    assert binding.prefill_workspace_bytes(2, 8, 100, 256) > 0           # any number of positions
     assert binding.prefill_workspace_bytes(2, 8, 512, 256) == 0          # the queries' positions must fit the memory
+    assert binding.prefill_workspace_bytes(2, 8, 128, 256, k=64) == 0
     a = ctypes.c_void_p(0x1000)
     pf = L.mqa_prefill_attention
-    assert pf(a, a, a, None, a, a, need, None, 2, 8, 100, 256, 128, 128, None) == binding.ERR_UNSUPPORTED
+    assert pf(a, a, a, None, a, a, need, None, 2, 8, 512, 256, 128, 128, None) == binding.ERR_UNSUPPORTED
     assert pf(a, a, a, None, a, a, need - 1, None, 2, 8, 128, 256, 128, 128, None) == binding.ERR_WORKSPACE_TOO_SMALL
     assert pf(None, a, a, None, a, a, need, None, 2, 8, 128, 256, 128, 128, None) == binding.ERR_INVALID_ARG
     assert pf(a, a, a, ctypes.c_void_p(0x1002), a, a, need, None, 2, 8, 128, 256, 128, 128, None) == binding.ERR_INVALID_ARG

@@ -62,6 +62,10 @@ SMALL = [
     (2, 3, 256, 300, [44, 0]),                  # a head count that does not divide 64
     (1, 32, 128, 1100, [900]),                  # long memory in front of few queries
     (5, 16, 64, 2048, [1984, 0, 63, 64, 1000]),
+    (2, 5, 100, 260, [160, 0]),                 # n is no multiple of anything: the last tile of a head is partly filled
+    (3, 2, 1, 700, [0, 699, 350]),              # one position: a decoding step
+    (1, 3, 129, 129, None),                     # one position in a tile of its own
+    (2, 4, 333, 1200, [867, 5]),
 ]
 
 
@@ -169,7 +173,7 @@ def test_two_runs_are_bit_identical():
 
 
 def test_what_is_not_supported_is_refused_before_any_launch():
-    b, h, n, m_max = 2, 4, 100, 256                        # n is not a multiple of 64
+    b, h, n, m_max = 2, 4, 300, 256                        # more positions than the memory holds
     assert mqa.prefill_workspace_bytes(b, h, n, m_max) == 0
     Q = torch.zeros(b, h, n, 128, dtype=torch.bfloat16, device=DEV)
     K = torch.zeros(b, m_max, 128, dtype=torch.bfloat16, device=DEV)
