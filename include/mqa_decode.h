@@ -341,15 +341,15 @@ size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v);
  *          paper's M = X case, the processing of a whole prompt).  A negative start[b] is taken as an empty memory
  *          for that sequence (zeros) and flagged LEN_CLAMPED, like a bad lens.
  *   O      [b, h, n, v] fp32, written           status   optional; LEN_CLAMPED, PIPELINE_TIMEOUT
- *   workspace   at least mqa_prefill_workspace_bytes(b, h, n, m_max, k, v) bytes; as for mqa_decode_step.
- * n a multiple of 128: one kernel made for this form (mqa_prefill_kernel).  A CTA takes 128 consecutive positions of
- * two heads of a sequence -- the heads share K and V, so each staged 128-row K/V tile serves 256 query rows -- with
- * the query rows as the rows of the tensor-core tiles (one thread owns one query row's logits, maximum and sum), the
- * weights handed to the second product through tensor memory, and cache rows beyond a tile's last position never
- * fetched.  The workspace is not touched.  Otherwise (n a multiple of 64 only): each run of 64 consecutive positions
- * of one head is given to the persistent decoding kernel as 64 query rows over the cache rows up to its last
- * position, at most 1024 such runs per launch.  Supported: k = v = 128, n a multiple of 64 (MQA_ERR_UNSUPPORTED
- * otherwise).  A memory that would pass m_max (start[b] + n > m_max) is cut at m_max and flagged LEN_CLAMPED.
+ *   workspace   at least mqa_prefill_workspace_bytes(b, h, n, m_max, k, v) bytes (see below).
+ * One launch of a kernel made for this form (mqa_prefill_kernel).  A CTA takes 128 consecutive positions of two heads
+ * of a sequence -- the heads share K and V, so each staged 128-row K/V tile serves 256 query rows -- with the query
+ * rows as the rows of the tensor-core tiles (one thread owns one query row's logits, maximum and sum), the weights
+ * handed to the second product through tensor memory, and cache rows beyond a tile's last position never fetched.
+ * Any n >= 1 (the last tile of a head may be partly filled); k = v = 128 (MQA_ERR_UNSUPPORTED otherwise, and for
+ * n > m_max).  A memory that would pass m_max (start[b] + n > m_max) is cut at m_max and flagged LEN_CLAMPED.  The
+ * workspace is not touched by the present kernel; the argument stays in the interface (pass at least
+ * mqa_prefill_workspace_bytes() bytes, which is small and non-zero for supported sizes, 0 otherwise).
  */
 int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int32_t* start, float* O,
                           void* workspace, size_t workspace_bytes, int32_t* status,

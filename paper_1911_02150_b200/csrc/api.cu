@@ -363,18 +363,17 @@ constexpr int kEarlyTestWithhold = 1 << 8;    // rides on `early`: MQA_STEP_TEST
 std::atomic<int> g_umma_opt_in[kMaxDevices][13];
 
 // b, h: the caller's sequences and query rows per sequence (the kernel is given the plan's: sequences x groups, 64 rows
-// each, where the plan has groups).  grp_in: the groups of a launch of the batched form; otherwise derived from the plan.
+// each, where the plan has groups).
 template <int HP, bool FUSED, bool GUESS = false, int GROUPED = 0>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
                 const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
-                int early = 0, const QueryGroups* grp_in = nullptr, long long q_rows = 0) {
+                int early = 0) {
     using Cfg = UmmaCfg<HP>;
     auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS, GROUPED>;
     static_assert(GROUPED == 0 || HP == 64, "groups hold 64 query rows");
-    constexpr int kSlot = GROUPED == 2 ? 9 : GROUPED == 1 ? 10 + (GUESS ? 2 : FUSED ? 1 : 0)
-                                                          : (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
-    const QueryGroups grp = grp_in ? *grp_in : QueryGroups{p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0, 0};
+    constexpr int kSlot = GROUPED == 1 ? 10 + (GUESS ? 2 : FUSED ? 1 : 0) : (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
+    const QueryGroups grp = {p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
@@ -396,7 +395,7 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     const long long rows = (long long)b * m_max;             // (b caches, however many schedule sequences look at each)
     if (!encode_cache_map(&map_k, K, rows, kUmmaStageRows) || !encode_cache_map(&map_v, V, rows, kUmmaStageRows) ||
         !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows) ||
-        !encode_cache_map(&map_q, q, q_rows > 0 ? q_rows : (long long)b * h, HP))
+        !encode_cache_map(&map_q, q, (long long)b * h, HP))
         return MQA_ERR_CUDA;
     const StreamWorkspace w = stream_workspace(p, workspace);
     // a cache that cannot stay in L2 from one step to the next is streamed through it with the evict-first policy
@@ -486,7 +485,7 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     int rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
     if (p.stream()) {
-        const QueryGroups grp = {p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0, 0};
+        const QueryGroups grp = {p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0};
         return launch_stream_combine(p, workspace, o, lens_advance, m_max, stream, grp);
     }
     if (p.n_splits <= 1) return MQA_OK;

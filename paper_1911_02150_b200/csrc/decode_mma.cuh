@@ -663,12 +663,9 @@ __host__ __device__ inline size_t stream_ml_bytes(int slots, int h) {
 }
 __host__ __device__ inline size_t stream_acc_bytes(int slots, int h) { return (size_t)slots * h * kHeadDim * sizeof(float); }
 
-// Several sequences of the schedule may stand for ONE cache, kGroupRows query rows each:
-//   * a sequence with more than 64 query rows (more heads than that, or beams x heads, all over one shared
-//     memory) is cut into groups of 64 rows, each a schedule sequence of its own over the same cache rows;
-//   * in the batched form of Section 3 (n query positions per head, the autoregressive mask of Section 2.3)
-//     a schedule sequence is 64 consecutive positions of one head: position p attends over the rows up to its
-//     own, so the group's cache ends with its last position and only its last 63 rows need a mask per column.
+// Several sequences of the schedule may stand for ONE cache, kGroupRows query rows each: a sequence with more than
+// 64 query rows (more heads than that, or beams x heads, all over one shared memory) is cut into groups of 64 rows,
+// each a schedule sequence of its own over the same cache rows.
 // Schedule sequence s of a launch is number sg = first + s of all of them; its cache is kv = sg / per_kv; its
 // query (and output) rows are rows kv * rows_per_kv + (sg % per_kv) * 64 .. of the [rows, 128] q (o) matrix.
 constexpr int kGroupRows = 64;
@@ -676,7 +673,6 @@ struct QueryGroups {
     int per_kv;         // schedule sequences per cache (0: the plain step, one sequence per cache, no other field used)
     int rows_per_kv;    // query rows per cache
     int first;          // number of this launch's first schedule sequence (a launch holds at most kStreamMaxSeqs)
-    int causal_every;   // 0, or groups per head: sequence sg holds the query positions 64 * (sg % causal_every) .. + 63
 };
 __device__ __forceinline__ int group_kv(const QueryGroups& g, int s) { return g.per_kv == 0 ? s : (g.first + s) / g.per_kv; }
 // first query row of schedule sequence s (h: query rows per sequence of the plain step)
@@ -692,14 +688,10 @@ __device__ __forceinline__ int group_rows(const QueryGroups& g, int s, int h) {
 }
 
 // Rows of its cache that schedule sequence s may look at, as lens says (read from L2: the kernels before and
-// after this one may write lens).  In the batched form lens[kv] (null: 0) is the memory position of the head's
-// first query, and the group's last position is its last row.
+// after this one may write lens).
 template <bool FUSED>
 __device__ __forceinline__ int read_len(const int32_t* lens, int s, const QueryGroups& g) {
-    if (g.per_kv == 0) return __ldcg(lens + s);
-    const int raw = lens ? __ldcg(lens + group_kv(g, s)) : 0;
-    if (g.causal_every == 0) return raw;
-    return raw < 0 ? raw : raw + kGroupRows * ((g.first + s) % g.causal_every + 1);
+    return __ldcg(lens + group_kv(g, s));
 }
 
 // Rows of sequence s this launch attends over, and whether the step appends to it.
@@ -729,7 +721,7 @@ template <bool FUSED, int THREADS, int PENALTY>
 __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ lens, float* __restrict__ o,
                                                  int32_t* __restrict__ status, int b, int h, int m_max, bool appending,
                                                  unsigned long long magic, int* prefix, int* rows_of, int* plan_sm,
-                                                 int solo_warp = -1, const QueryGroups grp = QueryGroups{0, 0, 0, 0}) {
+                                                 int solo_warp = -1, const QueryGroups grp = QueryGroups{0, 0, 0}) {
     const int cta = blockIdx.x, G = gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int planners = solo_warp >= 0 ? THREADS - 32 : THREADS;
@@ -809,7 +801,7 @@ template <bool FUSED, int PENALTY>
 __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, int b, int m_max, bool appending,
                                               unsigned long long magic, Segment* g, int* rows, int cluster = 1, int rank = 0,
                                               int stage_tiles = 4, bool* strided = nullptr,
-                                              const QueryGroups grp = QueryGroups{0, 0, 0, 0}) {
+                                              const QueryGroups grp = QueryGroups{0, 0, 0}) {
     if (strided) *strided = false;
     if (b > kFastSeqs) return false;
     const int cta = blockIdx.x, lane = threadIdx.x & 31;

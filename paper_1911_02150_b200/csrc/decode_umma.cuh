@@ -356,7 +356,7 @@ __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__
 // HP = head rows of the Q tile (h rounded up to 16, 32 or 64).  GUESS: built with the code that starts copies on a
 // guess before the wait (GUESS && early >= 2 below); kernels without it take early 0 or 1 only.
 // GROUPED: 0 = every schedule sequence has its own cache (the plain step: nothing of QueryGroups is compiled in);
-// 1 = groups of 64 query rows over shared caches; 2 = the batched form, with its mask per column.
+// 1 = groups of 64 query rows over shared caches.
 template <int HP, bool FUSED, bool GUESS = false, int GROUPED = 0>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -368,8 +368,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int early_arg,
                               int read_once, const QueryGroups grp_arg) {
     using Cfg = UmmaCfg<HP>;
-    constexpr bool CAUSAL = GROUPED == 2;
-    const QueryGroups grp = GROUPED ? grp_arg : QueryGroups{0, 0, 0, 0};
+    const QueryGroups grp = GROUPED ? grp_arg : QueryGroups{0, 0, 0};
     const int early = GUESS ? early_arg : (early_arg == 1 ? 1 : 0);
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
@@ -884,9 +883,6 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     const int fetched = min(kSubs, g.hi - u) * kTileRows;
                     const int valid = min(fetched, L - u * kTileRows);
                     const bool row_ok = t < valid;
-                    // batched form: column c of the group is query position (last position) - 63 + c and looks at the
-                    // rows up to its own, i.e. at this thread's row iff (rows from it to the end) + c >= 64
-                    const int to_end = L - (u * kTileRows + t);
                     if (ok) ok = mbar_wait(s_ready + sb * 8, (j >> 1) & 1);
                     if (tid == 0) ST(j, 2);
                     tc_fence_after();
@@ -912,8 +908,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         const float mv[4] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const bool seen = !CAUSAL || to_end + head0 + i + e >= kGroupRows;
-                            x[i + e] = row_ok && seen ? __fmul_rn(__uint_as_float(xr[i + e]), kLog2e) : -INFINITY;   // select, never multiply
+                            x[i + e] = row_ok ? __fmul_rn(__uint_as_float(xr[i + e]), kLog2e) : -INFINITY;   // select, never multiply
                             lead = fmaxf(lead, x[i + e] - mv[e]);           // (-inf) - (-inf) = NaN is ignored by fmaxf
                         }
                     }
@@ -934,8 +929,6 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                             float m_new = m_old;
 #pragma unroll
                             for (int w = 0; w < 4; ++w) m_new = fmaxf(m_new, red_m[w * HP + tid]);   // finite: the stage has a valid row
-                            // (batched form: a column may see none of a piece's rows; a finite stand-in gives it weight 0)
-                            if (CAUSAL) m_new = fmaxf(m_new, -1e30f);
                             f_sm[tid] = fast_exp2(m_old - m_new);            // 0 on the first stage, 1 if unchanged
                             m_sm[tid] = m_new;
                         }
