@@ -18,6 +18,7 @@
 #include "decode_umma.cuh"
 #include "decode_local.cuh"
 #include "prefill.cuh"
+#include "decode_wide.cuh"
 
 namespace mqa {
 namespace {
@@ -41,7 +42,7 @@ int sm_count() {
     return n;
 }
 
-enum class Kernel { kSimt, kMma1, kMma2, kUmma };
+enum class Kernel { kSimt, kMma1, kMma2, kUmma, kWide };
 constexpr int kMergeInKernelMaxPieces = 10;
 constexpr int kMaxClusterCtas = 4;            // a sequence's CTAs as one thread-block cluster.  Measured per step: clusters of 8
                                               // (16 sequences x 16384 rows) 43 us against 29 us without, clusters of 16
@@ -147,9 +148,32 @@ Plan plan_stream(int b, int h, int m_max) {
     return p;
 }
 
+// Fixed splits for the kernel with the query rows as tile rows (decode_wide.cuh: 33 .. 128 query rows per sequence): one
+// CTA per (sequence, split), about one CTA per SM, splits of whole 128-row stages and never shorter than two of them.
+Plan plan_wide(int b, int h, int m_max) {
+    Plan p;
+    p.units = (size_t)b * h;
+    p.b = b; p.h = h;
+    p.kernel = Kernel::kWide;
+    int want = sm_count() / b;
+    const int cap = m_max / (2 * kWideRows);
+    if (want > cap) want = cap;
+    if (want > 160) want = 160;                    // (the second pass merges up to 160 pieces in one go)
+    if (want < 1) want = 1;
+    int chunk = (m_max + want - 1) / want;
+    chunk = (chunk + kWideRows - 1) / kWideRows * kWideRows;
+    p.chunk_rows = chunk;
+    p.n_splits = (m_max + chunk - 1) / chunk;
+    return p;
+}
+
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // a row space too large for the 32-bit TMA coordinates goes to the general CUDA-core kernel
     if (!(multi_query && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
+#ifndef MQA_WIDE_MIN_H
+#define MQA_WIDE_MIN_H 65
+#endif
+    if (h >= MQA_WIDE_MIN_H && h <= kWideRows && m_max >= 1024 && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
     if (h > kGroupRows) {
         // more query rows than one tile of the tensor-core kernel holds (beams x heads, many heads): groups of 64
         // rows, each a sequence of the persistent kernel's schedule over the same cache
@@ -434,6 +458,35 @@ int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, 
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA; }
 
+int launch_wide(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o, float2* part_ml,
+                float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias,
+                const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
+    FusedArgs fa = {};
+    if (k_new) {
+        fa.k_new = static_cast<const uint4*>(k_new);
+        fa.v_new = static_cast<const uint4*>(v_new);
+        fa.K = static_cast<uint4*>(const_cast<void*>(K));
+        fa.V = static_cast<uint4*>(const_cast<void*>(V));
+    }
+    static std::atomic<int> opt_in[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
+    if (!opt_in[dev].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(mqa_decode_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return MQA_ERR_CUDA;
+        }
+        opt_in[dev].store(1, std::memory_order_release);
+    }
+    alignas(64) CUtensorMap map_q, map_k, map_v;
+    if (!encode_cache_map(&map_q, q, (long long)b * h, kWideRows) || !encode_cache_map(&map_k, K, (long long)b * m_max, kWideRows) ||
+        !encode_cache_map(&map_v, V, (long long)b * m_max, kWideRows))
+        return MQA_ERR_CUDA;
+    launch_dependent(mqa_decode_wide_kernel, (unsigned)((size_t)b * p.n_splits), (unsigned)kWideThreads, (size_t)kWideSmemBytes, stream, map_q,
+                     map_k, map_v, lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows, p.n_splits, len_bias, fa, lens_advance);
+    return launch_status();
+}
+
 int run_split(bool multi_query, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
               void* workspace, size_t workspace_bytes, int32_t* status,
               int b, int h, int m_max, int k, int v, cudaStream_t stream, int len_bias = 0, bool merge_in_kernel = false) {
@@ -447,6 +500,7 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
         return launch_umma_for<false>(p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge_in_kernel);
     float2* part_ml = partials_ml(workspace);
     float* part_acc = partials_acc(p, workspace);
+    if (p.kernel == Kernel::kWide) return launch_wide(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, len_bias);
     if (p.kernel == Kernel::kMma1)
         return launch_mma<1>(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, len_bias);
     if (p.kernel == Kernel::kMma2)
@@ -744,6 +798,16 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
                    : launch_mma<2>(p, q, K, V, lens, o, nullptr, nullptr, status, b, h, m_max, stream, 0, k_new, v_new,
                                    advance ? lens : nullptr, withhold);
     }
+    if (p.kernel == Kernel::kWide) {
+        // many query rows: the CTA whose rows hold the new one writes it; one split per sequence moves lens on itself,
+        // otherwise the second pass does.  One or two launches.
+        float2* part_ml = partials_ml(workspace);
+        float* part_acc = partials_acc(p, workspace);
+        rc = launch_wide(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new,
+                         p.n_splits == 1 && advance ? lens : nullptr);
+        if (rc || p.n_splits == 1) return rc;
+        return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr, true);
+    }
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits > 1) {
         // fixed splits: the CTA whose rows hold the new one writes it; the second pass moves lens on.  Two launches.
         float2* part_ml = partials_ml(workspace);
@@ -919,6 +983,7 @@ int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits == 1) return 1;   // one CTA per sequence does it all
     if (p.stream()) return 2;                          // pass with the append inside, second pass
     if (p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) return 2;   // fixed splits: the same two
+    if (p.kernel == Kernel::kWide) return p.n_splits == 1 ? 1 : 2;
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }
 
@@ -995,6 +1060,7 @@ const char* mqa_plan_kernel_name(int multi_query, int whole_step, int b, int h, 
         }
         case Kernel::kMma1: return "mqa_decode_split_mma_kernel<1>";
         case Kernel::kMma2: return "mqa_decode_split_mma_kernel<2>";
+        case Kernel::kWide: return "mqa_decode_wide_kernel";
         default: return "decode_split_simt_kernel";
     }
 }
