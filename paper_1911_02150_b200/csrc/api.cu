@@ -170,10 +170,10 @@ Plan plan_wide(int b, int h, int m_max) {
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // a row space too large for the 32-bit TMA coordinates goes to the general CUDA-core kernel
     if (!(multi_query && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
-#ifndef MQA_WIDE_MIN_H
-#define MQA_WIDE_MIN_H 65
-#endif
-    if (h >= MQA_WIDE_MIN_H && h <= kWideRows && m_max >= 1024 && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
+    // 33 .. 128 query rows per sequence: the kernel with the query rows as tile rows (measured against the streaming
+    // kernel's 64-row tile, per step: 32 x 64 rows x 8192: 30.5 vs 35.0 us; 128 x 64 x 2048: 26.2 vs 32.8; 4 x 48 x 4096:
+    // 10.8 vs 20.7; and against groups of 64 at 128 rows, 32 x 8192: 34.9 vs 68.8 us)
+    if (h > 32 && h <= kWideRows && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
     if (h > kGroupRows) {
         // more query rows than one tile of the tensor-core kernel holds (beams x heads, many heads): groups of 64
         // rows, each a sequence of the persistent kernel's schedule over the same cache

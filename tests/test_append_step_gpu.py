@@ -71,10 +71,11 @@ def lens_mix(b, m_max, seed):
 CASES = [
     # b, h, m_max: plans with the append inside the pass (persistent kernels) ...
     (40, 16, 1500), (160, 32, 333), (300, 8, 200), (37, 32, 4000), (64, 5, 777),
-    # ... the persistent tcgen05 kernel (h > 32) ...
-    (40, 48, 1500), (33, 64, 2100),
-    # ... more than 64 query rows per sequence: groups of 64 rows over the same cache, each storing the new row ...
-    (24, 128, 2048), (20, 96, 1500),
+    # ... 33 .. 128 query rows per sequence: the kernel with the query rows as tile rows (fixed splits; the CTA whose rows
+    # hold the new one stores it; one split per sequence moves lens on itself, else the second pass does) ...
+    (40, 48, 1500), (33, 64, 2100), (24, 128, 2048), (20, 96, 1500), (150, 33, 700), (1, 127, 20000), (5, 65, 129),
+    # ... more query rows than that: groups of 64 rows over the same cache, each storing the new row ...
+    (6, 200, 3000),
     # ... and plans that run as separate launches (small batches)
     (4, 8, 300), (1, 16, 20000), (2, 40, 600),
 ]

@@ -139,11 +139,15 @@ STREAM = [
     (160, 32, 333, 31),
     (3, 16, 9000, 32),      # few long sequences: cut into many pieces, merged by the second-pass kernel
     (1, 8, 20000, 33),
-    # more than 64 query rows per sequence (beams x heads over one shared memory, or many heads): groups of 64 rows
-    (32, 128, 2048, 34),    # 4 beams x 32 heads: two groups; 64 schedule sequences on 128 CTAs (clusters of two)
-    (40, 96, 1500, 35),     # a last group of 32 rows
+    # 33 .. 128 query rows per sequence (many heads, or beams x heads over one shared memory): the query rows are the tile rows
+    (32, 128, 2048, 34),    # 4 beams x 32 heads
+    (40, 96, 1500, 35),
+    (16, 65, 1100, 37),     # one warp of the tile holds a single row of the sequence
+    (150, 33, 700, 40),     # more sequences than SMs: one split each, short caches (two roundings of the weights)
+    (1, 127, 20000, 41),    # one sequence in many splits
+    (7, 100, 127, 42),      # less than one stage
+    # more than 128: groups of 64 rows on the streaming kernel
     (3, 200, 9000, 36),     # few long sequences, four groups (the last of 8 rows): second-pass kernel
-    (16, 65, 1100, 37),     # one row more than a group
     # batches that divide the grid are launched as clusters (16 and 8 CTAs here); with mixed lengths the clusters
     # change nothing and one CTA merges a sequence's many pieces
     (8, 16, 20000, 38),
