@@ -548,6 +548,8 @@ def main():
     ap.add_argument("--no-layer", action="store_true", help="skip the timing of the whole layer step (projections either side)")
     ap.add_argument("--prefill-only", default=None, metavar="B,H,N",
                     help="time only the batched (prefill) form at these sizes and print its block (what the ncu capture of that kernel runs)")
+    ap.add_argument("--step-only", default=None, metavar="B,H,M",
+                    help="time only the multi-query append-and-attend step of this shape (full caches) and print it")
     ap.add_argument("--no-line-sweep", action="store_true", help="skip the long-context sweep points of the default line")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true", help="run every workload, both variants, and write the table to --sweep-out")
@@ -580,6 +582,13 @@ def main():
     if args.prefill_only:
         pb, ph, pn = (int(x) for x in args.prefill_only.split(","))
         print(json.dumps({"prefill": prefill_block(mqa, device, 0, pb, ph, pn)}))
+        return
+    if args.step_only:
+        sb, sh, sm = (int(x) for x in args.step_only.split(","))
+        w2 = wl.Workload(f"step_b{sb}_h{sh}_m{sm}", b=sb, h=sh, m_max=sm, lens="full")
+        row = quick_point(mqa, "mqa", w2, device, steps=10, min_rotate_bytes=4 * L2_BYTES)
+        row["kernel"] = mqa.plan_kernel_name(True, True, sb, sh, sm)
+        print(json.dumps({"step": row}))
         return
 
     peak, peak_kind = measured_peak()

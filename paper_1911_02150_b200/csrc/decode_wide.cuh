@@ -313,19 +313,12 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         } else {
             named_barrier(1, 256);
             // (the loads from tensor memory below are warp-wide instructions: every lane executes them, whether or not
-            // its row is one of the sequence's h query rows; only the stores to global memory are per row)
+            // its row is one of the sequence's h query rows)
             const bool stored = r < h;
             const size_t unit = (size_t)seq * h + (stored ? r : 0);
-            float* dst = n_splits == 1 ? o + unit * kHeadDim : part_acc + (unit * n_splits + split) * kHeadDim;
             if (n_kv == 0) {
-                // nothing of this split lies inside the prefix: zeros (one split) or an empty piece
-                if (stored) {
-                    if (n_splits == 1) {
-                        for (int i = 0; i < kHeadDim; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
-                    } else {
-                        part_ml[unit * n_splits + split] = make_float2(-INFINITY, 0.f);
-                    }
-                }
+                // nothing of this split lies inside the prefix: zeros (one split, written below) or an empty piece
+                if (stored && n_splits > 1) part_ml[unit * n_splits + split] = make_float2(-INFINITY, 0.f);
             } else {
                 const float2 other = ex_ml[r];
                 const bool two = other.x != -INFINITY;                                 // warpgroup 1 had a stage
@@ -334,27 +327,43 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 const float tot = f0 * l + f1 * other.y;
                 const float scale = n_splits == 1 ? 1.f / tot : 1.f;
                 const float g0 = f0 * scale, g1 = f1 * scale;
+                // the merged row goes back to shared memory, in place of warpgroup 1's: a thread's row is 512 bytes, and
+                // stored from here it would leave as 32 separate 16-byte pieces per instruction (measured: 4.7 us for the
+                // CTA's 64 KB); all eight warps then copy whole rows out, 512 contiguous bytes per instruction
+                float4* my_row = reinterpret_cast<float4*>(base + kPfTileBytes + r * 512);   // (plain accesses: the eight loads of a
+                                                                                            // block go out together, ahead of its stores)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t y[32];
                     tmem_ld32(o_t + c * 32, y);
-                    tmem_wait_ld();
-                    if (stored) {
+                    float4 u[8];
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            float4 v = make_float4(__uint_as_float(y[i]) * g0, __uint_as_float(y[i + 1]) * g0, __uint_as_float(y[i + 2]) * g0,
-                                                   __uint_as_float(y[i + 3]) * g0);
-                            if (two) {
-                                float4 u;
-                                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(u.x), "=f"(u.y), "=f"(u.z), "=f"(u.w)
-                                             : "r"(ex_o + ((((c * 8 + (i >> 2)) ^ (r & 31)) << 4))));
-                                v.x = fmaf(u.x, g1, v.x); v.y = fmaf(u.y, g1, v.y); v.z = fmaf(u.z, g1, v.z); v.w = fmaf(u.w, g1, v.w);
-                            }
-                            *reinterpret_cast<float4*>(dst + c * 32 + i) = v;
-                        }
+                    for (int i = 0; i < 8; ++i) u[i] = two ? my_row[(c * 8 + i) ^ (r & 31)] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float4 v;
+                        v.x = fmaf(u[i].x, g1, __uint_as_float(y[4 * i]) * g0);
+                        v.y = fmaf(u[i].y, g1, __uint_as_float(y[4 * i + 1]) * g0);
+                        v.z = fmaf(u[i].z, g1, __uint_as_float(y[4 * i + 2]) * g0);
+                        v.w = fmaf(u[i].w, g1, __uint_as_float(y[4 * i + 3]) * g0);
+                        my_row[(c * 8 + i) ^ (r & 31)] = v;
                     }
                 }
                 if (stored && n_splits > 1) part_ml[unit * n_splits + split] = make_float2(top, tot);
+            }
+        }
+        // ---- all eight warps: the CTA's rows from shared memory to o (one split) or to its piece
+        named_barrier(2, 256);
+        if (n_kv > 0 || n_splits == 1) {
+            for (int item = threadIdx.x; item < kWideRows * 32; item += 256) {
+                const int row = item >> 5, c16 = item & 31;                             // (a warp: one row, its 32 pieces of 16 bytes)
+                if (row >= h) break;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (n_kv > 0) v = reinterpret_cast<const float4*>(base + kPfTileBytes + row * 512)[c16 ^ (row & 31)];
+                const size_t unit = (size_t)seq * h + row;
+                float* dst = n_splits == 1 ? o + unit * kHeadDim : part_acc + (unit * n_splits + split) * kHeadDim;
+                reinterpret_cast<float4*>(dst)[c16] = v;
             }
         }
         if (!ok) atomicExch(&timed_out, 1);
