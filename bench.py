@@ -661,6 +661,9 @@ def main():
         out["layer_step"] = layer_block(mqa, w, device, seed, max(3, min(args.steps, 20)))
         out["paper_incremental"] = paper_loop_block(mqa, device, seed)
         out["layer_step"]["projections_us"] = out["layer_step"]["us_per_step"] - blk["us_per_step"]
+    if not args.no_layer and world == 1:
+        out["prefill"] = prefill_block(mqa, device, seed)
+        out["beam4_rows"] = many_rows_block(mqa, device, seed, w)
     if not args.no_mha:
         sth = StepState(mqa, "mha", w, device, seed, min_rotate_bytes=2 * L2_BYTES)
         rh = run_variant(sth, max(3, min(args.steps, 20)), 3, device, sample_clocks=False, use_graph=not args.no_graph)
@@ -669,9 +672,6 @@ def main():
         out["mqa_speedup_over_mha"] = out["mha"]["us_per_step"] / blk["us_per_step"]
         del sth
         torch.cuda.empty_cache()
-    if not args.no_layer and world == 1:
-        out["prefill"] = prefill_block(mqa, device, seed)
-        out["beam4_rows"] = many_rows_block(mqa, device, seed, w)
     if not args.no_line_sweep and world == 1:
         # the other long-context points and the ragged batch: us, GB/s, fraction of 8 TB/s, launches, both variants
         out["sweep"] = [quick_point(mqa, variant, wl.WORKLOADS[name], device)
