@@ -1028,14 +1028,16 @@ int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int
         }
         opt_in[dev].store(1, std::memory_order_release);
     }
-    // a CTA per (tile of 128 positions, pair of heads, sequence); the last tile of a head may be partly filled
+    // a unit of work per (tile of 128 positions, pair of heads, sequence); the last tile of a head may be partly filled.
+    // One CTA per SM walks the units, longest first.
     const long long ctas = (long long)((n + kPfRows - 1) / kPfRows) * b * ((h + 1) / 2);
+    const unsigned grid = (unsigned)(ctas < sm_count() ? ctas : sm_count());
     alignas(64) CUtensorMap map_q, map_k, map_v;
     if (!encode_cache_map(&map_q, Q, (long long)b * h * n, kPfRows) || !encode_cache_map(&map_k, K, (long long)b * m_max, kPfRows) ||
         !encode_cache_map(&map_v, V, (long long)b * m_max, kPfRows))
         return MQA_ERR_CUDA;
-    launch_dependent(mqa_prefill_kernel, (unsigned)ctas, (unsigned)kPfThreads, (size_t)kPfSmemBytes, stream, map_q, map_k, map_v, start, O,
-                     status, b, h, n, m_max);
+    launch_dependent(mqa_prefill_kernel, grid, (unsigned)kPfThreads, (size_t)kPfSmemBytes, stream, map_q, map_k, map_v, start, O,
+                     status, b, h, n, m_max, (int)ctas);
     return launch_status();
 }
 

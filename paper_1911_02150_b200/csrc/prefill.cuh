@@ -32,7 +32,7 @@ constexpr int kPfProducerWarp = 8, kPfMmaWarp = 9;
 constexpr int kPfRegsSoftmax = 216, kPfRegsOther = 72;
 constexpr float kPfMaxLead = 8.f;                              // log2 units a logit may exceed its row's reference by
 // barriers: q_full, k_full/k_empty[2], v_full/v_empty[2], s_ready[2], p_ready[2], pv_done[2]
-constexpr int kPfBarriers = 1 + 2 * kPfKSlots + 2 * kPfVSlots + 6;
+constexpr int kPfBarriers = 1 + 2 * kPfKSlots + 2 * kPfVSlots + 6 + 1;       // (+ q_empty)
 constexpr int kPfSmemBytes = (2 + kPfKSlots + kPfVSlots) * kPfTileBytes + kPfBarriers * 8 + 16 + 1024 /* alignment slack */;
 static_assert(kPfSmemBytes <= 227 * 1024, "exceeds the shared memory of one SM");
 
@@ -59,25 +59,48 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
-// grid: x = ((n_tiles - 1 - position tile) * b + sequence) * head pairs + pair: the longest rows of work first.
+// One unit of work: 128 positions of a pair of heads of one sequence.  Units are numbered ((n_tiles - 1 - position tile) *
+// b + sequence) * head pairs + pair, the longest first; CTA c takes units c, c + grid, c + 2 grid, ... one after the other
+// (a persistent kernel: barriers, tensor memory and the K/V rings are set up once, and the next unit's Q and first stages
+// are fetched, and its first logits computed, while the softmax warps still write the unit before out).
+struct PfItem {
+    int seq, p0, head0, n_act, raw, L, n_kv;
+    bool hilo;
+    long long q_row0;
+};
+__device__ __forceinline__ PfItem pf_item(int item, const int32_t* __restrict__ start, int b, int h, int n, int m_max) {
+    PfItem it;
+    const int pairs = (h + 1) >> 1, n_tiles = (n + kPfRows - 1) / kPfRows;
+    const int pair = item % pairs;
+    it.seq = (item / pairs) % b;
+    it.p0 = (n_tiles - 1 - item / (pairs * b)) * kPfRows;        // first query position of the tile
+    it.head0 = 2 * pair;
+    it.n_act = it.head0 + 1 < h ? 2 : 1;                         // heads of the unit (an odd head count leaves one alone)
+    it.raw = start ? __ldg(start + it.seq) : 0;
+    // rows of the memory the tile's last position sees (the last tile of a head may hold fewer than 128 positions: the
+    // rows after them are computed on whatever the Q tile holds there and never stored); a memory that would pass m_max
+    // is cut there
+    it.L = it.raw + min(it.p0 + kPfRows, n);
+    if (it.L > m_max) it.L = m_max;
+    const bool empty = it.raw < 0 || it.L <= 0;                  // nothing to look at: zeros (like a bad lens)
+    it.n_kv = empty ? 0 : (it.L + kPfRows - 1) / kPfRows;        // stages
+    it.hilo = it.L < kSingleRoundingMinRows;
+    it.q_row0 = ((long long)it.seq * h + it.head0) * n + it.p0;  // row of head 0's first query in [b h n, 128]
+    return it;
+}
+
 __global__ void __launch_bounds__(kPfThreads, 1)
 mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ start, float* __restrict__ O,
-                   int32_t* __restrict__ status, int b, int h, int n, int m_max) {
+                   int32_t* __restrict__ status, int b, int h, int n, int m_max, int n_items) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pairs = (h + 1) >> 1, n_tiles = (n + kPfRows - 1) / kPfRows;
-    const int pair = blockIdx.x % pairs;
-    const int seq = (blockIdx.x / pairs) % b;
-    const int pt = n_tiles - 1 - blockIdx.x / (pairs * b);
-    const int p0 = pt * kPfRows;                                // first query position of the tile
-    const int head0 = 2 * pair;
-    const int n_act = head0 + 1 < h ? 2 : 1;                    // heads of this CTA (an odd head count leaves one alone)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);     // the 128-byte swizzle repeats every 1 KiB
     const uint32_t q_s = smem_addr(base);
     const uint32_t k_ring = q_s + 2 * kPfTileBytes, v_ring = k_ring + kPfKSlots * kPfTileBytes;
     const uint32_t bars = v_ring + kPfVSlots * kPfTileBytes;
+    const uint32_t q_empty = bars + 8 * (kPfBarriers - 1);       // the unit's Q tiles have been read for the last time
     const uint32_t q_full = bars, k_full = bars + 8, k_empty = k_full + 8 * kPfKSlots, v_full = k_empty + 8 * kPfKSlots,
                    v_empty = v_full + 8 * kPfVSlots, s_ready = v_empty + 8 * kPfVSlots, p_ready = s_ready + 16,
                    pv_done = p_ready + 16;
@@ -87,6 +110,7 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (threadIdx.x == 0) {
         prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
         mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
         for (int i = 0; i < kPfKSlots; ++i) { mbar_init(k_full + 8 * i, 1); mbar_init(k_empty + 8 * i, 1); }
         for (int i = 0; i < kPfVSlots; ++i) { mbar_init(v_full + 8 * i, 1); mbar_init(v_empty + 8 * i, 1); }
         for (int w = 0; w < 2; ++w) { mbar_init(s_ready + 8 * w, 1); mbar_init(p_ready + 8 * w, 4); mbar_init(pv_done + 8 * w, 1); }
@@ -104,102 +128,125 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t tmem_base = *tmem_slot;
     grid_dependency_wait();              // Q, K, V and start may come from the kernel before
     grid_launch_dependents();
-    const int raw = start ? __ldg(start + seq) : 0;
-    // rows of the memory this tile's last position sees (the last tile of a head may hold fewer than 128 positions: the
-    // rows after them are computed on whatever the Q tile holds there and never stored); a memory that would pass m_max
-    // is cut there (flagged)
-    int L = raw + min(p0 + kPfRows, n);
-    if (raw < 0 || raw + n > m_max) {
-        if (threadIdx.x == 0 && status) atomicOr(status, kStatusLenClamped);
-        if (L > m_max) L = m_max;
+    // the units of this CTA: c, 2G - 1 - c, 2G + c, 4G - 1 - c, ... (G CTAs; the units come longest first, so taking them
+    // forwards and backwards in turn evens the CTAs' totals out)
+    auto pf_unit = [&](int round) -> int {
+        const int G = (int)gridDim.x, c = (int)blockIdx.x;
+        return round * G + ((round & 1) ? G - 1 - c : c);
+    };
+    if (start && threadIdx.x < 32) {
+        // a start that is negative or leaves too little room is flagged once (its rows are zeros, or the memory is cut at m_max)
+        bool bad = false;
+        for (int i = blockIdx.x * 32 + threadIdx.x; i < b; i += gridDim.x * 32) bad = bad || start[i] < 0 || start[i] + n > m_max;
+        if (bad && status) atomicOr(status, kStatusLenClamped);
     }
-    const bool empty = raw < 0 || L <= 0;                      // nothing to look at: zeros (like a bad lens)
-    const int n_kv = empty ? 0 : (L + kPfRows - 1) / kPfRows;   // stages
-    const bool hilo = L < kSingleRoundingMinRows;
-    const long long q_row0 = ((long long)seq * h + head0) * n + p0;     // row of head 0's first query in [b h n, 128]
 
     if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPfRegsOther));
     if (warp == kPfProducerWarp) {
         // =============================================================== TMA producer
-        if (lane == 0 && n_kv > 0) {
+        if (lane == 0) {
             bool ok = true;
-            mbar_expect_tx(q_full, n_act * kPfTileBytes);
-            for (int w = 0; w < n_act; ++w)
-                for (int half = 0; half < 2; ++half)
-                    tma_load_2d(q_s + w * kPfTileBytes + half * kPfHalfBytes, &map_q, half * kBoxCols, (int)(q_row0 + (long long)w * n), q_full);
-            int issued_k = 0, issued_v = 0;
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const int y = seq * m_max + j * kPfRows;
-                const int ks = j % kPfKSlots, vs = j % kPfVSlots;
-                if (j >= kPfKSlots) ok = mbar_wait(k_empty + 8 * ks, ((j / kPfKSlots) - 1) & 1);
+            int g = 0, qi = 0;                                   // stages and units so far (they number the barriers' phases)
+            int issued_k = 0, issued_v = 0, issued_q = 0;
+            for (int round = 0, item; (item = pf_unit(round)) < n_items && ok; ++round) {
+                const PfItem it = pf_item(item, start, b, h, n, m_max);
+                if (it.n_kv == 0) continue;
+                if (qi > 0) ok = mbar_wait(q_empty, (qi - 1) & 1);            // the unit before has read its Q for the last time
                 if (!ok) break;
-                mbar_expect_tx(k_full + 8 * ks, kPfTileBytes);
-                tma_load_2d(k_ring + ks * kPfTileBytes, &map_k, 0, y, k_full + 8 * ks);
-                tma_load_2d(k_ring + ks * kPfTileBytes + kPfHalfBytes, &map_k, kBoxCols, y, k_full + 8 * ks);
-                issued_k = j + 1;
-                if (j >= kPfVSlots) ok = mbar_wait(v_empty + 8 * vs, ((j / kPfVSlots) - 1) & 1);
-                if (!ok) break;
-                mbar_expect_tx(v_full + 8 * vs, kPfTileBytes);
-                tma_load_2d(v_ring + vs * kPfTileBytes, &map_v, 0, y, v_full + 8 * vs);
-                tma_load_2d(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs);
-                issued_v = j + 1;
+                mbar_expect_tx(q_full, it.n_act * kPfTileBytes);
+                for (int w = 0; w < it.n_act; ++w)
+                    for (int half = 0; half < 2; ++half)
+                        tma_load_2d(q_s + w * kPfTileBytes + half * kPfHalfBytes, &map_q, half * kBoxCols, (int)(it.q_row0 + (long long)w * n), q_full);
+                issued_q = qi + 1;
+                for (int j = 0; j < it.n_kv && ok; ++j) {
+                    const int G = g + j;
+                    const int y = it.seq * m_max + j * kPfRows;
+                    const int ks = G % kPfKSlots, vs = G % kPfVSlots;
+                    if (G >= kPfKSlots) ok = mbar_wait(k_empty + 8 * ks, ((G / kPfKSlots) - 1) & 1);
+                    if (!ok) break;
+                    mbar_expect_tx(k_full + 8 * ks, kPfTileBytes);
+                    tma_load_2d(k_ring + ks * kPfTileBytes, &map_k, 0, y, k_full + 8 * ks);
+                    tma_load_2d(k_ring + ks * kPfTileBytes + kPfHalfBytes, &map_k, kBoxCols, y, k_full + 8 * ks);
+                    issued_k = G + 1;
+                    if (G >= kPfVSlots) ok = mbar_wait(v_empty + 8 * vs, ((G / kPfVSlots) - 1) & 1);
+                    if (!ok) break;
+                    mbar_expect_tx(v_full + 8 * vs, kPfTileBytes);
+                    tma_load_2d(v_ring + vs * kPfTileBytes, &map_v, 0, y, v_full + 8 * vs);
+                    tma_load_2d(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs);
+                    issued_v = G + 1;
+                }
+                g += it.n_kv;
+                ++qi;
             }
             if (!ok) {
                 // a wait ran out: the copies already started are given a bounded wait each before the CTA may leave
                 atomicExch(&timed_out, 1);
-                mbar_wait(q_full, 0);
-                for (int j = max(0, issued_k - kPfKSlots); j < issued_k; ++j) mbar_wait(k_full + 8 * (j % kPfKSlots), (j / kPfKSlots) & 1);
-                for (int j = max(0, issued_v - kPfVSlots); j < issued_v; ++j) mbar_wait(v_full + 8 * (j % kPfVSlots), (j / kPfVSlots) & 1);
+                if (issued_q > 0) mbar_wait(q_full, (issued_q - 1) & 1);
+                for (int G = max(0, issued_k - kPfKSlots); G < issued_k; ++G) mbar_wait(k_full + 8 * (G % kPfKSlots), (G / kPfKSlots) & 1);
+                for (int G = max(0, issued_v - kPfVSlots); G < issued_v; ++G) mbar_wait(v_full + 8 * (G % kPfVSlots), (G / kPfVSlots) & 1);
             }
         }
     } else if (warp == kPfMmaWarp) {
         // =============================================================== issuer of both products
-        if (lane == 0 && n_kv > 0) {
+        if (lane == 0) {
             constexpr uint32_t kIdescS = umma_idesc(128, 128, false, false);
             constexpr uint32_t kIdescO = umma_idesc(128, 128, false, true);
-            bool ok = mbar_wait(q_full, 0);
-            auto issue_s = [&](int w, int j) {                  // S_w = Q_w K_j^T into its 128 columns
-                const uint32_t k_s = k_ring + (j % kPfKSlots) * kPfTileBytes, qw = q_s + w * kPfTileBytes;
+            bool ok = true;
+            int g = 0, qi = 0, c_done[2] = {0, 0};               // stages, units, and stages of each head so far
+            for (int round = 0, item; (item = pf_unit(round)) < n_items && ok; ++round) {
+                const PfItem it = pf_item(item, start, b, h, n, m_max);
+                if (it.n_kv == 0) continue;
+                const int n_act = it.n_act, n_kv = it.n_kv;
+                auto issue_s = [&](int w, int G) {              // S_w = Q_w K^T into its 128 columns
+                    const uint32_t k_s = k_ring + (G % kPfKSlots) * kPfTileBytes, qw = q_s + w * kPfTileBytes;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {                // 8 k-steps of 16 columns; 4 per 64-column box
-                    const uint32_t off = (ks >> 2) * kPfHalfBytes + (ks & 3) * 32;
-                    umma_ss(tmem_base + w * 128, umma_desc(qw + off, 16, 1024), umma_desc(k_s + off, 16, 1024), kIdescS, ks ? 1u : 0u);
-                }
-                tc_commit(s_ready + 8 * w);
-            };
-            auto issue_pv = [&](int w, int j) {                 // O_w += P_w V_j: P from TMEM (bf16 pairs: 8 columns per 16 rows of V)
-                const uint32_t v_s = v_ring + (j % kPfVSlots) * kPfTileBytes;
-                for (int part = 0; part < (hilo ? 2 : 1); ++part) {
+                    for (int ks = 0; ks < 8; ++ks) {            // 8 k-steps of 16 columns; 4 per 64-column box
+                        const uint32_t off = (ks >> 2) * kPfHalfBytes + (ks & 3) * 32;
+                        umma_ss(tmem_base + w * 128, umma_desc(qw + off, 16, 1024), umma_desc(k_s + off, 16, 1024), kIdescS, ks ? 1u : 0u);
+                    }
+                    tc_commit(s_ready + 8 * w);
+                };
+                auto issue_pv = [&](int w, int G, bool first) {  // O_w += P_w V: P from TMEM (bf16 pairs: 8 columns per 16 rows of V)
+                    const uint32_t v_s = v_ring + (G % kPfVSlots) * kPfTileBytes;
+                    for (int part = 0; part < (it.hilo ? 2 : 1); ++part) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + (kk >> 1) * 32 + part * 16 + (kk & 1) * 8,
-                                umma_desc(v_s + kk * 2048, kPfHalfBytes, 1024), kIdescO, (j == 0 && part == 0 && kk == 0) ? 0u : 1u);
-                }
-                tc_commit(pv_done + 8 * w);
-            };
-            if (ok) ok = mbar_wait(k_full, 0);
-            tc_fence_after();
-            if (ok) {
-                for (int w = 0; w < n_act; ++w) issue_s(w, 0);
-                tc_commit(k_empty);
-            }
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const bool more = j + 1 < n_kv;
-                for (int w = 0; w < n_act && ok; ++w) {
-                    ok = mbar_wait(p_ready + 8 * w, j & 1);
-                    if (ok && w == 0) ok = mbar_wait(v_full + 8 * (j % kPfVSlots), (j / kPfVSlots) & 1);
-                    if (ok && w == 0 && more) ok = mbar_wait(k_full + 8 * ((j + 1) % kPfKSlots), ((j + 1) / kPfKSlots) & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    ST(j, 6 + w);
-                    issue_pv(w, j);
-                    if (w == n_act - 1) tc_commit(v_empty + 8 * (j % kPfVSlots));
-                    if (more) {
-                        issue_s(w, j + 1);
-                        if (w == n_act - 1) tc_commit(k_empty + 8 * ((j + 1) % kPfKSlots));
+                        for (int kk = 0; kk < 8; ++kk)
+                            umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + (kk >> 1) * 32 + part * 16 + (kk & 1) * 8,
+                                    umma_desc(v_s + kk * 2048, kPfHalfBytes, 1024), kIdescO, (first && part == 0 && kk == 0) ? 0u : 1u);
+                    }
+                    tc_commit(pv_done + 8 * w);
+                };
+                ok = mbar_wait(q_full, qi & 1);
+                if (ok) ok = mbar_wait(k_full + 8 * (g % kPfKSlots), (g / kPfKSlots) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                for (int w = 0; w < n_act; ++w) issue_s(w, g);
+                tc_commit(k_empty + 8 * (g % kPfKSlots));
+                if (n_kv == 1) tc_commit(q_empty);
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const bool more = j + 1 < n_kv;
+                    const int G = g + j;
+                    for (int w = 0; w < n_act && ok; ++w) {
+                        ok = mbar_wait(p_ready + 8 * w, (c_done[w] + j) & 1);
+                        if (ok && w == 0) ok = mbar_wait(v_full + 8 * (G % kPfVSlots), (G / kPfVSlots) & 1);
+                        if (ok && w == 0 && more) ok = mbar_wait(k_full + 8 * ((G + 1) % kPfKSlots), ((G + 1) / kPfKSlots) & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(w, G, j == 0);
+                        if (w == n_act - 1) tc_commit(v_empty + 8 * (G % kPfVSlots));
+                        if (more) {
+                            issue_s(w, G + 1);
+                            if (w == n_act - 1) {
+                                tc_commit(k_empty + 8 * ((G + 1) % kPfKSlots));
+                                if (j + 2 == n_kv) tc_commit(q_empty);       // the unit's last logits are on their way
+                            }
+                        }
                     }
                 }
+                g += n_kv;
+                ++qi;
+                for (int w = 0; w < n_act; ++w) c_done[w] += n_kv;
             }
             if (!ok) atomicExch(&timed_out, 1);
         }
@@ -208,138 +255,143 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPfRegsSoftmax));
         // =============================================================== softmax warps: one thread per query row
         const int w = warp >> 2, quarter = warp & 3, r = quarter * 32 + lane;
-        if (w < n_act) {
-            float* dst = O + (size_t)(q_row0 + (long long)w * n + r) * kHeadDim;
-            if (n_kv == 0) {
-                if (p0 + r < n)
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t s_t = lane_base + w * 128, o_t = lane_base + 256 + w * 128;
+        bool ok = true;
+        int g = 0, c_done = 0;                                   // stages of the CTA and of this head so far
+        for (int round = 0, item; (item = pf_unit(round)) < n_items; ++round) {
+            const PfItem it = pf_item(item, start, b, h, n, m_max);
+            if (w >= it.n_act) { g += it.n_kv; continue; }       // (an odd head count: the unit has one head)
+            const int p0 = it.p0, raw = it.raw;
+            float* dst = O + (size_t)(it.q_row0 + (long long)w * n + r) * kHeadDim;
+            const bool stored = p0 + r < n;                      // (a position of this head)
+            if (it.n_kv == 0) {
+                if (stored)
                     for (int i = 0; i < kHeadDim; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
-            } else {
-                const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-                const uint32_t s_t = lane_base + w * 128, o_t = lane_base + 256 + w * 128;
-                const int lim_first = min(raw + p0 + 1, L);               // rows the tile's first position sees
-                const int lim = min(raw + p0 + r + 1, L);                 // rows this thread's position sees: >= 1
-                const bool stored = p0 + r < n;                           // (a position of this head)
-                float m = -INFINITY, l = 0.f;                             // reference maximum (log2 units), sum of weights
-                bool ok = true;
-                for (int j = 0; j < n_kv; ++j) {
-                    const int k0 = j * kPfRows;
-                    if (ok) ok = mbar_wait(s_ready + 8 * w, j & 1);
-                    if (r == 0) ST(j, w * 3);
-                    tc_fence_after();
-                    const bool diag = k0 + kPfRows > lim_first;           // some position of the tile cannot see all of this stage
-                    // ---- the row's 128 logits, read once and kept in registers.  The mask of Section 2.3 is applied
-                    // by index, as a select: what lies behind a masked logit is never used.
-                    uint32_t x[128];
-                    tmem_ld_cols<128>(s_t, x);
-                    tmem_wait_ld();
-                    if (diag) {
-#pragma unroll
-                        for (int i = 0; i < 128; ++i)
-                            if (k0 + i >= lim) x[i] = 0xff800000u;        // -inf
-                    }
-                    float mx8[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1]));
-#pragma unroll
-                    for (int i = 8; i < 64; ++i) mx8[i & 7] = max3(mx8[i & 7], __uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1]));
-                    const float mx = max3(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * kLog2e;
-                    if (__any_sync(0xffffffffu, mx > m + kPfMaxLead)) {
-                        const float m_new = fmaxf(m, mx);
-                        if (j > 0) {
-                            const float f = fast_exp2(m - m_new);         // (m is finite from the first stage on)
-                            l *= f;
-                            if (ok) ok = mbar_wait(pv_done + 8 * w, (j - 1) & 1);    // O holds the stages before this one
-                            tc_fence_after();
-#pragma unroll 1
-                            for (int c = 0; c < 16; ++c) {
-                                uint32_t y[8];
-                                tmem_ld8(o_t + c * 8, y);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * f);
-                                tmem_st8(o_t + c * 8, y);
-                            }
-                        }
-                        m = m_new;
-                    }
-                    const unsigned long long neg_m2 = f2_pack(-m, -m), log2e2 = f2_pack(kLog2e, kLog2e);
-                    unsigned long long sum2[2] = {0ull, 0ull};
-                    if (hilo) {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t hi[16];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                float a0, a1;
-                                f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
-                                const float pa = fast_exp2(a0), pb = fast_exp2(a1);
-                                sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
-                                hi[i] = pack_bf16(pa, pb);
-                                x[c * 32 + i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
-                            }
-                            tmem_st16(s_t + c * 32, hi);
-                            tmem_st16(s_t + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 32]));
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t hi[16];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                float a0, a1;
-                                f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
-                                const float pa = fast_exp2(a0), pb = fast_exp2(a1);
-                                sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
-                                hi[i] = pack_bf16(pa, pb);
-                            }
-                            tmem_st16(s_t + c * 32, hi);
-                        }
-                    }
-                    {
-                        float s0, s1;
-                        f2_unpack(f2_add(sum2[0], sum2[1]), s0, s1);
-                        l += s0 + s1;
-                    }
-                    tmem_wait_st();
-                    tc_fence_before();
-                    if (w == 0 && j == n_kv - 1 && L < k0 + kPfRows) {
-                        // the last stage runs past the memory: the tensor core would multiply the zero weights with
-                        // whatever lies there (NaN * 0 = NaN), so those V rows are cleared first
-                        const int vs = j % kPfVSlots;
-                        if (ok) ok = mbar_wait(v_full + 8 * vs, (j / kPfVSlots) & 1);
-                        const uint32_t v_s = v_ring + vs * kPfTileBytes;
-                        const int first = L - k0;
-                        for (int i = r; i < (kPfRows - first) * 16; i += 128) {
-                            const int vrow = first + (i >> 4), ch = i & 15;
-                            const uint32_t a = v_s + (ch >> 3) * kPfHalfBytes + vrow * 128 + ((ch & 7) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
-                        }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(p_ready + 8 * w);
-                    if (r == 0) ST(j, w * 3 + 2);
-                }
-                // ---- the row of O, divided by the sum of its weights
-                if (ok) ok = mbar_wait(pv_done + 8 * w, (n_kv - 1) & 1);
-                tc_fence_after();
-                const float inv = 1.f / l;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t y[32];
-                    tmem_ld32(o_t + c * 32, y);
-                    tmem_wait_ld();
-                    if (stored) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<float4*>(dst + c * 32 + i) =
-                                make_float4(__uint_as_float(y[i]) * inv, __uint_as_float(y[i + 1]) * inv, __uint_as_float(y[i + 2]) * inv,
-                                            __uint_as_float(y[i + 3]) * inv);
-                    }
-                }
-                if (!ok) atomicExch(&timed_out, 1);
+                continue;
             }
+            const int lim_first = min(raw + p0 + 1, it.L);       // rows the tile's first position sees
+            const int lim = min(raw + p0 + r + 1, it.L);         // rows this thread's position sees: >= 1
+            float m = -INFINITY, l = 0.f;                        // reference maximum (log2 units), sum of weights
+            for (int j = 0; j < it.n_kv; ++j) {
+                const int k0 = j * kPfRows;
+                if (ok) ok = mbar_wait(s_ready + 8 * w, (c_done + j) & 1);
+                tc_fence_after();
+                const bool diag = k0 + kPfRows > lim_first;           // some position of the tile cannot see all of this stage
+                // ---- the row's 128 logits, read once and kept in registers.  The mask of Section 2.3 is applied
+                // by index, as a select: what lies behind a masked logit is never used.
+                uint32_t x[128];
+                tmem_ld_cols<128>(s_t, x);
+                tmem_wait_ld();
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (k0 + i >= lim) x[i] = 0xff800000u;        // -inf
+                }
+                float mx8[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1]));
+#pragma unroll
+                for (int i = 8; i < 64; ++i) mx8[i & 7] = max3(mx8[i & 7], __uint_as_float(x[2 * i]), __uint_as_float(x[2 * i + 1]));
+                const float mx = max3(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * kLog2e;
+                if (__any_sync(0xffffffffu, mx > m + kPfMaxLead)) {
+                    const float m_new = fmaxf(m, mx);
+                    if (j > 0) {
+                        const float f = fast_exp2(m - m_new);         // (m is finite from the first stage on)
+                        l *= f;
+                        if (ok) ok = mbar_wait(pv_done + 8 * w, (c_done + j - 1) & 1);    // O holds the stages before this one
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c = 0; c < 16; ++c) {
+                            uint32_t y[8];
+                            tmem_ld8(o_t + c * 8, y);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * f);
+                            tmem_st8(o_t + c * 8, y);
+                        }
+                    }
+                    m = m_new;
+                }
+                const unsigned long long neg_m2 = f2_pack(-m, -m), log2e2 = f2_pack(kLog2e, kLog2e);
+                unsigned long long sum2[2] = {0ull, 0ull};
+                if (it.hilo) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t hi[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float a0, a1;
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
+                            const float pa = fast_exp2(a0), pb = fast_exp2(a1);
+                            sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
+                            hi[i] = pack_bf16(pa, pb);
+                            x[c * 32 + i] = pack_bf16(pa - bf16_lo(hi[i]), pb - bf16_hi(hi[i]));
+                        }
+                        tmem_st16(s_t + c * 32, hi);
+                        tmem_st16(s_t + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 32]));
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t hi[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float a0, a1;
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(x[c * 32 + 2 * i]), __uint_as_float(x[c * 32 + 2 * i + 1])), log2e2, neg_m2), a0, a1);
+                            const float pa = fast_exp2(a0), pb = fast_exp2(a1);
+                            sum2[i & 1] = f2_add(sum2[i & 1], f2_pack(pa, pb));
+                            hi[i] = pack_bf16(pa, pb);
+                        }
+                        tmem_st16(s_t + c * 32, hi);
+                    }
+                }
+                {
+                    float s0, s1;
+                    f2_unpack(f2_add(sum2[0], sum2[1]), s0, s1);
+                    l += s0 + s1;
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                if (w == 0 && j == it.n_kv - 1 && it.L < k0 + kPfRows) {
+                    // the last stage runs past the memory: the tensor core would multiply the zero weights with
+                    // whatever lies there (NaN * 0 = NaN), so those V rows are cleared first
+                    const int vs = (g + j) % kPfVSlots;
+                    if (ok) ok = mbar_wait(v_full + 8 * vs, ((g + j) / kPfVSlots) & 1);
+                    const uint32_t v_s = v_ring + vs * kPfTileBytes;
+                    const int first = it.L - k0;
+                    for (int i = r; i < (kPfRows - first) * 16; i += 128) {
+                        const int vrow = first + (i >> 4), ch = i & 15;
+                        const uint32_t a = v_s + (ch >> 3) * kPfHalfBytes + vrow * 128 + ((ch & 7) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_ready + 8 * w);
+            }
+            // ---- the row of O, divided by the sum of its weights
+            if (ok) ok = mbar_wait(pv_done + 8 * w, (c_done + it.n_kv - 1) & 1);
+            tc_fence_after();
+            const float inv = 1.f / l;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t y[32];
+                tmem_ld32(o_t + c * 32, y);
+                tmem_wait_ld();
+                if (stored) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4*>(dst + c * 32 + i) =
+                            make_float4(__uint_as_float(y[i]) * inv, __uint_as_float(y[i + 1]) * inv, __uint_as_float(y[i + 2]) * inv,
+                                        __uint_as_float(y[i + 3]) * inv);
+                }
+            }
+            tc_fence_before();                                   // (the next unit's first product overwrites O once its weights are in)
+            g += it.n_kv;
+            c_done += it.n_kv;
         }
+        if (!ok) atomicExch(&timed_out, 1);
     }
     tc_fence_before();
     __syncthreads();
