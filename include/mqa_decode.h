@@ -343,8 +343,8 @@ size_t mqa_layer_workspace_bytes(int b, int h, int d, int m_max, int k, int v);
  *          for that sequence (zeros) and flagged LEN_CLAMPED, like a bad lens.
  *   O      [b, h, n, v] fp32, written           status   optional; LEN_CLAMPED, PIPELINE_TIMEOUT
  *   workspace   at least mqa_prefill_workspace_bytes(b, h, n, m_max, k, v) bytes (see below).
- * One launch of a kernel made for this form (mqa_prefill_kernel).  A CTA takes 128 consecutive positions of two heads
- * of a sequence -- the heads share K and V, so each staged 128-row K/V tile serves 256 query rows -- with the query
+ * One launch of a persistent kernel made for this form (mqa_prefill_kernel: a CTA per SM walks the units of work).  A
+ * unit is 128 consecutive positions of two heads of a sequence -- the heads share K and V, so each staged 128-row K/V tile serves 256 query rows -- with the query
  * rows as the rows of the tensor-core tiles (one thread owns one query row's logits, maximum and sum), the weights
  * handed to the second product through tensor memory, and cache rows beyond a tile's last position never fetched.
  * Any n >= 1 (the last tile of a head may be partly filled); k = v = 128 (MQA_ERR_UNSUPPORTED otherwise, and for
