@@ -460,7 +460,7 @@ int launch_status() { return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ER
 
 int launch_wide(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o, float2* part_ml,
                 float* part_acc, int32_t* status, int b, int h, int m_max, cudaStream_t stream, int len_bias,
-                const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr) {
+                const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr, bool withhold = false) {
     FusedArgs fa = {};
     if (k_new) {
         fa.k_new = static_cast<const uint4*>(k_new);
@@ -483,7 +483,8 @@ int launch_wide(const Plan& p, const void* q, const void* K, const void* V, cons
         !encode_cache_map(&map_v, V, (long long)b * m_max, kWideRows))
         return MQA_ERR_CUDA;
     launch_dependent(mqa_decode_wide_kernel, (unsigned)((size_t)b * p.n_splits), (unsigned)kWideThreads, (size_t)kWideSmemBytes, stream, map_q,
-                     map_k, map_v, lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows, p.n_splits, len_bias, fa, lens_advance);
+                     map_k, map_v, lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows, p.n_splits, len_bias, fa, lens_advance,
+                     withhold ? 1 : 0);
     return launch_status();
 }
 
@@ -804,7 +805,7 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
         float2* part_ml = partials_ml(workspace);
         float* part_acc = partials_acc(p, workspace);
         rc = launch_wide(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new,
-                         p.n_splits == 1 && advance ? lens : nullptr);
+                         p.n_splits == 1 && advance ? lens : nullptr, withhold);
         if (rc || p.n_splits == 1) return rc;
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr, true);
     }

@@ -39,7 +39,8 @@ __global__ void __launch_bounds__(kWideThreads, 1)
 mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ lens, float* __restrict__ o,
                        float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status, int h,
-                       int m_max, int chunk_rows, int n_splits, int len_bias, const FusedArgs fa, int32_t* __restrict__ lens_advance) {
+                       int m_max, int chunk_rows, int n_splits, int len_bias, const FusedArgs fa, int32_t* __restrict__ lens_advance,
+                       int withhold) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int seq = blockIdx.x / n_splits, split = blockIdx.x % n_splits;
 
@@ -120,7 +121,9 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     if (!ok) break;
                     mbar_expect_tx(v_full + 8 * vs, kPfTileBytes);
                     tma_load_2d_hint(v_ring + vs * kPfTileBytes, &map_v, 0, y, v_full + 8 * vs, policy);
-                    tma_load_2d_hint(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs, policy);
+                    // (for tests: one copy of the first CTA's second stage is never started, so that a wait runs out)
+                    if (!(withhold && blockIdx.x == 0 && j == 1))
+                        tma_load_2d_hint(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs, policy);
                     issued_v = j + 1;
                 }
                 if (!ok) {

@@ -28,6 +28,8 @@ def check_close(got, ref, what):
     (40, 16, 2048, False),      # persistent kernel, pieces merged through global memory
     (32, 32, 2048, True),       # persistent kernel launched as clusters, copies started on a guess
     (6, 8, 300, False),         # fixed-split kernel, one CTA per sequence
+    (20, 96, 2048, False),      # many query rows: the kernel with the query rows as tile rows, pieces and a second pass
+    (160, 40, 700, False),      # the same kernel, one split per sequence
 ])
 def test_a_wait_that_runs_out_is_reported_and_leaves_nothing_behind(b, h, m_max, chained):
     inp = wl.make_inputs(b, h, m_max, "mqa", seed=77, device=DEV)
