@@ -366,6 +366,15 @@ size_t mqa_prefill_workspace_bytes(int b, int h, int n, int m_max, int k, int v)
  */
 int mqa_set_wait_limit_cycles(long long cycles);
 
+/*
+ * mqa_set_test_withhold_copy -- for tests of the bounded waits of mqa_prefill_attention (which takes no flags): while
+ * on != 0, the kernel of the batched form never starts one on-chip copy of its first CTA's second stage, so that a
+ * wait runs out, MQA_STATUS_PIPELINE_TIMEOUT is flagged and the kernel returns by itself (O of that call is not
+ * valid).  Sets a variable on the current device, for kernels launched afterwards; synchronous, like
+ * mqa_set_wait_limit_cycles.  Off (0) by default.
+ */
+int mqa_set_test_withhold_copy(int on);
+
 /* mqa_status_string -- a static, human-readable name for a return code. */
 const char* mqa_status_string(int code);
 

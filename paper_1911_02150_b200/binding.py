@@ -25,7 +25,7 @@ EXPORTS = (
     "kv_cache_append", "mqa_decode_step", "mha_decode_step",
     "mqa_decode_step_split", "mqa_decode_step_combine",
     "mha_decode_step_split", "mha_decode_step_combine",
-    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_set_wait_limit_cycles", "mqa_prefill_attention", "mqa_prefill_workspace_bytes", "mqa_status_string", "mqa_decode_step_noalloc",
+    "mqa_workspace_bytes", "mqa_plan_splits", "mqa_plan_kernel_name", "mqa_set_wait_limit_cycles", "mqa_set_test_withhold_copy", "mqa_prefill_attention", "mqa_prefill_workspace_bytes", "mqa_status_string", "mqa_decode_step_noalloc",
     "mqa_decode_append_step", "mqa_append_step_launches",
     "mqa_layer_decode_step", "mqa_layer_workspace_bytes", "mqa_decode_local_step",
     "mqa_decode_append_step_host", "mqa_host_staging_bytes",
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.mqa_prefill_workspace_bytes.restype = sz
         L.mqa_set_wait_limit_cycles.argtypes = [ctypes.c_longlong]
         L.mqa_set_wait_limit_cycles.restype = I
+        L.mqa_set_test_withhold_copy.argtypes = [I]
+        L.mqa_set_test_withhold_copy.restype = I
         L.mqa_status_string.argtypes = [I]
         L.mqa_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -171,6 +173,11 @@ def _step_flags(advance, chained, withhold_copy=False) -> int:
     makes one bounded wait run out."""
     return ((STEP_ADVANCE if advance else 0) | (STEP_CHAINED if chained else 0) |
             (STEP_TEST_WRONG_GUESS if chained == "wrong-guess" else 0) | (STEP_TEST_WITHHOLD_COPY if withhold_copy else 0))
+
+
+def set_test_withhold_copy(on: bool) -> None:
+    """For tests: the batched form's kernel leaves one copy of its first CTA unstarted while this is on."""
+    _check(lib().mqa_set_test_withhold_copy(1 if on else 0), "mqa_set_test_withhold_copy")
 
 
 def set_wait_limit_cycles(cycles: int) -> None:

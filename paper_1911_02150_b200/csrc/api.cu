@@ -1042,6 +1042,15 @@ int mqa_prefill_attention(const void* Q, const void* K, const void* V, const int
     return launch_status();
 }
 
+int mqa_set_test_withhold_copy(int on) {
+    const int value = on ? 1 : 0;
+    if (cudaMemcpyToSymbol(g_test_withhold, &value, sizeof value) != cudaSuccess) {
+        cudaGetLastError();
+        return MQA_ERR_CUDA;
+    }
+    return MQA_OK;
+}
+
 int mqa_set_wait_limit_cycles(long long cycles) {
     const long long value = cycles > 0 ? cycles : kWaitLimitCycles;
     if (cudaMemcpyToSymbol(g_wait_limit_cycles, &value, sizeof value) != cudaSuccess) {

@@ -59,6 +59,10 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// For tests (mqa_set_test_withhold_copy): when non-zero, CTA 0 never starts one copy of the second stage of its first
+// unit, so that a bounded wait runs out.
+__device__ int g_test_withhold = 0;
+
 // One unit of work: 128 positions of a pair of heads of one sequence.  Units are numbered ((n_tiles - 1 - position tile) *
 // b + sequence) * head pairs + pair, the longest first; CTA c takes units c, c + grid, c + 2 grid, ... one after the other
 // (a persistent kernel: barriers, tensor memory and the K/V rings are set up once, and the next unit's Q and first stages
@@ -149,6 +153,7 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             bool ok = true;
             int g = 0, qi = 0;                                   // stages and units so far (they number the barriers' phases)
             int issued_k = 0, issued_v = 0, issued_q = 0;
+            const bool withhold = blockIdx.x == 0 && *reinterpret_cast<volatile int*>(&g_test_withhold) != 0;
             for (int round = 0, item; (item = pf_unit(round)) < n_items && ok; ++round) {
                 const PfItem it = pf_item(item, start, b, h, n, m_max);
                 if (it.n_kv == 0) continue;
@@ -173,7 +178,7 @@ mqa_prefill_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (!ok) break;
                     mbar_expect_tx(v_full + 8 * vs, kPfTileBytes);
                     tma_load_2d(v_ring + vs * kPfTileBytes, &map_v, 0, y, v_full + 8 * vs);
-                    tma_load_2d(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs);
+                    if (!(withhold && G == 1)) tma_load_2d(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs);
                     issued_v = G + 1;
                 }
                 g += it.n_kv;

@@ -64,3 +64,32 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_nothing_behind(b, h, m_max,
         assert np.array_equal(lens.cpu().numpy(), lens_h)
         check_close(o.cpu().numpy(), ref, f"call {rnd} after the timed-out one")
     assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)
+
+
+def test_the_batched_form_reports_a_wait_that_runs_out_and_is_correct_again_afterwards():
+    b, h, n, m_max = 3, 4, 512, 600
+    gen = torch.Generator(device=DEV).manual_seed(4)
+    Q = wl.bf16_normal((b, h, n, 128), 128 ** -0.5, gen, DEV)
+    K = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    V = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    st = np.array([88, 0, 31], np.int32)
+    start = torch.from_numpy(st).to(DEV)
+    O = torch.zeros(b, h, n, 128, dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(16, mqa.prefill_workspace_bytes(b, h, n, m_max)), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    try:
+        mqa.set_wait_limit_cycles(SHORT_LIMIT)
+        mqa.set_test_withhold_copy(True)
+        mqa.mqa_prefill_attention(Q, K, V, O, ws, start, status)
+        torch.cuda.synchronize()                     # the kernel came back by itself
+    finally:
+        mqa.set_test_withhold_copy(False)
+        mqa.set_wait_limit_cycles(0)
+    assert int(status.item()) & binding.STATUS_PIPELINE_TIMEOUT
+    status.zero_()
+    O.fill_(float("nan"))
+    mqa.mqa_prefill_attention(Q, K, V, O, ws, start, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = oracle.mqa_batched_attention(wl.bits(Q), wl.bits(K), wl.bits(V), st)
+    check_close(O.cpu().numpy(), ref, "the call after the timed-out one")
