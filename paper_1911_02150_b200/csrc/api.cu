@@ -191,7 +191,15 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
     }
     // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
-    if (b <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256) return plan_stream(b, h, m_max);
+    if (b <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256) {
+        const Plan p = plan_stream(b, h, m_max);
+        // few, long sequences, each cut into more pieces than one CTA merges inside the kernel: the streaming kernel would
+        // need its second pass as well, and the kernel with the query rows as tile rows (fixed splits, second pass) is
+        // then the quicker of the two (measured per step: 1 x 32 heads x 32768 rows 16.2 vs 18.5 us, 4 x 32 x 4096 10.5 vs
+        // 14.2, 8 x 32 x 32768 29.2 vs 30.6, 8 x 16 x 8192 16.1 vs 16.4)
+        if (!p.merge_in_kernel) return plan_wide(b, h, m_max);
+        return p;
+    }
     return h <= 32 ? plan_mma(b, h, m_max) : plan_simt(b, h, m_max);
 }
 
