@@ -674,8 +674,10 @@ def main():
         torch.cuda.empty_cache()
     if not args.no_line_sweep and world == 1:
         # the other long-context points and the ragged batch: us, GB/s, fraction of 8 TB/s, launches, both variants
-        out["sweep"] = [quick_point(mqa, variant, wl.WORKLOADS[name], device)
-                        for name in LINE_SWEEP for variant in ("mqa", "mha")]
+        # (all the multi-query points first: a point timed right after a multi-head point's gigabytes reads 10-15 % slower)
+        rows = {(name, variant): quick_point(mqa, variant, wl.WORKLOADS[name], device)
+                for variant in ("mqa", "mha") for name in LINE_SWEEP}
+        out["sweep"] = [rows[(name, variant)] for name in LINE_SWEEP for variant in ("mqa", "mha")]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, seed)
     if rank == 0:
