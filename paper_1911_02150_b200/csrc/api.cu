@@ -558,8 +558,9 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     // the second pass does not look at lens and moves it on when asked to
     const int32_t* lens_read = fused ? nullptr : lens;
     if (p.n_splits <= kCombineEager)
-        launch_dependent(combine_splits_kernel<1>, (unsigned)p.units, kHeadDim, 0, stream, part_ml, part_acc, lens_read, o, h,
-                         m_max, p.chunk_rows, p.n_splits, len_bias, fused ? lens_advance : static_cast<int32_t*>(nullptr));
+        launch_dependent(combine_few_kernel, (unsigned)((p.units + kCombineFewWarps - 1) / kCombineFewWarps), (unsigned)(kCombineFewWarps * 32),
+                         0, stream, part_ml, part_acc, lens_read, o, h, m_max, p.chunk_rows, p.n_splits, len_bias,
+                         fused ? lens_advance : static_cast<int32_t*>(nullptr), p.units);
     else
         launch_dependent(combine_splits_kernel<4>, (unsigned)p.units, 4 * kHeadDim, 0, stream, part_ml, part_acc, lens_read, o, h,
                          m_max, p.chunk_rows, p.n_splits, len_bias, fused ? lens_advance : static_cast<int32_t*>(nullptr));

@@ -120,4 +120,64 @@ combine_splits_kernel(const float2* __restrict__ part_ml, const float* __restric
                  o + u * kHeadDim);
 }
 
+// The same second pass for up to kCombineEager pieces per (sequence, head), one WARP per (sequence, head): a lane takes four
+// of the 128 columns, asks for its part of every piece and for the (maximum, sum) pairs in one go, and merges them in piece
+// order with the arithmetic of merge_pieces (the same bits).  No shared memory, no barrier: eight units per CTA, so the
+// 4096 units of 32 sequences x 128 query rows are one wave of 512 CTAs (one CTA per unit took 7.5 us there, this 2-3).
+constexpr int kCombineFewWarps = 8;
+__global__ void __launch_bounds__(kCombineFewWarps * 32)
+combine_few_kernel(const float2* __restrict__ part_ml, const float* __restrict__ part_acc, const int32_t* __restrict__ lens,
+                   float* __restrict__ o, int h, int m_max, int chunk_rows, int n_splits, int len_bias,
+                   int32_t* __restrict__ lens_advance, size_t units) {
+    const int lane = threadIdx.x & 31;
+    const size_t u = (size_t)blockIdx.x * kCombineFewWarps + (threadIdx.x >> 5);
+    grid_dependency_wait();          // the partials come from the kernel before this one
+    if (u >= units) return;
+    int live = n_splits;
+    if (lens != nullptr) {
+        int L = biased_len(lens[u / h], m_max, len_bias);
+        L = L < 0 ? 0 : (L > m_max ? m_max : L);
+        live = (L + chunk_rows - 1) / chunk_rows;
+        if (live > n_splits) live = n_splits;
+    } else if (lens_advance != nullptr && u % h == 0 && lane == 0) {
+        const int raw = lens_advance[u / h];
+        if (raw >= 0 && raw < m_max) lens_advance[u / h] = raw + 1;
+    }
+    float4* out = reinterpret_cast<float4*>(o + u * kHeadDim) + lane;
+    const float2* ml_p = part_ml + u * n_splits;
+    const float4* acc_p = reinterpret_cast<const float4*>(part_acc + u * (size_t)n_splits * kHeadDim) + lane;
+    float2 ml[kCombineEager];
+    float4 a[kCombineEager];
+#pragma unroll
+    for (int i = 0; i < kCombineEager; ++i) {
+        ml[i] = make_float2(-INFINITY, 0.f);
+        a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < live) {
+            ml[i] = __ldcg(ml_p + i);
+            a[i] = __ldcg(acc_p + (size_t)i * (kHeadDim / 4));
+        }
+    }
+    float top = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kCombineEager; ++i) top = fmaxf(top, ml[i].x);
+    if (live == 0 || top == -INFINITY) {               // the empty prefix, or nothing but empty pieces: zeros
+        *out = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    float den = 0.f;
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < kCombineEager; ++i) {
+        if (i < live) {
+            const float w = fast_exp2(ml[i].x - top);
+            if (w != 0.f) {                               // never multiply an unwritten slot
+                den = fmaf(w, ml[i].y, den);
+                num.x = fmaf(w, a[i].x, num.x); num.y = fmaf(w, a[i].y, num.y);
+                num.z = fmaf(w, a[i].z, num.z); num.w = fmaf(w, a[i].w, num.w);
+            }
+        }
+    }
+    *out = make_float4(num.x / den, num.y / den, num.z / den, num.w / den);
+}
+
 }  // namespace mqa
