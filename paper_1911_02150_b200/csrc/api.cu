@@ -155,7 +155,8 @@ Plan plan_wide(int b, int h, int m_max) {
     p.units = (size_t)b * h;
     p.b = b; p.h = h;
     p.kernel = Kernel::kWide;
-    int want = sm_count() / b;
+    const int tiles = (h + kWideRows - 1) / kWideRows;           // row tiles of 128 query rows (grid.y)
+    int want = sm_count() / (b * tiles);
     const int cap = m_max / (2 * kWideRows);
     if (want > cap) want = cap;
     if (want > 160) want = 160;                    // (the second pass merges up to 160 pieces in one go)
@@ -173,7 +174,9 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // 33 .. 128 query rows per sequence: the kernel with the query rows as tile rows (measured against the streaming
     // kernel's 64-row tile, per step: 32 x 64 rows x 8192: 30.5 vs 35.0 us; 128 x 64 x 2048: 26.2 vs 32.8; 4 x 48 x 4096:
     // 10.8 vs 20.7; and against groups of 64 at 128 rows, 32 x 8192: 34.9 vs 68.8 us)
-    if (h > 32 && h <= kWideRows && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
+    // (and beyond 128 rows as row tiles of 128 over the same cache rows: 32 x 256 rows x 8192: 43.6 us, against 122.7 us as
+    // four groups of 64 rows on the streaming kernel; 128 x 160 x 2048: 50.1 vs 103.2)
+    if (h > 32 && (h + kWideRows - 1) / kWideRows <= 65535 && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
     if (h > kGroupRows) {
         // more query rows than one tile of the tensor-core kernel holds (beams x heads, many heads): groups of 64
         // rows, each a sequence of the persistent kernel's schedule over the same cache
@@ -265,6 +268,22 @@ cudaError_t launch_dependent_clusters(unsigned cluster, void (*kernel)(Params...
         attr[1].val.clusterDim.x = cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
         cfg.numAttrs = 2;
     }
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
+template <typename... Params, typename... Args>
+cudaError_t launch_dependent_2d(void (*kernel)(Params...), unsigned grid_x, unsigned grid_y, unsigned block, size_t smem,
+                                cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid_x, grid_y);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
 }
 
@@ -490,7 +509,8 @@ int launch_wide(const Plan& p, const void* q, const void* K, const void* V, cons
     if (!encode_cache_map(&map_q, q, (long long)b * h, kWideRows) || !encode_cache_map(&map_k, K, (long long)b * m_max, kWideRows) ||
         !encode_cache_map(&map_v, V, (long long)b * m_max, kWideRows))
         return MQA_ERR_CUDA;
-    launch_dependent(mqa_decode_wide_kernel, (unsigned)((size_t)b * p.n_splits), (unsigned)kWideThreads, (size_t)kWideSmemBytes, stream, map_q,
+    launch_dependent_2d(mqa_decode_wide_kernel, (unsigned)((size_t)b * p.n_splits), (unsigned)((h + kWideRows - 1) / kWideRows),
+                        (unsigned)kWideThreads, (size_t)kWideSmemBytes, stream, map_q,
                      map_k, map_v, lens, o, part_ml, part_acc, status, h, m_max, p.chunk_rows, p.n_splits, len_bias, fa, lens_advance,
                      withhold ? 1 : 0);
     return launch_status();
@@ -813,9 +833,15 @@ static int append_step_impl(const void* q, void* K, void* V, const void* k_new, 
         // otherwise the second pass does.  One or two launches.
         float2* part_ml = partials_ml(workspace);
         float* part_acc = partials_acc(p, workspace);
+        // (one split and one tile of 128 rows: the CTA moves lens on itself)
+        const bool alone = p.n_splits == 1 && h <= kWideRows;
         rc = launch_wide(p, q, K, V, lens, o, part_ml, part_acc, status, b, h, m_max, stream, 0, k_new, v_new,
-                         p.n_splits == 1 && advance ? lens : nullptr, withhold);
-        if (rc || p.n_splits == 1) return rc;
+                         alone && advance ? lens : nullptr, withhold);
+        if (rc || alone) return rc;
+        if (p.n_splits == 1) {                                   // several row tiles read lens: moved on by a kernel of its own
+            if (advance) launch_dependent(lens_advance_kernel, (unsigned)((b + 255) / 256), 256u, 0, stream, lens, b, m_max);
+            return launch_status();
+        }
         return run_combine(true, lens, o, workspace, workspace_bytes, b, h, m_max, k, v, stream, 0, advance ? lens : nullptr, true);
     }
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits > 1) {
@@ -993,7 +1019,7 @@ int mqa_append_step_launches(int b, int h, int m_max, int k, int v) {
     if ((p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) && p.n_splits == 1) return 1;   // one CTA per sequence does it all
     if (p.stream()) return 2;                          // pass with the append inside, second pass
     if (p.kernel == Kernel::kMma1 || p.kernel == Kernel::kMma2) return 2;   // fixed splits: the same two
-    if (p.kernel == Kernel::kWide) return p.n_splits == 1 ? 1 : 2;
+    if (p.kernel == Kernel::kWide) return p.n_splits == 1 && h <= kWideRows ? 1 : 2;
     return 2 + (p.n_splits > 1 ? 1 : 0) + 1;           // append, pass, (second pass), lens advance
 }
 

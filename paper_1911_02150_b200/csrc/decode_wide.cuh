@@ -1,5 +1,5 @@
-// Multi-query decoding step for MANY query rows per sequence (33 .. 128: many heads, or beams x heads over one shared
-// memory, Section 4.2) -- the same three lines of Section 3 (logits = einsum(bhk,bmk->bhm), softmax over the valid
+// Multi-query decoding step for MANY query rows per sequence (33 and more: many heads, or beams x heads over one shared
+// memory, Section 4.2; 128 rows per CTA, more as grid.y row tiles over the same cache rows) -- the same three lines of Section 3 (logits = einsum(bhk,bmk->bhm), softmax over the valid
 // prefix, o = einsum(bhm,bmv->bhv)), with the query rows as the ROWS of the tensor-core tiles.
 //
 // The streaming kernel (decode_umma.cuh) puts the cache rows on the TMEM lanes and the heads on the columns, which is
@@ -34,7 +34,7 @@ constexpr int kWideBarriers = 1 + 2 * kWideKSlots + 2 * kWideVSlots + 6;
 constexpr int kWideSmemBytes = (1 + kWideKSlots + kWideVSlots) * kPfTileBytes + kWideBarriers * 8 + 16 + 1024 /* alignment slack */;
 static_assert(kWideSmemBytes + 1024 + 16 /* static */ <= 227 * 1024, "exceeds the shared memory of one SM");
 
-// grid: x = sequence * n_splits + split.  part_ml [b * h][n_splits], part_acc [b * h][n_splits][128] (combine.cuh).
+// grid: x = sequence * n_splits + split, y = tile of 128 query rows.  part_ml [b * h][n_splits], part_acc [b * h][n_splits][128] (combine.cuh).
 __global__ void __launch_bounds__(kWideThreads, 1)
 mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ lens, float* __restrict__ o,
@@ -43,6 +43,7 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                        int withhold) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int seq = blockIdx.x / n_splits, split = blockIdx.x % n_splits;
+    const int row0 = blockIdx.y * kWideRows;                   // this CTA's first query row of the sequence (more than 128: grid.y tiles)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);     // the 128-byte swizzle repeats every 1 KiB
@@ -83,9 +84,9 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     // second-pass kernel.
     const int raw = __ldcg(lens + seq);
     const bool appended = fa.k_new != nullptr && raw >= 0 && raw < m_max;
-    if (fa.k_new != nullptr && !appended && split == 0 && threadIdx.x == 0 && status)
+    if (fa.k_new != nullptr && !appended && split == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status)
         atomicOr(status, raw < 0 ? kStatusAppendNegative : kStatusAppendFull);
-    const int L = clamp_len(appended ? raw + 1 : biased_len(raw, m_max, len_bias), m_max, (split == 0 && threadIdx.x == 0) ? status : nullptr);
+    const int L = clamp_len(appended ? raw + 1 : biased_len(raw, m_max, len_bias), m_max, (split == 0 && blockIdx.y == 0 && threadIdx.x == 0) ? status : nullptr);
     const int r0 = split * chunk_rows, r1 = min(r0 + chunk_rows, L);           // this CTA's rows of the sequence's cache
     const int n_kv = r1 > r0 ? (r1 - r0 + kWideRows - 1) / kWideRows : 0;      // stages
     const bool hilo = L < kSingleRoundingMinRows;
@@ -105,7 +106,7 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 bool ok = true;
                 mbar_expect_tx(q_full, kPfTileBytes);
                 for (int half = 0; half < 2; ++half)
-                    tma_load_2d(q_s + half * kPfHalfBytes, &map_q, half * kBoxCols, seq * h, q_full);
+                    tma_load_2d(q_s + half * kPfHalfBytes, &map_q, half * kBoxCols, seq * h + row0, q_full);
                 const uint64_t policy = l2_stream_policy(true);     // the cache is read once per step
                 int issued_k = 0, issued_v = 0;
                 for (int j = 0; j < n_kv && ok; ++j) {
@@ -122,7 +123,7 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     mbar_expect_tx(v_full + 8 * vs, kPfTileBytes);
                     tma_load_2d_hint(v_ring + vs * kPfTileBytes, &map_v, 0, y, v_full + 8 * vs, policy);
                     // (for tests: one copy of the first CTA's second stage is never started, so that a wait runs out)
-                    if (!(withhold && blockIdx.x == 0 && j == 1))
+                    if (!(withhold && blockIdx.x == 0 && blockIdx.y == 0 && j == 1))
                         tma_load_2d_hint(v_ring + vs * kPfTileBytes + kPfHalfBytes, &map_v, kBoxCols, y, v_full + 8 * vs, policy);
                     issued_v = j + 1;
                 }
@@ -317,8 +318,8 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             named_barrier(1, 256);
             // (the loads from tensor memory below are warp-wide instructions: every lane executes them, whether or not
             // its row is one of the sequence's h query rows)
-            const bool stored = r < h;
-            const size_t unit = (size_t)seq * h + (stored ? r : 0);
+            const bool stored = row0 + r < h;
+            const size_t unit = (size_t)seq * h + (stored ? row0 + r : 0);
             if (n_kv == 0) {
                 // nothing of this split lies inside the prefix: zeros (one split, written below) or an empty piece
                 if (stored && n_splits > 1) part_ml[unit * n_splits + split] = make_float2(-INFINITY, 0.f);
@@ -361,10 +362,10 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         if (n_kv > 0 || n_splits == 1) {
             for (int item = threadIdx.x; item < kWideRows * 32; item += 256) {
                 const int row = item >> 5, c16 = item & 31;                             // (a warp: one row, its 32 pieces of 16 bytes)
-                if (row >= h) break;
+                if (row0 + row >= h) break;
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (n_kv > 0) v = reinterpret_cast<const float4*>(base + kPfTileBytes + row * 512)[c16 ^ (row & 31)];
-                const size_t unit = (size_t)seq * h + row;
+                const size_t unit = (size_t)seq * h + row0 + row;
                 float* dst = n_splits == 1 ? o + unit * kHeadDim : part_acc + (unit * n_splits + split) * kHeadDim;
                 reinterpret_cast<float4*>(dst)[c16] = v;
             }
@@ -378,7 +379,9 @@ mqa_decode_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         tmem_dealloc(tmem_base, 512);
     }
     if (threadIdx.x == 0 && timed_out && status) atomicOr(status, kStatusPipelineTimeout);
-    if (lens_advance && appended && n_splits == 1 && threadIdx.x == 0) lens_advance[seq] = raw + 1;   // (nobody else reads this sequence's length)
+    // (one split: lens is this CTA's to move on -- with several row tiles, the sequence's other CTAs read it too, so then the
+    // host leaves it to a kernel of its own)
+    if (lens_advance && appended && n_splits == 1 && threadIdx.x == 0) lens_advance[seq] = raw + 1;
 }
 
 }  // namespace mqa

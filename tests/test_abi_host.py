@@ -112,13 +112,13 @@ def test_plans_of_many_query_rows_and_of_the_batched_form(L):
     """More than 64 query rows per sequence are planned as groups of 64 on the tensor-core kernel, and the batched
     form's workspace and refusals are answered on the host (the plan assumes the 148 SMs of a B200 without a GPU)."""
     assert binding.plan_kernel_name(True, False, 32, 128, 8192) == "mqa_decode_wide_kernel"       # 65 .. 128 rows: rows as tile rows
-    assert binding.plan_kernel_name(True, False, 32, 192, 8192) == "mqa_decode_stream_umma_kernel<64>"   # beyond: groups of 64
+    assert binding.plan_kernel_name(True, False, 32, 192, 8192) == "mqa_decode_wide_kernel"       # beyond: tiles of 128 rows
     assert binding.plan_kernel_name(True, True, 32, 32, 8192) == "mqa_decode_stream_umma_kernel<32, fused, guess>"
     assert binding.plan_kernel_name(False, False, 32, 32, 8192) == "decode_split_simt_kernel"
     assert binding.plan_kernel_name(True, False, 0, 32, 8192) == ""
     assert binding.append_step_launches(32, 128, 8192) == 2
     assert binding.append_step_launches(256, 128, 8192) == 1
-    assert binding.append_step_launches(32, 192, 8192) == 1
+    assert binding.append_step_launches(32, 192, 8192) == 2
     assert binding.workspace_bytes(32, 128, 8192) >= binding.workspace_bytes(32, 64, 8192)
     need = binding.prefill_workspace_bytes(2, 8, 128, 256)
     assert need > 0

@@ -74,8 +74,9 @@ CASES = [
     # ... 33 .. 128 query rows per sequence: the kernel with the query rows as tile rows (fixed splits; the CTA whose rows
     # hold the new one stores it; one split per sequence moves lens on itself, else the second pass does) ...
     (40, 48, 1500), (33, 64, 2100), (24, 128, 2048), (20, 96, 1500), (150, 33, 700), (1, 127, 20000), (5, 65, 129),
-    # ... more query rows than that: groups of 64 rows over the same cache, each storing the new row ...
-    (6, 200, 3000),
+    # ... more query rows than that: row tiles of 128 over the same cache rows, each CTA of the row's split storing the
+    # new row; with one split per sequence lens is moved on by a kernel of its own ...
+    (6, 200, 3000), (80, 160, 600), (2, 129, 5000), (3, 300, 1500),
     # ... and plans that run as separate launches (small batches)
     (4, 8, 300), (1, 16, 20000), (2, 40, 600),
 ]

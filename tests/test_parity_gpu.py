@@ -146,8 +146,10 @@ STREAM = [
     (150, 33, 700, 40),     # more sequences than SMs: one split each, short caches (two roundings of the weights)
     (1, 127, 20000, 41),    # one sequence in many splits
     (7, 100, 127, 42),      # less than one stage
-    # more than 128: groups of 64 rows on the streaming kernel
-    (3, 200, 9000, 36),     # few long sequences, four groups (the last of 8 rows): second-pass kernel
+    # more than 128: row tiles of 128 on the same kernel
+    (3, 200, 9000, 36),     # few long sequences, two tiles (the second of 72 rows)
+    (80, 160, 600, 43),     # one split per sequence, two tiles
+    (4, 385, 2100, 44),     # four tiles, the last of one row
     # batches that divide the grid are launched as clusters (16 and 8 CTAs here); with mixed lengths the clusters
     # change nothing and one CTA merges a sequence's many pieces
     (8, 16, 20000, 38),
