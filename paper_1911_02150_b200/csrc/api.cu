@@ -57,9 +57,6 @@ struct Plan {
     int grid = 0;         // persistent kernel: number of CTAs
     Kernel kernel = Kernel::kSimt;
     bool merge_in_kernel = false;   // tcgen05 plan: pieces merged by the CTA that delivers a sequence's last one (single launch)
-    int groups = 1;       // tcgen05 plan for more than 64 query rows per sequence: groups of 64 rows, each a sequence of the
-                          // schedule over the same cache (then b = sequences x groups and h = 64: see QueryGroups)
-    int h_total = 0;      // query rows per sequence as the caller counts them
     bool stream() const { return kernel == Kernel::kUmma; }
 };
 
@@ -177,21 +174,6 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // (and beyond 128 rows as row tiles of 128 over the same cache rows: 32 x 256 rows x 8192: 43.6 us, against 122.7 us as
     // four groups of 64 rows on the streaming kernel; 128 x 160 x 2048: 50.1 vs 103.2)
     if (h > 32 && (h + kWideRows - 1) / kWideRows <= 65535 && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
-    if (h > kGroupRows) {
-        // more query rows than one tile of the tensor-core kernel holds (beams x heads, many heads): groups of 64
-        // rows, each a sequence of the persistent kernel's schedule over the same cache
-        const int groups = (h + kGroupRows - 1) / kGroupRows;
-        const long long seqs = (long long)b * groups;
-        const long long tiles = seqs * ((m_max + kTileRows - 1) / kTileRows);
-        if (seqs <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256 &&
-            (long long)b * h < 0x7fffffffLL) {
-            Plan p = plan_stream((int)seqs, kGroupRows, m_max);
-            p.groups = groups;
-            p.h_total = h;
-            return p;
-        }
-        return plan_simt(b, h, m_max);
-    }
     // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     if (b <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256) {
@@ -413,18 +395,16 @@ constexpr size_t kL2KeepBytes = 64u << 20;   // K and V together: half of the 12
 constexpr int kEarlyTestWithhold = 1 << 8;    // rides on `early`: MQA_STEP_TEST_WITHHOLD_COPY
 std::atomic<int> g_umma_opt_in[kMaxDevices][13];
 
-// b, h: the caller's sequences and query rows per sequence (the kernel is given the plan's: sequences x groups, 64 rows
-// each, where the plan has groups).
-template <int HP, bool FUSED, bool GUESS = false, int GROUPED = 0>
+// The streaming kernel serves up to 32 query rows per sequence (HP = 16 or 32); more go to decode_wide.cuh.
+template <int HP, bool FUSED, bool GUESS = false>
 int launch_umma(const Plan& p, const void* q, const void* K, const void* V, const int32_t* lens, float* o,
                 void* workspace, int32_t* status, int b, int h, int m_max, cudaStream_t stream, bool merge,
                 const void* k_new = nullptr, const void* v_new = nullptr, int32_t* lens_advance = nullptr,
                 int early = 0) {
     using Cfg = UmmaCfg<HP>;
-    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS, GROUPED>;
-    static_assert(GROUPED == 0 || HP == 64, "groups hold 64 query rows");
-    constexpr int kSlot = GROUPED == 1 ? 10 + (GUESS ? 2 : FUSED ? 1 : 0) : (HP == 16 ? 0 : (HP == 32 ? 1 : 2)) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
-    const QueryGroups grp = {p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0};
+    auto kernel = mqa_decode_stream_umma_kernel<HP, FUSED, GUESS>;
+    static_assert(HP == 16 || HP == 32, "padded head count");
+    constexpr int kSlot = (HP == 16 ? 0 : 1) * 3 + (GUESS ? 2 : FUSED ? 1 : 0);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return MQA_ERR_CUDA; }
     if (!g_umma_opt_in[dev][kSlot].load(std::memory_order_acquire)) {
@@ -443,7 +423,7 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
         fa.V = static_cast<uint4*>(const_cast<void*>(V));
     }
     alignas(64) CUtensorMap map_k, map_v, map_k_sub, map_v_sub, map_q;
-    const long long rows = (long long)b * m_max;             // (b caches, however many schedule sequences look at each)
+    const long long rows = (long long)b * m_max;
     if (!encode_cache_map(&map_k, K, rows, kUmmaStageRows) || !encode_cache_map(&map_v, V, rows, kUmmaStageRows) ||
         !encode_cache_map(&map_k_sub, K, rows) || !encode_cache_map(&map_v_sub, V, rows) ||
         !encode_cache_map(&map_q, q, (long long)b * h, HP))
@@ -458,7 +438,7 @@ int launch_umma(const Plan& p, const void* q, const void* K, const void* V, cons
     if (merge && p.grid % p.b == 0 && p.grid / p.b >= 2 && p.grid / p.b <= kMaxClusterCtas) cluster = (unsigned)(p.grid / p.b);
     launch_dependent_clusters(cluster, kernel, (unsigned)p.grid, kUmmaThreads, Cfg::kSmemBytes, stream, map_k, map_v, map_k_sub,
                               map_v_sub, map_q, lens, o, w.span, w.ml, w.acc, status, p.b, p.h, m_max, share_magic(p.grid), fa,
-                              merge ? w.ctrl : nullptr, lens_advance, early, read_once, grp);
+                              merge ? w.ctrl : nullptr, lens_advance, early, read_once);
     return cudaGetLastError() == cudaSuccess ? MQA_OK : MQA_ERR_CUDA;
 }
 
@@ -470,16 +450,12 @@ int launch_umma_for(const Plan& p, const void* q, const void* K, const void* V, 
 #define MQA_UMMA_ARGS p, q, K, V, lens, o, workspace, status, b, h, m_max, stream, merge, k_new, v_new, lens_advance, early
     if constexpr (FUSED) {
         if ((early & ~kEarlyTestWithhold) >= 2) {           // the kernels that carry the code for copies started on a guess
-            if (p.groups > 1) return launch_umma<64, true, true, 1>(MQA_UMMA_ARGS);
             if (p.h <= 16) return launch_umma<16, true, true>(MQA_UMMA_ARGS);
-            if (p.h <= 32) return launch_umma<32, true, true>(MQA_UMMA_ARGS);
-            return launch_umma<64, true, true>(MQA_UMMA_ARGS);
+            return launch_umma<32, true, true>(MQA_UMMA_ARGS);
         }
     }
-    if (p.groups > 1) return launch_umma<64, FUSED, false, 1>(MQA_UMMA_ARGS);
     if (p.h <= 16) return launch_umma<16, FUSED>(MQA_UMMA_ARGS);
-    if (p.h <= 32) return launch_umma<32, FUSED>(MQA_UMMA_ARGS);
-    return launch_umma<64, FUSED>(MQA_UMMA_ARGS);
+    return launch_umma<32, FUSED>(MQA_UMMA_ARGS);
 #undef MQA_UMMA_ARGS
 }
 
@@ -542,19 +518,18 @@ int run_split(bool multi_query, const void* q, const void* K, const void* V, con
 }
 
 // Second pass of the persistent kernel: one CTA per (schedule sequence, query row) merges the sequence's pieces.
-int launch_stream_combine(const Plan& p, const void* workspace, float* o, int32_t* lens_advance, int m_max, cudaStream_t stream,
-                          const QueryGroups& grp) {
+int launch_stream_combine(const Plan& p, const void* workspace, float* o, int32_t* lens_advance, int m_max, cudaStream_t stream) {
     const StreamWorkspace w = stream_workspace(p, workspace);
     const unsigned grid = (unsigned)((size_t)p.b * p.h);
     if (p.n_splits <= kCombineEager)
         launch_dependent(stream_combine_kernel<1>, grid, kHeadDim, 0, stream, w.span, w.ml, w.acc, o, p.b, p.h, lens_advance,
-                         m_max, share_magic(p.grid), grp);
+                         m_max, share_magic(p.grid));
     else if (p.n_splits <= 4 * kCombineEager)
         launch_dependent(stream_combine_kernel<4>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o, p.b, p.h,
-                         lens_advance, m_max, share_magic(p.grid), grp);
+                         lens_advance, m_max, share_magic(p.grid));
     else
         launch_dependent(stream_combine_kernel<kCombineManyGroups>, grid, 4 * kHeadDim, 0, stream, w.span, w.ml, w.acc, o,
-                         p.b, p.h, lens_advance, m_max, share_magic(p.grid), grp);
+                         p.b, p.h, lens_advance, m_max, share_magic(p.grid));
     return launch_status();
 }
 
@@ -568,8 +543,7 @@ int run_combine(bool multi_query, const int32_t* lens, float* o, const void* wor
     int rc = check_workspace(p, workspace, workspace_bytes);
     if (rc) return rc;
     if (p.stream()) {
-        const QueryGroups grp = {p.groups > 1 ? p.groups : 0, p.groups > 1 ? p.h_total : 0, 0};
-        return launch_stream_combine(p, workspace, o, lens_advance, m_max, stream, grp);
+        return launch_stream_combine(p, workspace, o, lens_advance, m_max, stream);
     }
     if (p.n_splits <= 1) return MQA_OK;
     const float2* part_ml = partials_ml(workspace);
@@ -1102,8 +1076,7 @@ const char* mqa_plan_kernel_name(int multi_query, int whole_step, int b, int h, 
         case Kernel::kUmma: {
             const bool guess = whole_step && p.merge_in_kernel && p.n_splits <= kGuessMaxPieces && p.chunk_rows >= kGuessMinShareRows;
             if (h <= 16) return !whole_step ? "mqa_decode_stream_umma_kernel<16>" : guess ? "mqa_decode_stream_umma_kernel<16, fused, guess>" : "mqa_decode_stream_umma_kernel<16, fused>";
-            if (h <= 32) return !whole_step ? "mqa_decode_stream_umma_kernel<32>" : guess ? "mqa_decode_stream_umma_kernel<32, fused, guess>" : "mqa_decode_stream_umma_kernel<32, fused>";
-            return !whole_step ? "mqa_decode_stream_umma_kernel<64>" : guess ? "mqa_decode_stream_umma_kernel<64, fused, guess>" : "mqa_decode_stream_umma_kernel<64, fused>";
+            return !whole_step ? "mqa_decode_stream_umma_kernel<32>" : guess ? "mqa_decode_stream_umma_kernel<32, fused, guess>" : "mqa_decode_stream_umma_kernel<32, fused>";
         }
         case Kernel::kMma1: return "mqa_decode_split_mma_kernel<1>";
         case Kernel::kMma2: return "mqa_decode_split_mma_kernel<2>";

@@ -663,36 +663,10 @@ __host__ __device__ inline size_t stream_ml_bytes(int slots, int h) {
 }
 __host__ __device__ inline size_t stream_acc_bytes(int slots, int h) { return (size_t)slots * h * kHeadDim * sizeof(float); }
 
-// Several sequences of the schedule may stand for ONE cache, kGroupRows query rows each: a sequence with more than
-// 64 query rows (more heads than that, or beams x heads, all over one shared memory) is cut into groups of 64 rows,
-// each a schedule sequence of its own over the same cache rows.
-// Schedule sequence s of a launch is number sg = first + s of all of them; its cache is kv = sg / per_kv; its
-// query (and output) rows are rows kv * rows_per_kv + (sg % per_kv) * 64 .. of the [rows, 128] q (o) matrix.
-constexpr int kGroupRows = 64;
-struct QueryGroups {
-    int per_kv;         // schedule sequences per cache (0: the plain step, one sequence per cache, no other field used)
-    int rows_per_kv;    // query rows per cache
-    int first;          // number of this launch's first schedule sequence (a launch holds at most kStreamMaxSeqs)
-};
-__device__ __forceinline__ int group_kv(const QueryGroups& g, int s) { return g.per_kv == 0 ? s : (g.first + s) / g.per_kv; }
-// first query row of schedule sequence s (h: query rows per sequence of the plain step)
-__device__ __forceinline__ long long group_row0(const QueryGroups& g, int s, int h) {
-    if (g.per_kv == 0) return (long long)s * h;
-    const int sg = g.first + s;
-    return (long long)(sg / g.per_kv) * g.rows_per_kv + (long long)(sg % g.per_kv) * kGroupRows;
-}
-__device__ __forceinline__ int group_rows(const QueryGroups& g, int s, int h) {
-    if (g.per_kv == 0) return h;
-    const int left = g.rows_per_kv - ((g.first + s) % g.per_kv) * kGroupRows;
-    return left < kGroupRows ? left : kGroupRows;
-}
-
-// Rows of its cache that schedule sequence s may look at, as lens says (read from L2: the kernels before and
-// after this one may write lens).
+// Rows of its cache that sequence s may look at, as lens says (read from L2: the kernels before and after this one may
+// write lens).
 template <bool FUSED>
-__device__ __forceinline__ int read_len(const int32_t* lens, int s, const QueryGroups& g) {
-    return __ldcg(lens + group_kv(g, s));
-}
+__device__ __forceinline__ int read_len(const int32_t* lens, int s) { return __ldcg(lens + s); }
 
 // Rows of sequence s this launch attends over, and whether the step appends to it.
 __device__ __forceinline__ int fused_rows(int raw, int m_max, bool appending, bool* can_append) {
@@ -721,7 +695,7 @@ template <bool FUSED, int THREADS, int PENALTY>
 __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ lens, float* __restrict__ o,
                                                  int32_t* __restrict__ status, int b, int h, int m_max, bool appending,
                                                  unsigned long long magic, int* prefix, int* rows_of, int* plan_sm,
-                                                 int solo_warp = -1, const QueryGroups grp = QueryGroups{0, 0, 0}) {
+                                                 int solo_warp = -1) {
     const int cta = blockIdx.x, G = gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int planners = solo_warp >= 0 ? THREADS - 32 : THREADS;
@@ -730,7 +704,7 @@ __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ len
         named_barrier(kPlanBarDone, THREADS);
     } else {
     for (int s = tix; s < b; s += planners) {
-        const int raw = read_len<FUSED>(lens, s, grp);
+        const int raw = read_len<FUSED>(lens, s);
         clamp_len(raw, m_max, cta == 0 ? status : nullptr);
         bool can_append;
         const int L = fused_rows(raw, m_max, appending, &can_append);
@@ -743,8 +717,8 @@ __device__ __forceinline__ SharePlan stream_plan(const int32_t* __restrict__ len
     if (solo_warp >= 0) named_barrier(kPlanBarInit, THREADS); else __syncthreads();
     for (int s = cta; s < b; s += G) {                     // the empty prefix gives zeros: all threads, 16 bytes each
         if ((rows_of[s] & (kAppendBit - 1)) != 0) continue;
-        float4* dst = reinterpret_cast<float4*>(o + (size_t)group_row0(grp, s, h) * kHeadDim);
-        for (int i = tix; i < group_rows(grp, s, h) * (kHeadDim / 4); i += planners) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4* dst = reinterpret_cast<float4*>(o + (size_t)s * h * kHeadDim);
+        for (int i = tix; i < h * (kHeadDim / 4); i += planners) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (warp == 0) {
         // inclusive scan of prefix[1..b] by one warp; the lane whose chunk holds this CTA's first position
@@ -800,8 +774,7 @@ constexpr int kFastSeqs = 256;
 template <bool FUSED, int PENALTY>
 __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, int b, int m_max, bool appending,
                                               unsigned long long magic, Segment* g, int* rows, int cluster = 1, int rank = 0,
-                                              int stage_tiles = 4, bool* strided = nullptr,
-                                              const QueryGroups grp = QueryGroups{0, 0, 0}) {
+                                              int stage_tiles = 4, bool* strided = nullptr) {
     if (strided) *strided = false;
     if (b > kFastSeqs) return false;
     const int cta = blockIdx.x, lane = threadIdx.x & 31;
@@ -813,7 +786,7 @@ __device__ __forceinline__ bool first_segment(const int32_t* __restrict__ lens, 
         tl[i] = 0; rw[i] = 0;
         if (i < per && base + i < b) {
             bool can_append;
-            const int L = fused_rows(read_len<FUSED>(lens, base + i, grp), m_max, appending, &can_append);
+            const int L = fused_rows(read_len<FUSED>(lens, base + i), m_max, appending, &can_append);
             tl[i] = L > 0 ? (L + kTileRows - 1) / kTileRows + PENALTY : 0;
             rw[i] = L | (appending && can_append ? kAppendBit : 0);
         }
@@ -882,16 +855,14 @@ template <int GROUPS>
 __global__ void __launch_bounds__(kHeadDim * (GROUPS >= 4 ? 4 : 1))
 stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restrict__ part_ml,
                       const float* __restrict__ part_acc, float* __restrict__ o, int b, int h,
-                      int32_t* lens_advance, int m_max, unsigned long long magic, const QueryGroups grp) {
+                      int32_t* lens_advance, int m_max, unsigned long long magic) {
     const int s = blockIdx.x / h, head = blockIdx.x % h;
     grid_dependency_wait();          // the slots come from the kernel before this one
-    // append-and-attend step: lens += 1 for a sequence that took a row (once per cache: by its first group)
-    if (lens_advance && head == 0 && threadIdx.x == 0 && (grp.per_kv == 0 || (grp.first + s) % grp.per_kv == 0)) {
-        const int kv = group_kv(grp, s);
-        const int raw = lens_advance[kv];
-        if (raw >= 0 && raw < m_max) lens_advance[kv] = raw + 1;
+    // append-and-attend step: lens += 1 for a sequence that took a row
+    if (lens_advance && head == 0 && threadIdx.x == 0) {
+        const int raw = lens_advance[s];
+        if (raw >= 0 && raw < m_max) lens_advance[s] = raw + 1;
     }
-    if (head >= group_rows(grp, s, h)) return;             // (a last group of fewer than 64 rows)
     const int2 span = seq_span[s];
     if (span.y <= span.x) return;
     const int T = seq_span[b].x;                        // length of the line (magic: the first pass's grid size, see share_begin)
@@ -905,7 +876,7 @@ stream_combine_kernel(const int2* __restrict__ seq_span, const float2* __restric
             return live ? __ldcg(part_ml + ((size_t)cta + s) * h + head) : make_float2(-INFINITY, 0.f);
         },
         [&](int i) { return part_acc + (((size_t)span.x + i + s) * h + head) * kHeadDim; },
-        o + ((size_t)group_row0(grp, s, h) + head) * kHeadDim);
+        o + ((size_t)s * h + head) * kHeadDim);
 }
 
 }  // namespace mqa

@@ -10,7 +10,7 @@
 //                                                                          B = P^T, written by the softmax warps
 //
 // so K and V are read from shared memory by the tensor core itself, once for all heads; the work
-// per stage grows with the padded head count HP (16, 32 or 64) and nothing is replicated.  In TMEM
+// per stage grows with the padded head count HP (16 or 32; more query rows per sequence run on decode_wide.cuh) and nothing is replicated.  In TMEM
 // a cache row of S^T is a lane, so a softmax thread owns one cache row of the stage (two threads
 // share a row's heads): masking by index is a per-thread decision and the weights need no exchange
 // between threads.  The reference maximum of a head is shared by all rows and moves only when some
@@ -53,7 +53,7 @@ constexpr float kMaxLead = 16.f;                                 // log2 units a
 
 template <int HP>
 struct UmmaCfg {
-    static_assert(HP == 16 || HP == 32 || HP == 64, "padded head count");
+    static_assert(HP == 16 || HP == 32, "padded head count (more query rows than 32: decode_wide.cuh)");
     static constexpr int kKSlots = 2, kVSlots = 3;
     static constexpr int kQBytes = HP * 256;                     // HP head rows x 128 columns bf16, two 64-column boxes
     // P^T tile: 128 cache rows x 128 bytes (64 bf16 head slots, HP used), 128-byte swizzle: an MN-major B
@@ -61,7 +61,7 @@ struct UmmaCfg {
     // the hi parts of two buffers (one rounding of P), or hi and lo of a single buffer (short prefixes).
     static constexpr int kPBytes = kUmmaStageRows * 128;
     static constexpr int kPTiles = 2;
-    static constexpr int kQBufs = HP <= 32 ? 2 : 1;             // 64 head rows: one Q buffer (shared memory)
+    static constexpr int kQBufs = 2;
     static constexpr int kHeadsPerThread = HP / 2;               // a cache row's heads are split over two warps
     static constexpr int kChunk = kHeadsPerThread < 32 ? kHeadsPerThread : 32;   // heads handled per TMEM load
     // per-quarter maxima and sums [4][HP] each, reference maxima, factors of the last move, 1/sum of two segments
@@ -298,7 +298,7 @@ __device__ __forceinline__ float warp_reduce_scatter(float (&v)[N], int lane) {
 
 // All the softmax threads of the CTA that delivered the last piece of sequence s: o[s] = the pieces held by
 // the CTAs lo..hi (those with a share of the line), merged in CTA order.  8 threads per head, 16 columns each.
-// o_rows: the sequence's rows of o (its first query row onwards), n_rows of them (h, or fewer in a last group of rows).
+// o_rows: the sequence's rows of o (its first query row onwards), n_rows of them.
 __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__ part_ml, const float* __restrict__ part_acc,
                                                    float* __restrict__ o_rows, int n_rows, int s, int h, int lo, int hi, int T,
                                                    unsigned long long magic, int tid) {
@@ -355,9 +355,7 @@ __device__ __forceinline__ void merge_sequence_pieces(const float2* __restrict__
 
 // HP = head rows of the Q tile (h rounded up to 16, 32 or 64).  GUESS: built with the code that starts copies on a
 // guess before the wait (GUESS && early >= 2 below); kernels without it take early 0 or 1 only.
-// GROUPED: 0 = every schedule sequence has its own cache (the plain step: nothing of QueryGroups is compiled in);
-// 1 = groups of 64 query rows over shared caches.
-template <int HP, bool FUSED, bool GUESS = false, int GROUPED = 0>
+template <int HP, bool FUSED, bool GUESS = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                               const __grid_constant__ CUtensorMap map_k_sub, const __grid_constant__ CUtensorMap map_v_sub,
@@ -366,9 +364,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                               float2* __restrict__ part_ml, float* __restrict__ part_acc, int32_t* __restrict__ status,
                               int b, int h, int m_max, unsigned long long magic, const FusedArgs fa,
                               unsigned long long* __restrict__ ctrl, int32_t* __restrict__ lens_advance, int early_arg,
-                              int read_once, const QueryGroups grp_arg) {
+                              int read_once) {
     using Cfg = UmmaCfg<HP>;
-    const QueryGroups grp = GROUPED ? grp_arg : QueryGroups{0, 0, 0};
     const int early = GUESS ? early_arg : (early_arg == 1 ? 1 : 0);
     constexpr int NK = Cfg::kKSlots, NV = Cfg::kVSlots, NQ = Cfg::kQBufs, CH = Cfg::kChunk, NCH = Cfg::kHeadsPerThread / CH;
     constexpr int kSubs = kUmmaStageRows / kTileRows;       // 4 sub-tiles of 32 rows per stage
@@ -436,12 +433,11 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     // new key row, lane l >= 16 of the new value row.  The row is loaded when its segment begins and stored (and
     // made visible to the copy engine) before the stage that contains it is fetched.
     auto row_load = [&](int s) -> uint4 {
-        const uint4* src = (lane < 16 ? fa.k_new : fa.v_new) + (size_t)group_kv(grp, s) * (kRowBytes / 16) + (lane & 15);
+        const uint4* src = (lane < 16 ? fa.k_new : fa.v_new) + (size_t)s * (kRowBytes / 16) + (lane & 15);
         return __ldg(src);
     };
     auto row_store = [&](int s, int new_row, uint4 value) {
-        // (groups of query rows over one cache each store the row before they fetch it: the same bytes)
-        uint4* dst = (lane < 16 ? fa.K : fa.V) + ((size_t)group_kv(grp, s) * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
+        uint4* dst = (lane < 16 ? fa.K : fa.V) + ((size_t)s * m_max + new_row) * (kRowBytes / 16) + (lane & 15);
         *dst = value;
         asm volatile("fence.proxy.async;" ::: "memory");   // the copy engine must see the row
         __syncwarp();
@@ -458,14 +454,14 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
         // the sequence's head rows (rows past h belong to the next sequence or read as zero: their
         // columns of S^T and O^T are never stored)
         if (lane == 0) mbar_expect_tx(q_full + qi * 8, Cfg::kQBytes);
-        tma_load_2d(q_s + qi * Cfg::kQBytes + lane * (Cfg::kQBytes / 2), &map_q, lane * kBoxCols, (int)group_row0(grp, s, h), q_full + qi * 8);
+        tma_load_2d(q_s + qi * Cfg::kQBytes + lane * (Cfg::kQBytes / 2), &map_q, lane * kBoxCols, s * h, q_full + qi * 8);
     };
     const uint64_t stream_policy = l2_stream_policy((read_once & 1) != 0);
     const bool withhold = (read_once & 2) != 0;             // for tests: one copy is never started, so that a wait runs out
     auto issue_stage = [&](int s, int u, int hi, int j) {   // lanes 0 to 3
         const int kv = lane >> 1, half = lane & 1;          // the K rows, then the V rows, each into its own ring
         const int nsub = min(kSubs, hi - u);
-        const int y = group_kv(grp, s) * m_max + u * kTileRows;
+        const int y = s * m_max + u * kTileRows;
         const int n_slots = kv ? NV : NK;
         const int slot = j % n_slots;
         const uint32_t full = (kv ? v_full : k_full) + slot * 8;
@@ -552,7 +548,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 Segment g = {};
                 int r = 0;
                 bool strided = false;
-                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r, cl, crank, kSubs, &strided, grp);
+                const bool found = first_segment<FUSED, kUmmaBoundaryPenalty>(lens, b, m_max, appending, magic, &g, &r, cl, crank, kSubs, &strided);
                 if (before && lane == 0) TS(8);
                 if (GUESS && before && early == 3) g.lo += kSubs;    // for tests: a guess that is one stage off
                 if (!before && GUESS && early >= 2) {
@@ -613,7 +609,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                         // CTAs: 26.9 us per step without, 26.2 / 26.0 / 26.5 / 27.2 us with 1 / 2 / 3 / 4 stages)
                         int u = g0.lo + pre_issued * ust;
                         for (int p = 0; p < kGuessL2Stages && (u + kSubs) * kTileRows <= stop_row && u + kSubs <= g0.hi; ++p, u += ust) {
-                            tma_prefetch_l2_2d((lane >> 1) ? &map_v : &map_k, (lane & 1) * kBoxCols, group_kv(grp, g0.s) * m_max + u * kTileRows);
+                            tma_prefetch_l2_2d((lane >> 1) ? &map_v : &map_k, (lane & 1) * kBoxCols, g0.s * m_max + u * kTileRows);
                         }
                     }
                 }
@@ -637,7 +633,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
 
     tc_fence_before();
     const SharePlan plan = stream_plan<FUSED, kUmmaThreads, kUmmaBoundaryPenalty>(lens, o, status, b, h, m_max, appending, magic, prefix,
-                                                            rows_of, plan_sm, kUmmaProducerWarp, grp);
+                                                            rows_of, plan_sm, kUmmaProducerWarp);
     const int T = plan.T, t_begin = plan.t_begin, t_end = plan.t_end, s_first = plan.s_first;
     tc_fence_after();
     // sequences of equal tile counts in a launch made of clusters: strided stages, pieces merged through the cluster
@@ -707,7 +703,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
             if (won) {
                 if (lens_advance)
                     for (int s = lane; s < b; s += 32)
-                        if (rows_of[s] & kAppendBit) lens_advance[group_kv(grp, s)] = rows_of[s] & (kAppendBit - 1);
+                        if (rows_of[s] & kAppendBit) lens_advance[s] = rows_of[s] & (kAppendBit - 1);
             }
         }
     } else if (warp == kUmmaSWarp) {
@@ -1040,8 +1036,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 }
                 piece_left = true;
                 pend = true;
-                pend_dst = (whole ? o + (size_t)group_row0(grp, s, h) * kHeadDim : via_cluster ? piece_acc : part_acc + slot * h * kHeadDim) + t;
-                pend_rows = whole ? group_rows(grp, s, h) : h;
+                pend_dst = (whole ? o + (size_t)s * h * kHeadDim : via_cluster ? piece_acc : part_acc + slot * h * kHeadDim) + t;
+                pend_rows = h;
                 pend_par = par;
                 pend_j = j - 1;
                 pend_s = s;
@@ -1059,8 +1055,8 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                 const int n_merge = merge_sm[0];
                 if (n_merge > 0) __threadfence();
                 for (int k = 0; k < n_merge; ++k)
-                    merge_sequence_pieces(part_ml, part_acc, o + (size_t)group_row0(grp, merge_sm[1 + 3 * k], h) * kHeadDim,
-                                          group_rows(grp, merge_sm[1 + 3 * k], h), merge_sm[1 + 3 * k], h, merge_sm[2 + 3 * k],
+                    merge_sequence_pieces(part_ml, part_acc, o + (size_t)merge_sm[1 + 3 * k] * h * kHeadDim,
+                                          h, merge_sm[1 + 3 * k], h, merge_sm[2 + 3 * k],
                                           merge_sm[3 + 3 * k], T, magic, tid);
             }
             if (!ok) atomicExch(&timed_out, 1);
@@ -1115,8 +1111,7 @@ mqa_decode_stream_umma_kernel(const __grid_constant__ CUtensorMap map_k, const _
                     }
                 }
                 const float inv = 1.f / den;
-                if (head >= group_rows(grp, s, h)) break;
-                *reinterpret_cast<float4*>(o + ((size_t)group_row0(grp, s, h) + head) * kHeadDim + c4 * 4) =
+                *reinterpret_cast<float4*>(o + ((size_t)s * h + head) * kHeadDim + c4 * 4) =
                     make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
             }
         }
