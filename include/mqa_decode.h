@@ -21,8 +21,8 @@
  *   - K, V, q, k_new, v_new hold bf16; o holds fp32; lens holds int32.
  *   - k == v == 128 is the only supported head width; h >= 1.  Many query rows per sequence (many heads;
  *     or beams x heads over one shared memory, passed as h = beams * heads) run on the tensor cores too:
- *     33 .. 128 rows on a kernel that puts the query rows on the rows of its tiles, more as groups of
- *     64 rows over the same cache.
+ *     more than 32 rows on a kernel that puts the query rows on the rows of its tiles (128 rows per
+ *     CTA; more as row tiles over the same cache rows).
  *   - `stream` is a cudaStream_t passed as a plain pointer (NULL = the legacy default stream).
  *     Calls only enqueue work on it: they never synchronise, never allocate device memory and
  *     never free anything.  The launch configuration is chosen from the integer arguments and
