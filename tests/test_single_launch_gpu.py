@@ -359,3 +359,44 @@ def test_the_configuration_the_bench_times_at_full_size():
         oracle.kv_cache_append(Kh, Vh, wl.bits(s["k_new"]), wl.bits(s["v_new"]), lens_h, True)
         assert np.array_equal(wl.bits(s["K"]), Kh) and np.array_equal(wl.bits(s["V"]), Vh)
         check_close(o.cpu().numpy(), oracle.mqa_decode_step(wl.bits(s["q"]), Kh, Vh, lens_h), "bench configuration")
+
+
+@pytest.mark.parametrize("rows", [64, 128])
+def test_the_many_rows_step_the_bench_times_at_full_size(rows):
+    """4 beams x 32 heads (and 64 rows) over the long-context workload's caches, as the bench's many-rows block launches
+    it: the append-and-attend step, lens not advanced, replayed from a CUDA graph over two cache sets.  Every output
+    against the oracle (all sequences, all rows), and the appended rows bit for bit."""
+    w = wl.WORKLOADS["long_context"]
+    b, h, m_max = w.b, rows, w.m_max
+    lens0 = wl.initial_lens(w, seed=0)
+    sets = [wl.make_inputs(b, h, m_max, "mqa", seed=80 + i, device=DEV) for i in range(2)]
+    before = [(wl.bits(s["K"]), wl.bits(s["V"])) for s in sets]
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    outs = [torch.full((b, h, 128), float("nan"), dtype=torch.float32, device=DEV) for _ in sets]
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    assert mqa.plan_kernel_name(True, True, b, h, m_max) == "mqa_decode_wide_kernel"
+    steps = [mqa.AppendStep(s["q"], s["K"], s["V"], s["k_new"], s["v_new"], lens_t, o, ws, status, advance=False, chained=True)
+             for s, o in zip(sets, outs)]
+    side = torch.cuda.Stream(device=DEV)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(4):
+            steps[i % 2](side)                                # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for o in outs:
+        o.fill_(float("nan"))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(6):
+            steps[i % 2](torch.cuda.current_stream())
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and np.array_equal(lens_t.cpu().numpy(), lens0)
+    for s, o, (Kb, Vb) in zip(sets, outs, before):
+        Kh, Vh, lens_h = Kb.copy(), Vb.copy(), lens0.copy()
+        oracle.kv_cache_append(Kh, Vh, wl.bits(s["k_new"]), wl.bits(s["v_new"]), lens_h, True)
+        assert np.array_equal(wl.bits(s["K"]), Kh) and np.array_equal(wl.bits(s["V"]), Vh)
+        check_close(o.cpu().numpy(), oracle.mqa_decode_step(wl.bits(s["q"]), Kh, Vh, lens_h), f"many rows ({rows}) at the bench's size")
