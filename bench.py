@@ -661,9 +661,24 @@ def main():
         out["layer_step"] = layer_block(mqa, w, device, seed, max(3, min(args.steps, 20)))
         out["paper_incremental"] = paper_loop_block(mqa, device, seed)
         out["layer_step"]["projections_us"] = out["layer_step"]["us_per_step"] - blk["us_per_step"]
+    # Order of the blocks: the multi-query points whose caches are below a gigabyte first, then the batched form, then the
+    # points and the multi-head blocks that stream gigabytes for long: a short step timed right after one of those reads
+    # 10-20 % slower (b=64 x m=4096: 28.6 us after them, 25.5 us before or alone), and so does the batched form (930 against
+    # 1000 TFLOP/s).
+    sweep_rows = {}
+    by_size = sorted(LINE_SWEEP, key=lambda n_: wl.WORKLOADS[n_].b * wl.WORKLOADS[n_].m_max)      # smallest caches first
+    small = [n_ for n_ in by_size if wl.WORKLOADS[n_].b * wl.WORKLOADS[n_].m_max * 512 <= (600 << 20)]
+    if not args.no_layer and world == 1:
+        out["beam4_rows"] = many_rows_block(mqa, device, seed, w)
+    if not args.no_line_sweep and world == 1:
+        for name in small:
+            sweep_rows[(name, "mqa")] = quick_point(mqa, "mqa", wl.WORKLOADS[name], device)
     if not args.no_layer and world == 1:
         out["prefill"] = prefill_block(mqa, device, seed)
-        out["beam4_rows"] = many_rows_block(mqa, device, seed, w)
+    if not args.no_line_sweep and world == 1:
+        for name in by_size:
+            if name not in small:
+                sweep_rows[(name, "mqa")] = quick_point(mqa, "mqa", wl.WORKLOADS[name], device)
     if not args.no_mha:
         sth = StepState(mqa, "mha", w, device, seed, min_rotate_bytes=2 * L2_BYTES)
         rh = run_variant(sth, max(3, min(args.steps, 20)), 3, device, sample_clocks=False, use_graph=not args.no_graph)
@@ -674,10 +689,9 @@ def main():
         torch.cuda.empty_cache()
     if not args.no_line_sweep and world == 1:
         # the other long-context points and the ragged batch: us, GB/s, fraction of 8 TB/s, launches, both variants
-        # (all the multi-query points first: a point timed right after a multi-head point's gigabytes reads 10-15 % slower)
-        rows = {(name, variant): quick_point(mqa, variant, wl.WORKLOADS[name], device)
-                for variant in ("mqa", "mha") for name in LINE_SWEEP}
-        out["sweep"] = [rows[(name, variant)] for name in LINE_SWEEP for variant in ("mqa", "mha")]
+        for name in LINE_SWEEP:
+            sweep_rows[(name, "mha")] = quick_point(mqa, "mha", wl.WORKLOADS[name], device)
+        out["sweep"] = [sweep_rows[(name, variant)] for name in LINE_SWEEP for variant in ("mqa", "mha")]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, seed)
     if rank == 0:
