@@ -100,3 +100,37 @@ def test_random_shape_batched_form(b, h, n, m_max, seed):
     assert int(status.item()) == 0
     ref = oracle.mqa_batched_attention(wl.bits(Q), wl.bits(K), wl.bits(V), st)
     check_close(O.cpu().numpy(), ref, f"batched b={b} h={h} n={n} m={m_max}")
+
+
+def test_mixed_back_to_back_launches_stay_bit_identical():
+    """The three kernels that take all of an SM's tensor memory (the streaming step, the many-rows step, the batched form),
+    launched back to back on one stream 200 times in turn (each may begin while the one before is finishing): every result
+    is bit for bit what the first round gave, and no wait ran out."""
+    b, h, m = 32, 32, 2048
+    a = wl.make_inputs(b, h, m, "mqa", seed=1, device=DEV)
+    c = wl.make_inputs(16, 96, 1100, "mqa", seed=2, device=DEV)
+    lens_a = torch.full((b,), m - 1, dtype=torch.int32, device=DEV)
+    lens_c = torch.from_numpy(np.random.default_rng(3).integers(0, 1100, size=16).astype(np.int32)).to(DEV)
+    ws_a, ws_c = mqa.alloc_workspace(b, h, m, DEV), mqa.alloc_workspace(16, 96, 1100, DEV)
+    o_a = torch.empty(b, h, 128, dtype=torch.float32, device=DEV)
+    o_c = torch.empty(16, 96, 128, dtype=torch.float32, device=DEV)
+    gen = torch.Generator(device=DEV).manual_seed(9)
+    Q = wl.bf16_normal((2, 5, 333, 128), 128 ** -0.5, gen, DEV)
+    K = wl.bf16_normal((2, 400, 128), 1.0, gen, DEV)
+    V = wl.bf16_normal((2, 400, 128), 1.0, gen, DEV)
+    O = torch.empty(2, 5, 333, 128, dtype=torch.float32, device=DEV)
+    ws_p = torch.empty(64, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    assert mqa.plan_kernel_name(True, True, b, h, m).startswith("mqa_decode_stream_umma_kernel")
+    assert mqa.plan_kernel_name(True, True, 16, 96, 1100) == "mqa_decode_wide_kernel"
+    first = None
+    for it in range(200):
+        mqa.mqa_decode_append_step(a["q"], a["K"], a["V"], a["k_new"], a["v_new"], lens_a, o_a, ws_a, status, advance=False, chained=it > 0)
+        mqa.mqa_prefill_attention(Q, K, V, O, ws_p, None, status)
+        mqa.mqa_decode_append_step(c["q"], c["K"], c["V"], c["k_new"], c["v_new"], lens_c, o_c, ws_c, status, advance=False)
+        if it % 40 == 0 or it == 199:
+            torch.cuda.synchronize()
+            cur = [t.clone().view(torch.int32) for t in (o_a, O, o_c)]
+            first = first or cur
+            assert all(torch.equal(x, y) for x, y in zip(first, cur)), f"round {it}"
+    assert int(status.item()) == 0
