@@ -183,3 +183,27 @@ def test_what_is_not_supported_is_refused_before_any_launch():
     assert e.value.code == binding.ERR_UNSUPPORTED
     torch.cuda.synchronize()
     assert bool((O == 7.0).all())
+
+
+def test_a_memory_that_would_pass_m_max_is_cut_there_and_flagged():
+    """start[b] + n > m_max: the positions past the end of the memory attend over all m_max rows (there is no row of
+    their own to add), LEN_CLAMPED is flagged, nothing outside K and V is read; the other sequences are not affected.
+    Checked row by row against the decoding step's oracle over min(start + t + 1, m_max) rows."""
+    b, h, n, m_max = 2, 4, 256, 600
+    gen = torch.Generator(device=DEV).manual_seed(31)
+    Q = wl.bf16_normal((b, h, n, 128), 128 ** -0.5, gen, DEV)
+    K = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    V = wl.bf16_normal((b, m_max, 128), 1.0, gen, DEV)
+    st = np.array([m_max - n + 70, 100], np.int32)          # the first sequence's last 70 positions have no row
+    O = torch.full((b, h, n, 128), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(16, mqa.prefill_workspace_bytes(b, h, n, m_max)), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mqa.mqa_prefill_attention(Q, K, V, O, ws, torch.from_numpy(st).to(DEV), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == binding.STATUS_LEN_CLAMPED
+    Oh = O.cpu().numpy()
+    assert np.all(np.isfinite(Oh))
+    for t in (0, 100, 185, 186, 200, 255):
+        lens = np.minimum(st + t + 1, m_max).astype(np.int32)
+        ref = oracle.mqa_decode_step(wl.bits(Q[:, :, t].contiguous()), wl.bits(K), wl.bits(V), lens)
+        check_close(Oh[:, :, t], ref, f"position {t}")
