@@ -373,6 +373,24 @@ def test_empty_and_out_of_range_lengths(variant):
     assert float(o2.abs().max()) == 0.0
 
 
+@pytest.mark.parametrize("b,h,m_max", [(40, 16, 1500), (24, 96, 2048), (6, 8, 300), (3, 200, 2100)])
+def test_split_and_combine_phases_equal_the_step_on_every_plan(b, h, m_max):
+    """The pass and the second pass on their own give the step's bits on the streaming kernel (whose step merges inside
+    the kernel), on the kernel with the query rows as tile rows (one and two row tiles) and on the fixed-split kernel."""
+    lens = _mixed_lens(b, m_max, seed=b + h)
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=12, device=DEV)
+    lens_t = torch.from_numpy(lens).to(DEV)
+    whole = gpu_step("mqa", inp["q"], inp["K"], inp["V"], lens_t)
+    o = torch.full_like(whole, float("nan"))
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    mqa.mqa_decode_step_split(inp["q"], inp["K"], inp["V"], lens_t, o, ws)
+    mqa.mqa_decode_step_combine(inp["q"], inp["K"], inp["V"], lens_t, o, ws)
+    torch.cuda.synchronize()
+    check_against_oracle("mqa", inp["q"], inp["K"], inp["V"], lens, o, f"split + combine b={b} h={h} m_max={m_max}", None)
+    if not mqa.plan_kernel_name(True, False, b, h, m_max).startswith("mqa_decode_stream_umma"):
+        assert torch.equal(o.view(torch.int32), whole.view(torch.int32))      # (the streaming step merges in another order)
+
+
 def test_split_and_combine_phases_equal_the_step():
     b, h, m_max = 4, 16, 9000
     lens = np.array([9000, 1, 4500, 8999], np.int32)
