@@ -437,12 +437,9 @@ def prefill_block(mqa, device, seed, b=32, h=32, n=4096):
     flops = 4 * 128 * h * b * n * (n + 1) // 2
     burst, sustained, kind = measured_tensor_peak()
     tf = flops / secs / 1e12
-    groups = b * h * (n // 64)
-    whole_tiles = n % 128 == 0          # the kernel of the batched form; otherwise groups of 64 rows on the decode kernel
     return {"b": b, "h": h, "n": n, "ms": secs * 1e3, "tflops": tf, "flops": flops, "bound": "tensor", "peak": sustained,
             "peak_kind": f"bf16 matmul, sustained, of {kind}", "frac": tf / sustained, "frac_of_burst_peak": tf / burst,
-            "launches": 1 if whole_tiles else -(-groups // 1024),
-            "kernel": "mqa_prefill_kernel" if whole_tiles else "mqa_decode_stream_umma_kernel<64, causal>",
+            "launches": 1, "kernel": "mqa_prefill_kernel",
             "status": int(status.item())}
 
 
