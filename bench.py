@@ -445,7 +445,7 @@ def prefill_block(mqa, device, seed, b=32, h=32, n=4096):
 
 def many_rows_block(mqa, device, seed, w, rows=128):
     """Beam search over one shared memory (Section 4.2: beam 4): beams x heads query rows per sequence, here 4 x 32 = 128
-    rows over the headline workload's caches, as groups of 64 rows on the tensor-core kernel.  us per step (attention over
+    rows over the headline workload's caches, on the kernel with the query rows as tile rows.  us per step (attention over
     the cache, caches rotated past L2), beside the 64-row figure."""
     out = {}
     for r in (64, rows):
