@@ -109,7 +109,7 @@ def test_binding_type_checks():
 
 
 def test_plans_of_many_query_rows_and_of_the_batched_form(L):
-    """More than 64 query rows per sequence are planned as groups of 64 on the tensor-core kernel, and the batched
+    """More than 32 query rows per sequence are planned on the kernel with the query rows as tile rows, and the batched
     form's workspace and refusals are answered on the host (the plan assumes the 148 SMs of a B200 without a GPU)."""
     assert binding.plan_kernel_name(True, False, 32, 128, 8192) == "mqa_decode_wide_kernel"       # 65 .. 128 rows: rows as tile rows
     assert binding.plan_kernel_name(True, False, 32, 192, 8192) == "mqa_decode_wide_kernel"       # beyond: tiles of 128 rows
