@@ -168,11 +168,11 @@ Plan plan_wide(int b, int h, int m_max) {
 Plan make_plan(bool multi_query, int b, int h, int m_max) {
     // a row space too large for the 32-bit TMA coordinates goes to the general CUDA-core kernel
     if (!(multi_query && (long long)b * m_max < 0x7fffffffLL)) return plan_simt(b, h, m_max);
-    // 33 .. 128 query rows per sequence: the kernel with the query rows as tile rows (measured against the streaming
-    // kernel's 64-row tile, per step: 32 x 64 rows x 8192: 30.5 vs 35.0 us; 128 x 64 x 2048: 26.2 vs 32.8; 4 x 48 x 4096:
-    // 10.8 vs 20.7; and against groups of 64 at 128 rows, 32 x 8192: 34.9 vs 68.8 us)
-    // (and beyond 128 rows as row tiles of 128 over the same cache rows: 32 x 256 rows x 8192: 43.6 us, against 122.7 us as
-    // four groups of 64 rows on the streaming kernel; 128 x 160 x 2048: 50.1 vs 103.2)
+    // More than 32 query rows per sequence: the kernel with the query rows as tile rows, 128 rows per CTA and more as row
+    // tiles over the same cache rows.  (The streaming kernel used to take up to 64 rows on a tile of its own and more as
+    // groups of 64: measured against that, per step, 32 x 64 rows x 8192: 30.5 vs 35.0 us; 128 x 64 x 2048: 26.2 vs 32.8;
+    // 4 x 48 x 4096: 10.8 vs 20.7; 32 x 128 x 8192: 34.9 vs 68.8; 32 x 256 x 8192: 43.6 vs 122.7; 128 x 160 x 2048: 50.1 vs
+    // 103.2 -- that tile and the groups are gone.)
     if (h > 32 && (h + kWideRows - 1) / kWideRows <= 65535 && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
     // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
