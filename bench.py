@@ -197,6 +197,21 @@ class StepState:
         self.host_o.copy_(self.o, non_blocking=True)
         stream.synchronize()
 
+    def capture_host_steps(self):
+        """The host-buffer call of every cache set captured once as a CUDA graph of its own (possible because nothing in
+        it is a transfer from pageable memory: a kernel fetches the pinned inputs, the kernels store o to the host)."""
+        self.host_graphs = []
+        for hs in self.host_steps:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                hs(torch.cuda.current_stream())
+            self.host_graphs.append(g)
+
+    def step_e2e_graph(self, i):
+        """step_e2e with the call replayed from its graph: the same work per token, one submission instead of two launches."""
+        self.host_graphs[i % len(self.host_graphs)].replay()
+        torch.cuda.current_stream().synchronize()
+
 
 def time_region(fn, steps, device):
     """Seconds for `steps` calls of fn(i), CUDA events on the launching stream, synchronised on both sides."""
@@ -326,9 +341,16 @@ def run_variant(st: StepState, steps, warmup, device, sample_clocks, use_graph=T
     # end to end with host buffers (eager: every step waits for its result)
     for i in range(3):
         st.step_e2e(i)
-    e2e_s = time_region(st.step_e2e, steps, device)
+    e2e_s = statistics.median(time_region(st.step_e2e, steps, device) for _ in range(5))
+    e2e_graph_s = None
+    if st.host_steps is not None and use_graph:
+        st.capture_host_steps()
+        for i in range(3):
+            st.step_e2e_graph(i)
+        e2e_graph_s = statistics.median(time_region(st.step_e2e_graph, steps, device) for _ in range(5))
     status = int(st.status.item())
-    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "status": status, "separate_s": sep_s, "isolated_s": isolated_s,
+    return {"secs": secs, "kernel_s": kernel_s, "e2e_s": e2e_s, "e2e_graph_s": e2e_graph_s, "status": status, "separate_s": sep_s,
+            "isolated_s": isolated_s,
             "clocks": sampler.summary() if sampler else None, "first_region_s": regions[0],
             "min_region_s": min(regions), "regions": len(regions), "graph": bool(use_graph)}
 
@@ -636,8 +658,13 @@ def main():
                                           "pair per launch: nothing of it overlaps a step before"}},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": st.h2d_bytes,
                 "d2h_bytes_per_step": st.d2h_bytes, "us_per_step": e2e_max / args.steps * 1e6,
-                "note": "per-step inputs q,k_new,v_new from pinned host memory, o read back; the KV cache is "
-                        "decoder state and stays resident in HBM"},
+                "us_per_step_graph_replay": r["e2e_graph_s"] / args.steps * 1e6 if r.get("e2e_graph_s") else None,
+                "note": ("mqa_decode_append_step_host, one call and one stream synchronisation per token: q, k_new, v_new "
+                         "fetched from pinned host memory by a kernel, o stored to pinned host memory by the kernels; "
+                         "us_per_step_graph_replay: the same call captured once per cache set and replayed; "
+                         if st.host_steps is not None else
+                         "per-step inputs q, k_new, v_new copied from pinned host memory, o copied back; ") +
+                        "the KV cache is decoder state and stays resident in HBM"},
         "gpu_launches": st.launches_per_step * args.steps,
         "clocks": r["clocks"],
     }

@@ -267,9 +267,13 @@ int mqa_append_step_launches(int b, int h, int m_max, int k, int v);
  * o is copied back, all enqueued on `stream` (nothing is synchronised: wait on the stream before reading o_host).
  * The cache, lens, workspace and status stay on the device as in mqa_decode_append_step.
  *
- *   q_host, k_new_host, v_new_host   HOST pointers, [b, h, k], [b, k], [b, v] bf16; pinned memory makes the copies
- *                     asynchronous.  When the three are packed back to back with each part padded to a multiple of
- *                     256 bytes they travel as one copy.
+ *   q_host, k_new_host, v_new_host   HOST pointers, [b, h, k], [b, k], [b, v] bf16.  Where all three are pinned memory
+ *                     that the device can address (cudaHostAlloc, cudaHostRegister), a kernel of this library fetches
+ *                     them into the staging buffer and the attention kernel behind it sets itself up and asks for its
+ *                     first stages of the cache meanwhile; they must then stay unchanged until the stream has passed
+ *                     this call's work.  Any other host memory goes by cudaMemcpyAsync (asynchronous for pinned
+ *                     memory; one copy when the three are packed back to back with each part padded to a multiple
+ *                     of 256 bytes, else three).
  *   o_host            HOST pointer, [b, h, v] fp32.  Pinned memory that the device can address (cudaHostAlloc,
  *                     cudaHostRegister) is written by the step's kernels themselves, with no copy after them;
  *                     any other host memory is filled by a copy from the staging buffer.  Either way it is

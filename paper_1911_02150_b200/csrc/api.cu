@@ -882,6 +882,16 @@ size_t mqa_host_staging_bytes(int b, int h, int k, int v) {
     return align256((size_t)b * h * k * 2) + 2 * align256((size_t)b * kHeadDim * 2) + align256((size_t)b * h * v * 4);
 }
 
+// The device's address of pinned host memory that it can reach (16-byte aligned), or null.
+static const void* host_device_pointer(const void* host) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+        aligned16(attr.devicePointer))
+        return attr.devicePointer;
+    cudaGetLastError();
+    return nullptr;
+}
+
 int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, const void* v_new_host, float* o_host,
                                 void* K, void* V, int32_t* lens, int advance, void* staging, size_t staging_bytes,
                                 void* workspace, size_t workspace_bytes, int32_t* status, int b, int h, int m_max, int k,
@@ -901,34 +911,46 @@ int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, cons
     const int bad = check_append_step(q_dev, K, V, k_dev, v_dev, lens, advance, o_dev, workspace, workspace_bytes, status, b, h,
                                       m_max, k, v);
     if (bad) return bad;
-    // the step's inputs: one copy when the caller packed them back to back (256-byte aligned parts), else three
+    // the step's inputs.  Pinned memory that this device can address: a kernel fetches them, and the attention kernel
+    // sets itself up and asks for its first stages while it does (what the layer step does behind its input projection).
+    // Otherwise copy-engine transfers: one when the caller packed them back to back (256-byte aligned parts), else three.
     const char* qh = static_cast<const char*>(q_host);
-    const bool packed = static_cast<const char*>(k_new_host) == qh + align256(q_bytes) &&
-                        static_cast<const char*>(v_new_host) == qh + align256(q_bytes) + align256(row_bytes);
-    if (packed) {
-        if (cudaMemcpyAsync(q_dev, qh, align256(q_bytes) + align256(row_bytes) + row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+    const void* q_map = host_device_pointer(q_host);
+    const void* k_map = host_device_pointer(k_new_host);
+    const void* v_map = host_device_pointer(v_new_host);
+    const bool by_kernel = q_map && k_map && v_map && q_bytes / 16 <= 0xffffffffull;
+    if (by_kernel) {
+        const StageInPart pq = {static_cast<const uint4*>(q_map), reinterpret_cast<uint4*>(q_dev), (unsigned)(q_bytes / 16)};
+        const StageInPart pk = {static_cast<const uint4*>(k_map), reinterpret_cast<uint4*>(k_dev), (unsigned)(row_bytes / 16)};
+        const StageInPart pv = {static_cast<const uint4*>(v_map), reinterpret_cast<uint4*>(v_dev), (unsigned)(row_bytes / 16)};
+        const size_t turns = (q_bytes / 16 + kStageInThreads - 1) / kStageInThreads;
+        const unsigned grid = (unsigned)(turns < (size_t)(2 * sm_count()) ? (turns ? turns : 1) : 2 * sm_count());
+        if (launch_dependent(stage_in_kernel, grid, (unsigned)kStageInThreads, 0, stream, pq, pk, pv) != cudaSuccess) {
             cudaGetLastError();
             return MQA_ERR_CUDA;
         }
     } else {
-        if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-            cudaMemcpyAsync(k_dev, k_new_host, row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-            cudaMemcpyAsync(v_dev, v_new_host, row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
-            cudaGetLastError();
-            return MQA_ERR_CUDA;
+        const bool packed = static_cast<const char*>(k_new_host) == qh + align256(q_bytes) &&
+                            static_cast<const char*>(v_new_host) == qh + align256(q_bytes) + align256(row_bytes);
+        if (packed) {
+            if (cudaMemcpyAsync(q_dev, qh, align256(q_bytes) + align256(row_bytes) + row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return MQA_ERR_CUDA;
+            }
+        } else {
+            if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+                cudaMemcpyAsync(k_dev, k_new_host, row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+                cudaMemcpyAsync(v_dev, v_new_host, row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return MQA_ERR_CUDA;
+            }
         }
     }
     // the result: where o_host is pinned memory that this device can address, the kernels store o there themselves
     // (posted writes that overlap the end of the step); otherwise it goes through the staging buffer and a copy
-    float* o_direct = nullptr;
-    cudaPointerAttributes attr;
-    if (cudaPointerGetAttributes(&attr, o_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
-        aligned16(attr.devicePointer))
-        o_direct = static_cast<float*>(attr.devicePointer);
-    else
-        cudaGetLastError();
+    float* o_direct = static_cast<float*>(const_cast<void*>(host_device_pointer(o_host)));
     const int rc = append_step_impl(q_dev, K, V, k_dev, v_dev, lens, advance, o_direct ? o_direct : o_dev, workspace,
-                                    workspace_bytes, status, b, h, m_max, k, v, stream_, false);
+                                    workspace_bytes, status, b, h, m_max, k, v, stream_, by_kernel);
     if (rc || o_direct) return rc;
     if (cudaMemcpyAsync(o_host, o_dev, o_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
         cudaGetLastError();

@@ -37,4 +37,23 @@ kv_cache_append_kernel(uint4* __restrict__ K, uint4* __restrict__ V,
     }
 }
 
+// The host-buffer step's inputs (q, the new key row, the new value row) from pinned host memory that the device can
+// address into the staging buffer, 16 bytes per thread and turn.  A kernel rather than a copy-engine transfer so that the
+// attention kernel behind it may set itself up and fetch its first stages meanwhile: like every kernel here it waits for
+// what is older, then lets its dependent start, and writes nothing but the staging buffer.
+constexpr int kStageInThreads = 256;
+struct StageInPart { const uint4* src; uint4* dst; unsigned n16; };
+
+__global__ void __launch_bounds__(kStageInThreads)
+stage_in_kernel(StageInPart q, StageInPart k_new, StageInPart v_new) {
+    grid_dependency_wait();          // the step before may still read the staging buffer
+    grid_launch_dependents();
+    const unsigned stride = gridDim.x * kStageInThreads;
+    const StageInPart parts[3] = {q, k_new, v_new};
+#pragma unroll
+    for (int p = 0; p < 3; ++p)
+        for (unsigned i = blockIdx.x * kStageInThreads + threadIdx.x; i < parts[p].n16; i += stride)
+            parts[p].dst[i] = __ldcv(parts[p].src + i);      // (host memory: read afresh, never from a cache line of an earlier step)
+}
+
 }  // namespace mqa

@@ -179,6 +179,37 @@ def test_host_buffer_entry_point_matches_the_device_one():
         assert torch.equal(Kc.view(torch.int16), inp["K"].view(torch.int16)) and torch.equal(lens_c, lens_a)
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("b,h,m_max", [(32, 32, 2048), (40, 16, 1500), (6, 48, 700), (4, 8, 100), (3, 130, 300), (150, 8, 1100)])
+def test_host_buffer_steps_in_a_loop_against_the_oracle(b, h, m_max, pinned):
+    """Five consecutive steps through the host-buffer entry point, bound once, the same host buffers refilled before each
+    step (pinned: the inputs are fetched by a kernel and o is stored to the host by the kernels; pageable: copies either
+    side): every step is the oracle's append and step on the grown cache, lens moves on, the cache holds the new rows."""
+    inp = wl.make_inputs(b, h, m_max, "mqa", seed=31, device=DEV)
+    lens0 = np.minimum(lens_mix(b, m_max, seed=31), m_max - 5).clip(0).astype(np.int32)
+    wl.poison_tail(inp["K"], lens0); wl.poison_tail(inp["V"], lens0)
+    Kh, Vh, lens_h = wl.bits(inp["K"]), wl.bits(inp["V"]), lens0.copy()
+    lens_t = torch.from_numpy(lens0).to(DEV)
+    hold = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    qh, kh, vh = (hold(torch.empty(tuple(inp[n].shape), dtype=torch.bfloat16)) for n in ("q", "k_new", "v_new"))
+    o_host = hold(torch.empty(b, h, 128, dtype=torch.float32))
+    staging = torch.empty(mqa.host_staging_bytes(b, h), dtype=torch.uint8, device=DEV)
+    ws = mqa.alloc_workspace(b, h, m_max, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    step = mqa.HostStep(qh, kh, vh, o_host, inp["K"], inp["V"], lens_t, staging, ws, status)
+    for t in range(5):
+        new = wl.make_inputs(b, h, 1, "mqa", seed=100 + t, device="cpu")
+        qh.copy_(new["q"]); kh.copy_(new["k_new"]); vh.copy_(new["v_new"])
+        o_host.fill_(float("nan"))
+        step()
+        torch.cuda.synchronize()
+        oracle.kv_cache_append(Kh, Vh, wl.bits(kh), wl.bits(vh), lens_h, True)
+        check_close(o_host.numpy(), oracle.mqa_decode_step(wl.bits(qh), Kh, Vh, lens_h), f"host step {t}")
+        assert np.array_equal(lens_t.cpu().numpy(), lens_h)
+    assert int(status.item()) == 0
+    assert np.array_equal(wl.bits(inp["K"]), Kh) and np.array_equal(wl.bits(inp["V"]), Vh)
+
+
 def test_bound_step_gives_what_the_call_gives():
     b, h, m_max = 40, 16, 1500
     inp = wl.make_inputs(b, h, m_max, "mqa", seed=22, device=DEV)
