@@ -92,7 +92,8 @@ Plan plan_mma(int b, int h, int m_max) {
     p.b = b; p.h = h;
     p.kernel = h <= 16 ? Kernel::kMma1 : Kernel::kMma2;
     const int ctas_per_sm = h <= 16 ? MmaCfg<1>::kMinBlocks : MmaCfg<2>::kMinBlocks;
-    const long slots = (long)sm_count() * ctas_per_sm;
+    const int sms = sm_count();
+    const long slots = (long)sms * ctas_per_sm;
     const double overhead_rows = 128.0;                               // start-up + merge, per CTA
     const double partial_rows = (double)h * (kHeadDim + 2) * 4 * 2 / (2.0 * kRowBytes);   // per split
     const int max_splits = m_max / 128 > 1 ? (m_max / 128 < 256 ? m_max / 128 : 256) : 1;
@@ -105,7 +106,7 @@ Plan plan_mma(int b, int h, int m_max) {
         const long ctas = (long)b * n;
         const long waves = (ctas + slots - 1) / slots;
         double cost = (double)waves * (chunk + overhead_rows) * ctas_per_sm;
-        if (n > 1) cost += (double)ctas * partial_rows / sm_count();
+        if (n > 1) cost += (double)ctas * partial_rows / sms;
         if (p.n_splits == 0 || cost < best) {
             best = cost;
             p.n_splits = n;
@@ -126,11 +127,12 @@ Plan plan_stream(int b, int h, int m_max) {
     // pieces (none when CTAs take whole sequences) and the CTAs that hold them finish together.  HBM is
     // saturated from about three quarters of the SMs on (measured: same pass time with 112..148 CTAs).
     // Among the multiples of the batch, first one that makes a sequence's CTAs a thread-block cluster.
-    p.grid = sm_count();
+    const int sms = sm_count();
+    p.grid = sms;
     bool found = false;
-    for (int g = sm_count(); g >= (3 * sm_count() + 3) / 4 && !found; --g)
+    for (int g = sms; g >= (3 * sms + 3) / 4 && !found; --g)
         if (b % g == 0 || (g % b == 0 && g / b <= kMaxClusterCtas)) { p.grid = g; found = true; }
-    for (int g = sm_count(); g >= (3 * sm_count() + 3) / 4 && !found; --g)
+    for (int g = sms; g >= (3 * sms + 3) / 4 && !found; --g)
         if (g % b == 0) { p.grid = g; found = true; }
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
     p.chunk_rows = (int)((tiles + p.grid - 1) / p.grid) * kTileRows;
@@ -176,7 +178,8 @@ Plan make_plan(bool multi_query, int b, int h, int m_max) {
     if (h > 32 && (h + kWideRows - 1) / kWideRows <= 65535 && (long long)b * h < 0x7fffffffLL) return plan_wide(b, h, m_max);
     // enough tiles to give every SM a real share: the persistent kernels; otherwise fixed splits
     const long long tiles = (long long)b * ((m_max + kTileRows - 1) / kTileRows);
-    if (b <= kStreamMaxSeqs && tiles >= 2LL * sm_count() && m_max >= 1024 && sm_count() <= 256) {
+    const int sms = sm_count();
+    if (b <= kStreamMaxSeqs && tiles >= 2LL * sms && m_max >= 1024 && sms <= 256) {
         const Plan p = plan_stream(b, h, m_max);
         // few, long sequences, each cut into more pieces than one CTA merges inside the kernel: the streaming kernel would
         // need its second pass as well, and the kernel with the query rows as tile rows (fixed splits, second pass) is
@@ -747,28 +750,31 @@ constexpr int kGuessMaxPieces = 6, kGuessMinShareRows = 8 * kUmmaStageRows;
 // Every check of mqa_decode_append_step that needs no launch: flags, pointers, sizes, the plan, the workspace.
 static int check_append_step(const void* q, const void* K, const void* V, const void* k_new, const void* v_new,
                              const int32_t* lens, int flags, const float* o, const void* workspace, size_t workspace_bytes,
-                             const int32_t* status, int b, int h, int m_max, int k, int v) {
+                             const int32_t* status, int b, int h, int m_max, int k, int v, Plan* plan) {
     if (flags & ~(MQA_STEP_ADVANCE | MQA_STEP_CHAINED | MQA_STEP_TEST_WRONG_GUESS | MQA_STEP_TEST_WITHHOLD_COPY)) return MQA_ERR_INVALID_ARG;
     int rc = check_step_args(q, K, V, lens, o, status, b, h, m_max, k, v);
     if (rc) return rc;
     if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return MQA_ERR_INVALID_ARG;
-    const Plan p = make_plan(true, b, h, m_max);
-    if (p.units * (size_t)p.n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
-    return check_workspace(p, workspace, workspace_bytes);
+    *plan = make_plan(true, b, h, m_max);
+    if (plan->units * (size_t)plan->n_splits > 0x7fffffffull) return MQA_ERR_UNSUPPORTED;
+    return check_workspace(*plan, workspace, workspace_bytes);
 }
 
 static int append_step_impl(const void* q, void* K, void* V, const void* k_new, const void* v_new, int32_t* lens,
                             int flags, float* o, void* workspace, size_t workspace_bytes, int32_t* status, int b,
-                            int h, int m_max, int k, int v, mqa_stream_t stream_, bool after_projection) {
-    int rc = check_append_step(q, K, V, k_new, v_new, lens, flags, o, workspace, workspace_bytes, status, b, h, m_max, k, v);
-    if (rc) return rc;
+                            int h, int m_max, int k, int v, mqa_stream_t stream_, bool after_projection,
+                            const Plan* checked = nullptr) {
+    // (checked: the caller has run check_append_step on these very arguments and passes the plan it gave)
+    Plan p;
+    int rc = MQA_OK;
+    if (checked) p = *checked;
+    else if ((rc = check_append_step(q, K, V, k_new, v_new, lens, flags, o, workspace, workspace_bytes, status, b, h, m_max, k, v, &p))) return rc;
     const int advance = flags & MQA_STEP_ADVANCE;
     int early = after_projection ? kEarlyAfterProjection
                 : !(flags & MQA_STEP_CHAINED) ? kEarlyNone
                 : (flags & MQA_STEP_TEST_WRONG_GUESS) ? kEarlyChainedWrongGuess : kEarlyChained;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const bool withhold = (flags & MQA_STEP_TEST_WITHHOLD_COPY) != 0;
-    const Plan p = make_plan(true, b, h, m_max);
     if (p.kernel == Kernel::kUmma) {
         // copies started on a guess pay where the step is one launch over long shares (measured: 0.4-0.7 us gained with
         // up to 6 pieces per sequence, 0.3-2.5 us lost with more pieces, short shares or a second-pass kernel)
@@ -908,8 +914,9 @@ int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, cons
     char* v_dev = k_dev + align256(row_bytes);
     float* o_dev = reinterpret_cast<float*>(v_dev + align256(row_bytes));
     // everything that can be refused is refused before the first copy is enqueued
+    Plan plan;
     const int bad = check_append_step(q_dev, K, V, k_dev, v_dev, lens, advance, o_dev, workspace, workspace_bytes, status, b, h,
-                                      m_max, k, v);
+                                      m_max, k, v, &plan);
     if (bad) return bad;
     // the step's inputs.  Pinned memory that this device can address: a kernel fetches them, and the attention kernel
     // sets itself up and asks for its first stages while it does (what the layer step does behind its input projection).
@@ -950,7 +957,7 @@ int mqa_decode_append_step_host(const void* q_host, const void* k_new_host, cons
     // (posted writes that overlap the end of the step); otherwise it goes through the staging buffer and a copy
     float* o_direct = static_cast<float*>(const_cast<void*>(host_device_pointer(o_host)));
     const int rc = append_step_impl(q_dev, K, V, k_dev, v_dev, lens, advance, o_direct ? o_direct : o_dev, workspace,
-                                    workspace_bytes, status, b, h, m_max, k, v, stream_, by_kernel);
+                                    workspace_bytes, status, b, h, m_max, k, v, stream_, by_kernel, &plan);
     if (rc || o_direct) return rc;
     if (cudaMemcpyAsync(o_host, o_dev, o_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
         cudaGetLastError();
