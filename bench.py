@@ -162,8 +162,9 @@ class StepState:
         if variant == "mqa":
             # the library's host-buffer call, bound once per cache set (what a decoding loop over fixed pinned buffers does)
             qh, kh, vh = self.host_views
+            self.e2e_stream = torch.cuda.current_stream(device)
             self.host_steps = [mqa.HostStep(qh, kh, vh, self.host_o, s["K"], s["V"], self.lens_before, self.staging, self.ws,
-                                            self.status, advance=False) for s in self.sets]
+                                            self.status, advance=False, stream=self.e2e_stream) for s in self.sets]
 
     def step(self, i):
         if self.bound_steps is not None:
@@ -183,12 +184,12 @@ class StepState:
         self.split_fn(s["q"], s["K"], s["V"], self.lens_after, self.o, self.ws, self.status)
 
     def step_e2e(self, i):
-        stream = torch.cuda.current_stream()
         if self.host_steps is not None:
-            # copies in, step, copy out: all enqueued by one C call on pinned host buffers
-            self.host_steps[i % len(self.host_steps)](stream)
-            stream.synchronize()                       # the caller needs o before the next token
+            # inputs in, step, o out: all enqueued by one C call on pinned host buffers (bound to the stream at set-up)
+            self.host_steps[i % len(self.host_steps)]()
+            self.e2e_stream.synchronize()              # the caller needs o before the next token
             return
+        stream = torch.cuda.current_stream()
         s = self.sets[i % len(self.sets)]
         self.dev_in.copy_(self.host_in, non_blocking=True)
         q, k_new, v_new = self.e2e_views

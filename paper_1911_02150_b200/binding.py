@@ -327,6 +327,12 @@ def mqa_decode_append_step(q, K, V, k_new, v_new, lens, o, workspace=None, statu
     return o
 
 
+def _as_c_args(fn, args):
+    """The argument tuple as instances of the function's declared ctypes types, made once: a call then converts nothing
+    (about a microsecond for the twenty arguments of a step)."""
+    return tuple(t(a) for t, a in zip(fn.argtypes, args))
+
+
 class AppendStep:
     """:func:`mqa_decode_append_step` bound once to its tensors: a decoding loop refills the same q, k_new and v_new
     buffers for every token, so the checks and the pointer marshalling (about 20 us of Python per call, several times
@@ -339,6 +345,7 @@ class AppendStep:
         self.args = _append_step_args(q, K, V, k_new, v_new, lens, o, workspace, status, advance, stream, chained)
         self.keep = (q, K, V, k_new, v_new, lens, o, workspace, status, stream)
         self.fn = lib().mqa_decode_append_step
+        self.args = _as_c_args(self.fn, self.args)
         self.o = o
 
     def __call__(self, stream=None):
@@ -480,6 +487,7 @@ class HostStep:
                                     chained)
         self.keep = (q_host, k_new_host, v_new_host, o_host, K, V, lens, staging, workspace, status, stream)
         self.fn = lib().mqa_decode_append_step_host
+        self.args = _as_c_args(self.fn, self.args)
         self.o_host = o_host
 
     def __call__(self, stream=None):
