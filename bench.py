@@ -12,6 +12,9 @@ workload is the long-context configuration (b=32, h=32, k=v=128, 8192-row cache)
 workloads (`--workload`, `--sweep`) are the parity configurations and the bandwidth sweep.
 Prints ONE JSON line (rank 0).  `value` is achieved HBM GB/s of the multi-query step
 (algorithmic bytes / time); the multi-head step on the same shapes is reported beside it.
+`e2e` is the same step through mqa_decode_append_step_host on pinned host buffers, one call and
+one stream synchronisation per token (median of five regions of K steps), and beside it the same
+call captured once per cache set as a CUDA graph and replayed.
 """
 from __future__ import annotations
 
